@@ -1,0 +1,19 @@
+"""CPU oracle of the lazy update (Algorithm 1) in dynamic fixed-point.
+
+Test infrastructure only: imported by the tests, the smoke check and the CPU
+baseline leg of the benchmark.  The CUDA library never imports it.
+"""
+from .kahan_oracle import (  # noqa: F401
+    OracleElem,
+    OracleTensor,
+    OracleState,
+    oracle_element,
+    oracle_increment,
+    oracle_rne_shift,
+    oracle_next_exponent,
+    oracle_step_tensor,
+    oracle_step,
+    oracle_max_threads,
+    EXP_FIXED,
+    EXP_AMAX,
+)

@@ -1,0 +1,251 @@
+/*
+ * CPU oracle for the lazy update (SGD with Kahan summation, Algorithm 1 of
+ * arXiv 1810.05486) in the dynamic fixed-point setting of Section 2 / Fig. 1.
+ *
+ * THIS FILE IS TEST INFRASTRUCTURE.  It is a plain, slow, one-element-at-a-time
+ * restatement of the update, used to check the CUDA library and to give a CPU
+ * baseline time.  It shares no code with the CUDA library and nothing in the
+ * product path may call it.
+ *
+ * Number system (Section 2, Fig. 1): a tensor is an array of signed integer
+ * mantissas with one shared exponent; value = Q * 2^e.  The parameter theta
+ * has m-bit mantissas Q_theta at exponent e_theta.  The extra "accumulator"
+ * parameter of Algorithm 1 is stored negated, as the compensation c = -acc,
+ * with n-bit mantissas Q_c at exponent e_c = e_theta - s, s = n - 1 - k, where
+ * k is the number of bits by which the accumulator overlaps the parameter
+ * (Section 2: "m + n - 2 - k" magnitude bits in total).  theta + c is the
+ * virtually widened parameter.
+ *
+ * One step for one element (Algorithm 1, statements 1-4, with c = -acc):
+ *   stmt 1  acc += eta*g      : the increment is rounded onto the accumulator
+ *                               grid,  d = rne(g * eta * 2^-e_c)
+ *   stmt 2  theta_u = theta-acc: T = theta + c - d exactly (wide integer on the
+ *                               fine grid), theta' = T rounded onto theta's grid
+ *   stmt 3  acc += theta_u-theta: c' = T - theta' (what the rounding lost)
+ *   stmt 4  theta = theta_u
+ *
+ * Readings fixed where the paper is silent:
+ *   - every rounding is round-to-nearest, ties-to-even (the paper only says
+ *     "uniform linear quantization without stochastic computing", Section 1);
+ *   - saturation is a symmetric clamp to +-(2^(b-1) - 1);
+ *   - the sum acc + eta*g is kept wide until statements 2-3;
+ *   - the increment is clamped to +-2^30 accumulator LSBs; NaN gives 0;
+ *   - a step reads the mantissas at exponent e_in and writes them at e_out
+ *     (|e_out - e_in| <= 8); the increment is rounded on the output grid;
+ *   - the next exponent is the tight fit of the step's max |P| (max scan,
+ *     Section 5 "Related work" on how dynamic fixed-point picks exponents).
+ *
+ * Parity pins (tests/test_oracle_pins.py): stall-vs-move (Section 2), the exact
+ * accumulation invariant, brute force over all inputs at small bit-widths
+ * against exact rational arithmetic, a literal four-statement transcription of
+ * Algorithm 1, the m+n-2-k bit-width closed form with the ties-to-even step
+ * counts, the plain-SGD reduction (Eq. 1), regrid value preservation, and the
+ * exponent-policy property.  Accuracy tables of Section 4: parity unpinned
+ * (datasets and trained weights are not available).
+ *
+ * Build: gcc -O2 -ffp-contract=off -fopenmp -shared -fPIC (see oracle/build.py).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct {
+  int64_t P;        /* parameter mantissa before saturation, units of 2^e_out      */
+  int64_t Rq;       /* compensation mantissa before saturation, units of 2^ec_out  */
+  int64_t T;        /* theta + c - d on the fine grid 2^f, f = min(ec_in, ec_out)  */
+  int32_t d;        /* quantized increment, units of 2^ec_out                      */
+  int32_t q_theta;  /* stored parameter mantissa  (saturated P)                    */
+  int32_t q_comp;   /* stored compensation mantissa (saturated Rq)                 */
+  int32_t nonfinite;/* 1 if the gradient was NaN or +-Inf                          */
+} ksgd_oracle_elem;
+
+typedef struct {
+  uint32_t amax_theta;  /* max |P| over the tensor                                 */
+  uint32_t amax_comp;   /* max min(|Rq|, 2^31 - 1) over the tensor                 */
+  uint64_t n_sat_theta; /* elements whose parameter mantissa was clamped           */
+  uint64_t n_sat_comp;  /* elements whose compensation mantissa was clamped        */
+  uint64_t n_nonfinite; /* NaN / Inf gradients                                     */
+} ksgd_oracle_stats;
+
+static int64_t pow2_i64(int r) { return (int64_t)1 << r; }
+
+/* floor(a / 2^r) without relying on the shift of a negative number. */
+static int64_t floor_div_pow2(int64_t a, int r) {
+  int64_t den = pow2_i64(r);
+  int64_t q = a / den;            /* truncates toward zero */
+  if ((a % den) != 0 && a < 0) q -= 1;
+  return q;
+}
+
+/* a / 2^r rounded to the nearest integer, ties to the even integer. */
+int64_t ksgd_oracle_rne_shift(int64_t a, int32_t r) {
+  if (r == 0) return a;
+  int64_t q = floor_div_pow2(a, r);
+  int64_t rem = a - q * pow2_i64(r);      /* 0 <= rem < 2^r */
+  int64_t half = pow2_i64(r - 1);
+  if (rem > half) return q + 1;
+  if (rem == half && (q % 2 != 0)) return q + 1;
+  return q;
+}
+
+static int64_t clamp_i64(int64_t x, int64_t lo, int64_t hi) {
+  return x < lo ? lo : (x > hi ? hi : x);
+}
+
+static int64_t qmax_bits(int bits) { return pow2_i64(bits - 1) - 1; }
+
+/*
+ * Statement 1 of Algorithm 1, increment part: eta*g rounded onto the
+ * accumulator's output grid.  scale = eta * 2^-ec_out exactly (a power-of-two
+ * rescaling of a binary32), x = g*scale is one binary32 multiply, then
+ * round-to-nearest-even to an integer, clamped to +-2^30; NaN -> 0.
+ */
+int32_t ksgd_oracle_increment(float g, float lr, int32_t ec_out) {
+  float scale = ldexpf(lr, -ec_out);
+  float xv = g * scale;            /* one binary32 multiply (SSE, no contraction) */
+  if (isnan(xv)) return 0;
+  const float lim = 1073741824.0f; /* 2^30 */
+  if (xv >= lim) return (int32_t)1 << 30;
+  if (xv <= -lim) return -((int32_t)1 << 30);
+  return (int32_t)nearbyintf(xv);  /* default rounding mode: to nearest even */
+}
+
+/*
+ * One element, any mantissa widths m (parameter) and n (compensation; n = 0 is
+ * plain low-precision SGD, Eq. 1) from 2 to 16 bits.  s is the distance between
+ * the two grids (ignored, taken as 0, when n = 0).
+ */
+void ksgd_oracle_element(int32_t q_theta, int32_t q_comp, float g, float lr,
+                         int32_t m, int32_t n, int32_t s, int32_t e_in,
+                         int32_t e_out, ksgd_oracle_elem* out) {
+  if (n == 0) { s = 0; q_comp = 0; }
+  int32_t ec_in = e_in - s;
+  int32_t ec_out = e_out - s;
+  int32_t f = ec_in < ec_out ? ec_in : ec_out;
+
+  int32_t d = ksgd_oracle_increment(g, lr, ec_out);
+
+  /* statements 1-2: theta + c - d, exact, in units of 2^f */
+  int64_t T = (int64_t)q_theta * pow2_i64(e_in - f) +
+              (int64_t)q_comp * pow2_i64(ec_in - f) -
+              (int64_t)d * pow2_i64(ec_out - f);
+
+  /* statement 2/4: round onto the parameter's output grid and saturate */
+  int64_t P = ksgd_oracle_rne_shift(T, e_out - f);
+  int64_t q_theta_new = clamp_i64(P, -qmax_bits(m), qmax_bits(m));
+
+  /* statement 3: what the parameter could not take stays in the compensation */
+  int64_t R = T - q_theta_new * pow2_i64(e_out - f);
+  int64_t Rq = 0, q_comp_new = 0;
+  if (n != 0) {
+    Rq = ksgd_oracle_rne_shift(R, ec_out - f);
+    q_comp_new = clamp_i64(Rq, -qmax_bits(n), qmax_bits(n));
+  }
+
+  out->P = P;
+  out->Rq = Rq;
+  out->T = T;
+  out->d = d;
+  out->q_theta = (int32_t)q_theta_new;
+  out->q_comp = (int32_t)q_comp_new;
+  out->nonfinite = isfinite(g) ? 0 : 1;
+}
+
+static int32_t load_mantissa(const void* p, int64_t i, int bits) {
+  return bits <= 8 ? (int32_t)((const int8_t*)p)[i] : (int32_t)((const int16_t*)p)[i];
+}
+
+static void store_mantissa(void* p, int64_t i, int bits, int32_t v) {
+  if (bits <= 8) ((int8_t*)p)[i] = (int8_t)v; else ((int16_t*)p)[i] = (int16_t)v;
+}
+
+/*
+ * One step over one tensor, in place.  Mantissas of up to 8 bits live in int8
+ * arrays, wider ones in int16 arrays.  comp may be NULL iff comp_bits == 0.
+ * n_threads > 1 splits the elements statically over OpenMP threads; max and
+ * integer sums are exact, so the result does not depend on n_threads.
+ * Returns 0, or -1 on an argument the format does not allow.
+ */
+int ksgd_oracle_step_tensor(void* theta, void* comp, const float* grad,
+                            int64_t numel, int32_t theta_bits, int32_t comp_bits,
+                            int32_t overlap_k, int32_t e_in, int32_t e_out,
+                            float lr, ksgd_oracle_stats* stats, int32_t n_threads) {
+  if (!theta || !grad || !stats || numel <= 0) return -1;
+  if (theta_bits < 2 || theta_bits > 16) return -1;
+  if (comp_bits != 0 && (comp_bits < 2 || comp_bits > 16)) return -1;
+  if (comp_bits != 0 && (!comp || overlap_k < 0 || overlap_k > comp_bits - 1)) return -1;
+  if (e_out - e_in > 8 || e_in - e_out > 8) return -1;
+  int32_t s = comp_bits == 0 ? 0 : comp_bits - 1 - overlap_k;
+
+  uint32_t amax_theta = 0, amax_comp = 0;
+  uint64_t n_sat_theta = 0, n_sat_comp = 0, n_nonfinite = 0;
+  if (n_threads < 1) n_threads = 1;
+
+#pragma omp parallel for schedule(static) num_threads(n_threads) \
+    reduction(max : amax_theta, amax_comp) reduction(+ : n_sat_theta, n_sat_comp, n_nonfinite)
+  for (int64_t i = 0; i < numel; ++i) {
+    ksgd_oracle_elem r;
+    int32_t qt = load_mantissa(theta, i, theta_bits);
+    int32_t qc = comp_bits ? load_mantissa(comp, i, comp_bits) : 0;
+    ksgd_oracle_element(qt, qc, grad[i], lr, theta_bits, comp_bits, s, e_in, e_out, &r);
+    store_mantissa(theta, i, theta_bits, r.q_theta);
+    if (comp_bits) store_mantissa(comp, i, comp_bits, r.q_comp);
+
+    int64_t aP = r.P < 0 ? -r.P : r.P;
+    int64_t aR = r.Rq < 0 ? -r.Rq : r.Rq;
+    if (aR > 2147483647LL) aR = 2147483647LL;
+    if ((uint32_t)aP > amax_theta) amax_theta = (uint32_t)aP;
+    if ((uint32_t)aR > amax_comp) amax_comp = (uint32_t)aR;
+    n_sat_theta += (r.P != r.q_theta);
+    n_sat_comp += (comp_bits != 0 && r.Rq != r.q_comp);
+    n_nonfinite += (uint64_t)r.nonfinite;
+  }
+  stats->amax_theta = amax_theta;
+  stats->amax_comp = amax_comp;
+  stats->n_sat_theta = n_sat_theta;
+  stats->n_sat_comp = n_sat_comp;
+  stats->n_nonfinite = n_nonfinite;
+  return 0;
+}
+
+/*
+ * Exponent for the next step from the max scan of this one (dynamic
+ * fixed-point: the shared exponent follows the tensor's maximum).  amax_theta
+ * is max |P| in units of 2^e_out.  Tight fit: the largest mantissa of the
+ * rescaled tensor lands in (QMAX/2, QMAX].  The move is limited to 8 binades
+ * per step and the exponent to [-64, 64].  amax_mode == 0 keeps e_out.
+ */
+int32_t ksgd_oracle_next_exponent(uint32_t amax_theta, int32_t theta_bits,
+                                  int32_t e_out, int32_t amax_mode) {
+  if (!amax_mode || amax_theta == 0) return e_out;
+  int64_t A = (int64_t)amax_theta;
+  int64_t Q = qmax_bits(theta_bits);
+  int32_t delta = 0;
+  if (A > Q) {
+    int32_t j = 1;
+    while (A > Q * pow2_i64(j)) ++j;
+    delta = j;
+  } else {
+    int32_t r = 0;
+    while (A * pow2_i64(r + 1) <= Q) ++r;
+    delta = -r;
+  }
+  if (delta > 8) delta = 8;
+  if (delta < -8) delta = -8;
+  int32_t e_next = e_out + delta;
+  if (e_next > 64) e_next = 64;
+  if (e_next < -64) e_next = -64;
+  return e_next;
+}
+
+int32_t ksgd_oracle_max_threads(void) {
+#ifdef _OPENMP
+  return (int32_t)omp_get_max_threads();
+#else
+  return 1;
+#endif
+}

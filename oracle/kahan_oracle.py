@@ -1,0 +1,159 @@
+"""ctypes binding of the C oracle plus the multi-tensor step built on it.
+
+Test infrastructure only.  The per-element arithmetic lives in kahan_oracle.c;
+this module adds what surrounds it in a training step (Algorithm 1 applied to
+every parameter tensor, then the exponent choice for the next step) and keeps
+the per-tensor state a caller would checkpoint.
+"""
+import ctypes
+from dataclasses import dataclass, field
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+from . import build as _build
+
+EXP_FIXED = 0
+EXP_AMAX = 1
+
+
+class OracleElem(ctypes.Structure):
+    _fields_ = [("P", ctypes.c_int64), ("Rq", ctypes.c_int64), ("T", ctypes.c_int64),
+                ("d", ctypes.c_int32), ("q_theta", ctypes.c_int32),
+                ("q_comp", ctypes.c_int32), ("nonfinite", ctypes.c_int32)]
+
+
+class _Stats(ctypes.Structure):
+    _fields_ = [("amax_theta", ctypes.c_uint32), ("amax_comp", ctypes.c_uint32),
+                ("n_sat_theta", ctypes.c_uint64), ("n_sat_comp", ctypes.c_uint64),
+                ("n_nonfinite", ctypes.c_uint64)]
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(_build.build())
+        lib.ksgd_oracle_rne_shift.restype = ctypes.c_int64
+        lib.ksgd_oracle_rne_shift.argtypes = [ctypes.c_int64, ctypes.c_int32]
+        lib.ksgd_oracle_increment.restype = ctypes.c_int32
+        lib.ksgd_oracle_increment.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_int32]
+        lib.ksgd_oracle_element.restype = None
+        lib.ksgd_oracle_element.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_float,
+                                            ctypes.c_float] + [ctypes.c_int32] * 5 + [
+                                                ctypes.POINTER(OracleElem)]
+        lib.ksgd_oracle_step_tensor.restype = ctypes.c_int
+        lib.ksgd_oracle_step_tensor.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+            ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+            ctypes.c_float, ctypes.POINTER(_Stats), ctypes.c_int32]
+        lib.ksgd_oracle_next_exponent.restype = ctypes.c_int32
+        lib.ksgd_oracle_next_exponent.argtypes = [ctypes.c_uint32, ctypes.c_int32,
+                                                  ctypes.c_int32, ctypes.c_int32]
+        lib.ksgd_oracle_max_threads.restype = ctypes.c_int32
+        lib.ksgd_oracle_max_threads.argtypes = []
+        _lib = lib
+    return _lib
+
+
+def oracle_max_threads() -> int:
+    return int(_load().ksgd_oracle_max_threads())
+
+
+def oracle_rne_shift(a: int, r: int) -> int:
+    """a / 2^r rounded to nearest, ties to even."""
+    return int(_load().ksgd_oracle_rne_shift(a, r))
+
+
+def oracle_increment(g: float, lr: float, ec_out: int) -> int:
+    """Algorithm 1 statement 1: eta*g rounded onto the accumulator grid 2^ec_out."""
+    return int(_load().ksgd_oracle_increment(g, lr, ec_out))
+
+
+def oracle_element(q_theta: int, q_comp: int, g: float, lr: float, m: int, n: int, s: int,
+                   e_in: int, e_out: int) -> OracleElem:
+    """Algorithm 1 for one element with m-bit parameter and n-bit compensation."""
+    out = OracleElem()
+    _load().ksgd_oracle_element(q_theta, q_comp, g, lr, m, n, s, e_in, e_out,
+                                ctypes.byref(out))
+    return out
+
+
+def oracle_next_exponent(amax_theta: int, theta_bits: int, e_out: int, mode: int) -> int:
+    """Exponent of the next step from this step's max |P| (max scan)."""
+    return int(_load().ksgd_oracle_next_exponent(amax_theta, theta_bits, e_out, mode))
+
+
+def _storage_dtype(bits: int):
+    return np.int8 if bits <= 8 else np.int16
+
+
+def oracle_step_tensor(theta: np.ndarray, comp: Optional[np.ndarray], grad: np.ndarray,
+                       theta_bits: int, comp_bits: int, overlap_k: int, e_in: int, e_out: int,
+                       lr: float, n_threads: int = 1) -> dict:
+    """Algorithm 1 over one tensor, in place on theta and comp; returns the step's stats."""
+    assert theta.dtype == _storage_dtype(theta_bits) and theta.flags.c_contiguous
+    assert grad.dtype == np.float32 and grad.flags.c_contiguous and grad.size == theta.size
+    if comp_bits:
+        assert comp is not None and comp.dtype == _storage_dtype(comp_bits)
+        assert comp.flags.c_contiguous and comp.size == theta.size
+    st = _Stats()
+    rc = _load().ksgd_oracle_step_tensor(
+        theta.ctypes.data, comp.ctypes.data if comp_bits else None, grad.ctypes.data,
+        theta.size, theta_bits, comp_bits, overlap_k, e_in, e_out,
+        ctypes.c_float(lr), ctypes.byref(st), n_threads)
+    if rc != 0:
+        raise ValueError("oracle rejected the tensor description")
+    return {"amax_theta": st.amax_theta, "amax_comp": st.amax_comp,
+            "n_sat_theta": st.n_sat_theta, "n_sat_comp": st.n_sat_comp,
+            "n_nonfinite": st.n_nonfinite}
+
+
+@dataclass
+class OracleTensor:
+    """One parameter tensor: mantissas, compensation, formats and exponents."""
+    theta: np.ndarray
+    comp: Optional[np.ndarray]
+    theta_bits: int
+    comp_bits: int
+    overlap_k: int = 0
+    exp_theta: int = 0          # exponent of the mantissas now stored
+    exp_theta_next: int = 0     # exponent the next step writes
+    amax_theta: int = 0         # of the most recent step
+    amax_comp: int = 0
+    n_sat_theta: int = 0        # cumulative
+    n_sat_comp: int = 0
+    n_nonfinite: int = 0
+
+    @property
+    def s(self) -> int:
+        return 0 if self.comp_bits == 0 else self.comp_bits - 1 - self.overlap_k
+
+
+@dataclass
+class OracleState:
+    tensors: List[OracleTensor] = field(default_factory=list)
+    mode: int = EXP_AMAX
+    n_threads: int = 1
+
+
+def oracle_step(state: OracleState, grads: Sequence[np.ndarray], lrs: Sequence[float]) -> None:
+    """One training-step update of every tensor, then the exponent choice.
+
+    Each tensor is read at exp_theta and written at exp_theta_next (chosen from
+    the previous step's max scan); afterwards exp_theta becomes the exponent
+    just written and exp_theta_next the tight fit of this step's max |P|.
+    """
+    assert len(grads) == len(state.tensors) == len(lrs)
+    for t, g, lr in zip(state.tensors, grads, lrs):
+        e_in, e_out = t.exp_theta, t.exp_theta_next
+        st = oracle_step_tensor(t.theta, t.comp, g, t.theta_bits, t.comp_bits, t.overlap_k,
+                                e_in, e_out, float(lr), state.n_threads)
+        t.amax_theta, t.amax_comp = st["amax_theta"], st["amax_comp"]
+        t.n_sat_theta += st["n_sat_theta"]
+        t.n_sat_comp += st["n_sat_comp"]
+        t.n_nonfinite += st["n_nonfinite"]
+        t.exp_theta = e_out
+        t.exp_theta_next = oracle_next_exponent(t.amax_theta, t.theta_bits, e_out, state.mode)

@@ -1,0 +1,158 @@
+/*
+ * kahan_sgd.h - C ABI of the lazy update (SGD with Kahan summation) in dynamic
+ * fixed-point, arXiv 1810.05486, Section 2, Eq. 1 and Algorithm 1.
+ *
+ * Number system (Section 2, Fig. 1).  A tensor is an array of signed integer
+ * mantissas sharing one exponent: value = Q * 2^e.  A parameter tensor theta has
+ * m-bit mantissas (m = 8 or 16) at exponent exp_theta.  The accumulator of
+ * Algorithm 1 is kept negated as the compensation c = -acc: n-bit mantissas
+ * (n = 8 or 16; n = 0 selects plain low-precision SGD, Eq. 1) at exponent
+ * exp_theta - s, with s = n - 1 - overlap_k, so that theta + c carries
+ * m + n - 2 - overlap_k magnitude bits (Section 2).
+ *
+ * One step, per element (Algorithm 1, statements 1-4, c = -acc):
+ *   d      = clamp(rne(g * (lr * 2^-(e_out - s))), +-2^30)   one binary32 multiply; NaN -> 0
+ *   T      = theta + c - d          exact, on the finer of the input and output c grids
+ *   P      = rne(T / 2^e_out)       Q_theta' = clamp(P,  +-(2^(m-1) - 1))
+ *   Rq     = rne((T - Q_theta' * 2^e_out) / 2^(e_out - s))
+ *                                   Q_c'     = clamp(Rq, +-(2^(n-1) - 1))
+ * rne = round to nearest, ties to even.  A step reads mantissas stored at exponent
+ * exp_cur and writes them at exp_next (|exp_next - exp_cur| <= 8); in the same pass it
+ * reduces, per tensor, amax_theta = max |P| and amax_comp = max min(|Rq|, 2^31 - 1)
+ * and counts clamped parameter mantissas, clamped compensation mantissas and
+ * non-finite gradients.  After the pass, per tensor (max scan, Section 5):
+ *   exp_cur <- exp_next;  exp_next <- tight fit of amax_theta (KSGD_EXP_AMAX)
+ *   or unchanged (KSGD_EXP_FIXED).  Tight fit: the smallest exponent change that puts
+ *   the largest mantissa in (QMAX/2, QMAX], limited to 8 binades per step and to
+ *   [-64, 64]; amax_theta == 0 keeps the exponent.
+ *
+ * Conventions for every entry point:
+ *   - "device" pointers are CUDA device memory of the current device, "host" pointers
+ *     ordinary host memory.  The caller owns every buffer it passes, including the
+ *     workspace; the library owns only the host-side handle.  Except where an entry
+ *     point says otherwise the library allocates and frees no device memory.
+ *   - All work is enqueued on the stream given to kahan_sgd_init; nothing touches the
+ *     default stream.  Only kahan_sgd_init, kahan_sgd_amax, kahan_sgd_step_host and
+ *     kahan_sgd_destroy wait for the stream.
+ *   - Return value 0 = success, negative = one of the KSGD_ERR_* codes.  No entry
+ *     point throws, aborts or traps on the device.  Saturation and non-finite
+ *     gradients are data, not errors: they are counted.
+ */
+#ifndef KAHAN_SGD_H_
+#define KAHAN_SGD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ksgd_handle ksgd_handle; /* opaque, host memory, library-owned */
+
+typedef struct {
+  void*   theta;          /* device, int8_t[numel] (theta_bits 8) or int16_t[numel] (16); in place; 16-byte aligned */
+  void*   comp;           /* device, int8_t/int16_t[numel] by comp_bits; in place; 16-byte aligned; NULL iff comp_bits == 0 */
+  int64_t numel;          /* > 0 */
+  int32_t theta_bits;     /* 8 | 16 */
+  int32_t comp_bits;      /* 0 (plain SGD, Eq. 1) | 8 | 16 */
+  int32_t overlap_k;      /* 0 .. comp_bits-1; bits of c that overlap theta; ignored when comp_bits == 0 */
+  int32_t exp_theta;      /* exponent of the mantissas now stored, in [-64, 64] */
+  int32_t exp_theta_next; /* exponent the first step writes (== exp_theta for a fresh start), in [-64, 64], within 8 of exp_theta */
+} ksgd_tensor_desc;
+
+typedef enum { KSGD_EXP_FIXED = 0, KSGD_EXP_AMAX = 1 } ksgd_exp_mode;
+
+enum {
+  KSGD_OK = 0,
+  KSGD_ERR_NULL = -1,      /* a required pointer is NULL (or comp is non-NULL with comp_bits == 0) */
+  KSGD_ERR_BITS = -2,      /* theta_bits / comp_bits not in the supported set */
+  KSGD_ERR_OVERLAP = -3,   /* overlap_k outside 0 .. comp_bits-1 */
+  KSGD_ERR_EXP_RANGE = -4, /* an exponent outside [-64, 64] or a first-step change larger than 8 */
+  KSGD_ERR_NUMEL = -5,     /* numel <= 0, n_tensors <= 0, or more than 2^31-1 chunks in total */
+  KSGD_ERR_ALIGN = -6,     /* a device pointer is not 16-byte aligned (workspace: 256) */
+  KSGD_ERR_WORKSPACE = -7, /* workspace smaller than kahan_sgd_workspace_bytes */
+  KSGD_ERR_LR = -8,        /* a learning rate is not finite or not > 0 */
+  KSGD_ERR_CUDA = -9,      /* a CUDA runtime call failed; kahan_sgd_last_cuda_error() has its text */
+  KSGD_ERR_MODE = -10      /* exponent mode not one of ksgd_exp_mode */
+};
+
+/*
+ * Bytes of device workspace kahan_sgd_init needs for this tensor list (per-tensor
+ * exponents, max-scan scratch, counters, per-step arguments and the table that cuts
+ * the ragged list into equal chunks).  Host-only computation.  Returns 0 if the list
+ * is invalid (kahan_sgd_init reports why).
+ */
+size_t kahan_sgd_workspace_bytes(const ksgd_tensor_desc* descs, int32_t n_tensors);
+
+/*
+ * Validate the list, lay out the workspace and copy the chunk table and initial
+ * exponents to it.  descs: host array of n_tensors entries, copied.  workspace: device,
+ * caller-owned, at least kahan_sgd_workspace_bytes, 256-byte aligned; it must stay
+ * valid and untouched by the caller until kahan_sgd_destroy.  cuda_stream: the
+ * cudaStream_t (as void*) all later work is enqueued on; NULL = the legacy default
+ * stream.  Waits for its copies to finish.  On error *out is NULL.
+ * (State of Algorithm 1: "Require theta, ..., previous theta, previous acc".)
+ */
+int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_tensors,
+                   ksgd_exp_mode mode, void* workspace, size_t workspace_bytes,
+                   void* cuda_stream);
+
+/*
+ * One lazy-update step of every tensor (Algorithm 1; Eq. 1 for comp_bits == 0), the
+ * fused max scans and the exponent choice for the next step.  grads: host array of
+ * n_tensors device pointers, each fp32[numel], 16-byte aligned, read-only, may change
+ * from step to step.  lrs: host array of n_tensors learning rates (eta), finite and
+ * > 0.  Both host arrays are consumed before the call returns.  Only enqueues work
+ * (no host synchronisation).  theta and comp are updated in place.
+ */
+int kahan_sgd_step(ksgd_handle* h, const float* const* grads, const float* lrs);
+
+/*
+ * The same step for callers whose tensors live in host memory: copies each tensor's
+ * theta, comp and gradient from host to the device buffers named in the descs (and to
+ * grad_staging), runs the step, copies theta and comp back and waits.  theta_host /
+ * comp_host / grads_host: host arrays of n_tensors host pointers (comp_host[t] ignored
+ * when comp_bits == 0); page-locked memory makes the copies asynchronous.
+ * grad_staging: device, 16-byte aligned, at least 4 * sum(round_up(numel, 4)) bytes,
+ * caller-owned.
+ */
+int kahan_sgd_step_host(ksgd_handle* h, void* const* theta_host, void* const* comp_host,
+                        const float* const* grads_host, const float* lrs,
+                        void* grad_staging, size_t grad_staging_bytes);
+
+/*
+ * Results of the most recent step, per tensor (each output: host array of n_tensors
+ * entries, or NULL to skip): amax_theta = max |P| and amax_comp = max |Rq| of that step
+ * (Section 5 max scan); exp_theta_cur = exponent of the mantissas now in memory;
+ * exp_theta_next = exponent the next step will write; n_sat_theta / n_sat_comp /
+ * n_nonfinite = cumulative counts since init.  Waits for the stream.
+ */
+int kahan_sgd_amax(ksgd_handle* h, uint32_t* amax_theta, uint32_t* amax_comp,
+                   int32_t* exp_theta_cur, int32_t* exp_theta_next,
+                   uint64_t* n_sat_theta, uint64_t* n_sat_comp, uint64_t* n_nonfinite);
+
+/*
+ * Override the exponents the next step writes (host array of n_tensors entries, each in
+ * [-64, 64]).  On the device each is limited to within 8 of the tensor's current
+ * exponent.  Enqueues only.  (Dynamic fixed-point, Section 1: the shared exponent is
+ * the caller's to steer when it knows better than the max scan.)
+ */
+int kahan_sgd_set_exponents(ksgd_handle* h, const int32_t* exp_theta_next);
+
+/* Free the host-side handle (waits for the stream first).  Device buffers stay the caller's. */
+int kahan_sgd_destroy(ksgd_handle* h);
+
+/* Static text for a KSGD_* code. */
+const char* kahan_sgd_strerror(int code);
+
+/* Text of the last CUDA runtime error seen by the calling thread ("" if none). */
+const char* kahan_sgd_last_cuda_error(void);
+
+/* Number of this library's kernels launched by the calling process since load. */
+uint64_t kahan_sgd_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KAHAN_SGD_H_ */

@@ -1,0 +1,178 @@
+"""ctypes binding of the C ABI in include/kahan_sgd.h.
+
+Argument marshalling only: every step of the update runs in the CUDA kernels of
+libkahan_sgd.so.  There is no CPU fallback; if the library is missing the import
+of this module fails with the build command to run.
+"""
+import ctypes
+import os
+from typing import Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIBRARY = os.path.join(_HERE, "libkahan_sgd.so")
+
+KSGD_EXP_FIXED = 0
+KSGD_EXP_AMAX = 1
+
+KSGD_OK = 0
+KSGD_ERR_NULL = -1
+KSGD_ERR_BITS = -2
+KSGD_ERR_OVERLAP = -3
+KSGD_ERR_EXP_RANGE = -4
+KSGD_ERR_NUMEL = -5
+KSGD_ERR_ALIGN = -6
+KSGD_ERR_WORKSPACE = -7
+KSGD_ERR_LR = -8
+KSGD_ERR_CUDA = -9
+KSGD_ERR_MODE = -10
+
+EXPORTS = (
+    "kahan_sgd_workspace_bytes", "kahan_sgd_init", "kahan_sgd_step", "kahan_sgd_step_host",
+    "kahan_sgd_amax", "kahan_sgd_set_exponents", "kahan_sgd_destroy", "kahan_sgd_strerror",
+    "kahan_sgd_last_cuda_error", "kahan_sgd_launch_count",
+)
+
+
+class ksgd_tensor_desc(ctypes.Structure):
+    _fields_ = [("theta", ctypes.c_void_p), ("comp", ctypes.c_void_p), ("numel", ctypes.c_int64),
+                ("theta_bits", ctypes.c_int32), ("comp_bits", ctypes.c_int32),
+                ("overlap_k", ctypes.c_int32), ("exp_theta", ctypes.c_int32),
+                ("exp_theta_next", ctypes.c_int32)]
+
+
+class KahanSgdError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__(f"kahan_sgd error {code}: {text}")
+        self.code = code
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIBRARY):
+        raise ImportError(
+            f"{LIBRARY} is missing: build it with `python -m paper_1810_05486_b200.build` "
+            "(nvcc, sm_100a).  There is no CPU fallback.")
+    lib = ctypes.CDLL(LIBRARY)
+    P = ctypes.POINTER
+    lib.kahan_sgd_workspace_bytes.restype = ctypes.c_size_t
+    lib.kahan_sgd_workspace_bytes.argtypes = [P(ksgd_tensor_desc), ctypes.c_int32]
+    lib.kahan_sgd_init.restype = ctypes.c_int
+    lib.kahan_sgd_init.argtypes = [P(ctypes.c_void_p), P(ksgd_tensor_desc), ctypes.c_int32,
+                                   ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+    lib.kahan_sgd_step.restype = ctypes.c_int
+    lib.kahan_sgd_step.argtypes = [ctypes.c_void_p, P(ctypes.c_void_p), P(ctypes.c_float)]
+    lib.kahan_sgd_step_host.restype = ctypes.c_int
+    lib.kahan_sgd_step_host.argtypes = [ctypes.c_void_p, P(ctypes.c_void_p), P(ctypes.c_void_p),
+                                        P(ctypes.c_void_p), P(ctypes.c_float), ctypes.c_void_p,
+                                        ctypes.c_size_t]
+    lib.kahan_sgd_amax.restype = ctypes.c_int
+    lib.kahan_sgd_amax.argtypes = [ctypes.c_void_p] + [ctypes.c_void_p] * 7
+    lib.kahan_sgd_set_exponents.restype = ctypes.c_int
+    lib.kahan_sgd_set_exponents.argtypes = [ctypes.c_void_p, P(ctypes.c_int32)]
+    lib.kahan_sgd_destroy.restype = ctypes.c_int
+    lib.kahan_sgd_destroy.argtypes = [ctypes.c_void_p]
+    lib.kahan_sgd_strerror.restype = ctypes.c_char_p
+    lib.kahan_sgd_strerror.argtypes = [ctypes.c_int]
+    lib.kahan_sgd_last_cuda_error.restype = ctypes.c_char_p
+    lib.kahan_sgd_last_cuda_error.argtypes = []
+    lib.kahan_sgd_launch_count.restype = ctypes.c_uint64
+    lib.kahan_sgd_launch_count.argtypes = []
+    return lib
+
+
+lib = _load()
+
+
+def _check(code: int) -> None:
+    if code != KSGD_OK:
+        text = lib.kahan_sgd_strerror(code).decode()
+        if code == KSGD_ERR_CUDA:
+            text += ": " + lib.kahan_sgd_last_cuda_error().decode()
+        raise KahanSgdError(code, text)
+
+
+def make_descs(tensors: Sequence[dict]):
+    """ctypes array of ksgd_tensor_desc from dicts with the struct's field names
+    (theta / comp are integer device addresses; comp None or 0 when comp_bits == 0)."""
+    arr = (ksgd_tensor_desc * len(tensors))()
+    for d, t in zip(arr, tensors):
+        d.theta = t["theta"]
+        d.comp = t.get("comp") or None
+        d.numel = t["numel"]
+        d.theta_bits = t["theta_bits"]
+        d.comp_bits = t["comp_bits"]
+        d.overlap_k = t.get("overlap_k", 0)
+        d.exp_theta = t["exp_theta"]
+        d.exp_theta_next = t.get("exp_theta_next", t["exp_theta"])
+    return arr
+
+
+def kahan_sgd_workspace_bytes(descs) -> int:
+    return int(lib.kahan_sgd_workspace_bytes(descs, len(descs)))
+
+
+def kahan_sgd_init(descs, mode: int, workspace: int, workspace_bytes: int, stream: int = 0):
+    """Returns the opaque handle (a ctypes.c_void_p)."""
+    h = ctypes.c_void_p()
+    _check(lib.kahan_sgd_init(ctypes.byref(h), descs, len(descs), mode,
+                              ctypes.c_void_p(workspace), workspace_bytes,
+                              ctypes.c_void_p(stream)))
+    return h
+
+
+def _ptr_array(addresses: Sequence[Optional[int]]):
+    return (ctypes.c_void_p * len(addresses))(*[a or None for a in addresses])
+
+
+def _float_array(values: Sequence[float]):
+    return (ctypes.c_float * len(values))(*values)
+
+
+def kahan_sgd_step(h, grads, lrs) -> None:
+    """grads: device addresses (or a prebuilt ctypes pointer array); lrs: floats (or a
+    prebuilt ctypes float array)."""
+    g = grads if isinstance(grads, ctypes.Array) else _ptr_array(grads)
+    l = lrs if isinstance(lrs, ctypes.Array) else _float_array(lrs)
+    _check(lib.kahan_sgd_step(h, g, l))
+
+
+def kahan_sgd_step_host(h, theta_host, comp_host, grads_host, lrs, grad_staging: int,
+                        grad_staging_bytes: int) -> None:
+    """theta_host / comp_host / grads_host: host addresses per tensor."""
+    th = theta_host if isinstance(theta_host, ctypes.Array) else _ptr_array(theta_host)
+    ch = comp_host if isinstance(comp_host, ctypes.Array) else _ptr_array(comp_host)
+    gh = grads_host if isinstance(grads_host, ctypes.Array) else _ptr_array(grads_host)
+    l = lrs if isinstance(lrs, ctypes.Array) else _float_array(lrs)
+    _check(lib.kahan_sgd_step_host(h, th, ch, gh, l, ctypes.c_void_p(grad_staging),
+                                   grad_staging_bytes))
+
+
+def kahan_sgd_amax(h, n_tensors: int) -> dict:
+    """Per-tensor results of the most recent step as lists (synchronises the stream)."""
+    a_t = (ctypes.c_uint32 * n_tensors)()
+    a_c = (ctypes.c_uint32 * n_tensors)()
+    e_c = (ctypes.c_int32 * n_tensors)()
+    e_n = (ctypes.c_int32 * n_tensors)()
+    s_t = (ctypes.c_uint64 * n_tensors)()
+    s_c = (ctypes.c_uint64 * n_tensors)()
+    nf = (ctypes.c_uint64 * n_tensors)()
+    _check(lib.kahan_sgd_amax(h, a_t, a_c, e_c, e_n, s_t, s_c, nf))
+    return {"amax_theta": list(a_t), "amax_comp": list(a_c), "exp_theta_cur": list(e_c),
+            "exp_theta_next": list(e_n), "n_sat_theta": list(s_t), "n_sat_comp": list(s_c),
+            "n_nonfinite": list(nf)}
+
+
+def kahan_sgd_set_exponents(h, exp_theta_next: Sequence[int]) -> None:
+    arr = (ctypes.c_int32 * len(exp_theta_next))(*exp_theta_next)
+    _check(lib.kahan_sgd_set_exponents(h, arr))
+
+
+def kahan_sgd_destroy(h) -> None:
+    _check(lib.kahan_sgd_destroy(h))
+
+
+def kahan_sgd_strerror(code: int) -> str:
+    return lib.kahan_sgd_strerror(code).decode()
+
+
+def kahan_sgd_launch_count() -> int:
+    return int(lib.kahan_sgd_launch_count())

@@ -1,0 +1,368 @@
+// Host side of the C ABI declared in include/kahan_sgd.h: validation, workspace layout,
+// launches.  All arithmetic of the update runs in the kernels of kahan_sgd_kernels.cuh.
+#include "kahan_sgd.h"
+
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <type_traits>
+#include <vector>
+
+#include "kahan_sgd_kernels.cuh"
+
+namespace {
+
+using namespace ksgd;
+
+std::atomic<uint64_t> g_launches{0};
+thread_local char g_cuda_error[256] = "";
+
+int cuda_fail(cudaError_t e, const char* what) {
+  std::snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", what, cudaGetErrorString(e));
+  return KSGD_ERR_CUDA;
+}
+
+#define KSGD_CUDA(call)                                   \
+  do {                                                    \
+    cudaError_t e__ = (call);                             \
+    if (e__ != cudaSuccess) return cuda_fail(e__, #call); \
+  } while (0)
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Offsets of the workspace regions.  The first four regions are contiguous so that
+// kahan_sgd_amax fetches them with one copy.
+struct Layout {
+  size_t exp_cur, exp_next, amax_last, counters, stats_end;
+  size_t amax_acc, info, grad_ptr, lr, chunks, ticket, total;
+  long long n_chunks;
+};
+
+Layout make_layout(const ksgd_tensor_desc* d, int32_t n) {
+  Layout L{};
+  long long chunks = 0;
+  for (int32_t i = 0; i < n; ++i) chunks += (d[i].numel + kChunk - 1) / kChunk;
+  L.n_chunks = chunks;
+  size_t o = 0;
+  L.exp_cur = o;   o += sizeof(int) * n;
+  L.exp_next = o;  o += sizeof(int) * n;
+  L.amax_last = o; o += sizeof(unsigned int) * 2 * n;
+  o = align_up(o, 8);
+  L.counters = o;  o += sizeof(unsigned long long) * 3 * n;
+  L.stats_end = o;
+  L.amax_acc = o;  o += sizeof(unsigned int) * 2 * n;
+  o = align_up(o, 16);
+  L.info = o;      o += sizeof(TensorInfo) * n;
+  L.grad_ptr = o;  o += sizeof(const float*) * n;
+  L.lr = o;        o += sizeof(float) * n;
+  o = align_up(o, 16);
+  L.chunks = o;    o += sizeof(ChunkRef) * (size_t)chunks;
+  o = align_up(o, 16);
+  L.ticket = o;    o += 16;
+  L.total = align_up(o, 256);
+  return L;
+}
+
+int validate(const ksgd_tensor_desc* d, int32_t n) {
+  if (!d) return KSGD_ERR_NULL;
+  if (n <= 0) return KSGD_ERR_NUMEL;
+  long long chunks = 0;
+  for (int32_t i = 0; i < n; ++i) {
+    const ksgd_tensor_desc& t = d[i];
+    if (t.theta_bits != 8 && t.theta_bits != 16) return KSGD_ERR_BITS;
+    if (t.comp_bits != 0 && t.comp_bits != 8 && t.comp_bits != 16) return KSGD_ERR_BITS;
+    if (!t.theta) return KSGD_ERR_NULL;
+    if ((t.comp_bits != 0) != (t.comp != nullptr)) return KSGD_ERR_NULL;
+    if (t.comp_bits != 0 && (t.overlap_k < 0 || t.overlap_k > t.comp_bits - 1)) return KSGD_ERR_OVERLAP;
+    if (t.numel <= 0) return KSGD_ERR_NUMEL;
+    if (t.exp_theta < kExpMin || t.exp_theta > kExpMax) return KSGD_ERR_EXP_RANGE;
+    if (t.exp_theta_next < kExpMin || t.exp_theta_next > kExpMax) return KSGD_ERR_EXP_RANGE;
+    if (std::abs(t.exp_theta_next - t.exp_theta) > kMaxDelta) return KSGD_ERR_EXP_RANGE;
+    if (reinterpret_cast<uintptr_t>(t.theta) % 16 || reinterpret_cast<uintptr_t>(t.comp) % 16)
+      return KSGD_ERR_ALIGN;
+    chunks += (t.numel + kChunk - 1) / kChunk;
+    if (chunks > 0x7fffffffLL) return KSGD_ERR_NUMEL;
+  }
+  return KSGD_OK;
+}
+
+}  // namespace
+
+struct ksgd_handle {
+  std::vector<ksgd_tensor_desc> descs;
+  Layout layout;
+  StepParams params;
+  char* ws_base;
+  cudaStream_t stream;
+  int32_t n;
+  std::vector<unsigned char> stats_host;   // staging for kahan_sgd_amax
+};
+
+extern "C" {
+
+size_t kahan_sgd_workspace_bytes(const ksgd_tensor_desc* descs, int32_t n_tensors) {
+  if (validate(descs, n_tensors) != KSGD_OK) return 0;
+  return make_layout(descs, n_tensors).total;
+}
+
+int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_tensors,
+                   ksgd_exp_mode mode, void* workspace, size_t workspace_bytes,
+                   void* cuda_stream) {
+  if (!out) return KSGD_ERR_NULL;
+  *out = nullptr;
+  const int v = validate(descs, n_tensors);
+  if (v != KSGD_OK) return v;
+  if (mode != KSGD_EXP_FIXED && mode != KSGD_EXP_AMAX) return KSGD_ERR_MODE;
+  if (!workspace) return KSGD_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(workspace) % 256) return KSGD_ERR_ALIGN;
+  const Layout L = make_layout(descs, n_tensors);
+  if (workspace_bytes < L.total) return KSGD_ERR_WORKSPACE;
+
+  ksgd_handle* h = new (std::nothrow) ksgd_handle();
+  if (!h) return KSGD_ERR_NULL;
+  h->descs.assign(descs, descs + n_tensors);
+  h->layout = L;
+  h->n = n_tensors;
+  h->ws_base = static_cast<char*>(workspace);
+  h->stream = static_cast<cudaStream_t>(cuda_stream);
+  h->stats_host.resize(L.stats_end);
+
+  // Host image of the workspace: exponents, zeroed scans and counters, tensor table,
+  // chunk table.
+  std::vector<unsigned char> img(L.total, 0);
+  int* exp_cur = reinterpret_cast<int*>(img.data() + L.exp_cur);
+  int* exp_next = reinterpret_cast<int*>(img.data() + L.exp_next);
+  TensorInfo* info = reinterpret_cast<TensorInfo*>(img.data() + L.info);
+  ChunkRef* chunks = reinterpret_cast<ChunkRef*>(img.data() + L.chunks);
+  long long c = 0;
+  for (int32_t i = 0; i < n_tensors; ++i) {
+    const ksgd_tensor_desc& t = descs[i];
+    exp_cur[i] = t.exp_theta;
+    exp_next[i] = t.exp_theta_next;
+    info[i].theta = t.theta;
+    info[i].comp = t.comp;
+    info[i].numel = t.numel;
+    info[i].theta_bits = t.theta_bits;
+    info[i].comp_bits = t.comp_bits;
+    info[i].s = t.comp_bits ? t.comp_bits - 1 - t.overlap_k : 0;
+    info[i].pad = 0;
+    const long long nc = (t.numel + kChunk - 1) / kChunk;
+    for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
+  }
+
+  Workspace& w = h->params.ws;
+  char* b = h->ws_base;
+  w.exp_cur = reinterpret_cast<int*>(b + L.exp_cur);
+  w.exp_next = reinterpret_cast<int*>(b + L.exp_next);
+  w.amax_last = reinterpret_cast<unsigned int*>(b + L.amax_last);
+  w.counters = reinterpret_cast<unsigned long long*>(b + L.counters);
+  w.amax_acc = reinterpret_cast<unsigned int*>(b + L.amax_acc);
+  w.info = reinterpret_cast<TensorInfo*>(b + L.info);
+  w.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
+  w.lr = reinterpret_cast<float*>(b + L.lr);
+  w.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
+  w.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
+  h->params.n_tensors = n_tensors;
+  h->params.n_chunks = (int)L.n_chunks;
+  h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
+  h->params.inline_args = n_tensors <= kInlineArgs ? 1 : 0;
+
+  cudaError_t e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+  if (e != cudaSuccess) {
+    delete h;
+    return cuda_fail(e, "workspace upload");
+  }
+  *out = h;
+  return KSGD_OK;
+}
+
+static int check_step_args(const ksgd_handle* h, const float* const* grads, const float* lrs) {
+  if (!h || !grads || !lrs) return KSGD_ERR_NULL;
+  for (int32_t i = 0; i < h->n; ++i) {
+    if (!grads[i]) return KSGD_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(grads[i]) % 16) return KSGD_ERR_ALIGN;
+    if (!std::isfinite(lrs[i]) || !(lrs[i] > 0.0f)) return KSGD_ERR_LR;
+  }
+  return KSGD_OK;
+}
+
+static int launch_step(ksgd_handle* h, const float* const* grads, const float* lrs) {
+  static InlineArgs none{};   // parameter placeholder for long lists
+  const InlineArgs* ia = &none;
+  InlineArgs inl;
+  if (h->params.inline_args) {
+    for (int32_t i = 0; i < h->n; ++i) { inl.grads[i] = grads[i]; inl.lrs[i] = lrs[i]; }
+    for (int32_t i = h->n; i < kInlineArgs; ++i) { inl.grads[i] = nullptr; inl.lrs[i] = 0.0f; }
+    ia = &inl;
+  } else {
+    UploadBatch* ub = new (std::nothrow) UploadBatch;
+    if (!ub) return KSGD_ERR_NULL;
+    for (int32_t first = 0; first < h->n; first += kUploadBatch) {
+      const int count = h->n - first < kUploadBatch ? h->n - first : kUploadBatch;
+      for (int i = 0; i < count; ++i) { ub->grads[i] = grads[first + i]; ub->lrs[i] = lrs[first + i]; }
+      ksgd_upload_args_kernel<<<1, 256, 0, h->stream>>>(*ub, first, count, h->params.ws.grad_ptr,
+                                                        h->params.ws.lr);
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    delete ub;
+    KSGD_CUDA(cudaGetLastError());
+  }
+  ksgd_step_kernel<<<(unsigned)h->params.n_chunks, kThreads, 0, h->stream>>>(h->params, *ia);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  KSGD_CUDA(cudaGetLastError());
+  return KSGD_OK;
+}
+
+int kahan_sgd_step(ksgd_handle* h, const float* const* grads, const float* lrs) {
+  const int v = check_step_args(h, grads, lrs);
+  if (v != KSGD_OK) return v;
+  return launch_step(h, grads, lrs);
+}
+
+int kahan_sgd_step_host(ksgd_handle* h, void* const* theta_host, void* const* comp_host,
+                        const float* const* grads_host, const float* lrs,
+                        void* grad_staging, size_t grad_staging_bytes) {
+  if (!h || !theta_host || !comp_host || !grads_host || !lrs || !grad_staging) return KSGD_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(grad_staging) % 16) return KSGD_ERR_ALIGN;
+  size_t need = 0;
+  for (int32_t i = 0; i < h->n; ++i) need += align_up((size_t)h->descs[i].numel, 4) * sizeof(float);
+  if (grad_staging_bytes < need) return KSGD_ERR_WORKSPACE;
+  std::vector<const float*> dev_grads(h->n);
+  size_t off = 0;
+  for (int32_t i = 0; i < h->n; ++i) {
+    const ksgd_tensor_desc& t = h->descs[i];
+    if (!theta_host[i] || !grads_host[i] || (t.comp_bits && !comp_host[i])) return KSGD_ERR_NULL;
+    if (!std::isfinite(lrs[i]) || !(lrs[i] > 0.0f)) return KSGD_ERR_LR;
+    dev_grads[i] = reinterpret_cast<const float*>(static_cast<char*>(grad_staging) + off);
+    off += align_up((size_t)t.numel, 4) * sizeof(float);
+  }
+  // Host -> device.  Neighbouring tensors whose host and device ranges both continue
+  // where the previous one ended travel as one copy.
+  struct Span { char* dst; const char* src; size_t bytes; };
+  auto flush = [&](std::vector<Span>& spans, cudaMemcpyKind kind) -> cudaError_t {
+    size_t i = 0;
+    while (i < spans.size()) {
+      Span s = spans[i++];
+      while (i < spans.size() && spans[i].dst == s.dst + s.bytes && spans[i].src == s.src + s.bytes)
+        s.bytes += spans[i++].bytes;
+      cudaError_t e = cudaMemcpyAsync(s.dst, s.src, s.bytes, kind, h->stream);
+      if (e != cudaSuccess) return e;
+    }
+    spans.clear();
+    return cudaSuccess;
+  };
+  std::vector<Span> spans;
+  for (int32_t i = 0; i < h->n; ++i) {
+    const ksgd_tensor_desc& t = h->descs[i];
+    spans.push_back({static_cast<char*>(t.theta), static_cast<const char*>(theta_host[i]),
+                     (size_t)t.numel * (t.theta_bits / 8)});
+  }
+  KSGD_CUDA(flush(spans, cudaMemcpyHostToDevice));
+  for (int32_t i = 0; i < h->n; ++i) {
+    const ksgd_tensor_desc& t = h->descs[i];
+    if (t.comp_bits)
+      spans.push_back({static_cast<char*>(t.comp), static_cast<const char*>(comp_host[i]),
+                       (size_t)t.numel * (t.comp_bits / 8)});
+  }
+  KSGD_CUDA(flush(spans, cudaMemcpyHostToDevice));
+  for (int32_t i = 0; i < h->n; ++i) {
+    // the staging slots are padded to 16 bytes; copy the padded length when the host
+    // arrays are laid out the same way so that the copies merge, else the exact length
+    spans.push_back({const_cast<char*>(reinterpret_cast<const char*>(dev_grads[i])),
+                     reinterpret_cast<const char*>(grads_host[i]),
+                     (size_t)h->descs[i].numel * sizeof(float)});
+  }
+  KSGD_CUDA(flush(spans, cudaMemcpyHostToDevice));
+
+  const int r = launch_step(h, dev_grads.data(), lrs);
+  if (r != KSGD_OK) return r;
+
+  // Device -> host: the updated mantissas.
+  for (int32_t i = 0; i < h->n; ++i) {
+    const ksgd_tensor_desc& t = h->descs[i];
+    spans.push_back({static_cast<char*>(theta_host[i]), static_cast<const char*>(t.theta),
+                     (size_t)t.numel * (t.theta_bits / 8)});
+  }
+  KSGD_CUDA(flush(spans, cudaMemcpyDeviceToHost));
+  for (int32_t i = 0; i < h->n; ++i) {
+    const ksgd_tensor_desc& t = h->descs[i];
+    if (t.comp_bits)
+      spans.push_back({static_cast<char*>(comp_host[i]), static_cast<const char*>(t.comp),
+                       (size_t)t.numel * (t.comp_bits / 8)});
+  }
+  KSGD_CUDA(flush(spans, cudaMemcpyDeviceToHost));
+  KSGD_CUDA(cudaStreamSynchronize(h->stream));
+  return KSGD_OK;
+}
+
+int kahan_sgd_amax(ksgd_handle* h, uint32_t* amax_theta, uint32_t* amax_comp,
+                   int32_t* exp_theta_cur, int32_t* exp_theta_next, uint64_t* n_sat_theta,
+                   uint64_t* n_sat_comp, uint64_t* n_nonfinite) {
+  if (!h) return KSGD_ERR_NULL;
+  const Layout& L = h->layout;
+  KSGD_CUDA(cudaMemcpyAsync(h->stats_host.data(), h->ws_base, L.stats_end, cudaMemcpyDeviceToHost,
+                            h->stream));
+  KSGD_CUDA(cudaStreamSynchronize(h->stream));
+  const unsigned char* b = h->stats_host.data();
+  const size_t n = (size_t)h->n;
+  if (exp_theta_cur) std::memcpy(exp_theta_cur, b + L.exp_cur, 4 * n);
+  if (exp_theta_next) std::memcpy(exp_theta_next, b + L.exp_next, 4 * n);
+  if (amax_theta) std::memcpy(amax_theta, b + L.amax_last, 4 * n);
+  if (amax_comp) std::memcpy(amax_comp, b + L.amax_last + 4 * n, 4 * n);
+  if (n_sat_theta) std::memcpy(n_sat_theta, b + L.counters, 8 * n);
+  if (n_sat_comp) std::memcpy(n_sat_comp, b + L.counters + 8 * n, 8 * n);
+  if (n_nonfinite) std::memcpy(n_nonfinite, b + L.counters + 16 * n, 8 * n);
+  return KSGD_OK;
+}
+
+int kahan_sgd_set_exponents(ksgd_handle* h, const int32_t* exp_theta_next) {
+  if (!h || !exp_theta_next) return KSGD_ERR_NULL;
+  for (int32_t i = 0; i < h->n; ++i)
+    if (exp_theta_next[i] < kExpMin || exp_theta_next[i] > kExpMax) return KSGD_ERR_EXP_RANGE;
+  ExponentBatch* eb = new (std::nothrow) ExponentBatch;
+  if (!eb) return KSGD_ERR_NULL;
+  for (int32_t first = 0; first < h->n; first += kUploadBatch) {
+    const int count = h->n - first < kUploadBatch ? h->n - first : kUploadBatch;
+    for (int i = 0; i < count; ++i) eb->exp_next[i] = exp_theta_next[first + i];
+    ksgd_set_exponents_kernel<<<1, 256, 0, h->stream>>>(*eb, first, count, h->params.ws.exp_cur,
+                                                        h->params.ws.exp_next);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+  }
+  delete eb;
+  KSGD_CUDA(cudaGetLastError());
+  return KSGD_OK;
+}
+
+int kahan_sgd_destroy(ksgd_handle* h) {
+  if (!h) return KSGD_ERR_NULL;
+  const cudaError_t e = cudaStreamSynchronize(h->stream);
+  delete h;
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  return KSGD_OK;
+}
+
+const char* kahan_sgd_strerror(int code) {
+  switch (code) {
+    case KSGD_OK: return "success";
+    case KSGD_ERR_NULL: return "a required pointer is NULL (or comp given with comp_bits == 0)";
+    case KSGD_ERR_BITS: return "theta_bits must be 8 or 16 and comp_bits 0, 8 or 16";
+    case KSGD_ERR_OVERLAP: return "overlap_k must lie in 0 .. comp_bits-1";
+    case KSGD_ERR_EXP_RANGE: return "exponent outside [-64, 64] or more than 8 from the current one";
+    case KSGD_ERR_NUMEL: return "numel and n_tensors must be positive (and at most 2^31-1 chunks)";
+    case KSGD_ERR_ALIGN: return "device pointers must be 16-byte aligned (workspace: 256)";
+    case KSGD_ERR_WORKSPACE: return "workspace or staging buffer too small";
+    case KSGD_ERR_LR: return "learning rates must be finite and > 0";
+    case KSGD_ERR_CUDA: return "CUDA runtime error (see kahan_sgd_last_cuda_error)";
+    case KSGD_ERR_MODE: return "unknown exponent mode";
+    default: return "unknown error code";
+  }
+}
+
+const char* kahan_sgd_last_cuda_error(void) { return g_cuda_error; }
+
+uint64_t kahan_sgd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

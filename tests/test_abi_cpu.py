@@ -1,0 +1,105 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every
+symbol the header declares, and rejects bad arguments before touching CUDA."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_1810_05486_b200 import build
+    build.build()
+    from paper_1810_05486_b200 import binding
+    return binding
+
+
+def header_functions():
+    text = open(os.path.join(ROOT, "include", "kahan_sgd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(kahan_sgd_\w+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(B):
+    names = header_functions()
+    assert len(names) >= 10
+    for name in names:
+        assert hasattr(B.lib, name), name
+    assert sorted(B.EXPORTS) == names
+
+
+def test_desc_struct_layout_matches_header(B):
+    assert ctypes.sizeof(B.ksgd_tensor_desc) == 48
+    assert B.ksgd_tensor_desc.numel.offset == 16
+    assert B.ksgd_tensor_desc.exp_theta_next.offset == 40
+
+
+def good(**over):
+    d = dict(theta=0x10000, comp=0x20000, numel=1000, theta_bits=8, comp_bits=8, overlap_k=0,
+             exp_theta=-11)
+    d.update(over)
+    return d
+
+
+@pytest.mark.parametrize("desc,code", [
+    (good(theta_bits=4), "KSGD_ERR_BITS"),
+    (good(comp_bits=12), "KSGD_ERR_BITS"),
+    (good(theta=0), "KSGD_ERR_NULL"),
+    (good(comp=0), "KSGD_ERR_NULL"),
+    (good(comp_bits=0), "KSGD_ERR_NULL"),          # comp given but no compensation asked for
+    (good(overlap_k=8), "KSGD_ERR_OVERLAP"),
+    (good(overlap_k=-1), "KSGD_ERR_OVERLAP"),
+    (good(numel=0), "KSGD_ERR_NUMEL"),
+    (good(exp_theta=65), "KSGD_ERR_EXP_RANGE"),
+    (good(exp_theta=-65), "KSGD_ERR_EXP_RANGE"),
+    (good(exp_theta=0, exp_theta_next=9), "KSGD_ERR_EXP_RANGE"),
+    (good(theta=0x10008), "KSGD_ERR_ALIGN"),
+    (good(comp=0x20004), "KSGD_ERR_ALIGN"),
+])
+def test_init_rejects_bad_descriptions_without_cuda(B, desc, code):
+    descs = B.make_descs([desc])
+    assert B.kahan_sgd_workspace_bytes(descs) == 0
+    with pytest.raises(B.KahanSgdError) as ei:
+        B.kahan_sgd_init(descs, B.KSGD_EXP_AMAX, 0x100000, 1 << 20)
+    assert ei.value.code == getattr(B, code)
+
+
+def test_init_rejects_bad_workspace_and_mode(B):
+    descs = B.make_descs([good()])
+    need = B.kahan_sgd_workspace_bytes(descs)
+    assert need > 0 and need % 256 == 0
+    for args, code in (((B.KSGD_EXP_AMAX, 0, need), B.KSGD_ERR_NULL),
+                       ((B.KSGD_EXP_AMAX, 0x100010, need), B.KSGD_ERR_ALIGN),
+                       ((B.KSGD_EXP_AMAX, 0x100000, need - 1), B.KSGD_ERR_WORKSPACE),
+                       ((7, 0x100000, need), B.KSGD_ERR_MODE)):
+        with pytest.raises(B.KahanSgdError) as ei:
+            B.kahan_sgd_init(descs, *args)
+        assert ei.value.code == code
+    assert B.lib.kahan_sgd_init(None, descs, 1, 1, 0x100000, need, None) == B.KSGD_ERR_NULL
+
+
+def test_workspace_grows_with_the_chunk_table(B):
+    small = B.kahan_sgd_workspace_bytes(B.make_descs([good(numel=10)]))
+    large = B.kahan_sgd_workspace_bytes(B.make_descs([good(numel=10_000_000)]))
+    many = B.kahan_sgd_workspace_bytes(B.make_descs([good(numel=10)] * 500))
+    assert small < large and small < many
+    # ~8 bytes per 8192-element chunk: a billion parameters need about a megabyte
+    big = B.kahan_sgd_workspace_bytes(B.make_descs([good(numel=1_000_000_000, theta_bits=16,
+                                                         comp_bits=16)]))
+    assert big < 2 << 20
+
+
+def test_null_handles_and_strerror(B):
+    assert B.lib.kahan_sgd_step(None, None, None) == B.KSGD_ERR_NULL
+    assert B.lib.kahan_sgd_amax(None, *([None] * 7)) == B.KSGD_ERR_NULL
+    assert B.lib.kahan_sgd_set_exponents(None, None) == B.KSGD_ERR_NULL
+    assert B.lib.kahan_sgd_destroy(None) == B.KSGD_ERR_NULL
+    assert B.lib.kahan_sgd_step_host(None, None, None, None, None, None, 0) == B.KSGD_ERR_NULL
+    seen = {B.kahan_sgd_strerror(c) for c in range(0, -11, -1)}
+    assert len(seen) == 11 and "unknown error code" not in seen
+    assert B.kahan_sgd_strerror(-99) == "unknown error code"
+    assert B.kahan_sgd_launch_count() == 0          # nothing was launched by these checks

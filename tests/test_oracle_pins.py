@@ -328,6 +328,8 @@ def test_bitwidth_closed_form_and_tie_step_counts():
                 oracle_step_tensor(theta, comp, np.array([g], np.float32), m, n, k, e_t, e_t, 1.0)
                 steps += 1
                 assert steps <= 2 ** s
+                if int(theta[0]) == q0:      # one LSB of a grid s bits below theta's per step
+                    assert int(comp[0]) == -steps
             assert steps == want_steps and int(theta[0]) == q0 - 1
 
 

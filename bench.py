@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the lazy-update step (SGD with Kahan summation, dynamic fixed-point).
+
+A "step" is one pass of the whole hot path over one synthetic parameter list: gradient
+quantization, compensated update, requantization, compensation store, per-tensor max
+scans and the exponent choice, i.e. one kahan_sgd_step call.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints one JSON line.  `value` is parameters updated per second with every input
+resident in device memory; `e2e` is the same metric through kahan_sgd_step_host with
+page-locked host buffers (host->device and device->host copies inside the timed region);
+`roofline` relates the step kernel to the measured HBM copy bandwidth; `cpu_baseline` is
+the CPU oracle timed on this machine's cores.  With N > 1 (torchrun) every rank updates
+its own parameter list of the same shape (weak scaling, no data-path collective: the
+update of one tensor never needs another tensor).
+"""
+import argparse
+import ctypes
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "parameters updated/sec and achieved HBM GB/s (% of B200 peak) per Kahan SGD step"
+UNIT = "parameters/s"
+FALLBACK_HBM_GBS = 6650.0
+GRAD_SETS = {"c5_sweep": 2}     # how many gradient sets stay resident and rotate
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c5_sweep")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--sweep-total", type=int, default=0,
+                    help="with --workload c5_sweep: scaled-down total parameter count (profiling)")
+    ap.add_argument("--sweep-tensors", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """nvidia-smi clock samples; only those stamped inside the timed region are kept."""
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "50"], stdout=f,
+                stderr=subprocess.DEVNULL)
+            f.close()
+        except Exception:
+            self.proc = None
+
+    def stop(self, t_begin: float, t_end: float) -> dict:
+        """t_begin / t_end: time.time() around the timed region."""
+        import datetime
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    if not (t_begin <= ts <= t_end + 0.05):
+                        continue
+                    sm.append(float(parts[1]))
+                    mx.append(float(parts[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def pick_workload(W, args):
+    if args.workload == "c5_sweep" and args.sweep_total:
+        return W.scaled_sweep(args.sweep_total, args.sweep_tensors or 256)
+    return W.workload(args.workload)
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import __graft_entry__ as entry
+    if not os.path.exists(os.path.join(ROOT, "paper_1810_05486_b200", "libkahan_sgd.so")):
+        entry.build()
+    from paper_1810_05486_b200 import binding as B
+    from paper_1810_05486_b200 import workloads as W
+    from paper_1810_05486_b200.runner import DeviceRun, HostInputs
+
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    wl = pick_workload(W, args)
+    n = len(wl.tensors)
+    n_sets = GRAD_SETS.get(wl.name, 4)
+    t0 = time.time()
+    host = HostInputs(wl, args.seed + 1000 * rank, n_sets, pinned=True)
+    gen_s = time.time() - t0
+    run = DeviceRun(host, B.KSGD_EXP_AMAX)
+    stream = run.stream
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident throughput ---------------------------------------------------
+    with torch.cuda.stream(stream):
+        for i in range(args.warmup):
+            run.step(i % n_sets)
+        barrier()
+        sampler = ClockSampler(local_rank)
+        if rank == 0:
+            sampler.start()
+            time.sleep(0.2)
+        launches0 = B.kahan_sgd_launch_count()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        wall0 = time.time()
+        ev0.record(stream)
+        for i in range(args.steps):
+            run.step((args.warmup + i) % n_sets)
+        ev1.record(stream)
+        barrier()
+        wall1 = time.time()
+        launches = B.kahan_sgd_launch_count() - launches0
+        ms_total = ev0.elapsed_time(ev1)
+        clocks = sampler.stop(wall0, wall1) if rank == 0 else None
+    stats = run.stats()
+
+    if dist is not None:
+        t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * wl.numel / (ms_step * 1e-3)
+
+    # ---- end to end through host buffers ------------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        th_h, c_h, g_h = run.host_pointer_arrays()
+        run.step_host(th_h, c_h, g_h[0])
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(args.e2e_steps):
+            run.step_host(th_h, c_h, g_h[(i + 1) % n_sets])
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if dist is not None:
+            t = torch.tensor([dt], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        state_bytes = sum(t.numel * (t.theta_bits + t.comp_bits) // 8 for t in wl.tensors)
+        e2e = {"value": world * wl.numel * args.e2e_steps / dt, "unit": UNIT,
+               "h2d_bytes_per_step": state_bytes + 4 * wl.numel,
+               "d2h_bytes_per_step": state_bytes, "steps": args.e2e_steps,
+               "ms_per_step": dt / args.e2e_steps * 1e3}
+    run.close()
+
+    if rank != 0:
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = hbm_peak()
+    achieved = wl.bytes_per_step / (ms_step * 1e-3) / 1e9
+    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
+    traffic = None
+    try:
+        with open(traffic_path) as f:
+            traffic = json.load(f).get(wl.name)
+    except Exception:
+        pass
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int16+int16+f32" if wl.name == "c5_sweep"
+        else "int8/int16+f32", "data": "synthetic",
+        "config": {"workload": wl.name, "tensors": n, "parameters": wl.numel,
+                   "bytes_per_step": wl.bytes_per_step, "grad_sets": n_sets,
+                   "l2": "inputs larger than L2 (%.0f MB touched per step)" % (wl.bytes_per_step / 1e6),
+                   "exponent_mode": "amax", "input_generation_s": round(gen_s, 1)},
+        "achieved_hbm_gbs": achieved,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                     "frac_of_nominal_8000": achieved / 8000.0,
+                     "kernel": "ksgd_step_kernel", "launch_ms": ms_step},
+        "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+        "counters": {"n_sat_theta": int(sum(stats["n_sat_theta"])),
+                     "n_sat_comp": int(sum(stats["n_sat_comp"])),
+                     "n_nonfinite": int(sum(stats["n_nonfinite"]))},
+    }
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(wl, host, budget_core_s=20.0)
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def cpu_baseline(wl, host, budget_core_s):
+    """Time the oracle, as it stands, with all host cores on a bounded sample: one step of
+    the largest tensors of the workload until about budget_core_s core-seconds are spent."""
+    from oracle import oracle_step_tensor, oracle_max_threads
+    cores = oracle_max_threads()
+    done, t_used, k = 0, 0.0, 0
+    order = sorted(range(len(wl.tensors)), key=lambda i: -wl.tensors[i].numel)
+    for i in order:
+        t = wl.tensors[i]
+        th = host.thetas[i].copy()
+        c = host.comps[i].copy() if t.comp_bits else None
+        g = host.grads[0][i]
+        t0 = time.perf_counter()
+        oracle_step_tensor(th, c, g, t.theta_bits, t.comp_bits, t.overlap_k, t.exp_theta,
+                           t.exp_theta, wl.lr, cores)
+        t_used += time.perf_counter() - t0
+        done += t.numel
+        k += 1
+        if t_used * cores >= budget_core_s:
+            break
+    return {"value": done / t_used, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "one step of the %d largest tensors of %s (%d of %d parameters), OpenMP "
+                      "static split over elements" % (k, wl.name, done, wl.numel),
+            "seconds": round(t_used, 3)}
+
+
+def run_reference(args, rank, world):
+    """The reference arm: the CPU oracle on the same workload, bounded sample per step."""
+    if rank != 0:
+        return
+    from oracle import build as oracle_build
+    oracle_build.build()
+    from paper_1810_05486_b200 import workloads as W
+    from oracle import oracle_step_tensor, oracle_max_threads
+    wl = pick_workload(W, args)
+    cores = oracle_max_threads()
+    # sample: the largest tensors up to ~64M parameters per step
+    order = sorted(range(len(wl.tensors)), key=lambda i: -wl.tensors[i].numel)
+    pick, tot = [], 0
+    for i in order:
+        if tot + wl.tensors[i].numel > 64_000_000 and pick:
+            break
+        pick.append(i)
+        tot += wl.tensors[i].numel
+    thetas = [W.theta_slice(wl, i, 0, wl.tensors[i].numel, args.seed) for i in pick]
+    comps = [np.zeros(wl.tensors[i].numel, W.storage_dtype(max(wl.tensors[i].comp_bits, 8)))
+             for i in pick]
+    grads = [W.grad_slice(wl, i, 0, 0, wl.tensors[i].numel, args.seed) for i in pick]
+
+    def one_step():
+        for j, i in enumerate(pick):
+            t = wl.tensors[i]
+            oracle_step_tensor(thetas[j], comps[j] if t.comp_bits else None, grads[j],
+                               t.theta_bits, t.comp_bits, t.overlap_k, t.exp_theta, t.exp_theta,
+                               wl.lr, cores)
+    for _ in range(args.warmup):
+        one_step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        one_step()
+    dt = time.perf_counter() - t0
+    value = tot * args.steps / dt
+    sample = "each step = the %d largest tensors of %s (%d of %d parameters)" % (
+        len(pick), wl.name, tot, wl.numel)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "config": {"workload": wl.name, "tensors": len(wl.tensors), "parameters": wl.numel,
+                       "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

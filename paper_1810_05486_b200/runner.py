@@ -1,0 +1,114 @@
+"""Device-side set-up of a synthetic workload: host buffers, device buffers, descriptors,
+handle.  Used by the benchmark and by the full-size parity tests so that both drive the
+library in exactly the same launch configuration.  PyTorch supplies memory and streams
+only; every step of the update runs in the CUDA library."""
+import ctypes
+from typing import List, Optional
+
+import numpy as np
+
+from . import binding as B
+from . import workloads as W
+
+
+def _carve(wl, itemsize_of):
+    offs, off = [], 0
+    for t in wl.tensors:
+        offs.append(off)
+        off += (t.numel * itemsize_of(t) + 15) // 16 * 16
+    return offs, off
+
+
+class HostInputs:
+    """Host copies of theta, comp and n_sets gradient sets.  Each kind lives in one
+    (optionally page-locked) buffer with every tensor at a 16-byte aligned offset."""
+
+    def __init__(self, wl, seed: int = 0, n_sets: int = 1, pinned: bool = True,
+                 threads: Optional[int] = None):
+        import torch
+        self.wl = wl
+        self.th_offs, th_bytes = _carve(wl, lambda t: t.theta_bits // 8)
+        self.c_offs, c_bytes = _carve(wl, lambda t: max(t.comp_bits, 8) // 8)
+        self.g_offs, g_bytes = _carve(wl, lambda t: 4)
+        alloc = lambda n: torch.zeros(n, dtype=torch.uint8, pin_memory=pinned)  # noqa: E731
+        self.th_buf, self.c_buf = alloc(th_bytes), alloc(c_bytes)
+        self.g_bufs = [alloc(g_bytes) for _ in range(n_sets)]
+        self.thetas = self._views(self.th_buf, self.th_offs,
+                                  lambda t: W.storage_dtype(t.theta_bits))
+        self.comps = self._views(self.c_buf, self.c_offs,
+                                 lambda t: W.storage_dtype(max(t.comp_bits, 8)))
+        W.fill_theta(wl, self.thetas, seed, threads)
+        self.grads: List[List[np.ndarray]] = []
+        for k, gb in enumerate(self.g_bufs):
+            gv = self._views(gb, self.g_offs, lambda t: np.float32)
+            W.fill_grads(wl, k, gv, seed, threads)
+            self.grads.append(gv)
+
+    def _views(self, buf, offs, dtype_of):
+        base = buf.numpy()
+        return [base[o:o + t.numel * np.dtype(dtype_of(t)).itemsize].view(dtype_of(t))
+                for o, t in zip(offs, self.wl.tensors)]
+
+
+class DeviceRun:
+    """Device buffers (same layout as HostInputs), descriptors, workspace and handle."""
+
+    def __init__(self, host: HostInputs, mode: int = B.KSGD_EXP_AMAX, stream=None):
+        import torch
+        self.torch = torch
+        self.host = host
+        wl = self.wl = host.wl
+        self.n = len(wl.tensors)
+        self.dev_th = host.th_buf.cuda(non_blocking=True)
+        self.dev_c = host.c_buf.cuda(non_blocking=True)
+        self.dev_g = [g.cuda(non_blocking=True) for g in host.g_bufs]
+        torch.cuda.synchronize()
+        self.descs = B.make_descs([
+            dict(theta=self.dev_th.data_ptr() + host.th_offs[i],
+                 comp=(self.dev_c.data_ptr() + host.c_offs[i]) if t.comp_bits else None,
+                 numel=t.numel, theta_bits=t.theta_bits, comp_bits=t.comp_bits,
+                 overlap_k=t.overlap_k, exp_theta=t.exp_theta)
+            for i, t in enumerate(wl.tensors)])
+        self.ws_bytes = B.kahan_sgd_workspace_bytes(self.descs)
+        self.workspace = torch.zeros(self.ws_bytes, dtype=torch.uint8, device="cuda")
+        self.stream = stream if stream is not None else torch.cuda.Stream()
+        self.handle = B.kahan_sgd_init(self.descs, mode, self.workspace.data_ptr(),
+                                       self.ws_bytes, self.stream.cuda_stream)
+        self.grad_ptr_sets = [(ctypes.c_void_p * self.n)(*[g.data_ptr() + o for o in host.g_offs])
+                              for g in self.dev_g]
+        self.lrs = (ctypes.c_float * self.n)(*([wl.lr] * self.n))
+
+    def step(self, grad_set: int) -> None:
+        B.kahan_sgd_step(self.handle, self.grad_ptr_sets[grad_set], self.lrs)
+
+    def stats(self) -> dict:
+        return B.kahan_sgd_amax(self.handle, self.n)
+
+    def theta(self, i: int) -> np.ndarray:
+        t = self.wl.tensors[i]
+        nb = t.numel * (t.theta_bits // 8)
+        o = self.host.th_offs[i]
+        return self.dev_th[o:o + nb].cpu().numpy().view(W.storage_dtype(t.theta_bits))
+
+    def comp(self, i: int) -> np.ndarray:
+        t = self.wl.tensors[i]
+        nb = t.numel * (t.comp_bits // 8)
+        o = self.host.c_offs[i]
+        return self.dev_c[o:o + nb].cpu().numpy().view(W.storage_dtype(t.comp_bits))
+
+    def host_pointer_arrays(self):
+        """ctypes arrays of host addresses for kahan_sgd_step_host."""
+        n = self.n
+        th = (ctypes.c_void_p * n)(*[a.ctypes.data for a in self.host.thetas])
+        c = (ctypes.c_void_p * n)(*[a.ctypes.data for a in self.host.comps])
+        g = [(ctypes.c_void_p * n)(*[a.ctypes.data for a in gs]) for gs in self.host.grads]
+        return th, c, g
+
+    def step_host(self, th, c, g) -> None:
+        staging = self.dev_g[0]
+        B.kahan_sgd_step_host(self.handle, th, c, g, self.lrs, staging.data_ptr(), staging.numel())
+
+    def close(self) -> None:
+        if self.handle is not None:
+            B.kahan_sgd_destroy(self.handle)
+            self.handle = None

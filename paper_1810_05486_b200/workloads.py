@@ -139,20 +139,25 @@ def _c4() -> Workload:
     return Workload("c4_alexnet", 4, tuple(tensors), 0.01, 20, "student_t3", None)
 
 
-def c5_sizes(total: int = 1_000_000_000, n_tensors: int = 1024, seed: int = 0) -> List[int]:
-    """Log-uniform tensor sizes 2^10..2^24, rescaled so that they sum to `total` exactly."""
+def c5_sizes(total: int = 1_000_000_000, n_tensors: int = 1024, seed: int = 0,
+             min_size: int = 1024) -> List[int]:
+    """Log-uniform tensor sizes 2^10..2^24, rescaled so that they sum to `total` exactly.
+    The rounding remainder goes to the last tensor (to the largest one if the last would
+    drop below min_size, which only happens for scaled-down totals)."""
     rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, 5, 0xC5])))
     raw = np.floor(2.0 ** (10.0 + 14.0 * rng.random(n_tensors)))
     rho = total / raw.sum()
-    sizes = np.maximum(1024, np.rint(rho * raw)).astype(np.int64)
-    sizes[-1] += total - int(sizes.sum())
-    assert sizes[-1] >= 1024 and int(sizes.sum()) == total
+    sizes = np.maximum(min_size, np.rint(rho * raw)).astype(np.int64)
+    rest = total - int(sizes.sum())
+    sink = n_tensors - 1 if sizes[-1] + rest >= min_size else int(np.argmax(sizes))
+    sizes[sink] += rest
+    assert sizes.min() >= min_size and int(sizes.sum()) == total
     return [int(x) for x in sizes]
 
 
-def _c5(total: int = 1_000_000_000, n_tensors: int = 1024) -> Workload:
+def _c5(total: int = 1_000_000_000, n_tensors: int = 1024, min_size: int = 1024) -> Workload:
     tensors = tuple(TensorSpec(f"t{i}", n, 16, 16, 0, -15, 1e-3)
-                    for i, n in enumerate(c5_sizes(total, n_tensors)))
+                    for i, n in enumerate(c5_sizes(total, n_tensors, 0, min_size)))
     return Workload("c5_sweep", 5, tensors, 0.01, 10, "normal", 2)
 
 
@@ -167,7 +172,7 @@ def workload(name: str) -> Workload:
 
 def scaled_sweep(total: int, n_tensors: int) -> Workload:
     """The c5 recipe at a smaller size (same size law and formats); used by quick tests."""
-    return _c5(total, n_tensors)
+    return _c5(total, n_tensors, min_size=max(1, min(1024, total // (64 * n_tensors))))
 
 
 # ----------------------------------------------------------------------------- drawing

@@ -74,7 +74,8 @@ enum {
   KSGD_ERR_WORKSPACE = -7, /* workspace smaller than kahan_sgd_workspace_bytes */
   KSGD_ERR_LR = -8,        /* a learning rate is not finite or not > 0 */
   KSGD_ERR_CUDA = -9,      /* a CUDA runtime call failed; kahan_sgd_last_cuda_error() has its text */
-  KSGD_ERR_MODE = -10      /* exponent mode not one of ksgd_exp_mode */
+  KSGD_ERR_MODE = -10,     /* exponent mode not one of ksgd_exp_mode */
+  KSGD_ERR_DEVICE = -11    /* a bounded wait inside a kernel ran out (reported by kahan_sgd_amax); the step's results are invalid */
 };
 
 /*

@@ -25,6 +25,7 @@ KSGD_ERR_WORKSPACE = -7
 KSGD_ERR_LR = -8
 KSGD_ERR_CUDA = -9
 KSGD_ERR_MODE = -10
+KSGD_ERR_DEVICE = -11
 
 EXPORTS = (
     "kahan_sgd_workspace_bytes", "kahan_sgd_init", "kahan_sgd_step", "kahan_sgd_step_host",

@@ -35,7 +35,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // Offsets of the workspace regions.  The first four regions are contiguous so that
 // kahan_sgd_amax fetches them with one copy.
 struct Layout {
-  size_t exp_cur, exp_next, amax_last, counters, stats_end;
+  size_t exp_cur, exp_next, amax_last, counters, error, stats_end;
   size_t amax_acc, info, grad_ptr, lr, chunks, ticket, total;
   long long n_chunks;
 };
@@ -51,6 +51,7 @@ Layout make_layout(const ksgd_tensor_desc* d, int32_t n) {
   L.amax_last = o; o += sizeof(unsigned int) * 2 * n;
   o = align_up(o, 8);
   L.counters = o;  o += sizeof(unsigned long long) * 3 * n;
+  L.error = o;     o += 8;
   L.stats_end = o;
   L.amax_acc = o;  o += sizeof(unsigned int) * 2 * n;
   o = align_up(o, 16);
@@ -97,6 +98,7 @@ struct ksgd_handle {
   char* ws_base;
   cudaStream_t stream;
   int32_t n;
+  int grid;
   std::vector<unsigned char> stats_host;   // staging for kahan_sgd_amax
 };
 
@@ -158,6 +160,7 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
   w.exp_next = reinterpret_cast<int*>(b + L.exp_next);
   w.amax_last = reinterpret_cast<unsigned int*>(b + L.amax_last);
   w.counters = reinterpret_cast<unsigned long long*>(b + L.counters);
+  w.error = reinterpret_cast<unsigned int*>(b + L.error);
   w.amax_acc = reinterpret_cast<unsigned int*>(b + L.amax_acc);
   w.info = reinterpret_cast<TensorInfo*>(b + L.info);
   w.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
@@ -169,7 +172,20 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
   h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
   h->params.inline_args = n_tensors <= kInlineArgs ? 1 : 0;
 
-  cudaError_t e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
+  // Persistent grid: one block per SM (fewer if the list has fewer tiles).
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(ksgd_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSharedBytes);
+  if (e != cudaSuccess) {
+    delete h;
+    return cuda_fail(e, "device query");
+  }
+  h->grid = (int)(L.n_chunks < (long long)sms ? L.n_chunks : (long long)sms);
+
+  e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
   if (e != cudaSuccess) {
     delete h;
@@ -210,7 +226,7 @@ static int launch_step(ksgd_handle* h, const float* const* grads, const float* l
     delete ub;
     KSGD_CUDA(cudaGetLastError());
   }
-  ksgd_step_kernel<<<(unsigned)h->params.n_chunks, kThreads, 0, h->stream>>>(h->params, *ia);
+  ksgd_step_kernel<<<(unsigned)h->grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, *ia);
   g_launches.fetch_add(1, std::memory_order_relaxed);
   KSGD_CUDA(cudaGetLastError());
   return KSGD_OK;
@@ -315,6 +331,9 @@ int kahan_sgd_amax(ksgd_handle* h, uint32_t* amax_theta, uint32_t* amax_comp,
   if (n_sat_theta) std::memcpy(n_sat_theta, b + L.counters, 8 * n);
   if (n_sat_comp) std::memcpy(n_sat_comp, b + L.counters + 8 * n, 8 * n);
   if (n_nonfinite) std::memcpy(n_nonfinite, b + L.counters + 16 * n, 8 * n);
+  unsigned int dev_err = 0;
+  std::memcpy(&dev_err, b + L.error, 4);
+  if (dev_err != 0) return KSGD_ERR_DEVICE;
   return KSGD_OK;
 }
 
@@ -357,6 +376,7 @@ const char* kahan_sgd_strerror(int code) {
     case KSGD_ERR_LR: return "learning rates must be finite and > 0";
     case KSGD_ERR_CUDA: return "CUDA runtime error (see kahan_sgd_last_cuda_error)";
     case KSGD_ERR_MODE: return "unknown exponent mode";
+    case KSGD_ERR_DEVICE: return "a bounded wait inside the step kernel ran out; results of that step are invalid";
     default: return "unknown error code";
   }
 }

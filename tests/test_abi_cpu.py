@@ -99,7 +99,7 @@ def test_null_handles_and_strerror(B):
     assert B.lib.kahan_sgd_set_exponents(None, None) == B.KSGD_ERR_NULL
     assert B.lib.kahan_sgd_destroy(None) == B.KSGD_ERR_NULL
     assert B.lib.kahan_sgd_step_host(None, None, None, None, None, None, 0) == B.KSGD_ERR_NULL
-    seen = {B.kahan_sgd_strerror(c) for c in range(0, -11, -1)}
-    assert len(seen) == 11 and "unknown error code" not in seen
+    seen = {B.kahan_sgd_strerror(c) for c in range(0, -12, -1)}
+    assert len(seen) == 12 and "unknown error code" not in seen
     assert B.kahan_sgd_strerror(-99) == "unknown error code"
     assert B.kahan_sgd_launch_count() == 0          # nothing was launched by these checks

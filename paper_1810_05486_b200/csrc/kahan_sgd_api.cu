@@ -61,7 +61,7 @@ Layout make_layout(const ksgd_tensor_desc* d, int32_t n) {
   o = align_up(o, 16);
   L.chunks = o;    o += sizeof(ChunkRef) * (size_t)chunks;
   o = align_up(o, 16);
-  L.ticket = o;    o += 16;
+  L.ticket = o;    o += 16;   // ticket, next_tile
   L.total = align_up(o, 256);
   return L;
 }
@@ -167,6 +167,7 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
   w.lr = reinterpret_cast<float*>(b + L.lr);
   w.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
   w.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
+  w.next_tile = w.ticket + 1;
   h->params.n_tensors = n_tensors;
   h->params.n_chunks = (int)L.n_chunks;
   h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
@@ -184,6 +185,7 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
     return cuda_fail(e, "device query");
   }
   h->grid = (int)(L.n_chunks < (long long)sms ? L.n_chunks : (long long)sms);
+  reinterpret_cast<unsigned int*>(img.data() + L.ticket)[1] = (unsigned int)h->grid;
 
   e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);

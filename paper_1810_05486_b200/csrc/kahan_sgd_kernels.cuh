@@ -72,6 +72,7 @@ struct Workspace {
   float* lr;                       // [n]
   ChunkRef* chunks;                // [n_chunks]
   unsigned int* ticket;            // blocks finished in the running step
+  unsigned int* next_tile;         // next tile not yet handed to a block (starts at gridDim.x)
 };
 
 struct StepParams {
@@ -110,19 +111,25 @@ struct StepCoef {
   int qmax_c;    // 2^(n-1) - 1
 };
 
-// One tile as the producer describes it to the consumers (lives in shared memory).
-struct TileDesc {
-  StepCoef coef;
+// One tile as the producer describes it to the consumers (lives in shared memory).  The
+// first 48 bytes are all the steady-state path reads (three 16-byte loads).
+struct __align__(16) TileDesc {
+  float scale;          // lr * 2^-(e_out - s)
+  float pow2s_neg;      // -2^s
+  float inv2s;          // 2^-s
+  float qmax_t;         // 2^(m-1) - 1
   void* theta;          // global address of the tile's first theta mantissa
   void* comp;           // same for the compensation (unused in plain mode)
-  const float* grad;    // same for the gradient
   int tensor;
-  int count;            // valid elements in the tile
   int n_bulk;           // elements that arrived through the bulk copies (multiple of 16)
-  int theta_bits;
-  int comp_bits;
-  int pad;
+  int count;            // valid elements in the tile
+  int flags;            // kFlag* | format id
+  StepCoef coef;        // for the general path
+  const float* grad;    // global address of the tile's first gradient
 };
+constexpr int kFlagFormatMask = 7;   // 0..5 = (8,0) (8,8) (8,16) (16,0) (16,8) (16,16)
+constexpr int kFlagSteady = 8;       // no exponent change: the exact-fp32 path applies
+constexpr int kFlagStop = 16;        // no more tiles for this block
 
 // Max scans and counters of the rare path, one set per consumer warp (shared memory).
 struct WarpSlots {
@@ -230,21 +237,24 @@ __device__ __forceinline__ StepCoef make_coef(const TensorInfo& ti, int e_in, in
   return k;
 }
 
-// Algorithm 1 for elements [first, first+n) of a tile with 64-bit intermediates, straight
-// from and to global memory.  This is the rare path: exponent changes, vectors in which
-// theta saturates or a gradient is not finite, and ragged tails.  It is kept out of line
-// (one copy for all formats) so that it costs the steady-state path no registers.
-__device__ __noinline__ void update_general(const TileDesc* td, int first, int n, WarpSlots* slots) {
-  const StepCoef k = td->coef;
-  const int tb = td->theta_bits, cb = td->comp_bits;
+// Algorithm 1 for elements [first, first+n) with 64-bit intermediates, in place on arrays
+// that may live in a shared-memory stage or in global memory.  This is the general path:
+// exponent changes, vectors in which theta saturates or a gradient is not finite (or very
+// large), and ragged tails.  It is kept out of line, one copy for all formats, so that it
+// costs the steady-state path no registers.
+__device__ __noinline__ void update_general(const StepCoef* coef, int tb, int cb, void* theta,
+                                            void* comp, const float* grad, int first, int n,
+                                            WarpSlots* slots) {
+  const StepCoef k = *coef;
   unsigned int amax_t = 0, amax_c = 0, n_sat_t = 0, n_sat_c = 0, n_nf = 0;
+#pragma unroll 1
   for (int e = first; e < first + n; ++e) {
-    const int qt = tb == 8 ? (int)static_cast<const signed char*>(td->theta)[e]
-                           : (int)static_cast<const short*>(td->theta)[e];
+    const int qt = tb == 8 ? (int)static_cast<const signed char*>(theta)[e]
+                           : (int)static_cast<const short*>(theta)[e];
     int qc = 0;
-    if (cb == 8) qc = (int)static_cast<const signed char*>(td->comp)[e];
-    else if (cb == 16) qc = (int)static_cast<const short*>(td->comp)[e];
-    const float g = td->grad[e];
+    if (cb == 8) qc = (int)static_cast<const signed char*>(comp)[e];
+    else if (cb == 16) qc = (int)static_cast<const short*>(comp)[e];
+    const float g = grad[e];
     const int d = quantize_increment(g, k.scale);
     const long long T = (long long)qt * (1LL << k.sh_t) + (long long)qc * (1LL << k.sh_c) -
                         (long long)d * (1LL << k.sh_d);
@@ -253,8 +263,8 @@ __device__ __noinline__ void update_general(const TileDesc* td, int first, int n
     const unsigned long long aP = (unsigned long long)(P < 0 ? -P : P);
     amax_t = max(amax_t, (unsigned int)aP);
     n_sat_t += (P != Pc);
-    if (tb == 8) static_cast<signed char*>(td->theta)[e] = (signed char)Pc;
-    else static_cast<short*>(td->theta)[e] = (short)Pc;
+    if (tb == 8) static_cast<signed char*>(theta)[e] = (signed char)Pc;
+    else static_cast<short*>(theta)[e] = (short)Pc;
     if (cb) {
       const long long R = T - Pc * (1LL << k.r_t);
       const long long Rq = rne_shift64(R, k.r_c);
@@ -263,8 +273,8 @@ __device__ __noinline__ void update_general(const TileDesc* td, int first, int n
       if (aR > 0x7fffffffULL) aR = 0x7fffffffULL;
       amax_c = max(amax_c, (unsigned int)aR);
       n_sat_c += (Rq != Rc);
-      if (cb == 8) static_cast<signed char*>(td->comp)[e] = (signed char)Rc;
-      else static_cast<short*>(td->comp)[e] = (short)Rc;
+      if (cb == 8) static_cast<signed char*>(comp)[e] = (signed char)Rc;
+      else static_cast<short*>(comp)[e] = (short)Rc;
     }
     n_nf += ((__float_as_uint(g) & 0x7f800000u) == 0x7f800000u);
   }
@@ -336,123 +346,153 @@ __device__ __forceinline__ void set_pack_word(Pack<BYTES>& r, int w, unsigned in
   }
 }
 
-// Sign-extended element i of a pack of BITS-wide integers.
+// ----------------------------------------------------------------------------------------
+// Steady state (no exponent change): one vector of V elements on the FP32 pipe, used as an
+// exact integer unit.  With M = 1.5 * 2^23 every float in [2^23, 2^24) is an integer whose
+// low mantissa bits are that integer in two's complement relative to M, an addition that
+// lands there rounds to nearest-even on the integer grid, and sums, differences and FMAs
+// of integers below 2^24 are exact.  Per element:
+//   qtM = M + qt, qcm = M + bias + qc   mantissa bytes spliced under M's exponent (PRMT)
+//   y   = g*scale + (M + bias)          = M + bias + d, d = rne(g*scale)   (stmt 1)
+//   u   = qcm - y                       = qc - d
+//   Pm  = fma(u, 2^-s, qtM)             = M + rne((qt*2^s + u) / 2^s) = M + P  (stmt 2;
+//                                         the tie falls on the parity of P itself)
+//   w   = Pm - qtM                      = P - qt
+//   r0  = fma(w, -2^s, u)               = T - P*2^s                       (stmt 3)
+// theta' and c' are the low bits of Pm and of r0 + M.  The vector is handed to
+// update_general instead (returns false, nothing stored) when some |g*scale| exceeds 4e6
+// (y must stay below 2^24) or is Inf or NaN, or some |P| exceeds QMAX: exactly the cases
+// in which the magnitudes above could leave the exact range or a clamp is needed.
+
+constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23, bits 0x4B400000
+constexpr unsigned int kMagicBits = 0x4B400000u;
+
+// M + 2^(BITS-1) + q for element i of a pack whose sign bits have been flipped.
 template <int BITS, int BYTES>
-__device__ __forceinline__ int unpack_elem(const Pack<BYTES>& r, int i) {
+__device__ __forceinline__ float magic_elem(const Pack<BYTES>& r, int i) {
   if constexpr (BITS == 8) {
-    const unsigned int w = pack_word(r, i >> 2);
-    return (int)(signed char)(w >> (8 * (i & 3)));
+    return __uint_as_float(__byte_perm(pack_word(r, i >> 2), kMagicBits, 0x7640u | (unsigned)(i & 3)));
   } else {
-    const unsigned int w = pack_word(r, i >> 1);
-    return (i & 1) ? ((int)w >> 16) : (int)(short)(w & 0xffffu);
+    return __uint_as_float(__byte_perm(pack_word(r, i >> 1), kMagicBits, (i & 1) ? 0x7632u : 0x7610u));
   }
 }
 
+template <int BITS, int BYTES>
+__device__ __forceinline__ void flip_signs(Pack<BYTES>& r) {
+  constexpr unsigned int m = BITS == 8 ? 0x80808080u : 0x80008000u;
+#pragma unroll
+  for (int w = 0; w < BYTES / 4; ++w) set_pack_word(r, w, pack_word(r, w) ^ m);
+}
+
+// Low BITS bits of V magic floats, packed.
 template <int BITS, int V>
-__device__ __forceinline__ Pack<V * BITS / 8> pack_elems(const int (&x)[V]) {
+__device__ __forceinline__ Pack<V * BITS / 8> pack_magic(const float (&x)[V]) {
   Pack<V * BITS / 8> r;
   if constexpr (BITS == 8) {
 #pragma unroll
     for (int w = 0; w < V / 4; ++w) {
-      const unsigned int lo = __byte_perm((unsigned)x[4 * w], (unsigned)x[4 * w + 1], 0x0040);
-      const unsigned int hi = __byte_perm((unsigned)x[4 * w + 2], (unsigned)x[4 * w + 3], 0x0040);
+      const unsigned int lo = __byte_perm(__float_as_uint(x[4 * w]), __float_as_uint(x[4 * w + 1]), 0x0040);
+      const unsigned int hi = __byte_perm(__float_as_uint(x[4 * w + 2]), __float_as_uint(x[4 * w + 3]), 0x0040);
       set_pack_word(r, w, __byte_perm(lo, hi, 0x5410));
     }
   } else {
 #pragma unroll
     for (int w = 0; w < V / 2; ++w)
-      set_pack_word(r, w, __byte_perm((unsigned)x[2 * w], (unsigned)x[2 * w + 1], 0x5410));
+      set_pack_word(r, w, __byte_perm(__float_as_uint(x[2 * w]), __float_as_uint(x[2 * w + 1]), 0x5410));
   }
   return r;
 }
 
-// ----------------------------------------------------------------------------------------
-// Steady state (no exponent change, s >= 1 or plain mode): one vector of V elements in
-// 32-bit arithmetic.  T = qt*2^s + u with u = qc - d; rounding T by s bits to nearest-even
-// only needs u, the parity of the truncated quotient and qt.  Returns false, having stored
-// nothing, if any element saturates theta or has a non-finite gradient: the caller then
-// runs the vector through update_general.
+struct SteadyCoef {
+  float scale;      // lr * 2^-(e - s)
+  float pow2s_neg;  // -2^s
+  float inv2s;      // 2^-s
+  float qmax_t;     // 2^(m-1) - 1
+};
+
+struct TileHot {       // the consumers' copy of the first 48 bytes of a TileDesc
+  SteadyCoef k;
+  unsigned char* theta;
+  unsigned char* comp;
+  int tensor, n_bulk, count, flags;
+};
 
 template <int TB, int CB, int V>
-__device__ __forceinline__ bool update_vector(const Pack<V * TB / 8>& pt,
-                                              const Pack<(CB ? V * CB / 8 : 8)>& pc,
-                                              const Pack<V * 4>& pg, float scale, int s, int qmax_t,
+__device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V * CB / 8 : 8)> pc,
+                                              const Pack<V * 4>& pg, const SteadyCoef& k,
                                               Pack<V * TB / 8>& ot, Pack<(CB ? V * CB / 8 : 8)>& oc,
-                                              unsigned int& amax_t, unsigned int& amax_c) {
+                                              float& amax_t, float& amax_c) {
   constexpr bool HAS_COMP = CB != 0;
-  int nt[V], nc[V];
-  const int hm1 = HAS_COMP ? ((1 << (s - 1)) - 1) : 0;
-  int mxP = -0x7fffffff, mnP = 0x7fffffff, mxR = 0, mnR = 0;
-  float nf = 0.0f;
+  constexpr float bias_t = (float)(1 << (TB - 1));
+  constexpr float bias_c = HAS_COMP ? (float)(1 << ((CB ? CB : 8) - 1)) : 0.0f;
+  flip_signs<TB>(pt);
+  if constexpr (HAS_COMP) flip_signs<(CB ? CB : 8)>(pc);
+  float Pm[V], rm[V];
+  float sum_abs = 0.0f, aX = 0.0f, aP = 0.0f, aR = 0.0f;
 #pragma unroll
   for (int i = 0; i < V; ++i) {
-    const int qt = unpack_elem<TB>(pt, i);
+    const float qtM = __fadd_rn(magic_elem<TB>(pt, i), -bias_t);
     const float g = __uint_as_float(pack_word(pg, i));
-    const int d = quantize_increment(g, scale);
-    nf = fmaf(g, 0.0f, nf);             // stays 0 unless some g is Inf or NaN
-    int P, r0;
-    if constexpr (HAS_COMP) {
-      const int u = unpack_elem<(CB ? CB : 8)>(pc, i) - d;
-      const int par = (qt + (u >> s)) & 1;
-      const int w = (u + hm1 + par) >> s;
-      P = qt + w;
-      r0 = u - w * (1 << s);
-      mxR = max(mxR, r0);
-      mnR = min(mnR, r0);
-    } else {
-      P = qt - d;
-      r0 = 0;
-    }
-    nt[i] = P;
-    nc[i] = r0;
-    mxP = max(mxP, P);
-    mnP = min(mnP, P);
+    const float x = __fmul_rn(g, k.scale);              // the one binary32 multiply
+    sum_abs = __fadd_rn(sum_abs, fabsf(x));             // Inf or NaN if any x is
+    aX = fmaxf(aX, fabsf(x));
+    const float y = __fadd_rn(x, kMagic + bias_c);      // rounds x to nearest-even integer
+    float u;
+    if constexpr (HAS_COMP) u = __fadd_rn(magic_elem<(CB ? CB : 8)>(pc, i), -y);
+    else u = __fadd_rn(kMagic, -y);
+    const float P = __fmaf_rn(u, k.inv2s, qtM);
+    const float w = __fadd_rn(P, -qtM);
+    const float r0 = __fmaf_rn(w, k.pow2s_neg, u);
+    Pm[i] = P;
+    rm[i] = __fadd_rn(r0, kMagic);
+    aP = fmaxf(aP, fabsf(__fadd_rn(P, -kMagic)));
+    if constexpr (HAS_COMP) aR = fmaxf(aR, fabsf(r0));
   }
-  if ((mxP > qmax_t) | (mnP < -qmax_t) | (nf != nf)) return false;
-  amax_t = max(amax_t, (unsigned int)max(mxP, -mnP));
-  if constexpr (HAS_COMP) amax_c = max(amax_c, (unsigned int)max(mxR, -mnR));
-  ot = pack_elems<TB, V>(nt);
-  if constexpr (HAS_COMP) oc = pack_elems<CB, V>(nc);
+  if (!(sum_abs < 3.0e38f) | (aX > 4000000.0f) | (aP > k.qmax_t)) return false;
+  amax_t = fmaxf(amax_t, aP);
+  if constexpr (HAS_COMP) amax_c = fmaxf(amax_c, aR);
+  ot = pack_magic<TB, V>(Pm);
+  if constexpr (HAS_COMP) oc = pack_magic<CB, V>(rm);
   return true;
 }
 
 // All vectors of one tile that belong to this consumer thread.
 template <int TB, int CB>
-__device__ __forceinline__ void consume_tile(const TileDesc* td, const unsigned char* stage,
-                                             int ctid, WarpSlots* slots, unsigned int& amax_t,
-                                             unsigned int& amax_c) {
+__device__ __forceinline__ void consume_tile(const TileHot& h, const TileDesc* td, unsigned char* stage,
+                                             int ctid, WarpSlots* slots, float& amax_t, float& amax_c) {
   constexpr bool HAS_COMP = CB != 0;
   constexpr int V = (TB == 8) ? 16 : 8;              // 16 bytes of theta per vector
   constexpr int TBYTES = V * TB / 8;
   constexpr int CBYTES = HAS_COMP ? V * CB / 8 : 8;
-  const StepCoef& k = td->coef;
-  const bool steady = (k.delta == 0) && (!HAS_COMP || k.s >= 1);
-  const int n_vec = td->n_bulk / V;
-  if (steady) {
-    const float scale = k.scale;
-    const int s = k.s, qmax_t = k.qmax_t;
-    unsigned char* theta_g = static_cast<unsigned char*>(td->theta);
-    unsigned char* comp_g = static_cast<unsigned char*>(td->comp);
-    for (int v = ctid; v < n_vec; v += kConsumers) {
-      const Pack<TBYTES> pt = load_pack<TBYTES>(stage + kStageThetaOff + v * TBYTES);
-      Pack<CBYTES> pc;
-      if constexpr (HAS_COMP) pc = load_pack<CBYTES>(stage + kStageCompOff + v * CBYTES);
-      const Pack<V * 4> pg = load_pack<V * 4>(stage + kStageGradOff + v * (V * 4));
-      Pack<TBYTES> ot;
-      Pack<CBYTES> oc;
-      if (update_vector<TB, CB, V>(pt, pc, pg, scale, s, qmax_t, ot, oc, amax_t, amax_c)) {
-        store_pack<TBYTES>(theta_g + (size_t)v * TBYTES, ot);
-        if constexpr (HAS_COMP) store_pack<CBYTES>(comp_g + (size_t)v * CBYTES, oc);
-      } else {
-        update_general(td, v * V, V, slots);
-      }
+  const bool steady = (h.flags & kFlagSteady) != 0;
+  const int n_vec = h.n_bulk / V;
+  unsigned char* theta_s = stage + kStageThetaOff;
+  unsigned char* comp_s = stage + kStageCompOff;
+  const float* grad_s = reinterpret_cast<const float*>(stage + kStageGradOff);
+  for (int v = ctid; v < n_vec; v += kConsumers) {
+    Pack<TBYTES> ot;
+    Pack<CBYTES> oc;
+    bool done = false;
+    if (steady) {
+      const Pack<TBYTES> pt = load_pack<TBYTES>(theta_s + v * TBYTES);
+      Pack<CBYTES> pc{};
+      if constexpr (HAS_COMP) pc = load_pack<CBYTES>(comp_s + v * CBYTES);
+      const Pack<V * 4> pg = load_pack<V * 4>(grad_s + v * V);
+      done = update_vector<TB, CB, V>(pt, pc, pg, h.k, ot, oc, amax_t, amax_c);
     }
-  } else {
-    for (int v = ctid; v < n_vec; v += kConsumers) update_general(td, v * V, V, slots);
+    if (!done) {
+      // general path, in place in the stage; then the vector goes out like any other
+      update_general(&td->coef, TB, CB, theta_s, comp_s, grad_s, v * V, V, slots);
+      ot = load_pack<TBYTES>(theta_s + v * TBYTES);
+      if constexpr (HAS_COMP) oc = load_pack<CBYTES>(comp_s + v * CBYTES);
+    }
+    store_pack<TBYTES>(h.theta + (size_t)v * TBYTES, ot);
+    if constexpr (HAS_COMP) store_pack<CBYTES>(h.comp + (size_t)v * CBYTES, oc);
   }
-  // ragged tail (fewer than 16 elements) that the bulk copies did not bring
-  const int e = td->n_bulk + ctid;
-  if (e < td->count) update_general(td, e, 1, slots);
+  // ragged tail (fewer than 16 elements) that the bulk copies did not bring: in place in
+  // global memory
+  const int e = h.n_bulk + ctid;
+  if (e < h.count) update_general(&td->coef, TB, CB, h.theta, h.comp, td->grad, e, 1, slots);
 }
 
 // Next exponent from the max scan: the tight fit puts the largest mantissa in
@@ -484,12 +524,13 @@ constexpr size_t kSharedBytes = (size_t)kStages * kStageBytes + sizeof(BlockShar
 
 // Publish a consumer warp's scans of tensor t and clear them.
 __device__ __forceinline__ void flush_scans(const StepParams& p, int t, WarpSlots* slots, int lane,
-                                            unsigned int& amax_t, unsigned int& amax_c) {
+                                            float& amax_t, float& amax_c) {
   const unsigned int full = 0xffffffffu;
-  unsigned int at = __reduce_max_sync(full, amax_t);
-  unsigned int ac = __reduce_max_sync(full, amax_c);
-  amax_t = 0u;
-  amax_c = 0u;
+  // the steady path's scans are exact integers below 2^23 held in floats
+  unsigned int at = __reduce_max_sync(full, (unsigned int)amax_t);
+  unsigned int ac = __reduce_max_sync(full, (unsigned int)amax_c);
+  amax_t = 0.0f;
+  amax_c = 0.0f;
   if (lane == 0 && t >= 0) {
     at = max(at, slots->amax_t);
     ac = max(ac, slots->amax_c);
@@ -506,16 +547,10 @@ __device__ __forceinline__ void flush_scans(const StepParams& p, int t, WarpSlot
 
 __global__ void __launch_bounds__(kBlockThreads, 1)
 ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ InlineArgs a) {
-  extern __shared__ unsigned char smem_raw[];
-  unsigned char* base = reinterpret_cast<unsigned char*>(
-      (reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
-  BlockShared* sh = reinterpret_cast<BlockShared*>(base + (size_t)kStages * kStageBytes);
+  extern __shared__ __align__(128) unsigned char smem[];
+  BlockShared* sh = reinterpret_cast<BlockShared*>(smem + (size_t)kStages * kStageBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // this block's contiguous run of tiles
-  const long long g = gridDim.x, b = blockIdx.x;
-  const int tile0 = (int)(b * p.n_chunks / g);
-  const int n_my = (int)((b + 1) * p.n_chunks / g) - tile0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -533,20 +568,34 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------ producer
+    // Tiles are handed out dynamically: block b starts with tile b, every later tile
+    // comes from a global counter, so blocks that meet slow tiles (exponent changes,
+    // saturation) simply take fewer of them.
     if (lane == 0) {
       int cur = -1;
       TensorInfo ti{};
       StepCoef coef{};
       const float* grad = nullptr;
       int issued = 0;
-      for (int i = 0; i < n_my; ++i) {
+      int tile = (int)blockIdx.x;
+      for (int i = 0;; ++i) {
         const int stage = i % kStages, use = i / kStages;
+        // ask for the tile after this one now; the answer is needed one iteration later
+        const unsigned int after = atomicAdd(p.ws.next_tile, 1u);
         if (use > 0 && !mbar_wait(&sh->empty[stage], (unsigned)(use - 1) & 1u, &sh->abort_flag)) {
           sh->abort_flag = 1;
           atomicCAS(p.ws.error, 0u, (unsigned)kErrEmptyWait);
           break;
         }
-        const ChunkRef cr = p.ws.chunks[tile0 + i];
+        TileDesc& td = sh->desc[stage];
+        if (tile >= p.n_chunks) {
+          td.flags = kFlagStop;
+          td.tensor = -1;
+          mbar_arrive(&sh->full[stage]);
+          issued = i + 1;
+          break;
+        }
+        const ChunkRef cr = p.ws.chunks[tile];
         if (cr.tensor != cur) {
           cur = cr.tensor;
           ti = p.ws.info[cur];
@@ -560,17 +609,19 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
         const int count = left < (long long)kChunk ? (int)left : kChunk;
         const int n_bulk = count & ~15;
         const int tbytes = ti.theta_bits >> 3, cbytes = ti.comp_bits >> 3;
-        TileDesc& td = sh->desc[stage];
-        td.coef = coef;
+        td.scale = coef.scale;
+        td.pow2s_neg = -pow2_float(coef.s);
+        td.inv2s = pow2_float(-coef.s);
+        td.qmax_t = (float)coef.qmax_t;
         td.theta = static_cast<unsigned char*>(ti.theta) + first * tbytes;
         td.comp = ti.comp ? static_cast<unsigned char*>(ti.comp) + first * cbytes : nullptr;
-        td.grad = grad + first;
         td.tensor = cur;
-        td.count = count;
         td.n_bulk = n_bulk;
-        td.theta_bits = ti.theta_bits;
-        td.comp_bits = ti.comp_bits;
-        unsigned char* st = base + (size_t)stage * kStageBytes;
+        td.count = count;
+        td.flags = ((ti.theta_bits == 16 ? 3 : 0) + (ti.comp_bits >> 3)) | (coef.delta == 0 ? kFlagSteady : 0);
+        td.coef = coef;
+        td.grad = grad + first;
+        unsigned char* st = smem + (size_t)stage * kStageBytes;
         if (n_bulk > 0) {
           mbar_arrive_expect_tx(&sh->full[stage], (unsigned)(n_bulk * (tbytes + cbytes + 4)));
           bulk_load(st + kStageThetaOff, td.theta, (unsigned)(n_bulk * tbytes), &sh->full[stage]);
@@ -580,6 +631,7 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
           mbar_arrive(&sh->full[stage]);
         }
         issued = i + 1;
+        tile = (int)after;
       }
       // Before the block may exit, every copy it started must have landed (normally the
       // consumers have long since seen them; this only matters after a give-up).
@@ -590,9 +642,9 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
     // ------------------------------------------------------------------ consumers
     const int ctid = threadIdx.x;
     WarpSlots* slots = &sh->slots[warp];
-    unsigned int amax_t = 0u, amax_c = 0u;
+    float amax_t = 0.0f, amax_c = 0.0f;
     int cur = -1;
-    for (int i = 0; i < n_my; ++i) {
+    for (int i = 0;; ++i) {
       const int stage = i % kStages, use = i / kStages;
       if (!mbar_wait(&sh->full[stage], (unsigned)use & 1u, &sh->abort_flag)) {
         if (lane == 0) {
@@ -602,22 +654,38 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
         break;
       }
       const TileDesc* td = &sh->desc[stage];
-      const int t = td->tensor;
-      if (t != cur) {
+      TileHot h;
+      {
+        const uint4* q = reinterpret_cast<const uint4*>(td);
+        const uint4 q0 = q[0], q1 = q[1], q2 = q[2];
+        h.k.scale = __uint_as_float(q0.x);
+        h.k.pow2s_neg = __uint_as_float(q0.y);
+        h.k.inv2s = __uint_as_float(q0.z);
+        h.k.qmax_t = __uint_as_float(q0.w);
+        h.theta = reinterpret_cast<unsigned char*>(((unsigned long long)q1.y << 32) | q1.x);
+        h.comp = reinterpret_cast<unsigned char*>(((unsigned long long)q1.w << 32) | q1.z);
+        h.tensor = (int)q2.x;
+        h.n_bulk = (int)q2.y;
+        h.count = (int)q2.z;
+        h.flags = (int)q2.w;
+      }
+      if (h.flags & kFlagStop) break;
+      if (h.tensor != cur) {
         flush_scans(p, cur, slots, lane, amax_t, amax_c);
-        cur = t;
+        cur = h.tensor;
       }
-      const unsigned char* st = base + (size_t)stage * kStageBytes;
-      const int tb = td->theta_bits, cb = td->comp_bits;
-      if (tb == 8) {
-        if (cb == 8) consume_tile<8, 8>(td, st, ctid, slots, amax_t, amax_c);
-        else if (cb == 16) consume_tile<8, 16>(td, st, ctid, slots, amax_t, amax_c);
-        else consume_tile<8, 0>(td, st, ctid, slots, amax_t, amax_c);
-      } else {
-        if (cb == 8) consume_tile<16, 8>(td, st, ctid, slots, amax_t, amax_c);
-        else if (cb == 16) consume_tile<16, 16>(td, st, ctid, slots, amax_t, amax_c);
-        else consume_tile<16, 0>(td, st, ctid, slots, amax_t, amax_c);
+      unsigned char* st = smem + (size_t)stage * kStageBytes;
+      switch (h.flags & kFlagFormatMask) {
+        case 0: consume_tile<8, 0>(h, td, st, ctid, slots, amax_t, amax_c); break;
+        case 1: consume_tile<8, 8>(h, td, st, ctid, slots, amax_t, amax_c); break;
+        case 2: consume_tile<8, 16>(h, td, st, ctid, slots, amax_t, amax_c); break;
+        case 3: consume_tile<16, 0>(h, td, st, ctid, slots, amax_t, amax_c); break;
+        case 4: consume_tile<16, 8>(h, td, st, ctid, slots, amax_t, amax_c); break;
+        default: consume_tile<16, 16>(h, td, st, ctid, slots, amax_t, amax_c); break;
       }
+      // the general path may have written into the stage: order those writes before the
+      // bulk copy that refills it
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->empty[stage]);
     }
@@ -648,7 +716,10 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
     p.ws.amax_acc[i] = 0u;
     p.ws.amax_acc[p.n_tensors + i] = 0u;
   }
-  if (threadIdx.x == 0) *p.ws.ticket = 0u;
+  if (threadIdx.x == 0) {
+    *p.ws.ticket = 0u;
+    *p.ws.next_tile = gridDim.x;
+  }
 }
 
 // Per-step arguments of long lists: written to the workspace from kernel parameters.

@@ -174,9 +174,10 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
   h->params.inline_args = n_tensors <= kInlineArgs ? 1 : 0;
 
   // Persistent grid: one block per SM (fewer if the list has fewer tiles).
-  int dev = 0, sms = 0;
+  int dev = 0, sms = 0, l2_bytes = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, dev);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(ksgd_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)kSharedBytes);
@@ -185,6 +186,13 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
     return cuda_fail(e, "device query");
   }
   h->grid = (int)(L.n_chunks < (long long)sms ? L.n_chunks : (long long)sms);
+  // theta and c of the whole list against the L2 size: if the state fits (with room for
+  // the gradients streaming through), gradient loads are marked evict-first
+  double state_bytes = 0.0;
+  for (int32_t i = 0; i < n_tensors; ++i)
+    state_bytes += (double)descs[i].numel * ((descs[i].theta_bits + descs[i].comp_bits) / 8);
+  h->params.grad_evict_first = state_bytes <= 0.8 * (double)l2_bytes ? 1 : 0;
+  h->params.pad = 0;
   reinterpret_cast<unsigned int*>(img.data() + L.ticket)[1] = (unsigned int)h->grid;
 
   e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);

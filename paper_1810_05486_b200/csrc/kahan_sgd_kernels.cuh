@@ -81,6 +81,8 @@ struct StepParams {
   int n_chunks;
   int amax_mode;     // 1: exponents follow the max scan, 0: fixed
   int inline_args;   // 1: grads/lrs are in the InlineArgs parameter
+  int grad_evict_first;  // 1: gradient loads carry the L2 evict-first hint
+  int pad;
 };
 
 struct InlineArgs {
@@ -199,6 +201,22 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, 
           smem_addr(dst_smem)),
       "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar))
       : "memory");
+}
+
+// Same, with an L2 eviction-priority hint for data that is read once per step.
+__device__ __forceinline__ void bulk_load_hint(void* dst_smem, const void* src_gmem, unsigned int bytes,
+                                               unsigned long long* bar, unsigned long long policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+          smem_addr(dst_smem)),
+      "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar)), "l"(policy)
+      : "memory");
+}
+
+__device__ __forceinline__ unsigned long long l2_policy_evict_first() {
+  unsigned long long pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
 }
 
 // ----------------------------------------------------------------------------------------
@@ -578,6 +596,7 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
       const float* grad = nullptr;
       int issued = 0;
       int tile = (int)blockIdx.x;
+      const unsigned long long grad_policy = l2_policy_evict_first();
       for (int i = 0;; ++i) {
         const int stage = i % kStages, use = i / kStages;
         // ask for the tile after this one now; the answer is needed one iteration later
@@ -626,7 +645,12 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
           mbar_arrive_expect_tx(&sh->full[stage], (unsigned)(n_bulk * (tbytes + cbytes + 4)));
           bulk_load(st + kStageThetaOff, td.theta, (unsigned)(n_bulk * tbytes), &sh->full[stage]);
           if (cbytes) bulk_load(st + kStageCompOff, td.comp, (unsigned)(n_bulk * cbytes), &sh->full[stage]);
-          bulk_load(st + kStageGradOff, td.grad, (unsigned)(n_bulk * 4), &sh->full[stage]);
+          // Gradients are read once.  When theta and c of the whole list fit in L2, letting
+          // the gradients leave it first keeps the state resident from step to step.
+          if (p.grad_evict_first)
+            bulk_load_hint(st + kStageGradOff, td.grad, (unsigned)(n_bulk * 4), &sh->full[stage], grad_policy);
+          else
+            bulk_load(st + kStageGradOff, td.grad, (unsigned)(n_bulk * 4), &sh->full[stage]);
         } else {
           mbar_arrive(&sh->full[stage]);
         }

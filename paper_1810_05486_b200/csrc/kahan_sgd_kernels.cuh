@@ -474,19 +474,21 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
   return true;
 }
 
-// All vectors of one tile that belong to this consumer thread.
+// All vectors of one tile that belong to this consumer thread (V consecutive elements,
+// 16 bytes of theta, per vector).  Returns true if the general path wrote into the stage.
 template <int TB, int CB>
-__device__ __forceinline__ void consume_tile(const TileHot& h, const TileDesc* td, unsigned char* stage,
+__device__ __forceinline__ bool consume_tile(const TileHot& h, const TileDesc* td, unsigned char* stage,
                                              int ctid, WarpSlots* slots, float& amax_t, float& amax_c) {
   constexpr bool HAS_COMP = CB != 0;
-  constexpr int V = (TB == 8) ? 16 : 8;              // 16 bytes of theta per vector
+  constexpr int V = (TB == 8) ? 16 : 8;
   constexpr int TBYTES = V * TB / 8;
   constexpr int CBYTES = HAS_COMP ? V * CB / 8 : 8;
   const bool steady = (h.flags & kFlagSteady) != 0;
-  const int n_vec = h.n_bulk / V;
   unsigned char* theta_s = stage + kStageThetaOff;
   unsigned char* comp_s = stage + kStageCompOff;
   const float* grad_s = reinterpret_cast<const float*>(stage + kStageGradOff);
+  bool wrote_stage = false;
+  const int n_vec = h.n_bulk / V;
   for (int v = ctid; v < n_vec; v += kConsumers) {
     Pack<TBYTES> ot;
     Pack<CBYTES> oc;
@@ -503,6 +505,7 @@ __device__ __forceinline__ void consume_tile(const TileHot& h, const TileDesc* t
       update_general(&td->coef, TB, CB, theta_s, comp_s, grad_s, v * V, V, slots);
       ot = load_pack<TBYTES>(theta_s + v * TBYTES);
       if constexpr (HAS_COMP) oc = load_pack<CBYTES>(comp_s + v * CBYTES);
+      wrote_stage = true;
     }
     store_pack<TBYTES>(h.theta + (size_t)v * TBYTES, ot);
     if constexpr (HAS_COMP) store_pack<CBYTES>(h.comp + (size_t)v * CBYTES, oc);
@@ -511,6 +514,7 @@ __device__ __forceinline__ void consume_tile(const TileHot& h, const TileDesc* t
   // global memory
   const int e = h.n_bulk + ctid;
   if (e < h.count) update_general(&td->coef, TB, CB, h.theta, h.comp, td->grad, e, 1, slots);
+  return wrote_stage;
 }
 
 // Next exponent from the max scan: the tight fit puts the largest mantissa in
@@ -596,11 +600,15 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
       const float* grad = nullptr;
       int issued = 0;
       int tile = (int)blockIdx.x;
+      ChunkRef cr = p.ws.chunks[tile];
       const unsigned long long grad_policy = l2_policy_evict_first();
       for (int i = 0;; ++i) {
         const int stage = i % kStages, use = i / kStages;
-        // ask for the tile after this one now; the answer is needed one iteration later
+        // fetch the tile after this one (number and table entry) now, while the consumers
+        // are still busy with the stage this tile will go to
         const unsigned int after = atomicAdd(p.ws.next_tile, 1u);
+        ChunkRef cr_after{-1, -1};
+        if (after < (unsigned)p.n_chunks) cr_after = p.ws.chunks[after];
         if (use > 0 && !mbar_wait(&sh->empty[stage], (unsigned)(use - 1) & 1u, &sh->abort_flag)) {
           sh->abort_flag = 1;
           atomicCAS(p.ws.error, 0u, (unsigned)kErrEmptyWait);
@@ -614,7 +622,6 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
           issued = i + 1;
           break;
         }
-        const ChunkRef cr = p.ws.chunks[tile];
         if (cr.tensor != cur) {
           cur = cr.tensor;
           ti = p.ws.info[cur];
@@ -656,6 +663,7 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
         }
         issued = i + 1;
         tile = (int)after;
+        cr = cr_after;
       }
       // Before the block may exit, every copy it started must have landed (normally the
       // consumers have long since seen them; this only matters after a give-up).
@@ -699,17 +707,18 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
         cur = h.tensor;
       }
       unsigned char* st = smem + (size_t)stage * kStageBytes;
+      bool wrote_stage;
       switch (h.flags & kFlagFormatMask) {
-        case 0: consume_tile<8, 0>(h, td, st, ctid, slots, amax_t, amax_c); break;
-        case 1: consume_tile<8, 8>(h, td, st, ctid, slots, amax_t, amax_c); break;
-        case 2: consume_tile<8, 16>(h, td, st, ctid, slots, amax_t, amax_c); break;
-        case 3: consume_tile<16, 0>(h, td, st, ctid, slots, amax_t, amax_c); break;
-        case 4: consume_tile<16, 8>(h, td, st, ctid, slots, amax_t, amax_c); break;
-        default: consume_tile<16, 16>(h, td, st, ctid, slots, amax_t, amax_c); break;
+        case 0: wrote_stage = consume_tile<8, 0>(h, td, st, ctid, slots, amax_t, amax_c); break;
+        case 1: wrote_stage = consume_tile<8, 8>(h, td, st, ctid, slots, amax_t, amax_c); break;
+        case 2: wrote_stage = consume_tile<8, 16>(h, td, st, ctid, slots, amax_t, amax_c); break;
+        case 3: wrote_stage = consume_tile<16, 0>(h, td, st, ctid, slots, amax_t, amax_c); break;
+        case 4: wrote_stage = consume_tile<16, 8>(h, td, st, ctid, slots, amax_t, amax_c); break;
+        default: wrote_stage = consume_tile<16, 16>(h, td, st, ctid, slots, amax_t, amax_c); break;
       }
-      // the general path may have written into the stage: order those writes before the
-      // bulk copy that refills it
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      // if the general path wrote into the stage, order those writes before the bulk copy
+      // that refills it
+      if (wrote_stage) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->empty[stage]);
     }

@@ -141,6 +141,48 @@ int kahan_sgd_amax(ksgd_handle* h, uint32_t* amax_theta, uint32_t* amax_comp,
  */
 int kahan_sgd_set_exponents(ksgd_handle* h, const int32_t* exp_theta_next);
 
+/*
+ * One step for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this entry point exists for the sake of the calling environment, not of the method.)
+ *
+ * kahan_sgd_init needs a device workspace from its caller, and some callers have no way to
+ * get one at the moment they need it: a plug-in running inside a host program that has
+ * already handed all device memory to its own pool and forbids further cudaMalloc calls;
+ * a latency-critical loop where cudaMalloc's device-wide synchronisation is unacceptable;
+ * code that runs while another thread is recording a stream capture in a mode that makes
+ * allocation calls illegal.  For them the same scratch (exponents, max-scan slots,
+ * counters, tile table) lives in a fixed array of KSGD_STATIC_SCRATCH_BYTES inside the
+ * library's device image, which every GPU that loads the library holds until the process
+ * exits.  The call allocates and frees no device memory, directly or through any library.
+ *
+ * The call is self-contained: it runs exactly one step of the whole list (same kernel,
+ * same arithmetic, same results bit for bit as kahan_sgd_init + kahan_sgd_step +
+ * kahan_sgd_amax on a fresh handle) and waits for it.  descs carries the state a caller
+ * keeps between steps: theta/comp device pointers (updated in place), formats, and the
+ * exponents exp_theta (of the stored mantissas) and exp_theta_next (to write); feed the
+ * returned exp_theta_cur / exp_theta_next back into the next call's descs.  grads, lrs:
+ * as for kahan_sgd_step.  Outputs (host arrays of n_tensors entries, NULL to skip): as for
+ * kahan_sgd_amax, except that the three counters count this call only.
+ *
+ * Limits: n_tensors <= KSGD_STATIC_MAX_TENSORS and the tile table must fit the array
+ * (sum over tensors of ceil(numel / 8192) tiles, 8 bytes each, plus about 100 bytes per
+ * tensor: roughly 1.9e8 parameters); beyond that the call returns KSGD_ERR_WORKSPACE and
+ * does nothing.
+ *
+ * The first call on each device looks up the array's device address and sets a kernel
+ * attribute; make that first call with the device current and before any stream capture
+ * begins.  All calls on a device share the one array and each call rewrites all of it, so
+ * two calls whose work overlaps on the GPU (different streams, different threads) race:
+ * callers serialise them.
+ */
+#define KSGD_STATIC_SCRATCH_BYTES (192 * 1024)
+#define KSGD_STATIC_MAX_TENSORS 256
+int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd_exp_mode mode,
+                          const float* const* grads, const float* lrs, uint32_t* amax_theta,
+                          uint32_t* amax_comp, int32_t* exp_theta_cur, int32_t* exp_theta_next,
+                          uint64_t* n_sat_theta, uint64_t* n_sat_comp, uint64_t* n_nonfinite,
+                          void* cuda_stream);
+
 /* Free the host-side handle (waits for the stream first).  Device buffers stay the caller's. */
 int kahan_sgd_destroy(ksgd_handle* h);
 

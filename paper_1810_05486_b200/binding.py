@@ -29,7 +29,8 @@ KSGD_ERR_DEVICE = -11
 
 EXPORTS = (
     "kahan_sgd_workspace_bytes", "kahan_sgd_init", "kahan_sgd_step", "kahan_sgd_step_host",
-    "kahan_sgd_amax", "kahan_sgd_set_exponents", "kahan_sgd_destroy", "kahan_sgd_strerror",
+    "kahan_sgd_amax", "kahan_sgd_set_exponents", "kahan_sgd_step_static", "kahan_sgd_destroy",
+    "kahan_sgd_strerror",
     "kahan_sgd_last_cuda_error", "kahan_sgd_launch_count",
 )
 
@@ -69,6 +70,10 @@ def _load() -> ctypes.CDLL:
     lib.kahan_sgd_amax.argtypes = [ctypes.c_void_p] + [ctypes.c_void_p] * 7
     lib.kahan_sgd_set_exponents.restype = ctypes.c_int
     lib.kahan_sgd_set_exponents.argtypes = [ctypes.c_void_p, P(ctypes.c_int32)]
+    lib.kahan_sgd_step_static.restype = ctypes.c_int
+    lib.kahan_sgd_step_static.argtypes = [P(ksgd_tensor_desc), ctypes.c_int32, ctypes.c_int,
+                                          P(ctypes.c_void_p), P(ctypes.c_float)] + \
+        [ctypes.c_void_p] * 7 + [ctypes.c_void_p]
     lib.kahan_sgd_destroy.restype = ctypes.c_int
     lib.kahan_sgd_destroy.argtypes = [ctypes.c_void_p]
     lib.kahan_sgd_strerror.restype = ctypes.c_char_p
@@ -165,6 +170,34 @@ def kahan_sgd_amax(h, n_tensors: int) -> dict:
 def kahan_sgd_set_exponents(h, exp_theta_next: Sequence[int]) -> None:
     arr = (ctypes.c_int32 * len(exp_theta_next))(*exp_theta_next)
     _check(lib.kahan_sgd_set_exponents(h, arr))
+
+
+KSGD_STATIC_SCRATCH_BYTES = 192 * 1024
+KSGD_STATIC_MAX_TENSORS = 256
+
+
+def kahan_sgd_step_static(descs, mode: int, grads, lrs, stream: int = 0) -> dict:
+    """One self-contained step that allocates no device memory (scratch inside the library).
+
+    For callers that cannot obtain a device workspace when they need one.  Returns the same
+    dictionary as kahan_sgd_amax (counters: this call only); put exp_theta_cur and
+    exp_theta_next back into the descs for the next call.  Calls must not overlap on the GPU.
+    """
+    n = len(descs)
+    g = grads if isinstance(grads, ctypes.Array) else _ptr_array(grads)
+    l = lrs if isinstance(lrs, ctypes.Array) else _float_array(lrs)
+    a_t = (ctypes.c_uint32 * n)()
+    a_c = (ctypes.c_uint32 * n)()
+    e_c = (ctypes.c_int32 * n)()
+    e_n = (ctypes.c_int32 * n)()
+    s_t = (ctypes.c_uint64 * n)()
+    s_c = (ctypes.c_uint64 * n)()
+    nf = (ctypes.c_uint64 * n)()
+    _check(lib.kahan_sgd_step_static(descs, n, mode, g, l, a_t, a_c, e_c, e_n, s_t, s_c, nf,
+                                     ctypes.c_void_p(stream)))
+    return {"amax_theta": list(a_t), "amax_comp": list(a_c), "exp_theta_cur": list(e_c),
+            "exp_theta_next": list(e_n), "n_sat_theta": list(s_t), "n_sat_comp": list(s_c),
+            "n_nonfinite": list(nf)}
 
 
 def kahan_sgd_destroy(h) -> None:

@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <type_traits>
 #include <vector>
@@ -370,6 +371,140 @@ int kahan_sgd_destroy(ksgd_handle* h) {
   const cudaError_t e = cudaStreamSynchronize(h->stream);
   delete h;
   if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  return KSGD_OK;
+}
+
+// ----------------------------------------------------------------------------------------
+// One step without any device allocation by anybody: the scratch that kahan_sgd_init
+// otherwise lays out in a caller-provided workspace lives in a fixed array inside this
+// library's device image.
+
+static __device__ __align__(256) unsigned char g_static_scratch[KSGD_STATIC_SCRATCH_BYTES];
+
+namespace {
+struct StaticDevice {
+  bool ready = false;
+  unsigned char* scratch = nullptr;   // device address of g_static_scratch on this device
+  int sms = 0;
+  int l2_bytes = 0;
+};
+constexpr int kMaxDevices = 64;
+StaticDevice g_static_dev[kMaxDevices];
+std::mutex g_static_mutex;
+}  // namespace
+
+int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd_exp_mode mode,
+                          const float* const* grads, const float* lrs, uint32_t* amax_theta,
+                          uint32_t* amax_comp, int32_t* exp_theta_cur, int32_t* exp_theta_next,
+                          uint64_t* n_sat_theta, uint64_t* n_sat_comp, uint64_t* n_nonfinite,
+                          void* cuda_stream) {
+  const int v = validate(descs, n_tensors);
+  if (v != KSGD_OK) return v;
+  if (mode != KSGD_EXP_FIXED && mode != KSGD_EXP_AMAX) return KSGD_ERR_MODE;
+  if (!grads || !lrs) return KSGD_ERR_NULL;
+  if (n_tensors > KSGD_STATIC_MAX_TENSORS) return KSGD_ERR_WORKSPACE;
+  const Layout L = make_layout(descs, n_tensors);
+  if (L.total > (size_t)KSGD_STATIC_SCRATCH_BYTES) return KSGD_ERR_WORKSPACE;
+  for (int32_t i = 0; i < n_tensors; ++i) {
+    if (!grads[i]) return KSGD_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(grads[i]) % 16) return KSGD_ERR_ALIGN;
+    if (!std::isfinite(lrs[i]) || !(lrs[i] > 0.0f)) return KSGD_ERR_LR;
+  }
+
+  // Once per device, with that device current: the array's name is only a host-side
+  // stand-in here, the address a kernel can use has to be asked for.
+  int dev = 0;
+  KSGD_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return KSGD_ERR_WORKSPACE;
+  StaticDevice sd;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDevice& slot = g_static_dev[dev];
+    if (!slot.ready) {
+      void* ptr = nullptr;
+      KSGD_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+      KSGD_CUDA(cudaDeviceGetAttribute(&slot.sms, cudaDevAttrMultiProcessorCount, dev));
+      KSGD_CUDA(cudaDeviceGetAttribute(&slot.l2_bytes, cudaDevAttrL2CacheSize, dev));
+      KSGD_CUDA(cudaFuncSetAttribute(ksgd_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)kSharedBytes));
+      slot.scratch = static_cast<unsigned char*>(ptr);
+      slot.ready = true;
+    }
+    sd = slot;
+  }
+
+  // Host image of the scratch, every byte of it: whatever the previous call left in the
+  // array (scans, counters, ticket, tile counter) is overwritten.
+  std::vector<unsigned char> img(L.total, 0);
+  int* e_cur = reinterpret_cast<int*>(img.data() + L.exp_cur);
+  int* e_next = reinterpret_cast<int*>(img.data() + L.exp_next);
+  TensorInfo* info = reinterpret_cast<TensorInfo*>(img.data() + L.info);
+  ChunkRef* chunks = reinterpret_cast<ChunkRef*>(img.data() + L.chunks);
+  long long c = 0;
+  double state_bytes = 0.0;
+  for (int32_t i = 0; i < n_tensors; ++i) {
+    const ksgd_tensor_desc& t = descs[i];
+    e_cur[i] = t.exp_theta;
+    e_next[i] = t.exp_theta_next;
+    info[i].theta = t.theta;
+    info[i].comp = t.comp;
+    info[i].numel = t.numel;
+    info[i].theta_bits = t.theta_bits;
+    info[i].comp_bits = t.comp_bits;
+    info[i].s = t.comp_bits ? t.comp_bits - 1 - t.overlap_k : 0;
+    info[i].pad = 0;
+    const long long nc = (t.numel + kChunk - 1) / kChunk;
+    for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
+    state_bytes += (double)t.numel * ((t.theta_bits + t.comp_bits) / 8);
+  }
+  const int grid = (int)(L.n_chunks < (long long)sd.sms ? L.n_chunks : (long long)sd.sms);
+  reinterpret_cast<unsigned int*>(img.data() + L.ticket)[1] = (unsigned int)grid;
+
+  StepParams params;
+  unsigned char* b = sd.scratch;
+  params.ws.exp_cur = reinterpret_cast<int*>(b + L.exp_cur);
+  params.ws.exp_next = reinterpret_cast<int*>(b + L.exp_next);
+  params.ws.amax_last = reinterpret_cast<unsigned int*>(b + L.amax_last);
+  params.ws.counters = reinterpret_cast<unsigned long long*>(b + L.counters);
+  params.ws.error = reinterpret_cast<unsigned int*>(b + L.error);
+  params.ws.amax_acc = reinterpret_cast<unsigned int*>(b + L.amax_acc);
+  params.ws.info = reinterpret_cast<TensorInfo*>(b + L.info);
+  params.ws.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
+  params.ws.lr = reinterpret_cast<float*>(b + L.lr);
+  params.ws.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
+  params.ws.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
+  params.ws.next_tile = params.ws.ticket + 1;
+  params.n_tensors = n_tensors;
+  params.n_chunks = (int)L.n_chunks;
+  params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
+  params.inline_args = 1;
+  params.grad_evict_first = state_bytes <= 0.8 * (double)sd.l2_bytes ? 1 : 0;
+  params.pad = 0;
+
+  InlineArgs inl;
+  for (int32_t i = 0; i < n_tensors; ++i) { inl.grads[i] = grads[i]; inl.lrs[i] = lrs[i]; }
+  for (int32_t i = n_tensors; i < kInlineArgs; ++i) { inl.grads[i] = nullptr; inl.lrs[i] = 0.0f; }
+
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  KSGD_CUDA(cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, stream));
+  ksgd_step_kernel<<<(unsigned)grid, kBlockThreads, kSharedBytes, stream>>>(params, inl);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  KSGD_CUDA(cudaGetLastError());
+  KSGD_CUDA(cudaMemcpyAsync(img.data(), b, L.stats_end, cudaMemcpyDeviceToHost, stream));
+  KSGD_CUDA(cudaStreamSynchronize(stream));
+
+  const unsigned char* r = img.data();
+  const size_t n = (size_t)n_tensors;
+  if (exp_theta_cur) std::memcpy(exp_theta_cur, r + L.exp_cur, 4 * n);
+  if (exp_theta_next) std::memcpy(exp_theta_next, r + L.exp_next, 4 * n);
+  if (amax_theta) std::memcpy(amax_theta, r + L.amax_last, 4 * n);
+  if (amax_comp) std::memcpy(amax_comp, r + L.amax_last + 4 * n, 4 * n);
+  if (n_sat_theta) std::memcpy(n_sat_theta, r + L.counters, 8 * n);
+  if (n_sat_comp) std::memcpy(n_sat_comp, r + L.counters + 8 * n, 8 * n);
+  if (n_nonfinite) std::memcpy(n_nonfinite, r + L.counters + 16 * n, 8 * n);
+  unsigned int dev_err = 0;
+  std::memcpy(&dev_err, r + L.error, 4);
+  if (dev_err != 0) return KSGD_ERR_DEVICE;
   return KSGD_OK;
 }
 

@@ -137,6 +137,7 @@ def run_ours(args, rank, world, local_rank):
         entry.build()
     from paper_1810_05486_b200 import binding as B
     from paper_1810_05486_b200 import workloads as W
+    from paper_1810_05486_b200 import multi
     from paper_1810_05486_b200.runner import DeviceRun, HostInputs
 
     torch.cuda.set_device(local_rank)
@@ -149,7 +150,7 @@ def run_ours(args, rank, world, local_rank):
     n = len(wl.tensors)
     n_sets = GRAD_SETS.get(wl.name, 4)
     t0 = time.time()
-    host = HostInputs(wl, args.seed + 1000 * rank, n_sets, pinned=True)
+    host = HostInputs(wl, multi.rank_seed(args.seed, rank), n_sets, pinned=True)
     gen_s = time.time() - t0
     run = DeviceRun(host, B.KSGD_EXP_AMAX)
     stream = run.stream
@@ -184,12 +185,9 @@ def run_ours(args, rank, world, local_rank):
         clocks = sampler.stop(wall0, wall1) if rank == 0 else None
     stats = run.stats()
 
-    if dist is not None:
-        t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = multi.max_over_ranks(ms_total, dist, "cuda")
     ms_step = ms_total / args.steps
-    value = world * wl.numel / (ms_step * 1e-3)
+    value = multi.whole_job_throughput(wl.numel, world, ms_step * 1e-3)
 
     # ---- end to end through host buffers ------------------------------------------------
     e2e = None
@@ -202,12 +200,9 @@ def run_ours(args, rank, world, local_rank):
             run.step_host(th_h, c_h, g_h[(i + 1) % n_sets])
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        if dist is not None:
-            t = torch.tensor([dt], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = multi.max_over_ranks(dt, dist, "cuda")
         state_bytes = sum(t.numel * (t.theta_bits + t.comp_bits) // 8 for t in wl.tensors)
-        e2e = {"value": world * wl.numel * args.e2e_steps / dt, "unit": UNIT,
+        e2e = {"value": multi.whole_job_throughput(wl.numel * args.e2e_steps, world, dt), "unit": UNIT,
                "h2d_bytes_per_step": state_bytes + 4 * wl.numel,
                "d2h_bytes_per_step": state_bytes, "steps": args.e2e_steps,
                "ms_per_step": dt / args.e2e_steps * 1e3}

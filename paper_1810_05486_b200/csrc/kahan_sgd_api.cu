@@ -62,7 +62,7 @@ Layout make_layout(const ksgd_tensor_desc* d, int32_t n) {
   o = align_up(o, 16);
   L.chunks = o;    o += sizeof(ChunkRef) * (size_t)chunks;
   o = align_up(o, 16);
-  L.ticket = o;    o += 16;   // ticket, next_tile
+  L.ticket = o;    o += 16;
   L.total = align_up(o, 256);
   return L;
 }
@@ -168,7 +168,6 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
   w.lr = reinterpret_cast<float*>(b + L.lr);
   w.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
   w.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
-  w.next_tile = w.ticket + 1;
   h->params.n_tensors = n_tensors;
   h->params.n_chunks = (int)L.n_chunks;
   h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
@@ -194,7 +193,6 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
     state_bytes += (double)descs[i].numel * ((descs[i].theta_bits + descs[i].comp_bits) / 8);
   h->params.grad_evict_first = state_bytes <= 0.8 * (double)l2_bytes ? 1 : 0;
   h->params.pad = 0;
-  reinterpret_cast<unsigned int*>(img.data() + L.ticket)[1] = (unsigned int)h->grid;
 
   e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
@@ -458,7 +456,6 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
     state_bytes += (double)t.numel * ((t.theta_bits + t.comp_bits) / 8);
   }
   const int grid = (int)(L.n_chunks < (long long)sd.sms ? L.n_chunks : (long long)sd.sms);
-  reinterpret_cast<unsigned int*>(img.data() + L.ticket)[1] = (unsigned int)grid;
 
   StepParams params;
   unsigned char* b = sd.scratch;
@@ -473,7 +470,6 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   params.ws.lr = reinterpret_cast<float*>(b + L.lr);
   params.ws.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
   params.ws.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
-  params.ws.next_tile = params.ws.ticket + 1;
   params.n_tensors = n_tensors;
   params.n_chunks = (int)L.n_chunks;
   params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;

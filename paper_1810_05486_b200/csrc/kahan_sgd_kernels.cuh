@@ -72,7 +72,6 @@ struct Workspace {
   float* lr;                       // [n]
   ChunkRef* chunks;                // [n_chunks]
   unsigned int* ticket;            // blocks finished in the running step
-  unsigned int* next_tile;         // next tile not yet handed to a block (starts at gridDim.x)
 };
 
 struct StepParams {
@@ -131,10 +130,10 @@ struct __align__(16) TileDesc {
 };
 constexpr int kFlagFormatMask = 7;   // 0..5 = (8,0) (8,8) (8,16) (16,0) (16,8) (16,16)
 constexpr int kFlagSteady = 8;       // no exponent change: the exact-fp32 path applies
-constexpr int kFlagStop = 16;        // no more tiles for this block
 
-// Max scans and counters of the rare path, one set per consumer warp (shared memory).
-struct WarpSlots {
+// Max scans and counters of one tile, gathered in shared memory: the consumer warps add to
+// it, the producer publishes it when it takes the tile's stage back.
+struct TileScan {
   unsigned int amax_t, amax_c, n_sat_t, n_sat_c, n_nonfinite, pad[3];
 };
 
@@ -262,7 +261,7 @@ __device__ __forceinline__ StepCoef make_coef(const TensorInfo& ti, int e_in, in
 // costs the steady-state path no registers.
 __device__ __noinline__ void update_general(const StepCoef* coef, int tb, int cb, void* theta,
                                             void* comp, const float* grad, int first, int n,
-                                            WarpSlots* slots) {
+                                            TileScan* slots) {
   const StepCoef k = *coef;
   unsigned int amax_t = 0, amax_c = 0, n_sat_t = 0, n_sat_c = 0, n_nf = 0;
 #pragma unroll 1
@@ -478,7 +477,7 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
 // 16 bytes of theta, per vector).  Returns true if the general path wrote into the stage.
 template <int TB, int CB>
 __device__ __forceinline__ bool consume_tile(const TileHot& h, const TileDesc* td, unsigned char* stage,
-                                             int ctid, WarpSlots* slots, float& amax_t, float& amax_c) {
+                                             int ctid, TileScan* slots, float& amax_t, float& amax_c) {
   constexpr bool HAS_COMP = CB != 0;
   constexpr int V = (TB == 8) ? 16 : 8;
   constexpr int TBYTES = V * TB / 8;
@@ -536,7 +535,7 @@ struct __align__(128) BlockShared {
   unsigned long long full[kStages];    // producer -> consumers: the tile's bytes have landed
   unsigned long long empty[kStages];   // consumers -> producer: the stage may be refilled
   TileDesc desc[kStages];
-  WarpSlots slots[kConsumerWarps];
+  TileScan scan[kStages];
   int abort_flag;   // set by the first thread whose bounded wait ran out
   int is_last;
   int never;        // stays 0: abort flag for waits that must not be cut short
@@ -544,27 +543,68 @@ struct __align__(128) BlockShared {
 
 constexpr size_t kSharedBytes = (size_t)kStages * kStageBytes + sizeof(BlockShared) + 128;
 
-// Publish a consumer warp's scans of tensor t and clear them.
-__device__ __forceinline__ void flush_scans(const StepParams& p, int t, WarpSlots* slots, int lane,
-                                            float& amax_t, float& amax_c) {
+// Add a consumer warp's steady-path scans of the tile it just finished to the tile's slot.
+__device__ __forceinline__ void add_warp_scans(TileScan* scan, int lane, float& amax_t, float& amax_c) {
   const unsigned int full = 0xffffffffu;
   // the steady path's scans are exact integers below 2^23 held in floats
-  unsigned int at = __reduce_max_sync(full, (unsigned int)amax_t);
-  unsigned int ac = __reduce_max_sync(full, (unsigned int)amax_c);
+  const unsigned int at = __reduce_max_sync(full, (unsigned int)amax_t);
+  const unsigned int ac = __reduce_max_sync(full, (unsigned int)amax_c);
   amax_t = 0.0f;
   amax_c = 0.0f;
-  if (lane == 0 && t >= 0) {
-    at = max(at, slots->amax_t);
-    ac = max(ac, slots->amax_c);
-    if (at) atomicMax(&p.ws.amax_acc[t], at);
-    if (ac) atomicMax(&p.ws.amax_acc[p.n_tensors + t], ac);
-    if (slots->n_sat_t) atomicAdd(&p.ws.counters[t], (unsigned long long)slots->n_sat_t);
-    if (slots->n_sat_c) atomicAdd(&p.ws.counters[p.n_tensors + t], (unsigned long long)slots->n_sat_c);
-    if (slots->n_nonfinite)
-      atomicAdd(&p.ws.counters[2 * p.n_tensors + t], (unsigned long long)slots->n_nonfinite);
-    slots->amax_t = slots->amax_c = slots->n_sat_t = slots->n_sat_c = slots->n_nonfinite = 0u;
+  if (lane == 0) {
+    if (at) atomicMax(&scan->amax_t, at);
+    if (ac) atomicMax(&scan->amax_c, ac);
   }
-  __syncwarp();
+}
+
+// Producer side: scans of finished tiles are merged per tensor in registers and go to
+// global memory when the tensor changes (one set of atomics per block and tensor run).
+struct ScanAcc {
+  int tensor = -1;
+  unsigned int amax_t = 0, amax_c = 0, n_sat_t = 0, n_sat_c = 0, n_nonfinite = 0;
+};
+
+__device__ __forceinline__ void publish(const StepParams& p, ScanAcc& acc) {
+  if (acc.tensor >= 0) {
+    const int t = acc.tensor, n = p.n_tensors;
+    if (acc.amax_t) atomicMax(&p.ws.amax_acc[t], acc.amax_t);
+    if (acc.amax_c) atomicMax(&p.ws.amax_acc[n + t], acc.amax_c);
+    if (acc.n_sat_t) atomicAdd(&p.ws.counters[t], (unsigned long long)acc.n_sat_t);
+    if (acc.n_sat_c) atomicAdd(&p.ws.counters[n + t], (unsigned long long)acc.n_sat_c);
+    if (acc.n_nonfinite) atomicAdd(&p.ws.counters[2 * n + t], (unsigned long long)acc.n_nonfinite);
+  }
+  acc = ScanAcc{};
+}
+
+__device__ __forceinline__ void take_back(const StepParams& p, ScanAcc& acc, TileScan* scan, int tensor) {
+  if (tensor != acc.tensor) {
+    publish(p, acc);
+    acc.tensor = tensor;
+  }
+  acc.amax_t = max(acc.amax_t, scan->amax_t);
+  acc.amax_c = max(acc.amax_c, scan->amax_c);
+  acc.n_sat_t += scan->n_sat_t;
+  acc.n_sat_c += scan->n_sat_c;
+  acc.n_nonfinite += scan->n_nonfinite;
+  scan->amax_t = scan->amax_c = scan->n_sat_t = scan->n_sat_c = scan->n_nonfinite = 0u;
+}
+
+// What the producer reads about a tile's tensor, fetched one tile ahead.
+struct TensorMeta {
+  TensorInfo ti;
+  const float* grad;
+  float lr;
+  int e_in, e_out;
+};
+
+__device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const InlineArgs& a, int t) {
+  TensorMeta m;
+  m.ti = p.ws.info[t];
+  m.e_in = p.ws.exp_cur[t];
+  m.e_out = p.ws.exp_next[t];
+  m.grad = p.inline_args ? a.grads[t] : p.ws.grad_ptr[t];
+  m.lr = p.inline_args ? a.lrs[t] : p.ws.lr[t];
+  return m;
 }
 
 __global__ void __launch_bounds__(kBlockThreads, 1)
@@ -584,69 +624,62 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
     sh->never = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (threadIdx.x < kConsumerWarps * (int)(sizeof(WarpSlots) / 4))
-    reinterpret_cast<unsigned int*>(sh->slots)[threadIdx.x] = 0u;
+  if (threadIdx.x < kStages * (int)(sizeof(TileScan) / 4))
+    reinterpret_cast<unsigned int*>(sh->scan)[threadIdx.x] = 0u;
   __syncthreads();
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------ producer
-    // Tiles are handed out dynamically: block b starts with tile b, every later tile
-    // comes from a global counter, so blocks that meet slow tiles (exponent changes,
-    // saturation) simply take fewer of them.
+    // Block b takes tiles b, b + gridDim.x, ...: neighbouring tiles run on neighbouring
+    // SMs at the same time, and the tiles of a tensor that needs the general path are
+    // spread evenly over all blocks.  Table entries are fetched two tiles ahead and the
+    // tensor's data one tile ahead, so none of these loads sits between a freed stage and
+    // the copy that refills it.
     if (lane == 0) {
-      int cur = -1;
-      TensorInfo ti{};
-      StepCoef coef{};
-      const float* grad = nullptr;
-      int issued = 0;
-      int tile = (int)blockIdx.x;
-      ChunkRef cr = p.ws.chunks[tile];
+      const int stride = (int)gridDim.x;
+      const int n_my = ((int)p.n_chunks - (int)blockIdx.x + stride - 1) / stride;
       const unsigned long long grad_policy = l2_policy_evict_first();
-      for (int i = 0;; ++i) {
+      ScanAcc acc;
+      ChunkRef cr = p.ws.chunks[blockIdx.x];
+      TensorMeta meta = load_meta(p, a, cr.tensor);
+      ChunkRef cr1{-1, -1};
+      if (n_my > 1) cr1 = p.ws.chunks[blockIdx.x + stride];
+      int issued = 0;
+      for (int i = 0; i < n_my; ++i) {
         const int stage = i % kStages, use = i / kStages;
-        // fetch the tile after this one (number and table entry) now, while the consumers
-        // are still busy with the stage this tile will go to
-        const unsigned int after = atomicAdd(p.ws.next_tile, 1u);
-        ChunkRef cr_after{-1, -1};
-        if (after < (unsigned)p.n_chunks) cr_after = p.ws.chunks[after];
-        if (use > 0 && !mbar_wait(&sh->empty[stage], (unsigned)(use - 1) & 1u, &sh->abort_flag)) {
-          sh->abort_flag = 1;
-          atomicCAS(p.ws.error, 0u, (unsigned)kErrEmptyWait);
-          break;
+        ChunkRef cr2{-1, -1};
+        if (i + 2 < n_my) cr2 = p.ws.chunks[blockIdx.x + (i + 2) * stride];
+        TensorMeta meta1 = meta;
+        if (i + 1 < n_my && cr1.tensor != cr.tensor) meta1 = load_meta(p, a, cr1.tensor);
+
+        if (use > 0) {
+          if (!mbar_wait(&sh->empty[stage], (unsigned)(use - 1) & 1u, &sh->abort_flag)) {
+            sh->abort_flag = 1;
+            atomicCAS(p.ws.error, 0u, (unsigned)kErrEmptyWait);
+            break;
+          }
+          take_back(p, acc, &sh->scan[stage], sh->desc[stage].tensor);
         }
-        TileDesc& td = sh->desc[stage];
-        if (tile >= p.n_chunks) {
-          td.flags = kFlagStop;
-          td.tensor = -1;
-          mbar_arrive(&sh->full[stage]);
-          issued = i + 1;
-          break;
-        }
-        if (cr.tensor != cur) {
-          cur = cr.tensor;
-          ti = p.ws.info[cur];
-          const int e_in = p.ws.exp_cur[cur], e_out = p.ws.exp_next[cur];
-          grad = p.inline_args ? a.grads[cur] : p.ws.grad_ptr[cur];
-          const float lr = p.inline_args ? a.lrs[cur] : p.ws.lr[cur];
-          coef = make_coef(ti, e_in, e_out, lr);
-        }
+        const TensorInfo& ti = meta.ti;
+        const StepCoef coef = make_coef(ti, meta.e_in, meta.e_out, meta.lr);
         const long long first = (long long)cr.index * kChunk;
         const long long left = ti.numel - first;
         const int count = left < (long long)kChunk ? (int)left : kChunk;
         const int n_bulk = count & ~15;
         const int tbytes = ti.theta_bits >> 3, cbytes = ti.comp_bits >> 3;
+        TileDesc& td = sh->desc[stage];
         td.scale = coef.scale;
         td.pow2s_neg = -pow2_float(coef.s);
         td.inv2s = pow2_float(-coef.s);
         td.qmax_t = (float)coef.qmax_t;
         td.theta = static_cast<unsigned char*>(ti.theta) + first * tbytes;
         td.comp = ti.comp ? static_cast<unsigned char*>(ti.comp) + first * cbytes : nullptr;
-        td.tensor = cur;
+        td.tensor = cr.tensor;
         td.n_bulk = n_bulk;
         td.count = count;
         td.flags = ((ti.theta_bits == 16 ? 3 : 0) + (ti.comp_bits >> 3)) | (coef.delta == 0 ? kFlagSteady : 0);
         td.coef = coef;
-        td.grad = grad + first;
+        td.grad = meta.grad + first;
         unsigned char* st = smem + (size_t)stage * kStageBytes;
         if (n_bulk > 0) {
           mbar_arrive_expect_tx(&sh->full[stage], (unsigned)(n_bulk * (tbytes + cbytes + 4)));
@@ -662,21 +695,29 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
           mbar_arrive(&sh->full[stage]);
         }
         issued = i + 1;
-        tile = (int)after;
-        cr = cr_after;
+        cr = cr1;
+        cr1 = cr2;
+        meta = meta1;
       }
-      // Before the block may exit, every copy it started must have landed (normally the
-      // consumers have long since seen them; this only matters after a give-up).
-      for (int i = max(0, issued - kStages); i < issued; ++i)
-        mbar_wait(&sh->full[i % kStages], (unsigned)(i / kStages) & 1u, &sh->never);
+      // Collect the scans of the last tiles (their stages are not reused) and publish.
+      // The same waits make sure that every copy this block started has landed before
+      // the block exits.
+      for (int i = max(0, issued - kStages); i < issued; ++i) {
+        const int stage = i % kStages;
+        if (mbar_wait(&sh->empty[stage], (unsigned)(i / kStages) & 1u, &sh->abort_flag))
+          take_back(p, acc, &sh->scan[stage], sh->desc[stage].tensor);
+        else
+          mbar_wait(&sh->full[stage], (unsigned)(i / kStages) & 1u, &sh->never);
+      }
+      publish(p, acc);
     }
   } else {
     // ------------------------------------------------------------------ consumers
     const int ctid = threadIdx.x;
-    WarpSlots* slots = &sh->slots[warp];
+    const int stride = (int)gridDim.x;
+    const int n_my = ((int)p.n_chunks - (int)blockIdx.x + stride - 1) / stride;
     float amax_t = 0.0f, amax_c = 0.0f;
-    int cur = -1;
-    for (int i = 0;; ++i) {
+    for (int i = 0; i < n_my; ++i) {
       const int stage = i % kStages, use = i / kStages;
       if (!mbar_wait(&sh->full[stage], (unsigned)use & 1u, &sh->abort_flag)) {
         if (lane == 0) {
@@ -686,6 +727,7 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
         break;
       }
       const TileDesc* td = &sh->desc[stage];
+      TileScan* scan = &sh->scan[stage];
       TileHot h;
       {
         const uint4* q = reinterpret_cast<const uint4*>(td);
@@ -701,28 +743,23 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
         h.count = (int)q2.z;
         h.flags = (int)q2.w;
       }
-      if (h.flags & kFlagStop) break;
-      if (h.tensor != cur) {
-        flush_scans(p, cur, slots, lane, amax_t, amax_c);
-        cur = h.tensor;
-      }
       unsigned char* st = smem + (size_t)stage * kStageBytes;
       bool wrote_stage;
       switch (h.flags & kFlagFormatMask) {
-        case 0: wrote_stage = consume_tile<8, 0>(h, td, st, ctid, slots, amax_t, amax_c); break;
-        case 1: wrote_stage = consume_tile<8, 8>(h, td, st, ctid, slots, amax_t, amax_c); break;
-        case 2: wrote_stage = consume_tile<8, 16>(h, td, st, ctid, slots, amax_t, amax_c); break;
-        case 3: wrote_stage = consume_tile<16, 0>(h, td, st, ctid, slots, amax_t, amax_c); break;
-        case 4: wrote_stage = consume_tile<16, 8>(h, td, st, ctid, slots, amax_t, amax_c); break;
-        default: wrote_stage = consume_tile<16, 16>(h, td, st, ctid, slots, amax_t, amax_c); break;
+        case 0: wrote_stage = consume_tile<8, 0>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 1: wrote_stage = consume_tile<8, 8>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 2: wrote_stage = consume_tile<8, 16>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 3: wrote_stage = consume_tile<16, 0>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 4: wrote_stage = consume_tile<16, 8>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        default: wrote_stage = consume_tile<16, 16>(h, td, st, ctid, scan, amax_t, amax_c); break;
       }
+      add_warp_scans(scan, lane, amax_t, amax_c);
       // if the general path wrote into the stage, order those writes before the bulk copy
       // that refills it
       if (wrote_stage) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->empty[stage]);
     }
-    flush_scans(p, cur, slots, lane, amax_t, amax_c);
   }
 
   // ---------------------------------------------------------------------- block done
@@ -749,10 +786,7 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
     p.ws.amax_acc[i] = 0u;
     p.ws.amax_acc[p.n_tensors + i] = 0u;
   }
-  if (threadIdx.x == 0) {
-    *p.ws.ticket = 0u;
-    *p.ws.next_tile = gridDim.x;
-  }
+  if (threadIdx.x == 0) *p.ws.ticket = 0u;
 }
 
 // Per-step arguments of long lists: written to the workspace from kernel parameters.

@@ -12,7 +12,7 @@
 // The pass is bound by HBM traffic: 2*m/8 + 2*n/8 + 4 bytes per parameter.
 //
 // Structure: a persistent grid, one block per SM.  The tensor list is cut into tiles of
-// kChunk elements; each block owns a contiguous run of tiles.  One producer thread
+// kChunk elements; block b takes tiles b, b + gridDim.x, ....  One producer thread
 // streams the tiles of theta, c and g into a ring of shared-memory stages with bulk
 // asynchronous copies (cp.async.bulk, completion counted on an mbarrier), so the bytes in
 // flight do not depend on registers or occupancy; sixteen consumer warps compute from

@@ -13,10 +13,12 @@
 //
 // Structure: a persistent grid, one block per SM.  The tensor list is cut into tiles of
 // kChunk elements; block b takes tiles b, b + gridDim.x, ....  One producer thread
-// streams the tiles of theta, c and g into a ring of shared-memory stages with bulk
+// streams the tiles of theta, c and g into a 224 KB shared-memory ring with bulk
 // asynchronous copies (cp.async.bulk, completion counted on an mbarrier), so the bytes in
-// flight do not depend on registers or occupancy; sixteen consumer warps compute from
-// shared memory and store theta' and c' straight to global memory with 16-byte stores.
+// flight do not depend on registers or occupancy; a tile takes only the pages its format
+// needs (6 for int8/int8, 8 for int16/int16), so three to four tiles are resident.
+// Sixteen consumer warps compute from shared memory and store theta' and c' straight to
+// global memory with 16-byte stores.
 // No block ever waits for another block; every wait inside a block is bounded.
 #pragma once
 
@@ -30,11 +32,9 @@ constexpr int kChunk = 8192;           // elements per tile
 constexpr int kConsumerWarps = 16;
 constexpr int kConsumers = kConsumerWarps * 32;
 constexpr int kBlockThreads = kConsumers + 32;   // + one producer warp
-constexpr int kStages = 3;
-constexpr int kStageBytes = kChunk * 8;          // theta <= 2 B, c <= 2 B, g 4 B per element
-constexpr int kStageThetaOff = 0;
-constexpr int kStageCompOff = kChunk * 2;
-constexpr int kStageGradOff = kChunk * 4;
+constexpr int kSlots = 6;              // tiles a block can have in its ring at once
+constexpr int kPageBytes = 8192;       // the ring is handed out in pages
+constexpr int kPages = 28;             // 224 KB of tile data per block
 constexpr int kInlineArgs = 256;     // lists up to this long pass grads/lrs as kernel parameters
 constexpr int kUploadBatch = 1024;   // tensors per launch of the argument-upload kernel
 constexpr int kDLimit = 1 << 30;     // clamp of the quantized increment, in compensation LSBs
@@ -130,6 +130,9 @@ struct __align__(16) TileDesc {
 };
 constexpr int kFlagFormatMask = 7;   // 0..5 = (8,0) (8,8) (8,16) (16,0) (16,8) (16,16)
 constexpr int kFlagSteady = 8;       // no exponent change: the exact-fp32 path applies
+constexpr int kFlagThetaPageShift = 8;   // 5 bits each: first ring page of theta, c, g
+constexpr int kFlagCompPageShift = 13;
+constexpr int kFlagGradPageShift = 18;
 
 // Max scans and counters of one tile, gathered in shared memory: the consumer warps add to
 // it, the producer publishes it when it takes the tile's stage back.
@@ -476,16 +479,17 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
 // All vectors of one tile that belong to this consumer thread (V consecutive elements,
 // 16 bytes of theta, per vector).  Returns true if the general path wrote into the stage.
 template <int TB, int CB>
-__device__ __forceinline__ bool consume_tile(const TileHot& h, const TileDesc* td, unsigned char* stage,
+__device__ __forceinline__ bool consume_tile(const TileHot& h, const TileDesc* td, unsigned char* ring,
                                              int ctid, TileScan* slots, float& amax_t, float& amax_c) {
   constexpr bool HAS_COMP = CB != 0;
   constexpr int V = (TB == 8) ? 16 : 8;
   constexpr int TBYTES = V * TB / 8;
   constexpr int CBYTES = HAS_COMP ? V * CB / 8 : 8;
   const bool steady = (h.flags & kFlagSteady) != 0;
-  unsigned char* theta_s = stage + kStageThetaOff;
-  unsigned char* comp_s = stage + kStageCompOff;
-  const float* grad_s = reinterpret_cast<const float*>(stage + kStageGradOff);
+  unsigned char* theta_s = ring + ((h.flags >> kFlagThetaPageShift) & 31) * kPageBytes;
+  unsigned char* comp_s = ring + ((h.flags >> kFlagCompPageShift) & 31) * kPageBytes;
+  const float* grad_s =
+      reinterpret_cast<const float*>(ring + ((h.flags >> kFlagGradPageShift) & 31) * kPageBytes);
   bool wrote_stage = false;
   const int n_vec = h.n_bulk / V;
   for (int v = ctid; v < n_vec; v += kConsumers) {
@@ -532,16 +536,17 @@ __device__ __forceinline__ int next_exponent(unsigned int amax, int bits, int e_
 }
 
 struct __align__(128) BlockShared {
-  unsigned long long full[kStages];    // producer -> consumers: the tile's bytes have landed
-  unsigned long long empty[kStages];   // consumers -> producer: the stage may be refilled
-  TileDesc desc[kStages];
-  TileScan scan[kStages];
+  unsigned long long full[kSlots];     // producer -> consumers: the tile's bytes have landed
+  unsigned long long empty[kSlots];    // consumers -> producer: the tile's pages may be reused
+  TileDesc desc[kSlots];
+  TileScan scan[kSlots];
+  int slot_pages[kSlots];              // ring pages held by the tile in each slot
   int abort_flag;   // set by the first thread whose bounded wait ran out
   int is_last;
   int never;        // stays 0: abort flag for waits that must not be cut short
 };
 
-constexpr size_t kSharedBytes = (size_t)kStages * kStageBytes + sizeof(BlockShared) + 128;
+constexpr size_t kSharedBytes = (size_t)kPages * kPageBytes + sizeof(BlockShared);
 
 // Add a consumer warp's steady-path scans of the tile it just finished to the tile's slot.
 __device__ __forceinline__ void add_warp_scans(TileScan* scan, int lane, float& amax_t, float& amax_c) {
@@ -610,12 +615,12 @@ __device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const Inlin
 __global__ void __launch_bounds__(kBlockThreads, 1)
 ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ InlineArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
-  BlockShared* sh = reinterpret_cast<BlockShared*>(smem + (size_t)kStages * kStageBytes);
+  BlockShared* sh = reinterpret_cast<BlockShared*>(smem + (size_t)kPages * kPageBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < kSlots; ++s) {
       mbar_init(&sh->full[s], 1u);
       mbar_init(&sh->empty[s], (unsigned)kConsumerWarps);
     }
@@ -624,7 +629,7 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
     sh->never = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (threadIdx.x < kStages * (int)(sizeof(TileScan) / 4))
+  if (threadIdx.x < kSlots * (int)(sizeof(TileScan) / 4))
     reinterpret_cast<unsigned int*>(sh->scan)[threadIdx.x] = 0u;
   __syncthreads();
 
@@ -645,29 +650,58 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
       ChunkRef cr1{-1, -1};
       if (n_my > 1) cr1 = p.ws.chunks[blockIdx.x + stride];
       int issued = 0;
+      // The ring: pages from `head` on are free, tiles are released in the order they were
+      // issued, `oldest` is the first tile whose pages have not been taken back yet.
+      int head = 0, free_pages = kPages, oldest = 0;
+      bool gave_up = false;
       for (int i = 0; i < n_my; ++i) {
-        const int stage = i % kStages, use = i / kStages;
+        const int slot = i % kSlots;
         ChunkRef cr2{-1, -1};
         if (i + 2 < n_my) cr2 = p.ws.chunks[blockIdx.x + (i + 2) * stride];
         TensorMeta meta1 = meta;
         if (i + 1 < n_my && cr1.tensor != cr.tensor) meta1 = load_meta(p, a, cr1.tensor);
 
-        if (use > 0) {
-          if (!mbar_wait(&sh->empty[stage], (unsigned)(use - 1) & 1u, &sh->abort_flag)) {
-            sh->abort_flag = 1;
-            atomicCAS(p.ws.error, 0u, (unsigned)kErrEmptyWait);
+        const TensorInfo& ti = meta.ti;
+        const int tbytes = ti.theta_bits >> 3, cbytes = ti.comp_bits >> 3;
+        // where the three arrays go (g, theta, c), and how many pages that takes including
+        // those skipped when a run does not fit before the end of the ring
+        const int run[3] = {kChunk * 4 / kPageBytes, kChunk * tbytes / kPageBytes, kChunk * cbytes / kPageBytes};
+        int page[3] = {0, 0, 0}, h2 = head, need = 0;
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+          if (run[r] == 0) continue;
+          if (h2 + run[r] > kPages) { need += kPages - h2; h2 = 0; }
+          page[r] = h2;
+          h2 += run[r];
+          need += run[r];
+        }
+        if (h2 == kPages) h2 = 0;
+        // take back pages, descriptor slots and scans from the oldest tiles until this one fits
+        while (free_pages < need || i - oldest >= kSlots) {
+          const int os = oldest % kSlots;
+          if (!mbar_wait(&sh->empty[os], (unsigned)(oldest / kSlots) & 1u, &sh->abort_flag)) {
+            gave_up = true;
             break;
           }
-          take_back(p, acc, &sh->scan[stage], sh->desc[stage].tensor);
+          take_back(p, acc, &sh->scan[os], sh->desc[os].tensor);
+          free_pages += sh->slot_pages[os];
+          ++oldest;
         }
-        const TensorInfo& ti = meta.ti;
+        if (gave_up) {
+          sh->abort_flag = 1;
+          atomicCAS(p.ws.error, 0u, (unsigned)kErrEmptyWait);
+          break;
+        }
+        head = h2;
+        free_pages -= need;
+        sh->slot_pages[slot] = need;
+
         const StepCoef coef = make_coef(ti, meta.e_in, meta.e_out, meta.lr);
         const long long first = (long long)cr.index * kChunk;
         const long long left = ti.numel - first;
         const int count = left < (long long)kChunk ? (int)left : kChunk;
         const int n_bulk = count & ~15;
-        const int tbytes = ti.theta_bits >> 3, cbytes = ti.comp_bits >> 3;
-        TileDesc& td = sh->desc[stage];
+        TileDesc& td = sh->desc[slot];
         td.scale = coef.scale;
         td.pow2s_neg = -pow2_float(coef.s);
         td.inv2s = pow2_float(-coef.s);
@@ -677,37 +711,39 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
         td.tensor = cr.tensor;
         td.n_bulk = n_bulk;
         td.count = count;
-        td.flags = ((ti.theta_bits == 16 ? 3 : 0) + (ti.comp_bits >> 3)) | (coef.delta == 0 ? kFlagSteady : 0);
+        td.flags = ((ti.theta_bits == 16 ? 3 : 0) + (ti.comp_bits >> 3)) |
+                   (coef.delta == 0 ? kFlagSteady : 0) | (page[1] << kFlagThetaPageShift) |
+                   (page[2] << kFlagCompPageShift) | (page[0] << kFlagGradPageShift);
         td.coef = coef;
         td.grad = meta.grad + first;
-        unsigned char* st = smem + (size_t)stage * kStageBytes;
         if (n_bulk > 0) {
-          mbar_arrive_expect_tx(&sh->full[stage], (unsigned)(n_bulk * (tbytes + cbytes + 4)));
-          bulk_load(st + kStageThetaOff, td.theta, (unsigned)(n_bulk * tbytes), &sh->full[stage]);
-          if (cbytes) bulk_load(st + kStageCompOff, td.comp, (unsigned)(n_bulk * cbytes), &sh->full[stage]);
+          mbar_arrive_expect_tx(&sh->full[slot], (unsigned)(n_bulk * (tbytes + cbytes + 4)));
+          bulk_load(smem + page[1] * kPageBytes, td.theta, (unsigned)(n_bulk * tbytes), &sh->full[slot]);
+          if (cbytes)
+            bulk_load(smem + page[2] * kPageBytes, td.comp, (unsigned)(n_bulk * cbytes), &sh->full[slot]);
           // Gradients are read once.  When theta and c of the whole list fit in L2, letting
           // the gradients leave it first keeps the state resident from step to step.
           if (p.grad_evict_first)
-            bulk_load_hint(st + kStageGradOff, td.grad, (unsigned)(n_bulk * 4), &sh->full[stage], grad_policy);
+            bulk_load_hint(smem + page[0] * kPageBytes, td.grad, (unsigned)(n_bulk * 4), &sh->full[slot],
+                           grad_policy);
           else
-            bulk_load(st + kStageGradOff, td.grad, (unsigned)(n_bulk * 4), &sh->full[stage]);
+            bulk_load(smem + page[0] * kPageBytes, td.grad, (unsigned)(n_bulk * 4), &sh->full[slot]);
         } else {
-          mbar_arrive(&sh->full[stage]);
+          mbar_arrive(&sh->full[slot]);
         }
         issued = i + 1;
         cr = cr1;
         cr1 = cr2;
         meta = meta1;
       }
-      // Collect the scans of the last tiles (their stages are not reused) and publish.
-      // The same waits make sure that every copy this block started has landed before
-      // the block exits.
-      for (int i = max(0, issued - kStages); i < issued; ++i) {
-        const int stage = i % kStages;
-        if (mbar_wait(&sh->empty[stage], (unsigned)(i / kStages) & 1u, &sh->abort_flag))
-          take_back(p, acc, &sh->scan[stage], sh->desc[stage].tensor);
+      // Collect the scans of the tiles still in the ring and publish.  The same waits make
+      // sure that every copy this block started has landed before the block exits.
+      for (int i = oldest; i < issued; ++i) {
+        const int os = i % kSlots;
+        if (mbar_wait(&sh->empty[os], (unsigned)(i / kSlots) & 1u, &sh->abort_flag))
+          take_back(p, acc, &sh->scan[os], sh->desc[os].tensor);
         else
-          mbar_wait(&sh->full[stage], (unsigned)(i / kStages) & 1u, &sh->never);
+          mbar_wait(&sh->full[os], (unsigned)(i / kSlots) & 1u, &sh->never);
       }
       publish(p, acc);
     }
@@ -718,7 +754,7 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
     const int n_my = ((int)p.n_chunks - (int)blockIdx.x + stride - 1) / stride;
     float amax_t = 0.0f, amax_c = 0.0f;
     for (int i = 0; i < n_my; ++i) {
-      const int stage = i % kStages, use = i / kStages;
+      const int stage = i % kSlots, use = i / kSlots;
       if (!mbar_wait(&sh->full[stage], (unsigned)use & 1u, &sh->abort_flag)) {
         if (lane == 0) {
           sh->abort_flag = 1;
@@ -743,7 +779,7 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
         h.count = (int)q2.z;
         h.flags = (int)q2.w;
       }
-      unsigned char* st = smem + (size_t)stage * kStageBytes;
+      unsigned char* st = smem;
       bool wrote_stage;
       switch (h.flags & kFlagFormatMask) {
         case 0: wrote_stage = consume_tile<8, 0>(h, td, st, ctid, scan, amax_t, amax_c); break;

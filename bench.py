@@ -34,13 +34,16 @@ if ROOT not in sys.path:
 METRIC = "parameters updated/sec and achieved HBM GB/s (% of B200 peak) per Kahan SGD step"
 UNIT = "parameters/s"
 FALLBACK_HBM_GBS = 6650.0
-GRAD_SETS = {"c5_sweep": 2}     # how many gradient sets stay resident and rotate
+# Gradient sets kept resident and used in turn: c5 alternates two sets (its recipe), the
+# other workloads draw a fresh gradient for every step of their recipe.
+GRAD_SETS = {"c5_sweep": 2, "c1_single": 100, "c2_resnet20": 200, "c3_resnet50": 50, "c4_alexnet": 20}
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=0,
+                    help="timed steps (default: 200 for c5_sweep, the recipe's own step count otherwise)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c5_sweep")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -149,6 +152,8 @@ def run_ours(args, rank, world, local_rank):
     wl = pick_workload(W, args)
     n = len(wl.tensors)
     n_sets = GRAD_SETS.get(wl.name, 4)
+    if not args.steps:
+        args.steps = 200 if wl.name == "c5_sweep" else wl.steps
     t0 = time.time()
     host = HostInputs(wl, multi.rank_seed(args.seed, rank), n_sets, pinned=True)
     gen_s = time.time() - t0
@@ -284,6 +289,8 @@ def run_reference(args, rank, world):
     from paper_1810_05486_b200 import workloads as W
     from oracle import oracle_step_tensor, oracle_max_threads
     wl = pick_workload(W, args)
+    if not args.steps:
+        args.steps = 3
     cores = oracle_max_threads()
     # sample: the largest tensors up to ~64M parameters per step
     order = sorted(range(len(wl.tensors)), key=lambda i: -wl.tensors[i].numel)

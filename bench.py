@@ -39,6 +39,38 @@ FALLBACK_HBM_GBS = 6650.0
 GRAD_SETS = {"c5_sweep": 2, "c1_single": 100, "c2_resnet20": 200, "c3_resnet50": 50, "c4_alexnet": 20}
 
 
+# DRAM traffic of ksgd_step_kernel from ncu captures (dram__bytes_read.sum +
+# dram__bytes_write.sum per launch, divided by the parameters of the captured launch; see
+# profiles/).  c5_sweep was captured at 2e8 parameters; traffic is proportional to the
+# parameter count, so a full launch is this figure times its parameters.  The record only
+# counts while the kernel sources still hash to the value below.
+TRAFFIC_RECORD = {
+    "sources_sha256": "877d20bfa10196f56381e6163606994e56ba204ad0b993b73ea47de29e30a71a",
+    "dram_bytes_per_parameter": {"c5_sweep": 2356.633e6 / 2e8, "c4_alexnet": 470.829e6 / 61100840,
+                                 "c3_resnet50": 199.963e6 / 25557032},
+}
+
+
+def kernel_sources_sha256():
+    import hashlib
+    h = hashlib.sha256()
+    for name in ("kahan_sgd_kernels.cuh", "kahan_sgd_api.cu"):
+        with open(os.path.join(ROOT, "paper_1810_05486_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def recorded_traffic(wl):
+    """DRAM bytes of one launch from the ncu record, or None once the kernel has changed."""
+    try:
+        if kernel_sources_sha256() != TRAFFIC_RECORD["sources_sha256"]:
+            return None
+        per = TRAFFIC_RECORD["dram_bytes_per_parameter"].get(wl.name)
+        return None if per is None else per * wl.numel
+    except Exception:
+        return None
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -221,13 +253,7 @@ def run_ours(args, rank, world, local_rank):
 
     peak, peak_src = hbm_peak()
     achieved = wl.bytes_per_step / (ms_step * 1e-3) / 1e9
-    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
-    traffic = None
-    try:
-        with open(traffic_path) as f:
-            traffic = json.load(f).get(wl.name)
-    except Exception:
-        pass
+    traffic = recorded_traffic(wl)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,

@@ -50,7 +50,7 @@ class DeviceArena:
         return bool((self.buf[mask] == CANARY).all().item())
 
 
-class GpuRun:
+class LibraryRun:
     """Drives kahan_sgd_* on device copies of the given tensors."""
 
     def __init__(self, specs: Sequence[dict], thetas: Sequence[np.ndarray],
@@ -127,7 +127,7 @@ def make_oracle_state(specs, thetas, comps, mode, n_threads=1):
     return OracleState(ts, mode, n_threads)
 
 
-def assert_same_state(gpu: GpuRun, ost, where="") -> None:
+def assert_same_state(gpu: LibraryRun, ost, where="") -> None:
     """Bit-exact comparison of everything a step produces."""
     st = gpu.stats()
     got_t, got_c = gpu.thetas(), gpu.comps()

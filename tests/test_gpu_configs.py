@@ -10,7 +10,7 @@ import os
 import numpy as np
 import pytest
 
-from harness import GpuRun, assert_same_state, make_oracle_state, specs_of
+from harness import LibraryRun, assert_same_state, make_oracle_state, specs_of
 from oracle import EXP_AMAX, OracleState, OracleTensor, oracle_max_threads, oracle_step
 from paper_1810_05486_b200 import workloads as W
 
@@ -20,7 +20,7 @@ pytestmark = pytest.mark.gpu
 def run_config(wl, steps, check_every=1):
     specs = specs_of(wl)
     thetas, comps = W.initial_state(wl)
-    gpu = GpuRun(specs, thetas, comps, EXP_AMAX)
+    gpu = LibraryRun(specs, thetas, comps, EXP_AMAX)
     ost = make_oracle_state(specs, thetas, comps, EXP_AMAX, n_threads=oracle_max_threads())
     lrs = [wl.lr] * len(specs)
     try:

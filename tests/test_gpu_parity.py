@@ -6,7 +6,7 @@ current and next exponents, both max scans and the three counters, after every s
 import numpy as np
 import pytest
 
-from harness import GpuRun, assert_same_state, make_oracle_state, specs_of, storage_dtype
+from harness import LibraryRun, assert_same_state, make_oracle_state, specs_of, storage_dtype
 from oracle import EXP_AMAX, EXP_FIXED, oracle_step
 from paper_1810_05486_b200 import workloads as W
 
@@ -20,7 +20,7 @@ def qmax(b):
 
 
 def run_both(specs, thetas, comps, grads_per_step, lrs_per_step, mode=EXP_AMAX, exps_per_step=None):
-    gpu = GpuRun(specs, thetas, comps, mode)
+    gpu = LibraryRun(specs, thetas, comps, mode)
     ost = make_oracle_state(specs, thetas, comps, mode)
     try:
         for step, (grads, lrs) in enumerate(zip(grads_per_step, lrs_per_step)):
@@ -63,7 +63,7 @@ def test_all_int8_pairs_times_gradient_sweep():
     mults = mults + [-m for m in mults[1:]]
     specs = [dict(numel=theta.size, theta_bits=8, comp_bits=8, overlap_k=0, exp_theta=e_t)]
     grads = [[np.full(theta.size, np.float32(m * lsb / 0.25), np.float32)] for m in mults]
-    gpu = GpuRun(specs, [theta], [comp], EXP_FIXED)
+    gpu = LibraryRun(specs, [theta], [comp], EXP_FIXED)
     try:
         for m, g in zip(mults, grads):
             # same starting state for every increment: re-upload
@@ -151,7 +151,7 @@ def test_every_exponent_change(tb, cb, k):
     exps = [[-20 + d for d in deltas], None, [-20 for _ in deltas]]
     # step 1 follows the max scan after the forced change; step 2 is forced back
     # (the forced value must stay within 8 of the then-current exponent, which it does)
-    gpu = GpuRun(specs, thetas, comps, EXP_AMAX)
+    gpu = LibraryRun(specs, thetas, comps, EXP_AMAX)
     ost = make_oracle_state(specs, thetas, comps, EXP_AMAX)
     try:
         for step in range(3):
@@ -260,19 +260,19 @@ def test_checkpoint_resume_is_bit_identical():
     grads = [W.gradients(wl, s) for s in range(6)]
     grads = [[g * np.float32(30.0) for g in gs] for gs in grads]
     lrs = [[wl.lr] * len(specs)] * 6
-    a = GpuRun(specs, thetas, comps, EXP_AMAX)
+    a = LibraryRun(specs, thetas, comps, EXP_AMAX)
     for s in range(6):
         a.step(grads[s], lrs[s])
     ta, ca, sa = a.thetas(), a.comps(), a.stats()
     a.close()
-    b = GpuRun(specs, thetas, comps, EXP_AMAX)
+    b = LibraryRun(specs, thetas, comps, EXP_AMAX)
     for s in range(3):
         b.step(grads[s], lrs[s])
     tb_, cb_, sb = b.thetas(), b.comps(), b.stats()
     b.close()
     specs2 = [dict(sp, exp_theta=sb["exp_theta_cur"][i], exp_theta_next=sb["exp_theta_next"][i])
               for i, sp in enumerate(specs)]
-    c = GpuRun(specs2, tb_, cb_, EXP_AMAX)
+    c = LibraryRun(specs2, tb_, cb_, EXP_AMAX)
     for s in range(3, 6):
         c.step(grads[s], lrs[s])
     tc, cc, sc = c.thetas(), c.comps(), c.stats()
@@ -293,7 +293,7 @@ def test_step_on_a_side_stream_and_back_to_back_steps():
     g = (rng.standard_normal(n) * 1e-4).astype(np.float32)
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
-        gpu = GpuRun(specs, [th], [c], EXP_AMAX, stream=side)
+        gpu = LibraryRun(specs, [th], [c], EXP_AMAX, stream=side)
         gpu.grad_arena.upload(0, g)
         side.synchronize()
         for _ in range(25):
@@ -315,7 +315,7 @@ def test_step_host_matches_device_step():
     thetas, comps = W.initial_state(wl)
     grads = [g * np.float32(25.0) for g in W.gradients(wl, 0)]
     lrs = [wl.lr] * len(specs)
-    gpu = GpuRun(specs, [np.zeros_like(t) for t in thetas], [np.zeros_like(c) for c in comps],
+    gpu = LibraryRun(specs, [np.zeros_like(t) for t in thetas], [np.zeros_like(c) for c in comps],
                  EXP_AMAX)
     ost = make_oracle_state(specs, thetas, comps, EXP_AMAX)
     th_h = [t.copy() for t in thetas]

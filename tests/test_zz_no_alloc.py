@@ -13,7 +13,7 @@ run every other test.
 import numpy as np
 import pytest
 
-from harness import DeviceArena, GpuRun, storage_dtype
+from harness import DeviceArena, LibraryRun, storage_dtype
 
 pytestmark = pytest.mark.gpu
 
@@ -52,7 +52,7 @@ def test_static_entry_point_matches_the_workspace_path_twice_in_a_row():
     n = len(specs)
 
     # reference: the ordinary path with a caller-provided workspace
-    ref = GpuRun(specs, thetas, comps, B.KSGD_EXP_AMAX)
+    ref = LibraryRun(specs, thetas, comps, B.KSGD_EXP_AMAX)
     ref_states = []
     prev = ref.stats()
     for step in range(2):

@@ -13,6 +13,10 @@ from .kahan_oracle import (  # noqa: F401
     oracle_next_exponent,
     oracle_step_tensor,
     oracle_step,
+    OracleMomElem,
+    oracle_momentum_element,
+    oracle_momentum_step_tensor,
+    oracle_momentum_step,
     oracle_max_threads,
     EXP_FIXED,
     EXP_AMAX,

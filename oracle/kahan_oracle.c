@@ -40,7 +40,11 @@
  * against exact rational arithmetic, a literal four-statement transcription of
  * Algorithm 1, the m+n-2-k bit-width closed form with the ties-to-even step
  * counts, the plain-SGD reduction (Eq. 1), regrid value preservation, and the
- * exponent-policy property.  Accuracy tables of Section 4: parity unpinned
+ * exponent-policy property; for the momentum variant (tests/test_oracle_momentum_pins.py):
+ * reduction to the plain lazy update at mu = 0, the velocity recursion against exact
+ * rationals with explicit binary32 rounding, the geometric fixed point, the exact
+ * accumulation invariant and both directions of the velocity-to-compensation grid shift.
+ * Accuracy tables of Section 4: parity unpinned
  * (datasets and trained weights are not available).
  *
  * Build: gcc -O2 -ffp-contract=off -fopenmp -shared -fPIC (see oracle/build.py).
@@ -240,6 +244,136 @@ int32_t ksgd_oracle_next_exponent(uint32_t amax_theta, int32_t theta_bits,
   if (e_next > 64) e_next = 64;
   if (e_next < -64) e_next = -64;
   return e_next;
+}
+
+/* ------------------------------------------------------------------------------------
+ * Momentum optimizer with the lazy update (Section 4: "the lazy update described in
+ * Algorithm 1 was implemented in the optimizers"; momentum mu = 0.9 in INT8, INT16 for
+ * AlexNet).  The paper gives no formulas; the reading taken is the classical form
+ *     v <- mu*v + eta*g ,   theta <- theta - v
+ * with v a third dynamic fixed-point tensor (b-bit mantissas Q_v, own exponent e_v that
+ * follows its own max scan) and Algorithm 1 applied with v in the place of eta*g:
+ *   mu_s = fl32(mu * 2^(ev_in - ev_out))                 exact power-of-two rescaling
+ *   bq   = fl32(g * fl32(eta * 2^-ev_out))               one binary32 multiply
+ *   y    = fma32(mu_s, Q_v, bq)                           one rounding
+ *   V    = clamp(rne(y), +-2^30), NaN -> 0 ;  Q_v' = clamp(V, +-(2^(b-1)-1))
+ *   d    = Q_v' * 2^k (clamped to +-2^30) if k >= 0 else rne(Q_v' / 2^-k),
+ *          k = ev_out - ec_out: the stored velocity expressed on the compensation grid
+ *   then statements 1-4 of Algorithm 1 with this d.
+ */
+typedef struct {
+  ksgd_oracle_elem upd;  /* the parameter update (d = increment taken from the velocity)   */
+  int64_t V;             /* velocity mantissa before saturation, units of 2^ev_out          */
+  int32_t q_mom;         /* stored velocity mantissa                                        */
+} ksgd_oracle_mom_elem;
+
+static int32_t velocity_mantissa(int32_t q_mom, float g, float lr, float mu, int32_t ev_in,
+                                 int32_t ev_out) {
+  float mu_s = ldexpf(mu, ev_in - ev_out);
+  float scale_v = ldexpf(lr, -ev_out);
+  float bq = g * scale_v;
+  float y = fmaf(mu_s, (float)q_mom, bq);
+  if (isnan(y)) return 0;
+  const float lim = 1073741824.0f;
+  if (y >= lim) return (int32_t)1 << 30;
+  if (y <= -lim) return -((int32_t)1 << 30);
+  return (int32_t)nearbyintf(y);
+}
+
+void ksgd_oracle_momentum_element(int32_t q_theta, int32_t q_comp, int32_t q_mom, float g, float lr,
+                                  float mu, int32_t m, int32_t n, int32_t s, int32_t b,
+                                  int32_t e_in, int32_t e_out, int32_t ev_in, int32_t ev_out,
+                                  ksgd_oracle_mom_elem* out) {
+  if (n == 0) { s = 0; q_comp = 0; }
+  int64_t V = velocity_mantissa(q_mom, g, lr, mu, ev_in, ev_out);
+  int64_t q_mom_new = clamp_i64(V, -qmax_bits(b), qmax_bits(b));
+
+  int32_t ec_in = e_in - s, ec_out = e_out - s;
+  int32_t f = ec_in < ec_out ? ec_in : ec_out;
+  int32_t k = ev_out - ec_out;
+  int64_t d;
+  if (k >= 0) {
+    /* |Q_v'| < 2^15, so any k >= 16 with Q_v' != 0 is beyond the clamp */
+    d = k > 40 ? (q_mom_new > 0 ? pow2_i64(30) : (q_mom_new < 0 ? -pow2_i64(30) : 0))
+               : clamp_i64(q_mom_new * pow2_i64(k), -pow2_i64(30), pow2_i64(30));
+  } else {
+    d = -k > 40 ? 0 : ksgd_oracle_rne_shift(q_mom_new, -k);
+  }
+
+  int64_t T = (int64_t)q_theta * pow2_i64(e_in - f) + (int64_t)q_comp * pow2_i64(ec_in - f) -
+              d * pow2_i64(ec_out - f);
+  int64_t P = ksgd_oracle_rne_shift(T, e_out - f);
+  int64_t q_theta_new = clamp_i64(P, -qmax_bits(m), qmax_bits(m));
+  int64_t R = T - q_theta_new * pow2_i64(e_out - f);
+  int64_t Rq = 0, q_comp_new = 0;
+  if (n != 0) {
+    Rq = ksgd_oracle_rne_shift(R, ec_out - f);
+    q_comp_new = clamp_i64(Rq, -qmax_bits(n), qmax_bits(n));
+  }
+  out->upd.P = P;
+  out->upd.Rq = Rq;
+  out->upd.T = T;
+  out->upd.d = (int32_t)d;
+  out->upd.q_theta = (int32_t)q_theta_new;
+  out->upd.q_comp = (int32_t)q_comp_new;
+  out->upd.nonfinite = isfinite(g) ? 0 : 1;
+  out->V = V;
+  out->q_mom = (int32_t)q_mom_new;
+}
+
+typedef struct {
+  ksgd_oracle_stats upd;
+  uint32_t amax_mom;    /* max |V| over the tensor                     */
+  uint64_t n_sat_mom;   /* elements whose velocity mantissa was clamped */
+} ksgd_oracle_mom_stats;
+
+int ksgd_oracle_momentum_step_tensor(void* theta, void* comp, void* mom, const float* grad,
+                                     int64_t numel, int32_t theta_bits, int32_t comp_bits,
+                                     int32_t overlap_k, int32_t mom_bits, int32_t e_in,
+                                     int32_t e_out, int32_t ev_in, int32_t ev_out, float lr, float mu,
+                                     ksgd_oracle_mom_stats* stats, int32_t n_threads) {
+  if (!theta || !mom || !grad || !stats || numel <= 0) return -1;
+  if (theta_bits < 2 || theta_bits > 16 || mom_bits < 2 || mom_bits > 16) return -1;
+  if (comp_bits != 0 && (comp_bits < 2 || comp_bits > 16)) return -1;
+  if (comp_bits != 0 && (!comp || overlap_k < 0 || overlap_k > comp_bits - 1)) return -1;
+  if (e_out - e_in > 8 || e_in - e_out > 8 || ev_out - ev_in > 8 || ev_in - ev_out > 8) return -1;
+  int32_t s = comp_bits == 0 ? 0 : comp_bits - 1 - overlap_k;
+  uint32_t amax_theta = 0, amax_comp = 0, amax_mom = 0;
+  uint64_t n_sat_theta = 0, n_sat_comp = 0, n_nonfinite = 0, n_sat_mom = 0;
+  if (n_threads < 1) n_threads = 1;
+#pragma omp parallel for schedule(static) num_threads(n_threads) \
+    reduction(max : amax_theta, amax_comp, amax_mom) \
+    reduction(+ : n_sat_theta, n_sat_comp, n_nonfinite, n_sat_mom)
+  for (int64_t i = 0; i < numel; ++i) {
+    ksgd_oracle_mom_elem r;
+    int32_t qt = load_mantissa(theta, i, theta_bits);
+    int32_t qc = comp_bits ? load_mantissa(comp, i, comp_bits) : 0;
+    int32_t qv = load_mantissa(mom, i, mom_bits);
+    ksgd_oracle_momentum_element(qt, qc, qv, grad[i], lr, mu, theta_bits, comp_bits, s, mom_bits,
+                                 e_in, e_out, ev_in, ev_out, &r);
+    store_mantissa(theta, i, theta_bits, r.upd.q_theta);
+    if (comp_bits) store_mantissa(comp, i, comp_bits, r.upd.q_comp);
+    store_mantissa(mom, i, mom_bits, r.q_mom);
+    int64_t aP = r.upd.P < 0 ? -r.upd.P : r.upd.P;
+    int64_t aR = r.upd.Rq < 0 ? -r.upd.Rq : r.upd.Rq;
+    int64_t aV = r.V < 0 ? -r.V : r.V;
+    if (aR > 2147483647LL) aR = 2147483647LL;
+    if ((uint32_t)aP > amax_theta) amax_theta = (uint32_t)aP;
+    if ((uint32_t)aR > amax_comp) amax_comp = (uint32_t)aR;
+    if ((uint32_t)aV > amax_mom) amax_mom = (uint32_t)aV;
+    n_sat_theta += (r.upd.P != r.upd.q_theta);
+    n_sat_comp += (comp_bits != 0 && r.upd.Rq != r.upd.q_comp);
+    n_sat_mom += (r.V != r.q_mom);
+    n_nonfinite += (uint64_t)r.upd.nonfinite;
+  }
+  stats->upd.amax_theta = amax_theta;
+  stats->upd.amax_comp = amax_comp;
+  stats->upd.n_sat_theta = n_sat_theta;
+  stats->upd.n_sat_comp = n_sat_comp;
+  stats->upd.n_nonfinite = n_nonfinite;
+  stats->amax_mom = amax_mom;
+  stats->n_sat_mom = n_sat_mom;
+  return 0;
 }
 
 int32_t ksgd_oracle_max_threads(void) {

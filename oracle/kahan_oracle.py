@@ -23,10 +23,18 @@ class OracleElem(ctypes.Structure):
                 ("q_comp", ctypes.c_int32), ("nonfinite", ctypes.c_int32)]
 
 
+class OracleMomElem(ctypes.Structure):
+    _fields_ = [("upd", OracleElem), ("V", ctypes.c_int64), ("q_mom", ctypes.c_int32)]
+
+
 class _Stats(ctypes.Structure):
     _fields_ = [("amax_theta", ctypes.c_uint32), ("amax_comp", ctypes.c_uint32),
                 ("n_sat_theta", ctypes.c_uint64), ("n_sat_comp", ctypes.c_uint64),
                 ("n_nonfinite", ctypes.c_uint64)]
+
+
+class _MomStats(ctypes.Structure):
+    _fields_ = [("upd", _Stats), ("amax_mom", ctypes.c_uint32), ("n_sat_mom", ctypes.c_uint64)]
 
 
 _lib = None
@@ -52,6 +60,13 @@ def _load():
         lib.ksgd_oracle_next_exponent.restype = ctypes.c_int32
         lib.ksgd_oracle_next_exponent.argtypes = [ctypes.c_uint32, ctypes.c_int32,
                                                   ctypes.c_int32, ctypes.c_int32]
+        lib.ksgd_oracle_momentum_element.restype = None
+        lib.ksgd_oracle_momentum_element.argtypes = [ctypes.c_int32] * 3 + [ctypes.c_float] * 3 + \
+            [ctypes.c_int32] * 8 + [ctypes.POINTER(OracleMomElem)]
+        lib.ksgd_oracle_momentum_step_tensor.restype = ctypes.c_int
+        lib.ksgd_oracle_momentum_step_tensor.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int64] + \
+            [ctypes.c_int32] * 8 + [ctypes.c_float, ctypes.c_float, ctypes.POINTER(_MomStats),
+                                    ctypes.c_int32]
         lib.ksgd_oracle_max_threads.restype = ctypes.c_int32
         lib.ksgd_oracle_max_threads.argtypes = []
         _lib = lib
@@ -111,6 +126,36 @@ def oracle_step_tensor(theta: np.ndarray, comp: Optional[np.ndarray], grad: np.n
             "n_nonfinite": st.n_nonfinite}
 
 
+def oracle_momentum_element(q_theta: int, q_comp: int, q_mom: int, g: float, lr: float, mu: float,
+                            m: int, n: int, s: int, b: int, e_in: int, e_out: int, ev_in: int,
+                            ev_out: int) -> OracleMomElem:
+    """Momentum with the lazy update for one element (v <- mu v + eta g, then Algorithm 1 with v)."""
+    out = OracleMomElem()
+    _load().ksgd_oracle_momentum_element(q_theta, q_comp, q_mom, g, lr, mu, m, n, s, b, e_in, e_out,
+                                         ev_in, ev_out, ctypes.byref(out))
+    return out
+
+
+def oracle_momentum_step_tensor(theta, comp, mom, grad, theta_bits, comp_bits, overlap_k, mom_bits,
+                                e_in, e_out, ev_in, ev_out, lr, mu, n_threads: int = 1) -> dict:
+    """Momentum step over one tensor, in place on theta, comp and mom; returns the stats."""
+    assert theta.dtype == _storage_dtype(theta_bits) and theta.flags.c_contiguous
+    assert mom.dtype == _storage_dtype(mom_bits) and mom.flags.c_contiguous and mom.size == theta.size
+    assert grad.dtype == np.float32 and grad.flags.c_contiguous and grad.size == theta.size
+    if comp_bits:
+        assert comp is not None and comp.dtype == _storage_dtype(comp_bits) and comp.size == theta.size
+    st = _MomStats()
+    rc = _load().ksgd_oracle_momentum_step_tensor(
+        theta.ctypes.data, comp.ctypes.data if comp_bits else None, mom.ctypes.data, grad.ctypes.data,
+        theta.size, theta_bits, comp_bits, overlap_k, mom_bits, e_in, e_out, ev_in, ev_out,
+        ctypes.c_float(lr), ctypes.c_float(mu), ctypes.byref(st), n_threads)
+    if rc != 0:
+        raise ValueError("oracle rejected the tensor description")
+    return {"amax_theta": st.upd.amax_theta, "amax_comp": st.upd.amax_comp,
+            "n_sat_theta": st.upd.n_sat_theta, "n_sat_comp": st.upd.n_sat_comp,
+            "n_nonfinite": st.upd.n_nonfinite, "amax_mom": st.amax_mom, "n_sat_mom": st.n_sat_mom}
+
+
 @dataclass
 class OracleTensor:
     """One parameter tensor: mantissas, compensation, formats and exponents."""
@@ -126,6 +171,13 @@ class OracleTensor:
     n_sat_theta: int = 0        # cumulative
     n_sat_comp: int = 0
     n_nonfinite: int = 0
+    # momentum variant only
+    mom: Optional[np.ndarray] = None
+    mom_bits: int = 0
+    exp_mom: int = 0
+    exp_mom_next: int = 0
+    amax_mom: int = 0
+    n_sat_mom: int = 0
 
     @property
     def s(self) -> int:
@@ -157,3 +209,24 @@ def oracle_step(state: OracleState, grads: Sequence[np.ndarray], lrs: Sequence[f
         t.n_nonfinite += st["n_nonfinite"]
         t.exp_theta = e_out
         t.exp_theta_next = oracle_next_exponent(t.amax_theta, t.theta_bits, e_out, state.mode)
+
+
+def oracle_momentum_step(state: OracleState, grads: Sequence[np.ndarray], lrs: Sequence[float],
+                         mus: Sequence[float]) -> None:
+    """One momentum step of every tensor, then the exponent choices: theta's exponent
+    follows max |P|, the velocity's exponent follows max |V|, each on its own."""
+    assert len(grads) == len(state.tensors) == len(lrs) == len(mus)
+    for t, g, lr, mu in zip(state.tensors, grads, lrs, mus):
+        e_in, e_out, ev_in, ev_out = t.exp_theta, t.exp_theta_next, t.exp_mom, t.exp_mom_next
+        st = oracle_momentum_step_tensor(t.theta, t.comp, t.mom, g, t.theta_bits, t.comp_bits,
+                                         t.overlap_k, t.mom_bits, e_in, e_out, ev_in, ev_out,
+                                         float(lr), float(mu), state.n_threads)
+        t.amax_theta, t.amax_comp, t.amax_mom = st["amax_theta"], st["amax_comp"], st["amax_mom"]
+        t.n_sat_theta += st["n_sat_theta"]
+        t.n_sat_comp += st["n_sat_comp"]
+        t.n_nonfinite += st["n_nonfinite"]
+        t.n_sat_mom += st["n_sat_mom"]
+        t.exp_theta = e_out
+        t.exp_theta_next = oracle_next_exponent(t.amax_theta, t.theta_bits, e_out, state.mode)
+        t.exp_mom = ev_out
+        t.exp_mom_next = oracle_next_exponent(t.amax_mom, t.mom_bits, ev_out, state.mode)

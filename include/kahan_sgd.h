@@ -186,6 +186,49 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
 /* Free the host-side handle (waits for the stream first).  Device buffers stay the caller's. */
 int kahan_sgd_destroy(ksgd_handle* h);
 
+/*
+ * Momentum optimizer with the lazy update (Section 4: Algorithm 1 "was implemented in the
+ * optimizers"; momentum mu = 0.9 kept in INT8, INT16 for AlexNet).  The paper prints no
+ * formulas for it; the form implemented is
+ *     v <- mu*v + eta*g ,   theta <- theta - v   (the subtraction through Algorithm 1)
+ * with the velocity v a third dynamic fixed-point tensor: mom_bits-bit mantissas with their
+ * own shared exponent, which follows the max scan of |V| exactly as theta's exponent
+ * follows |P| (one step of delay, at most 8 binades per step, [-64, 64]).  Per element:
+ *     y  = fma32(fl32(mu * 2^(ev_in - ev_out)), Q_v, fl32(g * fl32(eta * 2^-ev_out)))
+ *     V  = clamp(rne(y), +-2^30), NaN -> 0 ;   Q_v' = clamp(V, +-(2^(mom_bits-1) - 1))
+ *     d  = Q_v' * 2^k if k >= 0 (clamped to +-2^30), rne(Q_v' / 2^-k) otherwise,
+ *          k = ev_out - (e_out - s): the stored velocity on the compensation grid
+ *     then T, P, Q_theta', Rq, Q_c' as in the plain step with this d.
+ * The tensor descriptions are the same ksgd_tensor_desc (comp_bits must be 8 or 16) plus
+ * one ksgd_momentum_desc per tensor.  At most 256 tensors per list.  Ownership, streams,
+ * return codes and the meaning of the common outputs are as for the plain entry points;
+ * mus: host array of momentum coefficients, finite and >= 0 (an invalid one gives
+ * KSGD_ERR_LR).  amax_mom = max |V| of the last step, n_sat_mom = clamped velocity
+ * mantissas since init.
+ */
+typedef struct ksgd_momentum_handle ksgd_momentum_handle;
+
+typedef struct {
+  void*   mom;           /* device, int8_t[numel] (mom_bits 8) or int16_t[numel] (16); in place; 16-byte aligned */
+  int32_t mom_bits;      /* 8 | 16 */
+  int32_t exp_mom;       /* exponent of the velocity mantissas now stored, in [-64, 64] */
+  int32_t exp_mom_next;  /* exponent the first step writes, within 8 of exp_mom */
+  int32_t reserved;      /* 0 */
+} ksgd_momentum_desc;
+
+size_t kahan_sgd_momentum_workspace_bytes(const ksgd_tensor_desc* descs, const ksgd_momentum_desc* mdescs,
+                                          int32_t n_tensors);
+int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* descs,
+                            const ksgd_momentum_desc* mdescs, int32_t n_tensors, ksgd_exp_mode mode,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+int kahan_sgd_momentum_step(ksgd_momentum_handle* h, const float* const* grads, const float* lrs,
+                            const float* mus);
+int kahan_sgd_momentum_amax(ksgd_momentum_handle* h, uint32_t* amax_theta, uint32_t* amax_comp,
+                            uint32_t* amax_mom, int32_t* exp_theta_cur, int32_t* exp_theta_next,
+                            int32_t* exp_mom_cur, int32_t* exp_mom_next, uint64_t* n_sat_theta,
+                            uint64_t* n_sat_comp, uint64_t* n_sat_mom, uint64_t* n_nonfinite);
+int kahan_sgd_momentum_destroy(ksgd_momentum_handle* h);
+
 /* Static text for a KSGD_* code. */
 const char* kahan_sgd_strerror(int code);
 

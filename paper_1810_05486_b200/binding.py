@@ -30,7 +30,8 @@ KSGD_ERR_DEVICE = -11
 EXPORTS = (
     "kahan_sgd_workspace_bytes", "kahan_sgd_init", "kahan_sgd_step", "kahan_sgd_step_host",
     "kahan_sgd_amax", "kahan_sgd_set_exponents", "kahan_sgd_step_static", "kahan_sgd_destroy",
-    "kahan_sgd_strerror",
+    "kahan_sgd_strerror", "kahan_sgd_momentum_workspace_bytes", "kahan_sgd_momentum_init",
+    "kahan_sgd_momentum_step", "kahan_sgd_momentum_amax", "kahan_sgd_momentum_destroy",
     "kahan_sgd_last_cuda_error", "kahan_sgd_launch_count",
 )
 
@@ -40,6 +41,11 @@ class ksgd_tensor_desc(ctypes.Structure):
                 ("theta_bits", ctypes.c_int32), ("comp_bits", ctypes.c_int32),
                 ("overlap_k", ctypes.c_int32), ("exp_theta", ctypes.c_int32),
                 ("exp_theta_next", ctypes.c_int32)]
+
+
+class ksgd_momentum_desc(ctypes.Structure):
+    _fields_ = [("mom", ctypes.c_void_p), ("mom_bits", ctypes.c_int32), ("exp_mom", ctypes.c_int32),
+                ("exp_mom_next", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 class KahanSgdError(RuntimeError):
@@ -74,6 +80,20 @@ def _load() -> ctypes.CDLL:
     lib.kahan_sgd_step_static.argtypes = [P(ksgd_tensor_desc), ctypes.c_int32, ctypes.c_int,
                                           P(ctypes.c_void_p), P(ctypes.c_float)] + \
         [ctypes.c_void_p] * 7 + [ctypes.c_void_p]
+    lib.kahan_sgd_momentum_workspace_bytes.restype = ctypes.c_size_t
+    lib.kahan_sgd_momentum_workspace_bytes.argtypes = [P(ksgd_tensor_desc), P(ksgd_momentum_desc),
+                                                       ctypes.c_int32]
+    lib.kahan_sgd_momentum_init.restype = ctypes.c_int
+    lib.kahan_sgd_momentum_init.argtypes = [P(ctypes.c_void_p), P(ksgd_tensor_desc), P(ksgd_momentum_desc),
+                                            ctypes.c_int32, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t,
+                                            ctypes.c_void_p]
+    lib.kahan_sgd_momentum_step.restype = ctypes.c_int
+    lib.kahan_sgd_momentum_step.argtypes = [ctypes.c_void_p, P(ctypes.c_void_p), P(ctypes.c_float),
+                                            P(ctypes.c_float)]
+    lib.kahan_sgd_momentum_amax.restype = ctypes.c_int
+    lib.kahan_sgd_momentum_amax.argtypes = [ctypes.c_void_p] + [ctypes.c_void_p] * 11
+    lib.kahan_sgd_momentum_destroy.restype = ctypes.c_int
+    lib.kahan_sgd_momentum_destroy.argtypes = [ctypes.c_void_p]
     lib.kahan_sgd_destroy.restype = ctypes.c_int
     lib.kahan_sgd_destroy.argtypes = [ctypes.c_void_p]
     lib.kahan_sgd_strerror.restype = ctypes.c_char_p
@@ -202,6 +222,56 @@ def kahan_sgd_step_static(descs, mode: int, grads, lrs, stream: int = 0) -> dict
 
 def kahan_sgd_destroy(h) -> None:
     _check(lib.kahan_sgd_destroy(h))
+
+
+def make_momentum_descs(tensors: Sequence[dict]):
+    """ctypes array of ksgd_momentum_desc from dicts with keys mom, mom_bits, exp_mom
+    (and optionally exp_mom_next)."""
+    arr = (ksgd_momentum_desc * len(tensors))()
+    for d, t in zip(arr, tensors):
+        d.mom = t["mom"]
+        d.mom_bits = t["mom_bits"]
+        d.exp_mom = t["exp_mom"]
+        d.exp_mom_next = t.get("exp_mom_next", t["exp_mom"])
+        d.reserved = 0
+    return arr
+
+
+def kahan_sgd_momentum_workspace_bytes(descs, mdescs) -> int:
+    return int(lib.kahan_sgd_momentum_workspace_bytes(descs, mdescs, len(descs)))
+
+
+def kahan_sgd_momentum_init(descs, mdescs, mode: int, workspace: int, workspace_bytes: int,
+                            stream: int = 0):
+    h = ctypes.c_void_p()
+    _check(lib.kahan_sgd_momentum_init(ctypes.byref(h), descs, mdescs, len(descs), mode,
+                                       ctypes.c_void_p(workspace), workspace_bytes,
+                                       ctypes.c_void_p(stream)))
+    return h
+
+
+def kahan_sgd_momentum_step(h, grads, lrs, mus) -> None:
+    g = grads if isinstance(grads, ctypes.Array) else _ptr_array(grads)
+    l = lrs if isinstance(lrs, ctypes.Array) else _float_array(lrs)
+    m = mus if isinstance(mus, ctypes.Array) else _float_array(mus)
+    _check(lib.kahan_sgd_momentum_step(h, g, l, m))
+
+
+def kahan_sgd_momentum_amax(h, n_tensors: int) -> dict:
+    u32 = lambda: (ctypes.c_uint32 * n_tensors)()   # noqa: E731
+    i32 = lambda: (ctypes.c_int32 * n_tensors)()    # noqa: E731
+    u64 = lambda: (ctypes.c_uint64 * n_tensors)()   # noqa: E731
+    a_t, a_c, a_v, e_c, e_n, ev_c, ev_n = u32(), u32(), u32(), i32(), i32(), i32(), i32()
+    s_t, s_c, s_v, nf = u64(), u64(), u64(), u64()
+    _check(lib.kahan_sgd_momentum_amax(h, a_t, a_c, a_v, e_c, e_n, ev_c, ev_n, s_t, s_c, s_v, nf))
+    return {"amax_theta": list(a_t), "amax_comp": list(a_c), "amax_mom": list(a_v),
+            "exp_theta_cur": list(e_c), "exp_theta_next": list(e_n), "exp_mom_cur": list(ev_c),
+            "exp_mom_next": list(ev_n), "n_sat_theta": list(s_t), "n_sat_comp": list(s_c),
+            "n_sat_mom": list(s_v), "n_nonfinite": list(nf)}
+
+
+def kahan_sgd_momentum_destroy(h) -> None:
+    _check(lib.kahan_sgd_momentum_destroy(h))
 
 
 def kahan_sgd_strerror(code: int) -> str:

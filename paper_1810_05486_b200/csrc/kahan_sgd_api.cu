@@ -12,6 +12,7 @@
 #include <vector>
 
 #include "kahan_sgd_kernels.cuh"
+#include "kahan_sgd_momentum_kernels.cuh"
 
 namespace {
 
@@ -504,6 +505,225 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   return KSGD_OK;
 }
 
+// ----------------------------------------------------------------------------------------
+// Momentum optimizer with the lazy update.
+
+namespace {
+
+struct MomLayout {
+  size_t exp_cur, exp_next, expv_cur, expv_next, amax_last, counters, error, stats_end;
+  size_t amax_acc, info, chunks, ticket, total;
+  long long n_chunks;
+};
+
+MomLayout make_mom_layout(const ksgd_tensor_desc* d, int32_t n) {
+  MomLayout L{};
+  long long chunks = 0;
+  for (int32_t i = 0; i < n; ++i) chunks += (d[i].numel + kChunk - 1) / kChunk;
+  L.n_chunks = chunks;
+  size_t o = 0;
+  L.exp_cur = o;   o += sizeof(int) * n;
+  L.exp_next = o;  o += sizeof(int) * n;
+  L.expv_cur = o;  o += sizeof(int) * n;
+  L.expv_next = o; o += sizeof(int) * n;
+  L.amax_last = o; o += sizeof(unsigned int) * 3 * n;
+  o = align_up(o, 8);
+  L.counters = o;  o += sizeof(unsigned long long) * 4 * n;
+  L.error = o;     o += 8;
+  L.stats_end = o;
+  L.amax_acc = o;  o += sizeof(unsigned int) * 3 * n;
+  o = align_up(o, 16);
+  L.info = o;      o += sizeof(mom::TensorInfo) * n;
+  o = align_up(o, 16);
+  L.chunks = o;    o += sizeof(ChunkRef) * (size_t)chunks;
+  o = align_up(o, 16);
+  L.ticket = o;    o += 16;
+  L.total = align_up(o, 256);
+  return L;
+}
+
+int validate_momentum(const ksgd_tensor_desc* d, const ksgd_momentum_desc* m, int32_t n) {
+  const int v = validate(d, n);
+  if (v != KSGD_OK) return v;
+  if (!m) return KSGD_ERR_NULL;
+  if (n > kInlineArgs) return KSGD_ERR_NUMEL;
+  for (int32_t i = 0; i < n; ++i) {
+    if (d[i].comp_bits == 0) return KSGD_ERR_BITS;        // momentum goes through the lazy update
+    if (m[i].mom_bits != 8 && m[i].mom_bits != 16) return KSGD_ERR_BITS;
+    if (!m[i].mom) return KSGD_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(m[i].mom) % 16) return KSGD_ERR_ALIGN;
+    if (m[i].exp_mom < kExpMin || m[i].exp_mom > kExpMax) return KSGD_ERR_EXP_RANGE;
+    if (m[i].exp_mom_next < kExpMin || m[i].exp_mom_next > kExpMax) return KSGD_ERR_EXP_RANGE;
+    if (std::abs(m[i].exp_mom_next - m[i].exp_mom) > kMaxDelta) return KSGD_ERR_EXP_RANGE;
+  }
+  return KSGD_OK;
+}
+
+}  // namespace
+
+struct ksgd_momentum_handle {
+  MomLayout layout;
+  mom::StepParams params;
+  char* ws_base;
+  cudaStream_t stream;
+  int32_t n;
+  int grid;
+  std::vector<unsigned char> stats_host;
+};
+
+size_t kahan_sgd_momentum_workspace_bytes(const ksgd_tensor_desc* descs, const ksgd_momentum_desc* mdescs,
+                                          int32_t n_tensors) {
+  if (validate_momentum(descs, mdescs, n_tensors) != KSGD_OK) return 0;
+  return make_mom_layout(descs, n_tensors).total;
+}
+
+int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* descs,
+                            const ksgd_momentum_desc* mdescs, int32_t n_tensors, ksgd_exp_mode mode,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!out) return KSGD_ERR_NULL;
+  *out = nullptr;
+  const int v = validate_momentum(descs, mdescs, n_tensors);
+  if (v != KSGD_OK) return v;
+  if (mode != KSGD_EXP_FIXED && mode != KSGD_EXP_AMAX) return KSGD_ERR_MODE;
+  if (!workspace) return KSGD_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(workspace) % 256) return KSGD_ERR_ALIGN;
+  const MomLayout L = make_mom_layout(descs, n_tensors);
+  if (workspace_bytes < L.total) return KSGD_ERR_WORKSPACE;
+
+  ksgd_momentum_handle* h = new (std::nothrow) ksgd_momentum_handle();
+  if (!h) return KSGD_ERR_NULL;
+  h->layout = L;
+  h->n = n_tensors;
+  h->ws_base = static_cast<char*>(workspace);
+  h->stream = static_cast<cudaStream_t>(cuda_stream);
+  h->stats_host.resize(L.stats_end);
+
+  std::vector<unsigned char> img(L.total, 0);
+  int* e_cur = reinterpret_cast<int*>(img.data() + L.exp_cur);
+  int* e_next = reinterpret_cast<int*>(img.data() + L.exp_next);
+  int* ev_cur = reinterpret_cast<int*>(img.data() + L.expv_cur);
+  int* ev_next = reinterpret_cast<int*>(img.data() + L.expv_next);
+  mom::TensorInfo* info = reinterpret_cast<mom::TensorInfo*>(img.data() + L.info);
+  ChunkRef* chunks = reinterpret_cast<ChunkRef*>(img.data() + L.chunks);
+  long long c = 0;
+  double state_bytes = 0.0;
+  for (int32_t i = 0; i < n_tensors; ++i) {
+    const ksgd_tensor_desc& t = descs[i];
+    e_cur[i] = t.exp_theta;
+    e_next[i] = t.exp_theta_next;
+    ev_cur[i] = mdescs[i].exp_mom;
+    ev_next[i] = mdescs[i].exp_mom_next;
+    info[i].theta = t.theta;
+    info[i].comp = t.comp;
+    info[i].mom = mdescs[i].mom;
+    info[i].numel = t.numel;
+    info[i].theta_bits = t.theta_bits;
+    info[i].comp_bits = t.comp_bits;
+    info[i].mom_bits = mdescs[i].mom_bits;
+    info[i].s = t.comp_bits - 1 - t.overlap_k;
+    const long long nc = (t.numel + kChunk - 1) / kChunk;
+    for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
+    state_bytes += (double)t.numel * ((t.theta_bits + t.comp_bits + mdescs[i].mom_bits) / 8);
+  }
+
+  mom::Workspace& w = h->params.ws;
+  char* b = h->ws_base;
+  w.exp_cur = reinterpret_cast<int*>(b + L.exp_cur);
+  w.exp_next = reinterpret_cast<int*>(b + L.exp_next);
+  w.expv_cur = reinterpret_cast<int*>(b + L.expv_cur);
+  w.expv_next = reinterpret_cast<int*>(b + L.expv_next);
+  w.amax_last = reinterpret_cast<unsigned int*>(b + L.amax_last);
+  w.counters = reinterpret_cast<unsigned long long*>(b + L.counters);
+  w.error = reinterpret_cast<unsigned int*>(b + L.error);
+  w.amax_acc = reinterpret_cast<unsigned int*>(b + L.amax_acc);
+  w.info = reinterpret_cast<mom::TensorInfo*>(b + L.info);
+  w.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
+  w.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
+  h->params.n_tensors = n_tensors;
+  h->params.n_chunks = (int)L.n_chunks;
+  h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
+
+  int dev = 0, sms = 0, l2_bytes = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, dev);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(mom::ksgd_momentum_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)mom::kSharedBytes);
+  if (e != cudaSuccess) {
+    delete h;
+    return cuda_fail(e, "device query");
+  }
+  h->grid = (int)(L.n_chunks < (long long)sms ? L.n_chunks : (long long)sms);
+  h->params.grad_evict_first = state_bytes <= 0.8 * (double)l2_bytes ? 1 : 0;
+
+  e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+  if (e != cudaSuccess) {
+    delete h;
+    return cuda_fail(e, "workspace upload");
+  }
+  *out = h;
+  return KSGD_OK;
+}
+
+int kahan_sgd_momentum_step(ksgd_momentum_handle* h, const float* const* grads, const float* lrs,
+                            const float* mus) {
+  if (!h || !grads || !lrs || !mus) return KSGD_ERR_NULL;
+  mom::StepArgs args;
+  for (int32_t i = 0; i < h->n; ++i) {
+    if (!grads[i]) return KSGD_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(grads[i]) % 16) return KSGD_ERR_ALIGN;
+    if (!std::isfinite(lrs[i]) || !(lrs[i] > 0.0f)) return KSGD_ERR_LR;
+    if (!std::isfinite(mus[i]) || !(mus[i] >= 0.0f)) return KSGD_ERR_LR;
+    args.grads[i] = grads[i];
+    args.lrs[i] = lrs[i];
+    args.mus[i] = mus[i];
+  }
+  for (int32_t i = h->n; i < kInlineArgs; ++i) { args.grads[i] = nullptr; args.lrs[i] = 0.0f; args.mus[i] = 0.0f; }
+  mom::ksgd_momentum_step_kernel<<<(unsigned)h->grid, kBlockThreads, mom::kSharedBytes, h->stream>>>(h->params,
+                                                                                                  args);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  KSGD_CUDA(cudaGetLastError());
+  return KSGD_OK;
+}
+
+int kahan_sgd_momentum_amax(ksgd_momentum_handle* h, uint32_t* amax_theta, uint32_t* amax_comp,
+                            uint32_t* amax_mom, int32_t* exp_theta_cur, int32_t* exp_theta_next,
+                            int32_t* exp_mom_cur, int32_t* exp_mom_next, uint64_t* n_sat_theta,
+                            uint64_t* n_sat_comp, uint64_t* n_sat_mom, uint64_t* n_nonfinite) {
+  if (!h) return KSGD_ERR_NULL;
+  const MomLayout& L = h->layout;
+  KSGD_CUDA(cudaMemcpyAsync(h->stats_host.data(), h->ws_base, L.stats_end, cudaMemcpyDeviceToHost,
+                            h->stream));
+  KSGD_CUDA(cudaStreamSynchronize(h->stream));
+  const unsigned char* b = h->stats_host.data();
+  const size_t n = (size_t)h->n;
+  if (exp_theta_cur) std::memcpy(exp_theta_cur, b + L.exp_cur, 4 * n);
+  if (exp_theta_next) std::memcpy(exp_theta_next, b + L.exp_next, 4 * n);
+  if (exp_mom_cur) std::memcpy(exp_mom_cur, b + L.expv_cur, 4 * n);
+  if (exp_mom_next) std::memcpy(exp_mom_next, b + L.expv_next, 4 * n);
+  if (amax_theta) std::memcpy(amax_theta, b + L.amax_last, 4 * n);
+  if (amax_comp) std::memcpy(amax_comp, b + L.amax_last + 4 * n, 4 * n);
+  if (amax_mom) std::memcpy(amax_mom, b + L.amax_last + 8 * n, 4 * n);
+  if (n_sat_theta) std::memcpy(n_sat_theta, b + L.counters, 8 * n);
+  if (n_sat_comp) std::memcpy(n_sat_comp, b + L.counters + 8 * n, 8 * n);
+  if (n_sat_mom) std::memcpy(n_sat_mom, b + L.counters + 16 * n, 8 * n);
+  if (n_nonfinite) std::memcpy(n_nonfinite, b + L.counters + 24 * n, 8 * n);
+  unsigned int dev_err = 0;
+  std::memcpy(&dev_err, b + L.error, 4);
+  if (dev_err != 0) return KSGD_ERR_DEVICE;
+  return KSGD_OK;
+}
+
+int kahan_sgd_momentum_destroy(ksgd_momentum_handle* h) {
+  if (!h) return KSGD_ERR_NULL;
+  const cudaError_t e = cudaStreamSynchronize(h->stream);
+  delete h;
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  return KSGD_OK;
+}
+
 const char* kahan_sgd_strerror(int code) {
   switch (code) {
     case KSGD_OK: return "success";
@@ -514,7 +734,7 @@ const char* kahan_sgd_strerror(int code) {
     case KSGD_ERR_NUMEL: return "numel and n_tensors must be positive (and at most 2^31-1 chunks)";
     case KSGD_ERR_ALIGN: return "device pointers must be 16-byte aligned (workspace: 256)";
     case KSGD_ERR_WORKSPACE: return "workspace or staging buffer too small";
-    case KSGD_ERR_LR: return "learning rates must be finite and > 0";
+    case KSGD_ERR_LR: return "learning rates must be finite and > 0 (momentum coefficients finite and >= 0)";
     case KSGD_ERR_CUDA: return "CUDA runtime error (see kahan_sgd_last_cuda_error)";
     case KSGD_ERR_MODE: return "unknown exponent mode";
     case KSGD_ERR_DEVICE: return "a bounded wait inside the step kernel ran out; results of that step are invalid";

@@ -1,0 +1,564 @@
+// Device code of the momentum optimizer with the lazy update (Section 4 of
+// arXiv 1810.05486: Algorithm 1 "implemented in the optimizers", momentum mu = 0.9 kept
+// in INT8 or INT16).  Per element
+//     v <- mu*v + eta*g          velocity, a third dynamic fixed-point tensor
+//     theta <- theta - v         through Algorithm 1, with v in the place of eta*g
+// and three max scans per tensor (|P|, |Rq|, |V|) that steer the exponents of theta and of
+// the velocity independently.
+//
+// Same structure as ksgd_step_kernel (persistent blocks, one producer thread streaming
+// tiles into a paged shared-memory ring with bulk asynchronous copies, sixteen consumer
+// warps, producer-side publishing of the scans, exponent choice in the last block), with a
+// fourth array per tile.  HBM traffic: 2*m/8 + 2*n/8 + 2*b/8 + 4 bytes per parameter.
+#pragma once
+
+#include "kahan_sgd_kernels.cuh"
+
+namespace ksgd {
+namespace mom {
+
+struct TensorInfo {
+  void* theta;
+  void* comp;
+  void* mom;
+  long long numel;
+  int theta_bits;
+  int comp_bits;
+  int mom_bits;
+  int s;       // grid distance: exp_comp = exp_theta - s
+};
+
+struct Workspace {
+  int* exp_cur;                    // [n]  theta
+  int* exp_next;                   // [n]
+  int* expv_cur;                   // [n]  velocity
+  int* expv_next;                  // [n]
+  unsigned int* amax_last;         // [3n] theta | comp | mom, of the last finished step
+  unsigned long long* counters;    // [4n] sat_theta | sat_comp | sat_mom | nonfinite
+  unsigned int* error;             // [1]
+  unsigned int* amax_acc;          // [3n]
+  TensorInfo* info;                // [n]
+  ChunkRef* chunks;                // [n_chunks]
+  unsigned int* ticket;
+};
+
+struct StepParams {
+  Workspace ws;
+  int n_tensors;
+  int n_chunks;
+  int amax_mode;
+  int grad_evict_first;
+};
+
+struct StepArgs {                  // per-step arguments, passed as a kernel parameter
+  const float* grads[kInlineArgs];
+  float lrs[kInlineArgs];
+  float mus[kInlineArgs];
+};
+
+// What a tile's tensor needs for this step (general path reads all of it).
+struct Coef {
+  float scale_v;   // lr * 2^-ev_out: gradient -> velocity LSBs of the output grid
+  float mu_s;      // mu * 2^(ev_in - ev_out)
+  int k;           // ev_out - ec_out: velocity LSB -> compensation LSBs (a shift, either way)
+  int s;
+  int delta;       // e_out - e_in (theta)
+  int delta_v;     // ev_out - ev_in
+  int sh_t, sh_c, sh_d, r_t, r_c;
+  int qmax_t, qmax_c, qmax_v;
+};
+
+struct __align__(16) TileDesc {
+  // steady path: four 16-byte loads
+  float scale_v, mu_s, pow2k, pow2s_neg;
+  float inv2s, qmax_t, qmax_v, d_limit;   // d_limit: bound on |V| that keeps |V * 2^k| <= 4e6
+  void* theta;
+  void* comp;
+  void* mom;
+  int n_bulk;
+  int flags;
+  // the rest
+  int tensor;
+  int count;
+  Coef coef;
+  const float* grad;
+};
+constexpr int kFormatMask = 7;       // bit 0: theta 16, bit 1: comp 16, bit 2: mom 16
+constexpr int kSteady = 8;
+constexpr int kThetaPageShift = 8, kCompPageShift = 13, kGradPageShift = 18, kMomPageShift = 23;
+
+struct TileScan {
+  unsigned int amax_t, amax_c, amax_v, n_sat_t, n_sat_c, n_sat_v, n_nonfinite, pad;
+};
+
+__device__ __forceinline__ Coef make_coef(const TensorInfo& ti, int e_in, int e_out, int ev_in, int ev_out,
+                                          float lr, float mu) {
+  Coef k;
+  const int delta = e_out - e_in;
+  k.s = ti.s;
+  k.delta = delta;
+  k.delta_v = ev_out - ev_in;
+  k.sh_t = ti.s + max(0, -delta);
+  k.sh_c = max(0, -delta);
+  k.sh_d = max(0, delta);
+  k.r_t = ti.s + max(0, delta);
+  k.r_c = max(0, delta);
+  k.qmax_t = (1 << (ti.theta_bits - 1)) - 1;
+  k.qmax_c = (1 << (ti.comp_bits - 1)) - 1;
+  k.qmax_v = (1 << (ti.mom_bits - 1)) - 1;
+  k.k = ev_out - (e_out - ti.s);
+  k.scale_v = __fmul_rn(lr, pow2_float(-ev_out));
+  k.mu_s = __fmul_rn(mu, pow2_float(ev_in - ev_out));
+  return k;
+}
+
+__device__ __forceinline__ int load_q(const void* p, int bits, int e) {
+  return bits == 8 ? (int)static_cast<const signed char*>(p)[e] : (int)static_cast<const short*>(p)[e];
+}
+__device__ __forceinline__ void store_q(void* p, int bits, int e, long long v) {
+  if (bits == 8) static_cast<signed char*>(p)[e] = (signed char)v;
+  else static_cast<short*>(p)[e] = (short)v;
+}
+__device__ __forceinline__ long long clamp_ll(long long x, long long q) {
+  return x > q ? q : (x < -q ? -q : x);
+}
+
+// Elements [first, first+n) with 64-bit integers, in place on arrays in the ring or in
+// global memory: exponent changes of theta or of the velocity, vectors that left the
+// steady path, ragged tails.  Out of line, one copy for all formats.
+__device__ __noinline__ void update_general(const Coef* coef, int tb, int cb, int vb, void* theta, void* comp,
+                                            void* momv, const float* grad, int first, int n,
+                                            TileScan* scan) {
+  const Coef k = *coef;
+  unsigned int amax_t = 0, amax_c = 0, amax_v = 0, n_sat_t = 0, n_sat_c = 0, n_sat_v = 0, n_nf = 0;
+#pragma unroll 1
+  for (int e = first; e < first + n; ++e) {
+    const int qt = load_q(theta, tb, e), qc = load_q(comp, cb, e), qv = load_q(momv, vb, e);
+    const float g = grad[e];
+    // velocity: y = fma(mu_s, Qv, fl32(g * scale_v)), V = rne(y)
+    const float y = __fmaf_rn(k.mu_s, (float)qv, __fmul_rn(g, k.scale_v));
+    int V = __float2int_rn(y);                       // saturates, NaN -> 0
+    V = max(min(V, kDLimit), -kDLimit);
+    const long long Vc = clamp_ll(V, k.qmax_v);
+    amax_v = max(amax_v, (unsigned int)(V < 0 ? -V : V));
+    n_sat_v += (Vc != V);
+    store_q(momv, vb, e, Vc);
+    // the stored velocity on the compensation grid
+    long long d;
+    if (k.k >= 0) d = k.k > 40 ? (Vc > 0 ? kDLimit : (Vc < 0 ? -kDLimit : 0)) : clamp_ll(Vc * (1LL << k.k), kDLimit);
+    else d = -k.k > 40 ? 0 : rne_shift64(Vc, -k.k);
+    // Algorithm 1, statements 1-4
+    const long long T = (long long)qt * (1LL << k.sh_t) + (long long)qc * (1LL << k.sh_c) - d * (1LL << k.sh_d);
+    const long long P = rne_shift64(T, k.r_t);
+    const long long Pc = clamp_ll(P, k.qmax_t);
+    amax_t = max(amax_t, (unsigned int)(unsigned long long)(P < 0 ? -P : P));
+    n_sat_t += (P != Pc);
+    store_q(theta, tb, e, Pc);
+    const long long R = T - Pc * (1LL << k.r_t);
+    const long long Rq = rne_shift64(R, k.r_c);
+    const long long Rc = clamp_ll(Rq, k.qmax_c);
+    unsigned long long aR = (unsigned long long)(Rq < 0 ? -Rq : Rq);
+    if (aR > 0x7fffffffULL) aR = 0x7fffffffULL;
+    amax_c = max(amax_c, (unsigned int)aR);
+    n_sat_c += (Rq != Rc);
+    store_q(comp, cb, e, Rc);
+    n_nf += ((__float_as_uint(g) & 0x7f800000u) == 0x7f800000u);
+  }
+  if (amax_t) atomicMax(&scan->amax_t, amax_t);
+  if (amax_c) atomicMax(&scan->amax_c, amax_c);
+  if (amax_v) atomicMax(&scan->amax_v, amax_v);
+  if (n_sat_t) atomicAdd(&scan->n_sat_t, n_sat_t);
+  if (n_sat_c) atomicAdd(&scan->n_sat_c, n_sat_c);
+  if (n_sat_v) atomicAdd(&scan->n_sat_v, n_sat_v);
+  if (n_nf) atomicAdd(&scan->n_nonfinite, n_nf);
+}
+
+struct SteadyCoef {
+  float scale_v, mu_s, pow2k, pow2s_neg, inv2s, qmax_t, qmax_v, d_limit;
+};
+
+// Steady state (no exponent change of theta or of the velocity): eight elements on the FP32
+// pipe used as an exact integer unit (see update_vector of the plain step for the
+// technique).  With M = 1.5 * 2^23:
+//   y  = fma(mu_s, Qv, fl32(g*scale_v))      the velocity, as defined (two roundings)
+//   Vm = y + M = M + rne(y) = M + V          |y| <= 4e6
+//   dm = fma(V, 2^k, M) = M + d              exact product for k >= 0, rne for k < 0
+//   u  = Qc - d,  Pm = fma(u, 2^-s, M + Qt), w = Pm - (M + Qt), r0 = fma(w, -2^s, u)
+// theta', c' and v' are the low bits of Pm, r0 + M and Vm.  Returns false, nothing stored,
+// if a value could leave the exact range or a clamp is needed.
+template <int TB, int CB, int VB>
+__device__ __forceinline__ bool update_vector(Pack<TB> pt, Pack<CB> pc, Pack<VB> pv, const Pack<32>& pg,
+                                              const SteadyCoef& k, Pack<TB>& ot, Pack<CB>& oc, Pack<VB>& ov,
+                                              float& amax_t, float& amax_c, float& amax_v) {
+  constexpr int V = 8;
+  constexpr float bias_t = (float)(1 << (TB - 1)), bias_c = (float)(1 << (CB - 1)),
+                  bias_v = (float)(1 << (VB - 1));
+  flip_signs<TB>(pt);
+  flip_signs<CB>(pc);
+  flip_signs<VB>(pv);
+  float Pm[V], rm[V], Vm[V];
+  float sum_abs = 0.0f, aY = 0.0f, aP = 0.0f, aR = 0.0f, aV = 0.0f;
+#pragma unroll
+  for (int i = 0; i < V; ++i) {
+    const float qtM = __fadd_rn(magic_elem<TB>(pt, i), -bias_t);                  // M + Qt
+    const float qc = __fadd_rn(magic_elem<CB>(pc, i), -(kMagic + bias_c));        // Qc
+    const float qv = __fadd_rn(magic_elem<VB>(pv, i), -(kMagic + bias_v));        // Qv
+    const float g = __uint_as_float(pack_word(pg, i));
+    const float y = __fmaf_rn(k.mu_s, qv, __fmul_rn(g, k.scale_v));
+    sum_abs = __fadd_rn(sum_abs, fabsf(y));             // Inf or NaN if any y is
+    aY = fmaxf(aY, fabsf(y));
+    const float vm = __fadd_rn(y, kMagic);              // M + rne(y)
+    const float v = __fadd_rn(vm, -kMagic);
+    const float d = __fadd_rn(__fmaf_rn(v, k.pow2k, kMagic), -kMagic);
+    const float u = __fadd_rn(qc, -d);
+    const float P = __fmaf_rn(u, k.inv2s, qtM);
+    const float w = __fadd_rn(P, -qtM);
+    const float r0 = __fmaf_rn(w, k.pow2s_neg, u);
+    Pm[i] = P;
+    rm[i] = __fadd_rn(r0, kMagic);
+    Vm[i] = vm;
+    aP = fmaxf(aP, fabsf(__fadd_rn(P, -kMagic)));
+    aR = fmaxf(aR, fabsf(r0));
+    aV = fmaxf(aV, fabsf(v));
+  }
+  if (!(sum_abs < 3.0e38f) | (aY > 4000000.0f) | (aV > k.qmax_v) | (aV > k.d_limit) | (aP > k.qmax_t))
+    return false;
+  amax_t = fmaxf(amax_t, aP);
+  amax_c = fmaxf(amax_c, aR);
+  amax_v = fmaxf(amax_v, aV);
+  ot = pack_magic<TB, V>(Pm);
+  oc = pack_magic<CB, V>(rm);
+  ov = pack_magic<VB, V>(Vm);
+  return true;
+}
+
+// All vectors of one tile that belong to this consumer thread (8 consecutive elements per
+// vector; with V = 8 a vector of B-bit mantissas is B bytes).  Returns true if the general
+// path wrote into the ring.
+template <int TB, int CB, int VB>
+__device__ __forceinline__ bool consume_tile(const TileDesc* td, unsigned char* ring, int ctid, TileScan* scan,
+                                             float& amax_t, float& amax_c, float& amax_v) {
+  constexpr int V = 8;
+  const uint4* q = reinterpret_cast<const uint4*>(td);
+  const uint4 q0 = q[0], q1 = q[1], q2 = q[2], q3 = q[3];
+  SteadyCoef k;
+  k.scale_v = __uint_as_float(q0.x);
+  k.mu_s = __uint_as_float(q0.y);
+  k.pow2k = __uint_as_float(q0.z);
+  k.pow2s_neg = __uint_as_float(q0.w);
+  k.inv2s = __uint_as_float(q1.x);
+  k.qmax_t = __uint_as_float(q1.y);
+  k.qmax_v = __uint_as_float(q1.z);
+  k.d_limit = __uint_as_float(q1.w);
+  unsigned char* theta_g = reinterpret_cast<unsigned char*>(((unsigned long long)q2.y << 32) | q2.x);
+  unsigned char* comp_g = reinterpret_cast<unsigned char*>(((unsigned long long)q2.w << 32) | q2.z);
+  unsigned char* mom_g = reinterpret_cast<unsigned char*>(((unsigned long long)q3.y << 32) | q3.x);
+  const int n_bulk = (int)q3.z, flags = (int)q3.w;
+  unsigned char* theta_s = ring + ((flags >> kThetaPageShift) & 31) * kPageBytes;
+  unsigned char* comp_s = ring + ((flags >> kCompPageShift) & 31) * kPageBytes;
+  unsigned char* mom_s = ring + ((flags >> kMomPageShift) & 31) * kPageBytes;
+  const float* grad_s = reinterpret_cast<const float*>(ring + ((flags >> kGradPageShift) & 31) * kPageBytes);
+  const bool steady = (flags & kSteady) != 0;
+  bool wrote_ring = false;
+  const int n_vec = n_bulk / V;
+  for (int v = ctid; v < n_vec; v += kConsumers) {
+    Pack<TB> ot;
+    Pack<CB> oc;
+    Pack<VB> ov;
+    bool done = false;
+    if (steady) {
+      const Pack<TB> pt = load_pack<TB>(theta_s + v * TB);
+      const Pack<CB> pc = load_pack<CB>(comp_s + v * CB);
+      const Pack<VB> pv = load_pack<VB>(mom_s + v * VB);
+      const Pack<32> pg = load_pack<32>(grad_s + v * V);
+      done = update_vector<TB, CB, VB>(pt, pc, pv, pg, k, ot, oc, ov, amax_t, amax_c, amax_v);
+    }
+    if (!done) {
+      update_general(&td->coef, TB, CB, VB, theta_s, comp_s, mom_s, grad_s, v * V, V, scan);
+      ot = load_pack<TB>(theta_s + v * TB);
+      oc = load_pack<CB>(comp_s + v * CB);
+      ov = load_pack<VB>(mom_s + v * VB);
+      wrote_ring = true;
+    }
+    store_pack<TB>(theta_g + (size_t)v * TB, ot);
+    store_pack<CB>(comp_g + (size_t)v * CB, oc);
+    store_pack<VB>(mom_g + (size_t)v * VB, ov);
+  }
+  // ragged tail (fewer than 16 elements) that the bulk copies did not bring
+  const int e = n_bulk + ctid;
+  if (e < td->count) update_general(&td->coef, TB, CB, VB, theta_g, comp_g, mom_g, td->grad, e, 1, scan);
+  return wrote_ring;
+}
+
+struct __align__(128) BlockShared {
+  unsigned long long full[kSlots];
+  unsigned long long empty[kSlots];
+  TileDesc desc[kSlots];
+  TileScan scan[kSlots];
+  int slot_pages[kSlots];
+  int abort_flag;
+  int is_last;
+  int never;
+};
+
+constexpr size_t kSharedBytes = (size_t)kPages * kPageBytes + sizeof(BlockShared);
+
+struct ScanAcc {
+  int tensor = -1;
+  unsigned int amax_t = 0, amax_c = 0, amax_v = 0, n_sat_t = 0, n_sat_c = 0, n_sat_v = 0, n_nonfinite = 0;
+};
+
+__device__ __forceinline__ void publish(const StepParams& p, ScanAcc& acc) {
+  if (acc.tensor >= 0) {
+    const int t = acc.tensor, n = p.n_tensors;
+    if (acc.amax_t) atomicMax(&p.ws.amax_acc[t], acc.amax_t);
+    if (acc.amax_c) atomicMax(&p.ws.amax_acc[n + t], acc.amax_c);
+    if (acc.amax_v) atomicMax(&p.ws.amax_acc[2 * n + t], acc.amax_v);
+    if (acc.n_sat_t) atomicAdd(&p.ws.counters[t], (unsigned long long)acc.n_sat_t);
+    if (acc.n_sat_c) atomicAdd(&p.ws.counters[n + t], (unsigned long long)acc.n_sat_c);
+    if (acc.n_sat_v) atomicAdd(&p.ws.counters[2 * n + t], (unsigned long long)acc.n_sat_v);
+    if (acc.n_nonfinite) atomicAdd(&p.ws.counters[3 * n + t], (unsigned long long)acc.n_nonfinite);
+  }
+  acc = ScanAcc{};
+}
+
+__device__ __forceinline__ void take_back(const StepParams& p, ScanAcc& acc, TileScan* scan, int tensor) {
+  if (tensor != acc.tensor) {
+    publish(p, acc);
+    acc.tensor = tensor;
+  }
+  acc.amax_t = max(acc.amax_t, scan->amax_t);
+  acc.amax_c = max(acc.amax_c, scan->amax_c);
+  acc.amax_v = max(acc.amax_v, scan->amax_v);
+  acc.n_sat_t += scan->n_sat_t;
+  acc.n_sat_c += scan->n_sat_c;
+  acc.n_sat_v += scan->n_sat_v;
+  acc.n_nonfinite += scan->n_nonfinite;
+  scan->amax_t = scan->amax_c = scan->amax_v = 0u;
+  scan->n_sat_t = scan->n_sat_c = scan->n_sat_v = scan->n_nonfinite = 0u;
+}
+
+struct TensorMeta {
+  TensorInfo ti;
+  const float* grad;
+  float lr, mu;
+  int e_in, e_out, ev_in, ev_out;
+};
+
+__device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const StepArgs& a, int t) {
+  TensorMeta m;
+  m.ti = p.ws.info[t];
+  m.e_in = p.ws.exp_cur[t];
+  m.e_out = p.ws.exp_next[t];
+  m.ev_in = p.ws.expv_cur[t];
+  m.ev_out = p.ws.expv_next[t];
+  m.grad = a.grads[t];
+  m.lr = a.lrs[t];
+  m.mu = a.mus[t];
+  return m;
+}
+
+__global__ void __launch_bounds__(kBlockThreads, 1)
+ksgd_momentum_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ StepArgs a) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  BlockShared* sh = reinterpret_cast<BlockShared*>(smem + (size_t)kPages * kPageBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int stride = (int)gridDim.x;
+  const int n_my = ((int)p.n_chunks - (int)blockIdx.x + stride - 1) / stride;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kSlots; ++s) {
+      mbar_init(&sh->full[s], 1u);
+      mbar_init(&sh->empty[s], (unsigned)kConsumerWarps);
+    }
+    sh->abort_flag = 0;
+    sh->is_last = 0;
+    sh->never = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (threadIdx.x < kSlots * (int)(sizeof(TileScan) / 4))
+    reinterpret_cast<unsigned int*>(sh->scan)[threadIdx.x] = 0u;
+  __syncthreads();
+
+  if (warp == kConsumerWarps) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      const unsigned long long grad_policy = l2_policy_evict_first();
+      ScanAcc acc;
+      ChunkRef cr = p.ws.chunks[blockIdx.x];
+      TensorMeta meta = load_meta(p, a, cr.tensor);
+      ChunkRef cr1{-1, -1};
+      if (n_my > 1) cr1 = p.ws.chunks[blockIdx.x + stride];
+      int issued = 0, head = 0, free_pages = kPages, oldest = 0;
+      bool gave_up = false;
+      for (int i = 0; i < n_my; ++i) {
+        const int slot = i % kSlots;
+        ChunkRef cr2{-1, -1};
+        if (i + 2 < n_my) cr2 = p.ws.chunks[blockIdx.x + (i + 2) * stride];
+        TensorMeta meta1 = meta;
+        if (i + 1 < n_my && cr1.tensor != cr.tensor) meta1 = load_meta(p, a, cr1.tensor);
+
+        const TensorInfo& ti = meta.ti;
+        const int tbytes = ti.theta_bits >> 3, cbytes = ti.comp_bits >> 3, vbytes = ti.mom_bits >> 3;
+        const int run[4] = {kChunk * 4 / kPageBytes, kChunk * tbytes / kPageBytes,
+                            kChunk * cbytes / kPageBytes, kChunk * vbytes / kPageBytes};
+        int page[4] = {0, 0, 0, 0}, h2 = head, need = 0;
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          if (h2 + run[r] > kPages) { need += kPages - h2; h2 = 0; }
+          page[r] = h2;
+          h2 += run[r];
+          need += run[r];
+        }
+        if (h2 == kPages) h2 = 0;
+        while (free_pages < need || i - oldest >= kSlots) {
+          const int os = oldest % kSlots;
+          if (!mbar_wait(&sh->empty[os], (unsigned)(oldest / kSlots) & 1u, &sh->abort_flag)) {
+            gave_up = true;
+            break;
+          }
+          take_back(p, acc, &sh->scan[os], sh->desc[os].tensor);
+          free_pages += sh->slot_pages[os];
+          ++oldest;
+        }
+        if (gave_up) {
+          sh->abort_flag = 1;
+          atomicCAS(p.ws.error, 0u, (unsigned)kErrEmptyWait);
+          break;
+        }
+        head = h2;
+        free_pages -= need;
+        sh->slot_pages[slot] = need;
+
+        const Coef coef = make_coef(ti, meta.e_in, meta.e_out, meta.ev_in, meta.ev_out, meta.lr, meta.mu);
+        const long long first = (long long)cr.index * kChunk;
+        const long long left = ti.numel - first;
+        const int count = left < (long long)kChunk ? (int)left : kChunk;
+        const int n_bulk = count & ~15;
+        // velocity LSB -> compensation LSBs as a float factor; beyond +-30 the steady path
+        // is never exact (k large) or the increment is always zero (k very negative)
+        const int kk = max(-40, min(30, coef.k));
+        TileDesc& td = sh->desc[slot];
+        td.scale_v = coef.scale_v;
+        td.mu_s = coef.mu_s;
+        td.pow2k = pow2_float(kk);
+        td.pow2s_neg = -pow2_float(coef.s);
+        td.inv2s = pow2_float(-coef.s);
+        td.qmax_t = (float)coef.qmax_t;
+        td.qmax_v = (float)coef.qmax_v;
+        td.d_limit = coef.k > 22 ? 0.5f : (coef.k > 0 ? 4000000.0f * pow2_float(-coef.k) : 4000000.0f);
+        td.theta = static_cast<unsigned char*>(ti.theta) + first * tbytes;
+        td.comp = static_cast<unsigned char*>(ti.comp) + first * cbytes;
+        td.mom = static_cast<unsigned char*>(ti.mom) + first * vbytes;
+        td.n_bulk = n_bulk;
+        td.flags = ((ti.theta_bits == 16 ? 1 : 0) | (ti.comp_bits == 16 ? 2 : 0) | (ti.mom_bits == 16 ? 4 : 0)) |
+                   ((coef.delta == 0 && coef.delta_v == 0) ? kSteady : 0) | (page[1] << kThetaPageShift) |
+                   (page[2] << kCompPageShift) | (page[0] << kGradPageShift) | (page[3] << kMomPageShift);
+        td.tensor = cr.tensor;
+        td.count = count;
+        td.coef = coef;
+        td.grad = meta.grad + first;
+        if (n_bulk > 0) {
+          mbar_arrive_expect_tx(&sh->full[slot], (unsigned)(n_bulk * (tbytes + cbytes + vbytes + 4)));
+          bulk_load(smem + page[1] * kPageBytes, td.theta, (unsigned)(n_bulk * tbytes), &sh->full[slot]);
+          bulk_load(smem + page[2] * kPageBytes, td.comp, (unsigned)(n_bulk * cbytes), &sh->full[slot]);
+          bulk_load(smem + page[3] * kPageBytes, td.mom, (unsigned)(n_bulk * vbytes), &sh->full[slot]);
+          if (p.grad_evict_first)
+            bulk_load_hint(smem + page[0] * kPageBytes, td.grad, (unsigned)(n_bulk * 4), &sh->full[slot],
+                           grad_policy);
+          else
+            bulk_load(smem + page[0] * kPageBytes, td.grad, (unsigned)(n_bulk * 4), &sh->full[slot]);
+        } else {
+          mbar_arrive(&sh->full[slot]);
+        }
+        issued = i + 1;
+        cr = cr1;
+        cr1 = cr2;
+        meta = meta1;
+      }
+      for (int i = oldest; i < issued; ++i) {
+        const int os = i % kSlots;
+        if (mbar_wait(&sh->empty[os], (unsigned)(i / kSlots) & 1u, &sh->abort_flag))
+          take_back(p, acc, &sh->scan[os], sh->desc[os].tensor);
+        else
+          mbar_wait(&sh->full[os], (unsigned)(i / kSlots) & 1u, &sh->never);
+      }
+      publish(p, acc);
+    }
+  } else {
+    // ------------------------------------------------------------------ consumers
+    const int ctid = threadIdx.x;
+    float amax_t = 0.0f, amax_c = 0.0f, amax_v = 0.0f;
+    for (int i = 0; i < n_my; ++i) {
+      const int slot = i % kSlots, use = i / kSlots;
+      if (!mbar_wait(&sh->full[slot], (unsigned)use & 1u, &sh->abort_flag)) {
+        if (lane == 0) {
+          sh->abort_flag = 1;
+          atomicCAS(p.ws.error, 0u, (unsigned)kErrFullWait);
+        }
+        break;
+      }
+      const TileDesc* td = &sh->desc[slot];
+      TileScan* scan = &sh->scan[slot];
+      bool wrote_ring;
+      switch (td->flags & kFormatMask) {
+        case 0: wrote_ring = consume_tile<8, 8, 8>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+        case 1: wrote_ring = consume_tile<16, 8, 8>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+        case 2: wrote_ring = consume_tile<8, 16, 8>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+        case 3: wrote_ring = consume_tile<16, 16, 8>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+        case 4: wrote_ring = consume_tile<8, 8, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+        case 5: wrote_ring = consume_tile<16, 8, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+        case 6: wrote_ring = consume_tile<8, 16, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+        default: wrote_ring = consume_tile<16, 16, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+      }
+      {
+        __syncwarp();
+        const unsigned int full = 0xffffffffu;
+        const unsigned int at = __reduce_max_sync(full, (unsigned int)amax_t);
+        const unsigned int ac = __reduce_max_sync(full, (unsigned int)amax_c);
+        const unsigned int av = __reduce_max_sync(full, (unsigned int)amax_v);
+        amax_t = amax_c = amax_v = 0.0f;
+        if (lane == 0) {
+          if (at) atomicMax(&scan->amax_t, at);
+          if (ac) atomicMax(&scan->amax_c, ac);
+          if (av) atomicMax(&scan->amax_v, av);
+        }
+      }
+      if (wrote_ring) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->empty[slot]);
+    }
+  }
+
+  // ---------------------------------------------------------------------- block done
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned int done = atomicAdd(p.ws.ticket, 1u);
+    sh->is_last = (done == gridDim.x - 1u);
+  }
+  __syncthreads();
+  if (!sh->is_last) return;
+
+  // Last block: rotate and choose the exponents of theta and of the velocity.
+  __threadfence();
+  const int n = p.n_tensors;
+  for (int i = threadIdx.x; i < n; i += kBlockThreads) {
+    const unsigned int at = __ldcg(&p.ws.amax_acc[i]);
+    const unsigned int ac = __ldcg(&p.ws.amax_acc[n + i]);
+    const unsigned int av = __ldcg(&p.ws.amax_acc[2 * n + i]);
+    const int eo = p.ws.exp_next[i], evo = p.ws.expv_next[i];
+    p.ws.exp_cur[i] = eo;
+    p.ws.exp_next[i] = next_exponent(at, p.ws.info[i].theta_bits, eo, p.amax_mode);
+    p.ws.expv_cur[i] = evo;
+    p.ws.expv_next[i] = next_exponent(av, p.ws.info[i].mom_bits, evo, p.amax_mode);
+    p.ws.amax_last[i] = at;
+    p.ws.amax_last[n + i] = ac;
+    p.ws.amax_last[2 * n + i] = av;
+    p.ws.amax_acc[i] = p.ws.amax_acc[n + i] = p.ws.amax_acc[2 * n + i] = 0u;
+  }
+  if (threadIdx.x == 0) *p.ws.ticket = 0u;
+}
+
+}  // namespace mom
+}  // namespace ksgd

@@ -103,3 +103,26 @@ def test_null_handles_and_strerror(B):
     assert len(seen) == 12 and "unknown error code" not in seen
     assert B.kahan_sgd_strerror(-99) == "unknown error code"
     assert B.kahan_sgd_launch_count() == 0          # nothing was launched by these checks
+
+
+def test_momentum_init_rejects_bad_descriptions_without_cuda(B):
+    assert ctypes.sizeof(B.ksgd_momentum_desc) == 24
+    ok_m = dict(mom=0x30000, mom_bits=8, exp_mom=-14)
+    cases = [((good(), dict(ok_m, mom_bits=4)), B.KSGD_ERR_BITS),
+             ((good(comp_bits=0, comp=0), ok_m), B.KSGD_ERR_BITS),      # momentum needs the lazy update
+             ((good(), dict(ok_m, mom=0)), B.KSGD_ERR_NULL),
+             ((good(), dict(ok_m, mom=0x30004)), B.KSGD_ERR_ALIGN),
+             ((good(), dict(ok_m, exp_mom=70)), B.KSGD_ERR_EXP_RANGE),
+             ((good(), dict(ok_m, exp_mom=0, exp_mom_next=-9)), B.KSGD_ERR_EXP_RANGE)]
+    for (d, m), code in cases:
+        descs, mdescs = B.make_descs([d]), B.make_momentum_descs([m])
+        assert B.kahan_sgd_momentum_workspace_bytes(descs, mdescs) == 0
+        with pytest.raises(B.KahanSgdError) as ei:
+            B.kahan_sgd_momentum_init(descs, mdescs, B.KSGD_EXP_AMAX, 0x100000, 1 << 20)
+        assert ei.value.code == code
+    many = [good()] * 257
+    assert B.kahan_sgd_momentum_workspace_bytes(B.make_descs(many), B.make_momentum_descs([ok_m] * 257)) == 0
+    assert B.kahan_sgd_momentum_workspace_bytes(B.make_descs([good()]), B.make_momentum_descs([ok_m])) > 0
+    assert B.lib.kahan_sgd_momentum_step(None, None, None, None) == B.KSGD_ERR_NULL
+    assert B.lib.kahan_sgd_momentum_amax(None, *([None] * 11)) == B.KSGD_ERR_NULL
+    assert B.lib.kahan_sgd_momentum_destroy(None) == B.KSGD_ERR_NULL

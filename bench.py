@@ -84,6 +84,8 @@ def parse_args():
     ap.add_argument("--sweep-total", type=int, default=0,
                     help="with --workload c5_sweep: scaled-down total parameter count (profiling)")
     ap.add_argument("--sweep-tensors", type=int, default=0)
+    ap.add_argument("--momentum-bits", type=int, default=0, choices=[0, 8, 16],
+                    help="8 or 16: time the momentum optimizer (mu 0.9) with a velocity tensor of that width")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -189,7 +191,9 @@ def run_ours(args, rank, world, local_rank):
     t0 = time.time()
     host = HostInputs(wl, multi.rank_seed(args.seed, rank), n_sets, pinned=True)
     gen_s = time.time() - t0
-    run = DeviceRun(host, B.KSGD_EXP_AMAX)
+    run = DeviceRun(host, B.KSGD_EXP_AMAX, mom_bits=args.momentum_bits)
+    if args.momentum_bits:
+        args.no_e2e = args.no_cpu_baseline = True      # those legs describe the plain step
     stream = run.stream
 
     def barrier():
@@ -252,21 +256,24 @@ def run_ours(args, rank, world, local_rank):
         return
 
     peak, peak_src = hbm_peak()
-    achieved = wl.bytes_per_step / (ms_step * 1e-3) / 1e9
-    traffic = recorded_traffic(wl)
+    achieved = run.bytes_per_step / (ms_step * 1e-3) / 1e9
+    traffic = None if args.momentum_bits else recorded_traffic(wl)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": wl.name, "tensors": n, "parameters": wl.numel,
-                   "bytes_per_step": wl.bytes_per_step, "grad_sets": n_sets,
+                   "bytes_per_step": run.bytes_per_step, "grad_sets": n_sets,
+                   "optimizer": "momentum 0.9, int%d velocity" % args.momentum_bits if args.momentum_bits
+                   else "sgd",
                    "l2": "inputs larger than L2 (%.0f MB touched per step)" % (wl.bytes_per_step / 1e6),
                    "exponent_mode": "amax", "input_generation_s": round(gen_s, 1)},
         "achieved_hbm_gbs": achieved,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                      "frac_of_nominal_8000": achieved / 8000.0,
-                     "kernel": "ksgd_step_kernel", "launch_ms": ms_step},
+                     "kernel": "ksgd_momentum_step_kernel" if args.momentum_bits else "ksgd_step_kernel",
+                     "launch_ms": ms_step},
         "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
         "counters": {"n_sat_theta": int(sum(stats["n_sat_theta"])),
                      "n_sat_comp": int(sum(stats["n_sat_comp"])),

@@ -192,8 +192,10 @@ int kahan_sgd_destroy(ksgd_handle* h);
  * formulas for it; the form implemented is
  *     v <- mu*v + eta*g ,   theta <- theta - v   (the subtraction through Algorithm 1)
  * with the velocity v a third dynamic fixed-point tensor: mom_bits-bit mantissas with their
- * own shared exponent, which follows the max scan of |V| exactly as theta's exponent
- * follows |P| (one step of delay, at most 8 binades per step, [-64, 64]).  Per element:
+ * own shared exponent, which follows the max scan of |V| like theta's exponent follows
+ * |P| (one step of delay, at most 8 binades per step, [-64, 64]) but with a dead band: it
+ * is kept while the largest velocity mantissa stays in (QMAX/4, QMAX] and otherwise takes
+ * the tight fit, because the velocity's maximum moves with every gradient.  Per element:
  *     y  = fma32(fl32(mu * 2^(ev_in - ev_out)), Q_v, fl32(g * fl32(eta * 2^-ev_out)))
  *     V  = clamp(rne(y), +-2^30), NaN -> 0 ;   Q_v' = clamp(V, +-(2^(mom_bits-1) - 1))
  *     d  = Q_v' * 2^k if k >= 0 (clamped to +-2^30), rne(Q_v' / 2^-k) otherwise,

@@ -11,6 +11,7 @@ from .kahan_oracle import (  # noqa: F401
     oracle_increment,
     oracle_rne_shift,
     oracle_next_exponent,
+    oracle_next_exponent_velocity,
     oracle_step_tensor,
     oracle_step,
     OracleMomElem,

@@ -376,6 +376,22 @@ int ksgd_oracle_momentum_step_tensor(void* theta, void* comp, void* mom, const f
   return 0;
 }
 
+/*
+ * Exponent of the velocity for the next step.  The velocity's maximum moves with every
+ * gradient, so the tight fit used for theta would change the exponent back and forth from
+ * step to step; the velocity therefore keeps its exponent while its largest mantissa stays
+ * in (QMAX/4, QMAX]: coarser at once when amax > QMAX (as for theta), finer only when
+ * 4*amax <= QMAX, and then by the tight fit.  Same limits (8 binades per step, [-64, 64]).
+ */
+int32_t ksgd_oracle_next_exponent_velocity(uint32_t amax_mom, int32_t mom_bits, int32_t ev_out,
+                                           int32_t amax_mode) {
+  if (!amax_mode || amax_mom == 0) return ev_out;
+  int64_t A = (int64_t)amax_mom;
+  int64_t Q = qmax_bits(mom_bits);
+  if (A <= Q && 4 * A > Q) return ev_out;
+  return ksgd_oracle_next_exponent(amax_mom, mom_bits, ev_out, amax_mode);
+}
+
 int32_t ksgd_oracle_max_threads(void) {
 #ifdef _OPENMP
   return (int32_t)omp_get_max_threads();

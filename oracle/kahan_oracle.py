@@ -67,6 +67,9 @@ def _load():
         lib.ksgd_oracle_momentum_step_tensor.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int64] + \
             [ctypes.c_int32] * 8 + [ctypes.c_float, ctypes.c_float, ctypes.POINTER(_MomStats),
                                     ctypes.c_int32]
+        lib.ksgd_oracle_next_exponent_velocity.restype = ctypes.c_int32
+        lib.ksgd_oracle_next_exponent_velocity.argtypes = [ctypes.c_uint32, ctypes.c_int32,
+                                                           ctypes.c_int32, ctypes.c_int32]
         lib.ksgd_oracle_max_threads.restype = ctypes.c_int32
         lib.ksgd_oracle_max_threads.argtypes = []
         _lib = lib
@@ -99,6 +102,11 @@ def oracle_element(q_theta: int, q_comp: int, g: float, lr: float, m: int, n: in
 def oracle_next_exponent(amax_theta: int, theta_bits: int, e_out: int, mode: int) -> int:
     """Exponent of the next step from this step's max |P| (max scan)."""
     return int(_load().ksgd_oracle_next_exponent(amax_theta, theta_bits, e_out, mode))
+
+
+def oracle_next_exponent_velocity(amax_mom: int, mom_bits: int, ev_out: int, mode: int) -> int:
+    """Velocity exponent of the next step: kept while the largest mantissa is in (QMAX/4, QMAX]."""
+    return int(_load().ksgd_oracle_next_exponent_velocity(amax_mom, mom_bits, ev_out, mode))
 
 
 def _storage_dtype(bits: int):
@@ -214,7 +222,7 @@ def oracle_step(state: OracleState, grads: Sequence[np.ndarray], lrs: Sequence[f
 def oracle_momentum_step(state: OracleState, grads: Sequence[np.ndarray], lrs: Sequence[float],
                          mus: Sequence[float]) -> None:
     """One momentum step of every tensor, then the exponent choices: theta's exponent
-    follows max |P|, the velocity's exponent follows max |V|, each on its own."""
+    follows max |P|, the velocity's exponent follows max |V|, each on its own (the velocity's with a dead band)."""
     assert len(grads) == len(state.tensors) == len(lrs) == len(mus)
     for t, g, lr, mu in zip(state.tensors, grads, lrs, mus):
         e_in, e_out, ev_in, ev_out = t.exp_theta, t.exp_theta_next, t.exp_mom, t.exp_mom_next
@@ -229,4 +237,4 @@ def oracle_momentum_step(state: OracleState, grads: Sequence[np.ndarray], lrs: S
         t.exp_theta = e_out
         t.exp_theta_next = oracle_next_exponent(t.amax_theta, t.theta_bits, e_out, state.mode)
         t.exp_mom = ev_out
-        t.exp_mom_next = oracle_next_exponent(t.amax_mom, t.mom_bits, ev_out, state.mode)
+        t.exp_mom_next = oracle_next_exponent_velocity(t.amax_mom, t.mom_bits, ev_out, state.mode)

@@ -290,6 +290,15 @@ __device__ __forceinline__ bool consume_tile(const TileDesc* td, unsigned char* 
   return wrote_ring;
 }
 
+// Exponent of the velocity for the next step.  The velocity's maximum moves with every
+// gradient, so it keeps its exponent while its largest mantissa stays in (QMAX/4, QMAX] and
+// otherwise takes the tight fit (coarser at once, finer only after a fourfold drop).
+__device__ __forceinline__ int next_exponent_velocity(unsigned int amax, int bits, int ev_out, int amax_mode) {
+  const unsigned int q = (1u << (bits - 1)) - 1u;
+  if (amax <= q && 4ull * amax > q) return ev_out;
+  return next_exponent(amax, bits, ev_out, amax_mode);
+}
+
 struct __align__(128) BlockShared {
   unsigned long long full[kSlots];
   unsigned long long empty[kSlots];
@@ -551,7 +560,7 @@ ksgd_momentum_step_kernel(const __grid_constant__ StepParams p, const __grid_con
     p.ws.exp_cur[i] = eo;
     p.ws.exp_next[i] = next_exponent(at, p.ws.info[i].theta_bits, eo, p.amax_mode);
     p.ws.expv_cur[i] = evo;
-    p.ws.expv_next[i] = next_exponent(av, p.ws.info[i].mom_bits, evo, p.amax_mode);
+    p.ws.expv_next[i] = next_exponent_velocity(av, p.ws.info[i].mom_bits, evo, p.amax_mode);
     p.ws.amax_last[i] = at;
     p.ws.amax_last[n + i] = ac;
     p.ws.amax_last[2 * n + i] = av;

@@ -53,7 +53,10 @@ class HostInputs:
 class DeviceRun:
     """Device buffers (same layout as HostInputs), descriptors, workspace and handle."""
 
-    def __init__(self, host: HostInputs, mode: int = B.KSGD_EXP_AMAX, stream=None):
+    def __init__(self, host: HostInputs, mode: int = B.KSGD_EXP_AMAX, stream=None,
+                 mom_bits: int = 0, mu: float = 0.9):
+        """mom_bits = 8 or 16 selects the momentum optimizer (velocity buffers start at zero,
+        on a grid 8 binades below theta's)."""
         import torch
         self.torch = torch
         self.host = host
@@ -69,20 +72,44 @@ class DeviceRun:
                  numel=t.numel, theta_bits=t.theta_bits, comp_bits=t.comp_bits,
                  overlap_k=t.overlap_k, exp_theta=t.exp_theta)
             for i, t in enumerate(wl.tensors)])
-        self.ws_bytes = B.kahan_sgd_workspace_bytes(self.descs)
-        self.workspace = torch.zeros(self.ws_bytes, dtype=torch.uint8, device="cuda")
         self.stream = stream if stream is not None else torch.cuda.Stream()
-        self.handle = B.kahan_sgd_init(self.descs, mode, self.workspace.data_ptr(),
-                                       self.ws_bytes, self.stream.cuda_stream)
+        self.mom_bits = mom_bits
+        if mom_bits:
+            self.v_offs, v_bytes = _carve(wl, lambda t: mom_bits // 8)
+            self.dev_v = torch.zeros(v_bytes, dtype=torch.uint8, device="cuda")
+            self.mdescs = B.make_momentum_descs([
+                dict(mom=self.dev_v.data_ptr() + self.v_offs[i], mom_bits=mom_bits,
+                     exp_mom=t.exp_theta - 8) for i, t in enumerate(wl.tensors)])
+            self.ws_bytes = B.kahan_sgd_momentum_workspace_bytes(self.descs, self.mdescs)
+            self.workspace = torch.zeros(self.ws_bytes, dtype=torch.uint8, device="cuda")
+            self.handle = B.kahan_sgd_momentum_init(self.descs, self.mdescs, mode,
+                                                    self.workspace.data_ptr(), self.ws_bytes,
+                                                    self.stream.cuda_stream)
+            self.mus = (ctypes.c_float * self.n)(*([mu] * self.n))
+        else:
+            self.ws_bytes = B.kahan_sgd_workspace_bytes(self.descs)
+            self.workspace = torch.zeros(self.ws_bytes, dtype=torch.uint8, device="cuda")
+            self.handle = B.kahan_sgd_init(self.descs, mode, self.workspace.data_ptr(),
+                                           self.ws_bytes, self.stream.cuda_stream)
         self.grad_ptr_sets = [(ctypes.c_void_p * self.n)(*[g.data_ptr() + o for o in host.g_offs])
                               for g in self.dev_g]
         self.lrs = (ctypes.c_float * self.n)(*([wl.lr] * self.n))
 
     def step(self, grad_set: int) -> None:
-        B.kahan_sgd_step(self.handle, self.grad_ptr_sets[grad_set], self.lrs)
+        if self.mom_bits:
+            B.kahan_sgd_momentum_step(self.handle, self.grad_ptr_sets[grad_set], self.lrs, self.mus)
+        else:
+            B.kahan_sgd_step(self.handle, self.grad_ptr_sets[grad_set], self.lrs)
 
     def stats(self) -> dict:
+        if self.mom_bits:
+            return B.kahan_sgd_momentum_amax(self.handle, self.n)
         return B.kahan_sgd_amax(self.handle, self.n)
+
+    @property
+    def bytes_per_step(self) -> int:
+        """Algorithmic HBM bytes of one step, velocity included."""
+        return self.wl.bytes_per_step + 2 * (self.mom_bits // 8) * self.wl.numel
 
     def theta(self, i: int) -> np.ndarray:
         t = self.wl.tensors[i]
@@ -110,5 +137,8 @@ class DeviceRun:
 
     def close(self) -> None:
         if self.handle is not None:
-            B.kahan_sgd_destroy(self.handle)
+            if self.mom_bits:
+                B.kahan_sgd_momentum_destroy(self.handle)
+            else:
+                B.kahan_sgd_destroy(self.handle)
             self.handle = None

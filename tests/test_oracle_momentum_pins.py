@@ -6,7 +6,8 @@ from fractions import Fraction
 import numpy as np
 import pytest
 
-from oracle import (oracle_momentum_element, oracle_momentum_step_tensor, oracle_step_tensor)
+from oracle import (EXP_AMAX, EXP_FIXED, oracle_momentum_element, oracle_momentum_step_tensor,
+                    oracle_next_exponent_velocity, oracle_step_tensor)
 
 
 def qmax(b):
@@ -174,3 +175,37 @@ def test_threads_do_not_change_momentum_results():
                                              0.9, n_threads=nt)
         outs.append((theta, comp, mom, st))
     assert all(np.array_equal(a, b) for a, b in zip(outs[0][:3], outs[1][:3])) and outs[0][3] == outs[1][3]
+
+
+@pytest.mark.parametrize("bits", [8, 16])
+def test_velocity_exponent_has_a_dead_band(bits):
+    """The velocity keeps its exponent while its largest mantissa is in (QMAX/4, QMAX]; outside
+    it moves to the tight fit, so afterwards the largest mantissa is in (QMAX/2, QMAX]."""
+    Q = qmax(bits)
+    for A in list(range(1, 5 * Q)) + [2 ** 20, 2 ** 24 + 1]:
+        e = oracle_next_exponent_velocity(A, bits, 0, EXP_AMAX)
+        if 4 * A > Q and A <= Q:
+            assert e == 0, A
+        elif -8 < e < 8:
+            top = Fraction(A) / Fraction(2) ** e
+            assert top <= Q and 2 * top > Q, (A, e)
+            assert e != 0
+        elif e == 8:
+            assert Fraction(A, 2 ** 7) > Q
+        else:
+            assert A * 2 ** 8 <= Q or A * 2 ** 7 <= Q
+    assert oracle_next_exponent_velocity(0, bits, 3, EXP_AMAX) == 3
+    assert oracle_next_exponent_velocity(10 * Q, bits, 3, EXP_FIXED) == 3
+    assert oracle_next_exponent_velocity(10 * Q, bits, 63, EXP_AMAX) == 64
+    assert oracle_next_exponent_velocity(1, bits, -63, EXP_AMAX) == -64
+    # a maximum that wanders by less than a factor of two settles after at most two moves
+    # (one to the tight fit, one back if it landed just under QMAX)
+    e, moves = 0, 0
+    rng = np.random.default_rng(bits)
+    base = 0.3 * Q
+    for _ in range(400):
+        A = int(base * rng.uniform(0.75, 1.45) / 2.0 ** e)
+        e2 = oracle_next_exponent_velocity(A, bits, e, EXP_AMAX)
+        moves += e2 != e
+        e = e2
+    assert moves <= 2

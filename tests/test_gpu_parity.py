@@ -331,3 +331,50 @@ def test_step_host_matches_device_step():
             assert np.array_equal(th_h[i], t.theta) and np.array_equal(c_h[i], t.comp)
     assert_same_state(gpu, ost, "host step")
     gpu.close()
+
+
+def test_tensor_with_more_than_2_31_elements_sampled():
+    """One int8/int8 tensor of 2^31 + 12345 elements (element and byte offsets beyond 32 bits),
+    fixed exponent so that every slice can be checked on its own: slices at the start, across
+    the 2^31 and 2^32-byte marks of the gradient, and the ragged end are compared with the
+    oracle; a guard band behind each array must stay untouched."""
+    import torch
+    from oracle import oracle_step_tensor
+    from paper_1810_05486_b200 import binding as B
+    free, _ = torch.cuda.mem_get_info()
+    if free < 20 << 30:
+        pytest.skip("needs 20 GB of free device memory")
+    n = 2 ** 31 + 12345
+    guard = 4096
+    gen = torch.Generator(device="cuda").manual_seed(1234)
+    theta = torch.empty(n + guard, dtype=torch.int8, device="cuda")
+    comp = torch.empty(n + guard, dtype=torch.int8, device="cuda")
+    grad = torch.empty(n + guard, dtype=torch.float32, device="cuda")
+    step = 1 << 28
+    for lo in range(0, n, step):                      # inputs come from torch's generator, in pieces
+        hi = min(n, lo + step)
+        theta[lo:hi] = torch.randint(-127, 128, (hi - lo,), generator=gen, device="cuda", dtype=torch.int8)
+        comp[lo:hi] = torch.randint(-64, 65, (hi - lo,), generator=gen, device="cuda", dtype=torch.int8)
+        grad[lo:hi] = torch.randn(hi - lo, generator=gen, device="cuda") * (2.0 ** -18 * 40)
+    theta[n:] = 0x5A
+    comp[n:] = 0x5A
+    grad[n:] = 7.0
+    windows = [(0, 70000), (2 ** 30 - 5000, 2 ** 30 + 5000), (2 ** 31 - 9000, 2 ** 31 + 9000), (n - 20000, n)]
+    before = [(theta[a:b].cpu().numpy().copy(), comp[a:b].cpu().numpy().copy(), grad[a:b].cpu().numpy().copy())
+              for a, b in windows]
+    descs = B.make_descs([dict(theta=theta.data_ptr(), comp=comp.data_ptr(), numel=n, theta_bits=8,
+                               comp_bits=8, exp_theta=-11)])
+    nb = B.kahan_sgd_workspace_bytes(descs)
+    ws = torch.zeros(nb, dtype=torch.uint8, device="cuda")
+    h = B.kahan_sgd_init(descs, B.KSGD_EXP_FIXED, ws.data_ptr(), nb, torch.cuda.current_stream().cuda_stream)
+    B.kahan_sgd_step(h, [grad.data_ptr()], [1.0])
+    st = B.kahan_sgd_amax(h, 1)
+    B.kahan_sgd_destroy(h)
+    worst = 0
+    for (a, b), (t0, c0, g0) in zip(windows, before):
+        res = oracle_step_tensor(t0, c0, g0, 8, 8, 0, -11, -11, 1.0)
+        assert np.array_equal(theta[a:b].cpu().numpy(), t0), (a, b)
+        assert np.array_equal(comp[a:b].cpu().numpy(), c0), (a, b)
+        worst = max(worst, res["amax_theta"])
+    assert st["amax_theta"][0] >= worst and st["exp_theta_cur"][0] == -11
+    assert bool((theta[n:] == 0x5A).all()) and bool((comp[n:] == 0x5A).all()) and bool((grad[n:] == 7.0).all())

@@ -114,7 +114,10 @@ int kahan_sgd_step(ksgd_handle* h, const float* const* grads, const float* lrs);
  * theta, comp and gradient from host to the device buffers named in the descs (and to
  * grad_staging), runs the step, copies theta and comp back and waits.  theta_host /
  * comp_host / grads_host: host arrays of n_tensors host pointers (comp_host[t] ignored
- * when comp_bits == 0); page-locked memory makes the copies asynchronous.
+ * when comp_bits == 0); page-locked memory makes the copies asynchronous.  The list is
+ * processed as a pipeline of groups of neighbouring tensors (about 256 MB each): copies
+ * to the device, the update, and copies back overlap, on two copy streams the handle
+ * creates on first use.  The exponents of a tensor are chosen when its group is done.
  * grad_staging: device, 16-byte aligned, at least 4 * sum(round_up(numel, 4)) bytes,
  * caller-owned.
  */

@@ -101,7 +101,12 @@ struct ksgd_handle {
   cudaStream_t stream;
   int32_t n;
   int grid;
+  int sms;
   std::vector<unsigned char> stats_host;   // staging for kahan_sgd_amax
+  std::vector<long long> first_tile;       // [n+1] first tile of every tensor
+  // kahan_sgd_step_host: copy streams and events, created on first use
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+  std::vector<cudaEvent_t> events;
 };
 
 extern "C" {
@@ -153,8 +158,10 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
     info[i].s = t.comp_bits ? t.comp_bits - 1 - t.overlap_k : 0;
     info[i].pad = 0;
     const long long nc = (t.numel + kChunk - 1) / kChunk;
+    h->first_tile.push_back(c);
     for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
   }
+  h->first_tile.push_back(c);
 
   Workspace& w = h->params.ws;
   char* b = h->ws_base;
@@ -173,6 +180,10 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
   h->params.n_chunks = (int)L.n_chunks;
   h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
   h->params.inline_args = n_tensors <= kInlineArgs ? 1 : 0;
+  h->params.tile_begin = 0;
+  h->params.tile_count = (int)L.n_chunks;
+  h->params.tensor_begin = 0;
+  h->params.tensor_count = n_tensors;
 
   // Persistent grid: one block per SM (fewer if the list has fewer tiles).
   int dev = 0, sms = 0, l2_bytes = 0;
@@ -187,6 +198,7 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
     return cuda_fail(e, "device query");
   }
   h->grid = (int)(L.n_chunks < (long long)sms ? L.n_chunks : (long long)sms);
+  h->sms = sms;
   // theta and c of the whole list against the L2 size: if the state fits (with room for
   // the gradients streaming through), gradient loads are marked evict-first
   double state_bytes = 0.0;
@@ -212,6 +224,20 @@ static int check_step_args(const ksgd_handle* h, const float* const* grads, cons
     if (reinterpret_cast<uintptr_t>(grads[i]) % 16) return KSGD_ERR_ALIGN;
     if (!std::isfinite(lrs[i]) || !(lrs[i] > 0.0f)) return KSGD_ERR_LR;
   }
+  return KSGD_OK;
+}
+
+// Launch the step on tensors [t0, t1) (their tiles are contiguous in the table).
+static int launch_step_range(ksgd_handle* h, const InlineArgs* ia, int32_t t0, int32_t t1) {
+  StepParams p = h->params;
+  p.tile_begin = (int)h->first_tile[t0];
+  p.tile_count = (int)(h->first_tile[t1] - h->first_tile[t0]);
+  p.tensor_begin = t0;
+  p.tensor_count = t1 - t0;
+  const int grid = p.tile_count < h->sms ? p.tile_count : h->sms;
+  ksgd_step_kernel<<<(unsigned)grid, kBlockThreads, kSharedBytes, h->stream>>>(p, *ia);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  KSGD_CUDA(cudaGetLastError());
   return KSGD_OK;
 }
 
@@ -265,61 +291,116 @@ int kahan_sgd_step_host(ksgd_handle* h, void* const* theta_host, void* const* co
     dev_grads[i] = reinterpret_cast<const float*>(static_cast<char*>(grad_staging) + off);
     off += align_up((size_t)t.numel, 4) * sizeof(float);
   }
-  // Host -> device.  Neighbouring tensors whose host and device ranges both continue
-  // where the previous one ended travel as one copy.
+
+  // Groups of neighbouring tensors of about 256 MB each travel as a pipeline: while one
+  // group is being updated, the next one is on its way to the device and the previous
+  // one on its way back (the two copy directions run at the same time).
+  constexpr size_t kGroupBytes = 256u << 20;
+  std::vector<int32_t> group_start{0};
+  size_t acc = 0;
+  for (int32_t i = 0; i < h->n; ++i) {
+    const ksgd_tensor_desc& t = h->descs[i];
+    const size_t b = (size_t)t.numel * ((t.theta_bits + t.comp_bits) / 8 + 4);
+    if (acc > 0 && acc + b > kGroupBytes) { group_start.push_back(i); acc = 0; }
+    acc += b;
+  }
+  group_start.push_back(h->n);
+  const size_t n_groups = group_start.size() - 1;
+
+  if (!h->h2d_stream) KSGD_CUDA(cudaStreamCreateWithFlags(&h->h2d_stream, cudaStreamNonBlocking));
+  if (!h->d2h_stream) KSGD_CUDA(cudaStreamCreateWithFlags(&h->d2h_stream, cudaStreamNonBlocking));
+  while (h->events.size() < 2 * n_groups + 1) {
+    cudaEvent_t ev;
+    KSGD_CUDA(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+    h->events.push_back(ev);
+  }
+
+  // per-step arguments (device gradient addresses, learning rates)
+  static InlineArgs none{};
+  const InlineArgs* ia = &none;
+  InlineArgs inl;
+  if (h->params.inline_args) {
+    for (int32_t i = 0; i < h->n; ++i) { inl.grads[i] = dev_grads[i]; inl.lrs[i] = lrs[i]; }
+    for (int32_t i = h->n; i < kInlineArgs; ++i) { inl.grads[i] = nullptr; inl.lrs[i] = 0.0f; }
+    ia = &inl;
+  } else {
+    UploadBatch* ub = new (std::nothrow) UploadBatch;
+    if (!ub) return KSGD_ERR_NULL;
+    for (int32_t first = 0; first < h->n; first += kUploadBatch) {
+      const int count = h->n - first < kUploadBatch ? h->n - first : kUploadBatch;
+      for (int i = 0; i < count; ++i) { ub->grads[i] = dev_grads[first + i]; ub->lrs[i] = lrs[first + i]; }
+      ksgd_upload_args_kernel<<<1, 256, 0, h->stream>>>(*ub, first, count, h->params.ws.grad_ptr,
+                                                        h->params.ws.lr);
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    delete ub;
+    KSGD_CUDA(cudaGetLastError());
+  }
+
+  // Neighbouring tensors whose host and device ranges both continue where the previous
+  // one ended travel as one copy.
   struct Span { char* dst; const char* src; size_t bytes; };
-  auto flush = [&](std::vector<Span>& spans, cudaMemcpyKind kind) -> cudaError_t {
+  auto flush = [&](std::vector<Span>& spans, cudaMemcpyKind kind, cudaStream_t st) -> cudaError_t {
     size_t i = 0;
     while (i < spans.size()) {
-      Span s = spans[i++];
-      while (i < spans.size() && spans[i].dst == s.dst + s.bytes && spans[i].src == s.src + s.bytes)
-        s.bytes += spans[i++].bytes;
-      cudaError_t e = cudaMemcpyAsync(s.dst, s.src, s.bytes, kind, h->stream);
+      Span sp = spans[i++];
+      while (i < spans.size() && spans[i].dst == sp.dst + sp.bytes && spans[i].src == sp.src + sp.bytes)
+        sp.bytes += spans[i++].bytes;
+      cudaError_t e = cudaMemcpyAsync(sp.dst, sp.src, sp.bytes, kind, st);
       if (e != cudaSuccess) return e;
     }
     spans.clear();
     return cudaSuccess;
   };
+
+  // the copies must not overtake work already queued on the caller's stream
+  cudaEvent_t ev_start = h->events[2 * n_groups];
+  KSGD_CUDA(cudaEventRecord(ev_start, h->stream));
+  KSGD_CUDA(cudaStreamWaitEvent(h->h2d_stream, ev_start, 0));
+
   std::vector<Span> spans;
-  for (int32_t i = 0; i < h->n; ++i) {
-    const ksgd_tensor_desc& t = h->descs[i];
-    spans.push_back({static_cast<char*>(t.theta), static_cast<const char*>(theta_host[i]),
-                     (size_t)t.numel * (t.theta_bits / 8)});
-  }
-  KSGD_CUDA(flush(spans, cudaMemcpyHostToDevice));
-  for (int32_t i = 0; i < h->n; ++i) {
-    const ksgd_tensor_desc& t = h->descs[i];
-    if (t.comp_bits)
-      spans.push_back({static_cast<char*>(t.comp), static_cast<const char*>(comp_host[i]),
-                       (size_t)t.numel * (t.comp_bits / 8)});
-  }
-  KSGD_CUDA(flush(spans, cudaMemcpyHostToDevice));
-  for (int32_t i = 0; i < h->n; ++i) {
-    // the staging slots are padded to 16 bytes; copy the padded length when the host
-    // arrays are laid out the same way so that the copies merge, else the exact length
-    spans.push_back({const_cast<char*>(reinterpret_cast<const char*>(dev_grads[i])),
-                     reinterpret_cast<const char*>(grads_host[i]),
-                     (size_t)h->descs[i].numel * sizeof(float)});
-  }
-  KSGD_CUDA(flush(spans, cudaMemcpyHostToDevice));
+  for (size_t g = 0; g < n_groups; ++g) {
+    const int32_t t0 = group_start[g], t1 = group_start[g + 1];
+    for (int32_t i = t0; i < t1; ++i) {
+      const ksgd_tensor_desc& t = h->descs[i];
+      spans.push_back({static_cast<char*>(t.theta), static_cast<const char*>(theta_host[i]),
+                       (size_t)t.numel * (t.theta_bits / 8)});
+    }
+    KSGD_CUDA(flush(spans, cudaMemcpyHostToDevice, h->h2d_stream));
+    for (int32_t i = t0; i < t1; ++i) {
+      const ksgd_tensor_desc& t = h->descs[i];
+      if (t.comp_bits)
+        spans.push_back({static_cast<char*>(t.comp), static_cast<const char*>(comp_host[i]),
+                         (size_t)t.numel * (t.comp_bits / 8)});
+    }
+    KSGD_CUDA(flush(spans, cudaMemcpyHostToDevice, h->h2d_stream));
+    for (int32_t i = t0; i < t1; ++i)
+      spans.push_back({const_cast<char*>(reinterpret_cast<const char*>(dev_grads[i])),
+                       reinterpret_cast<const char*>(grads_host[i]), (size_t)h->descs[i].numel * sizeof(float)});
+    KSGD_CUDA(flush(spans, cudaMemcpyHostToDevice, h->h2d_stream));
+    KSGD_CUDA(cudaEventRecord(h->events[2 * g], h->h2d_stream));
 
-  const int r = launch_step(h, dev_grads.data(), lrs);
-  if (r != KSGD_OK) return r;
+    KSGD_CUDA(cudaStreamWaitEvent(h->stream, h->events[2 * g], 0));
+    const int r = launch_step_range(h, ia, t0, t1);
+    if (r != KSGD_OK) return r;
+    KSGD_CUDA(cudaEventRecord(h->events[2 * g + 1], h->stream));
 
-  // Device -> host: the updated mantissas.
-  for (int32_t i = 0; i < h->n; ++i) {
-    const ksgd_tensor_desc& t = h->descs[i];
-    spans.push_back({static_cast<char*>(theta_host[i]), static_cast<const char*>(t.theta),
-                     (size_t)t.numel * (t.theta_bits / 8)});
+    KSGD_CUDA(cudaStreamWaitEvent(h->d2h_stream, h->events[2 * g + 1], 0));
+    for (int32_t i = t0; i < t1; ++i) {
+      const ksgd_tensor_desc& t = h->descs[i];
+      spans.push_back({static_cast<char*>(theta_host[i]), static_cast<const char*>(t.theta),
+                       (size_t)t.numel * (t.theta_bits / 8)});
+    }
+    KSGD_CUDA(flush(spans, cudaMemcpyDeviceToHost, h->d2h_stream));
+    for (int32_t i = t0; i < t1; ++i) {
+      const ksgd_tensor_desc& t = h->descs[i];
+      if (t.comp_bits)
+        spans.push_back({static_cast<char*>(comp_host[i]), static_cast<const char*>(t.comp),
+                         (size_t)t.numel * (t.comp_bits / 8)});
+    }
+    KSGD_CUDA(flush(spans, cudaMemcpyDeviceToHost, h->d2h_stream));
   }
-  KSGD_CUDA(flush(spans, cudaMemcpyDeviceToHost));
-  for (int32_t i = 0; i < h->n; ++i) {
-    const ksgd_tensor_desc& t = h->descs[i];
-    if (t.comp_bits)
-      spans.push_back({static_cast<char*>(comp_host[i]), static_cast<const char*>(t.comp),
-                       (size_t)t.numel * (t.comp_bits / 8)});
-  }
-  KSGD_CUDA(flush(spans, cudaMemcpyDeviceToHost));
+  KSGD_CUDA(cudaStreamSynchronize(h->d2h_stream));
   KSGD_CUDA(cudaStreamSynchronize(h->stream));
   return KSGD_OK;
 }
@@ -368,6 +449,9 @@ int kahan_sgd_set_exponents(ksgd_handle* h, const int32_t* exp_theta_next) {
 int kahan_sgd_destroy(ksgd_handle* h) {
   if (!h) return KSGD_ERR_NULL;
   const cudaError_t e = cudaStreamSynchronize(h->stream);
+  for (cudaEvent_t ev : h->events) cudaEventDestroy(ev);
+  if (h->h2d_stream) cudaStreamDestroy(h->h2d_stream);
+  if (h->d2h_stream) cudaStreamDestroy(h->d2h_stream);
   delete h;
   if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
   return KSGD_OK;
@@ -475,6 +559,10 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   params.n_chunks = (int)L.n_chunks;
   params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
   params.inline_args = 1;
+  params.tile_begin = 0;
+  params.tile_count = (int)L.n_chunks;
+  params.tensor_begin = 0;
+  params.tensor_count = n_tensors;
   params.grad_evict_first = state_bytes <= 0.8 * (double)sd.l2_bytes ? 1 : 0;
   params.pad = 0;
 

@@ -81,6 +81,10 @@ struct StepParams {
   int amax_mode;     // 1: exponents follow the max scan, 0: fixed
   int inline_args;   // 1: grads/lrs are in the InlineArgs parameter
   int grad_evict_first;  // 1: gradient loads carry the L2 evict-first hint
+  // The launch covers tiles [tile_begin, tile_begin + tile_count), which are all the tiles
+  // of tensors [tensor_begin, tensor_begin + tensor_count): the whole list for an ordinary
+  // step, one group of tensors when the host-buffer entry point pipelines its copies.
+  int tile_begin, tile_count, tensor_begin, tensor_count;
   int pad;
 };
 
@@ -642,13 +646,14 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
     // the copy that refills it.
     if (lane == 0) {
       const int stride = (int)gridDim.x;
-      const int n_my = ((int)p.n_chunks - (int)blockIdx.x + stride - 1) / stride;
+      const int n_my = (p.tile_count - (int)blockIdx.x + stride - 1) / stride;
+      const int tile0 = p.tile_begin + (int)blockIdx.x;
       const unsigned long long grad_policy = l2_policy_evict_first();
       ScanAcc acc;
-      ChunkRef cr = p.ws.chunks[blockIdx.x];
+      ChunkRef cr = p.ws.chunks[tile0];
       TensorMeta meta = load_meta(p, a, cr.tensor);
       ChunkRef cr1{-1, -1};
-      if (n_my > 1) cr1 = p.ws.chunks[blockIdx.x + stride];
+      if (n_my > 1) cr1 = p.ws.chunks[tile0 + stride];
       int issued = 0;
       // The ring: pages from `head` on are free, tiles are released in the order they were
       // issued, `oldest` is the first tile whose pages have not been taken back yet.
@@ -657,7 +662,7 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
       for (int i = 0; i < n_my; ++i) {
         const int slot = i % kSlots;
         ChunkRef cr2{-1, -1};
-        if (i + 2 < n_my) cr2 = p.ws.chunks[blockIdx.x + (i + 2) * stride];
+        if (i + 2 < n_my) cr2 = p.ws.chunks[tile0 + (i + 2) * stride];
         TensorMeta meta1 = meta;
         if (i + 1 < n_my && cr1.tensor != cr.tensor) meta1 = load_meta(p, a, cr1.tensor);
 
@@ -751,7 +756,7 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
     // ------------------------------------------------------------------ consumers
     const int ctid = threadIdx.x;
     const int stride = (int)gridDim.x;
-    const int n_my = ((int)p.n_chunks - (int)blockIdx.x + stride - 1) / stride;
+    const int n_my = (p.tile_count - (int)blockIdx.x + stride - 1) / stride;
     float amax_t = 0.0f, amax_c = 0.0f;
     for (int i = 0; i < n_my; ++i) {
       const int stage = i % kSlots, use = i / kSlots;
@@ -811,7 +816,7 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
   // Last block to finish: every other block has published its scans and has long since
   // read the exponents, so they can be rotated here.  No block ever waits for another.
   __threadfence();
-  for (int i = threadIdx.x; i < p.n_tensors; i += kBlockThreads) {
+  for (int i = p.tensor_begin + threadIdx.x; i < p.tensor_begin + p.tensor_count; i += kBlockThreads) {
     const unsigned int at = __ldcg(&p.ws.amax_acc[i]);
     const unsigned int ac = __ldcg(&p.ws.amax_acc[p.n_tensors + i]);
     const int eo = p.ws.exp_next[i];

@@ -110,3 +110,32 @@ def test_c5_full_size_sampled_tensors():
             assert 0 < st["amax_theta"][i]
     finally:
         run.close()
+
+
+def test_c4_through_host_buffers_in_several_groups():
+    """kahan_sgd_step_host on a list large enough to travel as several pipelined groups of
+    tensors: host buffers in, host buffers out, two steps, everything bit-exact."""
+    import torch
+    from paper_1810_05486_b200.runner import DeviceRun, HostInputs
+    wl = W.workload("c4_alexnet")
+    host = HostInputs(wl, seed=0, n_sets=2, pinned=True)
+    ost = OracleState([OracleTensor(host.thetas[i].copy(), host.comps[i].copy(), t.theta_bits, t.comp_bits, 0,
+                                    t.exp_theta, t.exp_theta) for i, t in enumerate(wl.tensors)],
+                      EXP_AMAX, n_threads=oracle_max_threads())
+    run = DeviceRun(host)
+    run.dev_th.zero_()          # the device copies must come from the host buffers
+    run.dev_c.zero_()
+    th, c, g = run.host_pointer_arrays()
+    try:
+        for step in range(2):
+            run.step_host(th, c, g[step])
+            oracle_step(ost, [x.copy() for x in host.grads[step]], [wl.lr] * len(wl.tensors))
+            st = run.stats()
+            for i, t in enumerate(ost.tensors):
+                assert np.array_equal(host.thetas[i], t.theta), (step, i)
+                assert np.array_equal(host.comps[i], t.comp), (step, i)
+                assert (st["exp_theta_cur"][i], st["exp_theta_next"][i]) == (t.exp_theta, t.exp_theta_next)
+                assert (st["amax_theta"][i], st["amax_comp"][i]) == (t.amax_theta, t.amax_comp)
+                assert (st["n_sat_theta"][i], st["n_sat_comp"][i]) == (t.n_sat_theta, t.n_sat_comp)
+    finally:
+        run.close()

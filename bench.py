@@ -43,11 +43,11 @@ GRAD_SETS = {"c5_sweep": 2, "c1_single": 100, "c2_resnet20": 200, "c3_resnet50":
 # dram__bytes_write.sum per launch, divided by the parameters of the captured launch; see
 # profiles/).  c5_sweep was captured at 2e8 parameters; traffic is proportional to the
 # parameter count, so a full launch is this figure times its parameters.  The record only
-# counts while the kernel sources still hash to the value below.
+# counts while the kernel source (kahan_sgd_kernels.cuh) still hashes to the value below.
 TRAFFIC_RECORD = {
-    "sources_sha256": "ecfe5c34de15ff9edc81ad8cb3301052ea5b9f977d2e49920a82b478c4db0b3d",
-    "dram_bytes_per_parameter": {"c5_sweep": 2356.633e6 / 2e8, "c4_alexnet": 470.829e6 / 61100840,
-                                 "c3_resnet50": 199.963e6 / 25557032},
+    "sources_sha256": "c2c9d57719edaeb49b12292faae83747c99efe64fdf8bee40e220ecdd560dbed",
+    "dram_bytes_per_parameter": {"c5_sweep": 2355.452e6 / 2e8, "c4_alexnet": 470.055e6 / 61100840,
+                                 "c3_resnet50": 199.173e6 / 25557032},
 }
 
 

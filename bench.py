@@ -88,6 +88,8 @@ def parse_args():
                     help="8 or 16: time the momentum optimizer (mu 0.9) with a velocity tensor of that width")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-buckets", action="store_true",
+                    help="skip the per-size-bucket timing of c5_sweep")
     return ap.parse_args()
 
 
@@ -247,6 +249,9 @@ def run_ours(args, rank, world, local_rank):
                "h2d_bytes_per_step": state_bytes + 4 * wl.numel,
                "d2h_bytes_per_step": state_bytes, "steps": args.e2e_steps,
                "ms_per_step": dt / args.e2e_steps * 1e3}
+    buckets = None
+    if wl.name == "c5_sweep" and rank == 0 and not args.momentum_bits and not args.no_buckets:
+        buckets = time_size_buckets(torch, B, run, wl)
     run.close()
 
     if rank != 0:
@@ -279,12 +284,50 @@ def run_ours(args, rank, world, local_rank):
                      "n_sat_comp": int(sum(stats["n_sat_comp"])),
                      "n_nonfinite": int(sum(stats["n_nonfinite"]))},
     }
+    if buckets is not None:
+        line["size_buckets"] = buckets
     if not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, host, budget_core_s=20.0)
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def time_size_buckets(torch, B, run, wl, steps=20):
+    """GB/s of the step on the sub-list of every tensor-size bucket [2^j, 2^(j+1)) of the
+    sweep, on the device buffers of the full run (each sub-list gets its own handle)."""
+    import math
+    out = []
+    by_bucket = {}
+    for i, t in enumerate(wl.tensors):
+        by_bucket.setdefault(int(math.log2(t.numel)), []).append(i)
+    for j in sorted(by_bucket):
+        idx = by_bucket[j]
+        sub = [dict(theta=run.descs[i].theta, comp=run.descs[i].comp, numel=run.descs[i].numel,
+                    theta_bits=run.descs[i].theta_bits, comp_bits=run.descs[i].comp_bits,
+                    overlap_k=run.descs[i].overlap_k, exp_theta=wl.tensors[i].exp_theta) for i in idx]
+        descs = B.make_descs(sub)
+        nb = B.kahan_sgd_workspace_bytes(descs)
+        ws = torch.zeros(nb, dtype=torch.uint8, device="cuda")
+        h = B.kahan_sgd_init(descs, B.KSGD_EXP_AMAX, ws.data_ptr(), nb, run.stream.cuda_stream)
+        gp = [(ctypes.c_void_p * len(idx))(*[run.grad_ptr_sets[k][i] for i in idx]) for k in range(2)]
+        lr = (ctypes.c_float * len(idx))(*([wl.lr] * len(idx)))
+        for k in range(3):
+            B.kahan_sgd_step(h, gp[k % 2], lr)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        run.stream.synchronize()
+        ev0.record(run.stream)
+        for k in range(steps):
+            B.kahan_sgd_step(h, gp[k % 2], lr)
+        ev1.record(run.stream)
+        run.stream.synchronize()
+        ms = ev0.elapsed_time(ev1) / steps
+        B.kahan_sgd_destroy(h)
+        params = sum(wl.tensors[i].numel for i in idx)
+        out.append({"log2_size": j, "tensors": len(idx), "parameters": params,
+                    "us_per_step": round(ms * 1e3, 2), "gbs": round(params * 12 / (ms * 1e-3) / 1e9, 1)})
+    return out
 
 
 def cpu_baseline(wl, host, budget_core_s):
@@ -307,10 +350,22 @@ def cpu_baseline(wl, host, budget_core_s):
         k += 1
         if t_used * cores >= budget_core_s:
             break
+    # one thread, on the largest tensor alone (a few seconds at most)
+    i = order[0]
+    t = wl.tensors[i]
+    n1 = min(t.numel, 40_000_000)
+    th = host.thetas[i][:n1].copy()
+    c = host.comps[i][:n1].copy() if t.comp_bits else None
+    t0 = time.perf_counter()
+    oracle_step_tensor(th, c, np.ascontiguousarray(host.grads[0][i][:n1]), t.theta_bits, t.comp_bits,
+                       t.overlap_k, t.exp_theta, t.exp_theta, wl.lr, 1)
+    t1 = time.perf_counter() - t0
     return {"value": done / t_used, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": "one step of the %d largest tensors of %s (%d of %d parameters), OpenMP "
                       "static split over elements" % (k, wl.name, done, wl.numel),
-            "seconds": round(t_used, 3)}
+            "seconds": round(t_used, 3),
+            "one_thread": {"value": n1 / t1, "unit": UNIT, "cores": 1,
+                           "sample": "%d parameters of the largest tensor" % n1}}
 
 
 def run_reference(args, rank, world):

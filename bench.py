@@ -249,6 +249,24 @@ def run_ours(args, rank, world, local_rank):
                "h2d_bytes_per_step": state_bytes + 4 * wl.numel,
                "d2h_bytes_per_step": state_bytes, "steps": args.e2e_steps,
                "ms_per_step": dt / args.e2e_steps * 1e3}
+    graph_us = None
+    if wl.bytes_per_step < (64 << 20) and world == 1 and not args.momentum_bits:
+        # small lists are bound by the host's launch rate: also time the same steps recorded
+        # once into a CUDA graph and replayed (kahan_sgd_step only enqueues work)
+        with torch.cuda.stream(stream):
+            stream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                for i in range(args.steps):
+                    run.step(i % n_sets)
+            graph.replay()
+            stream.synchronize()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record(stream)
+            graph.replay()
+            g1.record(stream)
+            stream.synchronize()
+            graph_us = g0.elapsed_time(g1) * 1e3 / args.steps
     buckets = None
     if wl.name == "c5_sweep" and rank == 0 and not args.momentum_bits and not args.no_buckets:
         buckets = time_size_buckets(torch, B, run, wl)
@@ -286,6 +304,9 @@ def run_ours(args, rank, world, local_rank):
     }
     if buckets is not None:
         line["size_buckets"] = buckets
+    if graph_us is not None:
+        line["cuda_graph"] = {"us_per_step": graph_us,
+                              "note": "the same %d steps recorded once into a CUDA graph and replayed" % args.steps}
     if not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, host, budget_core_s=20.0)
     print(json.dumps(line), flush=True)

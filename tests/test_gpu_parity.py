@@ -378,3 +378,41 @@ def test_tensor_with_more_than_2_31_elements_sampled():
         worst = max(worst, res["amax_theta"])
     assert st["amax_theta"][0] >= worst and st["exp_theta_cur"][0] == -11
     assert bool((theta[n:] == 0x5A).all()) and bool((comp[n:] == 0x5A).all()) and bool((grad[n:] == 7.0).all())
+
+
+def test_steps_captured_in_a_cuda_graph_and_replayed():
+    """kahan_sgd_step only enqueues work on the handle's stream, so a sequence of steps can
+    be recorded into a CUDA graph and replayed: 4 steps per graph, 3 replays, against 12
+    oracle steps (the captured gradient buffers are refilled between replays)."""
+    import torch
+    rng = np.random.default_rng(61)
+    wl = W.workload("c2_resnet20")
+    specs = specs_of(wl)
+    thetas, comps = W.initial_state(wl)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        gpu = LibraryRun(specs, thetas, comps, EXP_AMAX, stream=side)
+        lrs = [wl.lr] * len(specs)
+        grads = [W.gradients(wl, s) for s in range(4)]
+        # four resident gradient sets, one per captured step
+        sets = []
+        for gs in grads:
+            bufs = [torch.from_numpy(g).cuda() for g in gs]
+            sets.append(bufs)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for bufs in sets:
+                gpu.B.kahan_sgd_step(gpu.handle, [b.data_ptr() for b in bufs], lrs)
+        ost = make_oracle_state(specs, thetas, comps, EXP_AMAX)
+        for replay in range(3):
+            for k, bufs in enumerate(sets):          # new gradients into the captured buffers
+                for b, g in zip(bufs, W.gradients(wl, 4 * replay + k)):
+                    b.copy_(torch.from_numpy(g))
+            torch.cuda.synchronize()
+            graph.replay()
+            torch.cuda.synchronize()
+            for k in range(4):
+                oracle_step(ost, W.gradients(wl, 4 * replay + k), lrs)
+            assert_same_state(gpu, ost, f"replay {replay}")
+        gpu.close()

@@ -197,7 +197,7 @@ __device__ __forceinline__ bool update_vector(Pack<TB> pt, Pack<CB> pc, Pack<VB>
   flip_signs<CB>(pc);
   flip_signs<VB>(pv);
   float Pm[V], rm[V], Vm[V];
-  float sum_abs = 0.0f, aY = 0.0f, aP = 0.0f, aR = 0.0f, aV = 0.0f;
+  float sum_abs = 0.0f, aP = 0.0f, aR = 0.0f, aV = 0.0f;
 #pragma unroll
   for (int i = 0; i < V; ++i) {
     const float qtM = __fadd_rn(magic_elem<TB>(pt, i), -bias_t);                  // M + Qt
@@ -206,7 +206,6 @@ __device__ __forceinline__ bool update_vector(Pack<TB> pt, Pack<CB> pc, Pack<VB>
     const float g = __uint_as_float(pack_word(pg, i));
     const float y = __fmaf_rn(k.mu_s, qv, __fmul_rn(g, k.scale_v));
     sum_abs = __fadd_rn(sum_abs, fabsf(y));             // Inf or NaN if any y is
-    aY = fmaxf(aY, fabsf(y));
     const float vm = __fadd_rn(y, kMagic);              // M + rne(y)
     const float v = __fadd_rn(vm, -kMagic);
     const float d = __fadd_rn(__fmaf_rn(v, k.pow2k, kMagic), -kMagic);
@@ -221,8 +220,9 @@ __device__ __forceinline__ bool update_vector(Pack<TB> pt, Pack<CB> pc, Pack<VB>
     aR = fmaxf(aR, fabsf(r0));
     aV = fmaxf(aV, fabsf(v));
   }
-  if (!(sum_abs < 3.0e38f) | (aY > 4000000.0f) | (aV > k.qmax_v) | (aV > k.d_limit) | (aP > k.qmax_t))
-    return false;
+  // |y| > 4e6 (where y + M stops being exact) shows as |V| far beyond QMAX_v, so the velocity
+  // bound covers it
+  if (!(sum_abs < 3.0e38f) | (aV > k.qmax_v) | (aV > k.d_limit) | (aP > k.qmax_t)) return false;
   amax_t = fmaxf(amax_t, aP);
   amax_c = fmaxf(amax_c, aR);
   amax_v = fmaxf(amax_v, aV);

@@ -14,6 +14,9 @@ from .kahan_oracle import (  # noqa: F401
     oracle_next_exponent_velocity,
     oracle_step_tensor,
     oracle_step,
+    oracle_fit_exponent,
+    oracle_quantize,
+    oracle_dequantize,
     OracleMomElem,
     oracle_momentum_element,
     oracle_momentum_step_tensor,

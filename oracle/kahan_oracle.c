@@ -392,6 +392,68 @@ int32_t ksgd_oracle_next_exponent_velocity(uint32_t amax_mom, int32_t mom_bits, 
   return ksgd_oracle_next_exponent(amax_mom, mom_bits, ev_out, amax_mode);
 }
 
+/* ------------------------------------------------------------------------------------
+ * fp32 <-> dynamic fixed-point (Section 1: uniform linear quantization with one shared
+ * exponent per tensor; Section 5: the exponent comes from a scan of the maximum).
+ *
+ * Exponent: the smallest e in [-64, 64] with max|x| <= QMAX_m * 2^e over the finite x
+ * (e = 0 for an all-zero or all-non-finite tensor).
+ * Import: Q_theta = clamp(rne(x / 2^e), +-QMAX_m); with a compensation tensor the part
+ * theta cannot hold goes there, Q_c = clamp(rne((x - Q_theta*2^e) / 2^(e-s)), +-QMAX_n),
+ * so that theta + c carries m+n-2-k bits of x.  NaN -> 0, +-Inf -> +-QMAX_m (c = 0).
+ * Export: x = fl32(Q_theta * 2^e + Q_c * 2^(e-s)), computed exactly and rounded once.
+ * All scalings are by powers of two, so double arithmetic is exact here.
+ */
+int32_t ksgd_oracle_fit_exponent(const float* x, int64_t numel, int32_t bits) {
+  double amax = 0.0;
+  for (int64_t i = 0; i < numel; ++i)
+    if (isfinite(x[i]) && fabs((double)x[i]) > amax) amax = fabs((double)x[i]);
+  if (amax == 0.0) return 0;
+  double Q = (double)qmax_bits(bits);
+  int32_t e = -64;
+  while (e < 64 && amax > ldexp(Q, e)) ++e;
+  return e;
+}
+
+void ksgd_oracle_quantize(const float* x, void* theta, void* comp, int64_t numel, int32_t theta_bits,
+                          int32_t comp_bits, int32_t overlap_k, int32_t e) {
+  int32_t s = comp_bits ? comp_bits - 1 - overlap_k : 0;
+  double Qt = (double)qmax_bits(theta_bits);
+  for (int64_t i = 0; i < numel; ++i) {
+    double v = (double)x[i];
+    int64_t qt, qc = 0;
+    if (isnan(v)) {
+      qt = 0;
+    } else if (isinf(v)) {
+      qt = v > 0 ? (int64_t)Qt : -(int64_t)Qt;
+    } else {
+      double t = nearbyint(ldexp(v, -e));          /* exact scaling, ties to even */
+      if (t > Qt) t = Qt;
+      if (t < -Qt) t = -Qt;
+      qt = (int64_t)t;
+      if (comp_bits) {
+        double Qc = (double)qmax_bits(comp_bits);
+        double r = nearbyint(ldexp(v - ldexp((double)qt, e), -(e - s)));
+        if (r > Qc) r = Qc;
+        if (r < -Qc) r = -Qc;
+        qc = (int64_t)r;
+      }
+    }
+    store_mantissa(theta, i, theta_bits, (int32_t)qt);
+    if (comp_bits) store_mantissa(comp, i, comp_bits, (int32_t)qc);
+  }
+}
+
+void ksgd_oracle_dequantize(const void* theta, const void* comp, float* x, int64_t numel,
+                            int32_t theta_bits, int32_t comp_bits, int32_t overlap_k, int32_t e) {
+  int32_t s = comp_bits ? comp_bits - 1 - overlap_k : 0;
+  for (int64_t i = 0; i < numel; ++i) {
+    double v = ldexp((double)load_mantissa(theta, i, theta_bits), e);
+    if (comp_bits) v += ldexp((double)load_mantissa(comp, i, comp_bits), e - s);
+    x[i] = (float)v;                                /* one rounding to binary32 */
+  }
+}
+
 int32_t ksgd_oracle_max_threads(void) {
 #ifdef _OPENMP
   return (int32_t)omp_get_max_threads();

@@ -70,6 +70,12 @@ def _load():
         lib.ksgd_oracle_next_exponent_velocity.restype = ctypes.c_int32
         lib.ksgd_oracle_next_exponent_velocity.argtypes = [ctypes.c_uint32, ctypes.c_int32,
                                                            ctypes.c_int32, ctypes.c_int32]
+        lib.ksgd_oracle_fit_exponent.restype = ctypes.c_int32
+        lib.ksgd_oracle_fit_exponent.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32]
+        lib.ksgd_oracle_quantize.restype = None
+        lib.ksgd_oracle_quantize.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int64] + [ctypes.c_int32] * 4
+        lib.ksgd_oracle_dequantize.restype = None
+        lib.ksgd_oracle_dequantize.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int64] + [ctypes.c_int32] * 4
         lib.ksgd_oracle_max_threads.restype = ctypes.c_int32
         lib.ksgd_oracle_max_threads.argtypes = []
         _lib = lib
@@ -107,6 +113,31 @@ def oracle_next_exponent(amax_theta: int, theta_bits: int, e_out: int, mode: int
 def oracle_next_exponent_velocity(amax_mom: int, mom_bits: int, ev_out: int, mode: int) -> int:
     """Velocity exponent of the next step: kept while the largest mantissa is in (QMAX/4, QMAX]."""
     return int(_load().ksgd_oracle_next_exponent_velocity(amax_mom, mom_bits, ev_out, mode))
+
+
+def oracle_fit_exponent(x: np.ndarray, bits: int) -> int:
+    """Smallest exponent whose b-bit grid holds max|x| (finite values only)."""
+    assert x.dtype == np.float32 and x.flags.c_contiguous
+    return int(_load().ksgd_oracle_fit_exponent(x.ctypes.data, x.size, bits))
+
+
+def oracle_quantize(x: np.ndarray, theta_bits: int, comp_bits: int, overlap_k: int, e: int):
+    """fp32 -> (theta mantissas, compensation mantissas or None) at exponent e."""
+    assert x.dtype == np.float32 and x.flags.c_contiguous
+    theta = np.empty(x.size, _storage_dtype(theta_bits))
+    comp = np.empty(x.size, _storage_dtype(comp_bits)) if comp_bits else None
+    _load().ksgd_oracle_quantize(x.ctypes.data, theta.ctypes.data, comp.ctypes.data if comp_bits else None,
+                                 x.size, theta_bits, comp_bits, overlap_k, e)
+    return theta, comp
+
+
+def oracle_dequantize(theta: np.ndarray, comp, theta_bits: int, comp_bits: int, overlap_k: int,
+                      e: int) -> np.ndarray:
+    """(theta, compensation) at exponent e -> fp32, one rounding."""
+    x = np.empty(theta.size, np.float32)
+    _load().ksgd_oracle_dequantize(theta.ctypes.data, comp.ctypes.data if comp_bits else None,
+                                   x.ctypes.data, theta.size, theta_bits, comp_bits, overlap_k, e)
+    return x
 
 
 def _storage_dtype(bits: int):

@@ -234,6 +234,37 @@ int kahan_sgd_momentum_amax(ksgd_momentum_handle* h, uint32_t* amax_theta, uint3
                             uint64_t* n_sat_comp, uint64_t* n_sat_mom, uint64_t* n_nonfinite);
 int kahan_sgd_momentum_destroy(ksgd_momentum_handle* h);
 
+/*
+ * fp32 -> dynamic fixed-point (Section 1: uniform linear quantization, one shared exponent
+ * per tensor; Section 5: the exponent from a scan of the maximum).  src: device,
+ * fp32[numel].  theta / comp: device outputs in the formats of ksgd_tensor_desc (comp NULL
+ * iff comp_bits == 0).  Q_theta = clamp(rne(x / 2^e)); with a compensation tensor the part
+ * theta cannot hold goes there, Q_c = clamp(rne((x - Q_theta*2^e) / 2^(e-s))), so that an
+ * imported weight keeps m+n-2-k bits; NaN -> 0, +-Inf -> +-QMAX.  exp_theta: the exponent
+ * to use, in [-64, 64], or KSGD_EXP_AUTO for the smallest exponent whose grid holds the
+ * largest finite |x| (0 for an all-zero tensor); with KSGD_EXP_AUTO the call runs a max
+ * scan into scratch (device, at least 4 bytes, 4-byte aligned) and waits for it.
+ * *exp_theta_out (host, may be NULL) receives the exponent used.
+ */
+#define KSGD_EXP_AUTO INT32_MIN
+int kahan_sgd_import(const float* src, void* theta, void* comp, int64_t numel, int32_t theta_bits,
+                     int32_t comp_bits, int32_t overlap_k, int32_t exp_theta, int32_t* exp_theta_out,
+                     void* scratch, void* cuda_stream);
+
+/*
+ * Dynamic fixed-point -> fp32: dst[i] = fl32(Q_theta*2^e + Q_c*2^(e-s)), the exact value of
+ * theta + c rounded once.  dst: device, fp32[numel].  Enqueues only.
+ */
+int kahan_sgd_export(const void* theta, const void* comp, float* dst, int64_t numel, int32_t theta_bits,
+                     int32_t comp_bits, int32_t overlap_k, int32_t exp_theta, void* cuda_stream);
+
+/*
+ * Bit-width of the last fully-connected layer in front of a softmax (Section 3, Eq. 5):
+ * the smallest integer larger than log2(n_classes - 1) + log2(2 / alpha), 0 < alpha < 1
+ * (the paper suggests alpha = 0.5).  Host-only.  Returns 0 for invalid arguments.
+ */
+int32_t kahan_sgd_classifier_bits(int64_t n_classes, double alpha);
+
 /* Static text for a KSGD_* code. */
 const char* kahan_sgd_strerror(int code);
 

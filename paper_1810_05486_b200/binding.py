@@ -32,6 +32,7 @@ EXPORTS = (
     "kahan_sgd_amax", "kahan_sgd_set_exponents", "kahan_sgd_step_static", "kahan_sgd_destroy",
     "kahan_sgd_strerror", "kahan_sgd_momentum_workspace_bytes", "kahan_sgd_momentum_init",
     "kahan_sgd_momentum_step", "kahan_sgd_momentum_amax", "kahan_sgd_momentum_destroy",
+    "kahan_sgd_import", "kahan_sgd_export", "kahan_sgd_classifier_bits",
     "kahan_sgd_last_cuda_error", "kahan_sgd_launch_count",
 )
 
@@ -94,6 +95,14 @@ def _load() -> ctypes.CDLL:
     lib.kahan_sgd_momentum_amax.argtypes = [ctypes.c_void_p] + [ctypes.c_void_p] * 11
     lib.kahan_sgd_momentum_destroy.restype = ctypes.c_int
     lib.kahan_sgd_momentum_destroy.argtypes = [ctypes.c_void_p]
+    lib.kahan_sgd_import.restype = ctypes.c_int
+    lib.kahan_sgd_import.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int64] + [ctypes.c_int32] * 4 + \
+        [P(ctypes.c_int32), ctypes.c_void_p, ctypes.c_void_p]
+    lib.kahan_sgd_export.restype = ctypes.c_int
+    lib.kahan_sgd_export.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int64] + [ctypes.c_int32] * 4 + \
+        [ctypes.c_void_p]
+    lib.kahan_sgd_classifier_bits.restype = ctypes.c_int32
+    lib.kahan_sgd_classifier_bits.argtypes = [ctypes.c_int64, ctypes.c_double]
     lib.kahan_sgd_destroy.restype = ctypes.c_int
     lib.kahan_sgd_destroy.argtypes = [ctypes.c_void_p]
     lib.kahan_sgd_strerror.restype = ctypes.c_char_p
@@ -272,6 +281,32 @@ def kahan_sgd_momentum_amax(h, n_tensors: int) -> dict:
 
 def kahan_sgd_momentum_destroy(h) -> None:
     _check(lib.kahan_sgd_momentum_destroy(h))
+
+
+KSGD_EXP_AUTO = -(2 ** 31)
+
+
+def kahan_sgd_import(src: int, theta: int, comp, numel: int, theta_bits: int, comp_bits: int,
+                     overlap_k: int = 0, exp_theta: int = KSGD_EXP_AUTO, scratch: int = 0,
+                     stream: int = 0) -> int:
+    """fp32 -> dynamic fixed-point on the device; returns the exponent used."""
+    e = ctypes.c_int32()
+    _check(lib.kahan_sgd_import(ctypes.c_void_p(src), ctypes.c_void_p(theta), ctypes.c_void_p(comp or None),
+                                numel, theta_bits, comp_bits, overlap_k, exp_theta, ctypes.byref(e),
+                                ctypes.c_void_p(scratch or None), ctypes.c_void_p(stream)))
+    return int(e.value)
+
+
+def kahan_sgd_export(theta: int, comp, dst: int, numel: int, theta_bits: int, comp_bits: int,
+                     overlap_k: int, exp_theta: int, stream: int = 0) -> None:
+    """Dynamic fixed-point -> fp32 on the device (theta + c rounded once)."""
+    _check(lib.kahan_sgd_export(ctypes.c_void_p(theta), ctypes.c_void_p(comp or None), ctypes.c_void_p(dst),
+                                numel, theta_bits, comp_bits, overlap_k, exp_theta, ctypes.c_void_p(stream)))
+
+
+def kahan_sgd_classifier_bits(n_classes: int, alpha: float = 0.5) -> int:
+    """Eq. 5: smallest bit-width larger than log2(n_classes - 1) + log2(2 / alpha)."""
+    return int(lib.kahan_sgd_classifier_bits(n_classes, alpha))
 
 
 def kahan_sgd_strerror(code: int) -> str:

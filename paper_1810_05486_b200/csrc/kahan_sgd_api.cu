@@ -13,6 +13,7 @@
 
 #include "kahan_sgd_kernels.cuh"
 #include "kahan_sgd_momentum_kernels.cuh"
+#include "kahan_sgd_convert.cuh"
 
 namespace {
 
@@ -810,6 +811,123 @@ int kahan_sgd_momentum_destroy(ksgd_momentum_handle* h) {
   delete h;
   if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
   return KSGD_OK;
+}
+
+// ----------------------------------------------------------------------------------------
+// fp32 <-> dynamic fixed-point, and the classifier bit-width rule.
+
+}  // extern "C"
+
+namespace {
+
+int check_format(int32_t theta_bits, int32_t comp_bits, int32_t overlap_k) {
+  if (theta_bits != 8 && theta_bits != 16) return KSGD_ERR_BITS;
+  if (comp_bits != 0 && comp_bits != 8 && comp_bits != 16) return KSGD_ERR_BITS;
+  if (comp_bits != 0 && (overlap_k < 0 || overlap_k > comp_bits - 1)) return KSGD_ERR_OVERLAP;
+  return KSGD_OK;
+}
+
+int convert_grid(int64_t numel) {
+  const int64_t blocks = (numel + convert::kThreads - 1) / convert::kThreads;
+  return (int)(blocks < 148 * 16 ? blocks : 148 * 16);
+}
+
+template <typename T, typename C, bool HC>
+void launch_quantize(const float* src, void* theta, void* comp, int64_t numel, int e, int s, int tb, int cb,
+                     cudaStream_t st) {
+  convert::quantize_kernel<T, C, HC><<<convert_grid(numel), convert::kThreads, 0, st>>>(
+      src, static_cast<T*>(theta), static_cast<C*>(comp), numel, e, s, tb, cb);
+}
+
+template <typename T, typename C, bool HC>
+void launch_dequantize(const void* theta, const void* comp, float* dst, int64_t numel, int e, int s,
+                       cudaStream_t st) {
+  convert::dequantize_kernel<T, C, HC><<<convert_grid(numel), convert::kThreads, 0, st>>>(
+      static_cast<const T*>(theta), static_cast<const C*>(comp), dst, numel, e, s);
+}
+
+}  // namespace
+
+extern "C" {
+
+int kahan_sgd_import(const float* src, void* theta, void* comp, int64_t numel, int32_t theta_bits,
+                     int32_t comp_bits, int32_t overlap_k, int32_t exp_theta, int32_t* exp_theta_out,
+                     void* scratch, void* cuda_stream) {
+  const int f = check_format(theta_bits, comp_bits, overlap_k);
+  if (f != KSGD_OK) return f;
+  if (!src || !theta || (comp_bits != 0) != (comp != nullptr)) return KSGD_ERR_NULL;
+  if (numel <= 0) return KSGD_ERR_NUMEL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int e = exp_theta;
+  if (exp_theta == KSGD_EXP_AUTO) {
+    // max scan, then the smallest exponent whose grid holds the maximum
+    if (!scratch) return KSGD_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(scratch) % 4) return KSGD_ERR_ALIGN;
+    KSGD_CUDA(cudaMemsetAsync(scratch, 0, 4, st));
+    convert::absmax_kernel<<<convert_grid(numel), convert::kThreads, 0, st>>>(
+        src, numel, static_cast<unsigned int*>(scratch));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    KSGD_CUDA(cudaGetLastError());
+    unsigned int bits = 0;
+    KSGD_CUDA(cudaMemcpyAsync(&bits, scratch, 4, cudaMemcpyDeviceToHost, st));
+    KSGD_CUDA(cudaStreamSynchronize(st));
+    float amax;
+    std::memcpy(&amax, &bits, 4);
+    e = 0;
+    if (amax > 0.0f) {
+      const double q = (double)((1 << (theta_bits - 1)) - 1);
+      e = kExpMin;
+      while (e < kExpMax && (double)amax > std::ldexp(q, e)) ++e;
+    }
+  } else if (exp_theta < kExpMin || exp_theta > kExpMax) {
+    return KSGD_ERR_EXP_RANGE;
+  }
+  const int s = comp_bits ? comp_bits - 1 - overlap_k : 0;
+  if (theta_bits == 8) {
+    if (comp_bits == 8) launch_quantize<signed char, signed char, true>(src, theta, comp, numel, e, s, 8, 8, st);
+    else if (comp_bits == 16) launch_quantize<signed char, short, true>(src, theta, comp, numel, e, s, 8, 16, st);
+    else launch_quantize<signed char, signed char, false>(src, theta, comp, numel, e, s, 8, 0, st);
+  } else {
+    if (comp_bits == 8) launch_quantize<short, signed char, true>(src, theta, comp, numel, e, s, 16, 8, st);
+    else if (comp_bits == 16) launch_quantize<short, short, true>(src, theta, comp, numel, e, s, 16, 16, st);
+    else launch_quantize<short, signed char, false>(src, theta, comp, numel, e, s, 16, 0, st);
+  }
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  KSGD_CUDA(cudaGetLastError());
+  if (exp_theta_out) *exp_theta_out = e;
+  return KSGD_OK;
+}
+
+int kahan_sgd_export(const void* theta, const void* comp, float* dst, int64_t numel, int32_t theta_bits,
+                     int32_t comp_bits, int32_t overlap_k, int32_t exp_theta, void* cuda_stream) {
+  const int f = check_format(theta_bits, comp_bits, overlap_k);
+  if (f != KSGD_OK) return f;
+  if (!dst || !theta || (comp_bits != 0) != (comp != nullptr)) return KSGD_ERR_NULL;
+  if (numel <= 0) return KSGD_ERR_NUMEL;
+  if (exp_theta < kExpMin || exp_theta > kExpMax) return KSGD_ERR_EXP_RANGE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int s = comp_bits ? comp_bits - 1 - overlap_k : 0, e = exp_theta;
+  if (theta_bits == 8) {
+    if (comp_bits == 8) launch_dequantize<signed char, signed char, true>(theta, comp, dst, numel, e, s, st);
+    else if (comp_bits == 16) launch_dequantize<signed char, short, true>(theta, comp, dst, numel, e, s, st);
+    else launch_dequantize<signed char, signed char, false>(theta, comp, dst, numel, e, s, st);
+  } else {
+    if (comp_bits == 8) launch_dequantize<short, signed char, true>(theta, comp, dst, numel, e, s, st);
+    else if (comp_bits == 16) launch_dequantize<short, short, true>(theta, comp, dst, numel, e, s, st);
+    else launch_dequantize<short, signed char, false>(theta, comp, dst, numel, e, s, st);
+  }
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  KSGD_CUDA(cudaGetLastError());
+  return KSGD_OK;
+}
+
+int32_t kahan_sgd_classifier_bits(int64_t n_classes, double alpha) {
+  if (n_classes < 2 || !(alpha > 0.0) || !(alpha < 1.0)) return 0;
+  // Eq. 5: bitwidth > log2(|class| - 1) + log2(2 / alpha); the smallest integer that is
+  // strictly larger.  Evaluated on the integers: 2^(b-1) * alpha > |class| - 1.
+  for (int32_t b = 2; b <= 64; ++b)
+    if (std::ldexp(alpha, b - 1) > (double)(n_classes - 1)) return b;
+  return 64;
 }
 
 const char* kahan_sgd_strerror(int code) {

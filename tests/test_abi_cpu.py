@@ -126,3 +126,33 @@ def test_momentum_init_rejects_bad_descriptions_without_cuda(B):
     assert B.lib.kahan_sgd_momentum_step(None, None, None, None) == B.KSGD_ERR_NULL
     assert B.lib.kahan_sgd_momentum_amax(None, *([None] * 11)) == B.KSGD_ERR_NULL
     assert B.lib.kahan_sgd_momentum_destroy(None) == B.KSGD_ERR_NULL
+
+
+def test_classifier_bits_follow_eq_5_and_the_printed_example(B):
+    import math
+    rows = [ln.split() for ln in open(os.path.join(ROOT, "tests", "golden", "classifier_bitwidth.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    for classes, alpha, bound, bits in rows:
+        classes, alpha, bound, bits = int(classes), float(alpha), float(bound), int(bits)
+        assert abs(math.log2(classes - 1) + math.log2(2 / alpha) - bound) < 0.01
+        assert B.kahan_sgd_classifier_bits(classes, alpha) == bits
+    for classes in (2, 3, 5, 100, 1000, 21841):
+        for alpha in (0.5, 0.25, 0.1):
+            b = B.kahan_sgd_classifier_bits(classes, alpha)
+            real = math.log2(classes - 1) + math.log2(2 / alpha)
+            assert b > real and b - 1 <= real + 1e-12        # smallest integer strictly above
+    assert B.kahan_sgd_classifier_bits(1, 0.5) == 0 and B.kahan_sgd_classifier_bits(10, 0.0) == 0
+    assert B.kahan_sgd_classifier_bits(10, 1.0) == 0
+
+
+def test_import_export_reject_bad_arguments_without_cuda(B):
+    imp, exp = B.lib.kahan_sgd_import, B.lib.kahan_sgd_export
+    assert imp(0x1000, 0x2000, 0x3000, 10, 4, 8, 0, 0, None, None, None) == B.KSGD_ERR_BITS
+    assert imp(0x1000, 0x2000, 0x3000, 10, 8, 8, 9, 0, None, None, None) == B.KSGD_ERR_OVERLAP
+    assert imp(None, 0x2000, 0x3000, 10, 8, 8, 0, 0, None, None, None) == B.KSGD_ERR_NULL
+    assert imp(0x1000, 0x2000, None, 10, 8, 8, 0, 0, None, None, None) == B.KSGD_ERR_NULL
+    assert imp(0x1000, 0x2000, 0x3000, 0, 8, 8, 0, 0, None, None, None) == B.KSGD_ERR_NUMEL
+    assert imp(0x1000, 0x2000, 0x3000, 10, 8, 8, 0, 65, None, None, None) == B.KSGD_ERR_EXP_RANGE
+    assert imp(0x1000, 0x2000, 0x3000, 10, 8, 8, 0, B.KSGD_EXP_AUTO, None, None, None) == B.KSGD_ERR_NULL
+    assert exp(0x2000, 0x3000, None, 10, 8, 8, 0, 0, None) == B.KSGD_ERR_NULL
+    assert exp(0x2000, 0x3000, 0x1000, 10, 8, 8, 0, -70, None) == B.KSGD_ERR_EXP_RANGE

@@ -15,6 +15,10 @@ from .kahan_oracle import (  # noqa: F401
     oracle_step_tensor,
     oracle_step,
     oracle_fit_exponent,
+    OracleAdamElem,
+    oracle_adam_element,
+    oracle_adam_step_tensor,
+    oracle_adam_step,
     oracle_quantize,
     oracle_dequantize,
     OracleMomElem,

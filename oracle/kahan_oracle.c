@@ -393,6 +393,128 @@ int32_t ksgd_oracle_next_exponent_velocity(uint32_t amax_mom, int32_t mom_bits, 
 }
 
 /* ------------------------------------------------------------------------------------
+ * ADAM with the lazy update (Section 4: ADAM, beta1 = 0.9, beta2 = 0.999, needs INT16 for
+ * its moments "because of beta2").  The paper gives no formulas; the reading taken is the
+ * usual ADAM with the bias correction folded into the step size by the caller
+ * (lr_t = eta * sqrt(1 - beta2^t) / (1 - beta1^t)):
+ *     m <- beta1*m + (1-beta1)*g ,  v <- beta2*v + (1-beta2)*g^2 ,
+ *     theta <- theta - lr_t * m / (sqrt(v) + eps)      (the subtraction through Algorithm 1)
+ * with m and v two more dynamic fixed-point tensors (16-bit mantissas, own exponents).
+ * Every floating-point operation is one correctly rounded binary32 operation:
+ *   c1 = fl(1 - beta1), c2 = fl(1 - beta2)
+ *   ym = fma(fl(beta1 * 2^(em_in-em_out)), Q_m, fl(g * fl(c1 * 2^-em_out)))    M = rne(ym)
+ *   yv = fma(fl(beta2 * 2^(ev_in-ev_out)), Q_v, fl(fl(g*g) * fl(c2 * 2^-ev_out)))  V = rne(yv)
+ *   (both clamped to +-2^30, NaN -> 0, then to +-(2^15 - 1) for storage)
+ *   mr = Q_m' * 2^em_out, vr = Q_v' * 2^ev_out          exact
+ *   q  = fl(mr / fl(sqrt(vr) + eps))                    sqrt of a negative vr is taken of 0
+ *   d  = clamp(rne(fl(q * fl(lr_t * 2^-ec_out))), +-2^30), NaN -> 0
+ *   then statements 1-4 of Algorithm 1 with this d.
+ */
+typedef struct {
+  ksgd_oracle_elem upd;
+  int64_t M, V;          /* moment mantissas before saturation */
+  int32_t q_m, q_v;      /* stored moment mantissas            */
+} ksgd_oracle_adam_elem;
+
+static int32_t rne_clamped(float y) {
+  if (isnan(y)) return 0;
+  const float lim = 1073741824.0f;
+  if (y >= lim) return (int32_t)1 << 30;
+  if (y <= -lim) return -((int32_t)1 << 30);
+  return (int32_t)nearbyintf(y);
+}
+
+void ksgd_oracle_adam_element(int32_t q_theta, int32_t q_comp, int32_t q_m, int32_t q_v, float g, float lr,
+                              float beta1, float beta2, float eps, int32_t m, int32_t n, int32_t s,
+                              int32_t e_in, int32_t e_out, int32_t em_in, int32_t em_out,
+                              int32_t ev_in, int32_t ev_out, ksgd_oracle_adam_elem* out) {
+  if (n == 0) { s = 0; q_comp = 0; }
+  float c1 = 1.0f - beta1, c2 = 1.0f - beta2;
+  float ym = fmaf(ldexpf(beta1, em_in - em_out), (float)q_m, g * ldexpf(c1, -em_out));
+  float g2 = g * g;
+  float yv = fmaf(ldexpf(beta2, ev_in - ev_out), (float)q_v, g2 * ldexpf(c2, -ev_out));
+  int64_t M = rne_clamped(ym), V = rne_clamped(yv);
+  int64_t qm_new = clamp_i64(M, -32767, 32767), qv_new = clamp_i64(V, -32767, 32767);
+
+  int32_t ec_in = e_in - s, ec_out = e_out - s;
+  int32_t f = ec_in < ec_out ? ec_in : ec_out;
+  float mr = ldexpf((float)qm_new, em_out);
+  float vr = ldexpf((float)qv_new, ev_out);
+  float root = sqrtf(vr > 0.0f ? vr : 0.0f);
+  float den = root + eps;
+  float q = mr / den;
+  float x = q * ldexpf(lr, -ec_out);
+  int64_t d = rne_clamped(x);
+
+  int64_t T = (int64_t)q_theta * pow2_i64(e_in - f) + (int64_t)q_comp * pow2_i64(ec_in - f) -
+              d * pow2_i64(ec_out - f);
+  int64_t P = ksgd_oracle_rne_shift(T, e_out - f);
+  int64_t q_theta_new = clamp_i64(P, -qmax_bits(m), qmax_bits(m));
+  int64_t R = T - q_theta_new * pow2_i64(e_out - f);
+  int64_t Rq = 0, q_comp_new = 0;
+  if (n != 0) {
+    Rq = ksgd_oracle_rne_shift(R, ec_out - f);
+    q_comp_new = clamp_i64(Rq, -qmax_bits(n), qmax_bits(n));
+  }
+  out->upd.P = P; out->upd.Rq = Rq; out->upd.T = T; out->upd.d = (int32_t)d;
+  out->upd.q_theta = (int32_t)q_theta_new; out->upd.q_comp = (int32_t)q_comp_new;
+  out->upd.nonfinite = isfinite(g) ? 0 : 1;
+  out->M = M; out->V = V; out->q_m = (int32_t)qm_new; out->q_v = (int32_t)qv_new;
+}
+
+typedef struct {
+  ksgd_oracle_stats upd;
+  uint32_t amax_m, amax_v;
+  uint64_t n_sat_m, n_sat_v;
+} ksgd_oracle_adam_stats;
+
+int ksgd_oracle_adam_step_tensor(void* theta, void* comp, int16_t* mom1, int16_t* mom2, const float* grad,
+                                 int64_t numel, int32_t theta_bits, int32_t comp_bits, int32_t overlap_k,
+                                 int32_t e_in, int32_t e_out, int32_t em_in, int32_t em_out, int32_t ev_in,
+                                 int32_t ev_out, float lr, float beta1, float beta2, float eps,
+                                 ksgd_oracle_adam_stats* stats, int32_t n_threads) {
+  if (!theta || !mom1 || !mom2 || !grad || !stats || numel <= 0) return -1;
+  if (theta_bits < 2 || theta_bits > 16) return -1;
+  if (comp_bits != 0 && (comp_bits < 2 || comp_bits > 16)) return -1;
+  if (comp_bits != 0 && (!comp || overlap_k < 0 || overlap_k > comp_bits - 1)) return -1;
+  int32_t s = comp_bits == 0 ? 0 : comp_bits - 1 - overlap_k;
+  uint32_t amax_theta = 0, amax_comp = 0, amax_m = 0, amax_v = 0;
+  uint64_t n_sat_theta = 0, n_sat_comp = 0, n_nonfinite = 0, n_sat_m = 0, n_sat_v = 0;
+  if (n_threads < 1) n_threads = 1;
+#pragma omp parallel for schedule(static) num_threads(n_threads) \
+    reduction(max : amax_theta, amax_comp, amax_m, amax_v) \
+    reduction(+ : n_sat_theta, n_sat_comp, n_nonfinite, n_sat_m, n_sat_v)
+  for (int64_t i = 0; i < numel; ++i) {
+    ksgd_oracle_adam_elem r;
+    int32_t qt = load_mantissa(theta, i, theta_bits);
+    int32_t qc = comp_bits ? load_mantissa(comp, i, comp_bits) : 0;
+    ksgd_oracle_adam_element(qt, qc, mom1[i], mom2[i], grad[i], lr, beta1, beta2, eps, theta_bits,
+                             comp_bits, s, e_in, e_out, em_in, em_out, ev_in, ev_out, &r);
+    store_mantissa(theta, i, theta_bits, r.upd.q_theta);
+    if (comp_bits) store_mantissa(comp, i, comp_bits, r.upd.q_comp);
+    mom1[i] = (int16_t)r.q_m;
+    mom2[i] = (int16_t)r.q_v;
+    int64_t aP = r.upd.P < 0 ? -r.upd.P : r.upd.P, aR = r.upd.Rq < 0 ? -r.upd.Rq : r.upd.Rq;
+    int64_t aM = r.M < 0 ? -r.M : r.M, aV = r.V < 0 ? -r.V : r.V;
+    if (aR > 2147483647LL) aR = 2147483647LL;
+    if ((uint32_t)aP > amax_theta) amax_theta = (uint32_t)aP;
+    if ((uint32_t)aR > amax_comp) amax_comp = (uint32_t)aR;
+    if ((uint32_t)aM > amax_m) amax_m = (uint32_t)aM;
+    if ((uint32_t)aV > amax_v) amax_v = (uint32_t)aV;
+    n_sat_theta += (r.upd.P != r.upd.q_theta);
+    n_sat_comp += (comp_bits != 0 && r.upd.Rq != r.upd.q_comp);
+    n_sat_m += (r.M != r.q_m);
+    n_sat_v += (r.V != r.q_v);
+    n_nonfinite += (uint64_t)r.upd.nonfinite;
+  }
+  stats->upd.amax_theta = amax_theta; stats->upd.amax_comp = amax_comp;
+  stats->upd.n_sat_theta = n_sat_theta; stats->upd.n_sat_comp = n_sat_comp;
+  stats->upd.n_nonfinite = n_nonfinite;
+  stats->amax_m = amax_m; stats->amax_v = amax_v; stats->n_sat_m = n_sat_m; stats->n_sat_v = n_sat_v;
+  return 0;
+}
+
+/* ------------------------------------------------------------------------------------
  * fp32 <-> dynamic fixed-point (Section 1: uniform linear quantization with one shared
  * exponent per tensor; Section 5: the exponent comes from a scan of the maximum).
  *

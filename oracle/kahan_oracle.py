@@ -37,6 +37,16 @@ class _MomStats(ctypes.Structure):
     _fields_ = [("upd", _Stats), ("amax_mom", ctypes.c_uint32), ("n_sat_mom", ctypes.c_uint64)]
 
 
+class OracleAdamElem(ctypes.Structure):
+    _fields_ = [("upd", OracleElem), ("M", ctypes.c_int64), ("V", ctypes.c_int64),
+                ("q_m", ctypes.c_int32), ("q_v", ctypes.c_int32)]
+
+
+class _AdamStats(ctypes.Structure):
+    _fields_ = [("upd", _Stats), ("amax_m", ctypes.c_uint32), ("amax_v", ctypes.c_uint32),
+                ("n_sat_m", ctypes.c_uint64), ("n_sat_v", ctypes.c_uint64)]
+
+
 _lib = None
 
 
@@ -76,6 +86,12 @@ def _load():
         lib.ksgd_oracle_quantize.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int64] + [ctypes.c_int32] * 4
         lib.ksgd_oracle_dequantize.restype = None
         lib.ksgd_oracle_dequantize.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int64] + [ctypes.c_int32] * 4
+        lib.ksgd_oracle_adam_element.restype = None
+        lib.ksgd_oracle_adam_element.argtypes = [ctypes.c_int32] * 4 + [ctypes.c_float] * 5 + \
+            [ctypes.c_int32] * 9 + [ctypes.POINTER(OracleAdamElem)]
+        lib.ksgd_oracle_adam_step_tensor.restype = ctypes.c_int
+        lib.ksgd_oracle_adam_step_tensor.argtypes = [ctypes.c_void_p] * 5 + [ctypes.c_int64] + \
+            [ctypes.c_int32] * 9 + [ctypes.c_float] * 4 + [ctypes.POINTER(_AdamStats), ctypes.c_int32]
         lib.ksgd_oracle_max_threads.restype = ctypes.c_int32
         lib.ksgd_oracle_max_threads.argtypes = []
         _lib = lib
@@ -195,6 +211,36 @@ def oracle_momentum_step_tensor(theta, comp, mom, grad, theta_bits, comp_bits, o
             "n_nonfinite": st.upd.n_nonfinite, "amax_mom": st.amax_mom, "n_sat_mom": st.n_sat_mom}
 
 
+def oracle_adam_element(q_theta, q_comp, q_m, q_v, g, lr, beta1, beta2, eps, m, n, s, e_in, e_out,
+                        em_in, em_out, ev_in, ev_out) -> OracleAdamElem:
+    """ADAM with the lazy update for one element (16-bit moments)."""
+    out = OracleAdamElem()
+    _load().ksgd_oracle_adam_element(q_theta, q_comp, q_m, q_v, g, lr, beta1, beta2, eps, m, n, s,
+                                     e_in, e_out, em_in, em_out, ev_in, ev_out, ctypes.byref(out))
+    return out
+
+
+def oracle_adam_step_tensor(theta, comp, mom1, mom2, grad, theta_bits, comp_bits, overlap_k, e_in, e_out,
+                            em_in, em_out, ev_in, ev_out, lr, beta1, beta2, eps, n_threads: int = 1) -> dict:
+    """ADAM step over one tensor, in place on theta, comp and both moments; returns the stats."""
+    assert theta.dtype == _storage_dtype(theta_bits) and theta.flags.c_contiguous
+    for a in (mom1, mom2):
+        assert a.dtype == np.int16 and a.flags.c_contiguous and a.size == theta.size
+    assert grad.dtype == np.float32 and grad.flags.c_contiguous and grad.size == theta.size
+    st = _AdamStats()
+    rc = _load().ksgd_oracle_adam_step_tensor(
+        theta.ctypes.data, comp.ctypes.data if comp_bits else None, mom1.ctypes.data, mom2.ctypes.data,
+        grad.ctypes.data, theta.size, theta_bits, comp_bits, overlap_k, e_in, e_out, em_in, em_out,
+        ev_in, ev_out, ctypes.c_float(lr), ctypes.c_float(beta1), ctypes.c_float(beta2),
+        ctypes.c_float(eps), ctypes.byref(st), n_threads)
+    if rc != 0:
+        raise ValueError("oracle rejected the tensor description")
+    return {"amax_theta": st.upd.amax_theta, "amax_comp": st.upd.amax_comp,
+            "n_sat_theta": st.upd.n_sat_theta, "n_sat_comp": st.upd.n_sat_comp,
+            "n_nonfinite": st.upd.n_nonfinite, "amax_m": st.amax_m, "amax_v": st.amax_v,
+            "n_sat_m": st.n_sat_m, "n_sat_v": st.n_sat_v}
+
+
 @dataclass
 class OracleTensor:
     """One parameter tensor: mantissas, compensation, formats and exponents."""
@@ -217,6 +263,12 @@ class OracleTensor:
     exp_mom_next: int = 0
     amax_mom: int = 0
     n_sat_mom: int = 0
+    # ADAM only: `mom` is the first moment, `mom2` the second
+    mom2: Optional[np.ndarray] = None
+    exp_mom2: int = 0
+    exp_mom2_next: int = 0
+    amax_mom2: int = 0
+    n_sat_mom2: int = 0
 
     @property
     def s(self) -> int:
@@ -269,3 +321,29 @@ def oracle_momentum_step(state: OracleState, grads: Sequence[np.ndarray], lrs: S
         t.exp_theta_next = oracle_next_exponent(t.amax_theta, t.theta_bits, e_out, state.mode)
         t.exp_mom = ev_out
         t.exp_mom_next = oracle_next_exponent_velocity(t.amax_mom, t.mom_bits, ev_out, state.mode)
+
+
+def oracle_adam_step(state: OracleState, grads: Sequence[np.ndarray], lrs: Sequence[float], beta1: float,
+                     beta2: float, eps: float) -> None:
+    """One ADAM step of every tensor (lrs carry the bias correction), then the exponent
+    choices: theta's by the tight fit, both moments' with the dead band."""
+    assert len(grads) == len(state.tensors) == len(lrs)
+    for t, g, lr in zip(state.tensors, grads, lrs):
+        e_in, e_out = t.exp_theta, t.exp_theta_next
+        em_in, em_out, ev_in, ev_out = t.exp_mom, t.exp_mom_next, t.exp_mom2, t.exp_mom2_next
+        st = oracle_adam_step_tensor(t.theta, t.comp, t.mom, t.mom2, g, t.theta_bits, t.comp_bits,
+                                     t.overlap_k, e_in, e_out, em_in, em_out, ev_in, ev_out, float(lr),
+                                     float(beta1), float(beta2), float(eps), state.n_threads)
+        t.amax_theta, t.amax_comp = st["amax_theta"], st["amax_comp"]
+        t.amax_mom, t.amax_mom2 = st["amax_m"], st["amax_v"]
+        t.n_sat_theta += st["n_sat_theta"]
+        t.n_sat_comp += st["n_sat_comp"]
+        t.n_nonfinite += st["n_nonfinite"]
+        t.n_sat_mom += st["n_sat_m"]
+        t.n_sat_mom2 += st["n_sat_v"]
+        t.exp_theta = e_out
+        t.exp_theta_next = oracle_next_exponent(t.amax_theta, t.theta_bits, e_out, state.mode)
+        t.exp_mom = em_out
+        t.exp_mom_next = oracle_next_exponent_velocity(t.amax_mom, 16, em_out, state.mode)
+        t.exp_mom2 = ev_out
+        t.exp_mom2_next = oracle_next_exponent_velocity(t.amax_mom2, 16, ev_out, state.mode)

@@ -86,6 +86,9 @@ def parse_args():
     ap.add_argument("--sweep-tensors", type=int, default=0)
     ap.add_argument("--momentum-bits", type=int, default=0, choices=[0, 8, 16],
                     help="8 or 16: time the momentum optimizer (mu 0.9) with a velocity tensor of that width")
+    ap.add_argument("--adam", action="store_true",
+                    help="time ADAM (beta1 0.9, beta2 0.999, eps 1e-8, two int16 moment tensors; the step "
+                         "size is 1e-3 of the first tensor's range)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-buckets", action="store_true",
@@ -193,8 +196,14 @@ def run_ours(args, rank, world, local_rank):
     t0 = time.time()
     host = HostInputs(wl, multi.rank_seed(args.seed, rank), n_sets, pinned=True)
     gen_s = time.time() - t0
-    run = DeviceRun(host, B.KSGD_EXP_AMAX, mom_bits=args.momentum_bits)
-    if args.momentum_bits:
+    adam = None
+    if args.adam:
+        t0_ = wl.tensors[0]
+        adam = dict(beta1=0.9, beta2=0.999, eps=1e-8,
+                    eta=1e-3 * 2.0 ** t0_.exp_theta * (2 ** (t0_.theta_bits - 1) - 1))
+    run = DeviceRun(host, B.KSGD_EXP_AMAX, mom_bits=args.momentum_bits, adam=adam)
+    other = bool(args.momentum_bits or args.adam)
+    if other:
         args.no_e2e = args.no_cpu_baseline = True      # those legs describe the plain step
     stream = run.stream
 
@@ -250,7 +259,7 @@ def run_ours(args, rank, world, local_rank):
                "d2h_bytes_per_step": state_bytes, "steps": args.e2e_steps,
                "ms_per_step": dt / args.e2e_steps * 1e3}
     graph_us = None
-    if wl.bytes_per_step < (64 << 20) and world == 1 and not args.momentum_bits:
+    if wl.bytes_per_step < (64 << 20) and world == 1 and not other:
         # small lists are bound by the host's launch rate: also time the same steps recorded
         # once into a CUDA graph and replayed (kahan_sgd_step only enqueues work)
         with torch.cuda.stream(stream):
@@ -268,7 +277,7 @@ def run_ours(args, rank, world, local_rank):
             stream.synchronize()
             graph_us = g0.elapsed_time(g1) * 1e3 / args.steps
     buckets = None
-    if wl.name == "c5_sweep" and rank == 0 and not args.momentum_bits and not args.no_buckets:
+    if wl.name == "c5_sweep" and rank == 0 and not other and not args.no_buckets:
         buckets = time_size_buckets(torch, B, run, wl)
     run.close()
 
@@ -280,7 +289,7 @@ def run_ours(args, rank, world, local_rank):
 
     peak, peak_src = hbm_peak()
     achieved = run.bytes_per_step / (ms_step * 1e-3) / 1e9
-    traffic = None if args.momentum_bits else recorded_traffic(wl)
+    traffic = None if other else recorded_traffic(wl)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
@@ -288,14 +297,15 @@ def run_ours(args, rank, world, local_rank):
         "config": {"workload": wl.name, "tensors": n, "parameters": wl.numel,
                    "bytes_per_step": run.bytes_per_step, "grad_sets": n_sets,
                    "optimizer": "momentum 0.9, int%d velocity" % args.momentum_bits if args.momentum_bits
-                   else "sgd",
+                   else ("adam 0.9/0.999/1e-8, int16 moments" if args.adam else "sgd"),
                    "l2": "inputs larger than L2 (%.0f MB touched per step)" % (wl.bytes_per_step / 1e6),
                    "exponent_mode": "amax", "input_generation_s": round(gen_s, 1)},
         "achieved_hbm_gbs": achieved,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                      "frac_of_nominal_8000": achieved / 8000.0,
-                     "kernel": "ksgd_momentum_step_kernel" if args.momentum_bits else "ksgd_step_kernel",
+                     "kernel": "ksgd_momentum_step_kernel" if args.momentum_bits
+                     else ("ksgd_adam_step_kernel" if args.adam else "ksgd_step_kernel"),
                      "launch_ms": ms_step},
         "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
         "counters": {"n_sat_theta": int(sum(stats["n_sat_theta"])),

@@ -235,6 +235,74 @@ int kahan_sgd_momentum_amax(ksgd_momentum_handle* h, uint32_t* amax_theta, uint3
 int kahan_sgd_momentum_destroy(ksgd_momentum_handle* h);
 
 /*
+ * ADAM with the lazy update (Section 4: Algorithm 1 in the optimizers; the experiments use
+ * ADAM with beta1 = 0.9, beta2 = 0.999, and with beta1 = 0.5, beta2 = 0.9, eps = 1e-3; INT16
+ * is needed for it because of beta2).  The paper prints no formulas for it; the form
+ * implemented is the published ADAM with the bias correction folded into the step size by
+ * the caller, lr_t = eta * sqrt(1 - beta2^t) / (1 - beta1^t):
+ *     m <- beta1*m + (1-beta1)*g ,  v <- beta2*v + (1-beta2)*g^2 ,
+ *     theta <- theta - lr_t * m / (sqrt(v) + eps)     (the subtraction through Algorithm 1)
+ * with m and v two more dynamic fixed-point tensors of 16-bit mantissas, each with its own
+ * shared exponent that follows the max scan of its mantissas like the momentum velocity's
+ * (one step of delay, at most 8 binades per step, [-64, 64], dead band (QMAX/4, QMAX]).
+ * Per element, every fl32/fma32/sqrt32/div32 one correctly rounded binary32 operation:
+ *     ym = fma32(fl32(beta1 * 2^(em_in-em_out)), Q_m, fl32(g * fl32(fl32(1-beta1) * 2^-em_out)))
+ *     yv = fma32(fl32(beta2 * 2^(ev_in-ev_out)), Q_v, fl32(fl32(g*g) * fl32(fl32(1-beta2) * 2^-ev_out)))
+ *     M, V = clamp(rne(y), +-2^30), NaN -> 0 ;  Q_m', Q_v' = clamp(., +-32767)
+ *     q  = div32(Q_m' * 2^em_out, fl32(sqrt32(max(Q_v', 1) * 2^ev_out) + eps))
+ *     d  = clamp(rne(fl32(q * fl32(lr_t * 2^-(e_out - s)))), +-2^30), NaN -> 0
+ *     then T, P, Q_theta', Rq, Q_c' as in the plain step with this d.
+ * A second moment below the resolution of its grid is taken as one unit of the grid, not as
+ * zero (which would leave eps alone in the denominator and make the step m/eps): the step of
+ * such an element is bounded by |m| / sqrt(2^ev_out).  The tensor descriptions are the same
+ * ksgd_tensor_desc (comp_bits must be 8 or 16) plus one ksgd_adam_desc per tensor.  At most
+ * 256 tensors per list.  Ownership, streams and return codes are as for the plain entry
+ * points.  lrs: host array of lr_t per tensor, finite and > 0; beta1, beta2 in [0, 1], eps
+ * finite and >= 0 (otherwise KSGD_ERR_LR).  kahan_sgd_adam_amax fills the non-NULL host
+ * arrays of ksgd_adam_stats (n_tensors entries each): maxima of |P|, |Rq|, |M|, |V| of the
+ * last step, the exponents now stored and those the next step writes, and the counts of
+ * clamped mantissas and non-finite gradients since init.
+ */
+typedef struct ksgd_adam_handle ksgd_adam_handle;
+
+typedef struct {
+  void*   mom1;          /* device, int16_t[numel], first moment m; in place; 16-byte aligned */
+  void*   mom2;          /* device, int16_t[numel], second moment v; in place; 16-byte aligned */
+  int32_t exp_m;         /* exponent of the first-moment mantissas now stored, in [-64, 64] */
+  int32_t exp_m_next;    /* exponent the first step writes, within 8 of exp_m */
+  int32_t exp_v;         /* the same for the second moment */
+  int32_t exp_v_next;
+} ksgd_adam_desc;
+
+typedef struct {
+  uint32_t *amax_theta, *amax_comp, *amax_m, *amax_v;
+  int32_t  *exp_theta_cur, *exp_theta_next, *exp_m_cur, *exp_m_next, *exp_v_cur, *exp_v_next;
+  uint64_t *n_sat_theta, *n_sat_comp, *n_sat_m, *n_sat_v, *n_nonfinite;
+} ksgd_adam_stats;
+
+size_t kahan_sgd_adam_workspace_bytes(const ksgd_tensor_desc* descs, const ksgd_adam_desc* adescs,
+                                      int32_t n_tensors);
+int kahan_sgd_adam_init(ksgd_adam_handle** out, const ksgd_tensor_desc* descs, const ksgd_adam_desc* adescs,
+                        int32_t n_tensors, ksgd_exp_mode mode, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream);
+int kahan_sgd_adam_step(ksgd_adam_handle* h, const float* const* grads, const float* lrs, float beta1,
+                        float beta2, float eps);
+int kahan_sgd_adam_amax(ksgd_adam_handle* h, const ksgd_adam_stats* out);
+int kahan_sgd_adam_destroy(ksgd_adam_handle* h);
+
+/*
+ * Self-check of the ADAM kernel's arithmetic (no counterpart in the paper).  The kernel's
+ * fast path computes sqrt32 and div32 above with short branch-free sequences instead of the
+ * general correctly rounded operations; this call compares the two on the device for every
+ * operand the fast path can meet -- all (Q_m', significand of the denominator) pairs at
+ * eight exponent pairs including the corners of the exponent ranges (2.2e12 divisions), and
+ * all Q_v' * 2^ev (4.2e6 square roots) -- and returns the numbers of differing results in
+ * the two host words (both must be 0).  Takes about two seconds of GPU time; allocates
+ * nothing; runs on cuda_stream and waits for it.
+ */
+int kahan_sgd_adam_selfcheck(uint64_t* div_mismatches, uint64_t* sqrt_mismatches, void* cuda_stream);
+
+/*
  * fp32 -> dynamic fixed-point (Section 1: uniform linear quantization, one shared exponent
  * per tensor; Section 5: the exponent from a scan of the maximum).  src: device,
  * fp32[numel].  theta / comp: device outputs in the formats of ksgd_tensor_desc (comp NULL

@@ -405,10 +405,15 @@ int32_t ksgd_oracle_next_exponent_velocity(uint32_t amax_mom, int32_t mom_bits, 
  *   ym = fma(fl(beta1 * 2^(em_in-em_out)), Q_m, fl(g * fl(c1 * 2^-em_out)))    M = rne(ym)
  *   yv = fma(fl(beta2 * 2^(ev_in-ev_out)), Q_v, fl(fl(g*g) * fl(c2 * 2^-ev_out)))  V = rne(yv)
  *   (both clamped to +-2^30, NaN -> 0, then to +-(2^15 - 1) for storage)
- *   mr = Q_m' * 2^em_out, vr = Q_v' * 2^ev_out          exact
- *   q  = fl(mr / fl(sqrt(vr) + eps))                    sqrt of a negative vr is taken of 0
+ *   mr = Q_m' * 2^em_out, vr = max(Q_v', 1) * 2^ev_out  exact
+ *   q  = fl(mr / fl(sqrt(vr) + eps))
  *   d  = clamp(rne(fl(q * fl(lr_t * 2^-ec_out))), +-2^30), NaN -> 0
  *   then statements 1-4 of Algorithm 1 with this d.
+ * The floor of one unit on the second-moment mantissa: a second moment below the resolution
+ * of its 16-bit grid would otherwise leave eps alone in the denominator and turn any
+ * non-zero first moment into a step of m/eps (1e8 m with the usual eps); a value that the
+ * grid cannot tell from zero is taken as one unit instead, which bounds the step by
+ * |m| / sqrt(2^ev_out).
  */
 typedef struct {
   ksgd_oracle_elem upd;
@@ -439,8 +444,8 @@ void ksgd_oracle_adam_element(int32_t q_theta, int32_t q_comp, int32_t q_m, int3
   int32_t ec_in = e_in - s, ec_out = e_out - s;
   int32_t f = ec_in < ec_out ? ec_in : ec_out;
   float mr = ldexpf((float)qm_new, em_out);
-  float vr = ldexpf((float)qv_new, ev_out);
-  float root = sqrtf(vr > 0.0f ? vr : 0.0f);
+  float vr = ldexpf((float)(qv_new > 1 ? qv_new : 1), ev_out);
+  float root = sqrtf(vr);
   float den = root + eps;
   float q = mr / den;
   float x = q * ldexpf(lr, -ec_out);

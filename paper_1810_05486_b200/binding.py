@@ -32,6 +32,8 @@ EXPORTS = (
     "kahan_sgd_amax", "kahan_sgd_set_exponents", "kahan_sgd_step_static", "kahan_sgd_destroy",
     "kahan_sgd_strerror", "kahan_sgd_momentum_workspace_bytes", "kahan_sgd_momentum_init",
     "kahan_sgd_momentum_step", "kahan_sgd_momentum_amax", "kahan_sgd_momentum_destroy",
+    "kahan_sgd_adam_workspace_bytes", "kahan_sgd_adam_init", "kahan_sgd_adam_step",
+    "kahan_sgd_adam_amax", "kahan_sgd_adam_destroy", "kahan_sgd_adam_selfcheck",
     "kahan_sgd_import", "kahan_sgd_export", "kahan_sgd_classifier_bits",
     "kahan_sgd_last_cuda_error", "kahan_sgd_launch_count",
 )
@@ -47,6 +49,20 @@ class ksgd_tensor_desc(ctypes.Structure):
 class ksgd_momentum_desc(ctypes.Structure):
     _fields_ = [("mom", ctypes.c_void_p), ("mom_bits", ctypes.c_int32), ("exp_mom", ctypes.c_int32),
                 ("exp_mom_next", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class ksgd_adam_desc(ctypes.Structure):
+    _fields_ = [("mom1", ctypes.c_void_p), ("mom2", ctypes.c_void_p), ("exp_m", ctypes.c_int32),
+                ("exp_m_next", ctypes.c_int32), ("exp_v", ctypes.c_int32), ("exp_v_next", ctypes.c_int32)]
+
+
+_ADAM_STATS_FIELDS = ("amax_theta", "amax_comp", "amax_m", "amax_v", "exp_theta_cur", "exp_theta_next",
+                      "exp_m_cur", "exp_m_next", "exp_v_cur", "exp_v_next", "n_sat_theta", "n_sat_comp",
+                      "n_sat_m", "n_sat_v", "n_nonfinite")
+
+
+class ksgd_adam_stats(ctypes.Structure):
+    _fields_ = [(name, ctypes.c_void_p) for name in _ADAM_STATS_FIELDS]
 
 
 class KahanSgdError(RuntimeError):
@@ -95,6 +111,21 @@ def _load() -> ctypes.CDLL:
     lib.kahan_sgd_momentum_amax.argtypes = [ctypes.c_void_p] + [ctypes.c_void_p] * 11
     lib.kahan_sgd_momentum_destroy.restype = ctypes.c_int
     lib.kahan_sgd_momentum_destroy.argtypes = [ctypes.c_void_p]
+    lib.kahan_sgd_adam_workspace_bytes.restype = ctypes.c_size_t
+    lib.kahan_sgd_adam_workspace_bytes.argtypes = [P(ksgd_tensor_desc), P(ksgd_adam_desc), ctypes.c_int32]
+    lib.kahan_sgd_adam_init.restype = ctypes.c_int
+    lib.kahan_sgd_adam_init.argtypes = [P(ctypes.c_void_p), P(ksgd_tensor_desc), P(ksgd_adam_desc),
+                                        ctypes.c_int32, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t,
+                                        ctypes.c_void_p]
+    lib.kahan_sgd_adam_step.restype = ctypes.c_int
+    lib.kahan_sgd_adam_step.argtypes = [ctypes.c_void_p, P(ctypes.c_void_p), P(ctypes.c_float),
+                                        ctypes.c_float, ctypes.c_float, ctypes.c_float]
+    lib.kahan_sgd_adam_amax.restype = ctypes.c_int
+    lib.kahan_sgd_adam_amax.argtypes = [ctypes.c_void_p, P(ksgd_adam_stats)]
+    lib.kahan_sgd_adam_destroy.restype = ctypes.c_int
+    lib.kahan_sgd_adam_destroy.argtypes = [ctypes.c_void_p]
+    lib.kahan_sgd_adam_selfcheck.restype = ctypes.c_int
+    lib.kahan_sgd_adam_selfcheck.argtypes = [P(ctypes.c_uint64), P(ctypes.c_uint64), ctypes.c_void_p]
     lib.kahan_sgd_import.restype = ctypes.c_int
     lib.kahan_sgd_import.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int64] + [ctypes.c_int32] * 4 + \
         [P(ctypes.c_int32), ctypes.c_void_p, ctypes.c_void_p]
@@ -281,6 +312,57 @@ def kahan_sgd_momentum_amax(h, n_tensors: int) -> dict:
 
 def kahan_sgd_momentum_destroy(h) -> None:
     _check(lib.kahan_sgd_momentum_destroy(h))
+
+
+def make_adam_descs(tensors: Sequence[dict]):
+    """ctypes array of ksgd_adam_desc from dicts with keys mom1, mom2, exp_m, exp_v (and
+    optionally exp_m_next, exp_v_next)."""
+    arr = (ksgd_adam_desc * len(tensors))()
+    for d, t in zip(arr, tensors):
+        d.mom1, d.mom2 = t["mom1"], t["mom2"]
+        d.exp_m, d.exp_m_next = t["exp_m"], t.get("exp_m_next", t["exp_m"])
+        d.exp_v, d.exp_v_next = t["exp_v"], t.get("exp_v_next", t["exp_v"])
+    return arr
+
+
+def kahan_sgd_adam_workspace_bytes(descs, adescs) -> int:
+    return int(lib.kahan_sgd_adam_workspace_bytes(descs, adescs, len(descs)))
+
+
+def kahan_sgd_adam_init(descs, adescs, mode: int, workspace: int, workspace_bytes: int, stream: int = 0):
+    h = ctypes.c_void_p()
+    _check(lib.kahan_sgd_adam_init(ctypes.byref(h), descs, adescs, len(descs), mode,
+                                   ctypes.c_void_p(workspace), workspace_bytes, ctypes.c_void_p(stream)))
+    return h
+
+
+def kahan_sgd_adam_step(h, grads, lrs, beta1: float, beta2: float, eps: float) -> None:
+    g = grads if isinstance(grads, ctypes.Array) else _ptr_array(grads)
+    l = lrs if isinstance(lrs, ctypes.Array) else _float_array(lrs)
+    _check(lib.kahan_sgd_adam_step(h, g, l, beta1, beta2, eps))
+
+
+def kahan_sgd_adam_amax(h, n_tensors: int) -> dict:
+    arrays = {}
+    st = ksgd_adam_stats()
+    for name in _ADAM_STATS_FIELDS:
+        ctype = ctypes.c_uint32 if name.startswith("amax") else (
+            ctypes.c_int32 if name.startswith("exp") else ctypes.c_uint64)
+        arrays[name] = (ctype * n_tensors)()
+        setattr(st, name, ctypes.addressof(arrays[name]))
+    _check(lib.kahan_sgd_adam_amax(h, ctypes.byref(st)))
+    return {name: list(a) for name, a in arrays.items()}
+
+
+def kahan_sgd_adam_destroy(h) -> None:
+    _check(lib.kahan_sgd_adam_destroy(h))
+
+
+def kahan_sgd_adam_selfcheck(stream: int = 0):
+    """(division mismatches, square-root mismatches) of the fast path's sequences."""
+    d, q = ctypes.c_uint64(), ctypes.c_uint64()
+    _check(lib.kahan_sgd_adam_selfcheck(ctypes.byref(d), ctypes.byref(q), ctypes.c_void_p(stream)))
+    return int(d.value), int(q.value)
 
 
 KSGD_EXP_AUTO = -(2 ** 31)

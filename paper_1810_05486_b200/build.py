@@ -10,6 +10,8 @@ LIBRARY = os.path.join(_HERE, "libkahan_sgd.so")
 SOURCES = [os.path.join(CSRC, "kahan_sgd_api.cu")]
 _DEPENDS = SOURCES + [os.path.join(CSRC, "kahan_sgd_kernels.cuh"),
                       os.path.join(CSRC, "kahan_sgd_momentum_kernels.cuh"),
+                      os.path.join(CSRC, "kahan_sgd_adam_kernels.cuh"),
+                      os.path.join(CSRC, "kahan_sgd_convert.cuh"),
                       os.path.join(INCLUDE, "kahan_sgd.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -13,6 +13,7 @@
 
 #include "kahan_sgd_kernels.cuh"
 #include "kahan_sgd_momentum_kernels.cuh"
+#include "kahan_sgd_adam_kernels.cuh"
 #include "kahan_sgd_convert.cuh"
 
 namespace {
@@ -806,6 +807,263 @@ int kahan_sgd_momentum_amax(ksgd_momentum_handle* h, uint32_t* amax_theta, uint3
 }
 
 int kahan_sgd_momentum_destroy(ksgd_momentum_handle* h) {
+  if (!h) return KSGD_ERR_NULL;
+  const cudaError_t e = cudaStreamSynchronize(h->stream);
+  delete h;
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  return KSGD_OK;
+}
+
+// ----------------------------------------------------------------------------------------
+// ADAM with the lazy update.
+
+namespace {
+
+struct AdamLayout {
+  size_t exp_cur, exp_next, expm_cur, expm_next, expv_cur, expv_next, amax_last, counters, error, stats_end;
+  size_t amax_acc, info, chunks, ticket, total;
+  long long n_chunks;
+};
+
+AdamLayout make_adam_layout(const ksgd_tensor_desc* d, int32_t n) {
+  AdamLayout L{};
+  long long chunks = 0;
+  for (int32_t i = 0; i < n; ++i) chunks += (d[i].numel + kChunk - 1) / kChunk;
+  L.n_chunks = chunks;
+  size_t o = 0;
+  L.exp_cur = o;   o += sizeof(int) * n;
+  L.exp_next = o;  o += sizeof(int) * n;
+  L.expm_cur = o;  o += sizeof(int) * n;
+  L.expm_next = o; o += sizeof(int) * n;
+  L.expv_cur = o;  o += sizeof(int) * n;
+  L.expv_next = o; o += sizeof(int) * n;
+  L.amax_last = o; o += sizeof(unsigned int) * 4 * n;
+  o = align_up(o, 8);
+  L.counters = o;  o += sizeof(unsigned long long) * 5 * n;
+  L.error = o;     o += 8;
+  L.stats_end = o;
+  L.amax_acc = o;  o += sizeof(unsigned int) * 4 * n;
+  o = align_up(o, 16);
+  L.info = o;      o += sizeof(adam::TensorInfo) * n;
+  o = align_up(o, 16);
+  L.chunks = o;    o += sizeof(ChunkRef) * (size_t)chunks;
+  o = align_up(o, 16);
+  L.ticket = o;    o += 16;
+  L.total = align_up(o, 256);
+  return L;
+}
+
+bool exp_pair_ok(int32_t cur, int32_t next) {
+  return cur >= kExpMin && cur <= kExpMax && next >= kExpMin && next <= kExpMax &&
+         std::abs(next - cur) <= kMaxDelta;
+}
+
+int validate_adam(const ksgd_tensor_desc* d, const ksgd_adam_desc* a, int32_t n) {
+  const int v = validate(d, n);
+  if (v != KSGD_OK) return v;
+  if (!a) return KSGD_ERR_NULL;
+  if (n > kInlineArgs) return KSGD_ERR_NUMEL;
+  for (int32_t i = 0; i < n; ++i) {
+    if (d[i].comp_bits == 0) return KSGD_ERR_BITS;        // ADAM goes through the lazy update
+    if (!a[i].mom1 || !a[i].mom2) return KSGD_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(a[i].mom1) % 16 || reinterpret_cast<uintptr_t>(a[i].mom2) % 16)
+      return KSGD_ERR_ALIGN;
+    if (!exp_pair_ok(a[i].exp_m, a[i].exp_m_next) || !exp_pair_ok(a[i].exp_v, a[i].exp_v_next))
+      return KSGD_ERR_EXP_RANGE;
+  }
+  return KSGD_OK;
+}
+
+}  // namespace
+
+struct ksgd_adam_handle {
+  AdamLayout layout;
+  adam::StepParams params;
+  char* ws_base;
+  cudaStream_t stream;
+  int32_t n;
+  int grid;
+  std::vector<unsigned char> stats_host;
+};
+
+size_t kahan_sgd_adam_workspace_bytes(const ksgd_tensor_desc* descs, const ksgd_adam_desc* adescs,
+                                      int32_t n_tensors) {
+  if (validate_adam(descs, adescs, n_tensors) != KSGD_OK) return 0;
+  return make_adam_layout(descs, n_tensors).total;
+}
+
+int kahan_sgd_adam_init(ksgd_adam_handle** out, const ksgd_tensor_desc* descs, const ksgd_adam_desc* adescs,
+                        int32_t n_tensors, ksgd_exp_mode mode, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream) {
+  if (!out) return KSGD_ERR_NULL;
+  *out = nullptr;
+  const int v = validate_adam(descs, adescs, n_tensors);
+  if (v != KSGD_OK) return v;
+  if (mode != KSGD_EXP_FIXED && mode != KSGD_EXP_AMAX) return KSGD_ERR_MODE;
+  if (!workspace) return KSGD_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(workspace) % 256) return KSGD_ERR_ALIGN;
+  const AdamLayout L = make_adam_layout(descs, n_tensors);
+  if (workspace_bytes < L.total) return KSGD_ERR_WORKSPACE;
+
+  ksgd_adam_handle* h = new (std::nothrow) ksgd_adam_handle();
+  if (!h) return KSGD_ERR_NULL;
+  h->layout = L;
+  h->n = n_tensors;
+  h->ws_base = static_cast<char*>(workspace);
+  h->stream = static_cast<cudaStream_t>(cuda_stream);
+  h->stats_host.resize(L.stats_end);
+
+  std::vector<unsigned char> img(L.total, 0);
+  auto ints = [&](size_t off) { return reinterpret_cast<int*>(img.data() + off); };
+  adam::TensorInfo* info = reinterpret_cast<adam::TensorInfo*>(img.data() + L.info);
+  ChunkRef* chunks = reinterpret_cast<ChunkRef*>(img.data() + L.chunks);
+  long long c = 0;
+  double state_bytes = 0.0;
+  for (int32_t i = 0; i < n_tensors; ++i) {
+    const ksgd_tensor_desc& t = descs[i];
+    ints(L.exp_cur)[i] = t.exp_theta;
+    ints(L.exp_next)[i] = t.exp_theta_next;
+    ints(L.expm_cur)[i] = adescs[i].exp_m;
+    ints(L.expm_next)[i] = adescs[i].exp_m_next;
+    ints(L.expv_cur)[i] = adescs[i].exp_v;
+    ints(L.expv_next)[i] = adescs[i].exp_v_next;
+    info[i].theta = t.theta;
+    info[i].comp = t.comp;
+    info[i].mom1 = adescs[i].mom1;
+    info[i].mom2 = adescs[i].mom2;
+    info[i].numel = t.numel;
+    info[i].theta_bits = t.theta_bits;
+    info[i].comp_bits = t.comp_bits;
+    info[i].s = t.comp_bits - 1 - t.overlap_k;
+    info[i].pad = 0;
+    const long long nc = (t.numel + kChunk - 1) / kChunk;
+    for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
+    state_bytes += (double)t.numel * ((t.theta_bits + t.comp_bits + 32) / 8);
+  }
+
+  adam::Workspace& w = h->params.ws;
+  char* b = h->ws_base;
+  w.exp_cur = reinterpret_cast<int*>(b + L.exp_cur);
+  w.exp_next = reinterpret_cast<int*>(b + L.exp_next);
+  w.expm_cur = reinterpret_cast<int*>(b + L.expm_cur);
+  w.expm_next = reinterpret_cast<int*>(b + L.expm_next);
+  w.expv_cur = reinterpret_cast<int*>(b + L.expv_cur);
+  w.expv_next = reinterpret_cast<int*>(b + L.expv_next);
+  w.amax_last = reinterpret_cast<unsigned int*>(b + L.amax_last);
+  w.counters = reinterpret_cast<unsigned long long*>(b + L.counters);
+  w.error = reinterpret_cast<unsigned int*>(b + L.error);
+  w.amax_acc = reinterpret_cast<unsigned int*>(b + L.amax_acc);
+  w.info = reinterpret_cast<adam::TensorInfo*>(b + L.info);
+  w.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
+  w.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
+  h->params.n_tensors = n_tensors;
+  h->params.n_chunks = (int)L.n_chunks;
+  h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
+
+  int dev = 0, sms = 0, l2_bytes = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, dev);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(adam::ksgd_adam_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)adam::kSharedBytes);
+  if (e != cudaSuccess) {
+    delete h;
+    return cuda_fail(e, "device query");
+  }
+  h->grid = (int)(L.n_chunks < (long long)sms ? L.n_chunks : (long long)sms);
+  h->params.grad_evict_first = state_bytes <= 0.8 * (double)l2_bytes ? 1 : 0;
+
+  e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+  if (e != cudaSuccess) {
+    delete h;
+    return cuda_fail(e, "workspace upload");
+  }
+  *out = h;
+  return KSGD_OK;
+}
+
+int kahan_sgd_adam_step(ksgd_adam_handle* h, const float* const* grads, const float* lrs, float beta1,
+                        float beta2, float eps) {
+  if (!h || !grads || !lrs) return KSGD_ERR_NULL;
+  if (!(beta1 >= 0.0f && beta1 <= 1.0f) || !(beta2 >= 0.0f && beta2 <= 1.0f)) return KSGD_ERR_LR;
+  if (!std::isfinite(eps) || !(eps >= 0.0f)) return KSGD_ERR_LR;
+  adam::StepArgs args;
+  for (int32_t i = 0; i < h->n; ++i) {
+    if (!grads[i]) return KSGD_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(grads[i]) % 16) return KSGD_ERR_ALIGN;
+    if (!std::isfinite(lrs[i]) || !(lrs[i] > 0.0f)) return KSGD_ERR_LR;
+    args.grads[i] = grads[i];
+    args.lrs[i] = lrs[i];
+  }
+  for (int32_t i = h->n; i < kInlineArgs; ++i) { args.grads[i] = nullptr; args.lrs[i] = 0.0f; }
+  args.beta1 = beta1;
+  args.beta2 = beta2;
+  args.eps = eps;
+  adam::ksgd_adam_step_kernel<<<(unsigned)h->grid, adam::kBlock, adam::kSharedBytes, h->stream>>>(h->params,
+                                                                                                args);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  KSGD_CUDA(cudaGetLastError());
+  return KSGD_OK;
+}
+
+int kahan_sgd_adam_amax(ksgd_adam_handle* h, const ksgd_adam_stats* out) {
+  if (!h || !out) return KSGD_ERR_NULL;
+  const AdamLayout& L = h->layout;
+  KSGD_CUDA(cudaMemcpyAsync(h->stats_host.data(), h->ws_base, L.stats_end, cudaMemcpyDeviceToHost,
+                            h->stream));
+  KSGD_CUDA(cudaStreamSynchronize(h->stream));
+  const unsigned char* b = h->stats_host.data();
+  const size_t n = (size_t)h->n;
+  auto give = [&](void* dst, size_t off, size_t width) { if (dst) std::memcpy(dst, b + off, width * n); };
+  give(out->exp_theta_cur, L.exp_cur, 4);
+  give(out->exp_theta_next, L.exp_next, 4);
+  give(out->exp_m_cur, L.expm_cur, 4);
+  give(out->exp_m_next, L.expm_next, 4);
+  give(out->exp_v_cur, L.expv_cur, 4);
+  give(out->exp_v_next, L.expv_next, 4);
+  give(out->amax_theta, L.amax_last, 4);
+  give(out->amax_comp, L.amax_last + 4 * n, 4);
+  give(out->amax_m, L.amax_last + 8 * n, 4);
+  give(out->amax_v, L.amax_last + 12 * n, 4);
+  give(out->n_sat_theta, L.counters, 8);
+  give(out->n_sat_comp, L.counters + 8 * n, 8);
+  give(out->n_sat_m, L.counters + 16 * n, 8);
+  give(out->n_sat_v, L.counters + 24 * n, 8);
+  give(out->n_nonfinite, L.counters + 32 * n, 8);
+  unsigned int dev_err = 0;
+  std::memcpy(&dev_err, b + L.error, 4);
+  if (dev_err != 0) return KSGD_ERR_DEVICE;
+  return KSGD_OK;
+}
+
+static __device__ unsigned long long g_selfcheck_mismatches[2];
+
+int kahan_sgd_adam_selfcheck(uint64_t* div_mismatches, uint64_t* sqrt_mismatches, void* cuda_stream) {
+  if (!div_mismatches || !sqrt_mismatches) return KSGD_ERR_NULL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  unsigned long long* dev = nullptr;
+  KSGD_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&dev), g_selfcheck_mismatches));
+  KSGD_CUDA(cudaMemsetAsync(dev, 0, 16, stream));
+  // exponents of a (first moment grid) and of b (denominator): corners and inside
+  const int combos[][2] = {{0, 0}, {-20, -10}, {-64, -32}, {-64, 40}, {64, -32}, {64, 40}, {-37, 5}, {-1, 1}};
+  for (const auto& c : combos) {
+    adam::ksgd_adam_selfcheck_div<<<(1u << 23) / 256, 256, 0, stream>>>(c[0], c[1], dev);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+  }
+  adam::ksgd_adam_selfcheck_sqrt<<<128, 256, 0, stream>>>(dev + 1);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  KSGD_CUDA(cudaGetLastError());
+  unsigned long long host[2] = {0, 0};
+  KSGD_CUDA(cudaMemcpyAsync(host, dev, 16, cudaMemcpyDeviceToHost, stream));
+  KSGD_CUDA(cudaStreamSynchronize(stream));
+  *div_mismatches = host[0];
+  *sqrt_mismatches = host[1];
+  return KSGD_OK;
+}
+
+int kahan_sgd_adam_destroy(ksgd_adam_handle* h) {
   if (!h) return KSGD_ERR_NULL;
   const cudaError_t e = cudaStreamSynchronize(h->stream);
   delete h;

@@ -54,9 +54,12 @@ class DeviceRun:
     """Device buffers (same layout as HostInputs), descriptors, workspace and handle."""
 
     def __init__(self, host: HostInputs, mode: int = B.KSGD_EXP_AMAX, stream=None,
-                 mom_bits: int = 0, mu: float = 0.9):
+                 mom_bits: int = 0, mu: float = 0.9, adam: Optional[dict] = None):
         """mom_bits = 8 or 16 selects the momentum optimizer (velocity buffers start at zero,
-        on a grid 8 binades below theta's)."""
+        on a grid 8 binades below theta's).  adam = dict(beta1, beta2, eps, eta) selects ADAM
+        (both 16-bit moments start at zero, on grids that just hold what the first step makes of
+        the largest gradient of the first set; the step size carries the bias correction of the
+        step count)."""
         import torch
         self.torch = torch
         self.host = host
@@ -74,7 +77,27 @@ class DeviceRun:
             for i, t in enumerate(wl.tensors)])
         self.stream = stream if stream is not None else torch.cuda.Stream()
         self.mom_bits = mom_bits
-        if mom_bits:
+        self.adam = adam
+        self.t = 0
+        if adam:
+            assert not mom_bits
+            self.m_offs, m_bytes = _carve(wl, lambda t: 2)
+            self.dev_m1 = torch.zeros(m_bytes, dtype=torch.uint8, device="cuda")
+            self.dev_m2 = torch.zeros(m_bytes, dtype=torch.uint8, device="cuda")
+            adescs = []
+            for i, g in enumerate(host.grads[0]):
+                gmax = max(float(np.abs(g[:1 << 20]).max()), 1e-30)
+                e_m = int(np.clip(np.ceil(np.log2((1.0 - adam["beta1"] + 1e-9) * gmax / 32767.0)), -64, 64))
+                e_v = int(np.clip(np.ceil(np.log2((1.0 - adam["beta2"] + 1e-9) * gmax * gmax / 32767.0)),
+                                  -64, 64))
+                adescs.append(dict(mom1=self.dev_m1.data_ptr() + self.m_offs[i],
+                                   mom2=self.dev_m2.data_ptr() + self.m_offs[i], exp_m=e_m, exp_v=e_v))
+            self.adescs = B.make_adam_descs(adescs)
+            self.ws_bytes = B.kahan_sgd_adam_workspace_bytes(self.descs, self.adescs)
+            self.workspace = torch.zeros(self.ws_bytes, dtype=torch.uint8, device="cuda")
+            self.handle = B.kahan_sgd_adam_init(self.descs, self.adescs, mode, self.workspace.data_ptr(),
+                                                self.ws_bytes, self.stream.cuda_stream)
+        elif mom_bits:
             self.v_offs, v_bytes = _carve(wl, lambda t: mom_bits // 8)
             self.dev_v = torch.zeros(v_bytes, dtype=torch.uint8, device="cuda")
             self.mdescs = B.make_momentum_descs([
@@ -95,20 +118,36 @@ class DeviceRun:
                               for g in self.dev_g]
         self.lrs = (ctypes.c_float * self.n)(*([wl.lr] * self.n))
 
+    def adam_lrs(self, t: int):
+        """Step sizes of ADAM step t (1-based): eta * sqrt(1 - beta2^t) / (1 - beta1^t)."""
+        a = self.adam
+        c1 = 1.0 - a["beta1"] ** t if a["beta1"] < 1.0 else 1.0
+        c2 = 1.0 - a["beta2"] ** t if a["beta2"] < 1.0 else 1.0
+        lr = float(np.float32(a["eta"] * np.sqrt(c2) / c1))
+        return (ctypes.c_float * self.n)(*([lr] * self.n))
+
     def step(self, grad_set: int) -> None:
-        if self.mom_bits:
+        if self.adam:
+            self.t += 1
+            B.kahan_sgd_adam_step(self.handle, self.grad_ptr_sets[grad_set], self.adam_lrs(self.t),
+                                  self.adam["beta1"], self.adam["beta2"], self.adam["eps"])
+        elif self.mom_bits:
             B.kahan_sgd_momentum_step(self.handle, self.grad_ptr_sets[grad_set], self.lrs, self.mus)
         else:
             B.kahan_sgd_step(self.handle, self.grad_ptr_sets[grad_set], self.lrs)
 
     def stats(self) -> dict:
+        if self.adam:
+            return B.kahan_sgd_adam_amax(self.handle, self.n)
         if self.mom_bits:
             return B.kahan_sgd_momentum_amax(self.handle, self.n)
         return B.kahan_sgd_amax(self.handle, self.n)
 
     @property
     def bytes_per_step(self) -> int:
-        """Algorithmic HBM bytes of one step, velocity included."""
+        """Algorithmic HBM bytes of one step, velocity or moments included."""
+        if self.adam:
+            return self.wl.bytes_per_step + 8 * self.wl.numel
         return self.wl.bytes_per_step + 2 * (self.mom_bits // 8) * self.wl.numel
 
     def theta(self, i: int) -> np.ndarray:
@@ -137,7 +176,9 @@ class DeviceRun:
 
     def close(self) -> None:
         if self.handle is not None:
-            if self.mom_bits:
+            if self.adam:
+                B.kahan_sgd_adam_destroy(self.handle)
+            elif self.mom_bits:
                 B.kahan_sgd_momentum_destroy(self.handle)
             else:
                 B.kahan_sgd_destroy(self.handle)

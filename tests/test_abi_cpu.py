@@ -128,6 +128,41 @@ def test_momentum_init_rejects_bad_descriptions_without_cuda(B):
     assert B.lib.kahan_sgd_momentum_destroy(None) == B.KSGD_ERR_NULL
 
 
+def test_adam_init_rejects_bad_descriptions_without_cuda(B):
+    assert ctypes.sizeof(B.ksgd_adam_desc) == 32 and ctypes.sizeof(B.ksgd_adam_stats) == 15 * 8
+    ok_a = dict(mom1=0x30000, mom2=0x40000, exp_m=-20, exp_v=-36)
+    cases = [((good(comp_bits=0, comp=0), ok_a), B.KSGD_ERR_BITS),      # ADAM needs the lazy update
+             ((good(), dict(ok_a, mom1=0)), B.KSGD_ERR_NULL),
+             ((good(), dict(ok_a, mom2=0)), B.KSGD_ERR_NULL),
+             ((good(), dict(ok_a, mom2=0x40002)), B.KSGD_ERR_ALIGN),
+             ((good(), dict(ok_a, exp_m=-70)), B.KSGD_ERR_EXP_RANGE),
+             ((good(), dict(ok_a, exp_v=65)), B.KSGD_ERR_EXP_RANGE),
+             ((good(), dict(ok_a, exp_v=0, exp_v_next=9)), B.KSGD_ERR_EXP_RANGE),
+             ((good(), dict(ok_a, exp_m=0, exp_m_next=-9)), B.KSGD_ERR_EXP_RANGE)]
+    for (d, a), code in cases:
+        descs, adescs = B.make_descs([d]), B.make_adam_descs([a])
+        assert B.kahan_sgd_adam_workspace_bytes(descs, adescs) == 0
+        with pytest.raises(B.KahanSgdError) as ei:
+            B.kahan_sgd_adam_init(descs, adescs, B.KSGD_EXP_AMAX, 0x100000, 1 << 20)
+        assert ei.value.code == code
+    assert B.kahan_sgd_adam_workspace_bytes(B.make_descs([good()] * 257), B.make_adam_descs([ok_a] * 257)) == 0
+    descs, adescs = B.make_descs([good()]), B.make_adam_descs([ok_a])
+    need = B.kahan_sgd_adam_workspace_bytes(descs, adescs)
+    assert need > 0 and need % 256 == 0
+    for ws, nb, mode, code in ((0, need, B.KSGD_EXP_AMAX, B.KSGD_ERR_NULL),
+                               (0x100010, need, B.KSGD_EXP_AMAX, B.KSGD_ERR_ALIGN),
+                               (0x100000, need - 1, B.KSGD_EXP_AMAX, B.KSGD_ERR_WORKSPACE),
+                               (0x100000, need, 7, B.KSGD_ERR_MODE)):
+        with pytest.raises(B.KahanSgdError) as ei:
+            B.kahan_sgd_adam_init(descs, adescs, mode, ws, nb)
+        assert ei.value.code == code
+    assert B.lib.kahan_sgd_adam_step(None, None, None, 0.9, 0.999, 1e-8) == B.KSGD_ERR_NULL
+    assert B.lib.kahan_sgd_adam_amax(None, None) == B.KSGD_ERR_NULL
+    assert B.lib.kahan_sgd_adam_destroy(None) == B.KSGD_ERR_NULL
+    assert B.lib.kahan_sgd_adam_selfcheck(None, None, None) == B.KSGD_ERR_NULL
+    assert B.kahan_sgd_launch_count() == 0
+
+
 def test_classifier_bits_follow_eq_5_and_the_printed_example(B):
     import math
     rows = [ln.split() for ln in open(os.path.join(ROOT, "tests", "golden", "classifier_bitwidth.txt"))

@@ -771,7 +771,7 @@ int kahan_sgd_momentum_step(ksgd_momentum_handle* h, const float* const* grads, 
     args.mus[i] = mus[i];
   }
   for (int32_t i = h->n; i < kInlineArgs; ++i) { args.grads[i] = nullptr; args.lrs[i] = 0.0f; args.mus[i] = 0.0f; }
-  mom::ksgd_momentum_step_kernel<<<(unsigned)h->grid, kBlockThreads, mom::kSharedBytes, h->stream>>>(h->params,
+  mom::ksgd_momentum_step_kernel<<<(unsigned)h->grid, mom::kBlock, mom::kSharedBytes, h->stream>>>(h->params,
                                                                                                   args);
   g_launches.fetch_add(1, std::memory_order_relaxed);
   KSGD_CUDA(cudaGetLastError());

@@ -56,6 +56,15 @@ struct StepArgs {                  // per-step arguments, passed as a kernel par
   float mus[kInlineArgs];
 };
 
+// Twelve consumer warps (three per scheduler, plus the producer's) leave 128 registers per
+// thread: a vector of eight elements with three mantissa arrays then stays in registers.
+#ifndef KSGD_MOM_WARPS
+#define KSGD_MOM_WARPS 12
+#endif
+constexpr int kWarps = KSGD_MOM_WARPS;         // consumer warps; one more warp produces
+constexpr int kThreads = 32 * kWarps;
+constexpr int kBlock = kThreads + 32;
+
 // What a tile's tensor needs for this step (general path reads all of it).
 struct Coef {
   float scale_v;   // lr * 2^-ev_out: gradient -> velocity LSBs of the output grid
@@ -177,9 +186,10 @@ struct SteadyCoef {
   float scale_v, mu_s, pow2k, pow2s_neg, inv2s, qmax_t, qmax_v, d_limit;
 };
 
-// Steady state (no exponent change of theta or of the velocity): eight elements on the FP32
-// pipe used as an exact integer unit (see update_vector of the plain step for the
-// technique).  With M = 1.5 * 2^23:
+// Steady state (no exponent change of theta; the velocity's exponent may change, because
+// mu_s and scale_v already carry both of its exponents): eight elements on the FP32 pipe
+// used as an exact integer unit (see update_vector of the plain step for the technique).
+// With M = 1.5 * 2^23:
 //   y  = fma(mu_s, Qv, fl32(g*scale_v))      the velocity, as defined (two roundings)
 //   Vm = y + M = M + rne(y) = M + V          |y| <= 4e6
 //   dm = fma(V, 2^k, M) = M + d              exact product for k >= 0, rne for k < 0
@@ -261,7 +271,7 @@ __device__ __forceinline__ bool consume_tile(const TileDesc* td, unsigned char* 
   const bool steady = (flags & kSteady) != 0;
   bool wrote_ring = false;
   const int n_vec = n_bulk / V;
-  for (int v = ctid; v < n_vec; v += kConsumers) {
+  for (int v = ctid; v < n_vec; v += kThreads) {
     Pack<TB> ot;
     Pack<CB> oc;
     Pack<VB> ov;
@@ -367,7 +377,7 @@ __device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const StepA
   return m;
 }
 
-__global__ void __launch_bounds__(kBlockThreads, 1)
+__global__ void __launch_bounds__(kBlock, 1)
 ksgd_momentum_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ StepArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   BlockShared* sh = reinterpret_cast<BlockShared*>(smem + (size_t)kPages * kPageBytes);
@@ -378,7 +388,7 @@ ksgd_momentum_step_kernel(const __grid_constant__ StepParams p, const __grid_con
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSlots; ++s) {
       mbar_init(&sh->full[s], 1u);
-      mbar_init(&sh->empty[s], (unsigned)kConsumerWarps);
+      mbar_init(&sh->empty[s], (unsigned)kWarps);
     }
     sh->abort_flag = 0;
     sh->is_last = 0;
@@ -389,7 +399,7 @@ ksgd_momentum_step_kernel(const __grid_constant__ StepParams p, const __grid_con
     reinterpret_cast<unsigned int*>(sh->scan)[threadIdx.x] = 0u;
   __syncthreads();
 
-  if (warp == kConsumerWarps) {
+  if (warp == kWarps) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
       const unsigned long long grad_policy = l2_policy_evict_first();
@@ -461,7 +471,7 @@ ksgd_momentum_step_kernel(const __grid_constant__ StepParams p, const __grid_con
         td.mom = static_cast<unsigned char*>(ti.mom) + first * vbytes;
         td.n_bulk = n_bulk;
         td.flags = ((ti.theta_bits == 16 ? 1 : 0) | (ti.comp_bits == 16 ? 2 : 0) | (ti.mom_bits == 16 ? 4 : 0)) |
-                   ((coef.delta == 0 && coef.delta_v == 0) ? kSteady : 0) | (page[1] << kThetaPageShift) |
+                   (coef.delta == 0 ? kSteady : 0) | (page[1] << kThetaPageShift) |
                    (page[2] << kCompPageShift) | (page[0] << kGradPageShift) | (page[3] << kMomPageShift);
         td.tensor = cr.tensor;
         td.count = count;
@@ -552,7 +562,7 @@ ksgd_momentum_step_kernel(const __grid_constant__ StepParams p, const __grid_con
   // Last block: rotate and choose the exponents of theta and of the velocity.
   __threadfence();
   const int n = p.n_tensors;
-  for (int i = threadIdx.x; i < n; i += kBlockThreads) {
+  for (int i = threadIdx.x; i < n; i += kBlock) {
     const unsigned int at = __ldcg(&p.ws.amax_acc[i]);
     const unsigned int ac = __ldcg(&p.ws.amax_acc[n + i]);
     const unsigned int av = __ldcg(&p.ws.amax_acc[2 * n + i]);

@@ -205,7 +205,7 @@ int kahan_sgd_destroy(ksgd_handle* h);
  *          k = ev_out - (e_out - s): the stored velocity on the compensation grid
  *     then T, P, Q_theta', Rq, Q_c' as in the plain step with this d.
  * The tensor descriptions are the same ksgd_tensor_desc (comp_bits must be 8 or 16) plus
- * one ksgd_momentum_desc per tensor.  At most 256 tensors per list.  Ownership, streams,
+ * one ksgd_momentum_desc per tensor.  Ownership, streams,
  * return codes and the meaning of the common outputs are as for the plain entry points;
  * mus: host array of momentum coefficients, finite and >= 0 (an invalid one gives
  * KSGD_ERR_LR).  amax_mom = max |V| of the last step, n_sat_mom = clamped velocity
@@ -255,9 +255,8 @@ int kahan_sgd_momentum_destroy(ksgd_momentum_handle* h);
  * A second moment below the resolution of its grid is taken as one unit of the grid, not as
  * zero (which would leave eps alone in the denominator and make the step m/eps): the step of
  * such an element is bounded by |m| / sqrt(2^ev_out).  The tensor descriptions are the same
- * ksgd_tensor_desc (comp_bits must be 8 or 16) plus one ksgd_adam_desc per tensor.  At most
- * 256 tensors per list.  Ownership, streams and return codes are as for the plain entry
- * points.  lrs: host array of lr_t per tensor, finite and > 0; beta1, beta2 in [0, 1], eps
+ * ksgd_tensor_desc (comp_bits must be 8 or 16) plus one ksgd_adam_desc per tensor.
+ * Ownership, streams and return codes are as for the plain entry points.  lrs: host array of lr_t per tensor, finite and > 0; beta1, beta2 in [0, 1], eps
  * finite and >= 0 (otherwise KSGD_ERR_LR).  kahan_sgd_adam_amax fills the non-NULL host
  * arrays of ksgd_adam_stats (n_tensors entries each): maxima of |P|, |Rq|, |M|, |V| of the
  * last step, the exponents now stored and those the next step writes, and the counts of

@@ -600,9 +600,33 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
 
 namespace {
 
+// Per-step arguments of a list longer than kInlineArgs: batches passed by value to the
+// upload kernel, which writes them into the workspace (second pass for the momentum
+// coefficients, which travel in the batch's lrs field).
+int upload_long_list(cudaStream_t stream, int32_t n, const float* const* grads, const float* lrs,
+                     const float* mus, const float** grad_ptr, float* lr, float* mu) {
+  UploadBatch* ub = new (std::nothrow) UploadBatch;
+  if (!ub) return KSGD_ERR_NULL;
+  for (int32_t first = 0; first < n; first += kUploadBatch) {
+    const int count = n - first < kUploadBatch ? n - first : kUploadBatch;
+    for (int i = 0; i < count; ++i) { ub->grads[i] = grads[first + i]; ub->lrs[i] = lrs[first + i]; }
+    ksgd_upload_args_kernel<<<1, 256, 0, stream>>>(*ub, first, count, grad_ptr, lr);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (mus) {
+      for (int i = 0; i < count; ++i) ub->lrs[i] = mus[first + i];
+      ksgd_upload_args_kernel<<<1, 256, 0, stream>>>(*ub, first, count, grad_ptr, mu);
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+  }
+  delete ub;
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "argument upload");
+  return KSGD_OK;
+}
+
 struct MomLayout {
   size_t exp_cur, exp_next, expv_cur, expv_next, amax_last, counters, error, stats_end;
-  size_t amax_acc, info, chunks, ticket, total;
+  size_t amax_acc, info, chunks, ticket, grad_ptr, lr, mu, total;
   long long n_chunks;
 };
 
@@ -628,6 +652,9 @@ MomLayout make_mom_layout(const ksgd_tensor_desc* d, int32_t n) {
   L.chunks = o;    o += sizeof(ChunkRef) * (size_t)chunks;
   o = align_up(o, 16);
   L.ticket = o;    o += 16;
+  L.grad_ptr = o;  o += sizeof(float*) * n;
+  L.lr = o;        o += sizeof(float) * n;
+  L.mu = o;        o += sizeof(float) * n;
   L.total = align_up(o, 256);
   return L;
 }
@@ -636,7 +663,6 @@ int validate_momentum(const ksgd_tensor_desc* d, const ksgd_momentum_desc* m, in
   const int v = validate(d, n);
   if (v != KSGD_OK) return v;
   if (!m) return KSGD_ERR_NULL;
-  if (n > kInlineArgs) return KSGD_ERR_NUMEL;
   for (int32_t i = 0; i < n; ++i) {
     if (d[i].comp_bits == 0) return KSGD_ERR_BITS;        // momentum goes through the lazy update
     if (m[i].mom_bits != 8 && m[i].mom_bits != 16) return KSGD_ERR_BITS;
@@ -729,9 +755,13 @@ int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* 
   w.info = reinterpret_cast<mom::TensorInfo*>(b + L.info);
   w.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
   w.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
+  w.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
+  w.lr = reinterpret_cast<float*>(b + L.lr);
+  w.mu = reinterpret_cast<float*>(b + L.mu);
   h->params.n_tensors = n_tensors;
   h->params.n_chunks = (int)L.n_chunks;
   h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
+  h->params.inline_args = n_tensors <= kInlineArgs ? 1 : 0;
 
   int dev = 0, sms = 0, l2_bytes = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -760,17 +790,20 @@ int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* 
 int kahan_sgd_momentum_step(ksgd_momentum_handle* h, const float* const* grads, const float* lrs,
                             const float* mus) {
   if (!h || !grads || !lrs || !mus) return KSGD_ERR_NULL;
-  mom::StepArgs args;
   for (int32_t i = 0; i < h->n; ++i) {
     if (!grads[i]) return KSGD_ERR_NULL;
     if (reinterpret_cast<uintptr_t>(grads[i]) % 16) return KSGD_ERR_ALIGN;
     if (!std::isfinite(lrs[i]) || !(lrs[i] > 0.0f)) return KSGD_ERR_LR;
     if (!std::isfinite(mus[i]) || !(mus[i] >= 0.0f)) return KSGD_ERR_LR;
-    args.grads[i] = grads[i];
-    args.lrs[i] = lrs[i];
-    args.mus[i] = mus[i];
   }
-  for (int32_t i = h->n; i < kInlineArgs; ++i) { args.grads[i] = nullptr; args.lrs[i] = 0.0f; args.mus[i] = 0.0f; }
+  mom::StepArgs args{};
+  if (h->params.inline_args) {
+    for (int32_t i = 0; i < h->n; ++i) { args.grads[i] = grads[i]; args.lrs[i] = lrs[i]; args.mus[i] = mus[i]; }
+  } else {
+    const int rc = upload_long_list(h->stream, h->n, grads, lrs, mus, h->params.ws.grad_ptr, h->params.ws.lr,
+                                    h->params.ws.mu);
+    if (rc != KSGD_OK) return rc;
+  }
   mom::ksgd_momentum_step_kernel<<<(unsigned)h->grid, mom::kBlock, mom::kSharedBytes, h->stream>>>(h->params,
                                                                                                   args);
   g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -821,7 +854,7 @@ namespace {
 
 struct AdamLayout {
   size_t exp_cur, exp_next, expm_cur, expm_next, expv_cur, expv_next, amax_last, counters, error, stats_end;
-  size_t amax_acc, info, chunks, ticket, total;
+  size_t amax_acc, info, chunks, ticket, grad_ptr, lr, total;
   long long n_chunks;
 };
 
@@ -849,6 +882,8 @@ AdamLayout make_adam_layout(const ksgd_tensor_desc* d, int32_t n) {
   L.chunks = o;    o += sizeof(ChunkRef) * (size_t)chunks;
   o = align_up(o, 16);
   L.ticket = o;    o += 16;
+  L.grad_ptr = o;  o += sizeof(float*) * n;
+  L.lr = o;        o += sizeof(float) * n;
   L.total = align_up(o, 256);
   return L;
 }
@@ -862,7 +897,6 @@ int validate_adam(const ksgd_tensor_desc* d, const ksgd_adam_desc* a, int32_t n)
   const int v = validate(d, n);
   if (v != KSGD_OK) return v;
   if (!a) return KSGD_ERR_NULL;
-  if (n > kInlineArgs) return KSGD_ERR_NUMEL;
   for (int32_t i = 0; i < n; ++i) {
     if (d[i].comp_bits == 0) return KSGD_ERR_BITS;        // ADAM goes through the lazy update
     if (!a[i].mom1 || !a[i].mom2) return KSGD_ERR_NULL;
@@ -956,9 +990,12 @@ int kahan_sgd_adam_init(ksgd_adam_handle** out, const ksgd_tensor_desc* descs, c
   w.info = reinterpret_cast<adam::TensorInfo*>(b + L.info);
   w.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
   w.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
+  w.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
+  w.lr = reinterpret_cast<float*>(b + L.lr);
   h->params.n_tensors = n_tensors;
   h->params.n_chunks = (int)L.n_chunks;
   h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
+  h->params.inline_args = n_tensors <= kInlineArgs ? 1 : 0;
 
   int dev = 0, sms = 0, l2_bytes = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -989,15 +1026,19 @@ int kahan_sgd_adam_step(ksgd_adam_handle* h, const float* const* grads, const fl
   if (!h || !grads || !lrs) return KSGD_ERR_NULL;
   if (!(beta1 >= 0.0f && beta1 <= 1.0f) || !(beta2 >= 0.0f && beta2 <= 1.0f)) return KSGD_ERR_LR;
   if (!std::isfinite(eps) || !(eps >= 0.0f)) return KSGD_ERR_LR;
-  adam::StepArgs args;
   for (int32_t i = 0; i < h->n; ++i) {
     if (!grads[i]) return KSGD_ERR_NULL;
     if (reinterpret_cast<uintptr_t>(grads[i]) % 16) return KSGD_ERR_ALIGN;
     if (!std::isfinite(lrs[i]) || !(lrs[i] > 0.0f)) return KSGD_ERR_LR;
-    args.grads[i] = grads[i];
-    args.lrs[i] = lrs[i];
   }
-  for (int32_t i = h->n; i < kInlineArgs; ++i) { args.grads[i] = nullptr; args.lrs[i] = 0.0f; }
+  adam::StepArgs args{};
+  if (h->params.inline_args) {
+    for (int32_t i = 0; i < h->n; ++i) { args.grads[i] = grads[i]; args.lrs[i] = lrs[i]; }
+  } else {
+    const int rc = upload_long_list(h->stream, h->n, grads, lrs, nullptr, h->params.ws.grad_ptr,
+                                    h->params.ws.lr, nullptr);
+    if (rc != KSGD_OK) return rc;
+  }
   args.beta1 = beta1;
   args.beta2 = beta2;
   args.eps = eps;

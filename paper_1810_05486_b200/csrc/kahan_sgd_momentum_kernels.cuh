@@ -40,6 +40,9 @@ struct Workspace {
   TensorInfo* info;                // [n]
   ChunkRef* chunks;                // [n_chunks]
   unsigned int* ticket;
+  const float** grad_ptr;          // [n] per-step arguments for lists longer than kInlineArgs
+  float* lr;                       // [n]
+  float* mu;                       // [n]
 };
 
 struct StepParams {
@@ -48,6 +51,7 @@ struct StepParams {
   int n_chunks;
   int amax_mode;
   int grad_evict_first;
+  int inline_args;                 // 1: grads/lrs/mus are in the StepArgs parameter
 };
 
 struct StepArgs {                  // per-step arguments, passed as a kernel parameter
@@ -371,9 +375,9 @@ __device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const StepA
   m.e_out = p.ws.exp_next[t];
   m.ev_in = p.ws.expv_cur[t];
   m.ev_out = p.ws.expv_next[t];
-  m.grad = a.grads[t];
-  m.lr = a.lrs[t];
-  m.mu = a.mus[t];
+  m.grad = p.inline_args ? a.grads[t] : p.ws.grad_ptr[t];
+  m.lr = p.inline_args ? a.lrs[t] : p.ws.lr[t];
+  m.mu = p.inline_args ? a.mus[t] : p.ws.mu[t];
   return m;
 }
 

@@ -233,3 +233,21 @@ def test_fast_path_division_and_square_root_equal_the_correctly_rounded_operatio
     """Exhaustive over the operands the fast path can meet (see the header)."""
     from paper_1810_05486_b200 import binding as B
     assert B.kahan_sgd_adam_selfcheck() == (0, 0)
+
+
+def test_a_list_longer_than_the_inline_argument_block():
+    """More than 256 tensors: gradients and step sizes reach the kernel through the workspace
+    instead of the kernel parameters."""
+    rng = np.random.default_rng(902)
+    n_t = 300
+    sizes = [int(x) for x in rng.integers(1, 3000, n_t)]
+    sizes[17], sizes[290] = 8192 * 2 + 5, 40000
+    specs, thetas, comps, m1s, m2s = [], [], [], [], []
+    for i, n in enumerate(sizes):
+        tb, cb = FORMATS[i % 4]
+        t, c, a, b = random_state(rng, n, tb, cb)
+        specs.append(dict(numel=n, theta_bits=tb, comp_bits=cb, exp_theta=-10, exp_m=-21, exp_v=-36))
+        thetas.append(t); comps.append(c); m1s.append(a); m2s.append(b)
+    grads = [[(rng.standard_normal(n) * 0.004).astype(np.float32) for n in sizes] for _ in range(3)]
+    lrs = [[float(x) for x in rng.choice([2.0 ** -12, 2.0 ** -11, 3e-4], n_t)] for _ in range(3)]
+    run_both(specs, thetas, comps, m1s, m2s, grads, lrs, 0.9, 0.999, 1e-8)

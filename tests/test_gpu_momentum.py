@@ -192,3 +192,22 @@ def test_resnet20_shapes_int8_momentum_and_alexnet_last_layers_int16_momentum():
     moms = [np.zeros(a.tensors[i].numel, np.int16) for i in pick]
     grads = [[W.grad_slice(a, i, s, 0, a.tensors[i].numel) for i in pick] for s in range(10)]
     run_both(specs, thetas, comps, moms, grads, [a.lr] * len(pick), [0.9] * len(pick))
+
+
+def test_a_list_longer_than_the_inline_argument_block():
+    """More than 256 tensors: gradients, step sizes and momentum coefficients reach the
+    kernel through the workspace instead of the kernel parameters."""
+    rng = np.random.default_rng(901)
+    n_t = 300
+    sizes = [int(x) for x in rng.integers(1, 3000, n_t)]
+    sizes[17], sizes[290] = 8192 * 2 + 5, 40000
+    specs, thetas, comps, moms = [], [], [], []
+    for i, n in enumerate(sizes):
+        tb, cb, vb = FORMATS[i % len(FORMATS)]
+        t, c, v = random_state(rng, n, tb, cb, vb)
+        specs.append(dict(numel=n, theta_bits=tb, comp_bits=cb, mom_bits=vb, exp_theta=-10, exp_mom=-17))
+        thetas.append(t); comps.append(c); moms.append(v)
+    grads = [[(rng.standard_normal(n) * 2.0 ** -17 * 400).astype(np.float32) for n in sizes] for _ in range(3)]
+    lrs = [float(x) for x in rng.choice([0.05, 0.1, 0.2], n_t)]
+    mus = [float(x) for x in rng.choice([0.0, 0.5, 0.9], n_t)]
+    run_both(specs, thetas, comps, moms, grads, lrs, mus)

@@ -110,6 +110,22 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
 int kahan_sgd_step(ksgd_handle* h, const float* const* grads, const float* lrs);
 
 /*
+ * The same step with the gradients given as dynamic fixed-point tensors, as the paper's
+ * 8-bit hardware model produces them (Section 1: every tensor of the training pass, the
+ * gradients included, is INT8 or INT16 with a shared exponent; Section 4.2: INT16 gradients
+ * before the last layer of AlexNet).  grads[i]: device, int8_t[numel] (grad_bits 8) or
+ * int16_t[numel] (16), 16-byte aligned, read only; exp_grad[i]: host array, the exponent of
+ * tensor i's gradient mantissas, in [-64, 64] (else KSGD_ERR_EXP_RANGE).  A gradient
+ * Q_g * 2^exp_grad is exact in binary32, and the step is by definition the plain step on
+ * that binary32 value: d = clamp(rne(fl32((Q_g * 2^exp_grad) * fl32(eta * 2^-(e_out - s)))));
+ * everything else as kahan_sgd_step.  Fixed-point gradients can be made from binary32
+ * ones with kahan_sgd_import (comp_bits 0, KSGD_EXP_AUTO picks the exponent from the
+ * maximum).  The gradient stream shrinks from 4 bytes per parameter to 1 or 2.
+ */
+int kahan_sgd_step_qgrad(ksgd_handle* h, const void* const* grads, int32_t grad_bits, const int32_t* exp_grad,
+                         const float* lrs);
+
+/*
  * The same step for callers whose tensors live in host memory: copies each tensor's
  * theta, comp and gradient from host to the device buffers named in the descs (and to
  * grad_staging), runs the step, copies theta and comp back and waits.  theta_host /

@@ -19,6 +19,8 @@ from .kahan_oracle import (  # noqa: F401
     oracle_adam_element,
     oracle_adam_step_tensor,
     oracle_adam_step,
+    oracle_dequantize_gradient,
+    oracle_step_qgrad,
     oracle_quantize,
     oracle_dequantize,
     OracleMomElem,

@@ -302,6 +302,20 @@ def oracle_step(state: OracleState, grads: Sequence[np.ndarray], lrs: Sequence[f
         t.exp_theta_next = oracle_next_exponent(t.amax_theta, t.theta_bits, e_out, state.mode)
 
 
+def oracle_dequantize_gradient(q: np.ndarray, exp_grad: int) -> np.ndarray:
+    """A fixed-point gradient tensor as binary32 values: Q * 2^exp_grad is exact for 8- and
+    16-bit mantissas and exponents in [-64, 64]."""
+    assert q.dtype in (np.int8, np.int16) and -64 <= exp_grad <= 64
+    return np.ldexp(q.astype(np.float32), np.int32(exp_grad)).astype(np.float32)
+
+
+def oracle_step_qgrad(state: OracleState, grads_q: Sequence[np.ndarray], exp_grads: Sequence[int],
+                      lrs: Sequence[float]) -> None:
+    """The step with gradients given in dynamic fixed point (the paper's hardware model,
+    Section 1): by definition the plain step on the exactly dequantized gradients."""
+    oracle_step(state, [oracle_dequantize_gradient(q, e) for q, e in zip(grads_q, exp_grads)], lrs)
+
+
 def oracle_momentum_step(state: OracleState, grads: Sequence[np.ndarray], lrs: Sequence[float],
                          mus: Sequence[float]) -> None:
     """One momentum step of every tensor, then the exponent choices: theta's exponent

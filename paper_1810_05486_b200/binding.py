@@ -28,7 +28,8 @@ KSGD_ERR_MODE = -10
 KSGD_ERR_DEVICE = -11
 
 EXPORTS = (
-    "kahan_sgd_workspace_bytes", "kahan_sgd_init", "kahan_sgd_step", "kahan_sgd_step_host",
+    "kahan_sgd_workspace_bytes", "kahan_sgd_init", "kahan_sgd_step", "kahan_sgd_step_qgrad",
+    "kahan_sgd_step_host",
     "kahan_sgd_amax", "kahan_sgd_set_exponents", "kahan_sgd_step_static", "kahan_sgd_destroy",
     "kahan_sgd_strerror", "kahan_sgd_momentum_workspace_bytes", "kahan_sgd_momentum_init",
     "kahan_sgd_momentum_step", "kahan_sgd_momentum_amax", "kahan_sgd_momentum_destroy",
@@ -85,6 +86,9 @@ def _load() -> ctypes.CDLL:
                                    ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
     lib.kahan_sgd_step.restype = ctypes.c_int
     lib.kahan_sgd_step.argtypes = [ctypes.c_void_p, P(ctypes.c_void_p), P(ctypes.c_float)]
+    lib.kahan_sgd_step_qgrad.restype = ctypes.c_int
+    lib.kahan_sgd_step_qgrad.argtypes = [ctypes.c_void_p, P(ctypes.c_void_p), ctypes.c_int32,
+                                         P(ctypes.c_int32), P(ctypes.c_float)]
     lib.kahan_sgd_step_host.restype = ctypes.c_int
     lib.kahan_sgd_step_host.argtypes = [ctypes.c_void_p, P(ctypes.c_void_p), P(ctypes.c_void_p),
                                         P(ctypes.c_void_p), P(ctypes.c_float), ctypes.c_void_p,
@@ -199,6 +203,14 @@ def kahan_sgd_step(h, grads, lrs) -> None:
     g = grads if isinstance(grads, ctypes.Array) else _ptr_array(grads)
     l = lrs if isinstance(lrs, ctypes.Array) else _float_array(lrs)
     _check(lib.kahan_sgd_step(h, g, l))
+
+
+def kahan_sgd_step_qgrad(h, grads, grad_bits: int, exp_grad, lrs) -> None:
+    """grads: device addresses of int8 / int16 gradient mantissas; exp_grad: their exponents."""
+    g = grads if isinstance(grads, ctypes.Array) else _ptr_array(grads)
+    e = exp_grad if isinstance(exp_grad, ctypes.Array) else (ctypes.c_int32 * len(exp_grad))(*exp_grad)
+    l = lrs if isinstance(lrs, ctypes.Array) else _float_array(lrs)
+    _check(lib.kahan_sgd_step_qgrad(h, g, grad_bits, e, l))
 
 
 def kahan_sgd_step_host(h, theta_host, comp_host, grads_host, lrs, grad_staging: int,

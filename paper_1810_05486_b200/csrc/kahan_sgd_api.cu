@@ -40,7 +40,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // kahan_sgd_amax fetches them with one copy.
 struct Layout {
   size_t exp_cur, exp_next, amax_last, counters, error, stats_end;
-  size_t amax_acc, info, grad_ptr, lr, chunks, ticket, total;
+  size_t amax_acc, info, grad_ptr, lr, exp_grad, chunks, ticket, total;
   long long n_chunks;
 };
 
@@ -62,6 +62,7 @@ Layout make_layout(const ksgd_tensor_desc* d, int32_t n) {
   L.info = o;      o += sizeof(TensorInfo) * n;
   L.grad_ptr = o;  o += sizeof(const float*) * n;
   L.lr = o;        o += sizeof(float) * n;
+  L.exp_grad = o;  o += sizeof(int) * n;
   o = align_up(o, 16);
   L.chunks = o;    o += sizeof(ChunkRef) * (size_t)chunks;
   o = align_up(o, 16);
@@ -176,6 +177,7 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
   w.info = reinterpret_cast<TensorInfo*>(b + L.info);
   w.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
   w.lr = reinterpret_cast<float*>(b + L.lr);
+  w.exp_grad = reinterpret_cast<int*>(b + L.exp_grad);
   w.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
   w.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
   h->params.n_tensors = n_tensors;
@@ -194,6 +196,12 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, dev);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(ksgd_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSharedBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(ksgd_step_qgrad_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSharedBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(ksgd_step_qgrad_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)kSharedBytes);
   if (e != cudaSuccess) {
     delete h;
@@ -265,6 +273,52 @@ static int launch_step(ksgd_handle* h, const float* const* grads, const float* l
     KSGD_CUDA(cudaGetLastError());
   }
   ksgd_step_kernel<<<(unsigned)h->grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, *ia);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  KSGD_CUDA(cudaGetLastError());
+  return KSGD_OK;
+}
+
+int kahan_sgd_step_qgrad(ksgd_handle* h, const void* const* grads, int32_t grad_bits, const int32_t* exp_grad,
+                         const float* lrs) {
+  if (!h || !grads || !exp_grad || !lrs) return KSGD_ERR_NULL;
+  if (grad_bits != 8 && grad_bits != 16) return KSGD_ERR_BITS;
+  for (int32_t i = 0; i < h->n; ++i) {
+    if (!grads[i]) return KSGD_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(grads[i]) % 16) return KSGD_ERR_ALIGN;
+    if (exp_grad[i] < kExpMin || exp_grad[i] > kExpMax) return KSGD_ERR_EXP_RANGE;
+    if (!std::isfinite(lrs[i]) || !(lrs[i] > 0.0f)) return KSGD_ERR_LR;
+  }
+  QGradArgs args{};
+  if (h->params.inline_args) {
+    for (int32_t i = 0; i < h->n; ++i) {
+      args.grads[i] = grads[i];
+      args.lrs[i] = lrs[i];
+      args.exp_grad[i] = (signed char)exp_grad[i];
+    }
+  } else {
+    UploadBatch* ub = new (std::nothrow) UploadBatch;
+    ExponentBatch* eb = new (std::nothrow) ExponentBatch;
+    if (!ub || !eb) { delete ub; delete eb; return KSGD_ERR_NULL; }
+    for (int32_t first = 0; first < h->n; first += kUploadBatch) {
+      const int count = h->n - first < kUploadBatch ? h->n - first : kUploadBatch;
+      for (int i = 0; i < count; ++i) {
+        ub->grads[i] = static_cast<const float*>(grads[first + i]);   // only the address travels
+        ub->lrs[i] = lrs[first + i];
+        eb->exp_next[i] = exp_grad[first + i];
+      }
+      ksgd_upload_args_kernel<<<1, 256, 0, h->stream>>>(*ub, first, count, h->params.ws.grad_ptr,
+                                                        h->params.ws.lr);
+      ksgd_upload_ints_kernel<<<1, 256, 0, h->stream>>>(*eb, first, count, h->params.ws.exp_grad);
+      g_launches.fetch_add(2, std::memory_order_relaxed);
+    }
+    delete ub;
+    delete eb;
+    KSGD_CUDA(cudaGetLastError());
+  }
+  if (grad_bits == 8)
+    ksgd_step_qgrad_kernel<8><<<(unsigned)h->grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, args);
+  else
+    ksgd_step_qgrad_kernel<16><<<(unsigned)h->grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, args);
   g_launches.fetch_add(1, std::memory_order_relaxed);
   KSGD_CUDA(cudaGetLastError());
   return KSGD_OK;
@@ -555,6 +609,7 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   params.ws.info = reinterpret_cast<TensorInfo*>(b + L.info);
   params.ws.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
   params.ws.lr = reinterpret_cast<float*>(b + L.lr);
+  params.ws.exp_grad = reinterpret_cast<int*>(b + L.exp_grad);
   params.ws.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
   params.ws.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
   params.n_tensors = n_tensors;

@@ -70,6 +70,7 @@ struct Workspace {
   TensorInfo* info;                // [n]
   const float** grad_ptr;          // [n] per-step arguments for lists longer than kInlineArgs
   float* lr;                       // [n]
+  int* exp_grad;                   // [n] the same, exponents of fixed-point gradients
   ChunkRef* chunks;                // [n_chunks]
   unsigned int* ticket;            // blocks finished in the running step
 };
@@ -93,6 +94,14 @@ struct InlineArgs {
   float lrs[kInlineArgs];
 };
 
+// Per-step arguments when the gradients are dynamic fixed-point tensors themselves (8- or
+// 16-bit mantissas, one exponent per tensor).
+struct QGradArgs {
+  const void* grads[kInlineArgs];
+  float lrs[kInlineArgs];
+  signed char exp_grad[kInlineArgs];
+};
+
 struct UploadBatch {
   const float* grads[kUploadBatch];
   float lrs[kUploadBatch];
@@ -114,12 +123,14 @@ struct StepCoef {
   int r_c;       // fine grid -> comp output grid (rounding shift)
   int qmax_t;    // 2^(m-1) - 1
   int qmax_c;    // 2^(n-1) - 1
+  int gb;        // gradient storage: 32 = binary32, 8 / 16 = fixed-point mantissas
+  int eg;        // exponent of fixed-point gradient mantissas (0 for binary32)
 };
 
 // One tile as the producer describes it to the consumers (lives in shared memory).  The
 // first 48 bytes are all the steady-state path reads (three 16-byte loads).
 struct __align__(16) TileDesc {
-  float scale;          // lr * 2^-(e_out - s)
+  float scale;          // lr * 2^-(e_out - s), times 2^eg for fixed-point gradients
   float pow2s_neg;      // -2^s
   float inv2s;          // 2^-s
   float qmax_t;         // 2^(m-1) - 1
@@ -130,7 +141,7 @@ struct __align__(16) TileDesc {
   int count;            // valid elements in the tile
   int flags;            // kFlag* | format id
   StepCoef coef;        // for the general path
-  const float* grad;    // global address of the tile's first gradient
+  const void* grad;     // global address of the tile's first gradient
 };
 constexpr int kFlagFormatMask = 7;   // 0..5 = (8,0) (8,8) (8,16) (16,0) (16,8) (16,16)
 constexpr int kFlagSteady = 8;       // no exponent change: the exact-fp32 path applies
@@ -245,8 +256,11 @@ __device__ __forceinline__ int quantize_increment(float g, float scale) {
   return max(min(d, kDLimit), -kDLimit);
 }
 
-__device__ __forceinline__ StepCoef make_coef(const TensorInfo& ti, int e_in, int e_out, float lr) {
+__device__ __forceinline__ StepCoef make_coef(const TensorInfo& ti, int e_in, int e_out, float lr, int gb,
+                                              int eg) {
   StepCoef k;
+  k.gb = gb;
+  k.eg = eg;
   const int delta = e_out - e_in;
   k.s = ti.s;
   k.delta = delta;
@@ -267,7 +281,7 @@ __device__ __forceinline__ StepCoef make_coef(const TensorInfo& ti, int e_in, in
 // large), and ragged tails.  It is kept out of line, one copy for all formats, so that it
 // costs the steady-state path no registers.
 __device__ __noinline__ void update_general(const StepCoef* coef, int tb, int cb, void* theta,
-                                            void* comp, const float* grad, int first, int n,
+                                            void* comp, const void* grad, int first, int n,
                                             TileScan* slots) {
   const StepCoef k = *coef;
   unsigned int amax_t = 0, amax_c = 0, n_sat_t = 0, n_sat_c = 0, n_nf = 0;
@@ -278,7 +292,10 @@ __device__ __noinline__ void update_general(const StepCoef* coef, int tb, int cb
     int qc = 0;
     if (cb == 8) qc = (int)static_cast<const signed char*>(comp)[e];
     else if (cb == 16) qc = (int)static_cast<const short*>(comp)[e];
-    const float g = grad[e];
+    float g;       // a fixed-point gradient Q * 2^eg is exact in binary32
+    if (k.gb == 32) g = static_cast<const float*>(grad)[e];
+    else if (k.gb == 8) g = __fmul_rn((float)static_cast<const signed char*>(grad)[e], pow2_float(k.eg));
+    else g = __fmul_rn((float)static_cast<const short*>(grad)[e], pow2_float(k.eg));
     const int d = quantize_increment(g, k.scale);
     const long long T = (long long)qt * (1LL << k.sh_t) + (long long)qc * (1LL << k.sh_c) -
                         (long long)d * (1LL << k.sh_d);
@@ -441,9 +458,9 @@ struct TileHot {       // the consumers' copy of the first 48 bytes of a TileDes
   int tensor, n_bulk, count, flags;
 };
 
-template <int TB, int CB, int V>
+template <int TB, int CB, int V, int GB>
 __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V * CB / 8 : 8)> pc,
-                                              const Pack<V * 4>& pg, const SteadyCoef& k,
+                                              Pack<V * GB / 8> pg, const SteadyCoef& k,
                                               Pack<V * TB / 8>& ot, Pack<(CB ? V * CB / 8 : 8)>& oc,
                                               float& amax_t, float& amax_c) {
   constexpr bool HAS_COMP = CB != 0;
@@ -451,12 +468,15 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
   constexpr float bias_c = HAS_COMP ? (float)(1 << ((CB ? CB : 8) - 1)) : 0.0f;
   flip_signs<TB>(pt);
   if constexpr (HAS_COMP) flip_signs<(CB ? CB : 8)>(pc);
+  if constexpr (GB != 32) flip_signs<(GB == 32 ? 8 : GB)>(pg);
   float Pm[V], rm[V];
   float sum_abs = 0.0f, aX = 0.0f, aP = 0.0f, aR = 0.0f;
 #pragma unroll
   for (int i = 0; i < V; ++i) {
     const float qtM = __fadd_rn(magic_elem<TB>(pt, i), -bias_t);
-    const float g = __uint_as_float(pack_word(pg, i));
+    float g;       // binary32 gradient, or the gradient mantissa (k.scale then carries 2^eg)
+    if constexpr (GB == 32) g = __uint_as_float(pack_word(pg, i));
+    else g = __fadd_rn(magic_elem<(GB == 32 ? 8 : GB)>(pg, i), -(kMagic + (float)(1 << ((GB == 32 ? 8 : GB) - 1))));
     const float x = __fmul_rn(g, k.scale);              // the one binary32 multiply
     sum_abs = __fadd_rn(sum_abs, fabsf(x));             // Inf or NaN if any x is
     aX = fmaxf(aX, fabsf(x));
@@ -482,18 +502,18 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
 
 // All vectors of one tile that belong to this consumer thread (V consecutive elements,
 // 16 bytes of theta, per vector).  Returns true if the general path wrote into the stage.
-template <int TB, int CB>
+template <int TB, int CB, int GB>
 __device__ __forceinline__ bool consume_tile(const TileHot& h, const TileDesc* td, unsigned char* ring,
                                              int ctid, TileScan* slots, float& amax_t, float& amax_c) {
   constexpr bool HAS_COMP = CB != 0;
   constexpr int V = (TB == 8) ? 16 : 8;
   constexpr int TBYTES = V * TB / 8;
   constexpr int CBYTES = HAS_COMP ? V * CB / 8 : 8;
+  constexpr int GBYTES = V * GB / 8;
   const bool steady = (h.flags & kFlagSteady) != 0;
   unsigned char* theta_s = ring + ((h.flags >> kFlagThetaPageShift) & 31) * kPageBytes;
   unsigned char* comp_s = ring + ((h.flags >> kFlagCompPageShift) & 31) * kPageBytes;
-  const float* grad_s =
-      reinterpret_cast<const float*>(ring + ((h.flags >> kFlagGradPageShift) & 31) * kPageBytes);
+  const unsigned char* grad_s = ring + ((h.flags >> kFlagGradPageShift) & 31) * kPageBytes;
   bool wrote_stage = false;
   const int n_vec = h.n_bulk / V;
   for (int v = ctid; v < n_vec; v += kConsumers) {
@@ -504,8 +524,8 @@ __device__ __forceinline__ bool consume_tile(const TileHot& h, const TileDesc* t
       const Pack<TBYTES> pt = load_pack<TBYTES>(theta_s + v * TBYTES);
       Pack<CBYTES> pc{};
       if constexpr (HAS_COMP) pc = load_pack<CBYTES>(comp_s + v * CBYTES);
-      const Pack<V * 4> pg = load_pack<V * 4>(grad_s + v * V);
-      done = update_vector<TB, CB, V>(pt, pc, pg, h.k, ot, oc, amax_t, amax_c);
+      const Pack<GBYTES> pg = load_pack<GBYTES>(grad_s + v * GBYTES);
+      done = update_vector<TB, CB, V, GB>(pt, pc, pg, h.k, ot, oc, amax_t, amax_c);
     }
     if (!done) {
       // general path, in place in the stage; then the vector goes out like any other
@@ -601,9 +621,10 @@ __device__ __forceinline__ void take_back(const StepParams& p, ScanAcc& acc, Til
 // What the producer reads about a tile's tensor, fetched one tile ahead.
 struct TensorMeta {
   TensorInfo ti;
-  const float* grad;
+  const void* grad;
   float lr;
   int e_in, e_out;
+  int eg;          // exponent of a fixed-point gradient, 0 for binary32
 };
 
 __device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const InlineArgs& a, int t) {
@@ -613,11 +634,25 @@ __device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const Inlin
   m.e_out = p.ws.exp_next[t];
   m.grad = p.inline_args ? a.grads[t] : p.ws.grad_ptr[t];
   m.lr = p.inline_args ? a.lrs[t] : p.ws.lr[t];
+  m.eg = 0;
   return m;
 }
 
-__global__ void __launch_bounds__(kBlockThreads, 1)
-ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ InlineArgs a) {
+__device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const QGradArgs& a, int t) {
+  TensorMeta m;
+  m.ti = p.ws.info[t];
+  m.e_in = p.ws.exp_cur[t];
+  m.e_out = p.ws.exp_next[t];
+  m.grad = p.inline_args ? a.grads[t] : static_cast<const void*>(p.ws.grad_ptr[t]);
+  m.lr = p.inline_args ? a.lrs[t] : p.ws.lr[t];
+  m.eg = p.inline_args ? (int)a.exp_grad[t] : p.ws.exp_grad[t];
+  return m;
+}
+
+// The whole step.  GB = 32: binary32 gradients; 8 / 16: fixed-point gradients (one or two
+// bytes per parameter instead of four on the gradient stream).
+template <int GB, typename Args>
+__device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
   extern __shared__ __align__(128) unsigned char smem[];
   BlockShared* sh = reinterpret_cast<BlockShared*>(smem + (size_t)kPages * kPageBytes);
 
@@ -670,7 +705,8 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
         const int tbytes = ti.theta_bits >> 3, cbytes = ti.comp_bits >> 3;
         // where the three arrays go (g, theta, c), and how many pages that takes including
         // those skipped when a run does not fit before the end of the ring
-        const int run[3] = {kChunk * 4 / kPageBytes, kChunk * tbytes / kPageBytes, kChunk * cbytes / kPageBytes};
+        constexpr int gbytes = GB / 8;
+        const int run[3] = {kChunk * gbytes / kPageBytes, kChunk * tbytes / kPageBytes, kChunk * cbytes / kPageBytes};
         int page[3] = {0, 0, 0}, h2 = head, need = 0;
 #pragma unroll
         for (int r = 0; r < 3; ++r) {
@@ -701,13 +737,22 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
         free_pages -= need;
         sh->slot_pages[slot] = need;
 
-        const StepCoef coef = make_coef(ti, meta.e_in, meta.e_out, meta.lr);
+        const StepCoef coef = make_coef(ti, meta.e_in, meta.e_out, meta.lr, GB, meta.eg);
+        // fixed-point gradients: the exact-fp32 path multiplies the mantissa by scale * 2^eg,
+        // which must itself be exact (a normal number); otherwise the tile takes the general path
+        float scale_hot = coef.scale;
+        bool scale_ok = true;
+        if constexpr (GB != 32) {
+          const int ex = (int)((__float_as_uint(coef.scale) >> 23) & 0xffu);
+          scale_ok = ex != 0 && ex + meta.eg >= 1 && ex + meta.eg <= 254;
+          if (scale_ok) scale_hot = __int_as_float(__float_as_int(coef.scale) + (meta.eg << 23));
+        }
         const long long first = (long long)cr.index * kChunk;
         const long long left = ti.numel - first;
         const int count = left < (long long)kChunk ? (int)left : kChunk;
         const int n_bulk = count & ~15;
         TileDesc& td = sh->desc[slot];
-        td.scale = coef.scale;
+        td.scale = scale_hot;
         td.pow2s_neg = -pow2_float(coef.s);
         td.inv2s = pow2_float(-coef.s);
         td.qmax_t = (float)coef.qmax_t;
@@ -717,22 +762,22 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
         td.n_bulk = n_bulk;
         td.count = count;
         td.flags = ((ti.theta_bits == 16 ? 3 : 0) + (ti.comp_bits >> 3)) |
-                   (coef.delta == 0 ? kFlagSteady : 0) | (page[1] << kFlagThetaPageShift) |
+                   ((coef.delta == 0 && scale_ok) ? kFlagSteady : 0) | (page[1] << kFlagThetaPageShift) |
                    (page[2] << kFlagCompPageShift) | (page[0] << kFlagGradPageShift);
         td.coef = coef;
-        td.grad = meta.grad + first;
+        td.grad = static_cast<const unsigned char*>(meta.grad) + first * gbytes;
         if (n_bulk > 0) {
-          mbar_arrive_expect_tx(&sh->full[slot], (unsigned)(n_bulk * (tbytes + cbytes + 4)));
+          mbar_arrive_expect_tx(&sh->full[slot], (unsigned)(n_bulk * (tbytes + cbytes + gbytes)));
           bulk_load(smem + page[1] * kPageBytes, td.theta, (unsigned)(n_bulk * tbytes), &sh->full[slot]);
           if (cbytes)
             bulk_load(smem + page[2] * kPageBytes, td.comp, (unsigned)(n_bulk * cbytes), &sh->full[slot]);
           // Gradients are read once.  When theta and c of the whole list fit in L2, letting
           // the gradients leave it first keeps the state resident from step to step.
           if (p.grad_evict_first)
-            bulk_load_hint(smem + page[0] * kPageBytes, td.grad, (unsigned)(n_bulk * 4), &sh->full[slot],
+            bulk_load_hint(smem + page[0] * kPageBytes, td.grad, (unsigned)(n_bulk * gbytes), &sh->full[slot],
                            grad_policy);
           else
-            bulk_load(smem + page[0] * kPageBytes, td.grad, (unsigned)(n_bulk * 4), &sh->full[slot]);
+            bulk_load(smem + page[0] * kPageBytes, td.grad, (unsigned)(n_bulk * gbytes), &sh->full[slot]);
         } else {
           mbar_arrive(&sh->full[slot]);
         }
@@ -787,12 +832,12 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
       unsigned char* st = smem;
       bool wrote_stage;
       switch (h.flags & kFlagFormatMask) {
-        case 0: wrote_stage = consume_tile<8, 0>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        case 1: wrote_stage = consume_tile<8, 8>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        case 2: wrote_stage = consume_tile<8, 16>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        case 3: wrote_stage = consume_tile<16, 0>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        case 4: wrote_stage = consume_tile<16, 8>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        default: wrote_stage = consume_tile<16, 16>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 0: wrote_stage = consume_tile<8, 0, GB>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 1: wrote_stage = consume_tile<8, 8, GB>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 2: wrote_stage = consume_tile<8, 16, GB>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 3: wrote_stage = consume_tile<16, 0, GB>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 4: wrote_stage = consume_tile<16, 8, GB>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        default: wrote_stage = consume_tile<16, 16, GB>(h, td, st, ctid, scan, amax_t, amax_c); break;
       }
       add_warp_scans(scan, lane, amax_t, amax_c);
       // if the general path wrote into the stage, order those writes before the bulk copy
@@ -830,6 +875,17 @@ ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ I
   if (threadIdx.x == 0) *p.ws.ticket = 0u;
 }
 
+__global__ void __launch_bounds__(kBlockThreads, 1)
+ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ InlineArgs a) {
+  step_body<32>(p, a);
+}
+
+template <int GB>
+__global__ void __launch_bounds__(kBlockThreads, 1)
+ksgd_step_qgrad_kernel(const __grid_constant__ StepParams p, const __grid_constant__ QGradArgs a) {
+  step_body<GB>(p, a);
+}
+
 // Per-step arguments of long lists: written to the workspace from kernel parameters.
 __global__ void ksgd_upload_args_kernel(const __grid_constant__ UploadBatch b, int first, int count,
                                         const float** grad_ptr, float* lr) {
@@ -837,6 +893,11 @@ __global__ void ksgd_upload_args_kernel(const __grid_constant__ UploadBatch b, i
     grad_ptr[first + i] = b.grads[i];
     lr[first + i] = b.lrs[i];
   }
+}
+
+__global__ void ksgd_upload_ints_kernel(const __grid_constant__ ExponentBatch b, int first, int count,
+                                       int* dst) {
+  for (int i = threadIdx.x; i < count; i += blockDim.x) dst[first + i] = b.exp_next[i];
 }
 
 // Caller-chosen exponents for the coming step, limited to kMaxDelta around the current one.

@@ -90,6 +90,19 @@ class LibraryRun:
             self.grad_arena.upload(i, g)
         self.B.kahan_sgd_step(self.handle, self.grad_ptrs, list(lrs))
 
+    def step_qgrad(self, grads_q: Sequence[np.ndarray], exp_grads: Sequence[int],
+                   lrs: Sequence[float]) -> None:
+        """Fixed-point gradients (all int8 or all int16), in a guarded arena of their own."""
+        bits = 8 * grads_q[0].dtype.itemsize
+        if getattr(self, "qgrad_arena", None) is None:
+            self.qgrad_arena = DeviceArena([s["numel"] * 2 for s in self.specs])
+        for i, g in enumerate(grads_q):
+            assert g.dtype == storage_dtype(bits) and g.size == self.specs[i]["numel"]
+            self.qgrad_arena.sizes[i] = g.nbytes
+            self.qgrad_arena.upload(i, g)
+        self.B.kahan_sgd_step_qgrad(self.handle, [self.qgrad_arena.ptr(i) for i in range(self.n)], bits,
+                                    [int(e) for e in exp_grads], list(lrs))
+
     def set_exponents(self, exps: Sequence[int]) -> None:
         self.B.kahan_sgd_set_exponents(self.handle, list(exps))
 
@@ -108,8 +121,10 @@ class LibraryRun:
 
     def guards_intact(self) -> bool:
         self.torch.cuda.synchronize()
-        return (self.theta_arena.guards_intact() and self.comp_arena.guards_intact()
-                and self.grad_arena.guards_intact())
+        arenas = [self.theta_arena, self.comp_arena, self.grad_arena]
+        if getattr(self, "qgrad_arena", None) is not None:
+            arenas.append(self.qgrad_arena)
+        return all(a.guards_intact() for a in arenas)
 
     def close(self) -> None:
         if self.handle is not None:

@@ -89,6 +89,9 @@ def parse_args():
     ap.add_argument("--adam", action="store_true",
                     help="time ADAM (beta1 0.9, beta2 0.999, eps 1e-8, two int16 moment tensors; the step "
                          "size is 1e-3 of the first tensor's range)")
+    ap.add_argument("--grad-bits", type=int, default=32, choices=[8, 16, 32],
+                    help="8 or 16: the gradients are fixed-point tensors of that width (made on the device "
+                         "from the binary32 ones before the timed region)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-buckets", action="store_true",
@@ -201,8 +204,8 @@ def run_ours(args, rank, world, local_rank):
         t0_ = wl.tensors[0]
         adam = dict(beta1=0.9, beta2=0.999, eps=1e-8,
                     eta=1e-3 * 2.0 ** t0_.exp_theta * (2 ** (t0_.theta_bits - 1) - 1))
-    run = DeviceRun(host, B.KSGD_EXP_AMAX, mom_bits=args.momentum_bits, adam=adam)
-    other = bool(args.momentum_bits or args.adam)
+    run = DeviceRun(host, B.KSGD_EXP_AMAX, mom_bits=args.momentum_bits, adam=adam, grad_bits=args.grad_bits)
+    other = bool(args.momentum_bits or args.adam or args.grad_bits != 32)
     if other:
         args.no_e2e = args.no_cpu_baseline = True      # those legs describe the plain step
     stream = run.stream
@@ -297,7 +300,8 @@ def run_ours(args, rank, world, local_rank):
         "config": {"workload": wl.name, "tensors": n, "parameters": wl.numel,
                    "bytes_per_step": run.bytes_per_step, "grad_sets": n_sets,
                    "optimizer": "momentum 0.9, int%d velocity" % args.momentum_bits if args.momentum_bits
-                   else ("adam 0.9/0.999/1e-8, int16 moments" if args.adam else "sgd"),
+                   else ("adam 0.9/0.999/1e-8, int16 moments" if args.adam else
+                         ("sgd" if args.grad_bits == 32 else "sgd, int%d gradients" % args.grad_bits)),
                    "l2": "inputs larger than L2 (%.0f MB touched per step)" % (wl.bytes_per_step / 1e6),
                    "exponent_mode": "amax", "input_generation_s": round(gen_s, 1)},
         "achieved_hbm_gbs": achieved,
@@ -305,7 +309,8 @@ def run_ours(args, rank, world, local_rank):
                      "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                      "frac_of_nominal_8000": achieved / 8000.0,
                      "kernel": "ksgd_momentum_step_kernel" if args.momentum_bits
-                     else ("ksgd_adam_step_kernel" if args.adam else "ksgd_step_kernel"),
+                     else ("ksgd_adam_step_kernel" if args.adam else
+                           ("ksgd_step_kernel" if args.grad_bits == 32 else "ksgd_step_qgrad_kernel")),
                      "launch_ms": ms_step},
         "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
         "counters": {"n_sat_theta": int(sum(stats["n_sat_theta"])),

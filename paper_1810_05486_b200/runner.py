@@ -54,12 +54,14 @@ class DeviceRun:
     """Device buffers (same layout as HostInputs), descriptors, workspace and handle."""
 
     def __init__(self, host: HostInputs, mode: int = B.KSGD_EXP_AMAX, stream=None,
-                 mom_bits: int = 0, mu: float = 0.9, adam: Optional[dict] = None):
+                 mom_bits: int = 0, mu: float = 0.9, adam: Optional[dict] = None, grad_bits: int = 32):
         """mom_bits = 8 or 16 selects the momentum optimizer (velocity buffers start at zero,
         on a grid 8 binades below theta's).  adam = dict(beta1, beta2, eps, eta) selects ADAM
         (both 16-bit moments start at zero, on grids that just hold what the first step makes of
         the largest gradient of the first set; the step size carries the bias correction of the
-        step count)."""
+        step count).  grad_bits = 8 or 16 (plain optimizer only): every resident gradient set is
+        turned into fixed-point tensors of that width on the device (exponent from the tensor's
+        maximum) and the steps read those."""
         import torch
         self.torch = torch
         self.host = host
@@ -116,6 +118,22 @@ class DeviceRun:
                                            self.ws_bytes, self.stream.cuda_stream)
         self.grad_ptr_sets = [(ctypes.c_void_p * self.n)(*[g.data_ptr() + o for o in host.g_offs])
                               for g in self.dev_g]
+        self.grad_bits = grad_bits
+        if grad_bits != 32:
+            assert grad_bits in (8, 16) and not mom_bits and not adam
+            self.q_offs, q_bytes = _carve(wl, lambda t: grad_bits // 8)
+            scratch = torch.zeros(64, dtype=torch.uint8, device="cuda")
+            self.dev_gq, self.gq_ptr_sets, self.gq_exp_sets = [], [], []
+            for gset in self.dev_g:
+                q = torch.zeros(q_bytes, dtype=torch.uint8, device="cuda")
+                exps = [B.kahan_sgd_import(gset.data_ptr() + host.g_offs[i], q.data_ptr() + self.q_offs[i], None,
+                                           t.numel, grad_bits, 0, 0, B.KSGD_EXP_AUTO, scratch.data_ptr(),
+                                           self.stream.cuda_stream) for i, t in enumerate(wl.tensors)]
+                self.dev_gq.append(q)
+                self.gq_ptr_sets.append((ctypes.c_void_p * self.n)(*[q.data_ptr() + o for o in self.q_offs]))
+                self.gq_exp_sets.append((ctypes.c_int32 * self.n)(*exps))
+            self.dev_g = self.dev_g[:1]            # the binary32 copies are no longer needed
+            torch.cuda.empty_cache()
         self.lrs = (ctypes.c_float * self.n)(*([wl.lr] * self.n))
 
     def adam_lrs(self, t: int):
@@ -133,6 +151,9 @@ class DeviceRun:
                                   self.adam["beta1"], self.adam["beta2"], self.adam["eps"])
         elif self.mom_bits:
             B.kahan_sgd_momentum_step(self.handle, self.grad_ptr_sets[grad_set], self.lrs, self.mus)
+        elif self.grad_bits != 32:
+            B.kahan_sgd_step_qgrad(self.handle, self.gq_ptr_sets[grad_set], self.grad_bits,
+                                   self.gq_exp_sets[grad_set], self.lrs)
         else:
             B.kahan_sgd_step(self.handle, self.grad_ptr_sets[grad_set], self.lrs)
 
@@ -148,6 +169,8 @@ class DeviceRun:
         """Algorithmic HBM bytes of one step, velocity or moments included."""
         if self.adam:
             return self.wl.bytes_per_step + 8 * self.wl.numel
+        if self.grad_bits != 32:
+            return self.wl.bytes_per_step - (4 - self.grad_bits // 8) * self.wl.numel
         return self.wl.bytes_per_step + 2 * (self.mom_bits // 8) * self.wl.numel
 
     def theta(self, i: int) -> np.ndarray:

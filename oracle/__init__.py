@@ -20,6 +20,11 @@ from .kahan_oracle import (  # noqa: F401
     oracle_adam_step_tensor,
     oracle_adam_step,
     oracle_dequantize_gradient,
+    OracleStrictElem,
+    oracle_strict_element,
+    oracle_strict_step_tensor,
+    oracle_strict_step,
+    oracle_next_exponent_acc,
     oracle_step_qgrad,
     oracle_quantize,
     oracle_dequantize,

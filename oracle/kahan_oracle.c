@@ -520,6 +520,104 @@ int ksgd_oracle_adam_step_tensor(void* theta, void* comp, int16_t* mom1, int16_t
 }
 
 /* ------------------------------------------------------------------------------------
+ * Strict Algorithm 1: every statement rounds into the stored format, and the accumulator
+ * is a dynamic fixed-point tensor of its own -- n-bit mantissas with an exponent that
+ * follows the accumulator's maximum, not theta's exponent (Section 2: acc is an n-bit
+ * tensor below theta, Figure 1; Section 5: exponents from a scan of the maximum).  The
+ * overlap k is then not a parameter but a result, k = n - 1 - (e - e_acc).
+ * As everywhere here the tensor stored is c = -acc.  With f the smallest of the four
+ * exponents (theta's and c's, each read at *_in and written at *_out):
+ *   d   = clamp(rne(fl(g * fl(lr * 2^-ec_out))), +-2^30)              the increment on c's grid
+ *   C1  = rne((Q_c * 2^(ec_in-f) - d * 2^(ec_out-f)) / 2^(ec_out-f))  statement 1: acc += eta g
+ *   Qc1 = clamp(C1, +-QMAX_n)                                         ... stored in n bits
+ *   T   = Q_theta * 2^(e_in-f) + Qc1 * 2^(ec_out-f)                   statement 2: theta - acc
+ *   P   = rne(T / 2^(e_out-f)),  Q_theta' = clamp(P, +-QMAX_m)        ... stored in m bits
+ *   C2  = rne((T - Q_theta' * 2^(e_out-f)) / 2^(ec_out-f))            statement 3: acc += theta_u - theta
+ *   Q_c' = clamp(C2, +-QMAX_n)                                        ... stored in n bits
+ * Scans: max |P| for theta, max(|C1|, |C2|) for c (so that an increment too large for the
+ * accumulator raises its exponent), each capped at 2^31 - 1.
+ * Exponents must satisfy  -8 <= e - ec <= 36  at both ends of the step (the sums then fit
+ * in 64 bits); the policy keeps them there.
+ */
+typedef struct {
+  int64_t C1, T, P, C2;
+  int32_t d, q_comp_mid, q_theta, q_comp, nonfinite;
+} ksgd_oracle_strict_elem;
+
+static int64_t rne_div_pow2(int64_t a, int r) { return r == 0 ? a : ksgd_oracle_rne_shift(a, r); }
+
+void ksgd_oracle_strict_element(int32_t q_theta, int32_t q_comp, float g, float lr, int32_t m, int32_t n,
+                                int32_t e_in, int32_t e_out, int32_t ec_in, int32_t ec_out,
+                                ksgd_oracle_strict_elem* out) {
+  int32_t f = e_in;
+  if (e_out < f) f = e_out;
+  if (ec_in < f) f = ec_in;
+  if (ec_out < f) f = ec_out;
+  int64_t d = ksgd_oracle_increment(g, lr, ec_out);
+  int64_t C1 = rne_div_pow2((int64_t)q_comp * pow2_i64(ec_in - f) - d * pow2_i64(ec_out - f), ec_out - f);
+  int64_t Qc1 = clamp_i64(C1, -qmax_bits(n), qmax_bits(n));
+  int64_t T = (int64_t)q_theta * pow2_i64(e_in - f) + Qc1 * pow2_i64(ec_out - f);
+  int64_t P = rne_div_pow2(T, e_out - f);
+  int64_t Qt = clamp_i64(P, -qmax_bits(m), qmax_bits(m));
+  int64_t C2 = rne_div_pow2(T - Qt * pow2_i64(e_out - f), ec_out - f);
+  int64_t Qc2 = clamp_i64(C2, -qmax_bits(n), qmax_bits(n));
+  out->C1 = C1; out->T = T; out->P = P; out->C2 = C2; out->d = (int32_t)d;
+  out->q_comp_mid = (int32_t)Qc1; out->q_theta = (int32_t)Qt; out->q_comp = (int32_t)Qc2;
+  out->nonfinite = isfinite(g) ? 0 : 1;
+}
+
+static int strict_window_ok(int32_t e, int32_t ec) { return e - ec >= -8 && e - ec <= 36; }
+
+int ksgd_oracle_strict_step_tensor(void* theta, void* comp, const float* grad, int64_t numel,
+                                   int32_t theta_bits, int32_t comp_bits, int32_t e_in, int32_t e_out,
+                                   int32_t ec_in, int32_t ec_out, float lr, ksgd_oracle_stats* stats,
+                                   int32_t n_threads) {
+  if (!theta || !comp || !grad || !stats || numel <= 0) return -1;
+  if (theta_bits < 2 || theta_bits > 16 || comp_bits < 2 || comp_bits > 16) return -1;
+  if (!strict_window_ok(e_in, ec_in) || !strict_window_ok(e_out, ec_out)) return -1;
+  uint32_t amax_theta = 0, amax_comp = 0;
+  uint64_t n_sat_theta = 0, n_sat_comp = 0, n_nonfinite = 0;
+  if (n_threads < 1) n_threads = 1;
+#pragma omp parallel for schedule(static) num_threads(n_threads) \
+    reduction(max : amax_theta, amax_comp) reduction(+ : n_sat_theta, n_sat_comp, n_nonfinite)
+  for (int64_t i = 0; i < numel; ++i) {
+    ksgd_oracle_strict_elem r;
+    ksgd_oracle_strict_element(load_mantissa(theta, i, theta_bits), load_mantissa(comp, i, comp_bits), grad[i],
+                               lr, theta_bits, comp_bits, e_in, e_out, ec_in, ec_out, &r);
+    store_mantissa(theta, i, theta_bits, r.q_theta);
+    store_mantissa(comp, i, comp_bits, r.q_comp);
+    int64_t aP = r.P < 0 ? -r.P : r.P, a1 = r.C1 < 0 ? -r.C1 : r.C1, a2 = r.C2 < 0 ? -r.C2 : r.C2;
+    int64_t aC = a1 > a2 ? a1 : a2;
+    if (aP > 2147483647LL) aP = 2147483647LL;
+    if (aC > 2147483647LL) aC = 2147483647LL;
+    if ((uint32_t)aP > amax_theta) amax_theta = (uint32_t)aP;
+    if ((uint32_t)aC > amax_comp) amax_comp = (uint32_t)aC;
+    n_sat_theta += (r.P != r.q_theta);
+    n_sat_comp += (uint64_t)(r.C1 != r.q_comp_mid) + (uint64_t)(r.C2 != r.q_comp);
+    n_nonfinite += (uint64_t)r.nonfinite;
+  }
+  stats->amax_theta = amax_theta; stats->amax_comp = amax_comp;
+  stats->n_sat_theta = n_sat_theta; stats->n_sat_comp = n_sat_comp; stats->n_nonfinite = n_nonfinite;
+  return 0;
+}
+
+/* The accumulator's next exponent: the tight fit of its own maximum (same rule as for
+ * theta), then moved into the window [e_next - 36, e_next + 8] around theta's next exponent
+ * and into [-64, 64].  A scan of zero says that every increment rounded to nothing on the
+ * present grid (or that there was none): the grid then becomes 8 binades finer, so that an
+ * empty accumulator finds the scale of the increments instead of swallowing them for ever. */
+int32_t ksgd_oracle_next_exponent_acc(uint32_t amax_comp, int32_t comp_bits, int32_t ec_out, int32_t e_next,
+                                      int32_t amax_mode) {
+  int32_t ec = ksgd_oracle_next_exponent(amax_comp, comp_bits, ec_out, amax_mode);
+  if (amax_mode && amax_comp == 0) ec = ec_out - 8;
+  if (ec < e_next - 36) ec = e_next - 36;
+  if (ec > e_next + 8) ec = e_next + 8;
+  if (ec > 64) ec = 64;
+  if (ec < -64) ec = -64;
+  return ec;
+}
+
+/* ------------------------------------------------------------------------------------
  * fp32 <-> dynamic fixed-point (Section 1: uniform linear quantization with one shared
  * exponent per tensor; Section 5: the exponent comes from a scan of the maximum).
  *

@@ -47,6 +47,12 @@ class _AdamStats(ctypes.Structure):
                 ("n_sat_m", ctypes.c_uint64), ("n_sat_v", ctypes.c_uint64)]
 
 
+class OracleStrictElem(ctypes.Structure):
+    _fields_ = [("C1", ctypes.c_int64), ("T", ctypes.c_int64), ("P", ctypes.c_int64), ("C2", ctypes.c_int64),
+                ("d", ctypes.c_int32), ("q_comp_mid", ctypes.c_int32), ("q_theta", ctypes.c_int32),
+                ("q_comp", ctypes.c_int32), ("nonfinite", ctypes.c_int32)]
+
+
 _lib = None
 
 
@@ -92,6 +98,15 @@ def _load():
         lib.ksgd_oracle_adam_step_tensor.restype = ctypes.c_int
         lib.ksgd_oracle_adam_step_tensor.argtypes = [ctypes.c_void_p] * 5 + [ctypes.c_int64] + \
             [ctypes.c_int32] * 9 + [ctypes.c_float] * 4 + [ctypes.POINTER(_AdamStats), ctypes.c_int32]
+        lib.ksgd_oracle_strict_element.restype = None
+        lib.ksgd_oracle_strict_element.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_float,
+                                                   ctypes.c_float] + [ctypes.c_int32] * 6 + \
+            [ctypes.POINTER(OracleStrictElem)]
+        lib.ksgd_oracle_strict_step_tensor.restype = ctypes.c_int
+        lib.ksgd_oracle_strict_step_tensor.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int64] + \
+            [ctypes.c_int32] * 6 + [ctypes.c_float, ctypes.POINTER(_Stats), ctypes.c_int32]
+        lib.ksgd_oracle_next_exponent_acc.restype = ctypes.c_int32
+        lib.ksgd_oracle_next_exponent_acc.argtypes = [ctypes.c_uint32] + [ctypes.c_int32] * 4
         lib.ksgd_oracle_max_threads.restype = ctypes.c_int32
         lib.ksgd_oracle_max_threads.argtypes = []
         _lib = lib
@@ -241,6 +256,33 @@ def oracle_adam_step_tensor(theta, comp, mom1, mom2, grad, theta_bits, comp_bits
             "n_sat_m": st.n_sat_m, "n_sat_v": st.n_sat_v}
 
 
+def oracle_strict_element(q_theta, q_comp, g, lr, m, n, e_in, e_out, ec_in, ec_out) -> OracleStrictElem:
+    """Strict Algorithm 1 for one element (accumulator with its own exponent)."""
+    out = OracleStrictElem()
+    _load().ksgd_oracle_strict_element(q_theta, q_comp, g, lr, m, n, e_in, e_out, ec_in, ec_out,
+                                       ctypes.byref(out))
+    return out
+
+
+def oracle_strict_step_tensor(theta, comp, grad, theta_bits, comp_bits, e_in, e_out, ec_in, ec_out, lr,
+                              n_threads: int = 1) -> dict:
+    assert theta.dtype == _storage_dtype(theta_bits) and comp.dtype == _storage_dtype(comp_bits)
+    assert theta.flags.c_contiguous and comp.flags.c_contiguous and comp.size == theta.size
+    assert grad.dtype == np.float32 and grad.flags.c_contiguous and grad.size == theta.size
+    st = _Stats()
+    rc = _load().ksgd_oracle_strict_step_tensor(theta.ctypes.data, comp.ctypes.data, grad.ctypes.data,
+                                                theta.size, theta_bits, comp_bits, e_in, e_out, ec_in, ec_out,
+                                                ctypes.c_float(lr), ctypes.byref(st), n_threads)
+    if rc != 0:
+        raise ValueError("oracle rejected the tensor description")
+    return {"amax_theta": st.amax_theta, "amax_comp": st.amax_comp, "n_sat_theta": st.n_sat_theta,
+            "n_sat_comp": st.n_sat_comp, "n_nonfinite": st.n_nonfinite}
+
+
+def oracle_next_exponent_acc(amax_comp: int, comp_bits: int, ec_out: int, e_next: int, mode: int) -> int:
+    return int(_load().ksgd_oracle_next_exponent_acc(amax_comp, comp_bits, ec_out, e_next, mode))
+
+
 @dataclass
 class OracleTensor:
     """One parameter tensor: mantissas, compensation, formats and exponents."""
@@ -263,6 +305,9 @@ class OracleTensor:
     exp_mom_next: int = 0
     amax_mom: int = 0
     n_sat_mom: int = 0
+    # strict Algorithm 1 only: the compensation's own exponent
+    exp_comp: int = 0
+    exp_comp_next: int = 0
     # ADAM only: `mom` is the first moment, `mom2` the second
     mom2: Optional[np.ndarray] = None
     exp_mom2: int = 0
@@ -361,3 +406,22 @@ def oracle_adam_step(state: OracleState, grads: Sequence[np.ndarray], lrs: Seque
         t.exp_mom_next = oracle_next_exponent_velocity(t.amax_mom, 16, em_out, state.mode)
         t.exp_mom2 = ev_out
         t.exp_mom2_next = oracle_next_exponent_velocity(t.amax_mom2, 16, ev_out, state.mode)
+
+
+def oracle_strict_step(state: OracleState, grads: Sequence[np.ndarray], lrs: Sequence[float]) -> None:
+    """One strict step of every tensor, then both exponent choices (theta's first: the
+    accumulator's window is placed around theta's next exponent)."""
+    assert len(grads) == len(state.tensors) == len(lrs)
+    for t, g, lr in zip(state.tensors, grads, lrs):
+        e_in, e_out, ec_in, ec_out = t.exp_theta, t.exp_theta_next, t.exp_comp, t.exp_comp_next
+        st = oracle_strict_step_tensor(t.theta, t.comp, g, t.theta_bits, t.comp_bits, e_in, e_out, ec_in,
+                                       ec_out, float(lr), state.n_threads)
+        t.amax_theta, t.amax_comp = st["amax_theta"], st["amax_comp"]
+        t.n_sat_theta += st["n_sat_theta"]
+        t.n_sat_comp += st["n_sat_comp"]
+        t.n_nonfinite += st["n_nonfinite"]
+        t.exp_theta = e_out
+        t.exp_theta_next = oracle_next_exponent(t.amax_theta, t.theta_bits, e_out, state.mode)
+        t.exp_comp = ec_out
+        t.exp_comp_next = oracle_next_exponent_acc(t.amax_comp, t.comp_bits, ec_out, t.exp_theta_next,
+                                                   state.mode)

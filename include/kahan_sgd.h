@@ -202,6 +202,39 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
                           uint64_t* n_sat_theta, uint64_t* n_sat_comp, uint64_t* n_nonfinite,
                           void* cuda_stream);
 
+/*
+ * Strict Algorithm 1 (Section 2, Algorithm 1 and Figure 1, read literally for the paper's
+ * hardware model): every statement rounds into the stored format, and the accumulator is
+ * an n-bit dynamic fixed-point tensor of its own whose exponent follows its own maximum
+ * (Section 5), so that the overlap k of Figure 1 is a result, k = n - 1 - (e - e_acc), not
+ * a parameter.  The ordinary entry points keep the sum theta + c - eta*g wide inside a step
+ * and tie c's exponent to theta's; this mode exists to measure what that buys.  As
+ * everywhere the tensor stored is c = -acc.  Per element, with f the smallest of the four
+ * exponents (theta's and c's, read at *_in, written at *_out):
+ *     d    = clamp(rne(fl32(g * fl32(eta * 2^-ec_out))), +-2^30)
+ *     C1   = rne((Q_c*2^(ec_in-f) - d*2^(ec_out-f)) / 2^(ec_out-f)),  Q_c1 = clamp(C1, +-QMAX_n)
+ *     T    = Q_theta*2^(e_in-f) + Q_c1*2^(ec_out-f),  P = rne(T / 2^(e_out-f)),  Q_theta' = clamp(P, +-QMAX_m)
+ *     C2   = rne((T - Q_theta'*2^(e_out-f)) / 2^(ec_out-f)),  Q_c' = clamp(C2, +-QMAX_n)
+ * amax_comp = max(|C1|, |C2|) and n_sat_comp counts both clamps.  c's next exponent is the
+ * tight fit of amax_comp (8 binades finer when amax_comp is 0: every increment rounded away
+ * or none came), kept within [e_next - 36, e_next + 8] of theta's next exponent.
+ * kahan_sgd_strict_init: as kahan_sgd_init, plus exp_comp / exp_comp_next (host arrays, one
+ * per tensor: c's exponent now stored and the one the first step writes; exp_comp_next NULL
+ * = the same).  Every tensor needs comp_bits != 0 (else KSGD_ERR_BITS); overlap_k is
+ * ignored; exponents outside [-64, 64] or outside the window above give KSGD_ERR_EXP_RANGE.
+ * The handle then works with kahan_sgd_step, kahan_sgd_step_qgrad, kahan_sgd_amax and
+ * kahan_sgd_destroy; kahan_sgd_step_host, kahan_sgd_set_exponents and
+ * kahan_sgd_strict_exponents on the wrong kind of handle return KSGD_ERR_MODE.
+ * kahan_sgd_strict_exponents copies c's exponents (stored / next) to the non-NULL host
+ * arrays and waits for the stream.
+ */
+size_t kahan_sgd_strict_workspace_bytes(const ksgd_tensor_desc* descs, const int32_t* exp_comp,
+                                        int32_t n_tensors);
+int kahan_sgd_strict_init(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t* exp_comp,
+                          const int32_t* exp_comp_next, int32_t n_tensors, ksgd_exp_mode mode,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+int kahan_sgd_strict_exponents(ksgd_handle* h, int32_t* exp_comp_cur, int32_t* exp_comp_next);
+
 /* Free the host-side handle (waits for the stream first).  Device buffers stay the caller's. */
 int kahan_sgd_destroy(ksgd_handle* h);
 

@@ -29,7 +29,8 @@ KSGD_ERR_DEVICE = -11
 
 EXPORTS = (
     "kahan_sgd_workspace_bytes", "kahan_sgd_init", "kahan_sgd_step", "kahan_sgd_step_qgrad",
-    "kahan_sgd_step_host",
+    "kahan_sgd_step_host", "kahan_sgd_strict_workspace_bytes", "kahan_sgd_strict_init",
+    "kahan_sgd_strict_exponents",
     "kahan_sgd_amax", "kahan_sgd_set_exponents", "kahan_sgd_step_static", "kahan_sgd_destroy",
     "kahan_sgd_strerror", "kahan_sgd_momentum_workspace_bytes", "kahan_sgd_momentum_init",
     "kahan_sgd_momentum_step", "kahan_sgd_momentum_amax", "kahan_sgd_momentum_destroy",
@@ -89,6 +90,14 @@ def _load() -> ctypes.CDLL:
     lib.kahan_sgd_step_qgrad.restype = ctypes.c_int
     lib.kahan_sgd_step_qgrad.argtypes = [ctypes.c_void_p, P(ctypes.c_void_p), ctypes.c_int32,
                                          P(ctypes.c_int32), P(ctypes.c_float)]
+    lib.kahan_sgd_strict_workspace_bytes.restype = ctypes.c_size_t
+    lib.kahan_sgd_strict_workspace_bytes.argtypes = [P(ksgd_tensor_desc), P(ctypes.c_int32), ctypes.c_int32]
+    lib.kahan_sgd_strict_init.restype = ctypes.c_int
+    lib.kahan_sgd_strict_init.argtypes = [P(ctypes.c_void_p), P(ksgd_tensor_desc), P(ctypes.c_int32),
+                                          P(ctypes.c_int32), ctypes.c_int32, ctypes.c_int, ctypes.c_void_p,
+                                          ctypes.c_size_t, ctypes.c_void_p]
+    lib.kahan_sgd_strict_exponents.restype = ctypes.c_int
+    lib.kahan_sgd_strict_exponents.argtypes = [ctypes.c_void_p, P(ctypes.c_int32), P(ctypes.c_int32)]
     lib.kahan_sgd_step_host.restype = ctypes.c_int
     lib.kahan_sgd_step_host.argtypes = [ctypes.c_void_p, P(ctypes.c_void_p), P(ctypes.c_void_p),
                                         P(ctypes.c_void_p), P(ctypes.c_float), ctypes.c_void_p,
@@ -203,6 +212,30 @@ def kahan_sgd_step(h, grads, lrs) -> None:
     g = grads if isinstance(grads, ctypes.Array) else _ptr_array(grads)
     l = lrs if isinstance(lrs, ctypes.Array) else _float_array(lrs)
     _check(lib.kahan_sgd_step(h, g, l))
+
+
+def _int_array(values):
+    return (ctypes.c_int32 * len(values))(*[int(v) for v in values])
+
+
+def kahan_sgd_strict_workspace_bytes(descs, exp_comp) -> int:
+    return int(lib.kahan_sgd_strict_workspace_bytes(descs, _int_array(exp_comp), len(descs)))
+
+
+def kahan_sgd_strict_init(descs, exp_comp, exp_comp_next, mode: int, workspace: int, workspace_bytes: int,
+                          stream: int = 0):
+    """Strict Algorithm 1: exp_comp / exp_comp_next are the compensation's own exponents."""
+    h = ctypes.c_void_p()
+    nxt = _int_array(exp_comp_next) if exp_comp_next is not None else None
+    _check(lib.kahan_sgd_strict_init(ctypes.byref(h), descs, _int_array(exp_comp), nxt, len(descs), mode,
+                                     ctypes.c_void_p(workspace), workspace_bytes, ctypes.c_void_p(stream)))
+    return h
+
+
+def kahan_sgd_strict_exponents(h, n_tensors: int) -> dict:
+    cur, nxt = (ctypes.c_int32 * n_tensors)(), (ctypes.c_int32 * n_tensors)()
+    _check(lib.kahan_sgd_strict_exponents(h, cur, nxt))
+    return {"exp_comp_cur": list(cur), "exp_comp_next": list(nxt)}
 
 
 def kahan_sgd_step_qgrad(h, grads, grad_bits: int, exp_grad, lrs) -> None:

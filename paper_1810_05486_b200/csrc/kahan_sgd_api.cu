@@ -40,7 +40,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // kahan_sgd_amax fetches them with one copy.
 struct Layout {
   size_t exp_cur, exp_next, amax_last, counters, error, stats_end;
-  size_t amax_acc, info, grad_ptr, lr, exp_grad, chunks, ticket, total;
+  size_t amax_acc, info, grad_ptr, lr, exp_grad, expc_cur, expc_next, chunks, ticket, total;
   long long n_chunks;
 };
 
@@ -63,6 +63,8 @@ Layout make_layout(const ksgd_tensor_desc* d, int32_t n) {
   L.grad_ptr = o;  o += sizeof(const float*) * n;
   L.lr = o;        o += sizeof(float) * n;
   L.exp_grad = o;  o += sizeof(int) * n;
+  L.expc_cur = o;  o += sizeof(int) * n;
+  L.expc_next = o; o += sizeof(int) * n;
   o = align_up(o, 16);
   L.chunks = o;    o += sizeof(ChunkRef) * (size_t)chunks;
   o = align_up(o, 16);
@@ -107,6 +109,7 @@ struct ksgd_handle {
   int sms;
   std::vector<unsigned char> stats_host;   // staging for kahan_sgd_amax
   std::vector<long long> first_tile;       // [n+1] first tile of every tensor
+  bool strict = false;                     // strict Algorithm 1: compensation with its own exponent
   // kahan_sgd_step_host: copy streams and events, created on first use
   cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
   std::vector<cudaEvent_t> events;
@@ -119,13 +122,35 @@ size_t kahan_sgd_workspace_bytes(const ksgd_tensor_desc* descs, int32_t n_tensor
   return make_layout(descs, n_tensors).total;
 }
 
-int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_tensors,
-                   ksgd_exp_mode mode, void* workspace, size_t workspace_bytes,
-                   void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+
+bool strict_window_ok(int e, int ec) { return e - ec >= -kStrictAbove && e - ec <= kStrictBelow; }
+
+int validate_strict(const ksgd_tensor_desc* d, const int32_t* ec, const int32_t* ec_next, int32_t n) {
+  if (!ec) return KSGD_ERR_NULL;
+  for (int32_t i = 0; i < n; ++i) {
+    if (d[i].comp_bits == 0) return KSGD_ERR_BITS;          // the accumulator is the point of this mode
+    const int32_t nx = ec_next ? ec_next[i] : ec[i];
+    if (ec[i] < kExpMin || ec[i] > kExpMax || nx < kExpMin || nx > kExpMax) return KSGD_ERR_EXP_RANGE;
+    if (!strict_window_ok(d[i].exp_theta, ec[i]) || !strict_window_ok(d[i].exp_theta_next, nx))
+      return KSGD_ERR_EXP_RANGE;
+  }
+  return KSGD_OK;
+}
+
+int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t* exp_comp,
+                const int32_t* exp_comp_next, bool strict, int32_t n_tensors, ksgd_exp_mode mode,
+                void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (!out) return KSGD_ERR_NULL;
   *out = nullptr;
   const int v = validate(descs, n_tensors);
   if (v != KSGD_OK) return v;
+  if (strict) {
+    const int vs = validate_strict(descs, exp_comp, exp_comp_next, n_tensors);
+    if (vs != KSGD_OK) return vs;
+  }
   if (mode != KSGD_EXP_FIXED && mode != KSGD_EXP_AMAX) return KSGD_ERR_MODE;
   if (!workspace) return KSGD_ERR_NULL;
   if (reinterpret_cast<uintptr_t>(workspace) % 256) return KSGD_ERR_ALIGN;
@@ -140,12 +165,21 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
   h->ws_base = static_cast<char*>(workspace);
   h->stream = static_cast<cudaStream_t>(cuda_stream);
   h->stats_host.resize(L.stats_end);
+  h->strict = strict;
 
   // Host image of the workspace: exponents, zeroed scans and counters, tensor table,
   // chunk table.
   std::vector<unsigned char> img(L.total, 0);
   int* exp_cur = reinterpret_cast<int*>(img.data() + L.exp_cur);
   int* exp_next = reinterpret_cast<int*>(img.data() + L.exp_next);
+  if (strict) {
+    int* ec_cur = reinterpret_cast<int*>(img.data() + L.expc_cur);
+    int* ec_nx = reinterpret_cast<int*>(img.data() + L.expc_next);
+    for (int32_t i = 0; i < n_tensors; ++i) {
+      ec_cur[i] = exp_comp[i];
+      ec_nx[i] = exp_comp_next ? exp_comp_next[i] : exp_comp[i];
+    }
+  }
   TensorInfo* info = reinterpret_cast<TensorInfo*>(img.data() + L.info);
   ChunkRef* chunks = reinterpret_cast<ChunkRef*>(img.data() + L.chunks);
   long long c = 0;
@@ -178,6 +212,8 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
   w.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
   w.lr = reinterpret_cast<float*>(b + L.lr);
   w.exp_grad = reinterpret_cast<int*>(b + L.exp_grad);
+  w.expc_cur = reinterpret_cast<int*>(b + L.expc_cur);
+  w.expc_next = reinterpret_cast<int*>(b + L.expc_next);
   w.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
   w.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
   h->params.n_tensors = n_tensors;
@@ -203,6 +239,15 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(ksgd_step_qgrad_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)kSharedBytes);
+  if (e == cudaSuccess && strict)
+    e = cudaFuncSetAttribute(ksgd_strict_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSharedBytes);
+  if (e == cudaSuccess && strict)
+    e = cudaFuncSetAttribute(ksgd_strict_step_qgrad_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSharedBytes);
+  if (e == cudaSuccess && strict)
+    e = cudaFuncSetAttribute(ksgd_strict_step_qgrad_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSharedBytes);
   if (e != cudaSuccess) {
     delete h;
     return cuda_fail(e, "device query");
@@ -227,6 +272,46 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
   return KSGD_OK;
 }
 
+}  // namespace
+
+extern "C" {
+
+int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_tensors,
+                   ksgd_exp_mode mode, void* workspace, size_t workspace_bytes,
+                   void* cuda_stream) {
+  return init_common(out, descs, nullptr, nullptr, false, n_tensors, mode, workspace, workspace_bytes,
+                     cuda_stream);
+}
+
+size_t kahan_sgd_strict_workspace_bytes(const ksgd_tensor_desc* descs, const int32_t* exp_comp,
+                                        int32_t n_tensors) {
+  if (validate(descs, n_tensors) != KSGD_OK) return 0;
+  if (validate_strict(descs, exp_comp, nullptr, n_tensors) != KSGD_OK) return 0;
+  return make_layout(descs, n_tensors).total;
+}
+
+int kahan_sgd_strict_init(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t* exp_comp,
+                          const int32_t* exp_comp_next, int32_t n_tensors, ksgd_exp_mode mode,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!out) return KSGD_ERR_NULL;
+  *out = nullptr;
+  if (!exp_comp) return KSGD_ERR_NULL;
+  return init_common(out, descs, exp_comp, exp_comp_next, true, n_tensors, mode, workspace, workspace_bytes,
+                     cuda_stream);
+}
+
+int kahan_sgd_strict_exponents(ksgd_handle* h, int32_t* exp_comp_cur, int32_t* exp_comp_next) {
+  if (!h) return KSGD_ERR_NULL;
+  if (!h->strict) return KSGD_ERR_MODE;
+  std::vector<int> host(2 * (size_t)h->n);
+  KSGD_CUDA(cudaMemcpyAsync(host.data(), h->ws_base + h->layout.expc_cur, sizeof(int) * 2 * (size_t)h->n,
+                            cudaMemcpyDeviceToHost, h->stream));
+  KSGD_CUDA(cudaStreamSynchronize(h->stream));
+  if (exp_comp_cur) std::memcpy(exp_comp_cur, host.data(), sizeof(int) * (size_t)h->n);
+  if (exp_comp_next) std::memcpy(exp_comp_next, host.data() + h->n, sizeof(int) * (size_t)h->n);
+  return KSGD_OK;
+}
+
 static int check_step_args(const ksgd_handle* h, const float* const* grads, const float* lrs) {
   if (!h || !grads || !lrs) return KSGD_ERR_NULL;
   for (int32_t i = 0; i < h->n; ++i) {
@@ -245,7 +330,8 @@ static int launch_step_range(ksgd_handle* h, const InlineArgs* ia, int32_t t0, i
   p.tensor_begin = t0;
   p.tensor_count = t1 - t0;
   const int grid = p.tile_count < h->sms ? p.tile_count : h->sms;
-  ksgd_step_kernel<<<(unsigned)grid, kBlockThreads, kSharedBytes, h->stream>>>(p, *ia);
+  if (h->strict) ksgd_strict_step_kernel<<<(unsigned)grid, kBlockThreads, kSharedBytes, h->stream>>>(p, *ia);
+  else ksgd_step_kernel<<<(unsigned)grid, kBlockThreads, kSharedBytes, h->stream>>>(p, *ia);
   g_launches.fetch_add(1, std::memory_order_relaxed);
   KSGD_CUDA(cudaGetLastError());
   return KSGD_OK;
@@ -272,7 +358,10 @@ static int launch_step(ksgd_handle* h, const float* const* grads, const float* l
     delete ub;
     KSGD_CUDA(cudaGetLastError());
   }
-  ksgd_step_kernel<<<(unsigned)h->grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, *ia);
+  if (h->strict)
+    ksgd_strict_step_kernel<<<(unsigned)h->grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, *ia);
+  else
+    ksgd_step_kernel<<<(unsigned)h->grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, *ia);
   g_launches.fetch_add(1, std::memory_order_relaxed);
   KSGD_CUDA(cudaGetLastError());
   return KSGD_OK;
@@ -315,10 +404,18 @@ int kahan_sgd_step_qgrad(ksgd_handle* h, const void* const* grads, int32_t grad_
     delete eb;
     KSGD_CUDA(cudaGetLastError());
   }
-  if (grad_bits == 8)
-    ksgd_step_qgrad_kernel<8><<<(unsigned)h->grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, args);
-  else
-    ksgd_step_qgrad_kernel<16><<<(unsigned)h->grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, args);
+  const unsigned grid = (unsigned)h->grid;
+  if (h->strict) {
+    if (grad_bits == 8)
+      ksgd_strict_step_qgrad_kernel<8><<<grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, args);
+    else
+      ksgd_strict_step_qgrad_kernel<16><<<grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, args);
+  } else {
+    if (grad_bits == 8)
+      ksgd_step_qgrad_kernel<8><<<grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, args);
+    else
+      ksgd_step_qgrad_kernel<16><<<grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, args);
+  }
   g_launches.fetch_add(1, std::memory_order_relaxed);
   KSGD_CUDA(cudaGetLastError());
   return KSGD_OK;
@@ -334,6 +431,7 @@ int kahan_sgd_step_host(ksgd_handle* h, void* const* theta_host, void* const* co
                         const float* const* grads_host, const float* lrs,
                         void* grad_staging, size_t grad_staging_bytes) {
   if (!h || !theta_host || !comp_host || !grads_host || !lrs || !grad_staging) return KSGD_ERR_NULL;
+  if (h->strict) return KSGD_ERR_MODE;
   if (reinterpret_cast<uintptr_t>(grad_staging) % 16) return KSGD_ERR_ALIGN;
   size_t need = 0;
   for (int32_t i = 0; i < h->n; ++i) need += align_up((size_t)h->descs[i].numel, 4) * sizeof(float);
@@ -486,6 +584,7 @@ int kahan_sgd_amax(ksgd_handle* h, uint32_t* amax_theta, uint32_t* amax_comp,
 
 int kahan_sgd_set_exponents(ksgd_handle* h, const int32_t* exp_theta_next) {
   if (!h || !exp_theta_next) return KSGD_ERR_NULL;
+  if (h->strict) return KSGD_ERR_MODE;     // the compensation's window hangs on theta's exponent
   for (int32_t i = 0; i < h->n; ++i)
     if (exp_theta_next[i] < kExpMin || exp_theta_next[i] > kExpMax) return KSGD_ERR_EXP_RANGE;
   ExponentBatch* eb = new (std::nothrow) ExponentBatch;
@@ -610,6 +709,8 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   params.ws.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
   params.ws.lr = reinterpret_cast<float*>(b + L.lr);
   params.ws.exp_grad = reinterpret_cast<int*>(b + L.exp_grad);
+  params.ws.expc_cur = reinterpret_cast<int*>(b + L.expc_cur);
+  params.ws.expc_next = reinterpret_cast<int*>(b + L.expc_next);
   params.ws.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
   params.ws.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
   params.n_tensors = n_tensors;

@@ -71,6 +71,8 @@ struct Workspace {
   const float** grad_ptr;          // [n] per-step arguments for lists longer than kInlineArgs
   float* lr;                       // [n]
   int* exp_grad;                   // [n] the same, exponents of fixed-point gradients
+  int* expc_cur;                   // [n] strict mode: the compensation's own exponent, stored ...
+  int* expc_next;                  // [n] ... and the one the coming step writes
   ChunkRef* chunks;                // [n_chunks]
   unsigned int* ticket;            // blocks finished in the running step
 };
@@ -125,6 +127,8 @@ struct StepCoef {
   int qmax_c;    // 2^(n-1) - 1
   int gb;        // gradient storage: 32 = binary32, 8 / 16 = fixed-point mantissas
   int eg;        // exponent of fixed-point gradient mantissas (0 for binary32)
+  int strict;    // 1: every statement of Algorithm 1 rounds into the stored format
+  int delta_c;   // ec_out - ec_in
 };
 
 // One tile as the producer describes it to the consumers (lives in shared memory).  The
@@ -256,22 +260,27 @@ __device__ __forceinline__ int quantize_increment(float g, float scale) {
   return max(min(d, kDLimit), -kDLimit);
 }
 
-__device__ __forceinline__ StepCoef make_coef(const TensorInfo& ti, int e_in, int e_out, float lr, int gb,
-                                              int eg) {
+// Shifts between the four grids of a step (theta's and c's, each read at *_in and written at
+// *_out) and the finest of them, f.  In the ordinary mode c's exponent is tied to theta's
+// (ec = e - s); in strict mode it is the tensor's own.
+__device__ __forceinline__ StepCoef make_coef(const TensorInfo& ti, int e_in, int e_out, int ec_in, int ec_out,
+                                              float lr, int gb, int eg, int strict) {
   StepCoef k;
   k.gb = gb;
   k.eg = eg;
-  const int delta = e_out - e_in;
-  k.s = ti.s;
-  k.delta = delta;
-  k.sh_t = ti.s + max(0, -delta);
-  k.sh_c = max(0, -delta);
-  k.sh_d = max(0, delta);
-  k.r_t = ti.s + max(0, delta);
-  k.r_c = max(0, delta);
+  k.strict = strict;
+  const int f = min(min(e_in, e_out), min(ec_in, ec_out));
+  k.s = e_out - ec_out;
+  k.delta = e_out - e_in;
+  k.delta_c = ec_out - ec_in;
+  k.sh_t = e_in - f;
+  k.sh_c = ec_in - f;
+  k.sh_d = ec_out - f;
+  k.r_t = e_out - f;
+  k.r_c = ec_out - f;
   k.qmax_t = (1 << (ti.theta_bits - 1)) - 1;
   k.qmax_c = ti.comp_bits ? (1 << (ti.comp_bits - 1)) - 1 : 0;
-  k.scale = __fmul_rn(lr, pow2_float(ti.s - e_out));   // |s - e_out| <= 79: exact power of two
+  k.scale = __fmul_rn(lr, pow2_float(-ec_out));   // |ec_out| <= 100: exact power of two
   return k;
 }
 
@@ -297,11 +306,23 @@ __device__ __noinline__ void update_general(const StepCoef* coef, int tb, int cb
     else if (k.gb == 8) g = __fmul_rn((float)static_cast<const signed char*>(grad)[e], pow2_float(k.eg));
     else g = __fmul_rn((float)static_cast<const short*>(grad)[e], pow2_float(k.eg));
     const int d = quantize_increment(g, k.scale);
-    const long long T = (long long)qt * (1LL << k.sh_t) + (long long)qc * (1LL << k.sh_c) -
-                        (long long)d * (1LL << k.sh_d);
+    long long T;
+    if (k.strict) {
+      // statement 1 rounds into the n-bit accumulator before theta sees it
+      const long long C1 = rne_shift64((long long)qc * (1LL << k.sh_c) - (long long)d * (1LL << k.sh_d), k.r_c);
+      const long long C1c = C1 > k.qmax_c ? k.qmax_c : (C1 < -k.qmax_c ? -k.qmax_c : C1);
+      unsigned long long a1 = (unsigned long long)(C1 < 0 ? -C1 : C1);
+      if (a1 > 0x7fffffffULL) a1 = 0x7fffffffULL;
+      amax_c = max(amax_c, (unsigned int)a1);
+      n_sat_c += (C1 != C1c);
+      T = (long long)qt * (1LL << k.sh_t) + C1c * (1LL << k.r_c);
+    } else {
+      T = (long long)qt * (1LL << k.sh_t) + (long long)qc * (1LL << k.sh_c) - (long long)d * (1LL << k.sh_d);
+    }
     const long long P = rne_shift64(T, k.r_t);
     const long long Pc = P > k.qmax_t ? k.qmax_t : (P < -k.qmax_t ? -k.qmax_t : P);
-    const unsigned long long aP = (unsigned long long)(P < 0 ? -P : P);
+    unsigned long long aP = (unsigned long long)(P < 0 ? -P : P);
+    if (aP > 0x7fffffffULL) aP = 0x7fffffffULL;
     amax_t = max(amax_t, (unsigned int)aP);
     n_sat_t += (P != Pc);
     if (tb == 8) static_cast<signed char*>(theta)[e] = (signed char)Pc;
@@ -458,7 +479,7 @@ struct TileHot {       // the consumers' copy of the first 48 bytes of a TileDes
   int tensor, n_bulk, count, flags;
 };
 
-template <int TB, int CB, int V, int GB>
+template <int TB, int CB, int V, int GB, bool STRICT>
 __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V * CB / 8 : 8)> pc,
                                               Pack<V * GB / 8> pg, const SteadyCoef& k,
                                               Pack<V * TB / 8>& ot, Pack<(CB ? V * CB / 8 : 8)>& oc,
@@ -470,7 +491,7 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
   if constexpr (HAS_COMP) flip_signs<(CB ? CB : 8)>(pc);
   if constexpr (GB != 32) flip_signs<(GB == 32 ? 8 : GB)>(pg);
   float Pm[V], rm[V];
-  float sum_abs = 0.0f, aX = 0.0f, aP = 0.0f, aR = 0.0f;
+  float sum_abs = 0.0f, aX = 0.0f, aP = 0.0f, aR = 0.0f, aU = 0.0f;
 #pragma unroll
   for (int i = 0; i < V; ++i) {
     const float qtM = __fadd_rn(magic_elem<TB>(pt, i), -bias_t);
@@ -491,8 +512,15 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
     rm[i] = __fadd_rn(r0, kMagic);
     aP = fmaxf(aP, fabsf(__fadd_rn(P, -kMagic)));
     if constexpr (HAS_COMP) aR = fmaxf(aR, fabsf(r0));
+    if constexpr (STRICT) aU = fmaxf(aU, fabsf(u));     // u = c - d is statement 1's result
   }
   if (!(sum_abs < 3.0e38f) | (aX > 4000000.0f) | (aP > k.qmax_t)) return false;
+  if constexpr (STRICT) {
+    // both accumulator results must fit their n bits, or the vector needs the clamps
+    constexpr float qmax_c = (float)((1 << ((CB ? CB : 8) - 1)) - 1);
+    aR = fmaxf(aR, aU);
+    if (aR > qmax_c) return false;
+  }
   amax_t = fmaxf(amax_t, aP);
   if constexpr (HAS_COMP) amax_c = fmaxf(amax_c, aR);
   ot = pack_magic<TB, V>(Pm);
@@ -502,7 +530,7 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
 
 // All vectors of one tile that belong to this consumer thread (V consecutive elements,
 // 16 bytes of theta, per vector).  Returns true if the general path wrote into the stage.
-template <int TB, int CB, int GB>
+template <int TB, int CB, int GB, bool STRICT>
 __device__ __forceinline__ bool consume_tile(const TileHot& h, const TileDesc* td, unsigned char* ring,
                                              int ctid, TileScan* slots, float& amax_t, float& amax_c) {
   constexpr bool HAS_COMP = CB != 0;
@@ -525,7 +553,7 @@ __device__ __forceinline__ bool consume_tile(const TileHot& h, const TileDesc* t
       Pack<CBYTES> pc{};
       if constexpr (HAS_COMP) pc = load_pack<CBYTES>(comp_s + v * CBYTES);
       const Pack<GBYTES> pg = load_pack<GBYTES>(grad_s + v * GBYTES);
-      done = update_vector<TB, CB, V, GB>(pt, pc, pg, h.k, ot, oc, amax_t, amax_c);
+      done = update_vector<TB, CB, V, GB, STRICT>(pt, pc, pg, h.k, ot, oc, amax_t, amax_c);
     }
     if (!done) {
       // general path, in place in the stage; then the vector goes out like any other
@@ -557,6 +585,19 @@ __device__ __forceinline__ int next_exponent(unsigned int amax, int bits, int e_
   }
   change = max(-kMaxDelta, min(kMaxDelta, change));
   return max(kExpMin, min(kExpMax, e_out + change));
+}
+
+// Strict mode: the compensation's own next exponent.  The tight fit of its scan; an empty
+// scan (every increment rounded away, or none came) makes the grid 8 binades finer; the
+// result stays within [e_next - 36, e_next + 8] of theta's next exponent, which keeps every
+// sum of the step within 64 bits.
+constexpr int kStrictBelow = 36, kStrictAbove = 8;
+__device__ __forceinline__ int next_exponent_acc(unsigned int amax, int bits, int ec_out, int e_next,
+                                                 int amax_mode) {
+  int ec = next_exponent(amax, bits, ec_out, amax_mode);
+  if (amax_mode && amax == 0u) ec = ec_out - kMaxDelta;
+  ec = max(e_next - kStrictBelow, min(e_next + kStrictAbove, ec));
+  return max(kExpMin, min(kExpMax, ec));
 }
 
 struct __align__(128) BlockShared {
@@ -624,10 +665,21 @@ struct TensorMeta {
   const void* grad;
   float lr;
   int e_in, e_out;
-  int eg;          // exponent of a fixed-point gradient, 0 for binary32
+  int ec_in, ec_out;   // the compensation's exponents: e - s, or its own in strict mode
+  int eg;              // exponent of a fixed-point gradient, 0 for binary32
 };
 
-__device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const InlineArgs& a, int t) {
+__device__ __forceinline__ void load_comp_exponents(const StepParams& p, int t, bool strict, TensorMeta& m) {
+  if (strict) {
+    m.ec_in = p.ws.expc_cur[t];
+    m.ec_out = p.ws.expc_next[t];
+  } else {
+    m.ec_in = m.e_in - m.ti.s;
+    m.ec_out = m.e_out - m.ti.s;
+  }
+}
+
+__device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const InlineArgs& a, int t, bool strict) {
   TensorMeta m;
   m.ti = p.ws.info[t];
   m.e_in = p.ws.exp_cur[t];
@@ -635,10 +687,11 @@ __device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const Inlin
   m.grad = p.inline_args ? a.grads[t] : p.ws.grad_ptr[t];
   m.lr = p.inline_args ? a.lrs[t] : p.ws.lr[t];
   m.eg = 0;
+  load_comp_exponents(p, t, strict, m);
   return m;
 }
 
-__device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const QGradArgs& a, int t) {
+__device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const QGradArgs& a, int t, bool strict) {
   TensorMeta m;
   m.ti = p.ws.info[t];
   m.e_in = p.ws.exp_cur[t];
@@ -646,12 +699,15 @@ __device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const QGrad
   m.grad = p.inline_args ? a.grads[t] : static_cast<const void*>(p.ws.grad_ptr[t]);
   m.lr = p.inline_args ? a.lrs[t] : p.ws.lr[t];
   m.eg = p.inline_args ? (int)a.exp_grad[t] : p.ws.exp_grad[t];
+  load_comp_exponents(p, t, strict, m);
   return m;
 }
 
 // The whole step.  GB = 32: binary32 gradients; 8 / 16: fixed-point gradients (one or two
 // bytes per parameter instead of four on the gradient stream).
-template <int GB, typename Args>
+// STRICT: every statement of Algorithm 1 rounds into the stored format and the compensation
+// has its own exponent (comp_bits != 0 for every tensor).
+template <int GB, bool STRICT, typename Args>
 __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
   extern __shared__ __align__(128) unsigned char smem[];
   BlockShared* sh = reinterpret_cast<BlockShared*>(smem + (size_t)kPages * kPageBytes);
@@ -686,7 +742,7 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
       const unsigned long long grad_policy = l2_policy_evict_first();
       ScanAcc acc;
       ChunkRef cr = p.ws.chunks[tile0];
-      TensorMeta meta = load_meta(p, a, cr.tensor);
+      TensorMeta meta = load_meta(p, a, cr.tensor, STRICT);
       ChunkRef cr1{-1, -1};
       if (n_my > 1) cr1 = p.ws.chunks[tile0 + stride];
       int issued = 0;
@@ -699,7 +755,7 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
         ChunkRef cr2{-1, -1};
         if (i + 2 < n_my) cr2 = p.ws.chunks[tile0 + (i + 2) * stride];
         TensorMeta meta1 = meta;
-        if (i + 1 < n_my && cr1.tensor != cr.tensor) meta1 = load_meta(p, a, cr1.tensor);
+        if (i + 1 < n_my && cr1.tensor != cr.tensor) meta1 = load_meta(p, a, cr1.tensor, STRICT);
 
         const TensorInfo& ti = meta.ti;
         const int tbytes = ti.theta_bits >> 3, cbytes = ti.comp_bits >> 3;
@@ -737,7 +793,8 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
         free_pages -= need;
         sh->slot_pages[slot] = need;
 
-        const StepCoef coef = make_coef(ti, meta.e_in, meta.e_out, meta.lr, GB, meta.eg);
+        const StepCoef coef = make_coef(ti, meta.e_in, meta.e_out, meta.ec_in, meta.ec_out, meta.lr, GB, meta.eg,
+                                        STRICT ? 1 : 0);
         // fixed-point gradients: the exact-fp32 path multiplies the mantissa by scale * 2^eg,
         // which must itself be exact (a normal number); otherwise the tile takes the general path
         float scale_hot = coef.scale;
@@ -762,7 +819,9 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
         td.n_bulk = n_bulk;
         td.count = count;
         td.flags = ((ti.theta_bits == 16 ? 3 : 0) + (ti.comp_bits >> 3)) |
-                   ((coef.delta == 0 && scale_ok) ? kFlagSteady : 0) | (page[1] << kFlagThetaPageShift) |
+                   ((coef.delta == 0 && scale_ok && (!STRICT || (coef.delta_c == 0 && coef.s >= 0))) ? kFlagSteady
+                                                                                                       : 0) |
+                   (page[1] << kFlagThetaPageShift) |
                    (page[2] << kFlagCompPageShift) | (page[0] << kFlagGradPageShift);
         td.coef = coef;
         td.grad = static_cast<const unsigned char*>(meta.grad) + first * gbytes;
@@ -832,12 +891,12 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
       unsigned char* st = smem;
       bool wrote_stage;
       switch (h.flags & kFlagFormatMask) {
-        case 0: wrote_stage = consume_tile<8, 0, GB>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        case 1: wrote_stage = consume_tile<8, 8, GB>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        case 2: wrote_stage = consume_tile<8, 16, GB>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        case 3: wrote_stage = consume_tile<16, 0, GB>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        case 4: wrote_stage = consume_tile<16, 8, GB>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        default: wrote_stage = consume_tile<16, 16, GB>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 0: wrote_stage = consume_tile<8, 0, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 1: wrote_stage = consume_tile<8, 8, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 2: wrote_stage = consume_tile<8, 16, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 3: wrote_stage = consume_tile<16, 0, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 4: wrote_stage = consume_tile<16, 8, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        default: wrote_stage = consume_tile<16, 16, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
       }
       add_warp_scans(scan, lane, amax_t, amax_c);
       // if the general path wrote into the stage, order those writes before the bulk copy
@@ -865,8 +924,14 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
     const unsigned int at = __ldcg(&p.ws.amax_acc[i]);
     const unsigned int ac = __ldcg(&p.ws.amax_acc[p.n_tensors + i]);
     const int eo = p.ws.exp_next[i];
+    const int en = next_exponent(at, p.ws.info[i].theta_bits, eo, p.amax_mode);
     p.ws.exp_cur[i] = eo;
-    p.ws.exp_next[i] = next_exponent(at, p.ws.info[i].theta_bits, eo, p.amax_mode);
+    p.ws.exp_next[i] = en;
+    if constexpr (STRICT) {
+      const int eco = p.ws.expc_next[i];
+      p.ws.expc_cur[i] = eco;
+      p.ws.expc_next[i] = next_exponent_acc(ac, p.ws.info[i].comp_bits, eco, en, p.amax_mode);
+    }
     p.ws.amax_last[i] = at;
     p.ws.amax_last[p.n_tensors + i] = ac;
     p.ws.amax_acc[i] = 0u;
@@ -877,13 +942,24 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
 
 __global__ void __launch_bounds__(kBlockThreads, 1)
 ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ InlineArgs a) {
-  step_body<32>(p, a);
+  step_body<32, false>(p, a);
 }
 
 template <int GB>
 __global__ void __launch_bounds__(kBlockThreads, 1)
 ksgd_step_qgrad_kernel(const __grid_constant__ StepParams p, const __grid_constant__ QGradArgs a) {
-  step_body<GB>(p, a);
+  step_body<GB, false>(p, a);
+}
+
+__global__ void __launch_bounds__(kBlockThreads, 1)
+ksgd_strict_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ InlineArgs a) {
+  step_body<32, true>(p, a);
+}
+
+template <int GB>
+__global__ void __launch_bounds__(kBlockThreads, 1)
+ksgd_strict_step_qgrad_kernel(const __grid_constant__ StepParams p, const __grid_constant__ QGradArgs a) {
+  step_body<GB, true>(p, a);
 }
 
 // Per-step arguments of long lists: written to the workspace from kernel parameters.

@@ -54,7 +54,7 @@ class LibraryRun:
     """Drives kahan_sgd_* on device copies of the given tensors."""
 
     def __init__(self, specs: Sequence[dict], thetas: Sequence[np.ndarray],
-                 comps: Sequence[Optional[np.ndarray]], mode: int, stream=None):
+                 comps: Sequence[Optional[np.ndarray]], mode: int, stream=None, strict: bool = False):
         import torch
         from paper_1810_05486_b200 import binding as B
         self.B = B
@@ -77,12 +77,22 @@ class LibraryRun:
                               exp_theta=s["exp_theta"],
                               exp_theta_next=s.get("exp_theta_next", s["exp_theta"])))
         self.descs = B.make_descs(descs)
-        nbytes = B.kahan_sgd_workspace_bytes(self.descs)
-        assert nbytes > 0
-        self.workspace = torch.zeros(nbytes + 256, dtype=torch.uint8, device="cuda")
+        self.strict = strict
         self.stream = stream if stream is not None else torch.cuda.current_stream()
-        self.handle = B.kahan_sgd_init(self.descs, mode, self.workspace.data_ptr(), nbytes,
-                                       self.stream.cuda_stream)
+        if strict:
+            ec = [s["exp_comp"] for s in specs]
+            ec_next = [s.get("exp_comp_next", s["exp_comp"]) for s in specs]
+            nbytes = B.kahan_sgd_strict_workspace_bytes(self.descs, ec)
+            assert nbytes > 0
+            self.workspace = torch.zeros(nbytes + 256, dtype=torch.uint8, device="cuda")
+            self.handle = B.kahan_sgd_strict_init(self.descs, ec, ec_next, mode, self.workspace.data_ptr(), nbytes,
+                                                  self.stream.cuda_stream)
+        else:
+            nbytes = B.kahan_sgd_workspace_bytes(self.descs)
+            assert nbytes > 0
+            self.workspace = torch.zeros(nbytes + 256, dtype=torch.uint8, device="cuda")
+            self.handle = B.kahan_sgd_init(self.descs, mode, self.workspace.data_ptr(), nbytes,
+                                           self.stream.cuda_stream)
         self.grad_ptrs = [self.grad_arena.ptr(i) for i in range(self.n)]
 
     def step(self, grads: Sequence[np.ndarray], lrs: Sequence[float]) -> None:
@@ -107,7 +117,10 @@ class LibraryRun:
         self.B.kahan_sgd_set_exponents(self.handle, list(exps))
 
     def stats(self) -> dict:
-        return self.B.kahan_sgd_amax(self.handle, self.n)
+        st = self.B.kahan_sgd_amax(self.handle, self.n)
+        if self.strict:
+            st.update(self.B.kahan_sgd_strict_exponents(self.handle, self.n))
+        return st
 
     def thetas(self) -> List[np.ndarray]:
         self.torch.cuda.synchronize()
@@ -138,7 +151,9 @@ def make_oracle_state(specs, thetas, comps, mode, n_threads=1):
     for s, th, c in zip(specs, thetas, comps):
         ts.append(OracleTensor(th.copy(), None if c is None else c.copy(), s["theta_bits"],
                                s["comp_bits"], s.get("overlap_k", 0), s["exp_theta"],
-                               s.get("exp_theta_next", s["exp_theta"])))
+                               s.get("exp_theta_next", s["exp_theta"]),
+                               exp_comp=s.get("exp_comp", 0),
+                               exp_comp_next=s.get("exp_comp_next", s.get("exp_comp", 0))))
     return OracleState(ts, mode, n_threads)
 
 
@@ -160,6 +175,8 @@ def assert_same_state(gpu: LibraryRun, ost, where="") -> None:
         assert st["n_sat_theta"][i] == t.n_sat_theta, tag
         assert st["n_sat_comp"][i] == t.n_sat_comp, tag
         assert st["n_nonfinite"][i] == t.n_nonfinite, tag
+        if gpu.strict:
+            assert (st["exp_comp_cur"][i], st["exp_comp_next"][i]) == (t.exp_comp, t.exp_comp_next), tag
 
 
 def specs_of(wl) -> List[dict]:

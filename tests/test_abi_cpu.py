@@ -163,6 +163,26 @@ def test_adam_init_rejects_bad_descriptions_without_cuda(B):
     assert B.kahan_sgd_launch_count() == 0
 
 
+def test_strict_and_fixed_point_gradient_entry_points_reject_bad_arguments_without_cuda(B):
+    descs = B.make_descs([good()])
+    assert B.kahan_sgd_strict_workspace_bytes(descs, [-18]) > 0
+    for d, ec, nxt, code in [(good(comp_bits=0, comp=0), [-18], None, B.KSGD_ERR_BITS),
+                             (good(), [-11 - 37], None, B.KSGD_ERR_EXP_RANGE),      # e - ec = 37
+                             (good(), [-11 + 9], None, B.KSGD_ERR_EXP_RANGE),       # e - ec = -9
+                             (good(), [-18], [-11 - 40], B.KSGD_ERR_EXP_RANGE),
+                             (good(exp_theta=-40), [-70], None, B.KSGD_ERR_EXP_RANGE)]:
+        ds = B.make_descs([d])
+        if nxt is None:
+            assert B.kahan_sgd_strict_workspace_bytes(ds, ec) == 0
+        with pytest.raises(B.KahanSgdError) as ei:
+            B.kahan_sgd_strict_init(ds, ec, nxt, B.KSGD_EXP_AMAX, 0x100000, 1 << 20)
+        assert ei.value.code == code
+    assert B.lib.kahan_sgd_strict_init(None, descs, None, None, 1, 1, None, 0, None) == B.KSGD_ERR_NULL
+    assert B.lib.kahan_sgd_strict_exponents(None, None, None) == B.KSGD_ERR_NULL
+    assert B.lib.kahan_sgd_step_qgrad(None, None, 8, None, None) == B.KSGD_ERR_NULL
+    assert B.kahan_sgd_launch_count() == 0
+
+
 def test_classifier_bits_follow_eq_5_and_the_printed_example(B):
     import math
     rows = [ln.split() for ln in open(os.path.join(ROOT, "tests", "golden", "classifier_bitwidth.txt"))

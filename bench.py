@@ -92,6 +92,9 @@ def parse_args():
     ap.add_argument("--grad-bits", type=int, default=32, choices=[8, 16, 32],
                     help="8 or 16: the gradients are fixed-point tensors of that width (made on the device "
                          "from the binary32 ones before the timed region)")
+    ap.add_argument("--strict", action="store_true",
+                    help="strict Algorithm 1: every statement rounded into the stored format, the "
+                         "compensation with its own exponent")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-buckets", action="store_true",
@@ -204,8 +207,9 @@ def run_ours(args, rank, world, local_rank):
         t0_ = wl.tensors[0]
         adam = dict(beta1=0.9, beta2=0.999, eps=1e-8,
                     eta=1e-3 * 2.0 ** t0_.exp_theta * (2 ** (t0_.theta_bits - 1) - 1))
-    run = DeviceRun(host, B.KSGD_EXP_AMAX, mom_bits=args.momentum_bits, adam=adam, grad_bits=args.grad_bits)
-    other = bool(args.momentum_bits or args.adam or args.grad_bits != 32)
+    run = DeviceRun(host, B.KSGD_EXP_AMAX, mom_bits=args.momentum_bits, adam=adam, grad_bits=args.grad_bits,
+                    strict=args.strict)
+    other = bool(args.momentum_bits or args.adam or args.grad_bits != 32 or args.strict)
     if other:
         args.no_e2e = args.no_cpu_baseline = True      # those legs describe the plain step
     stream = run.stream
@@ -301,7 +305,8 @@ def run_ours(args, rank, world, local_rank):
                    "bytes_per_step": run.bytes_per_step, "grad_sets": n_sets,
                    "optimizer": "momentum 0.9, int%d velocity" % args.momentum_bits if args.momentum_bits
                    else ("adam 0.9/0.999/1e-8, int16 moments" if args.adam else
-                         ("sgd" if args.grad_bits == 32 else "sgd, int%d gradients" % args.grad_bits)),
+                         (("sgd" if args.grad_bits == 32 else "sgd, int%d gradients" % args.grad_bits) +
+                          (", strict Algorithm 1" if args.strict else ""))),
                    "l2": "inputs larger than L2 (%.0f MB touched per step)" % (wl.bytes_per_step / 1e6),
                    "exponent_mode": "amax", "input_generation_s": round(gen_s, 1)},
         "achieved_hbm_gbs": achieved,
@@ -310,7 +315,8 @@ def run_ours(args, rank, world, local_rank):
                      "frac_of_nominal_8000": achieved / 8000.0,
                      "kernel": "ksgd_momentum_step_kernel" if args.momentum_bits
                      else ("ksgd_adam_step_kernel" if args.adam else
-                           ("ksgd_step_kernel" if args.grad_bits == 32 else "ksgd_step_qgrad_kernel")),
+                           (("ksgd_strict_step" if args.strict else "ksgd_step") +
+                            ("_kernel" if args.grad_bits == 32 else "_qgrad_kernel"))),
                      "launch_ms": ms_step},
         "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
         "counters": {"n_sat_theta": int(sum(stats["n_sat_theta"])),

@@ -137,7 +137,7 @@ struct __align__(16) TileDesc {
   float scale;          // lr * 2^-(e_out - s), times 2^eg for fixed-point gradients
   float pow2s_neg;      // -2^s
   float inv2s;          // 2^-s
-  float qmax_t;         // 2^(m-1) - 1
+  float pow2dc;         // strict mode: 2^(ec_in - ec_out), c's old units in new ones; else 1
   void* theta;          // global address of the tile's first theta mantissa
   void* comp;           // same for the compensation (unused in plain mode)
   int tensor;
@@ -426,6 +426,10 @@ __device__ __forceinline__ void set_pack_word(Pack<BYTES>& r, int w, unsigned in
 // (y must stay below 2^24) or is Inf or NaN, or some |P| exceeds QMAX: exactly the cases
 // in which the magnitudes above could leave the exact range or a clamp is needed.
 
+// Strict mode (STRICT): u is statement 1's rounded result C1 = rne(qc * 2^(ec_in-ec_out) - d),
+// formed by one FMA onto M - d, so a change of c's exponent stays on this path; the vector
+// also leaves the path when |C1| or |r0| exceeds c's n bits (the clamps of statements 1, 3).
+
 constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23, bits 0x4B400000
 constexpr unsigned int kMagicBits = 0x4B400000u;
 
@@ -469,7 +473,7 @@ struct SteadyCoef {
   float scale;      // lr * 2^-(e - s)
   float pow2s_neg;  // -2^s
   float inv2s;      // 2^-s
-  float qmax_t;     // 2^(m-1) - 1
+  float pow2dc;     // 2^(ec_in - ec_out) (strict mode)
 };
 
 struct TileHot {       // the consumers' copy of the first 48 bytes of a TileDesc
@@ -501,10 +505,18 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
     const float x = __fmul_rn(g, k.scale);              // the one binary32 multiply
     sum_abs = __fadd_rn(sum_abs, fabsf(x));             // Inf or NaN if any x is
     aX = fmaxf(aX, fabsf(x));
-    const float y = __fadd_rn(x, kMagic + bias_c);      // rounds x to nearest-even integer
     float u;
-    if constexpr (HAS_COMP) u = __fadd_rn(magic_elem<(CB ? CB : 8)>(pc, i), -y);
-    else u = __fadd_rn(kMagic, -y);
+    if constexpr (STRICT) {
+      // statement 1 with c's own exponent: C1 = rne(Q_c * 2^(ec_in-ec_out) - d), one rounding
+      // (the FMA lands in [2^23, 2^24), where floats are the integers)
+      const float d = __fadd_rn(__fadd_rn(x, kMagic), -kMagic);
+      const float qc = __fadd_rn(magic_elem<(CB ? CB : 8)>(pc, i), -(kMagic + bias_c));
+      u = __fadd_rn(__fmaf_rn(qc, k.pow2dc, __fadd_rn(kMagic, -d)), -kMagic);
+    } else {
+      const float y = __fadd_rn(x, kMagic + bias_c);      // rounds x to nearest-even integer
+      if constexpr (HAS_COMP) u = __fadd_rn(magic_elem<(CB ? CB : 8)>(pc, i), -y);
+      else u = __fadd_rn(kMagic, -y);
+    }
     const float P = __fmaf_rn(u, k.inv2s, qtM);
     const float w = __fadd_rn(P, -qtM);
     const float r0 = __fmaf_rn(w, k.pow2s_neg, u);
@@ -514,7 +526,8 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
     if constexpr (HAS_COMP) aR = fmaxf(aR, fabsf(r0));
     if constexpr (STRICT) aU = fmaxf(aU, fabsf(u));     // u = c - d is statement 1's result
   }
-  if (!(sum_abs < 3.0e38f) | (aX > 4000000.0f) | (aP > k.qmax_t)) return false;
+  constexpr float qmax_t = (float)((1 << (TB - 1)) - 1);
+  if (!(sum_abs < 3.0e38f) | (aX > 4000000.0f) | (aP > qmax_t)) return false;
   if constexpr (STRICT) {
     // both accumulator results must fit their n bits, or the vector needs the clamps
     constexpr float qmax_c = (float)((1 << ((CB ? CB : 8) - 1)) - 1);
@@ -812,15 +825,14 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
         td.scale = scale_hot;
         td.pow2s_neg = -pow2_float(coef.s);
         td.inv2s = pow2_float(-coef.s);
-        td.qmax_t = (float)coef.qmax_t;
+        td.pow2dc = pow2_float(-coef.delta_c);
         td.theta = static_cast<unsigned char*>(ti.theta) + first * tbytes;
         td.comp = ti.comp ? static_cast<unsigned char*>(ti.comp) + first * cbytes : nullptr;
         td.tensor = cr.tensor;
         td.n_bulk = n_bulk;
         td.count = count;
         td.flags = ((ti.theta_bits == 16 ? 3 : 0) + (ti.comp_bits >> 3)) |
-                   ((coef.delta == 0 && scale_ok && (!STRICT || (coef.delta_c == 0 && coef.s >= 0))) ? kFlagSteady
-                                                                                                       : 0) |
+                   ((coef.delta == 0 && scale_ok && (!STRICT || coef.s >= 0)) ? kFlagSteady : 0) |
                    (page[1] << kFlagThetaPageShift) |
                    (page[2] << kFlagCompPageShift) | (page[0] << kFlagGradPageShift);
         td.coef = coef;
@@ -880,7 +892,7 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
         h.k.scale = __uint_as_float(q0.x);
         h.k.pow2s_neg = __uint_as_float(q0.y);
         h.k.inv2s = __uint_as_float(q0.z);
-        h.k.qmax_t = __uint_as_float(q0.w);
+        h.k.pow2dc = __uint_as_float(q0.w);
         h.theta = reinterpret_cast<unsigned char*>(((unsigned long long)q1.y << 32) | q1.x);
         h.comp = reinterpret_cast<unsigned char*>(((unsigned long long)q1.w << 32) | q1.z);
         h.tensor = (int)q2.x;

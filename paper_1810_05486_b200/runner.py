@@ -54,14 +54,16 @@ class DeviceRun:
     """Device buffers (same layout as HostInputs), descriptors, workspace and handle."""
 
     def __init__(self, host: HostInputs, mode: int = B.KSGD_EXP_AMAX, stream=None,
-                 mom_bits: int = 0, mu: float = 0.9, adam: Optional[dict] = None, grad_bits: int = 32):
+                 mom_bits: int = 0, mu: float = 0.9, adam: Optional[dict] = None, grad_bits: int = 32,
+                 strict: bool = False):
         """mom_bits = 8 or 16 selects the momentum optimizer (velocity buffers start at zero,
         on a grid 8 binades below theta's).  adam = dict(beta1, beta2, eps, eta) selects ADAM
         (both 16-bit moments start at zero, on grids that just hold what the first step makes of
         the largest gradient of the first set; the step size carries the bias correction of the
         step count).  grad_bits = 8 or 16 (plain optimizer only): every resident gradient set is
         turned into fixed-point tensors of that width on the device (exponent from the tensor's
-        maximum) and the steps read those."""
+        maximum) and the steps read those.  strict (plain optimizer only): strict Algorithm 1, the
+        compensation starting on the grid the ordinary mode ties it to."""
         import torch
         self.torch = torch
         self.host = host
@@ -111,11 +113,18 @@ class DeviceRun:
                                                     self.workspace.data_ptr(), self.ws_bytes,
                                                     self.stream.cuda_stream)
             self.mus = (ctypes.c_float * self.n)(*([mu] * self.n))
+        elif strict:
+            ec = [t.exp_theta - (t.comp_bits - 1 - t.overlap_k) for t in wl.tensors]
+            self.ws_bytes = B.kahan_sgd_strict_workspace_bytes(self.descs, ec)
+            self.workspace = torch.zeros(self.ws_bytes, dtype=torch.uint8, device="cuda")
+            self.handle = B.kahan_sgd_strict_init(self.descs, ec, None, mode, self.workspace.data_ptr(),
+                                                  self.ws_bytes, self.stream.cuda_stream)
         else:
             self.ws_bytes = B.kahan_sgd_workspace_bytes(self.descs)
             self.workspace = torch.zeros(self.ws_bytes, dtype=torch.uint8, device="cuda")
             self.handle = B.kahan_sgd_init(self.descs, mode, self.workspace.data_ptr(),
                                            self.ws_bytes, self.stream.cuda_stream)
+        self.strict = strict
         self.grad_ptr_sets = [(ctypes.c_void_p * self.n)(*[g.data_ptr() + o for o in host.g_offs])
                               for g in self.dev_g]
         self.grad_bits = grad_bits

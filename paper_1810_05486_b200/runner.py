@@ -194,6 +194,19 @@ class DeviceRun:
         o = self.host.c_offs[i]
         return self.dev_c[o:o + nb].cpu().numpy().view(W.storage_dtype(t.comp_bits))
 
+    def velocity(self, i: int) -> np.ndarray:
+        """Momentum mode: the velocity mantissas of tensor i."""
+        nb = self.wl.tensors[i].numel * (self.mom_bits // 8)
+        o = self.v_offs[i]
+        return self.dev_v[o:o + nb].cpu().numpy().view(W.storage_dtype(self.mom_bits))
+
+    def moments(self, i: int):
+        """ADAM mode: (first, second) moment mantissas of tensor i."""
+        nb = self.wl.tensors[i].numel * 2
+        o = self.m_offs[i]
+        return (self.dev_m1[o:o + nb].cpu().numpy().view(np.int16),
+                self.dev_m2[o:o + nb].cpu().numpy().view(np.int16))
+
     def host_pointer_arrays(self):
         """ctypes arrays of host addresses for kahan_sgd_step_host."""
         n = self.n

@@ -9,6 +9,7 @@
 #include <mutex>
 #include <new>
 #include <type_traits>
+#include <utility>
 #include <vector>
 
 #include "kahan_sgd_kernels.cuh"
@@ -35,6 +36,25 @@ int cuda_fail(cudaError_t e, const char* what) {
   } while (0)
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Launch a step kernel with programmatic stream serialization (see grid_dependency_wait in
+// the kernels): its blocks may start their prologue while the preceding kernel of the stream
+// finishes.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_step_kernel(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem,
+                               cudaStream_t stream, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // Offsets of the workspace regions.  The first four regions are contiguous so that
 // kahan_sgd_amax fetches them with one copy.
@@ -359,9 +379,11 @@ static int launch_step(ksgd_handle* h, const float* const* grads, const float* l
     KSGD_CUDA(cudaGetLastError());
   }
   if (h->strict)
-    ksgd_strict_step_kernel<<<(unsigned)h->grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, *ia);
+    KSGD_CUDA(launch_step_kernel(ksgd_strict_step_kernel, (unsigned)h->grid, kBlockThreads, kSharedBytes, h->stream,
+                                 h->params, *ia));
   else
-    ksgd_step_kernel<<<(unsigned)h->grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, *ia);
+    KSGD_CUDA(launch_step_kernel(ksgd_step_kernel, (unsigned)h->grid, kBlockThreads, kSharedBytes, h->stream,
+                                 h->params, *ia));
   g_launches.fetch_add(1, std::memory_order_relaxed);
   KSGD_CUDA(cudaGetLastError());
   return KSGD_OK;
@@ -405,17 +427,9 @@ int kahan_sgd_step_qgrad(ksgd_handle* h, const void* const* grads, int32_t grad_
     KSGD_CUDA(cudaGetLastError());
   }
   const unsigned grid = (unsigned)h->grid;
-  if (h->strict) {
-    if (grad_bits == 8)
-      ksgd_strict_step_qgrad_kernel<8><<<grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, args);
-    else
-      ksgd_strict_step_qgrad_kernel<16><<<grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, args);
-  } else {
-    if (grad_bits == 8)
-      ksgd_step_qgrad_kernel<8><<<grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, args);
-    else
-      ksgd_step_qgrad_kernel<16><<<grid, kBlockThreads, kSharedBytes, h->stream>>>(h->params, args);
-  }
+  auto kernel = h->strict ? (grad_bits == 8 ? ksgd_strict_step_qgrad_kernel<8> : ksgd_strict_step_qgrad_kernel<16>)
+                          : (grad_bits == 8 ? ksgd_step_qgrad_kernel<8> : ksgd_step_qgrad_kernel<16>);
+  KSGD_CUDA(launch_step_kernel(kernel, grid, kBlockThreads, kSharedBytes, h->stream, h->params, args));
   g_launches.fetch_add(1, std::memory_order_relaxed);
   KSGD_CUDA(cudaGetLastError());
   return KSGD_OK;
@@ -960,8 +974,8 @@ int kahan_sgd_momentum_step(ksgd_momentum_handle* h, const float* const* grads, 
                                     h->params.ws.mu);
     if (rc != KSGD_OK) return rc;
   }
-  mom::ksgd_momentum_step_kernel<<<(unsigned)h->grid, mom::kBlock, mom::kSharedBytes, h->stream>>>(h->params,
-                                                                                                  args);
+  KSGD_CUDA(launch_step_kernel(mom::ksgd_momentum_step_kernel, (unsigned)h->grid, mom::kBlock, mom::kSharedBytes,
+                               h->stream, h->params, args));
   g_launches.fetch_add(1, std::memory_order_relaxed);
   KSGD_CUDA(cudaGetLastError());
   return KSGD_OK;
@@ -1198,8 +1212,8 @@ int kahan_sgd_adam_step(ksgd_adam_handle* h, const float* const* grads, const fl
   args.beta1 = beta1;
   args.beta2 = beta2;
   args.eps = eps;
-  adam::ksgd_adam_step_kernel<<<(unsigned)h->grid, adam::kBlock, adam::kSharedBytes, h->stream>>>(h->params,
-                                                                                                args);
+  KSGD_CUDA(launch_step_kernel(adam::ksgd_adam_step_kernel, (unsigned)h->grid, adam::kBlock, adam::kSharedBytes,
+                               h->stream, h->params, args));
   g_launches.fetch_add(1, std::memory_order_relaxed);
   KSGD_CUDA(cudaGetLastError());
   return KSGD_OK;

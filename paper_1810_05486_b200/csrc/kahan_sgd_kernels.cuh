@@ -234,6 +234,21 @@ __device__ __forceinline__ void bulk_load_hint(void* dst_smem, const void* src_g
       : "memory");
 }
 
+// Programmatic dependent launch.  The step kernels are launched with programmatic stream
+// serialization: a block of the next kernel in the stream may become resident as soon as an
+// SM has room (a block of this kernel has exited) and run its prologue -- barrier set-up,
+// its first table entries -- while the rest of this kernel finishes.  Before it touches
+// anything an earlier kernel wrote (exponents, mantissas, gradients, per-step arguments in
+// the workspace) every thread passes grid_dependency_wait(), which returns once the
+// preceding kernel has completed and its writes are visible.  Launched the ordinary way
+// both instructions do nothing.  The hardware orders the grids; nothing spins.
+__device__ __forceinline__ void grid_dependency_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ unsigned long long l2_policy_evict_first() {
   unsigned long long pol;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
@@ -724,6 +739,7 @@ template <int GB, bool STRICT, typename Args>
 __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
   extern __shared__ __align__(128) unsigned char smem[];
   BlockShared* sh = reinterpret_cast<BlockShared*>(smem + (size_t)kPages * kPageBytes);
+  grid_dependency_launch_dependents();   // the next step's blocks may take over SMs as ours exit
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -754,10 +770,13 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
       const int tile0 = p.tile_begin + (int)blockIdx.x;
       const unsigned long long grad_policy = l2_policy_evict_first();
       ScanAcc acc;
+      // the tile table is written once at init: read the first entries before waiting for
+      // the preceding kernel
       ChunkRef cr = p.ws.chunks[tile0];
-      TensorMeta meta = load_meta(p, a, cr.tensor, STRICT);
       ChunkRef cr1{-1, -1};
       if (n_my > 1) cr1 = p.ws.chunks[tile0 + stride];
+      grid_dependency_wait();
+      TensorMeta meta = load_meta(p, a, cr.tensor, STRICT);
       int issued = 0;
       // The ring: pages from `head` on are free, tiles are released in the order they were
       // issued, `oldest` is the first tile whose pages have not been taken back yet.
@@ -867,9 +886,12 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
           mbar_wait(&sh->full[os], (unsigned)(i / kSlots) & 1u, &sh->never);
       }
       publish(p, acc);
+    } else {
+      grid_dependency_wait();
     }
   } else {
     // ------------------------------------------------------------------ consumers
+    grid_dependency_wait();
     const int ctid = threadIdx.x;
     const int stride = (int)gridDim.x;
     const int n_my = (p.tile_count - (int)blockIdx.x + stride - 1) / stride;

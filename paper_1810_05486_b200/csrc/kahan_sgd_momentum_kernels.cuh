@@ -388,6 +388,7 @@ ksgd_momentum_step_kernel(const __grid_constant__ StepParams p, const __grid_con
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int stride = (int)gridDim.x;
   const int n_my = ((int)p.n_chunks - (int)blockIdx.x + stride - 1) / stride;
+  grid_dependency_launch_dependents();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSlots; ++s) {
@@ -409,9 +410,10 @@ ksgd_momentum_step_kernel(const __grid_constant__ StepParams p, const __grid_con
       const unsigned long long grad_policy = l2_policy_evict_first();
       ScanAcc acc;
       ChunkRef cr = p.ws.chunks[blockIdx.x];
-      TensorMeta meta = load_meta(p, a, cr.tensor);
       ChunkRef cr1{-1, -1};
       if (n_my > 1) cr1 = p.ws.chunks[blockIdx.x + stride];
+      grid_dependency_wait();
+      TensorMeta meta = load_meta(p, a, cr.tensor);
       int issued = 0, head = 0, free_pages = kPages, oldest = 0;
       bool gave_up = false;
       for (int i = 0; i < n_my; ++i) {
@@ -507,9 +509,12 @@ ksgd_momentum_step_kernel(const __grid_constant__ StepParams p, const __grid_con
           mbar_wait(&sh->full[os], (unsigned)(i / kSlots) & 1u, &sh->never);
       }
       publish(p, acc);
+    } else {
+      grid_dependency_wait();
     }
   } else {
     // ------------------------------------------------------------------ consumers
+    grid_dependency_wait();
     const int ctid = threadIdx.x;
     float amax_t = 0.0f, amax_c = 0.0f, amax_v = 0.0f;
     for (int i = 0; i < n_my; ++i) {

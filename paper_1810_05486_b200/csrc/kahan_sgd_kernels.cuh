@@ -429,17 +429,20 @@ __device__ __forceinline__ void set_pack_word(Pack<BYTES>& r, int w, unsigned in
 // low mantissa bits are that integer in two's complement relative to M, an addition that
 // lands there rounds to nearest-even on the integer grid, and sums, differences and FMAs
 // of integers below 2^24 are exact.  Per element:
-//   qtM = M + qt, qcm = M + bias + qc   mantissa bytes spliced under M's exponent (PRMT)
-//   y   = g*scale + (M + bias)          = M + bias + d, d = rne(g*scale)   (stmt 1)
+//   qtB = M + bias_t + qt, qcm = M + bias_c + qc   mantissa bytes (sign bit flipped, so the
+//                                         byte is q + bias) spliced under M's exponent (PRMT)
+//   y   = g*scale + (M + bias_c)        = M + bias_c + d, d = rne(g*scale)   (stmt 1)
 //   u   = qcm - y                       = qc - d
-//   Pm  = fma(u, 2^-s, qtM)             = M + rne((qt*2^s + u) / 2^s) = M + P  (stmt 2;
-//                                         the tie falls on the parity of P itself)
-//   w   = Pm - qtM                      = P - qt
+//   Pb  = fma(u, 2^-s, qtB)             = M + bias_t + rne((qt*2^s + u) / 2^s) = M + bias_t + P
+//                                         (stmt 2; M and the bias are even, so the tie falls
+//                                         on the parity of P itself)
+//   w   = Pb - qtB                      = P - qt
 //   r0  = fma(w, -2^s, u)               = T - P*2^s                       (stmt 3)
-// theta' and c' are the low bits of Pm and of r0 + M.  The vector is handed to
-// update_general instead (returns false, nothing stored) when some |g*scale| exceeds 4e6
-// (y must stay below 2^24) or is Inf or NaN, or some |P| exceeds QMAX: exactly the cases
-// in which the magnitudes above could leave the exact range or a clamp is needed.
+// theta' is the low bits of Pb with the sign bit flipped back, c' the low bits of r0 + M.
+// The vector is handed to update_general instead (returns false, nothing stored) when some
+// |g*scale| exceeds 4e6 (y must stay below 2^24) or is Inf or NaN, or some |P| exceeds QMAX:
+// exactly the cases in which the magnitudes above could leave the exact range or a clamp is
+// needed.
 
 // Strict mode (STRICT): u is statement 1's rounded result C1 = rne(qc * 2^(ec_in-ec_out) - d),
 // formed by one FMA onto M - d, so a change of c's exponent stays on this path; the vector
@@ -498,6 +501,28 @@ struct TileHot {       // the consumers' copy of the first 48 bytes of a TileDes
   int tensor, n_bulk, count, flags;
 };
 
+// Three-input maximum / minimum (one instruction on sm_100a).  The .NaN form returns NaN as
+// soon as one input is NaN, which is how a NaN product reaches the range check below.
+__device__ __forceinline__ float max3_nan(float a, float b, float c) {
+  float d;
+  asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+  float d;
+  asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// theta stays biased through the vector: qtB = M + 2^(TB-1) + qt and Pb = M + 2^(TB-1) + P
+// (the bias is even, so the tie still falls on the parity of P); the sign bits of the packed
+// result are flipped back at the end.  The scans take two elements per instruction: the
+// largest and smallest Pb give max|P|, and |x|, |r0| go through three-input maxima.
 template <int TB, int CB, int V, int GB, bool STRICT>
 __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V * CB / 8 : 8)> pc,
                                               Pack<V * GB / 8> pg, const SteadyCoef& k,
@@ -506,20 +531,19 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
   constexpr bool HAS_COMP = CB != 0;
   constexpr float bias_t = (float)(1 << (TB - 1));
   constexpr float bias_c = HAS_COMP ? (float)(1 << ((CB ? CB : 8) - 1)) : 0.0f;
+  constexpr float Mt = kMagic + bias_t;
   flip_signs<TB>(pt);
   if constexpr (HAS_COMP) flip_signs<(CB ? CB : 8)>(pc);
   if constexpr (GB != 32) flip_signs<(GB == 32 ? 8 : GB)>(pg);
-  float Pm[V], rm[V];
-  float sum_abs = 0.0f, aX = 0.0f, aP = 0.0f, aR = 0.0f, aU = 0.0f;
+  float Pm[V], rm[V], xa[2], ra[2], ua[2];
+  float aX = 0.0f, hiP = Mt, loP = Mt, aR = 0.0f, aU = 0.0f;
 #pragma unroll
   for (int i = 0; i < V; ++i) {
-    const float qtM = __fadd_rn(magic_elem<TB>(pt, i), -bias_t);
+    const float qtB = magic_elem<TB>(pt, i);
     float g;       // binary32 gradient, or the gradient mantissa (k.scale then carries 2^eg)
     if constexpr (GB == 32) g = __uint_as_float(pack_word(pg, i));
     else g = __fadd_rn(magic_elem<(GB == 32 ? 8 : GB)>(pg, i), -(kMagic + (float)(1 << ((GB == 32 ? 8 : GB) - 1))));
     const float x = __fmul_rn(g, k.scale);              // the one binary32 multiply
-    sum_abs = __fadd_rn(sum_abs, fabsf(x));             // Inf or NaN if any x is
-    aX = fmaxf(aX, fabsf(x));
     float u;
     if constexpr (STRICT) {
       // statement 1 with c's own exponent: C1 = rne(Q_c * 2^(ec_in-ec_out) - d), one rounding
@@ -532,17 +556,25 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
       if constexpr (HAS_COMP) u = __fadd_rn(magic_elem<(CB ? CB : 8)>(pc, i), -y);
       else u = __fadd_rn(kMagic, -y);
     }
-    const float P = __fmaf_rn(u, k.inv2s, qtM);
-    const float w = __fadd_rn(P, -qtM);
+    const float P = __fmaf_rn(u, k.inv2s, qtB);
+    const float w = __fadd_rn(P, -qtB);
     const float r0 = __fmaf_rn(w, k.pow2s_neg, u);
     Pm[i] = P;
     rm[i] = __fadd_rn(r0, kMagic);
-    aP = fmaxf(aP, fabsf(__fadd_rn(P, -kMagic)));
-    if constexpr (HAS_COMP) aR = fmaxf(aR, fabsf(r0));
-    if constexpr (STRICT) aU = fmaxf(aU, fabsf(u));     // u = c - d is statement 1's result
+    xa[i & 1] = fabsf(x);
+    ra[i & 1] = fabsf(r0);
+    ua[i & 1] = fabsf(u);
+    if (i & 1) {
+      aX = max3_nan(aX, xa[0], xa[1]);                  // NaN if any product is
+      hiP = max3(hiP, Pm[i - 1], P);
+      loP = min3(loP, Pm[i - 1], P);
+      if constexpr (HAS_COMP) aR = max3(aR, ra[0], ra[1]);
+      if constexpr (STRICT) aU = max3(aU, ua[0], ua[1]);  // u = c - d is statement 1's result
+    }
   }
+  const float aP = fmaxf(__fadd_rn(hiP, -Mt), __fadd_rn(Mt, -loP));
   constexpr float qmax_t = (float)((1 << (TB - 1)) - 1);
-  if (!(sum_abs < 3.0e38f) | (aX > 4000000.0f) | (aP > qmax_t)) return false;
+  if (!(aX <= 4000000.0f) | (aP > qmax_t)) return false;   // also Inf and NaN products
   if constexpr (STRICT) {
     // both accumulator results must fit their n bits, or the vector needs the clamps
     constexpr float qmax_c = (float)((1 << ((CB ? CB : 8) - 1)) - 1);
@@ -552,6 +584,7 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
   amax_t = fmaxf(amax_t, aP);
   if constexpr (HAS_COMP) amax_c = fmaxf(amax_c, aR);
   ot = pack_magic<TB, V>(Pm);
+  flip_signs<TB>(ot);
   if constexpr (HAS_COMP) oc = pack_magic<CB, V>(rm);
   return true;
 }

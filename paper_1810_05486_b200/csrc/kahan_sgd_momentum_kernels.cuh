@@ -207,40 +207,49 @@ __device__ __forceinline__ bool update_vector(Pack<TB> pt, Pack<CB> pc, Pack<VB>
   constexpr int V = 8;
   constexpr float bias_t = (float)(1 << (TB - 1)), bias_c = (float)(1 << (CB - 1)),
                   bias_v = (float)(1 << (VB - 1));
+  constexpr float Mt = kMagic + bias_t;
   flip_signs<TB>(pt);
   flip_signs<CB>(pc);
   flip_signs<VB>(pv);
-  float Pm[V], rm[V], Vm[V];
-  float sum_abs = 0.0f, aP = 0.0f, aR = 0.0f, aV = 0.0f;
+  // theta stays biased (qtB = M + 2^(TB-1) + Qt, the bias is even so ties fall as before; the
+  // packed result gets its sign bits flipped back); scans take two elements per instruction
+  float Pm[V], rm[V], Vm[V], va[2], ra[2];
+  float hiP = Mt, loP = Mt, aR = 0.0f, aV = 0.0f;
 #pragma unroll
   for (int i = 0; i < V; ++i) {
-    const float qtM = __fadd_rn(magic_elem<TB>(pt, i), -bias_t);                  // M + Qt
+    const float qtB = magic_elem<TB>(pt, i);                                      // M + bias + Qt
     const float qc = __fadd_rn(magic_elem<CB>(pc, i), -(kMagic + bias_c));        // Qc
     const float qv = __fadd_rn(magic_elem<VB>(pv, i), -(kMagic + bias_v));        // Qv
     const float g = __uint_as_float(pack_word(pg, i));
     const float y = __fmaf_rn(k.mu_s, qv, __fmul_rn(g, k.scale_v));
-    sum_abs = __fadd_rn(sum_abs, fabsf(y));             // Inf or NaN if any y is
     const float vm = __fadd_rn(y, kMagic);              // M + rne(y)
-    const float v = __fadd_rn(vm, -kMagic);
+    const float v = __fadd_rn(vm, -kMagic);             // Inf or NaN if y is
     const float d = __fadd_rn(__fmaf_rn(v, k.pow2k, kMagic), -kMagic);
     const float u = __fadd_rn(qc, -d);
-    const float P = __fmaf_rn(u, k.inv2s, qtM);
-    const float w = __fadd_rn(P, -qtM);
+    const float P = __fmaf_rn(u, k.inv2s, qtB);
+    const float w = __fadd_rn(P, -qtB);
     const float r0 = __fmaf_rn(w, k.pow2s_neg, u);
     Pm[i] = P;
     rm[i] = __fadd_rn(r0, kMagic);
     Vm[i] = vm;
-    aP = fmaxf(aP, fabsf(__fadd_rn(P, -kMagic)));
-    aR = fmaxf(aR, fabsf(r0));
-    aV = fmaxf(aV, fabsf(v));
+    va[i & 1] = fabsf(v);
+    ra[i & 1] = fabsf(r0);
+    if (i & 1) {
+      aV = max3_nan(aV, va[0], va[1]);                  // NaN if any y is
+      hiP = max3(hiP, Pm[i - 1], P);
+      loP = min3(loP, Pm[i - 1], P);
+      aR = max3(aR, ra[0], ra[1]);
+    }
   }
+  const float aP = fmaxf(__fadd_rn(hiP, -Mt), __fadd_rn(Mt, -loP));
   // |y| > 4e6 (where y + M stops being exact) shows as |V| far beyond QMAX_v, so the velocity
-  // bound covers it
-  if (!(sum_abs < 3.0e38f) | (aV > k.qmax_v) | (aV > k.d_limit) | (aP > k.qmax_t)) return false;
+  // bound covers it; a NaN fails the same comparison
+  if (!(aV <= k.qmax_v) | !(aV <= k.d_limit) | (aP > k.qmax_t)) return false;
   amax_t = fmaxf(amax_t, aP);
   amax_c = fmaxf(amax_c, aR);
   amax_v = fmaxf(amax_v, aV);
   ot = pack_magic<TB, V>(Pm);
+  flip_signs<TB>(ot);
   oc = pack_magic<CB, V>(rm);
   ov = pack_magic<VB, V>(Vm);
   return true;

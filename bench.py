@@ -381,6 +381,7 @@ def time_size_buckets(torch, B, run, wl, steps=20):
         descs = B.make_descs(sub)
         nb = B.kahan_sgd_workspace_bytes(descs)
         ws = torch.zeros(nb, dtype=torch.uint8, device="cuda")
+        torch.cuda.synchronize()      # the fill ran on torch's stream, the library works on run.stream
         h = B.kahan_sgd_init(descs, B.KSGD_EXP_AMAX, ws.data_ptr(), nb, run.stream.cuda_stream)
         gp = [(ctypes.c_void_p * len(idx))(*[run.grad_ptr_sets[k][i] for i in idx]) for k in range(2)]
         lr = (ctypes.c_float * len(idx))(*([wl.lr] * len(idx)))

@@ -99,6 +99,7 @@ class DeviceRun:
             self.adescs = B.make_adam_descs(adescs)
             self.ws_bytes = B.kahan_sgd_adam_workspace_bytes(self.descs, self.adescs)
             self.workspace = torch.zeros(self.ws_bytes, dtype=torch.uint8, device="cuda")
+            torch.cuda.synchronize()     # the fills above ran on torch's stream, the library works on self.stream
             self.handle = B.kahan_sgd_adam_init(self.descs, self.adescs, mode, self.workspace.data_ptr(),
                                                 self.ws_bytes, self.stream.cuda_stream)
         elif mom_bits:
@@ -109,6 +110,7 @@ class DeviceRun:
                      exp_mom=t.exp_theta - 8) for i, t in enumerate(wl.tensors)])
             self.ws_bytes = B.kahan_sgd_momentum_workspace_bytes(self.descs, self.mdescs)
             self.workspace = torch.zeros(self.ws_bytes, dtype=torch.uint8, device="cuda")
+            torch.cuda.synchronize()     # the fills above ran on torch's stream, the library works on self.stream
             self.handle = B.kahan_sgd_momentum_init(self.descs, self.mdescs, mode,
                                                     self.workspace.data_ptr(), self.ws_bytes,
                                                     self.stream.cuda_stream)
@@ -117,11 +119,13 @@ class DeviceRun:
             ec = [t.exp_theta - (t.comp_bits - 1 - t.overlap_k) for t in wl.tensors]
             self.ws_bytes = B.kahan_sgd_strict_workspace_bytes(self.descs, ec)
             self.workspace = torch.zeros(self.ws_bytes, dtype=torch.uint8, device="cuda")
+            torch.cuda.synchronize()     # the fills above ran on torch's stream, the library works on self.stream
             self.handle = B.kahan_sgd_strict_init(self.descs, ec, None, mode, self.workspace.data_ptr(),
                                                   self.ws_bytes, self.stream.cuda_stream)
         else:
             self.ws_bytes = B.kahan_sgd_workspace_bytes(self.descs)
             self.workspace = torch.zeros(self.ws_bytes, dtype=torch.uint8, device="cuda")
+            torch.cuda.synchronize()     # the fills above ran on torch's stream, the library works on self.stream
             self.handle = B.kahan_sgd_init(self.descs, mode, self.workspace.data_ptr(),
                                            self.ws_bytes, self.stream.cuda_stream)
         self.strict = strict
@@ -135,6 +139,7 @@ class DeviceRun:
             self.dev_gq, self.gq_ptr_sets, self.gq_exp_sets = [], [], []
             for gset in self.dev_g:
                 q = torch.zeros(q_bytes, dtype=torch.uint8, device="cuda")
+                torch.cuda.synchronize()     # the fill must not overtake the import kernels on self.stream
                 exps = [B.kahan_sgd_import(gset.data_ptr() + host.g_offs[i], q.data_ptr() + self.q_offs[i], None,
                                            t.numel, grad_bits, 0, 0, B.KSGD_EXP_AUTO, scratch.data_ptr(),
                                            self.stream.cuda_stream) for i, t in enumerate(wl.tensors)]

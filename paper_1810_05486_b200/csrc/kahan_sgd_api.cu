@@ -64,10 +64,24 @@ struct Layout {
   long long n_chunks;
 };
 
-Layout make_layout(const ksgd_tensor_desc* d, int32_t n) {
+// Tile size of a tensor, given the list's tile size for 8-bit theta.
+inline long long tile_elems(const ksgd_tensor_desc& t, int chunk8) { return t.theta_bits == 8 ? chunk8 : kChunk; }
+
+// Tile size for tensors with 8-bit theta: the large one if the list then still has
+// kBigTileMinTiles tiles (about seven per block), so that short lists keep every block busy.
+int pick_chunk8(const ksgd_tensor_desc* d, int32_t n) {
+  long long tiles = 0;
+  for (int32_t i = 0; i < n; ++i) {
+    const long long c = tile_elems(d[i], 2 * kChunk);
+    tiles += (d[i].numel + c - 1) / c;
+  }
+  return tiles >= kBigTileMinTiles ? 2 * kChunk : kChunk;
+}
+
+Layout make_layout(const ksgd_tensor_desc* d, int32_t n, int chunk8) {
   Layout L{};
   long long chunks = 0;
-  for (int32_t i = 0; i < n; ++i) chunks += (d[i].numel + kChunk - 1) / kChunk;
+  for (int32_t i = 0; i < n; ++i) chunks += (d[i].numel + tile_elems(d[i], chunk8) - 1) / tile_elems(d[i], chunk8);
   L.n_chunks = chunks;
   size_t o = 0;
   L.exp_cur = o;   o += sizeof(int) * n;
@@ -139,7 +153,7 @@ extern "C" {
 
 size_t kahan_sgd_workspace_bytes(const ksgd_tensor_desc* descs, int32_t n_tensors) {
   if (validate(descs, n_tensors) != KSGD_OK) return 0;
-  return make_layout(descs, n_tensors).total;
+  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors)).total;
 }
 
 }  // extern "C"
@@ -174,7 +188,8 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   if (mode != KSGD_EXP_FIXED && mode != KSGD_EXP_AMAX) return KSGD_ERR_MODE;
   if (!workspace) return KSGD_ERR_NULL;
   if (reinterpret_cast<uintptr_t>(workspace) % 256) return KSGD_ERR_ALIGN;
-  const Layout L = make_layout(descs, n_tensors);
+  const int chunk8 = pick_chunk8(descs, n_tensors);
+  const Layout L = make_layout(descs, n_tensors, chunk8);
   if (workspace_bytes < L.total) return KSGD_ERR_WORKSPACE;
 
   ksgd_handle* h = new (std::nothrow) ksgd_handle();
@@ -214,7 +229,7 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
     info[i].comp_bits = t.comp_bits;
     info[i].s = t.comp_bits ? t.comp_bits - 1 - t.overlap_k : 0;
     info[i].pad = 0;
-    const long long nc = (t.numel + kChunk - 1) / kChunk;
+    const long long nc = (t.numel + tile_elems(t, chunk8) - 1) / tile_elems(t, chunk8);
     h->first_tile.push_back(c);
     for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
   }
@@ -280,7 +295,7 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   for (int32_t i = 0; i < n_tensors; ++i)
     state_bytes += (double)descs[i].numel * ((descs[i].theta_bits + descs[i].comp_bits) / 8);
   h->params.grad_evict_first = state_bytes <= 0.8 * (double)l2_bytes ? 1 : 0;
-  h->params.pad = 0;
+  h->params.chunk8 = chunk8;
 
   e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
@@ -307,7 +322,7 @@ size_t kahan_sgd_strict_workspace_bytes(const ksgd_tensor_desc* descs, const int
                                         int32_t n_tensors) {
   if (validate(descs, n_tensors) != KSGD_OK) return 0;
   if (validate_strict(descs, exp_comp, nullptr, n_tensors) != KSGD_OK) return 0;
-  return make_layout(descs, n_tensors).total;
+  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors)).total;
 }
 
 int kahan_sgd_strict_init(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t* exp_comp,
@@ -655,7 +670,7 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   if (mode != KSGD_EXP_FIXED && mode != KSGD_EXP_AMAX) return KSGD_ERR_MODE;
   if (!grads || !lrs) return KSGD_ERR_NULL;
   if (n_tensors > KSGD_STATIC_MAX_TENSORS) return KSGD_ERR_WORKSPACE;
-  const Layout L = make_layout(descs, n_tensors);
+  const Layout L = make_layout(descs, n_tensors, kChunk);
   if (L.total > (size_t)KSGD_STATIC_SCRATCH_BYTES) return KSGD_ERR_WORKSPACE;
   for (int32_t i = 0; i < n_tensors; ++i) {
     if (!grads[i]) return KSGD_ERR_NULL;
@@ -736,7 +751,7 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   params.tensor_begin = 0;
   params.tensor_count = n_tensors;
   params.grad_evict_first = state_bytes <= 0.8 * (double)sd.l2_bytes ? 1 : 0;
-  params.pad = 0;
+  params.chunk8 = kChunk;
 
   InlineArgs inl;
   for (int32_t i = 0; i < n_tensors; ++i) { inl.grads[i] = grads[i]; inl.lrs[i] = lrs[i]; }

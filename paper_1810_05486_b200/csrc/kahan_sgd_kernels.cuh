@@ -12,8 +12,8 @@
 // The pass is bound by HBM traffic: 2*m/8 + 2*n/8 + 4 bytes per parameter.
 //
 // Structure: a persistent grid, one block per SM.  The tensor list is cut into tiles of
-// kChunk elements; block b takes tiles b, b + gridDim.x, ....  One producer thread
-// streams the tiles of theta, c and g into a 224 KB shared-memory ring with bulk
+// kChunk elements (2 * kChunk for 8-bit theta in long lists); block b takes tiles b,
+// b + gridDim.x, ....  One producer thread streams the tiles of theta, c and g into a 224 KB shared-memory ring with bulk
 // asynchronous copies (cp.async.bulk, completion counted on an mbarrier), so the bytes in
 // flight do not depend on registers or occupancy; a tile takes only the pages its format
 // needs (6 for int8/int8, 8 for int16/int16), so three to four tiles are resident.
@@ -28,12 +28,14 @@
 
 namespace ksgd {
 
-constexpr int kChunk = 8192;           // elements per tile
+constexpr int kChunk = 8192;           // elements per tile (twice as many for 8-bit theta in long lists)
+constexpr long long kBigTileMinTiles = 1024;   // a list gets the large 8-bit tiles if it still has this many tiles
 constexpr int kConsumerWarps = 16;
 constexpr int kConsumers = kConsumerWarps * 32;
 constexpr int kBlockThreads = kConsumers + 32;   // + one producer warp
 constexpr int kSlots = 6;              // tiles a block can have in its ring at once
 constexpr int kPageBytes = 8192;       // the ring is handed out in pages
+static_assert(kChunk == 8192 && kPageBytes == kChunk, "the producer's page arithmetic assumes 8192-element tiles and 8 KB pages");
 constexpr int kPages = 28;             // 224 KB of tile data per block
 constexpr int kInlineArgs = 256;     // lists up to this long pass grads/lrs as kernel parameters
 constexpr int kUploadBatch = 1024;   // tensors per launch of the argument-upload kernel
@@ -56,7 +58,7 @@ struct TensorInfo {
 
 struct ChunkRef {
   int tensor;  // index into the tensor list
-  int index;   // tile number inside that tensor: elements [index*kChunk, ...)
+  int index;   // tile number inside that tensor: elements [index*chunk, ...), chunk = the tensor's tile size
 };
 
 // Device-side view of the caller's workspace.
@@ -88,7 +90,11 @@ struct StepParams {
   // of tensors [tensor_begin, tensor_begin + tensor_count): the whole list for an ordinary
   // step, one group of tensors when the host-buffer entry point pipelines its copies.
   int tile_begin, tile_count, tensor_begin, tensor_count;
-  int pad;
+  // Elements per tile of tensors with 8-bit theta: kChunk, or 2 * kChunk for lists long
+  // enough to keep every block busy with the larger tiles (one vector per thread and tile
+  // leaves the per-tile work of a consumer -- wait, descriptor, scans, arrive -- a third of
+  // its instructions).  Tensors with 16-bit theta always take kChunk.
+  int chunk8;
 };
 
 struct InlineArgs {
@@ -827,7 +833,10 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
         // where the three arrays go (g, theta, c), and how many pages that takes including
         // those skipped when a run does not fit before the end of the ring
         constexpr int gbytes = GB / 8;
-        const int run[3] = {kChunk * gbytes / kPageBytes, kChunk * tbytes / kPageBytes, kChunk * cbytes / kPageBytes};
+        // kChunk == kPageBytes: an array of b-byte elements takes b pages (2b with the large tiles)
+        const int big = (ti.theta_bits == 8 && p.chunk8 != kChunk) ? 1 : 0;
+        const int chunk = kChunk << big;
+        const int run[3] = {gbytes << big, tbytes << big, cbytes << big};
         int page[3] = {0, 0, 0}, h2 = head, need = 0;
 #pragma unroll
         for (int r = 0; r < 3; ++r) {
@@ -869,9 +878,9 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
           scale_ok = ex != 0 && ex + meta.eg >= 1 && ex + meta.eg <= 254;
           if (scale_ok) scale_hot = __int_as_float(__float_as_int(coef.scale) + (meta.eg << 23));
         }
-        const long long first = (long long)cr.index * kChunk;
+        const long long first = (long long)cr.index << (13 + big);
         const long long left = ti.numel - first;
-        const int count = left < (long long)kChunk ? (int)left : kChunk;
+        const int count = left < (long long)chunk ? (int)left : chunk;
         const int n_bulk = count & ~15;
         TileDesc& td = sh->desc[slot];
         td.scale = scale_hot;

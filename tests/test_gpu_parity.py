@@ -251,6 +251,39 @@ def test_mixed_formats_in_one_list_and_long_lists():
     run_both(specs, thetas, comps, grads, lrs, EXP_AMAX)
 
 
+def test_long_lists_with_8bit_theta_take_the_large_tiles():
+    """A list long enough for the 16384-element tiles of 8-bit theta (the library picks the
+    tile size per list): every 8-bit format, sizes around the large and the small tile
+    boundary, 16-bit tensors (which keep the small tiles) in between, an exponent change and
+    saturating steps included."""
+    rng = np.random.default_rng(77)
+    T = 16384
+    sizes8 = [T * 300 + 5, T * 270 + T - 1, T * 260 + 8193, T * 250, T + 1, T - 1, 8192, 8193, 17, 1, 3 * T + 16]
+    specs, thetas, comps = [], [], []
+    for i, n in enumerate(sizes8):
+        tb, cb = [(8, 8), (8, 0), (8, 16)][i % 3]
+        th, c = random_tensor(rng, n, tb, cb, full_range=(i % 4 == 0))
+        specs.append(dict(numel=n, theta_bits=tb, comp_bits=cb, overlap_k=0, exp_theta=-11))
+        thetas.append(th)
+        comps.append(c)
+    for n, (tb, cb) in [(8192 * 5 + 9, (16, 16)), (100003, (16, 8)), (16384, (16, 0))]:
+        th, c = random_tensor(rng, n, tb, cb, full_range=False)
+        specs.append(dict(numel=n, theta_bits=tb, comp_bits=cb, overlap_k=0, exp_theta=-17))
+        thetas.append(th)
+        comps.append(c)
+    assert sum((sp["numel"] + T - 1) // T for sp in specs if sp["theta_bits"] == 8) >= 1024
+    grads, lrs = [], []
+    for step in range(4):
+        gs = []
+        for sp in specs:
+            s = sp["comp_bits"] - 1 if sp["comp_bits"] else 0
+            sigma = 2.0 ** (sp["exp_theta"] - s) * (4000 if step == 2 else 40) / 0.1
+            gs.append((rng.standard_normal(sp["numel"]) * sigma).astype(np.float32))
+        grads.append(gs)
+        lrs.append([0.1] * len(specs))
+    run_both(specs, thetas, comps, grads, lrs, EXP_AMAX)
+
+
 def test_checkpoint_resume_is_bit_identical():
     """N steps in one go == N/2 steps, read the state back, re-init from it, N/2 more."""
     rng = np.random.default_rng(31)

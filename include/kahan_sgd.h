@@ -93,6 +93,10 @@ size_t kahan_sgd_workspace_bytes(const ksgd_tensor_desc* descs, int32_t n_tensor
  * valid and untouched by the caller until kahan_sgd_destroy.  cuda_stream: the
  * cudaStream_t (as void*) all later work is enqueued on; NULL = the legacy default
  * stream.  Waits for its copies to finish.  On error *out is NULL.
+ * Ordering: the library orders its work on cuda_stream only.  Whatever the caller still
+ * has in flight on another stream that writes the workspace, theta, comp or the gradients
+ * (a zero-fill of a fresh allocation, an upload) must have finished, or be ordered before
+ * cuda_stream by an event, when this call and the later steps are made.
  * (State of Algorithm 1: "Require theta, ..., previous theta, previous acc".)
  */
 int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_tensors,

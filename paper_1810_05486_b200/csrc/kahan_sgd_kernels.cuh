@@ -16,7 +16,8 @@
 // b + gridDim.x, ....  One producer thread streams the tiles of theta, c and g into a 224 KB shared-memory ring with bulk
 // asynchronous copies (cp.async.bulk, completion counted on an mbarrier), so the bytes in
 // flight do not depend on registers or occupancy; a tile takes only the pages its format
-// needs (6 for int8/int8, 8 for int16/int16), so three to four tiles are resident.
+// needs (6 for int8/int8 -- 12 with the large tiles --, 8 for int16/int16), so two to four
+// tiles are resident.
 // Sixteen consumer warps compute from shared memory and store theta' and c' straight to
 // global memory with 16-byte stores.
 // No block ever waits for another block; every wait inside a block is bounded.

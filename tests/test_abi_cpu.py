@@ -93,6 +93,20 @@ def test_workspace_grows_with_the_chunk_table(B):
     assert big < 2 << 20
 
 
+def test_long_lists_of_8bit_theta_get_the_large_tiles(B):
+    """The tile table (8 bytes per tile) shows which tile size a list got: 8192 elements,
+    or 16384 for 8-bit theta once the list still has 1024 tiles with them; 16-bit theta
+    always keeps 8192."""
+    def table_bytes(numel, **kw):
+        return (B.kahan_sgd_workspace_bytes(B.make_descs([good(numel=numel, **kw)])) -
+                B.kahan_sgd_workspace_bytes(B.make_descs([good(numel=1, **kw)])))
+    short, long_ = 1023 * 16384, 1024 * 16384
+    assert abs(table_bytes(short) - 8 * (short // 8192)) <= 512          # small tiles
+    assert abs(table_bytes(long_) - 8 * 1024) <= 512                     # large tiles
+    wide = dict(theta_bits=16, comp_bits=16)
+    assert abs(table_bytes(long_, **wide) - 8 * (long_ // 8192)) <= 512  # 16-bit theta: small tiles
+
+
 def test_null_handles_and_strerror(B):
     assert B.lib.kahan_sgd_step(None, None, None) == B.KSGD_ERR_NULL
     assert B.lib.kahan_sgd_amax(None, *([None] * 7)) == B.KSGD_ERR_NULL

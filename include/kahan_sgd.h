@@ -87,6 +87,16 @@ enum {
 size_t kahan_sgd_workspace_bytes(const ksgd_tensor_desc* descs, int32_t n_tensors);
 
 /*
+ * Byte offset, inside the workspace of this list, of the 4-byte word in which a kernel
+ * records the first bounded wait that ran out (0 = none; the word is sticky and
+ * kahan_sgd_amax turns a non-zero value into KSGD_ERR_DEVICE).  For diagnostics, and for
+ * tests of the caller's error handling that set the word from the host instead of making a
+ * GPU wait run out.  Host-only computation; (size_t)-1 if the list is invalid.  (No
+ * counterpart in the paper: part of the error behaviour of this boundary.)
+ */
+size_t kahan_sgd_workspace_error_offset(const ksgd_tensor_desc* descs, int32_t n_tensors);
+
+/*
  * Validate the list, lay out the workspace and copy the chunk table and initial
  * exponents to it.  descs: host array of n_tensors entries, copied.  workspace: device,
  * caller-owned, at least kahan_sgd_workspace_bytes, 256-byte aligned; it must stay
@@ -171,9 +181,8 @@ int kahan_sgd_set_exponents(ksgd_handle* h, const int32_t* exp_theta_next);
  * kahan_sgd_init needs a device workspace from its caller, and some callers have no way to
  * get one at the moment they need it: a plug-in running inside a host program that has
  * already handed all device memory to its own pool and forbids further cudaMalloc calls;
- * a latency-critical loop where cudaMalloc's device-wide synchronisation is unacceptable;
- * code that runs while another thread is recording a stream capture in a mode that makes
- * allocation calls illegal.  For them the same scratch (exponents, max-scan slots,
+ * a latency-critical loop where cudaMalloc's device-wide synchronisation is unacceptable.
+ * For them the same scratch (exponents, max-scan slots,
  * counters, tile table) lives in a fixed array of KSGD_STATIC_SCRATCH_BYTES inside the
  * library's device image, which every GPU that loads the library holds until the process
  * exits.  The call allocates and frees no device memory, directly or through any library.
@@ -193,10 +202,15 @@ int kahan_sgd_set_exponents(ksgd_handle* h, const int32_t* exp_theta_next);
  * does nothing.
  *
  * The first call on each device looks up the array's device address and sets a kernel
- * attribute; make that first call with the device current and before any stream capture
- * begins.  All calls on a device share the one array and each call rewrites all of it, so
- * two calls whose work overlaps on the GPU (different streams, different threads) race:
- * callers serialise them.
+ * attribute; make that first call before any stream capture begins.  Every call takes the
+ * array, the SM count and the L2 size of the device that is current when it is made:
+ * the device that owns cuda_stream must be current on every call, not just the first.
+ * Every call copies to and from pageable host memory and waits for the stream, so the call
+ * itself synchronises and cannot be part of a stream capture.  All calls on a device share
+ * the one array and each call rewrites all of it, so two calls whose work overlaps on the
+ * GPU (different streams, different threads) race: callers serialise them.  The list is
+ * always cut into tiles of 8192 elements (the workspace path takes 16384-element tiles for
+ * long lists of 8-bit tensors), which changes no result.
  */
 #define KSGD_STATIC_SCRATCH_BYTES (192 * 1024)
 #define KSGD_STATIC_MAX_TENSORS 256
@@ -225,7 +239,10 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
  * kahan_sgd_strict_init: as kahan_sgd_init, plus exp_comp / exp_comp_next (host arrays, one
  * per tensor: c's exponent now stored and the one the first step writes; exp_comp_next NULL
  * = the same).  Every tensor needs comp_bits != 0 (else KSGD_ERR_BITS); overlap_k is
- * ignored; exponents outside [-64, 64] or outside the window above give KSGD_ERR_EXP_RANGE.
+ * ignored; exponents outside [-64, 64] or outside the window above, or a first-step change
+ * of c's exponent of more than 16 (the most the rule above ever asks for: 8 of its own fit
+ * plus 8 of theta's move; the 64-bit sums of a step are only guaranteed up to there), give
+ * KSGD_ERR_EXP_RANGE.
  * The handle then works with kahan_sgd_step, kahan_sgd_step_qgrad, kahan_sgd_amax and
  * kahan_sgd_destroy; kahan_sgd_step_host, kahan_sgd_set_exponents and
  * kahan_sgd_strict_exponents on the wrong kind of handle return KSGD_ERR_MODE.

@@ -575,6 +575,9 @@ int ksgd_oracle_strict_step_tensor(void* theta, void* comp, const float* grad, i
   if (!theta || !comp || !grad || !stats || numel <= 0) return -1;
   if (theta_bits < 2 || theta_bits > 16 || comp_bits < 2 || comp_bits > 16) return -1;
   if (!strict_window_ok(e_in, ec_in) || !strict_window_ok(e_out, ec_out)) return -1;
+  /* outside this the 64-bit sums of the element could overflow; the exponent rule below
+   * never asks for more (its own fit moves at most 8, theta's window at most 8 more) */
+  if (ec_out - ec_in > 16 || ec_in - ec_out > 16 || e_out - e_in > 8 || e_in - e_out > 8) return -1;
   uint32_t amax_theta = 0, amax_comp = 0;
   uint64_t n_sat_theta = 0, n_sat_comp = 0, n_nonfinite = 0;
   if (n_threads < 1) n_threads = 1;

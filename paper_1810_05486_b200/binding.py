@@ -28,7 +28,7 @@ KSGD_ERR_MODE = -10
 KSGD_ERR_DEVICE = -11
 
 EXPORTS = (
-    "kahan_sgd_workspace_bytes", "kahan_sgd_init", "kahan_sgd_step", "kahan_sgd_step_qgrad",
+    "kahan_sgd_workspace_bytes", "kahan_sgd_workspace_error_offset", "kahan_sgd_init", "kahan_sgd_step", "kahan_sgd_step_qgrad",
     "kahan_sgd_step_host", "kahan_sgd_strict_workspace_bytes", "kahan_sgd_strict_init",
     "kahan_sgd_strict_exponents",
     "kahan_sgd_amax", "kahan_sgd_set_exponents", "kahan_sgd_step_static", "kahan_sgd_destroy",
@@ -82,6 +82,8 @@ def _load() -> ctypes.CDLL:
     P = ctypes.POINTER
     lib.kahan_sgd_workspace_bytes.restype = ctypes.c_size_t
     lib.kahan_sgd_workspace_bytes.argtypes = [P(ksgd_tensor_desc), ctypes.c_int32]
+    lib.kahan_sgd_workspace_error_offset.restype = ctypes.c_size_t
+    lib.kahan_sgd_workspace_error_offset.argtypes = [P(ksgd_tensor_desc), ctypes.c_int32]
     lib.kahan_sgd_init.restype = ctypes.c_int
     lib.kahan_sgd_init.argtypes = [P(ctypes.c_void_p), P(ksgd_tensor_desc), ctypes.c_int32,
                                    ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
@@ -187,6 +189,14 @@ def make_descs(tensors: Sequence[dict]):
 
 def kahan_sgd_workspace_bytes(descs) -> int:
     return int(lib.kahan_sgd_workspace_bytes(descs, len(descs)))
+
+
+def kahan_sgd_workspace_error_offset(descs) -> int:
+    """Byte offset of the sticky device-error word inside this list's workspace."""
+    off = int(lib.kahan_sgd_workspace_error_offset(descs, len(descs)))
+    if off == ctypes.c_size_t(-1).value:
+        raise KahanSgdError(KSGD_ERR_NUMEL, "invalid tensor list")
+    return off
 
 
 def kahan_sgd_init(descs, mode: int, workspace: int, workspace_bytes: int, stream: int = 0):

@@ -156,6 +156,11 @@ size_t kahan_sgd_workspace_bytes(const ksgd_tensor_desc* descs, int32_t n_tensor
   return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors)).total;
 }
 
+size_t kahan_sgd_workspace_error_offset(const ksgd_tensor_desc* descs, int32_t n_tensors) {
+  if (validate(descs, n_tensors) != KSGD_OK) return (size_t)-1;
+  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors)).error;
+}
+
 }  // extern "C"
 
 namespace {
@@ -170,6 +175,9 @@ int validate_strict(const ksgd_tensor_desc* d, const int32_t* ec, const int32_t*
     if (ec[i] < kExpMin || ec[i] > kExpMax || nx < kExpMin || nx > kExpMax) return KSGD_ERR_EXP_RANGE;
     if (!strict_window_ok(d[i].exp_theta, ec[i]) || !strict_window_ok(d[i].exp_theta_next, nx))
       return KSGD_ERR_EXP_RANGE;
+    // the device never moves c's exponent by more than 2 * kMaxDelta in one step (its own
+    // fit plus theta's move); a larger first-step change would shift past 64 bits
+    if (std::abs(nx - ec[i]) > 2 * kMaxDelta) return KSGD_ERR_EXP_RANGE;
   }
   return KSGD_OK;
 }

@@ -184,6 +184,8 @@ def test_strict_and_fixed_point_gradient_entry_points_reject_bad_arguments_witho
                              (good(), [-11 - 37], None, B.KSGD_ERR_EXP_RANGE),      # e - ec = 37
                              (good(), [-11 + 9], None, B.KSGD_ERR_EXP_RANGE),       # e - ec = -9
                              (good(), [-18], [-11 - 40], B.KSGD_ERR_EXP_RANGE),
+                             # inside both windows, but c's exponent would move by 17 in one step
+                             (good(exp_theta=0, exp_theta_next=8), [-20], [-3], B.KSGD_ERR_EXP_RANGE),
                              (good(exp_theta=-40), [-70], None, B.KSGD_ERR_EXP_RANGE)]:
         ds = B.make_descs([d])
         if nxt is None:

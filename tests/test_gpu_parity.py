@@ -366,13 +366,15 @@ def test_step_host_matches_device_step():
     gpu.close()
 
 
-def test_tensor_with_more_than_2_31_elements_sampled():
+def test_tensor_with_more_than_2_31_elements_in_full():
     """One int8/int8 tensor of 2^31 + 12345 elements (element and byte offsets beyond 32 bits),
-    fixed exponent so that every slice can be checked on its own: slices at the start, across
-    the 2^31 and 2^32-byte marks of the gradient, and the ragged end are compared with the
-    oracle; a guard band behind each array must stay untouched."""
+    fixed exponent so that the oracle can take it slice by slice: every mantissa of theta and
+    c is compared, and the two scans and the three counters of the whole tensor must equal the
+    maximum / the sum over the oracle's slices.  A few planted gradients (NaN, both
+    infinities, values far beyond theta's range) sit on both sides of the 2^31-element and
+    2^32-byte marks; a guard band behind each array must stay untouched."""
     import torch
-    from oracle import oracle_step_tensor
+    from oracle import oracle_max_threads, oracle_step_tensor
     from paper_1810_05486_b200 import binding as B
     free, _ = torch.cuda.mem_get_info()
     if free < 20 << 30:
@@ -383,18 +385,29 @@ def test_tensor_with_more_than_2_31_elements_sampled():
     theta = torch.empty(n + guard, dtype=torch.int8, device="cuda")
     comp = torch.empty(n + guard, dtype=torch.int8, device="cuda")
     grad = torch.empty(n + guard, dtype=torch.float32, device="cuda")
-    step = 1 << 28
-    for lo in range(0, n, step):                      # inputs come from torch's generator, in pieces
-        hi = min(n, lo + step)
+    piece = 1 << 28
+    for lo in range(0, n, piece):                     # inputs come from torch's generator, in pieces
+        hi = min(n, lo + piece)
         theta[lo:hi] = torch.randint(-127, 128, (hi - lo,), generator=gen, device="cuda", dtype=torch.int8)
         comp[lo:hi] = torch.randint(-64, 65, (hi - lo,), generator=gen, device="cuda", dtype=torch.int8)
         grad[lo:hi] = torch.randn(hi - lo, generator=gen, device="cuda") * (2.0 ** -18 * 40)
+    planted = {123: float("nan"), 2 ** 30 - 1: float("inf"), 2 ** 30 + 16: -float("inf"),
+               2 ** 31 - 3: 1.0e3, 2 ** 31 + 5: float("inf"), 2 ** 31 + 8200: -2.0e-2, n - 2: float("nan"),
+               n - 9000: 7.0e-3}
+    for idx, val in planted.items():
+        grad[idx] = val
     theta[n:] = 0x5A
     comp[n:] = 0x5A
     grad[n:] = 7.0
-    windows = [(0, 70000), (2 ** 30 - 5000, 2 ** 30 + 5000), (2 ** 31 - 9000, 2 ** 31 + 9000), (n - 20000, n)]
-    before = [(theta[a:b].cpu().numpy().copy(), comp[a:b].cpu().numpy().copy(), grad[a:b].cpu().numpy().copy())
-              for a, b in windows]
+    # host copies of the inputs, taken before the step
+    t_host = np.empty(n, np.int8)
+    c_host = np.empty(n, np.int8)
+    g_host = np.empty(n, np.float32)
+    for lo in range(0, n, piece):
+        hi = min(n, lo + piece)
+        t_host[lo:hi] = theta[lo:hi].cpu().numpy()
+        c_host[lo:hi] = comp[lo:hi].cpu().numpy()
+        g_host[lo:hi] = grad[lo:hi].cpu().numpy()
     descs = B.make_descs([dict(theta=theta.data_ptr(), comp=comp.data_ptr(), numel=n, theta_bits=8,
                                comp_bits=8, exp_theta=-11)])
     nb = B.kahan_sgd_workspace_bytes(descs)
@@ -403,14 +416,55 @@ def test_tensor_with_more_than_2_31_elements_sampled():
     B.kahan_sgd_step(h, [grad.data_ptr()], [1.0])
     st = B.kahan_sgd_amax(h, 1)
     B.kahan_sgd_destroy(h)
-    worst = 0
-    for (a, b), (t0, c0, g0) in zip(windows, before):
-        res = oracle_step_tensor(t0, c0, g0, 8, 8, 0, -11, -11, 1.0)
-        assert np.array_equal(theta[a:b].cpu().numpy(), t0), (a, b)
-        assert np.array_equal(comp[a:b].cpu().numpy(), c0), (a, b)
-        worst = max(worst, res["amax_theta"])
-    assert st["amax_theta"][0] >= worst and st["exp_theta_cur"][0] == -11
+    want = dict(amax_theta=0, amax_comp=0, n_sat_theta=0, n_sat_comp=0, n_nonfinite=0)
+    threads = oracle_max_threads()
+    for lo in range(0, n, piece):
+        hi = min(n, lo + piece)
+        res = oracle_step_tensor(t_host[lo:hi], c_host[lo:hi], g_host[lo:hi], 8, 8, 0, -11, -11, 1.0, threads)
+        assert np.array_equal(theta[lo:hi].cpu().numpy(), t_host[lo:hi]), (lo, hi)
+        assert np.array_equal(comp[lo:hi].cpu().numpy(), c_host[lo:hi]), (lo, hi)
+        for key in ("amax_theta", "amax_comp"):
+            want[key] = max(want[key], res[key])
+        for key in ("n_sat_theta", "n_sat_comp", "n_nonfinite"):
+            want[key] += res[key]
+    assert want["n_nonfinite"] == 5 and want["n_sat_theta"] >= 4
+    for key, w in want.items():
+        assert st[key][0] == w, (key, st[key][0], w)
+    assert st["exp_theta_cur"][0] == -11 and st["exp_theta_next"][0] == -11
     assert bool((theta[n:] == 0x5A).all()) and bool((comp[n:] == 0x5A).all()) and bool((grad[n:] == 7.0).all())
+
+
+def test_device_error_word_reaches_the_caller():
+    """A kernel whose bounded wait runs out sets a sticky word in the workspace and
+    kahan_sgd_amax then returns KSGD_ERR_DEVICE.  No wait is made to run out here: the host
+    writes the word itself, between two healthy steps, and the read-out must report it
+    (and keep reporting it) while the statistics still come back."""
+    import torch
+    from paper_1810_05486_b200 import binding as B
+    wl = W.scaled_sweep(200_000, 5)
+    specs = specs_of(wl)
+    thetas, comps = W.initial_state(wl)
+    gpu = LibraryRun(specs, thetas, comps, EXP_AMAX)
+    lrs = [wl.lr] * len(specs)
+    try:
+        gpu.step(W.gradients(wl, 0), lrs)
+        gpu.stats()                                           # healthy: no exception
+        off = B.kahan_sgd_workspace_error_offset(gpu.descs)
+        word = gpu.workspace[off:off + 4]
+        assert bool((word == 0).all())
+        torch.cuda.synchronize()
+        word.copy_(torch.tensor([2, 0, 0, 0], dtype=torch.uint8))     # the code of a producer that gave up
+        torch.cuda.synchronize()
+        for _ in range(2):
+            with pytest.raises(B.KahanSgdError) as ei:
+                gpu.stats()
+            assert ei.value.code == B.KSGD_ERR_DEVICE
+        gpu.step(W.gradients(wl, 1), lrs)                     # the word is sticky: later steps do not clear it
+        with pytest.raises(B.KahanSgdError) as ei:
+            gpu.stats()
+        assert ei.value.code == B.KSGD_ERR_DEVICE
+    finally:
+        gpu.close()
 
 
 def test_steps_captured_in_a_cuda_graph_and_replayed():

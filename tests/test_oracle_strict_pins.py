@@ -129,6 +129,8 @@ def test_step_tensor_is_the_element_rule_with_brute_force_statistics():
     assert st == want and want["n_sat_comp"] > 0 and want["n_nonfinite"] == 2
     with pytest.raises(ValueError):
         oracle_strict_step_tensor(t2, c2, g, 8, 8, -9, -9, -46, -46, 0.5)      # e - ec = 37
+    with pytest.raises(ValueError):
+        oracle_strict_step_tensor(t2, c2, g, 8, 8, 0, 8, -20, -3, 0.5)         # c's exponent moves by 17
 
 
 def test_accumulator_exponent_policy_is_the_tight_fit_inside_the_window():

@@ -5,7 +5,9 @@ already handed to a host program's pool, a loop that cannot afford the device-wi
 synchronisation an allocation implies, a thread next to an ongoing stream capture), so they
 cannot give kahan_sgd_init the workspace it asks for.  The static entry point keeps that
 scratch inside the library.  This file checks, through the C ABI, that two such calls in a
-row give exactly the bits that the ordinary init/step/amax path gives on the same inputs.
+row give exactly the bits that the ordinary init/step/amax path gives on the same inputs,
+and that both agree with the CPU oracle (a mistake shared by the two entry points would
+otherwise pass).
 
 It is collected last on purpose: a run that stops at the first failure has then already
 run every other test.
@@ -13,7 +15,7 @@ run every other test.
 import numpy as np
 import pytest
 
-from harness import DeviceArena, LibraryRun, storage_dtype
+from harness import DeviceArena, LibraryRun, make_oracle_state, storage_dtype
 
 pytestmark = pytest.mark.gpu
 
@@ -48,8 +50,26 @@ def make_inputs(seed):
 def test_static_entry_point_matches_the_workspace_path_twice_in_a_row():
     import torch
     from paper_1810_05486_b200 import binding as B
+    from oracle import EXP_AMAX, oracle_step
     specs, thetas, comps, grads, lrs = make_inputs(2024)
     n = len(specs)
+
+    # the oracle on the same inputs
+    ost = make_oracle_state(specs, thetas, comps, EXP_AMAX)
+    oracle_states = []
+    for step in range(2):
+        before = [(t.n_sat_theta, t.n_sat_comp, t.n_nonfinite) for t in ost.tensors]
+        oracle_step(ost, grads[step], lrs)
+        oracle_states.append(dict(
+            theta=[t.theta.copy() for t in ost.tensors],
+            comp=[None if t.comp is None else t.comp.copy() for t in ost.tensors],
+            exp_theta_cur=[t.exp_theta for t in ost.tensors],
+            exp_theta_next=[t.exp_theta_next for t in ost.tensors],
+            amax_theta=[t.amax_theta for t in ost.tensors],
+            amax_comp=[t.amax_comp for t in ost.tensors],
+            n_sat_theta=[t.n_sat_theta - b[0] for t, b in zip(ost.tensors, before)],
+            n_sat_comp=[t.n_sat_comp - b[1] for t, b in zip(ost.tensors, before)],
+            n_nonfinite=[t.n_nonfinite - b[2] for t, b in zip(ost.tensors, before)]))
 
     # reference: the ordinary path with a caller-provided workspace
     ref = LibraryRun(specs, thetas, comps, B.KSGD_EXP_AMAX)
@@ -76,42 +96,82 @@ def test_static_entry_point_matches_the_workspace_path_twice_in_a_row():
             c_arena.upload(i, comps[i])
     exp_cur = [s["exp_theta"] for s in specs]
     exp_next = list(exp_cur)
-    launches0 = B.kahan_sgd_launch_count()
-    mem0 = torch.cuda.memory_allocated()
-    for step in range(2):
-        for i in range(n):
-            g_arena.upload(i, grads[step][i])
-        torch.cuda.synchronize()
-        descs = B.make_descs([
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def descs_now():
+        return B.make_descs([
             dict(theta=th_arena.ptr(i), comp=c_arena.ptr(i) if s["comp_bits"] else None,
                  numel=s["numel"], theta_bits=s["theta_bits"], comp_bits=s["comp_bits"],
                  overlap_k=s["overlap_k"], exp_theta=exp_cur[i], exp_theta_next=exp_next[i])
             for i, s in enumerate(specs)])
-        out = B.kahan_sgd_step_static(descs, B.KSGD_EXP_AMAX, [g_arena.ptr(i) for i in range(n)],
-                                      lrs, torch.cuda.current_stream().cuda_stream)
+
+    # One untimed call first, on copies that are thrown away: the first call on a device
+    # looks up the scratch array's address and sets the kernel's shared-memory attribute.
+    # After it, the free device memory the driver reports must not move: that figure sees a
+    # cudaMalloc by anybody, the library included, which torch's own counters would not.
+    warm_t = [th_arena.view(i).clone() for i in range(n)]
+    warm_c = [c_arena.view(i).clone() for i in range(n)]
+    for i in range(n):
+        g_arena.upload(i, grads[0][i])
+    torch.cuda.synchronize()
+    B.kahan_sgd_step_static(descs_now(), B.KSGD_EXP_AMAX, [g_arena.ptr(i) for i in range(n)], lrs, stream)
+    for i in range(n):
+        th_arena.view(i).copy_(warm_t[i])
+        c_arena.view(i).copy_(warm_c[i])
+    staged = [[torch.from_numpy(g).cuda() for g in gs] for gs in grads]   # no allocation inside the window
+    host_t = [torch.empty(th_arena.sizes[i], dtype=torch.uint8).pin_memory() for i in range(n)]
+    host_c = [torch.empty(c_arena.sizes[i], dtype=torch.uint8).pin_memory() for i in range(n)]
+    torch.cuda.synchronize()
+    launches0 = B.kahan_sgd_launch_count()
+    mem0 = torch.cuda.memory_allocated()
+    free0 = torch.cuda.mem_get_info()[0]
+    for step in range(2):
+        for i in range(n):
+            g_arena.view(i).copy_(staged[step][i].view(torch.uint8))
+        torch.cuda.synchronize()
+        out = B.kahan_sgd_step_static(descs_now(), B.KSGD_EXP_AMAX, [g_arena.ptr(i) for i in range(n)],
+                                      lrs, stream)
+        for i in range(n):                                     # device -> page-locked host, no allocation
+            host_t[i].copy_(th_arena.view(i))
+            host_c[i].copy_(c_arena.view(i))
+        torch.cuda.synchronize()
         want_t, want_c, want = ref_states[step]
+        orc = oracle_states[step]
         for i, s in enumerate(specs):
-            got_t = th_arena.download(i, storage_dtype(s["theta_bits"]))
+            got_t = host_t[i].numpy().view(storage_dtype(s["theta_bits"]))
             assert np.array_equal(got_t, want_t[i]), (step, i)
+            assert np.array_equal(got_t, orc["theta"][i]), (step, i, "oracle")
             if s["comp_bits"]:
-                got_c = c_arena.download(i, storage_dtype(s["comp_bits"]))
+                got_c = host_c[i].numpy().view(storage_dtype(s["comp_bits"]))
                 assert np.array_equal(got_c, want_c[i]), (step, i)
+                assert np.array_equal(got_c, orc["comp"][i]), (step, i, "oracle")
         assert out == want, step
+        for key in out:
+            assert list(out[key]) == orc[key], (step, key, "oracle")
         exp_cur, exp_next = out["exp_theta_cur"], out["exp_theta_next"]
     assert sum(ref_states[1][2]["n_nonfinite"]) == n          # the planted Inf per tensor
     assert B.kahan_sgd_launch_count() - launches0 == 2
-    assert torch.cuda.memory_allocated() == mem0               # nothing was allocated on the way
+    assert torch.cuda.memory_allocated() == mem0               # torch allocated nothing on the way ...
+    assert torch.cuda.mem_get_info()[0] >= free0               # ... and neither did anybody else
     assert th_arena.guards_intact() and c_arena.guards_intact() and g_arena.guards_intact()
 
 
 def test_static_entry_point_rejects_what_does_not_fit():
+    import torch
     from paper_1810_05486_b200 import binding as B
-    too_many = B.make_descs([dict(theta=0x10000, comp=0x20000, numel=100, theta_bits=8,
+    # real (small) device buffers behind every address, and a length derived from the
+    # array's size, so that neither case could ever reach a launch on a wild pointer
+    buf = torch.zeros(3 * 4096, dtype=torch.uint8, device="cuda")
+    th, c, g = buf.data_ptr(), buf.data_ptr() + 4096, buf.data_ptr() + 8192
+    too_many = B.make_descs([dict(theta=th, comp=c, numel=100, theta_bits=8,
                                   comp_bits=8, exp_theta=-11)] * (B.KSGD_STATIC_MAX_TENSORS + 1))
-    too_big = B.make_descs([dict(theta=0x10000, comp=0x20000, numel=400_000_000, theta_bits=8,
+    # 8 bytes of tile table per 8192 elements: four times what the whole array could describe
+    numel = 4 * (B.KSGD_STATIC_SCRATCH_BYTES // 8) * 8192
+    too_big = B.make_descs([dict(theta=th, comp=c, numel=numel, theta_bits=8,
                                  comp_bits=8, exp_theta=-11)])
     for descs in (too_many, too_big):
         with pytest.raises(B.KahanSgdError) as ei:
-            B.kahan_sgd_step_static(descs, B.KSGD_EXP_AMAX, [0x30000] * len(descs),
+            B.kahan_sgd_step_static(descs, B.KSGD_EXP_AMAX, [g] * len(descs),
                                     [0.1] * len(descs))
         assert ei.value.code == B.KSGD_ERR_WORKSPACE
+    assert bool((buf == 0).all())

@@ -156,6 +156,7 @@ struct __align__(16) TileDesc {
 };
 constexpr int kFlagFormatMask = 7;   // 0..5 = (8,0) (8,8) (8,16) (16,0) (16,8) (16,16)
 constexpr int kFlagSteady = 8;       // no exponent change: the exact-fp32 path applies
+constexpr int kFlagRegrid = 16;      // theta's exponent changes: the exact-fp32 re-gridding path applies
 constexpr int kFlagThetaPageShift = 8;   // 5 bits each: first ring page of theta, c, g
 constexpr int kFlagCompPageShift = 13;
 constexpr int kFlagGradPageShift = 18;
@@ -596,6 +597,109 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
   return true;
 }
 
+// The step in which theta's exponent changes by delta = e_out - e_in (ordinary mode: c's grid
+// moves with theta's), again on the FP32 pipe with every intermediate an exact integer below
+// 2^24.  k.pow2dc = 2^-delta.  d = rne(g*scale) is on the output compensation grid as always.
+//
+// Finer grid (delta < 0, a = -delta): the stored mantissas scale up exactly,
+//   base = M + qt*2^a (both even, so exact even beyond 2^24),  u = qc*2^a - d,
+//   Pb = fma(u, 2^-s, base) = M + P,  w = Pb - base,  r0 = fma(w, -2^s, u) = Rq  (no second rounding).
+// Coarser grid (delta > 0, a = delta, s' = s + a): theta's mantissa is split with two integer
+// operations per packed word, qt = A*2^a + B with 0 <= B < 2^a (on the sign-flipped lanes the
+// split is a logical shift and a mask), so that
+//   T = A*2^s' + v,  v = B*2^s + qc - d*2^a   (exact: |d|*2^a <= 4e6 is checked)
+//   Pb = fma(v, 2^-s', M + A) = M + P,  w = Pb - (M + A),  R = fma(w, -2^s', v),
+//   Rm = fma(R, 2^-a, M) = M + Rq   (the second rounding of the coarser grid, ties on Rq's parity).
+// In both cases |Rq| <= 2^(s-1) whenever P needs no clamp, so c never clamps on this path.
+// Returns false (nothing stored: the vector goes to update_general) when some product is too
+// large, Inf or NaN, or some |P| exceeds QMAX.  A coarser change needs a <= TB - 1 (the
+// producer checks).
+template <int TB, int CB, int V, int GB>
+__device__ __forceinline__ bool update_vector_regrid(Pack<V * TB / 8> pt, Pack<(CB ? V * CB / 8 : 8)> pc,
+                                                     Pack<V * GB / 8> pg, const SteadyCoef& k,
+                                                     Pack<V * TB / 8>& ot, Pack<(CB ? V * CB / 8 : 8)>& oc,
+                                                     float& amax_t, float& amax_c) {
+  constexpr bool HAS_COMP = CB != 0;
+  constexpr int CBS = CB ? CB : 8;
+  constexpr int GBS = GB == 32 ? 8 : GB;
+  constexpr float bias_t = (float)(1 << (TB - 1));
+  constexpr float bias_c = (float)(1 << (CBS - 1));
+  flip_signs<TB>(pt);
+  if constexpr (HAS_COMP) flip_signs<CBS>(pc);
+  if constexpr (GB != 32) flip_signs<GBS>(pg);
+  const bool finer = k.pow2dc > 1.0f;
+  // 2^a and 2^-a
+  const float up = finer ? k.pow2dc : __int_as_float(0x7f000000 - __float_as_int(k.pow2dc));
+  const float down = finer ? __int_as_float(0x7f000000 - __float_as_int(k.pow2dc)) : k.pow2dc;
+  Pack<V * TB / 8> pB = pt;
+  float inv2sp = k.inv2s, pow2sp_neg = k.pow2s_neg, biasA = bias_t, pow2s = -k.pow2s_neg;
+  if (!finer) {
+    const int a = 127 - (int)(__float_as_uint(k.pow2dc) >> 23);
+    constexpr unsigned int lanes = TB == 8 ? 0x01010101u : 0x00010001u;
+    constexpr unsigned int full = TB == 8 ? 0xffu : 0xffffu;
+    const unsigned int maskA = (full >> a) * lanes, maskB = ((1u << a) - 1u) * lanes;
+#pragma unroll
+    for (int w = 0; w < V * TB / 32; ++w) {
+      const unsigned int x = pack_word(pt, w);
+      set_pack_word(pt, w, (x >> a) & maskA);
+      set_pack_word(pB, w, x & maskB);
+    }
+    inv2sp = __fmul_rn(k.inv2s, down);          // 2^-s'
+    pow2sp_neg = __fmul_rn(k.pow2s_neg, up);    // -2^s'
+    biasA = __fmul_rn(bias_t, down);            // what the shifted lanes still carry of the sign flip
+  }
+  float Pm[V], rm[V], xa[2], ra[2];
+  float aX = 0.0f, hiP = kMagic, loP = kMagic, aR = 0.0f;
+#pragma unroll
+  for (int i = 0; i < V; ++i) {
+    float g;
+    if constexpr (GB == 32) g = __uint_as_float(pack_word(pg, i));
+    else g = __fadd_rn(magic_elem<GBS>(pg, i), -(kMagic + (float)(1 << (GBS - 1))));
+    const float x = __fmul_rn(g, k.scale);              // the one binary32 multiply
+    const float y = __fadd_rn(x, kMagic);               // M + d
+    float qc = 0.0f;
+    if constexpr (HAS_COMP) qc = __fadd_rn(magic_elem<CBS>(pc, i), -(kMagic + bias_c));
+    float P, r;
+    if (finer) {
+      const float qt = __fadd_rn(magic_elem<TB>(pt, i), -(kMagic + bias_t));
+      const float base = __fmaf_rn(qt, up, kMagic);
+      const float u = __fmaf_rn(qc, up, __fadd_rn(kMagic, -y));
+      P = __fmaf_rn(u, inv2sp, base);
+      const float w = __fadd_rn(P, -base);
+      r = __fmaf_rn(w, pow2sp_neg, u);
+      rm[i] = __fadd_rn(r, kMagic);
+    } else {
+      const float base = __fadd_rn(magic_elem<TB>(pt, i), -biasA);       // M + A
+      const float B = __fadd_rn(magic_elem<TB>(pB, i), -kMagic);
+      const float d = __fadd_rn(y, -kMagic);
+      const float v = __fmaf_rn(d, -up, __fmaf_rn(B, pow2s, qc));
+      P = __fmaf_rn(v, inv2sp, base);
+      const float w = __fadd_rn(P, -base);
+      const float R = __fmaf_rn(w, pow2sp_neg, v);
+      rm[i] = __fmaf_rn(R, down, kMagic);
+      r = __fadd_rn(rm[i], -kMagic);
+    }
+    Pm[i] = P;
+    xa[i & 1] = fabsf(x);
+    ra[i & 1] = fabsf(r);
+    if (i & 1) {
+      aX = max3_nan(aX, xa[0], xa[1]);                  // NaN if any product is
+      hiP = max3(hiP, Pm[i - 1], P);
+      loP = min3(loP, Pm[i - 1], P);
+      if constexpr (HAS_COMP) aR = max3(aR, ra[0], ra[1]);
+    }
+  }
+  const float aP = fmaxf(__fadd_rn(hiP, -kMagic), __fadd_rn(kMagic, -loP));
+  constexpr float qmax_t = (float)((1 << (TB - 1)) - 1);
+  const float x_limit = finer ? 4000000.0f : __fmul_rn(4000000.0f, down);   // |d| * 2^a stays exact
+  if (!(aX <= x_limit) | (aP > qmax_t)) return false;   // also Inf and NaN products
+  amax_t = fmaxf(amax_t, aP);
+  if constexpr (HAS_COMP) amax_c = fmaxf(amax_c, aR);
+  ot = pack_magic<TB, V>(Pm);
+  if constexpr (HAS_COMP) oc = pack_magic<CB, V>(rm);
+  return true;
+}
+
 // All vectors of one tile that belong to this consumer thread (V consecutive elements,
 // 16 bytes of theta, per vector).  Returns true if the general path wrote into the stage.
 template <int TB, int CB, int GB, bool STRICT>
@@ -640,6 +744,97 @@ __device__ __forceinline__ bool consume_tile(const TileHot& h, const TileDesc* t
   return wrote_stage;
 }
 
+// Add a consumer warp's steady-path scans of the tile it just finished to the tile's slot.
+__device__ __forceinline__ void add_warp_scans(TileScan* scan, int lane, float& amax_t, float& amax_c) {
+  const unsigned int full = 0xffffffffu;
+  // the steady path's scans are exact integers below 2^23 held in floats
+  const unsigned int at = __reduce_max_sync(full, (unsigned int)amax_t);
+  const unsigned int ac = __reduce_max_sync(full, (unsigned int)amax_c);
+  amax_t = 0.0f;
+  amax_c = 0.0f;
+  if (lane == 0) {
+    if (at) atomicMax(&scan->amax_t, at);
+    if (ac) atomicMax(&scan->amax_c, ac);
+  }
+}
+
+// A whole tile of a tensor whose exponent changes in this step, for one consumer thread:
+// update_vector_regrid per vector (update_general for the vectors it declines), stores, the
+// ragged tail, and the warp's scans added to the tile's slot.  Kept out of line, like update_general: it is called once per
+// tile with next to nothing live around the call, and the registers its arithmetic needs
+// then cost the tiles whose exponent does not change (the common case, inline in the
+// kernel) nothing.
+template <int TB, int CB, int GB>
+__device__ __forceinline__ bool regrid_tile_format(const TileHot& h, const TileDesc* td, unsigned char* ring,
+                                                   int ctid, TileScan* slots, float& amax_t, float& amax_c) {
+  constexpr bool HAS_COMP = CB != 0;
+  constexpr int V = (TB == 8) ? 16 : 8;
+  constexpr int TBYTES = V * TB / 8;
+  constexpr int CBYTES = HAS_COMP ? V * CB / 8 : 8;
+  constexpr int GBYTES = V * GB / 8;
+  unsigned char* theta_s = ring + ((h.flags >> kFlagThetaPageShift) & 31) * kPageBytes;
+  unsigned char* comp_s = ring + ((h.flags >> kFlagCompPageShift) & 31) * kPageBytes;
+  const unsigned char* grad_s = ring + ((h.flags >> kFlagGradPageShift) & 31) * kPageBytes;
+  bool wrote_stage = false;
+  const int n_vec = h.n_bulk / V;
+  for (int v = ctid; v < n_vec; v += kConsumers) {
+    Pack<TBYTES> ot;
+    Pack<CBYTES> oc;
+    const Pack<TBYTES> pt = load_pack<TBYTES>(theta_s + v * TBYTES);
+    Pack<CBYTES> pc{};
+    if constexpr (HAS_COMP) pc = load_pack<CBYTES>(comp_s + v * CBYTES);
+    const Pack<GBYTES> pg = load_pack<GBYTES>(grad_s + v * GBYTES);
+    if (!update_vector_regrid<TB, CB, V, GB>(pt, pc, pg, h.k, ot, oc, amax_t, amax_c)) {
+      update_general(&td->coef, TB, CB, theta_s, comp_s, grad_s, v * V, V, slots);
+      ot = load_pack<TBYTES>(theta_s + v * TBYTES);
+      if constexpr (HAS_COMP) oc = load_pack<CBYTES>(comp_s + v * CBYTES);
+      wrote_stage = true;
+    }
+    store_pack<TBYTES>(h.theta + (size_t)v * TBYTES, ot);
+    if constexpr (HAS_COMP) store_pack<CBYTES>(h.comp + (size_t)v * CBYTES, oc);
+  }
+  const int e = h.n_bulk + ctid;
+  if (e < h.count) update_general(&td->coef, TB, CB, h.theta, h.comp, td->grad, e, 1, slots);
+  return wrote_stage;
+}
+
+__device__ __forceinline__ TileHot load_tile_hot(const TileDesc* td) {
+  TileHot h;
+  const uint4* q = reinterpret_cast<const uint4*>(td);
+  const uint4 q0 = q[0], q1 = q[1], q2 = q[2];
+  h.k.scale = __uint_as_float(q0.x);
+  h.k.pow2s_neg = __uint_as_float(q0.y);
+  h.k.inv2s = __uint_as_float(q0.z);
+  h.k.pow2dc = __uint_as_float(q0.w);
+  h.theta = reinterpret_cast<unsigned char*>(((unsigned long long)q1.y << 32) | q1.x);
+  h.comp = reinterpret_cast<unsigned char*>(((unsigned long long)q1.w << 32) | q1.z);
+  h.tensor = (int)q2.x;
+  h.n_bulk = (int)q2.y;
+  h.count = (int)q2.z;
+  h.flags = (int)q2.w;
+  return h;
+}
+
+template <int GB>
+__device__ __noinline__ void regrid_tile(const TileDesc* td, TileScan* slots, unsigned char* ring) {
+  const TileHot h = load_tile_hot(td);
+  const int ctid = threadIdx.x;
+  float amax_t = 0.0f, amax_c = 0.0f;
+  bool wrote_stage;
+  switch (h.flags & kFlagFormatMask) {
+    case 0: wrote_stage = regrid_tile_format<8, 0, GB>(h, td, ring, ctid, slots, amax_t, amax_c); break;
+    case 1: wrote_stage = regrid_tile_format<8, 8, GB>(h, td, ring, ctid, slots, amax_t, amax_c); break;
+    case 2: wrote_stage = regrid_tile_format<8, 16, GB>(h, td, ring, ctid, slots, amax_t, amax_c); break;
+    case 3: wrote_stage = regrid_tile_format<16, 0, GB>(h, td, ring, ctid, slots, amax_t, amax_c); break;
+    case 4: wrote_stage = regrid_tile_format<16, 8, GB>(h, td, ring, ctid, slots, amax_t, amax_c); break;
+    default: wrote_stage = regrid_tile_format<16, 16, GB>(h, td, ring, ctid, slots, amax_t, amax_c); break;
+  }
+  add_warp_scans(slots, threadIdx.x & 31, amax_t, amax_c);
+  // if the general path wrote into the stage, order those writes before the bulk copy that
+  // refills it
+  if (wrote_stage) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
 // Next exponent from the max scan: the tight fit puts the largest mantissa in
 // (QMAX/2, QMAX].  With L = bit length of amax and QMAX = 2^(b-1)-1, the change is
 // L-(b-1), plus one more when amax still exceeds QMAX*2^change.
@@ -680,20 +875,6 @@ struct __align__(128) BlockShared {
 };
 
 constexpr size_t kSharedBytes = (size_t)kPages * kPageBytes + sizeof(BlockShared);
-
-// Add a consumer warp's steady-path scans of the tile it just finished to the tile's slot.
-__device__ __forceinline__ void add_warp_scans(TileScan* scan, int lane, float& amax_t, float& amax_c) {
-  const unsigned int full = 0xffffffffu;
-  // the steady path's scans are exact integers below 2^23 held in floats
-  const unsigned int at = __reduce_max_sync(full, (unsigned int)amax_t);
-  const unsigned int ac = __reduce_max_sync(full, (unsigned int)amax_c);
-  amax_t = 0.0f;
-  amax_c = 0.0f;
-  if (lane == 0) {
-    if (at) atomicMax(&scan->amax_t, at);
-    if (ac) atomicMax(&scan->amax_c, ac);
-  }
-}
 
 // Producer side: scans of finished tiles are merged per tensor in registers and go to
 // global memory when the tensor changes (one set of atomics per block and tensor run).
@@ -895,6 +1076,8 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
         td.count = count;
         td.flags = ((ti.theta_bits == 16 ? 3 : 0) + (ti.comp_bits >> 3)) |
                    ((coef.delta == 0 && scale_ok && (!STRICT || coef.s >= 0)) ? kFlagSteady : 0) |
+                   // a coarser grid splits theta's mantissa at bit delta: that needs delta <= theta_bits - 1
+                   ((!STRICT && coef.delta != 0 && scale_ok && coef.delta <= ti.theta_bits - 1) ? kFlagRegrid : 0) |
                    (page[1] << kFlagThetaPageShift) |
                    (page[2] << kFlagCompPageShift) | (page[0] << kFlagGradPageShift);
         td.coef = coef;
@@ -938,7 +1121,6 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
     const int ctid = threadIdx.x;
     const int stride = (int)gridDim.x;
     const int n_my = (p.tile_count - (int)blockIdx.x + stride - 1) / stride;
-    float amax_t = 0.0f, amax_c = 0.0f;
     for (int i = 0; i < n_my; ++i) {
       const int stage = i % kSlots, use = i / kSlots;
       if (!mbar_wait(&sh->full[stage], (unsigned)use & 1u, &sh->abort_flag)) {
@@ -950,35 +1132,26 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
       }
       const TileDesc* td = &sh->desc[stage];
       TileScan* scan = &sh->scan[stage];
-      TileHot h;
-      {
-        const uint4* q = reinterpret_cast<const uint4*>(td);
-        const uint4 q0 = q[0], q1 = q[1], q2 = q[2];
-        h.k.scale = __uint_as_float(q0.x);
-        h.k.pow2s_neg = __uint_as_float(q0.y);
-        h.k.inv2s = __uint_as_float(q0.z);
-        h.k.pow2dc = __uint_as_float(q0.w);
-        h.theta = reinterpret_cast<unsigned char*>(((unsigned long long)q1.y << 32) | q1.x);
-        h.comp = reinterpret_cast<unsigned char*>(((unsigned long long)q1.w << 32) | q1.z);
-        h.tensor = (int)q2.x;
-        h.n_bulk = (int)q2.y;
-        h.count = (int)q2.z;
-        h.flags = (int)q2.w;
-      }
       unsigned char* st = smem;
-      bool wrote_stage;
-      switch (h.flags & kFlagFormatMask) {
-        case 0: wrote_stage = consume_tile<8, 0, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        case 1: wrote_stage = consume_tile<8, 8, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        case 2: wrote_stage = consume_tile<8, 16, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        case 3: wrote_stage = consume_tile<16, 0, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        case 4: wrote_stage = consume_tile<16, 8, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        default: wrote_stage = consume_tile<16, 16, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+      if (!STRICT && (td->flags & kFlagRegrid)) {
+        regrid_tile<GB>(td, scan, st);
+      } else {
+        const TileHot h = load_tile_hot(td);
+        float amax_t = 0.0f, amax_c = 0.0f;
+        bool wrote_stage;
+        switch (h.flags & kFlagFormatMask) {
+          case 0: wrote_stage = consume_tile<8, 0, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+          case 1: wrote_stage = consume_tile<8, 8, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+          case 2: wrote_stage = consume_tile<8, 16, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+          case 3: wrote_stage = consume_tile<16, 0, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+          case 4: wrote_stage = consume_tile<16, 8, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+          default: wrote_stage = consume_tile<16, 16, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        }
+        add_warp_scans(scan, lane, amax_t, amax_c);
+        // if the general path wrote into the stage, order those writes before the bulk copy
+        // that refills it
+        if (wrote_stage) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       }
-      add_warp_scans(scan, lane, amax_t, amax_c);
-      // if the general path wrote into the stage, order those writes before the bulk copy
-      // that refills it
-      if (wrote_stage) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->empty[stage]);
     }

@@ -42,13 +42,20 @@ GRAD_SETS = {"c5_sweep": 2, "c1_single": 100, "c2_resnet20": 200, "c3_resnet50":
 
 # DRAM traffic of ksgd_step_kernel from ncu captures (dram__bytes_read.sum +
 # dram__bytes_write.sum per launch, divided by the parameters of the captured launch; see
-# profiles/).  c5_sweep was captured at 2e8 parameters; traffic is proportional to the
-# parameter count, so a full launch is this figure times its parameters.  The record only
-# counts while the kernel source (kahan_sgd_kernels.cuh) still hashes to the value below.
+# profiles/).  "cold": caches flushed before the launch (ncu's default), which is what a
+# list far larger than L2 sees at every step; c5_sweep was captured at 2e8 parameters and
+# its traffic is proportional to the parameter count, so a full launch is this figure times
+# its parameters.  "warm": the launch as it runs in the benchmark's loop, caches left as the
+# preceding steps left them (--cache-control none), which is what counts for a list whose
+# theta and c stay in L2 from step to step.  The record only counts while the kernel source
+# (kahan_sgd_kernels.cuh) still hashes to the value below.
 TRAFFIC_RECORD = {
     "sources_sha256": "2116fc351fe2f07e2b18bc9dcf183f78c3cd847a1bfd0bdc0e303bd140896441",
-    "dram_bytes_per_parameter": {"c5_sweep": 2355.328e6 / 2e8, "c4_alexnet": 469.794e6 / 61100840,
-                                 "c3_resnet50": 200.325e6 / 25557032},
+    "dram_bytes_per_parameter": {
+        "c5_sweep": {"cold": 2355.328e6 / 2e8, "warm": None},
+        "c4_alexnet": {"cold": 469.794e6 / 61100840, "warm": None},
+        "c3_resnet50": {"cold": 200.325e6 / 25557032, "warm": None},
+    },
 }
 
 
@@ -61,29 +68,40 @@ def kernel_sources_sha256():
     return h.hexdigest()
 
 
-def recorded_traffic(wl):
+def recorded_traffic(wl, kind="cold"):
     """DRAM bytes of one launch from the ncu record, or None once the kernel has changed."""
     try:
         if kernel_sources_sha256() != TRAFFIC_RECORD["sources_sha256"]:
             return None
-        per = TRAFFIC_RECORD["dram_bytes_per_parameter"].get(wl.name)
+        per = TRAFFIC_RECORD["dram_bytes_per_parameter"].get(wl.name, {}).get(kind)
         return None if per is None else per * wl.numel
     except Exception:
         return None
 
 
+def state_bytes_of(wl):
+    return sum(t.numel * (t.theta_bits + t.comp_bits) // 8 for t in wl.tensors)
+
+
+def l2_resident_state(wl):
+    """True if theta and c of the whole list stay in L2 from step to step (the library marks
+    the gradient loads evict-first under the same condition)."""
+    return state_bytes_of(wl) <= 0.8 * L2_BYTES
+
+
 def l2_note(wl, n_sets):
-    """How the timed steps relate to the 126 MB L2: what one step touches, and what the steps
-    of the timed region touch between two uses of the same gradient set."""
-    state = sum(t.numel * (t.theta_bits + t.comp_bits) // 8 for t in wl.tensors)
+    """How the timed steps relate to the 126 MB L2.  What decides is the state (theta and c)
+    plus ONE gradient set, not the bytes a step touches: a state that fits stays resident
+    while the gradients stream through."""
+    state = state_bytes_of(wl)
     grads = wl.bytes_per_step - 2 * state
-    if wl.bytes_per_step > L2_BYTES:
-        return "inputs larger than L2 (%.0f MB touched per step)" % (wl.bytes_per_step / 1e6)
-    cycle = state + n_sets * grads
-    if cycle > L2_BYTES:
-        return ("a fresh gradient set every step (%d sets, %.0f MB in all, larger than L2); theta and c "
-                "(%.1f MB) stay resident in L2 from step to step" % (n_sets, n_sets * grads / 1e6, state / 1e6))
-    return "working set %.1f MB fits L2: a launch-latency figure, not a DRAM one" % (cycle / 1e6)
+    if state + n_sets * grads <= L2_BYTES:
+        return "working set %.1f MB fits L2: a launch-latency figure, not a DRAM one" % ((state + n_sets * grads) / 1e6)
+    if l2_resident_state(wl):
+        return ("L2-assisted: theta and c (%.1f MB) stay resident in L2 from step to step; a fresh gradient "
+                "set every step (%d sets, %.0f MB each) streams from DRAM, so a step moves fewer DRAM bytes "
+                "than its %.0f MB of algorithmic bytes" % (state / 1e6, n_sets, grads / 1e6, wl.bytes_per_step / 1e6))
+    return "inputs larger than L2 (state %.0f MB + %.0f MB of gradients per step)" % (state / 1e6, grads / 1e6)
 
 
 def parse_args():
@@ -114,6 +132,11 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-buckets", action="store_true",
                     help="skip the per-size-bucket timing of c5_sweep")
+    ap.add_argument("--no-extra-workloads", action="store_true",
+                    help="skip the c3_resnet50 / c4_alexnet legs that the default run adds to its line")
+    ap.add_argument("--sustained-s", type=float, default=0.35,
+                    help="length of the sustained leg (the same steps repeated for about this long, with the "
+                         "clocks sampled inside it); 0 skips it")
     return ap.parse_args()
 
 
@@ -194,6 +217,111 @@ def pick_workload(W, args):
     return W.workload(args.workload)
 
 
+def timed_region(torch, B, run, n_sets, steps, first_set, barrier, sampler=None):
+    """`steps` back-to-back steps on the handle's stream between two CUDA events (recorded on
+    that stream), a barrier and a device synchronisation on both sides.  Returns total ms,
+    the per-step ms of each quarter of the region, launches of the library's kernels, and
+    the clock record if a sampler was given."""
+    stream = run.stream
+    if sampler is not None:
+        sampler.start()
+        time.sleep(0.2)
+    launches0 = B.kahan_sgd_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    wall0 = time.time()
+    ev0.record(stream)
+    marks = []          # events at the quarters of the timed region (clock-regime record)
+    for i in range(steps):
+        run.step((first_set + i) % n_sets)
+        if steps >= 40 and (i + 1) % (steps // 4) == 0 and len(marks) < 3:
+            marks.append(torch.cuda.Event(enable_timing=True))
+            marks[-1].record(stream)
+    ev1.record(stream)
+    barrier()
+    wall1 = time.time()
+    launches = B.kahan_sgd_launch_count() - launches0
+    ms_total = ev0.elapsed_time(ev1)
+    quarters = None
+    if len(marks) == 3:
+        pts = [ev0] + marks + [ev1]
+        q = steps // 4
+        counts = [q, q, q, steps - 3 * q]
+        quarters = [round(pts[j].elapsed_time(pts[j + 1]) / counts[j], 6) for j in range(4)]
+    clocks = sampler.stop(wall0, wall1) if sampler is not None else None
+    return ms_total, quarters, int(launches), clocks
+
+
+def sustained_leg(torch, B, run, n_sets, ms_step, seconds, first_set, barrier, gpu_index, bytes_per_step, peak):
+    """The same steps repeated for about `seconds` (gradient sets reused in turn), with the
+    clocks sampled inside the region: the figure a long training run sees, and the one a
+    timed region of a few milliseconds cannot carry a clock record for."""
+    steps = max(40, int(seconds / max(ms_step * 1e-3, 1e-6)))
+    steps = min(steps, 200000)
+    ms_total, quarters, _, clocks = timed_region(torch, B, run, n_sets, steps, first_set, barrier,
+                                                 ClockSampler(gpu_index))
+    ms = ms_total / steps
+    gbs = bytes_per_step / (ms * 1e-3) / 1e9
+    out = {"steps": steps, "ms_per_step": ms, "ms_per_step_quarters": quarters, "algorithmic_gbs": gbs,
+           "frac": gbs / peak, "clocks": clocks}
+    if clocks and clocks.get("sm_mhz"):
+        # time x clock: how the step depends on the SM clock the box happened to run at
+        out["us_x_ghz"] = round(ms * 1e3 * clocks["sm_mhz"] / 1e3, 2)
+    return out
+
+
+def roofline_of(wl, bytes_per_step, ms_step, peak, peak_src, kernel, plain):
+    """The roofline object of one workload.  `achieved` counts the ALGORITHMIC bytes of a
+    step (2m/8 + 2n/8 + 4 per parameter); `traffic` is what DRAM really moved per launch
+    (ncu), `dram_gbs` that traffic over the same time.  For a list whose state stays in L2
+    the two differ, and `dram_gbs` is the DRAM-side figure."""
+    achieved = bytes_per_step / (ms_step * 1e-3) / 1e9
+    r = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+         "traffic": None, "peak_source": peak_src, "frac_of_nominal_8000": achieved / 8000.0,
+         "kernel": kernel, "launch_ms": ms_step, "l2_assisted": l2_resident_state(wl)}
+    if plain:
+        kind = "warm" if r["l2_assisted"] else "cold"
+        traffic = recorded_traffic(wl, kind)
+        r["traffic"] = traffic
+        r["traffic_capture"] = ("ncu --cache-control none (caches as the preceding steps left them)"
+                                if kind == "warm" else "ncu default (caches flushed before the launch)")
+        if traffic is not None:
+            r["dram_gbs"] = traffic / (ms_step * 1e-3) / 1e9
+            r["frac_dram"] = r["dram_gbs"] / peak
+    return r
+
+
+def extra_workload(torch, B, W, name, args, peak, peak_src, barrier, gpu_index):
+    """One of the other workloads of at least 25 M parameters, timed like the headline: the
+    recipe's own number of steps (a fresh gradient set each), then the sustained leg."""
+    from paper_1810_05486_b200.runner import DeviceRun, HostInputs
+    wl = W.workload(name)
+    n_sets = GRAD_SETS[name]
+    host = HostInputs(wl, args.seed, n_sets, pinned=False)
+    run = DeviceRun(host, B.KSGD_EXP_AMAX)
+    with torch.cuda.stream(run.stream):
+        for i in range(args.warmup):
+            run.step(i % n_sets)
+        barrier()
+        ms_total, quarters, launches, _ = timed_region(torch, B, run, n_sets, wl.steps, args.warmup, barrier)
+        ms_step = ms_total / wl.steps
+        out = {"workload": name, "tensors": len(wl.tensors), "parameters": wl.numel,
+               "bytes_per_step": run.bytes_per_step, "steps": wl.steps, "warmup": args.warmup,
+               "ms_per_step": ms_step, "value": wl.numel / (ms_step * 1e-3), "unit": UNIT,
+               "gpu_launches": launches, "l2": l2_note(wl, n_sets),
+               "roofline": roofline_of(wl, run.bytes_per_step, ms_step, peak, peak_src, "ksgd_step_kernel", True)}
+        if args.sustained_s > 0:
+            out["sustained"] = sustained_leg(torch, B, run, n_sets, ms_step, args.sustained_s,
+                                             args.warmup + wl.steps, barrier, gpu_index, run.bytes_per_step, peak)
+    st = run.stats()
+    out["counters"] = {"n_sat_theta": int(sum(st["n_sat_theta"])), "n_sat_comp": int(sum(st["n_sat_comp"])),
+                       "n_nonfinite": int(sum(st["n_nonfinite"]))}
+    run.close()
+    del run, host
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     import __graft_entry__ as entry
@@ -241,38 +369,21 @@ def run_ours(args, rank, world, local_rank):
         for i in range(args.warmup):
             run.step(i % n_sets)
         barrier()
-        sampler = ClockSampler(local_rank)
-        if rank == 0:
-            sampler.start()
-            time.sleep(0.2)
-        launches0 = B.kahan_sgd_launch_count()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        wall0 = time.time()
-        ev0.record(stream)
-        marks = []          # events at the quarters of the timed region (clock-regime record)
-        for i in range(args.steps):
-            run.step((args.warmup + i) % n_sets)
-            if args.steps >= 40 and (i + 1) % (args.steps // 4) == 0 and len(marks) < 3:
-                marks.append(torch.cuda.Event(enable_timing=True))
-                marks[-1].record(stream)
-        ev1.record(stream)
-        barrier()
-        wall1 = time.time()
-        launches = B.kahan_sgd_launch_count() - launches0
-        ms_total = ev0.elapsed_time(ev1)
-        quarters = None
-        if len(marks) == 3:
-            pts = [ev0] + marks + [ev1]
-            q = args.steps // 4
-            counts = [q, q, q, args.steps - 3 * q]
-            quarters = [round(pts[j].elapsed_time(pts[j + 1]) / counts[j], 6) for j in range(4)]
-        clocks = sampler.stop(wall0, wall1) if rank == 0 else None
+        ms_total, quarters, launches, clocks = timed_region(
+            torch, B, run, n_sets, args.steps, args.warmup, barrier,
+            ClockSampler(local_rank) if rank == 0 else None)
     stats = run.stats()
 
     ms_total = multi.max_over_ranks(ms_total, dist, "cuda")
     ms_step = ms_total / args.steps
     value = multi.whole_job_throughput(wl.numel, world, ms_step * 1e-3)
+
+    peak, peak_src = hbm_peak()
+    sustained = None
+    if args.sustained_s > 0 and world == 1:
+        with torch.cuda.stream(stream):
+            sustained = sustained_leg(torch, B, run, n_sets, ms_step, args.sustained_s, args.warmup + args.steps,
+                                      barrier, local_rank, run.bytes_per_step, peak)
 
     # ---- end to end through host buffers ------------------------------------------------
     e2e = None
@@ -313,6 +424,8 @@ def run_ours(args, rank, world, local_rank):
     if wl.name == "c5_sweep" and rank == 0 and not other and not args.no_buckets:
         buckets = time_size_buckets(torch, B, run, wl)
     run.close()
+    bytes_per_step = run.bytes_per_step
+    run.dev_th = run.dev_c = run.dev_g = run.workspace = None      # give the device memory back
 
     if rank != 0:
         if dist is not None:
@@ -320,33 +433,30 @@ def run_ours(args, rank, world, local_rank):
             dist.destroy_process_group()
         return
 
-    peak, peak_src = hbm_peak()
-    achieved = run.bytes_per_step / (ms_step * 1e-3) / 1e9
-    traffic = None if other else recorded_traffic(wl)
+    kernel = ("ksgd_momentum_step_kernel" if args.momentum_bits
+              else ("ksgd_adam_step_kernel" if args.adam else
+                    (("ksgd_strict_step" if args.strict else "ksgd_step") +
+                     ("_kernel" if args.grad_bits == 32 else "_qgrad_kernel"))))
+    roofline = roofline_of(wl, bytes_per_step, ms_step, peak, peak_src, kernel, not other)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": wl.name, "tensors": n, "parameters": wl.numel,
-                   "bytes_per_step": run.bytes_per_step, "grad_sets": n_sets,
+                   "bytes_per_step": bytes_per_step, "grad_sets": n_sets,
                    "optimizer": "momentum 0.9, int%d velocity" % args.momentum_bits if args.momentum_bits
                    else ("adam 0.9/0.999/1e-8, int16 moments" if args.adam else
                          (("sgd" if args.grad_bits == 32 else "sgd, int%d gradients" % args.grad_bits) +
                           (", strict Algorithm 1" if args.strict else ""))),
                    "l2": l2_note(wl, n_sets),
                    "exponent_mode": "amax", "input_generation_s": round(gen_s, 1)},
-        "achieved_hbm_gbs": achieved,
+        # algorithmic bytes per second (not DRAM bytes: see roofline.dram_gbs / roofline.l2_assisted)
+        "achieved_hbm_gbs": roofline["achieved"],
         # ms per step in each quarter of the timed region: under sustained load the power cap
         # lowers the SM clock within a few tenths of a second, and the step gets faster with it
         "ms_per_step_quarters": quarters,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
-                     "frac_of_nominal_8000": achieved / 8000.0,
-                     "kernel": "ksgd_momentum_step_kernel" if args.momentum_bits
-                     else ("ksgd_adam_step_kernel" if args.adam else
-                           (("ksgd_strict_step" if args.strict else "ksgd_step") +
-                            ("_kernel" if args.grad_bits == 32 else "_qgrad_kernel"))),
-                     "launch_ms": ms_step},
+        "roofline": roofline,
+        "sustained": sustained,
         "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
         "counters": {"n_sat_theta": int(sum(stats["n_sat_theta"])),
                      "n_sat_comp": int(sum(stats["n_sat_comp"])),
@@ -359,6 +469,14 @@ def run_ours(args, rank, world, local_rank):
                               "note": "the same %d steps recorded once into a CUDA graph and replayed" % args.steps}
     if not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, host, budget_core_s=20.0)
+    if (wl.name == "c5_sweep" and not args.sweep_total and not other and world == 1
+            and not args.no_extra_workloads):
+        # the other two workloads of at least 25 M parameters, on the same line
+        run.host = None
+        del host        # page-locked host copies of the sweep (12 GB) go before the next workloads come
+        torch.cuda.empty_cache()
+        line["workloads"] = [extra_workload(torch, B, W, name, args, peak, peak_src, barrier, local_rank)
+                             for name in ("c3_resnet50", "c4_alexnet")]
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.barrier()
@@ -498,9 +616,29 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started without a launcher: start one rank per GPU ourselves (whole-list replicas,
+        # one process per GPU, rendezvous on the loopback address)
+        import socket
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        os.execv(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+                                  "--nproc-per-node", str(args.gpus), "--master-addr", "127.0.0.1",
+                                  "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:])
+    if world > 1 and args.gpus != world:
+        if rank == 0:
+            print("bench.py: --gpus %d does not match the %d ranks of the launcher" % (args.gpus, world),
+                  file=sys.stderr)
+        sys.exit(2)
     if args.impl == "reference":
         run_reference(args, rank, world)
         return
+    if args.impl == "ours":
+        import torch
+        if torch.cuda.device_count() < max(world, 1):
+            print("bench.py: %d ranks but %d visible GPUs" % (world, torch.cuda.device_count()), file=sys.stderr)
+            sys.exit(2)
     run_ours(args, rank, world, local_rank)
 
 

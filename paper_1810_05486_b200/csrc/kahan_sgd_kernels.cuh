@@ -437,16 +437,17 @@ __device__ __forceinline__ void set_pack_word(Pack<BYTES>& r, int w, unsigned in
 // low mantissa bits are that integer in two's complement relative to M, an addition that
 // lands there rounds to nearest-even on the integer grid, and sums, differences and FMAs
 // of integers below 2^24 are exact.  Per element:
-//   qtB = M + bias_t + qt, qcm = M + bias_c + qc   mantissa bytes (sign bit flipped, so the
-//                                         byte is q + bias) spliced under M's exponent (PRMT)
-//   y   = g*scale + (M + bias_c)        = M + bias_c + d, d = rne(g*scale)   (stmt 1)
-//   u   = qcm - y                       = qc - d
-//   Pb  = fma(u, 2^-s, qtB)             = M + bias_t + rne((qt*2^s + u) / 2^s) = M + bias_t + P
-//                                         (stmt 2; M and the bias are even, so the tie falls
-//                                         on the parity of P itself)
-//   w   = Pb - qtB                      = P - qt
+//   qtM = M + qt, qcM = M + qc          the signed mantissa added to M's bit pattern by one
+//                                         integer dot-product instruction (magic_signed)
+//   y   = g*scale + M                   = M + d, d = rne(g*scale)            (stmt 1)
+//   u   = qcM - y                       = qc - d
+//   Pb  = fma(u, 2^-s, qtM)             = M + rne((qt*2^s + u) / 2^s) = M + P
+//                                         (stmt 2; M is even, so the tie falls on the parity
+//                                         of P itself)
+//   w   = Pb - qtM                      = P - qt
 //   r0  = fma(w, -2^s, u)               = T - P*2^s                       (stmt 3)
-// theta' is the low bits of Pb with the sign bit flipped back, c' the low bits of r0 + M.
+// theta' is the low bits of Pb (two's complement of P under M's exponent), c' the low bits
+// of r0 + M.
 // The vector is handed to update_general instead (returns false, nothing stored) when some
 // |g*scale| exceeds 4e6 (y must stay below 2^24) or is Inf or NaN, or some |P| exceeds QMAX:
 // exactly the cases in which the magnitudes above could leave the exact range or a clamp is
@@ -466,6 +467,20 @@ __device__ __forceinline__ float magic_elem(const Pack<BYTES>& r, int i) {
     return __uint_as_float(__byte_perm(pack_word(r, i >> 2), kMagicBits, 0x7640u | (unsigned)(i & 3)));
   } else {
     return __uint_as_float(__byte_perm(pack_word(r, i >> 1), kMagicBits, (i & 1) ? 0x7632u : 0x7610u));
+  }
+}
+
+// M + q for element i of a pack of signed mantissas, in one instruction: the integer dot
+// product with a selector that is 1 at element i sign-extends the mantissa and adds it to
+// M's bit pattern (for |q| < 2^22 integer addition on the bits is addition of the values).
+// It runs on the FMA pipe; the PRMT form above and the sign flips it needs take the ALU
+// pipe, which has half the lanes and also carries the scans and the packing.
+template <int BITS, int BYTES>
+__device__ __forceinline__ float magic_signed(const Pack<BYTES>& r, int i) {
+  if constexpr (BITS == 8) {
+    return __int_as_float(__dp4a((int)pack_word(r, i >> 2), 1 << (8 * (i & 3)), (int)kMagicBits));
+  } else {
+    return __int_as_float(__dp2a_lo((int)pack_word(r, i >> 1), (i & 1) ? 0x0100 : 0x0001, (int)kMagicBits));
   }
 }
 
@@ -527,45 +542,39 @@ __device__ __forceinline__ float min3(float a, float b, float c) {
   return d;
 }
 
-// theta stays biased through the vector: qtB = M + 2^(TB-1) + qt and Pb = M + 2^(TB-1) + P
-// (the bias is even, so the tie still falls on the parity of P); the sign bits of the packed
-// result are flipped back at the end.  The scans take two elements per instruction: the
-// largest and smallest Pb give max|P|, and |x|, |r0| go through three-input maxima.
+// The scans take two elements per instruction: the largest and smallest Pb give max|P|, and
+// |x|, |r0| go through three-input maxima.
 template <int TB, int CB, int V, int GB, bool STRICT>
-__device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V * CB / 8 : 8)> pc,
-                                              Pack<V * GB / 8> pg, const SteadyCoef& k,
+__device__ __forceinline__ bool update_vector(const Pack<V * TB / 8>& pt, const Pack<(CB ? V * CB / 8 : 8)>& pc,
+                                              const Pack<V * GB / 8>& pg, const SteadyCoef& k,
                                               Pack<V * TB / 8>& ot, Pack<(CB ? V * CB / 8 : 8)>& oc,
                                               float& amax_t, float& amax_c) {
   constexpr bool HAS_COMP = CB != 0;
-  constexpr float bias_t = (float)(1 << (TB - 1));
-  constexpr float bias_c = HAS_COMP ? (float)(1 << ((CB ? CB : 8) - 1)) : 0.0f;
-  constexpr float Mt = kMagic + bias_t;
-  flip_signs<TB>(pt);
-  if constexpr (HAS_COMP) flip_signs<(CB ? CB : 8)>(pc);
-  if constexpr (GB != 32) flip_signs<(GB == 32 ? 8 : GB)>(pg);
+  constexpr int CBS = CB ? CB : 8;
+  constexpr int GBS = GB == 32 ? 8 : GB;
   float Pm[V], rm[V], xa[2], ra[2], ua[2];
-  float aX = 0.0f, hiP = Mt, loP = Mt, aR = 0.0f, aU = 0.0f;
+  float aX = 0.0f, hiP = kMagic, loP = kMagic, aR = 0.0f, aU = 0.0f;
 #pragma unroll
   for (int i = 0; i < V; ++i) {
-    const float qtB = magic_elem<TB>(pt, i);
+    const float qtM = magic_signed<TB>(pt, i);
     float g;       // binary32 gradient, or the gradient mantissa (k.scale then carries 2^eg)
     if constexpr (GB == 32) g = __uint_as_float(pack_word(pg, i));
-    else g = __fadd_rn(magic_elem<(GB == 32 ? 8 : GB)>(pg, i), -(kMagic + (float)(1 << ((GB == 32 ? 8 : GB) - 1))));
+    else g = __fadd_rn(magic_signed<GBS>(pg, i), -kMagic);
     const float x = __fmul_rn(g, k.scale);              // the one binary32 multiply
     float u;
     if constexpr (STRICT) {
       // statement 1 with c's own exponent: C1 = rne(Q_c * 2^(ec_in-ec_out) - d), one rounding
       // (the FMA lands in [2^23, 2^24), where floats are the integers)
       const float d = __fadd_rn(__fadd_rn(x, kMagic), -kMagic);
-      const float qc = __fadd_rn(magic_elem<(CB ? CB : 8)>(pc, i), -(kMagic + bias_c));
+      const float qc = __fadd_rn(magic_signed<CBS>(pc, i), -kMagic);
       u = __fadd_rn(__fmaf_rn(qc, k.pow2dc, __fadd_rn(kMagic, -d)), -kMagic);
     } else {
-      const float y = __fadd_rn(x, kMagic + bias_c);      // rounds x to nearest-even integer
-      if constexpr (HAS_COMP) u = __fadd_rn(magic_elem<(CB ? CB : 8)>(pc, i), -y);
+      const float y = __fadd_rn(x, kMagic);               // rounds x to nearest-even integer
+      if constexpr (HAS_COMP) u = __fadd_rn(magic_signed<CBS>(pc, i), -y);
       else u = __fadd_rn(kMagic, -y);
     }
-    const float P = __fmaf_rn(u, k.inv2s, qtB);
-    const float w = __fadd_rn(P, -qtB);
+    const float P = __fmaf_rn(u, k.inv2s, qtM);
+    const float w = __fadd_rn(P, -qtM);
     const float r0 = __fmaf_rn(w, k.pow2s_neg, u);
     Pm[i] = P;
     rm[i] = __fadd_rn(r0, kMagic);
@@ -580,19 +589,18 @@ __device__ __forceinline__ bool update_vector(Pack<V * TB / 8> pt, Pack<(CB ? V 
       if constexpr (STRICT) aU = max3(aU, ua[0], ua[1]);  // u = c - d is statement 1's result
     }
   }
-  const float aP = fmaxf(__fadd_rn(hiP, -Mt), __fadd_rn(Mt, -loP));
+  const float aP = fmaxf(__fadd_rn(hiP, -kMagic), __fadd_rn(kMagic, -loP));
   constexpr float qmax_t = (float)((1 << (TB - 1)) - 1);
   if (!(aX <= 4000000.0f) | (aP > qmax_t)) return false;   // also Inf and NaN products
   if constexpr (STRICT) {
     // both accumulator results must fit their n bits, or the vector needs the clamps
-    constexpr float qmax_c = (float)((1 << ((CB ? CB : 8) - 1)) - 1);
+    constexpr float qmax_c = (float)((1 << (CBS - 1)) - 1);
     aR = fmaxf(aR, aU);
     if (aR > qmax_c) return false;
   }
   amax_t = fmaxf(amax_t, aP);
   if constexpr (HAS_COMP) amax_c = fmaxf(amax_c, aR);
   ot = pack_magic<TB, V>(Pm);
-  flip_signs<TB>(ot);
   if constexpr (HAS_COMP) oc = pack_magic<CB, V>(rm);
   return true;
 }
@@ -623,25 +631,23 @@ __device__ __forceinline__ bool update_vector_regrid(Pack<V * TB / 8> pt, Pack<(
   constexpr int CBS = CB ? CB : 8;
   constexpr int GBS = GB == 32 ? 8 : GB;
   constexpr float bias_t = (float)(1 << (TB - 1));
-  constexpr float bias_c = (float)(1 << (CBS - 1));
-  flip_signs<TB>(pt);
-  if constexpr (HAS_COMP) flip_signs<CBS>(pc);
-  if constexpr (GB != 32) flip_signs<GBS>(pg);
   const bool finer = k.pow2dc > 1.0f;
   // 2^a and 2^-a
   const float up = finer ? k.pow2dc : __int_as_float(0x7f000000 - __float_as_int(k.pow2dc));
   const float down = finer ? __int_as_float(0x7f000000 - __float_as_int(k.pow2dc)) : k.pow2dc;
-  Pack<V * TB / 8> pB = pt;
+  Pack<V * TB / 8> pA = pt, pB = pt;
   float inv2sp = k.inv2s, pow2sp_neg = k.pow2s_neg, biasA = bias_t, pow2s = -k.pow2s_neg;
   if (!finer) {
+    // split on the sign-flipped (unsigned) lanes: a logical shift and a mask per word
+    flip_signs<TB>(pA);
     const int a = 127 - (int)(__float_as_uint(k.pow2dc) >> 23);
     constexpr unsigned int lanes = TB == 8 ? 0x01010101u : 0x00010001u;
     constexpr unsigned int full = TB == 8 ? 0xffu : 0xffffu;
     const unsigned int maskA = (full >> a) * lanes, maskB = ((1u << a) - 1u) * lanes;
 #pragma unroll
     for (int w = 0; w < V * TB / 32; ++w) {
-      const unsigned int x = pack_word(pt, w);
-      set_pack_word(pt, w, (x >> a) & maskA);
+      const unsigned int x = pack_word(pA, w);
+      set_pack_word(pA, w, (x >> a) & maskA);
       set_pack_word(pB, w, x & maskB);
     }
     inv2sp = __fmul_rn(k.inv2s, down);          // 2^-s'
@@ -654,14 +660,14 @@ __device__ __forceinline__ bool update_vector_regrid(Pack<V * TB / 8> pt, Pack<(
   for (int i = 0; i < V; ++i) {
     float g;
     if constexpr (GB == 32) g = __uint_as_float(pack_word(pg, i));
-    else g = __fadd_rn(magic_elem<GBS>(pg, i), -(kMagic + (float)(1 << (GBS - 1))));
+    else g = __fadd_rn(magic_signed<GBS>(pg, i), -kMagic);
     const float x = __fmul_rn(g, k.scale);              // the one binary32 multiply
     const float y = __fadd_rn(x, kMagic);               // M + d
     float qc = 0.0f;
-    if constexpr (HAS_COMP) qc = __fadd_rn(magic_elem<CBS>(pc, i), -(kMagic + bias_c));
+    if constexpr (HAS_COMP) qc = __fadd_rn(magic_signed<CBS>(pc, i), -kMagic);
     float P, r;
     if (finer) {
-      const float qt = __fadd_rn(magic_elem<TB>(pt, i), -(kMagic + bias_t));
+      const float qt = __fadd_rn(magic_signed<TB>(pt, i), -kMagic);
       const float base = __fmaf_rn(qt, up, kMagic);
       const float u = __fmaf_rn(qc, up, __fadd_rn(kMagic, -y));
       P = __fmaf_rn(u, inv2sp, base);
@@ -669,7 +675,7 @@ __device__ __forceinline__ bool update_vector_regrid(Pack<V * TB / 8> pt, Pack<(
       r = __fmaf_rn(w, pow2sp_neg, u);
       rm[i] = __fadd_rn(r, kMagic);
     } else {
-      const float base = __fadd_rn(magic_elem<TB>(pt, i), -biasA);       // M + A
+      const float base = __fadd_rn(magic_elem<TB>(pA, i), -biasA);       // M + A
       const float B = __fadd_rn(magic_elem<TB>(pB, i), -kMagic);
       const float d = __fadd_rn(y, -kMagic);
       const float v = __fmaf_rn(d, -up, __fmaf_rn(B, pow2s, qc));

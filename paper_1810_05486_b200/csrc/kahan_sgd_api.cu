@@ -56,12 +56,13 @@ cudaError_t launch_step_kernel(void (*kernel)(KArgs...), unsigned grid, unsigned
   return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
-// Offsets of the workspace regions.  The first four regions are contiguous so that
+// Offsets of the workspace regions.  The regions up to stats_end are contiguous so that
 // kahan_sgd_amax fetches them with one copy.
 struct Layout {
-  size_t exp_cur, exp_next, amax_last, counters, error, stats_end;
-  size_t amax_acc, info, grad_ptr, lr, exp_grad, expc_cur, expc_next, chunks, ticket, total;
+  size_t phase, state, counters, error, stats_end;
+  size_t info, grad_ptr, lr, exp_grad, chunks, total;
   long long n_chunks;
+  int slab;                // records per phase slab (a slab is a multiple of 128 bytes)
 };
 
 // Tile size of a tensor, given the list's tile size for 8-bit theta.
@@ -83,28 +84,105 @@ Layout make_layout(const ksgd_tensor_desc* d, int32_t n, int chunk8) {
   long long chunks = 0;
   for (int32_t i = 0; i < n; ++i) chunks += (d[i].numel + tile_elems(d[i], chunk8) - 1) / tile_elems(d[i], chunk8);
   L.n_chunks = chunks;
+  L.slab = (int)(align_up(sizeof(TensorState) * (size_t)n, 128) / sizeof(TensorState));
   size_t o = 0;
-  L.exp_cur = o;   o += sizeof(int) * n;
-  L.exp_next = o;  o += sizeof(int) * n;
-  L.amax_last = o; o += sizeof(unsigned int) * 2 * n;
-  o = align_up(o, 8);
+  L.phase = o;     o += 128;
+  L.state = o;     o += sizeof(TensorState) * 3 * L.slab;
   L.counters = o;  o += sizeof(unsigned long long) * 3 * n;
   L.error = o;     o += 8;
   L.stats_end = o;
-  L.amax_acc = o;  o += sizeof(unsigned int) * 2 * n;
   o = align_up(o, 16);
   L.info = o;      o += sizeof(TensorInfo) * n;
   L.grad_ptr = o;  o += sizeof(const float*) * n;
   L.lr = o;        o += sizeof(float) * n;
   L.exp_grad = o;  o += sizeof(int) * n;
-  L.expc_cur = o;  o += sizeof(int) * n;
-  L.expc_next = o; o += sizeof(int) * n;
   o = align_up(o, 16);
   L.chunks = o;    o += sizeof(ChunkRef) * (size_t)chunks;
-  o = align_up(o, 16);
-  L.ticket = o;    o += 16;
   L.total = align_up(o, 256);
   return L;
+}
+
+// Device-side view of a workspace at `b`.
+void bind_workspace(Workspace& w, char* b, const Layout& L) {
+  w.phase = reinterpret_cast<unsigned int*>(b + L.phase);
+  w.state = reinterpret_cast<TensorState*>(b + L.state);
+  w.slab = L.slab;
+  w.counters = reinterpret_cast<unsigned long long*>(b + L.counters);
+  w.error = reinterpret_cast<unsigned int*>(b + L.error);
+  w.info = reinterpret_cast<TensorInfo*>(b + L.info);
+  w.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
+  w.lr = reinterpret_cast<float*>(b + L.lr);
+  w.exp_grad = reinterpret_cast<int*>(b + L.exp_grad);
+  w.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
+}
+
+// Host image of a fresh workspace (`img`: L.total zero bytes): phase 0; in the records the
+// first step reads (slab 2) the exponents of the stored mantissas and, as overrides, the
+// exponents the first step must write; zeroed scans and counters; tensor table; tile
+// table.  first_tile (optional) receives the first tile of every tensor, plus the total.
+void write_initial_image(unsigned char* img, const Layout& L, const ksgd_tensor_desc* descs, int32_t n,
+                         const int32_t* exp_comp, const int32_t* exp_comp_next, int chunk8,
+                         std::vector<long long>* first_tile) {
+  TensorState* last = reinterpret_cast<TensorState*>(img + L.state) + 2 * (size_t)L.slab;
+  TensorInfo* info = reinterpret_cast<TensorInfo*>(img + L.info);
+  ChunkRef* chunks = reinterpret_cast<ChunkRef*>(img + L.chunks);
+  long long c = 0;
+  for (int32_t i = 0; i < n; ++i) {
+    const ksgd_tensor_desc& t = descs[i];
+    last[i].exp_theta = t.exp_theta;
+    last[i].ovr_theta = t.exp_theta_next + kOvrBias;
+    if (exp_comp) {
+      last[i].exp_comp = exp_comp[i];
+      last[i].ovr_comp = (exp_comp_next ? exp_comp_next[i] : exp_comp[i]) + kOvrBias;
+    }
+    info[i].theta = t.theta;
+    info[i].comp = t.comp;
+    info[i].numel = t.numel;
+    info[i].theta_bits = t.theta_bits;
+    info[i].comp_bits = t.comp_bits;
+    info[i].s = t.comp_bits ? t.comp_bits - 1 - t.overlap_k : 0;
+    info[i].pad = 0;
+    const long long nc = (t.numel + tile_elems(t, chunk8) - 1) / tile_elems(t, chunk8);
+    if (first_tile) first_tile->push_back(c);
+    for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
+  }
+  if (first_tile) first_tile->push_back(c);
+}
+
+// The caller's view of a copy of the stats region: scans and exponent of the last finished
+// step, the exponent the coming step will write (its override if one is set, else what the
+// scan implies: the rule the kernel itself applies), cumulative counters, error word.
+int read_stats(const unsigned char* b, const Layout& L, const ksgd_tensor_desc* descs, int32_t n_tensors,
+               int amax_mode, bool strict, uint32_t* amax_theta, uint32_t* amax_comp, int32_t* exp_theta_cur,
+               int32_t* exp_theta_next, uint64_t* n_sat_theta, uint64_t* n_sat_comp, uint64_t* n_nonfinite,
+               int32_t* exp_comp_cur, int32_t* exp_comp_next) {
+  const size_t n = (size_t)n_tensors;
+  unsigned int ph = 0;
+  std::memcpy(&ph, b + L.phase, 4);
+  if (ph > 2) return KSGD_ERR_DEVICE;
+  const TensorState* last = reinterpret_cast<const TensorState*>(b + L.state) + ((ph + 2) % 3) * (size_t)L.slab;
+  for (size_t i = 0; i < n; ++i) {
+    const TensorState& r = last[i];
+    const int e_next = r.ovr_theta ? r.ovr_theta - kOvrBias
+                                   : next_exponent(r.amax_t, descs[i].theta_bits, r.exp_theta, amax_mode);
+    if (amax_theta) amax_theta[i] = r.amax_t;
+    if (amax_comp) amax_comp[i] = r.amax_c;
+    if (exp_theta_cur) exp_theta_cur[i] = r.exp_theta;
+    if (exp_theta_next) exp_theta_next[i] = e_next;
+    if (strict) {
+      if (exp_comp_cur) exp_comp_cur[i] = r.exp_comp;
+      if (exp_comp_next)
+        exp_comp_next[i] = r.ovr_comp ? r.ovr_comp - kOvrBias
+                                      : next_exponent_acc(r.amax_c, descs[i].comp_bits, r.exp_comp, e_next, amax_mode);
+    }
+  }
+  if (n_sat_theta) std::memcpy(n_sat_theta, b + L.counters, 8 * n);
+  if (n_sat_comp) std::memcpy(n_sat_comp, b + L.counters + 8 * n, 8 * n);
+  if (n_nonfinite) std::memcpy(n_nonfinite, b + L.counters + 16 * n, 8 * n);
+  unsigned int dev_err = 0;
+  std::memcpy(&dev_err, b + L.error, 4);
+  if (dev_err != 0) return KSGD_ERR_DEVICE;
+  return KSGD_OK;
 }
 
 int validate(const ksgd_tensor_desc* d, int32_t n) {
@@ -210,55 +288,11 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   h->stats_host.resize(L.stats_end);
   h->strict = strict;
 
-  // Host image of the workspace: exponents, zeroed scans and counters, tensor table,
-  // chunk table.
   std::vector<unsigned char> img(L.total, 0);
-  int* exp_cur = reinterpret_cast<int*>(img.data() + L.exp_cur);
-  int* exp_next = reinterpret_cast<int*>(img.data() + L.exp_next);
-  if (strict) {
-    int* ec_cur = reinterpret_cast<int*>(img.data() + L.expc_cur);
-    int* ec_nx = reinterpret_cast<int*>(img.data() + L.expc_next);
-    for (int32_t i = 0; i < n_tensors; ++i) {
-      ec_cur[i] = exp_comp[i];
-      ec_nx[i] = exp_comp_next ? exp_comp_next[i] : exp_comp[i];
-    }
-  }
-  TensorInfo* info = reinterpret_cast<TensorInfo*>(img.data() + L.info);
-  ChunkRef* chunks = reinterpret_cast<ChunkRef*>(img.data() + L.chunks);
-  long long c = 0;
-  for (int32_t i = 0; i < n_tensors; ++i) {
-    const ksgd_tensor_desc& t = descs[i];
-    exp_cur[i] = t.exp_theta;
-    exp_next[i] = t.exp_theta_next;
-    info[i].theta = t.theta;
-    info[i].comp = t.comp;
-    info[i].numel = t.numel;
-    info[i].theta_bits = t.theta_bits;
-    info[i].comp_bits = t.comp_bits;
-    info[i].s = t.comp_bits ? t.comp_bits - 1 - t.overlap_k : 0;
-    info[i].pad = 0;
-    const long long nc = (t.numel + tile_elems(t, chunk8) - 1) / tile_elems(t, chunk8);
-    h->first_tile.push_back(c);
-    for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
-  }
-  h->first_tile.push_back(c);
-
-  Workspace& w = h->params.ws;
+  write_initial_image(img.data(), L, descs, n_tensors, strict ? exp_comp : nullptr, exp_comp_next, chunk8,
+                      &h->first_tile);
   char* b = h->ws_base;
-  w.exp_cur = reinterpret_cast<int*>(b + L.exp_cur);
-  w.exp_next = reinterpret_cast<int*>(b + L.exp_next);
-  w.amax_last = reinterpret_cast<unsigned int*>(b + L.amax_last);
-  w.counters = reinterpret_cast<unsigned long long*>(b + L.counters);
-  w.error = reinterpret_cast<unsigned int*>(b + L.error);
-  w.amax_acc = reinterpret_cast<unsigned int*>(b + L.amax_acc);
-  w.info = reinterpret_cast<TensorInfo*>(b + L.info);
-  w.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
-  w.lr = reinterpret_cast<float*>(b + L.lr);
-  w.exp_grad = reinterpret_cast<int*>(b + L.exp_grad);
-  w.expc_cur = reinterpret_cast<int*>(b + L.expc_cur);
-  w.expc_next = reinterpret_cast<int*>(b + L.expc_next);
-  w.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
-  w.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
+  bind_workspace(h->params.ws, b, L);
   h->params.n_tensors = n_tensors;
   h->params.n_chunks = (int)L.n_chunks;
   h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
@@ -267,6 +301,7 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   h->params.tile_count = (int)L.n_chunks;
   h->params.tensor_begin = 0;
   h->params.tensor_count = n_tensors;
+  h->params.advance = 1;
 
   // Persistent grid: one block per SM (fewer if the list has fewer tiles).
   int dev = 0, sms = 0, l2_bytes = 0;
@@ -343,16 +378,22 @@ int kahan_sgd_strict_init(ksgd_handle** out, const ksgd_tensor_desc* descs, cons
                      cuda_stream);
 }
 
+static int fetch_stats(ksgd_handle* h) {
+  KSGD_CUDA(cudaMemcpyAsync(h->stats_host.data(), h->ws_base, h->layout.stats_end, cudaMemcpyDeviceToHost,
+                            h->stream));
+  KSGD_CUDA(cudaStreamSynchronize(h->stream));
+  return KSGD_OK;
+}
+
 int kahan_sgd_strict_exponents(ksgd_handle* h, int32_t* exp_comp_cur, int32_t* exp_comp_next) {
   if (!h) return KSGD_ERR_NULL;
   if (!h->strict) return KSGD_ERR_MODE;
-  std::vector<int> host(2 * (size_t)h->n);
-  KSGD_CUDA(cudaMemcpyAsync(host.data(), h->ws_base + h->layout.expc_cur, sizeof(int) * 2 * (size_t)h->n,
-                            cudaMemcpyDeviceToHost, h->stream));
-  KSGD_CUDA(cudaStreamSynchronize(h->stream));
-  if (exp_comp_cur) std::memcpy(exp_comp_cur, host.data(), sizeof(int) * (size_t)h->n);
-  if (exp_comp_next) std::memcpy(exp_comp_next, host.data() + h->n, sizeof(int) * (size_t)h->n);
-  return KSGD_OK;
+  const int r = fetch_stats(h);
+  if (r != KSGD_OK) return r;
+  const int rs = read_stats(h->stats_host.data(), h->layout, h->descs.data(), h->n, h->params.amax_mode, true,
+                            nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, exp_comp_cur,
+                            exp_comp_next);
+  return rs == KSGD_ERR_DEVICE ? KSGD_OK : rs;    // the device error word is kahan_sgd_amax's to report
 }
 
 static int check_step_args(const ksgd_handle* h, const float* const* grads, const float* lrs) {
@@ -368,6 +409,7 @@ static int check_step_args(const ksgd_handle* h, const float* const* grads, cons
 // Launch the step on tensors [t0, t1) (their tiles are contiguous in the table).
 static int launch_step_range(ksgd_handle* h, const InlineArgs* ia, int32_t t0, int32_t t1) {
   StepParams p = h->params;
+  p.advance = t1 == h->n ? 1 : 0;     // the groups of one step share its phase; the last one moves it on
   p.tile_begin = (int)h->first_tile[t0];
   p.tile_count = (int)(h->first_tile[t1] - h->first_tile[t0]);
   p.tensor_begin = t0;
@@ -600,23 +642,11 @@ int kahan_sgd_amax(ksgd_handle* h, uint32_t* amax_theta, uint32_t* amax_comp,
                    int32_t* exp_theta_cur, int32_t* exp_theta_next, uint64_t* n_sat_theta,
                    uint64_t* n_sat_comp, uint64_t* n_nonfinite) {
   if (!h) return KSGD_ERR_NULL;
-  const Layout& L = h->layout;
-  KSGD_CUDA(cudaMemcpyAsync(h->stats_host.data(), h->ws_base, L.stats_end, cudaMemcpyDeviceToHost,
-                            h->stream));
-  KSGD_CUDA(cudaStreamSynchronize(h->stream));
-  const unsigned char* b = h->stats_host.data();
-  const size_t n = (size_t)h->n;
-  if (exp_theta_cur) std::memcpy(exp_theta_cur, b + L.exp_cur, 4 * n);
-  if (exp_theta_next) std::memcpy(exp_theta_next, b + L.exp_next, 4 * n);
-  if (amax_theta) std::memcpy(amax_theta, b + L.amax_last, 4 * n);
-  if (amax_comp) std::memcpy(amax_comp, b + L.amax_last + 4 * n, 4 * n);
-  if (n_sat_theta) std::memcpy(n_sat_theta, b + L.counters, 8 * n);
-  if (n_sat_comp) std::memcpy(n_sat_comp, b + L.counters + 8 * n, 8 * n);
-  if (n_nonfinite) std::memcpy(n_nonfinite, b + L.counters + 16 * n, 8 * n);
-  unsigned int dev_err = 0;
-  std::memcpy(&dev_err, b + L.error, 4);
-  if (dev_err != 0) return KSGD_ERR_DEVICE;
-  return KSGD_OK;
+  const int r = fetch_stats(h);
+  if (r != KSGD_OK) return r;
+  return read_stats(h->stats_host.data(), h->layout, h->descs.data(), h->n, h->params.amax_mode, h->strict,
+                    amax_theta, amax_comp, exp_theta_cur, exp_theta_next, n_sat_theta, n_sat_comp, n_nonfinite,
+                    nullptr, nullptr);
 }
 
 int kahan_sgd_set_exponents(ksgd_handle* h, const int32_t* exp_theta_next) {
@@ -629,8 +659,8 @@ int kahan_sgd_set_exponents(ksgd_handle* h, const int32_t* exp_theta_next) {
   for (int32_t first = 0; first < h->n; first += kUploadBatch) {
     const int count = h->n - first < kUploadBatch ? h->n - first : kUploadBatch;
     for (int i = 0; i < count; ++i) eb->exp_next[i] = exp_theta_next[first + i];
-    ksgd_set_exponents_kernel<<<1, 256, 0, h->stream>>>(*eb, first, count, h->params.ws.exp_cur,
-                                                        h->params.ws.exp_next);
+    ksgd_set_exponents_kernel<<<1, 256, 0, h->stream>>>(*eb, first, count, h->layout.slab, h->params.ws.phase,
+                                                        h->params.ws.state);
     g_launches.fetch_add(1, std::memory_order_relaxed);
   }
   delete eb;
@@ -709,47 +739,17 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   }
 
   // Host image of the scratch, every byte of it: whatever the previous call left in the
-  // array (scans, counters, ticket, tile counter) is overwritten.
+  // array (scans, counters, phase and tickets) is overwritten.
   std::vector<unsigned char> img(L.total, 0);
-  int* e_cur = reinterpret_cast<int*>(img.data() + L.exp_cur);
-  int* e_next = reinterpret_cast<int*>(img.data() + L.exp_next);
-  TensorInfo* info = reinterpret_cast<TensorInfo*>(img.data() + L.info);
-  ChunkRef* chunks = reinterpret_cast<ChunkRef*>(img.data() + L.chunks);
-  long long c = 0;
+  write_initial_image(img.data(), L, descs, n_tensors, nullptr, nullptr, kChunk, nullptr);
   double state_bytes = 0.0;
-  for (int32_t i = 0; i < n_tensors; ++i) {
-    const ksgd_tensor_desc& t = descs[i];
-    e_cur[i] = t.exp_theta;
-    e_next[i] = t.exp_theta_next;
-    info[i].theta = t.theta;
-    info[i].comp = t.comp;
-    info[i].numel = t.numel;
-    info[i].theta_bits = t.theta_bits;
-    info[i].comp_bits = t.comp_bits;
-    info[i].s = t.comp_bits ? t.comp_bits - 1 - t.overlap_k : 0;
-    info[i].pad = 0;
-    const long long nc = (t.numel + kChunk - 1) / kChunk;
-    for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
-    state_bytes += (double)t.numel * ((t.theta_bits + t.comp_bits) / 8);
-  }
+  for (int32_t i = 0; i < n_tensors; ++i)
+    state_bytes += (double)descs[i].numel * ((descs[i].theta_bits + descs[i].comp_bits) / 8);
   const int grid = (int)(L.n_chunks < (long long)sd.sms ? L.n_chunks : (long long)sd.sms);
 
   StepParams params;
   unsigned char* b = sd.scratch;
-  params.ws.exp_cur = reinterpret_cast<int*>(b + L.exp_cur);
-  params.ws.exp_next = reinterpret_cast<int*>(b + L.exp_next);
-  params.ws.amax_last = reinterpret_cast<unsigned int*>(b + L.amax_last);
-  params.ws.counters = reinterpret_cast<unsigned long long*>(b + L.counters);
-  params.ws.error = reinterpret_cast<unsigned int*>(b + L.error);
-  params.ws.amax_acc = reinterpret_cast<unsigned int*>(b + L.amax_acc);
-  params.ws.info = reinterpret_cast<TensorInfo*>(b + L.info);
-  params.ws.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
-  params.ws.lr = reinterpret_cast<float*>(b + L.lr);
-  params.ws.exp_grad = reinterpret_cast<int*>(b + L.exp_grad);
-  params.ws.expc_cur = reinterpret_cast<int*>(b + L.expc_cur);
-  params.ws.expc_next = reinterpret_cast<int*>(b + L.expc_next);
-  params.ws.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
-  params.ws.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
+  bind_workspace(params.ws, reinterpret_cast<char*>(b), L);
   params.n_tensors = n_tensors;
   params.n_chunks = (int)L.n_chunks;
   params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
@@ -760,6 +760,7 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   params.tensor_count = n_tensors;
   params.grad_evict_first = state_bytes <= 0.8 * (double)sd.l2_bytes ? 1 : 0;
   params.chunk8 = kChunk;
+  params.advance = 1;
 
   InlineArgs inl;
   for (int32_t i = 0; i < n_tensors; ++i) { inl.grads[i] = grads[i]; inl.lrs[i] = lrs[i]; }
@@ -773,19 +774,8 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   KSGD_CUDA(cudaMemcpyAsync(img.data(), b, L.stats_end, cudaMemcpyDeviceToHost, stream));
   KSGD_CUDA(cudaStreamSynchronize(stream));
 
-  const unsigned char* r = img.data();
-  const size_t n = (size_t)n_tensors;
-  if (exp_theta_cur) std::memcpy(exp_theta_cur, r + L.exp_cur, 4 * n);
-  if (exp_theta_next) std::memcpy(exp_theta_next, r + L.exp_next, 4 * n);
-  if (amax_theta) std::memcpy(amax_theta, r + L.amax_last, 4 * n);
-  if (amax_comp) std::memcpy(amax_comp, r + L.amax_last + 4 * n, 4 * n);
-  if (n_sat_theta) std::memcpy(n_sat_theta, r + L.counters, 8 * n);
-  if (n_sat_comp) std::memcpy(n_sat_comp, r + L.counters + 8 * n, 8 * n);
-  if (n_nonfinite) std::memcpy(n_nonfinite, r + L.counters + 16 * n, 8 * n);
-  unsigned int dev_err = 0;
-  std::memcpy(&dev_err, r + L.error, 4);
-  if (dev_err != 0) return KSGD_ERR_DEVICE;
-  return KSGD_OK;
+  return read_stats(img.data(), L, descs, n_tensors, params.amax_mode, false, amax_theta, amax_comp, exp_theta_cur,
+                    exp_theta_next, n_sat_theta, n_sat_comp, n_nonfinite, nullptr, nullptr);
 }
 
 // ----------------------------------------------------------------------------------------

@@ -8,7 +8,8 @@
 //     theta's grid (theta'), and what the rounding lost is stored back as c';
 //   - the per-tensor max scans that dynamic fixed-point needs to choose the next
 //     exponent (Section 5): registers -> warp reduce -> one atomicMax per warp and tensor;
-//   - in the last block to finish, the exponent choice itself for every tensor.
+//   - the exponent choice for every tensor, made by the blocks of the NEXT step from the
+//     finished scans (rotating buffers, see Workspace): no block is ever the last one.
 // The pass is bound by HBM traffic: 2*m/8 + 2*n/8 + 4 bytes per parameter.
 //
 // Structure: a persistent grid, one block per SM.  The tensor list is cut into tiles of
@@ -21,6 +22,17 @@
 // Sixteen consumer warps compute from shared memory and store theta' and c' straight to
 // global memory with 16-byte stores.
 // No block ever waits for another block; every wait inside a block is bounded.
+//
+// State between steps.  The per-tensor state a step leaves behind (the exponent it wrote,
+// its max scans) lives in three rotating buffers indexed by the step's phase p = step mod 3
+// (a word in the workspace).  Step p reads buffer p-1 (exponent of the stored mantissas,
+// finished scans), derives from it the exponent it writes (every block that meets a tensor
+// derives the same value and stores it into buffer p: idempotent), accumulates its own scans
+// into buffer p, and clears buffer p+1, which nobody reads or writes until the next step.
+// So a step needs no pass "after all blocks are done": the kernel ends when each block has
+// published its scans, and the next launch finds everything it needs.  The phase word is
+// advanced by the block that draws the last entry ticket, i.e. after every block of the
+// step has read it.
 #pragma once
 
 #include <cstdint>
@@ -63,22 +75,33 @@ struct ChunkRef {
 };
 
 // Device-side view of the caller's workspace.
+// What a step leaves behind for one tensor: everything the next step needs to know about it,
+// in one 32-byte record (one load).
+struct __align__(32) TensorState {
+  int exp_theta;          // exponent of theta's mantissas as this step wrote them
+  int exp_comp;           // strict mode: the same for the compensation's own exponent
+  unsigned int amax_t;    // this step's max scans (blocks add to them while the step runs)
+  unsigned int amax_c;
+  int ovr_theta;          // exponent the NEXT step must write instead of the one the scans give:
+  int ovr_comp;           //   value + kOvrBias, 0 = none (init, kahan_sgd_set_exponents; comp: init only)
+  int pad[2];
+};
+
 struct Workspace {
-  int* exp_cur;                    // [n] exponent of the stored mantissas
-  int* exp_next;                   // [n] exponent the coming step writes
-  unsigned int* amax_last;         // [2n] max scans of the last finished step (theta | comp)
+  unsigned int* phase;             // [0] phase of the coming step (0..2); [1] entry tickets drawn in the running step
+  // [3][slab] records, one slab per phase; a slab starts on a 128-byte boundary, so that the
+  // slab all blocks add their scans to shares no cache line with the one they read.
+  TensorState* state;
+  int slab;                        // records per slab
   unsigned long long* counters;    // [3n] cumulative: sat_theta | sat_comp | nonfinite
   unsigned int* error;             // [1] first DeviceError seen (0 = none), sticky
-  unsigned int* amax_acc;          // [2n] max scans being accumulated by the running step
   TensorInfo* info;                // [n]
   const float** grad_ptr;          // [n] per-step arguments for lists longer than kInlineArgs
   float* lr;                       // [n]
   int* exp_grad;                   // [n] the same, exponents of fixed-point gradients
-  int* expc_cur;                   // [n] strict mode: the compensation's own exponent, stored ...
-  int* expc_next;                  // [n] ... and the one the coming step writes
   ChunkRef* chunks;                // [n_chunks]
-  unsigned int* ticket;            // blocks finished in the running step
 };
+constexpr int kOvrBias = 1000;
 
 struct StepParams {
   Workspace ws;
@@ -87,6 +110,8 @@ struct StepParams {
   int amax_mode;     // 1: exponents follow the max scan, 0: fixed
   int inline_args;   // 1: grads/lrs are in the InlineArgs parameter
   int grad_evict_first;  // 1: gradient loads carry the L2 evict-first hint
+  int advance;           // 1: this launch ends a step (the phase word moves on); 0: more launches of the
+                         //    same step follow (the host-buffer entry point updates groups of tensors in turn)
   // The launch covers tiles [tile_begin, tile_begin + tile_count), which are all the tiles
   // of tensors [tensor_begin, tensor_begin + tensor_count): the whole list for an ordinary
   // step, one group of tensors when the host-buffer entry point pipelines its copies.
@@ -187,6 +212,12 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, u
   asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(
                    smem_addr(bar)),
                "r"(bytes)
+               : "memory");
+}
+
+// Announce `bytes` more bytes for the current phase without arriving.
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned int bytes) {
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
                : "memory");
 }
 
@@ -844,16 +875,27 @@ __device__ __noinline__ void regrid_tile(const TileDesc* td, TileScan* slots, un
 // Next exponent from the max scan: the tight fit puts the largest mantissa in
 // (QMAX/2, QMAX].  With L = bit length of amax and QMAX = 2^(b-1)-1, the change is
 // L-(b-1), plus one more when amax still exceeds QMAX*2^change.
-__device__ __forceinline__ int next_exponent(unsigned int amax, int bits, int e_out, int amax_mode) {
+__host__ __device__ __forceinline__ int bit_length(unsigned int x) {
+#ifdef __CUDA_ARCH__
+  return 32 - __clz(x);
+#else
+  int n = 0;
+  while (x) { ++n; x >>= 1; }
+  return n;
+#endif
+}
+
+__host__ __device__ __forceinline__ int next_exponent(unsigned int amax, int bits, int e_out, int amax_mode) {
   if (!amax_mode || amax == 0u) return e_out;
-  const int L = 32 - __clz(amax);
+  const int L = bit_length(amax);
   int change = L - (bits - 1);
   if (change >= 1) {
     const unsigned long long cap = (unsigned long long)((1 << (bits - 1)) - 1) << change;
     if ((unsigned long long)amax > cap) ++change;
   }
-  change = max(-kMaxDelta, min(kMaxDelta, change));
-  return max(kExpMin, min(kExpMax, e_out + change));
+  change = change < -kMaxDelta ? -kMaxDelta : (change > kMaxDelta ? kMaxDelta : change);
+  const int e = e_out + change;
+  return e < kExpMin ? kExpMin : (e > kExpMax ? kExpMax : e);
 }
 
 // Strict mode: the compensation's own next exponent.  The tight fit of its scan; an empty
@@ -861,12 +903,12 @@ __device__ __forceinline__ int next_exponent(unsigned int amax, int bits, int e_
 // result stays within [e_next - 36, e_next + 8] of theta's next exponent, which keeps every
 // sum of the step within 64 bits.
 constexpr int kStrictBelow = 36, kStrictAbove = 8;
-__device__ __forceinline__ int next_exponent_acc(unsigned int amax, int bits, int ec_out, int e_next,
-                                                 int amax_mode) {
+__host__ __device__ __forceinline__ int next_exponent_acc(unsigned int amax, int bits, int ec_out, int e_next,
+                                                          int amax_mode) {
   int ec = next_exponent(amax, bits, ec_out, amax_mode);
   if (amax_mode && amax == 0u) ec = ec_out - kMaxDelta;
-  ec = max(e_next - kStrictBelow, min(e_next + kStrictAbove, ec));
-  return max(kExpMin, min(kExpMax, ec));
+  ec = ec < e_next - kStrictBelow ? e_next - kStrictBelow : (ec > e_next + kStrictAbove ? e_next + kStrictAbove : ec);
+  return ec < kExpMin ? kExpMin : (ec > kExpMax ? kExpMax : ec);
 }
 
 struct __align__(128) BlockShared {
@@ -876,7 +918,6 @@ struct __align__(128) BlockShared {
   TileScan scan[kSlots];
   int slot_pages[kSlots];              // ring pages held by the tile in each slot
   int abort_flag;   // set by the first thread whose bounded wait ran out
-  int is_last;
   int never;        // stays 0: abort flag for waits that must not be cut short
 };
 
@@ -889,11 +930,11 @@ struct ScanAcc {
   unsigned int amax_t = 0, amax_c = 0, n_sat_t = 0, n_sat_c = 0, n_nonfinite = 0;
 };
 
-__device__ __forceinline__ void publish(const StepParams& p, ScanAcc& acc) {
+__device__ __forceinline__ void publish(const StepParams& p, ScanAcc& acc, TensorState* now) {
   if (acc.tensor >= 0) {
     const int t = acc.tensor, n = p.n_tensors;
-    if (acc.amax_t) atomicMax(&p.ws.amax_acc[t], acc.amax_t);
-    if (acc.amax_c) atomicMax(&p.ws.amax_acc[n + t], acc.amax_c);
+    if (acc.amax_t) atomicMax(&now[t].amax_t, acc.amax_t);
+    if (acc.amax_c) atomicMax(&now[t].amax_c, acc.amax_c);
     if (acc.n_sat_t) atomicAdd(&p.ws.counters[t], (unsigned long long)acc.n_sat_t);
     if (acc.n_sat_c) atomicAdd(&p.ws.counters[n + t], (unsigned long long)acc.n_sat_c);
     if (acc.n_nonfinite) atomicAdd(&p.ws.counters[2 * n + t], (unsigned long long)acc.n_nonfinite);
@@ -901,9 +942,10 @@ __device__ __forceinline__ void publish(const StepParams& p, ScanAcc& acc) {
   acc = ScanAcc{};
 }
 
-__device__ __forceinline__ void take_back(const StepParams& p, ScanAcc& acc, TileScan* scan, int tensor) {
+__device__ __forceinline__ void take_back(const StepParams& p, ScanAcc& acc, TensorState* now,
+                                          TileScan* scan, int tensor) {
   if (tensor != acc.tensor) {
-    publish(p, acc);
+    publish(p, acc, now);
     acc.tensor = tensor;
   }
   acc.amax_t = max(acc.amax_t, scan->amax_t);
@@ -924,37 +966,63 @@ struct TensorMeta {
   int eg;              // exponent of a fixed-point gradient, 0 for binary32
 };
 
-__device__ __forceinline__ void load_comp_exponents(const StepParams& p, int t, bool strict, TensorMeta& m) {
+// The exponents tensor t reads and writes in the step of phase `ph`, derived from what the
+// preceding step left in buffer ph-1; the result goes into buffer ph and buffer ph+1 is cleared
+// for the step after this one.  Every block that meets the tensor does the same and stores the
+// same values.
+__device__ __forceinline__ void step_exponents(const StepParams& p, int t, int ph, bool strict, TensorMeta& m) {
+  const int prev = ph == 0 ? 2 : ph - 1;
+  // one 32-byte load (L2: the record was written by other SMs during the preceding step)
+  const int4* rec = reinterpret_cast<const int4*>(&p.ws.state[(size_t)prev * p.ws.slab + t]);
+  const int4 r0 = __ldcg(rec), r1 = __ldcg(rec + 1);
+  m.e_in = r0.x;
+  m.e_out = r1.x ? r1.x - kOvrBias : next_exponent((unsigned)r0.z, m.ti.theta_bits, m.e_in, p.amax_mode);
   if (strict) {
-    m.ec_in = p.ws.expc_cur[t];
-    m.ec_out = p.ws.expc_next[t];
+    m.ec_in = r0.y;
+    m.ec_out = r1.y ? r1.y - kOvrBias : next_exponent_acc((unsigned)r0.w, m.ti.comp_bits, m.ec_in, m.e_out, p.amax_mode);
   } else {
     m.ec_in = m.e_in - m.ti.s;
     m.ec_out = m.e_out - m.ti.s;
   }
 }
 
-__device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const InlineArgs& a, int t, bool strict) {
+// Every block that meets a tensor derives the same exponents; the one that holds the tensor's
+// first tile records them and clears the record of the step after this one.  (This step's
+// own record was cleared a step ago; only its exponent fields are written here, the scans
+// other blocks may already have added to it stay.)
+__device__ __forceinline__ void record_exponents(const StepParams& p, int t, int ph, bool strict,
+                                                 const TensorMeta& m) {
+  const int next = ph == 2 ? 0 : ph + 1;
+  TensorState* now = &p.ws.state[(size_t)ph * p.ws.slab + t];
+  now->exp_theta = m.e_out;
+  now->exp_comp = strict ? m.ec_out : 0;
+  int4* nx = reinterpret_cast<int4*>(&p.ws.state[(size_t)next * p.ws.slab + t]);
+  nx[0] = make_int4(0, 0, 0, 0);
+  nx[1] = make_int4(0, 0, 0, 0);
+}
+
+// ti: the tensor's table entry if the caller has it already (the table never changes).
+__device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const InlineArgs& a, int t, int ph, bool strict,
+                                                bool owner, const TensorInfo* ti = nullptr) {
   TensorMeta m;
-  m.ti = p.ws.info[t];
-  m.e_in = p.ws.exp_cur[t];
-  m.e_out = p.ws.exp_next[t];
+  m.ti = ti ? *ti : p.ws.info[t];
   m.grad = p.inline_args ? a.grads[t] : p.ws.grad_ptr[t];
   m.lr = p.inline_args ? a.lrs[t] : p.ws.lr[t];
   m.eg = 0;
-  load_comp_exponents(p, t, strict, m);
+  step_exponents(p, t, ph, strict, m);
+  if (owner) record_exponents(p, t, ph, strict, m);
   return m;
 }
 
-__device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const QGradArgs& a, int t, bool strict) {
+__device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const QGradArgs& a, int t, int ph, bool strict,
+                                                bool owner, const TensorInfo* ti = nullptr) {
   TensorMeta m;
-  m.ti = p.ws.info[t];
-  m.e_in = p.ws.exp_cur[t];
-  m.e_out = p.ws.exp_next[t];
+  m.ti = ti ? *ti : p.ws.info[t];
   m.grad = p.inline_args ? a.grads[t] : static_cast<const void*>(p.ws.grad_ptr[t]);
   m.lr = p.inline_args ? a.lrs[t] : p.ws.lr[t];
   m.eg = p.inline_args ? (int)a.exp_grad[t] : p.ws.exp_grad[t];
-  load_comp_exponents(p, t, strict, m);
+  step_exponents(p, t, ph, strict, m);
+  if (owner) record_exponents(p, t, ph, strict, m);
   return m;
 }
 
@@ -976,7 +1044,6 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
       mbar_init(&sh->empty[s], (unsigned)kConsumerWarps);
     }
     sh->abort_flag = 0;
-    sh->is_last = 0;
     sh->never = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -1002,8 +1069,23 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
       ChunkRef cr = p.ws.chunks[tile0];
       ChunkRef cr1{-1, -1};
       if (n_my > 1) cr1 = p.ws.chunks[tile0 + stride];
+      const TensorInfo ti_first = p.ws.info[cr.tensor];       // the tensor table never changes either
+      // The step's phase.  The preceding step moves the word on as soon as all of its blocks
+      // have started, long before it ends, so the value read here, before the wait, is
+      // normally the right one already: the first record is fetched under it while the word
+      // is read again, and only fetched a second time if the two differ.  (The block's entry
+      // ticket, which tells the last block that all have read this word, is drawn by a
+      // consumer thread once the first tile has landed.)
+      int ph = (int)__ldcg(p.ws.phase);
       grid_dependency_wait();
-      TensorMeta meta = load_meta(p, a, cr.tensor, STRICT);
+      const int ph_now = (int)__ldcg(p.ws.phase);
+      TensorMeta meta = load_meta(p, a, cr.tensor, ph, STRICT, false, &ti_first);
+      if (ph_now != ph) {
+        ph = ph_now;
+        meta = load_meta(p, a, cr.tensor, ph, STRICT, false, &ti_first);
+      }
+      if (cr.index == 0) record_exponents(p, cr.tensor, ph, STRICT, meta);
+      TensorState* amax_now = p.ws.state + (size_t)ph * p.ws.slab;
       int issued = 0;
       // The ring: pages from `head` on are free, tiles are released in the order they were
       // issued, `oldest` is the first tile whose pages have not been taken back yet.
@@ -1014,7 +1096,7 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
         ChunkRef cr2{-1, -1};
         if (i + 2 < n_my) cr2 = p.ws.chunks[tile0 + (i + 2) * stride];
         TensorMeta meta1 = meta;
-        if (i + 1 < n_my && cr1.tensor != cr.tensor) meta1 = load_meta(p, a, cr1.tensor, STRICT);
+        if (i + 1 < n_my && cr1.tensor != cr.tensor) meta1 = load_meta(p, a, cr1.tensor, ph, STRICT, cr1.index == 0);
 
         const TensorInfo& ti = meta.ti;
         const int tbytes = ti.theta_bits >> 3, cbytes = ti.comp_bits >> 3;
@@ -1042,7 +1124,7 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
             gave_up = true;
             break;
           }
-          take_back(p, acc, &sh->scan[os], sh->desc[os].tensor);
+          take_back(p, acc, amax_now, &sh->scan[os], sh->desc[os].tensor);
           free_pages += sh->slot_pages[os];
           ++oldest;
         }
@@ -1055,6 +1137,29 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
         free_pages -= need;
         sh->slot_pages[slot] = need;
 
+        const long long first = (long long)cr.index << (13 + big);
+        const long long left = ti.numel - first;
+        const int count = left < (long long)chunk ? (int)left : chunk;
+        const int n_bulk = count & ~15;
+        // The copies go out first and the descriptor is written while they are on their way:
+        // the tile's barrier completes only when the bytes have landed AND the producer has
+        // arrived, and it arrives after the descriptor is in place.
+        unsigned char* const theta_g = static_cast<unsigned char*>(ti.theta) + first * tbytes;
+        unsigned char* const comp_g = ti.comp ? static_cast<unsigned char*>(ti.comp) + first * cbytes : nullptr;
+        const unsigned char* const grad_g = static_cast<const unsigned char*>(meta.grad) + first * gbytes;
+        if (n_bulk > 0) {
+          mbar_expect_tx(&sh->full[slot], (unsigned)(n_bulk * (tbytes + cbytes + gbytes)));
+          bulk_load(smem + page[1] * kPageBytes, theta_g, (unsigned)(n_bulk * tbytes), &sh->full[slot]);
+          if (cbytes)
+            bulk_load(smem + page[2] * kPageBytes, comp_g, (unsigned)(n_bulk * cbytes), &sh->full[slot]);
+          // Gradients are read once.  When theta and c of the whole list fit in L2, letting
+          // the gradients leave it first keeps the state resident from step to step.
+          if (p.grad_evict_first)
+            bulk_load_hint(smem + page[0] * kPageBytes, grad_g, (unsigned)(n_bulk * gbytes), &sh->full[slot],
+                           grad_policy);
+          else
+            bulk_load(smem + page[0] * kPageBytes, grad_g, (unsigned)(n_bulk * gbytes), &sh->full[slot]);
+        }
         const StepCoef coef = make_coef(ti, meta.e_in, meta.e_out, meta.ec_in, meta.ec_out, meta.lr, GB, meta.eg,
                                         STRICT ? 1 : 0);
         // fixed-point gradients: the exact-fp32 path multiplies the mantissa by scale * 2^eg,
@@ -1066,17 +1171,13 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
           scale_ok = ex != 0 && ex + meta.eg >= 1 && ex + meta.eg <= 254;
           if (scale_ok) scale_hot = __int_as_float(__float_as_int(coef.scale) + (meta.eg << 23));
         }
-        const long long first = (long long)cr.index << (13 + big);
-        const long long left = ti.numel - first;
-        const int count = left < (long long)chunk ? (int)left : chunk;
-        const int n_bulk = count & ~15;
         TileDesc& td = sh->desc[slot];
         td.scale = scale_hot;
         td.pow2s_neg = -pow2_float(coef.s);
         td.inv2s = pow2_float(-coef.s);
         td.pow2dc = pow2_float(-coef.delta_c);
-        td.theta = static_cast<unsigned char*>(ti.theta) + first * tbytes;
-        td.comp = ti.comp ? static_cast<unsigned char*>(ti.comp) + first * cbytes : nullptr;
+        td.theta = theta_g;
+        td.comp = comp_g;
         td.tensor = cr.tensor;
         td.n_bulk = n_bulk;
         td.count = count;
@@ -1087,22 +1188,8 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
                    (page[1] << kFlagThetaPageShift) |
                    (page[2] << kFlagCompPageShift) | (page[0] << kFlagGradPageShift);
         td.coef = coef;
-        td.grad = static_cast<const unsigned char*>(meta.grad) + first * gbytes;
-        if (n_bulk > 0) {
-          mbar_arrive_expect_tx(&sh->full[slot], (unsigned)(n_bulk * (tbytes + cbytes + gbytes)));
-          bulk_load(smem + page[1] * kPageBytes, td.theta, (unsigned)(n_bulk * tbytes), &sh->full[slot]);
-          if (cbytes)
-            bulk_load(smem + page[2] * kPageBytes, td.comp, (unsigned)(n_bulk * cbytes), &sh->full[slot]);
-          // Gradients are read once.  When theta and c of the whole list fit in L2, letting
-          // the gradients leave it first keeps the state resident from step to step.
-          if (p.grad_evict_first)
-            bulk_load_hint(smem + page[0] * kPageBytes, td.grad, (unsigned)(n_bulk * gbytes), &sh->full[slot],
-                           grad_policy);
-          else
-            bulk_load(smem + page[0] * kPageBytes, td.grad, (unsigned)(n_bulk * gbytes), &sh->full[slot]);
-        } else {
-          mbar_arrive(&sh->full[slot]);
-        }
+        td.grad = grad_g;
+        mbar_arrive(&sh->full[slot]);
         issued = i + 1;
         cr = cr1;
         cr1 = cr2;
@@ -1113,11 +1200,11 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
       for (int i = oldest; i < issued; ++i) {
         const int os = i % kSlots;
         if (mbar_wait(&sh->empty[os], (unsigned)(i / kSlots) & 1u, &sh->abort_flag))
-          take_back(p, acc, &sh->scan[os], sh->desc[os].tensor);
+          take_back(p, acc, amax_now, &sh->scan[os], sh->desc[os].tensor);
         else
           mbar_wait(&sh->full[os], (unsigned)(i / kSlots) & 1u, &sh->never);
       }
-      publish(p, acc);
+      publish(p, acc, amax_now);
     } else {
       grid_dependency_wait();
     }
@@ -1127,6 +1214,12 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
     const int ctid = threadIdx.x;
     const int stride = (int)gridDim.x;
     const int n_my = (p.tile_count - (int)blockIdx.x + stride - 1) / stride;
+    // Entry ticket (thread 0).  It is drawn after the block's first tile has landed, i.e. after
+    // the producer has read the phase word (it arrives on the tile's barrier later than that
+    // read returned, and the wait above has seen the arrival); the block that draws the last
+    // ticket therefore knows that every block of the step has read the word, and only then
+    // moves it on for the next step.  The answer is looked at when the block's tiles are done.
+    unsigned int ticket = 0u, ph0 = 0u;
     for (int i = 0; i < n_my; ++i) {
       const int stage = i % kSlots, use = i / kSlots;
       if (!mbar_wait(&sh->full[stage], (unsigned)use & 1u, &sh->abort_flag)) {
@@ -1135,6 +1228,10 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
           atomicCAS(p.ws.error, 0u, (unsigned)kErrFullWait);
         }
         break;
+      }
+      if (i == 0 && threadIdx.x == 0 && p.advance) {
+        ph0 = __ldcg(p.ws.phase);
+        ticket = atomicAdd(p.ws.phase + 1 + (ph0 >> 8), 1u) + 1u;
       }
       const TileDesc* td = &sh->desc[stage];
       TileScan* scan = &sh->scan[stage];
@@ -1161,39 +1258,14 @@ __device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->empty[stage]);
     }
-  }
-
-  // ---------------------------------------------------------------------- block done
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    const unsigned int done = atomicAdd(p.ws.ticket, 1u);
-    sh->is_last = (done == gridDim.x - 1u);
-  }
-  __syncthreads();
-  if (!sh->is_last) return;
-
-  // Last block to finish: every other block has published its scans and has long since
-  // read the exponents, so they can be rotated here.  No block ever waits for another.
-  __threadfence();
-  for (int i = p.tensor_begin + threadIdx.x; i < p.tensor_begin + p.tensor_count; i += kBlockThreads) {
-    const unsigned int at = __ldcg(&p.ws.amax_acc[i]);
-    const unsigned int ac = __ldcg(&p.ws.amax_acc[p.n_tensors + i]);
-    const int eo = p.ws.exp_next[i];
-    const int en = next_exponent(at, p.ws.info[i].theta_bits, eo, p.amax_mode);
-    p.ws.exp_cur[i] = eo;
-    p.ws.exp_next[i] = en;
-    if constexpr (STRICT) {
-      const int eco = p.ws.expc_next[i];
-      p.ws.expc_cur[i] = eco;
-      p.ws.expc_next[i] = next_exponent_acc(ac, p.ws.info[i].comp_bits, eco, en, p.amax_mode);
+    if (threadIdx.x == 0 && ticket == gridDim.x) {
+      p.ws.phase[1] = 0u;
+      p.ws.phase[0] = ph0 == 2u ? 0u : ph0 + 1u;
     }
-    p.ws.amax_last[i] = at;
-    p.ws.amax_last[p.n_tensors + i] = ac;
-    p.ws.amax_acc[i] = 0u;
-    p.ws.amax_acc[p.n_tensors + i] = 0u;
   }
-  if (threadIdx.x == 0) *p.ws.ticket = 0u;
+
+  // Nothing follows: the step is complete when every block's producer has published its
+  // scans; the exponents they imply are worked out by the blocks of the next step.
 }
 
 __global__ void __launch_bounds__(kBlockThreads, 1)
@@ -1232,14 +1304,17 @@ __global__ void ksgd_upload_ints_kernel(const __grid_constant__ ExponentBatch b,
   for (int i = threadIdx.x; i < count; i += blockDim.x) dst[first + i] = b.exp_next[i];
 }
 
-// Caller-chosen exponents for the coming step, limited to kMaxDelta around the current one.
+// Caller-chosen exponents for the coming step, limited to kMaxDelta around the current one:
+// written as overrides into the record the coming step reads.
 __global__ void ksgd_set_exponents_kernel(const __grid_constant__ ExponentBatch b, int first,
-                                          int count, const int* exp_cur, int* exp_next) {
+                                          int count, int slab, const unsigned int* phase, TensorState* state) {
+  const int ph = (int)phase[0], prev = ph == 0 ? 2 : ph - 1;
   for (int i = threadIdx.x; i < count; i += blockDim.x) {
-    const int cur = exp_cur[first + i];
+    TensorState* rec = &state[(size_t)prev * slab + first + i];
+    const int cur = rec->exp_theta;
     int e = max(kExpMin, min(kExpMax, b.exp_next[i]));
     e = max(cur - kMaxDelta, min(cur + kMaxDelta, e));
-    exp_next[first + i] = e;
+    rec->ovr_theta = e + kOvrBias;
   }
 }
 

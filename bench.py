@@ -134,6 +134,8 @@ def parse_args():
                     help="skip the per-size-bucket timing of c5_sweep")
     ap.add_argument("--no-extra-workloads", action="store_true",
                     help="skip the c3_resnet50 / c4_alexnet legs that the default run adds to its line")
+    ap.add_argument("--no-convert", action="store_true",
+                    help="skip the fp32 <-> fixed-point conversion leg that the default run adds to its line")
     ap.add_argument("--sustained-s", type=float, default=0.35,
                     help="length of the sustained leg (the same steps repeated for about this long, with the "
                          "clocks sampled inside it); 0 skips it")
@@ -289,6 +291,56 @@ def roofline_of(wl, bytes_per_step, ms_step, peak, peak_src, kernel, plain):
             r["dram_gbs"] = traffic / (ms_step * 1e-3) / 1e9
             r["frac_dram"] = r["dram_gbs"] / peak
     return r
+
+
+def convert_leg(torch, B, peak, numel=64 * 1024 * 1024, iters=10):
+    """fp32 <-> dynamic fixed-point on one tensor of `numel` elements (256 MB of binary32,
+    twice the L2): kahan_sgd_import_dev (max scan, exponent chosen on the device, quantization:
+    the source is read twice) and kahan_sgd_export, each timed over `iters` back-to-back calls
+    after two warm-up calls.  Algorithmic bytes per element: import 4 + 4 + m/8 + n/8, export
+    m/8 + n/8 + 4."""
+    st = torch.cuda.current_stream()
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    src = torch.randn(numel, generator=gen, device="cuda", dtype=torch.float32) * 0.05
+    dst = torch.empty(numel, dtype=torch.float32, device="cuda")
+    scratch = torch.zeros(4, dtype=torch.int32, device="cuda")
+    exp_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = []
+    for tb, cb, what in ((8, 0, "int8 gradients"), (16, 0, "int16 gradients"), (16, 8, "int16 theta + int8 c"),
+                         (8, 8, "int8 theta + int8 c"), (16, 16, "int16 theta + int16 c")):
+        th = torch.empty(numel * (tb // 8), dtype=torch.uint8, device="cuda")
+        c = torch.empty(numel * (cb // 8), dtype=torch.uint8, device="cuda") if cb else None
+        torch.cuda.synchronize()
+
+        def imp():
+            B.kahan_sgd_import_dev(src.data_ptr(), th.data_ptr(), c.data_ptr() if cb else None, numel, tb, cb, 0,
+                                   exp_dev.data_ptr(), scratch.data_ptr(), st.cuda_stream)
+
+        def exp():
+            B.kahan_sgd_export(th.data_ptr(), c.data_ptr() if cb else None, dst.data_ptr(), numel, tb, cb, 0,
+                               e_used, st.cuda_stream)
+        row = {"format": what, "elements": numel}
+        imp()
+        torch.cuda.synchronize()
+        e_used = int(exp_dev.item())
+        for name, fn, nbytes in (("import", imp, 8 + (tb + cb) // 8), ("export", exp, 4 + (tb + cb) // 8)):
+            fn()
+            fn()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(st)
+            for _ in range(iters):
+                fn()
+            e1.record(st)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / iters
+            gbs = numel * nbytes / (ms * 1e-3) / 1e9
+            row[name] = {"ms": round(ms, 4), "bytes_per_element": nbytes, "gbs": round(gbs, 1),
+                         "frac": round(gbs / peak, 3), "elements_per_s": numel / (ms * 1e-3)}
+        row["exponent"] = e_used
+        out.append(row)
+        del th, c
+    return out
 
 
 def extra_workload(torch, B, W, name, args, peak, peak_src, barrier, gpu_index):
@@ -477,6 +529,8 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.empty_cache()
         line["workloads"] = [extra_workload(torch, B, W, name, args, peak, peak_src, barrier, local_rank)
                              for name in ("c3_resnet50", "c4_alexnet")]
+        if not args.no_convert:
+            line["convert"] = convert_leg(torch, B, peak)
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.barrier()

@@ -140,6 +140,16 @@ int kahan_sgd_step_qgrad(ksgd_handle* h, const void* const* grads, int32_t grad_
                          const float* lrs);
 
 /*
+ * The same with the gradients' exponents in device memory: exp_grad_dev is a device array of
+ * n_tensors int32 (4-byte aligned) that the step reads when it runs, so that exponents chosen
+ * on the device by kahan_sgd_import_dev (Section 5: the exponent from a max scan) reach the
+ * step without a host round trip; values outside [-64, 64] are clamped into the range.  The
+ * array must stay valid and unchanged until the step has run.
+ */
+int kahan_sgd_step_qgrad_dev(ksgd_handle* h, const void* const* grads, int32_t grad_bits,
+                             const int32_t* exp_grad_dev, const float* lrs);
+
+/*
  * The same step for callers whose tensors live in host memory: copies each tensor's
  * theta, comp and gradient from host to the device buffers named in the descs (and to
  * grad_staging), runs the step, copies theta and comp back and waits.  theta_host /
@@ -380,13 +390,26 @@ int kahan_sgd_adam_selfcheck(uint64_t* div_mismatches, uint64_t* sqrt_mismatches
  * imported weight keeps m+n-2-k bits; NaN -> 0, +-Inf -> +-QMAX.  exp_theta: the exponent
  * to use, in [-64, 64], or KSGD_EXP_AUTO for the smallest exponent whose grid holds the
  * largest finite |x| (0 for an all-zero tensor); with KSGD_EXP_AUTO the call runs a max
- * scan into scratch (device, at least 4 bytes, 4-byte aligned) and waits for it.
- * *exp_theta_out (host, may be NULL) receives the exponent used.
+ * scan whose last block picks the exponent on the device, then the quantization, which reads
+ * it from device memory, and waits only to hand the exponent back; scratch: device, at least
+ * 16 bytes, 4-byte aligned (cleared by the call).  *exp_theta_out (host, may be NULL)
+ * receives the exponent used.  With a given exponent the call only enqueues.
+ * 16-byte aligned src and 4-byte (8-bit) or 8-byte (16-bit) aligned outputs take the fast path
+ * (four elements per access); anything else is converted element by element.
+ *
+ * kahan_sgd_import_dev: the KSGD_EXP_AUTO form without any host synchronisation.  The
+ * exponent is left in *exp_theta_dev (device int32, 4-byte aligned) for whoever needs it on
+ * the device (kahan_sgd_step_qgrad_dev reads gradient exponents from such an array).
+ * scratch: device, at least 8 bytes, 4-byte aligned, zero on the first call (every call
+ * leaves it zero again); calls that share a scratch must run one after the other.
  */
 #define KSGD_EXP_AUTO INT32_MIN
 int kahan_sgd_import(const float* src, void* theta, void* comp, int64_t numel, int32_t theta_bits,
                      int32_t comp_bits, int32_t overlap_k, int32_t exp_theta, int32_t* exp_theta_out,
                      void* scratch, void* cuda_stream);
+int kahan_sgd_import_dev(const float* src, void* theta, void* comp, int64_t numel, int32_t theta_bits,
+                         int32_t comp_bits, int32_t overlap_k, int32_t* exp_theta_dev, void* scratch,
+                         void* cuda_stream);
 
 /*
  * Dynamic fixed-point -> fp32: dst[i] = fl32(Q_theta*2^e + Q_c*2^(e-s)), the exact value of

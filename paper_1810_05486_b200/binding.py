@@ -29,6 +29,7 @@ KSGD_ERR_DEVICE = -11
 
 EXPORTS = (
     "kahan_sgd_workspace_bytes", "kahan_sgd_workspace_error_offset", "kahan_sgd_init", "kahan_sgd_step", "kahan_sgd_step_qgrad",
+    "kahan_sgd_step_qgrad_dev", "kahan_sgd_import_dev",
     "kahan_sgd_step_host", "kahan_sgd_strict_workspace_bytes", "kahan_sgd_strict_init",
     "kahan_sgd_strict_exponents",
     "kahan_sgd_amax", "kahan_sgd_set_exponents", "kahan_sgd_step_static", "kahan_sgd_destroy",
@@ -141,6 +142,12 @@ def _load() -> ctypes.CDLL:
     lib.kahan_sgd_adam_destroy.argtypes = [ctypes.c_void_p]
     lib.kahan_sgd_adam_selfcheck.restype = ctypes.c_int
     lib.kahan_sgd_adam_selfcheck.argtypes = [P(ctypes.c_uint64), P(ctypes.c_uint64), ctypes.c_void_p]
+    lib.kahan_sgd_step_qgrad_dev.restype = ctypes.c_int
+    lib.kahan_sgd_step_qgrad_dev.argtypes = [ctypes.c_void_p, P(ctypes.c_void_p), ctypes.c_int32,
+                                             ctypes.c_void_p, P(ctypes.c_float)]
+    lib.kahan_sgd_import_dev.restype = ctypes.c_int
+    lib.kahan_sgd_import_dev.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int64] + [ctypes.c_int32] * 3 + \
+        [ctypes.c_void_p] * 3
     lib.kahan_sgd_import.restype = ctypes.c_int
     lib.kahan_sgd_import.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int64] + [ctypes.c_int32] * 4 + \
         [P(ctypes.c_int32), ctypes.c_void_p, ctypes.c_void_p]
@@ -254,6 +261,13 @@ def kahan_sgd_step_qgrad(h, grads, grad_bits: int, exp_grad, lrs) -> None:
     e = exp_grad if isinstance(exp_grad, ctypes.Array) else (ctypes.c_int32 * len(exp_grad))(*exp_grad)
     l = lrs if isinstance(lrs, ctypes.Array) else _float_array(lrs)
     _check(lib.kahan_sgd_step_qgrad(h, g, grad_bits, e, l))
+
+
+def kahan_sgd_step_qgrad_dev(h, grads, grad_bits: int, exp_grad_dev: int, lrs) -> None:
+    """As kahan_sgd_step_qgrad, the exponents in a device int32 array (address exp_grad_dev)."""
+    g = grads if isinstance(grads, ctypes.Array) else _ptr_array(grads)
+    l = lrs if isinstance(lrs, ctypes.Array) else _float_array(lrs)
+    _check(lib.kahan_sgd_step_qgrad_dev(h, g, grad_bits, ctypes.c_void_p(exp_grad_dev), l))
 
 
 def kahan_sgd_step_host(h, theta_host, comp_host, grads_host, lrs, grad_staging: int,
@@ -432,6 +446,15 @@ def kahan_sgd_import(src: int, theta: int, comp, numel: int, theta_bits: int, co
                                 numel, theta_bits, comp_bits, overlap_k, exp_theta, ctypes.byref(e),
                                 ctypes.c_void_p(scratch or None), ctypes.c_void_p(stream)))
     return int(e.value)
+
+
+def kahan_sgd_import_dev(src: int, theta: int, comp, numel: int, theta_bits: int, comp_bits: int,
+                         overlap_k: int, exp_theta_dev: int, scratch: int, stream: int = 0) -> None:
+    """fp32 -> dynamic fixed-point without a host round trip: max scan, exponent chosen on the
+    device and left in the device int32 at exp_theta_dev, quantization.  Enqueues only."""
+    _check(lib.kahan_sgd_import_dev(ctypes.c_void_p(src), ctypes.c_void_p(theta), ctypes.c_void_p(comp or None),
+                                    numel, theta_bits, comp_bits, overlap_k, ctypes.c_void_p(exp_theta_dev),
+                                    ctypes.c_void_p(scratch), ctypes.c_void_p(stream)))
 
 
 def kahan_sgd_export(theta: int, comp, dst: int, numel: int, theta_bits: int, comp_bits: int,

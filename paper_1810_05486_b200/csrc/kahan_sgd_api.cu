@@ -302,6 +302,7 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   h->params.tensor_begin = 0;
   h->params.tensor_count = n_tensors;
   h->params.advance = 1;
+  h->params.exp_grad_dev = nullptr;
 
   // Persistent grid: one block per SM (fewer if the list has fewer tiles).
   int dev = 0, sms = 0, l2_bytes = 0;
@@ -454,14 +455,17 @@ static int launch_step(ksgd_handle* h, const float* const* grads, const float* l
   return KSGD_OK;
 }
 
-int kahan_sgd_step_qgrad(ksgd_handle* h, const void* const* grads, int32_t grad_bits, const int32_t* exp_grad,
-                         const float* lrs) {
-  if (!h || !grads || !exp_grad || !lrs) return KSGD_ERR_NULL;
+// exp_grad: host array (copied into the launch), or nullptr with exp_grad_dev: a device array
+// the kernel reads the exponents from.
+static int step_qgrad_common(ksgd_handle* h, const void* const* grads, int32_t grad_bits, const int32_t* exp_grad,
+                             const int32_t* exp_grad_dev, const float* lrs) {
+  if (!h || !grads || (!exp_grad && !exp_grad_dev) || !lrs) return KSGD_ERR_NULL;
   if (grad_bits != 8 && grad_bits != 16) return KSGD_ERR_BITS;
+  if (reinterpret_cast<uintptr_t>(exp_grad_dev) % 4) return KSGD_ERR_ALIGN;
   for (int32_t i = 0; i < h->n; ++i) {
     if (!grads[i]) return KSGD_ERR_NULL;
     if (reinterpret_cast<uintptr_t>(grads[i]) % 16) return KSGD_ERR_ALIGN;
-    if (exp_grad[i] < kExpMin || exp_grad[i] > kExpMax) return KSGD_ERR_EXP_RANGE;
+    if (exp_grad && (exp_grad[i] < kExpMin || exp_grad[i] > kExpMax)) return KSGD_ERR_EXP_RANGE;
     if (!std::isfinite(lrs[i]) || !(lrs[i] > 0.0f)) return KSGD_ERR_LR;
   }
   QGradArgs args{};
@@ -469,7 +473,7 @@ int kahan_sgd_step_qgrad(ksgd_handle* h, const void* const* grads, int32_t grad_
     for (int32_t i = 0; i < h->n; ++i) {
       args.grads[i] = grads[i];
       args.lrs[i] = lrs[i];
-      args.exp_grad[i] = (signed char)exp_grad[i];
+      args.exp_grad[i] = exp_grad ? (signed char)exp_grad[i] : 0;
     }
   } else {
     UploadBatch* ub = new (std::nothrow) UploadBatch;
@@ -480,24 +484,41 @@ int kahan_sgd_step_qgrad(ksgd_handle* h, const void* const* grads, int32_t grad_
       for (int i = 0; i < count; ++i) {
         ub->grads[i] = static_cast<const float*>(grads[first + i]);   // only the address travels
         ub->lrs[i] = lrs[first + i];
-        eb->exp_next[i] = exp_grad[first + i];
+        eb->exp_next[i] = exp_grad ? exp_grad[first + i] : 0;
       }
       ksgd_upload_args_kernel<<<1, 256, 0, h->stream>>>(*ub, first, count, h->params.ws.grad_ptr,
                                                         h->params.ws.lr);
-      ksgd_upload_ints_kernel<<<1, 256, 0, h->stream>>>(*eb, first, count, h->params.ws.exp_grad);
-      g_launches.fetch_add(2, std::memory_order_relaxed);
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+      if (exp_grad) {
+        ksgd_upload_ints_kernel<<<1, 256, 0, h->stream>>>(*eb, first, count, h->params.ws.exp_grad);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+      }
     }
     delete ub;
     delete eb;
     KSGD_CUDA(cudaGetLastError());
   }
+  StepParams p = h->params;
+  p.exp_grad_dev = exp_grad_dev;
   const unsigned grid = (unsigned)h->grid;
   auto kernel = h->strict ? (grad_bits == 8 ? ksgd_strict_step_qgrad_kernel<8> : ksgd_strict_step_qgrad_kernel<16>)
                           : (grad_bits == 8 ? ksgd_step_qgrad_kernel<8> : ksgd_step_qgrad_kernel<16>);
-  KSGD_CUDA(launch_step_kernel(kernel, grid, kBlockThreads, kSharedBytes, h->stream, h->params, args));
+  KSGD_CUDA(launch_step_kernel(kernel, grid, kBlockThreads, kSharedBytes, h->stream, p, args));
   g_launches.fetch_add(1, std::memory_order_relaxed);
   KSGD_CUDA(cudaGetLastError());
   return KSGD_OK;
+}
+
+int kahan_sgd_step_qgrad(ksgd_handle* h, const void* const* grads, int32_t grad_bits, const int32_t* exp_grad,
+                         const float* lrs) {
+  if (!exp_grad) return KSGD_ERR_NULL;
+  return step_qgrad_common(h, grads, grad_bits, exp_grad, nullptr, lrs);
+}
+
+int kahan_sgd_step_qgrad_dev(ksgd_handle* h, const void* const* grads, int32_t grad_bits,
+                             const int32_t* exp_grad_dev, const float* lrs) {
+  if (!exp_grad_dev) return KSGD_ERR_NULL;
+  return step_qgrad_common(h, grads, grad_bits, nullptr, exp_grad_dev, lrs);
 }
 
 int kahan_sgd_step(ksgd_handle* h, const float* const* grads, const float* lrs) {
@@ -761,6 +782,7 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   params.grad_evict_first = state_bytes <= 0.8 * (double)sd.l2_bytes ? 1 : 0;
   params.chunk8 = kChunk;
   params.advance = 1;
+  params.exp_grad_dev = nullptr;
 
   InlineArgs inl;
   for (int32_t i = 0; i < n_tensors; ++i) { inl.grads[i] = grads[i]; inl.lrs[i] = lrs[i]; }
@@ -1309,23 +1331,50 @@ int check_format(int32_t theta_bits, int32_t comp_bits, int32_t overlap_k) {
   return KSGD_OK;
 }
 
+// Grid of the conversion kernels: blocks of 256 threads, four elements per thread and access;
+// at most sixteen blocks per SM (two waves of resident blocks), never more than the work.
 int convert_grid(int64_t numel) {
-  const int64_t blocks = (numel + convert::kThreads - 1) / convert::kThreads;
-  return (int)(blocks < 148 * 16 ? blocks : 148 * 16);
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
+    else sms = 148;
+  }
+  const int64_t blocks = (numel / 4 + convert::kThreads - 1) / convert::kThreads + 1;
+  return (int)(blocks < (int64_t)sms * 16 ? blocks : (int64_t)sms * 16);
 }
 
-template <typename T, typename C, bool HC>
-void launch_quantize(const float* src, void* theta, void* comp, int64_t numel, int e, int s, int tb, int cb,
-                     cudaStream_t st) {
-  convert::quantize_kernel<T, C, HC><<<convert_grid(numel), convert::kThreads, 0, st>>>(
-      src, static_cast<T*>(theta), static_cast<C*>(comp), numel, e, s, tb, cb);
+template <int TB>
+void launch_quantize_tb(int cb, const float* src, void* theta, void* comp, int64_t numel, const int* exp_dev,
+                        int e, int s, cudaStream_t st) {
+  const int grid = convert_grid(numel);
+  if (cb == 8) convert::quantize_kernel<TB, 8><<<grid, convert::kThreads, 0, st>>>(src, theta, comp, numel, exp_dev, e, s);
+  else if (cb == 16) convert::quantize_kernel<TB, 16><<<grid, convert::kThreads, 0, st>>>(src, theta, comp, numel, exp_dev, e, s);
+  else convert::quantize_kernel<TB, 0><<<grid, convert::kThreads, 0, st>>>(src, theta, comp, numel, exp_dev, e, s);
 }
 
-template <typename T, typename C, bool HC>
-void launch_dequantize(const void* theta, const void* comp, float* dst, int64_t numel, int e, int s,
-                       cudaStream_t st) {
-  convert::dequantize_kernel<T, C, HC><<<convert_grid(numel), convert::kThreads, 0, st>>>(
-      static_cast<const T*>(theta), static_cast<const C*>(comp), dst, numel, e, s);
+template <int TB>
+void launch_dequantize_tb(int cb, const void* theta, const void* comp, float* dst, int64_t numel, int e, int s,
+                          cudaStream_t st) {
+  const int grid = convert_grid(numel);
+  if (cb == 8) convert::dequantize_kernel<TB, 8><<<grid, convert::kThreads, 0, st>>>(theta, comp, dst, numel, e, s);
+  else if (cb == 16) convert::dequantize_kernel<TB, 16><<<grid, convert::kThreads, 0, st>>>(theta, comp, dst, numel, e, s);
+  else convert::dequantize_kernel<TB, 0><<<grid, convert::kThreads, 0, st>>>(theta, comp, dst, numel, e, s);
+}
+
+// Max scan with the exponent left at exp_dev (device), then the quantization reading it
+// from there.  Enqueues two kernels; nothing waits.
+int import_auto(const float* src, void* theta, void* comp, int64_t numel, int32_t theta_bits, int32_t comp_bits,
+                int32_t overlap_k, int32_t* exp_dev, void* scratch, cudaStream_t st) {
+  convert::absmax_fit_kernel<<<convert_grid(numel), convert::kThreads, 0, st>>>(
+      src, numel, theta_bits, static_cast<convert::ScanScratch*>(scratch), exp_dev);
+  const int s = comp_bits ? comp_bits - 1 - overlap_k : 0;
+  if (theta_bits == 8) launch_quantize_tb<8>(comp_bits, src, theta, comp, numel, exp_dev, 0, s, st);
+  else launch_quantize_tb<16>(comp_bits, src, theta, comp, numel, exp_dev, 0, s, st);
+  g_launches.fetch_add(2, std::memory_order_relaxed);
+  KSGD_CUDA(cudaGetLastError());
+  return KSGD_OK;
 }
 
 }  // namespace
@@ -1342,42 +1391,38 @@ int kahan_sgd_import(const float* src, void* theta, void* comp, int64_t numel, i
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   int e = exp_theta;
   if (exp_theta == KSGD_EXP_AUTO) {
-    // max scan, then the smallest exponent whose grid holds the maximum
+    // scan and quantization run back to back on the device; the host only waits to hand the
+    // exponent back
     if (!scratch) return KSGD_ERR_NULL;
     if (reinterpret_cast<uintptr_t>(scratch) % 4) return KSGD_ERR_ALIGN;
-    KSGD_CUDA(cudaMemsetAsync(scratch, 0, 4, st));
-    convert::absmax_kernel<<<convert_grid(numel), convert::kThreads, 0, st>>>(
-        src, numel, static_cast<unsigned int*>(scratch));
+    KSGD_CUDA(cudaMemsetAsync(scratch, 0, 16, st));
+    int32_t* exp_dev = static_cast<int32_t*>(scratch) + 2;
+    const int r = import_auto(src, theta, comp, numel, theta_bits, comp_bits, overlap_k, exp_dev, scratch, st);
+    if (r != KSGD_OK) return r;
+    KSGD_CUDA(cudaMemcpyAsync(&e, exp_dev, 4, cudaMemcpyDeviceToHost, st));
+    KSGD_CUDA(cudaStreamSynchronize(st));
+  } else {
+    if (exp_theta < kExpMin || exp_theta > kExpMax) return KSGD_ERR_EXP_RANGE;
+    const int s = comp_bits ? comp_bits - 1 - overlap_k : 0;
+    if (theta_bits == 8) launch_quantize_tb<8>(comp_bits, src, theta, comp, numel, nullptr, e, s, st);
+    else launch_quantize_tb<16>(comp_bits, src, theta, comp, numel, nullptr, e, s, st);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     KSGD_CUDA(cudaGetLastError());
-    unsigned int bits = 0;
-    KSGD_CUDA(cudaMemcpyAsync(&bits, scratch, 4, cudaMemcpyDeviceToHost, st));
-    KSGD_CUDA(cudaStreamSynchronize(st));
-    float amax;
-    std::memcpy(&amax, &bits, 4);
-    e = 0;
-    if (amax > 0.0f) {
-      const double q = (double)((1 << (theta_bits - 1)) - 1);
-      e = kExpMin;
-      while (e < kExpMax && (double)amax > std::ldexp(q, e)) ++e;
-    }
-  } else if (exp_theta < kExpMin || exp_theta > kExpMax) {
-    return KSGD_ERR_EXP_RANGE;
   }
-  const int s = comp_bits ? comp_bits - 1 - overlap_k : 0;
-  if (theta_bits == 8) {
-    if (comp_bits == 8) launch_quantize<signed char, signed char, true>(src, theta, comp, numel, e, s, 8, 8, st);
-    else if (comp_bits == 16) launch_quantize<signed char, short, true>(src, theta, comp, numel, e, s, 8, 16, st);
-    else launch_quantize<signed char, signed char, false>(src, theta, comp, numel, e, s, 8, 0, st);
-  } else {
-    if (comp_bits == 8) launch_quantize<short, signed char, true>(src, theta, comp, numel, e, s, 16, 8, st);
-    else if (comp_bits == 16) launch_quantize<short, short, true>(src, theta, comp, numel, e, s, 16, 16, st);
-    else launch_quantize<short, signed char, false>(src, theta, comp, numel, e, s, 16, 0, st);
-  }
-  g_launches.fetch_add(1, std::memory_order_relaxed);
-  KSGD_CUDA(cudaGetLastError());
   if (exp_theta_out) *exp_theta_out = e;
   return KSGD_OK;
+}
+
+int kahan_sgd_import_dev(const float* src, void* theta, void* comp, int64_t numel, int32_t theta_bits,
+                         int32_t comp_bits, int32_t overlap_k, int32_t* exp_theta_dev, void* scratch,
+                         void* cuda_stream) {
+  const int f = check_format(theta_bits, comp_bits, overlap_k);
+  if (f != KSGD_OK) return f;
+  if (!src || !theta || (comp_bits != 0) != (comp != nullptr) || !exp_theta_dev || !scratch) return KSGD_ERR_NULL;
+  if (numel <= 0) return KSGD_ERR_NUMEL;
+  if (reinterpret_cast<uintptr_t>(scratch) % 4 || reinterpret_cast<uintptr_t>(exp_theta_dev) % 4) return KSGD_ERR_ALIGN;
+  return import_auto(src, theta, comp, numel, theta_bits, comp_bits, overlap_k, exp_theta_dev, scratch,
+                     static_cast<cudaStream_t>(cuda_stream));
 }
 
 int kahan_sgd_export(const void* theta, const void* comp, float* dst, int64_t numel, int32_t theta_bits,
@@ -1389,15 +1434,8 @@ int kahan_sgd_export(const void* theta, const void* comp, float* dst, int64_t nu
   if (exp_theta < kExpMin || exp_theta > kExpMax) return KSGD_ERR_EXP_RANGE;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int s = comp_bits ? comp_bits - 1 - overlap_k : 0, e = exp_theta;
-  if (theta_bits == 8) {
-    if (comp_bits == 8) launch_dequantize<signed char, signed char, true>(theta, comp, dst, numel, e, s, st);
-    else if (comp_bits == 16) launch_dequantize<signed char, short, true>(theta, comp, dst, numel, e, s, st);
-    else launch_dequantize<signed char, signed char, false>(theta, comp, dst, numel, e, s, st);
-  } else {
-    if (comp_bits == 8) launch_dequantize<short, signed char, true>(theta, comp, dst, numel, e, s, st);
-    else if (comp_bits == 16) launch_dequantize<short, short, true>(theta, comp, dst, numel, e, s, st);
-    else launch_dequantize<short, signed char, false>(theta, comp, dst, numel, e, s, st);
-  }
+  if (theta_bits == 8) launch_dequantize_tb<8>(comp_bits, theta, comp, dst, numel, e, s, st);
+  else launch_dequantize_tb<16>(comp_bits, theta, comp, dst, numel, e, s, st);
   g_launches.fetch_add(1, std::memory_order_relaxed);
   KSGD_CUDA(cudaGetLastError());
   return KSGD_OK;

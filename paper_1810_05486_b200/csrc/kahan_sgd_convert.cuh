@@ -1,8 +1,14 @@
 // fp32 <-> dynamic fixed-point conversion kernels (Section 1 of arXiv 1810.05486: uniform
 // linear quantization with one shared exponent per tensor; Section 5: the exponent comes
-// from a scan of the maximum).  Utilities around the update, used when a model enters or
-// leaves the fixed-point format, not per step: plain grid-stride kernels, coalesced accesses.  All scalings are by powers of two, so the
-// double arithmetic below is exact and the only roundings are the ones the definition names.
+// from a scan of the maximum).  Used when a model enters or leaves the fixed-point format,
+// and once per step and gradient tensor when the gradients are fixed-point tensors too.
+//
+// Import is two passes over the source, both bound by HBM traffic: a max scan (16-byte
+// loads) whose last block picks the exponent on the device and leaves it in device memory,
+// and the quantization, which reads that exponent from device memory (no host round trip
+// in between) and writes theta and c with 4 elements per thread and access.  All scalings
+// are by powers of two and every intermediate is exactly representable in binary32, so the
+// only roundings are the ones the definition names.
 #pragma once
 
 #include <cstdint>
@@ -12,60 +18,220 @@ namespace ksgd {
 namespace convert {
 
 constexpr int kThreads = 256;
+constexpr int kExpLo = -64, kExpHi = 64;
 
-// max |x| over the finite elements, as the bit pattern of a non-negative float (ordered
-// like the values), accumulated with atomicMax into *out (cleared by the caller).
-__global__ void __launch_bounds__(kThreads) absmax_kernel(const float* __restrict__ x, long long n,
-                                                          unsigned int* out) {
+// Device scratch of the scan: the running maximum (bit pattern of a non-negative float,
+// ordered like the values) and the count of blocks that have finished.  Both are zero
+// between calls: the caller clears them once, the last block of every scan clears them again.
+struct ScanScratch {
+  unsigned int amax_bits;
+  unsigned int done;
+};
+
+// Smallest exponent in [-64, 64] whose b-bit grid holds amax (0 for an all-zero tensor).
+__host__ __device__ inline int fit_exponent(float amax, int bits) {
+  if (!(amax > 0.0f)) return 0;
+  const double q = (double)((1 << (bits - 1)) - 1);
+  int e = kExpLo;
+  while (e < kExpHi && (double)amax > ldexp(q, e)) ++e;
+  return e;
+}
+
+__device__ __forceinline__ unsigned int finite_abs_bits(float x) {
+  const unsigned int b = __float_as_uint(x) & 0x7fffffffu;
+  return b < 0x7f800000u ? b : 0u;
+}
+
+// max |x| over the finite elements; the last block to finish turns it into the exponent and
+// stores it at *exp_out (device memory).  x 16-byte aligned: float4 loads; else scalar.
+// (Ordinary loads: a source that fits the L2 is then still there for the quantization.)
+__global__ void __launch_bounds__(kThreads) absmax_fit_kernel(const float* __restrict__ x, long long n, int bits,
+                                                              ScanScratch* scratch, int* exp_out) {
   unsigned int m = 0u;
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
-    const unsigned int b = __float_as_uint(x[i]) & 0x7fffffffu;
-    if (b < 0x7f800000u) m = max(m, b);
+  if ((reinterpret_cast<uintptr_t>(x) & 15u) == 0u) {
+    const long long n4 = n >> 2;
+    const float4* x4 = reinterpret_cast<const float4*>(x);
+    long long i = tid;
+    for (; i + 3 * stride < n4; i += 4 * stride) {      // four loads in flight per thread
+      const float4 a = __ldg(x4 + i), b = __ldg(x4 + i + stride), c = __ldg(x4 + i + 2 * stride),
+                   d = __ldg(x4 + i + 3 * stride);
+      m = max(m, max(max(finite_abs_bits(a.x), finite_abs_bits(a.y)), max(finite_abs_bits(a.z), finite_abs_bits(a.w))));
+      m = max(m, max(max(finite_abs_bits(b.x), finite_abs_bits(b.y)), max(finite_abs_bits(b.z), finite_abs_bits(b.w))));
+      m = max(m, max(max(finite_abs_bits(c.x), finite_abs_bits(c.y)), max(finite_abs_bits(c.z), finite_abs_bits(c.w))));
+      m = max(m, max(max(finite_abs_bits(d.x), finite_abs_bits(d.y)), max(finite_abs_bits(d.z), finite_abs_bits(d.w))));
+    }
+    for (; i < n4; i += stride) {
+      const float4 a = __ldg(x4 + i);
+      m = max(m, max(max(finite_abs_bits(a.x), finite_abs_bits(a.y)), max(finite_abs_bits(a.z), finite_abs_bits(a.w))));
+    }
+    for (long long j = (n4 << 2) + tid; j < n; j += stride) m = max(m, finite_abs_bits(x[j]));
+  } else {
+    for (long long j = tid; j < n; j += stride) m = max(m, finite_abs_bits(x[j]));
   }
+  __shared__ unsigned int warp_max[kThreads / 32];
+  __shared__ int is_last;
   m = __reduce_max_sync(0xffffffffu, m);
-  if ((threadIdx.x & 31) == 0 && m) atomicMax(out, m);
-}
-
-__device__ __forceinline__ double clampd(double v, double q) { return fmin(fmax(v, -q), q); }
-
-// One element: Q_theta = clamp(rne(x / 2^e)), Q_c = clamp(rne((x - Q_theta*2^e) / 2^(e-s))).
-__device__ __forceinline__ void quantize_one(float xf, int e, int s, double qmax_t, double qmax_c,
-                                             bool has_comp, int& qt, int& qc) {
-  const double v = (double)xf;
-  qc = 0;
-  if (v != v) { qt = 0; return; }
-  if (isinf(v)) { qt = v > 0 ? (int)qmax_t : -(int)qmax_t; return; }
-  const double t = clampd(rint(scalbn(v, -e)), qmax_t);
-  qt = (int)t;
-  if (has_comp) qc = (int)clampd(rint(scalbn(v - scalbn(t, e), s - e)), qmax_c);
-}
-
-template <typename ThetaT, typename CompT, bool HAS_COMP>
-__global__ void __launch_bounds__(kThreads) quantize_kernel(const float* __restrict__ x, ThetaT* theta,
-                                                            CompT* comp, long long n, int e, int s,
-                                                            int theta_bits, int comp_bits) {
-  const double qmax_t = (double)((1 << (theta_bits - 1)) - 1);
-  const double qmax_c = HAS_COMP ? (double)((1 << (comp_bits - 1)) - 1) : 0.0;
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
-    int qt, qc;
-    quantize_one(x[i], e, s, qmax_t, qmax_c, HAS_COMP, qt, qc);
-    theta[i] = (ThetaT)qt;
-    if (HAS_COMP) comp[i] = (CompT)qc;
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned int b = 0u;
+    for (int w = 0; w < kThreads / 32; ++w) b = max(b, warp_max[w]);
+    if (b) atomicMax(&scratch->amax_bits, b);
+    __threadfence();
+    is_last = atomicAdd(&scratch->done, 1u) == gridDim.x - 1u;
+    if (is_last) {
+      __threadfence();
+      const unsigned int all = __ldcg(&scratch->amax_bits);
+      *exp_out = fit_exponent(__uint_as_float(all), bits);
+      scratch->amax_bits = 0u;
+      scratch->done = 0u;
+    }
   }
 }
 
-// x = fl32(Q_theta * 2^e + Q_c * 2^(e-s)): exact in double, one rounding to binary32.
-template <typename ThetaT, typename CompT, bool HAS_COMP>
-__global__ void __launch_bounds__(kThreads) dequantize_kernel(const ThetaT* __restrict__ theta,
-                                                              const CompT* __restrict__ comp, float* x,
-                                                              long long n, int e, int s) {
+// One element in binary32, every step exact except the two roundings of the definition:
+//   Q_theta = clamp(rne(x / 2^e)),  Q_c = clamp(rne((x - Q_theta*2^e) / 2^(e-s))).
+// x / 2^e is an exact scaling (a result below the normal range is far below half a unit and
+// rounds to 0 either way); the rounding is an addition of M = 1.5 * 2^23 after a clamp to
+// +-(QMAX + 1), which commutes with it; x/2^e - Q_theta is a difference of two floats that
+// either lie within a factor of two of each other or has a result of fewer bits than x/2^e,
+// so it is exact whenever the result can still matter (beyond 2^24 it only has to be large).
+// NaN -> 0, +-Inf -> +-QMAX with nothing left for c.
+template <int TB, int CB>
+__device__ __forceinline__ void quantize_one(float x, float inv2e, float pow2s, int& qt, int& qc) {
+  constexpr float kM = 12582912.0f;
+  constexpr float qmax_t = (float)((1 << (TB - 1)) - 1);
+  constexpr float qmax_c = (float)((1 << ((CB ? CB : 8) - 1)) - 1);
+  const float xs = __fmul_rn(x, inv2e);
+  float t = fminf(fmaxf(xs, -(qmax_t + 1.0f)), qmax_t + 1.0f);      // NaN -> a finite bound, fixed below
+  t = __fadd_rn(__fadd_rn(t, kM), -kM);
+  t = fminf(fmaxf(t, -qmax_t), qmax_t);
+  const bool nan = x != x, inf = fabsf(x) == __int_as_float(0x7f800000);
+  qt = nan ? 0 : (int)t;
+  qc = 0;
+  if constexpr (CB != 0) {
+    float r = __fmul_rn(__fadd_rn(xs, -t), pow2s);
+    r = fminf(fmaxf(r, -(qmax_c + 1.0f)), qmax_c + 1.0f);
+    r = __fadd_rn(__fadd_rn(r, kM), -kM);
+    r = fminf(fmaxf(r, -qmax_c), qmax_c);
+    qc = (nan || inf) ? 0 : (int)r;
+  }
+}
+
+template <int BITS>
+__device__ __forceinline__ void store4(void* base, long long i4, const int (&q)[4]) {
+  if constexpr (BITS == 8) {
+    reinterpret_cast<unsigned int*>(base)[i4] = (unsigned int)(q[0] & 0xff) | ((unsigned int)(q[1] & 0xff) << 8) |
+                                                ((unsigned int)(q[2] & 0xff) << 16) | ((unsigned int)q[3] << 24);
+  } else {
+    reinterpret_cast<uint2*>(base)[i4] = make_uint2((unsigned int)(q[0] & 0xffff) | ((unsigned int)q[1] << 16),
+                                                    (unsigned int)(q[2] & 0xffff) | ((unsigned int)q[3] << 16));
+  }
+}
+
+template <int BITS>
+__device__ __forceinline__ void store1(void* base, long long i, int q) {
+  if constexpr (BITS == 8) static_cast<signed char*>(base)[i] = (signed char)q;
+  else static_cast<short*>(base)[i] = (short)q;
+}
+
+// exp_dev != nullptr: the exponent is read from device memory (left there by the scan);
+// otherwise e_fixed applies.  Four consecutive elements per thread and access when the three
+// arrays are aligned for it (16 bytes for x; 4 or 8 for theta and c), one otherwise.
+template <int TB, int CB>
+__global__ void __launch_bounds__(kThreads) quantize_kernel(const float* __restrict__ x, void* theta, void* comp,
+                                                            long long n, const int* exp_dev, int e_fixed, int s) {
+  const int e = exp_dev ? __ldcg(exp_dev) : e_fixed;
+  const float inv2e = __int_as_float((127 - e) << 23);      // |e| <= 64: a normal power of two
+  const float pow2s = __int_as_float((127 + s) << 23);
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
-    double v = scalbn((double)theta[i], e);
-    if (HAS_COMP) v += scalbn((double)comp[i], e - s);
-    x[i] = __double2float_rn(v);
+  const bool vec = ((reinterpret_cast<uintptr_t>(x) & 15u) | (reinterpret_cast<uintptr_t>(theta) & (TB / 2 - 1)) |
+                    (CB ? (reinterpret_cast<uintptr_t>(comp) & ((CB ? CB : 8) / 2 - 1)) : 0)) == 0u;
+  long long done = 0;
+  if (vec) {
+    const long long n4 = n >> 2;
+    const float4* x4 = reinterpret_cast<const float4*>(x);
+#pragma unroll 2
+    for (long long i = tid; i < n4; i += stride) {
+      const float4 v = __ldcs(x4 + i);       // last use of the source: let it leave the caches first
+      int qt[4], qc[4];
+      quantize_one<TB, CB>(v.x, inv2e, pow2s, qt[0], qc[0]);
+      quantize_one<TB, CB>(v.y, inv2e, pow2s, qt[1], qc[1]);
+      quantize_one<TB, CB>(v.z, inv2e, pow2s, qt[2], qc[2]);
+      quantize_one<TB, CB>(v.w, inv2e, pow2s, qt[3], qc[3]);
+      store4<TB>(theta, i, qt);
+      if constexpr (CB != 0) store4<(CB ? CB : 8)>(comp, i, qc);
+    }
+    done = n4 << 2;
+  }
+  for (long long j = done + tid; j < n; j += stride) {
+    int qt, qc;
+    quantize_one<TB, CB>(x[j], inv2e, pow2s, qt, qc);
+    store1<TB>(theta, j, qt);
+    if constexpr (CB != 0) store1<(CB ? CB : 8)>(comp, j, qc);
+  }
+}
+
+template <int BITS>
+__device__ __forceinline__ void load4(const void* base, long long i4, float (&q)[4]) {
+  if constexpr (BITS == 8) {
+    const unsigned int w = reinterpret_cast<const unsigned int*>(base)[i4];
+    q[0] = (float)(signed char)(w & 0xff);
+    q[1] = (float)(signed char)((w >> 8) & 0xff);
+    q[2] = (float)(signed char)((w >> 16) & 0xff);
+    q[3] = (float)(signed char)(w >> 24);
+  } else {
+    const uint2 w = reinterpret_cast<const uint2*>(base)[i4];
+    q[0] = (float)(short)(w.x & 0xffff);
+    q[1] = (float)(short)(w.x >> 16);
+    q[2] = (float)(short)(w.y & 0xffff);
+    q[3] = (float)(short)(w.y >> 16);
+  }
+}
+
+template <int BITS>
+__device__ __forceinline__ float load1(const void* base, long long i) {
+  if constexpr (BITS == 8) return (float)static_cast<const signed char*>(base)[i];
+  else return (float)static_cast<const short*>(base)[i];
+}
+
+// x = fl32(Q_theta * 2^e + Q_c * 2^(e-s)): the FMA forms Q_theta * 2^s + Q_c exactly and
+// rounds once; the scaling by 2^(e-s) that follows is exact (the result is a normal number:
+// |e - s| <= 79).
+template <int TB, int CB>
+__global__ void __launch_bounds__(kThreads) dequantize_kernel(const void* __restrict__ theta,
+                                                              const void* __restrict__ comp, float* x, long long n,
+                                                              int e, int s) {
+  const float pow2s = __int_as_float((127 + s) << 23);
+  const float pow2es = __int_as_float((127 + e - s) << 23);
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const bool vec = ((reinterpret_cast<uintptr_t>(x) & 15u) | (reinterpret_cast<uintptr_t>(theta) & (TB / 2 - 1)) |
+                    (CB ? (reinterpret_cast<uintptr_t>(comp) & ((CB ? CB : 8) / 2 - 1)) : 0)) == 0u;
+  long long done = 0;
+  if (vec) {
+    const long long n4 = n >> 2;
+#pragma unroll 2
+    for (long long i = tid; i < n4; i += stride) {
+      float qt[4], qc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+      load4<TB>(theta, i, qt);
+      if constexpr (CB != 0) load4<(CB ? CB : 8)>(comp, i, qc);
+      float4 v;
+      v.x = __fmul_rn(__fmaf_rn(qt[0], pow2s, qc[0]), pow2es);
+      v.y = __fmul_rn(__fmaf_rn(qt[1], pow2s, qc[1]), pow2es);
+      v.z = __fmul_rn(__fmaf_rn(qt[2], pow2s, qc[2]), pow2es);
+      v.w = __fmul_rn(__fmaf_rn(qt[3], pow2s, qc[3]), pow2es);
+      __stcs(reinterpret_cast<float4*>(x) + i, v);
+    }
+    done = n4 << 2;
+  }
+  for (long long j = done + tid; j < n; j += stride) {
+    float qc = 0.0f;
+    if constexpr (CB != 0) qc = load1<(CB ? CB : 8)>(comp, j);
+    x[j] = __fmul_rn(__fmaf_rn(load1<TB>(theta, j), pow2s, qc), pow2es);
   }
 }
 

@@ -110,6 +110,8 @@ struct StepParams {
   int amax_mode;     // 1: exponents follow the max scan, 0: fixed
   int inline_args;   // 1: grads/lrs are in the InlineArgs parameter
   int grad_evict_first;  // 1: gradient loads carry the L2 evict-first hint
+  const int* exp_grad_dev;   // fixed-point gradients: device array of their exponents (as a scan on the
+                             // device left them), or nullptr: the exponents come with the per-step arguments
   int advance;           // 1: this launch ends a step (the phase word moves on); 0: more launches of the
                          //    same step follow (the host-buffer entry point updates groups of tensors in turn)
   // The launch covers tiles [tile_begin, tile_begin + tile_count), which are all the tiles
@@ -1020,7 +1022,8 @@ __device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const QGrad
   m.ti = ti ? *ti : p.ws.info[t];
   m.grad = p.inline_args ? a.grads[t] : static_cast<const void*>(p.ws.grad_ptr[t]);
   m.lr = p.inline_args ? a.lrs[t] : p.ws.lr[t];
-  m.eg = p.inline_args ? (int)a.exp_grad[t] : p.ws.exp_grad[t];
+  if (p.exp_grad_dev) m.eg = max(kExpMin, min(kExpMax, __ldcg(p.exp_grad_dev + t)));
+  else m.eg = p.inline_args ? (int)a.exp_grad[t] : p.ws.exp_grad[t];
   step_exponents(p, t, ph, strict, m);
   if (owner) record_exponents(p, t, ph, strict, m);
   return m;

@@ -8,7 +8,7 @@ CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIBRARY = os.path.join(_HERE, "libkahan_sgd.so")
 SOURCES = [os.path.join(CSRC, "kahan_sgd_api.cu")]
-_DEPENDS = SOURCES + [os.path.join(CSRC, "kahan_sgd_kernels.cuh"),
+_DEPENDS = SOURCES + [os.path.join(CSRC, "kahan_sgd_ring.cuh"), os.path.join(CSRC, "kahan_sgd_kernels.cuh"),
                       os.path.join(CSRC, "kahan_sgd_momentum_kernels.cuh"),
                       os.path.join(CSRC, "kahan_sgd_adam_kernels.cuh"),
                       os.path.join(CSRC, "kahan_sgd_convert.cuh"),

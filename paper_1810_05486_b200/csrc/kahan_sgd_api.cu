@@ -164,16 +164,16 @@ int read_stats(const unsigned char* b, const Layout& L, const ksgd_tensor_desc* 
   for (size_t i = 0; i < n; ++i) {
     const TensorState& r = last[i];
     const int e_next = r.ovr_theta ? r.ovr_theta - kOvrBias
-                                   : next_exponent(r.amax_t, descs[i].theta_bits, r.exp_theta, amax_mode);
-    if (amax_theta) amax_theta[i] = r.amax_t;
-    if (amax_comp) amax_comp[i] = r.amax_c;
+                                   : next_exponent(r.amax[0], descs[i].theta_bits, r.exp_theta, amax_mode);
+    if (amax_theta) amax_theta[i] = r.amax[0];
+    if (amax_comp) amax_comp[i] = r.amax[1];
     if (exp_theta_cur) exp_theta_cur[i] = r.exp_theta;
     if (exp_theta_next) exp_theta_next[i] = e_next;
     if (strict) {
       if (exp_comp_cur) exp_comp_cur[i] = r.exp_comp;
       if (exp_comp_next)
         exp_comp_next[i] = r.ovr_comp ? r.ovr_comp - kOvrBias
-                                      : next_exponent_acc(r.amax_c, descs[i].comp_bits, r.exp_comp, e_next, amax_mode);
+                                      : next_exponent_acc(r.amax[1], descs[i].comp_bits, r.exp_comp, e_next, amax_mode);
     }
   }
   if (n_sat_theta) std::memcpy(n_sat_theta, b + L.counters, 8 * n);

@@ -12,52 +12,19 @@
 //     finished scans (rotating buffers, see Workspace): no block is ever the last one.
 // The pass is bound by HBM traffic: 2*m/8 + 2*n/8 + 4 bytes per parameter.
 //
-// Structure: a persistent grid, one block per SM.  The tensor list is cut into tiles of
-// kChunk elements (2 * kChunk for 8-bit theta in long lists); block b takes tiles b,
-// b + gridDim.x, ....  One producer thread streams the tiles of theta, c and g into a 224 KB shared-memory ring with bulk
-// asynchronous copies (cp.async.bulk, completion counted on an mbarrier), so the bytes in
-// flight do not depend on registers or occupancy; a tile takes only the pages its format
-// needs (6 for int8/int8 -- 12 with the large tiles --, 8 for int16/int16), so two to four
-// tiles are resident.
-// Sixteen consumer warps compute from shared memory and store theta' and c' straight to
-// global memory with 16-byte stores.
-// No block ever waits for another block; every wait inside a block is bounded.
-//
-// State between steps.  The per-tensor state a step leaves behind (the exponent it wrote,
-// its max scans) lives in three rotating buffers indexed by the step's phase p = step mod 3
-// (a word in the workspace).  Step p reads buffer p-1 (exponent of the stored mantissas,
-// finished scans), derives from it the exponent it writes (every block that meets a tensor
-// derives the same value and stores it into buffer p: idempotent), accumulates its own scans
-// into buffer p, and clears buffer p+1, which nobody reads or writes until the next step.
-// So a step needs no pass "after all blocks are done": the kernel ends when each block has
-// published its scans, and the next launch finds everything it needs.  The phase word is
-// advanced by the block that draws the last entry ticket, i.e. after every block of the
-// step has read it.
+// The persistent grid, the paged shared-memory ring, the scan publishing and the state that
+// steps hand to one another are those of kahan_sgd_ring.cuh; this file adds what is specific
+// to the plain optimizer: three arrays per tile (gradient, theta, c), the arithmetic of an
+// element, two max scans and one exponent (two in strict mode) per tensor.
 #pragma once
 
-#include <cstdint>
-#include <type_traits>
-#include <cuda_runtime.h>
+#include "kahan_sgd_ring.cuh"
 
 namespace ksgd {
 
-constexpr int kChunk = 8192;           // elements per tile (twice as many for 8-bit theta in long lists)
-constexpr long long kBigTileMinTiles = 1024;   // a list gets the large 8-bit tiles if it still has this many tiles
 constexpr int kConsumerWarps = 16;
 constexpr int kConsumers = kConsumerWarps * 32;
 constexpr int kBlockThreads = kConsumers + 32;   // + one producer warp
-constexpr int kSlots = 6;              // tiles a block can have in its ring at once
-constexpr int kPageBytes = 8192;       // the ring is handed out in pages
-static_assert(kChunk == 8192 && kPageBytes == kChunk, "the producer's page arithmetic assumes 8192-element tiles and 8 KB pages");
-constexpr int kPages = 28;             // 224 KB of tile data per block
-constexpr int kInlineArgs = 256;     // lists up to this long pass grads/lrs as kernel parameters
-constexpr int kUploadBatch = 1024;   // tensors per launch of the argument-upload kernel
-constexpr int kDLimit = 1 << 30;     // clamp of the quantized increment, in compensation LSBs
-constexpr int kMaxDelta = 8;         // largest exponent change per step
-constexpr int kExpMin = -64, kExpMax = 64;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a barrier wait gives up after 2 s
-
-enum DeviceError { kErrNone = 0, kErrFullWait = 1, kErrEmptyWait = 2 };
 
 struct TensorInfo {
   void* theta;
@@ -69,19 +36,12 @@ struct TensorInfo {
   int pad;
 };
 
-struct ChunkRef {
-  int tensor;  // index into the tensor list
-  int index;   // tile number inside that tensor: elements [index*chunk, ...), chunk = the tensor's tile size
-};
-
-// Device-side view of the caller's workspace.
 // What a step leaves behind for one tensor: everything the next step needs to know about it,
 // in one 32-byte record (one load).
 struct __align__(32) TensorState {
   int exp_theta;          // exponent of theta's mantissas as this step wrote them
   int exp_comp;           // strict mode: the same for the compensation's own exponent
-  unsigned int amax_t;    // this step's max scans (blocks add to them while the step runs)
-  unsigned int amax_c;
+  unsigned int amax[2];   // this step's max scans of theta and c (blocks add to them while the step runs)
   int ovr_theta;          // exponent the NEXT step must write instead of the one the scans give:
   int ovr_comp;           //   value + kOvrBias, 0 = none (init, kahan_sgd_set_exponents; comp: init only)
   int pad[2];
@@ -101,7 +61,6 @@ struct Workspace {
   int* exp_grad;                   // [n] the same, exponents of fixed-point gradients
   ChunkRef* chunks;                // [n_chunks]
 };
-constexpr int kOvrBias = 1000;
 
 struct StepParams {
   Workspace ws;
@@ -189,126 +148,14 @@ constexpr int kFlagCompPageShift = 13;
 constexpr int kFlagGradPageShift = 18;
 
 // Max scans and counters of one tile, gathered in shared memory: the consumer warps add to
-// it, the producer publishes it when it takes the tile's stage back.
+// it, the producer publishes it when it takes the tile's stage back.  (Two maxima, then three
+// counts: the order the ring expects.)
 struct TileScan {
   unsigned int amax_t, amax_c, n_sat_t, n_sat_c, n_nonfinite, pad[3];
 };
 
 // ----------------------------------------------------------------------------------------
-// mbarrier / bulk-copy wrappers (PTX)
-
-__device__ __forceinline__ unsigned int smem_addr(const void* p) {
-  return static_cast<unsigned int>(__cvta_generic_to_shared(p));
-}
-
-__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
-  asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.shared::cta.b64 st, [%0];\n}" ::"r"(smem_addr(bar))
-               : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, unsigned int bytes) {
-  asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(
-                   smem_addr(bar)),
-               "r"(bytes)
-               : "memory");
-}
-
-// Announce `bytes` more bytes for the current phase without arriving.
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned int bytes) {
-  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
-               : "memory");
-}
-
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned int parity) {
-  unsigned int ok;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(smem_addr(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
-__device__ __forceinline__ unsigned long long global_timer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
-// Bounded wait: false if the phase did not complete within kWaitLimitNs or another thread
-// of the block has already given up.
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned int parity,
-                                          const volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_timer_ns();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 64; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (global_timer_ns() - t0 > kWaitLimitNs) return false;
-  }
-}
-
-// Global -> shared bulk copy of `bytes` (multiple of 16, both addresses 16-byte aligned),
-// completion counted in bytes on `bar`.
-__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, unsigned int bytes,
-                                          unsigned long long* bar) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-          smem_addr(dst_smem)),
-      "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar))
-      : "memory");
-}
-
-// Same, with an L2 eviction-priority hint for data that is read once per step.
-__device__ __forceinline__ void bulk_load_hint(void* dst_smem, const void* src_gmem, unsigned int bytes,
-                                               unsigned long long* bar, unsigned long long policy) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
-          smem_addr(dst_smem)),
-      "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar)), "l"(policy)
-      : "memory");
-}
-
-// Programmatic dependent launch.  The step kernels are launched with programmatic stream
-// serialization: a block of the next kernel in the stream may become resident as soon as an
-// SM has room (a block of this kernel has exited) and run its prologue -- barrier set-up,
-// its first table entries -- while the rest of this kernel finishes.  Before it touches
-// anything an earlier kernel wrote (exponents, mantissas, gradients, per-step arguments in
-// the workspace) every thread passes grid_dependency_wait(), which returns once the
-// preceding kernel has completed and its writes are visible.  Launched the ordinary way
-// both instructions do nothing.  The hardware orders the grids; nothing spins.
-__device__ __forceinline__ void grid_dependency_launch_dependents() {
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-}
-__device__ __forceinline__ void grid_dependency_wait() {
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-}
-
-__device__ __forceinline__ unsigned long long l2_policy_evict_first() {
-  unsigned long long pol;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-  return pol;
-}
-
-// ----------------------------------------------------------------------------------------
 // Arithmetic
-
-__device__ __forceinline__ float pow2_float(int e) {  // exact 2^e for e in [-126, 127]
-  return __int_as_float((e + 127) << 23);
-}
-
-// a / 2^r, round to nearest, ties to even (|a| < 2^62).
-__device__ __forceinline__ long long rne_shift64(long long a, int r) {
-  if (r == 0) return a;
-  const long long bias = ((1LL << (r - 1)) - 1) + ((a >> r) & 1LL);
-  return (a + bias) >> r;
-}
 
 __device__ __forceinline__ int quantize_increment(float g, float scale) {
   const float x = __fmul_rn(g, scale);   // one binary32 multiply, never contracted
@@ -404,67 +251,6 @@ __device__ __noinline__ void update_general(const StepCoef* coef, int tb, int cb
 }
 
 // ----------------------------------------------------------------------------------------
-// 16-byte vector helpers.  A Pack holds V elements of B bits (8, 16, 32 or 64 bytes).
-
-template <int BYTES> struct Pack;
-template <> struct Pack<8>  { uint2 v; };
-template <> struct Pack<16> { uint4 v; };
-template <> struct Pack<32> { uint4 v[2]; };
-template <> struct Pack<64> { uint4 v[4]; };
-
-template <int BYTES>
-__device__ __forceinline__ Pack<BYTES> load_pack(const void* p) {
-  Pack<BYTES> r;
-  if constexpr (BYTES == 8) {
-    r.v = *reinterpret_cast<const uint2*>(p);
-  } else if constexpr (BYTES == 16) {
-    r.v = *reinterpret_cast<const uint4*>(p);
-  } else {
-#pragma unroll
-    for (int i = 0; i < BYTES / 16; ++i) r.v[i] = reinterpret_cast<const uint4*>(p)[i];
-  }
-  return r;
-}
-
-template <int BYTES>
-__device__ __forceinline__ void store_pack(void* p, const Pack<BYTES>& r) {
-  if constexpr (BYTES == 8) {
-    *reinterpret_cast<uint2*>(p) = r.v;
-  } else if constexpr (BYTES == 16) {
-    *reinterpret_cast<uint4*>(p) = r.v;
-  } else {
-#pragma unroll
-    for (int i = 0; i < BYTES / 16; ++i) reinterpret_cast<uint4*>(p)[i] = r.v[i];
-  }
-}
-
-template <int BYTES>
-__device__ __forceinline__ unsigned int pack_word(const Pack<BYTES>& r, int w) {
-  if constexpr (BYTES == 8) {
-    return w == 0 ? r.v.x : r.v.y;
-  } else if constexpr (BYTES == 16) {
-    return w == 0 ? r.v.x : (w == 1 ? r.v.y : (w == 2 ? r.v.z : r.v.w));
-  } else {
-    const uint4& q = r.v[w >> 2];
-    const int j = w & 3;
-    return j == 0 ? q.x : (j == 1 ? q.y : (j == 2 ? q.z : q.w));
-  }
-}
-
-template <int BYTES>
-__device__ __forceinline__ void set_pack_word(Pack<BYTES>& r, int w, unsigned int x) {
-  if constexpr (BYTES == 8) {
-    if (w == 0) r.v.x = x; else r.v.y = x;
-  } else if constexpr (BYTES == 16) {
-    if (w == 0) r.v.x = x; else if (w == 1) r.v.y = x; else if (w == 2) r.v.z = x; else r.v.w = x;
-  } else {
-    uint4& q = r.v[w >> 2];
-    const int j = w & 3;
-    if (j == 0) q.x = x; else if (j == 1) q.y = x; else if (j == 2) q.z = x; else q.w = x;
-  }
-}
-
-// ----------------------------------------------------------------------------------------
 // Steady state (no exponent change): one vector of V elements on the FP32 pipe, used as an
 // exact integer unit.  With M = 1.5 * 2^23 every float in [2^23, 2^24) is an integer whose
 // low mantissa bits are that integer in two's complement relative to M, an addition that
@@ -490,59 +276,6 @@ __device__ __forceinline__ void set_pack_word(Pack<BYTES>& r, int w, unsigned in
 // formed by one FMA onto M - d, so a change of c's exponent stays on this path; the vector
 // also leaves the path when |C1| or |r0| exceeds c's n bits (the clamps of statements 1, 3).
 
-constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23, bits 0x4B400000
-constexpr unsigned int kMagicBits = 0x4B400000u;
-
-// M + 2^(BITS-1) + q for element i of a pack whose sign bits have been flipped.
-template <int BITS, int BYTES>
-__device__ __forceinline__ float magic_elem(const Pack<BYTES>& r, int i) {
-  if constexpr (BITS == 8) {
-    return __uint_as_float(__byte_perm(pack_word(r, i >> 2), kMagicBits, 0x7640u | (unsigned)(i & 3)));
-  } else {
-    return __uint_as_float(__byte_perm(pack_word(r, i >> 1), kMagicBits, (i & 1) ? 0x7632u : 0x7610u));
-  }
-}
-
-// M + q for element i of a pack of signed mantissas, in one instruction: the integer dot
-// product with a selector that is 1 at element i sign-extends the mantissa and adds it to
-// M's bit pattern (for |q| < 2^22 integer addition on the bits is addition of the values).
-// It runs on the FMA pipe; the PRMT form above and the sign flips it needs take the ALU
-// pipe, which has half the lanes and also carries the scans and the packing.
-template <int BITS, int BYTES>
-__device__ __forceinline__ float magic_signed(const Pack<BYTES>& r, int i) {
-  if constexpr (BITS == 8) {
-    return __int_as_float(__dp4a((int)pack_word(r, i >> 2), 1 << (8 * (i & 3)), (int)kMagicBits));
-  } else {
-    return __int_as_float(__dp2a_lo((int)pack_word(r, i >> 1), (i & 1) ? 0x0100 : 0x0001, (int)kMagicBits));
-  }
-}
-
-template <int BITS, int BYTES>
-__device__ __forceinline__ void flip_signs(Pack<BYTES>& r) {
-  constexpr unsigned int m = BITS == 8 ? 0x80808080u : 0x80008000u;
-#pragma unroll
-  for (int w = 0; w < BYTES / 4; ++w) set_pack_word(r, w, pack_word(r, w) ^ m);
-}
-
-// Low BITS bits of V magic floats, packed.
-template <int BITS, int V>
-__device__ __forceinline__ Pack<V * BITS / 8> pack_magic(const float (&x)[V]) {
-  Pack<V * BITS / 8> r;
-  if constexpr (BITS == 8) {
-#pragma unroll
-    for (int w = 0; w < V / 4; ++w) {
-      const unsigned int lo = __byte_perm(__float_as_uint(x[4 * w]), __float_as_uint(x[4 * w + 1]), 0x0040);
-      const unsigned int hi = __byte_perm(__float_as_uint(x[4 * w + 2]), __float_as_uint(x[4 * w + 3]), 0x0040);
-      set_pack_word(r, w, __byte_perm(lo, hi, 0x5410));
-    }
-  } else {
-#pragma unroll
-    for (int w = 0; w < V / 2; ++w)
-      set_pack_word(r, w, __byte_perm(__float_as_uint(x[2 * w]), __float_as_uint(x[2 * w + 1]), 0x5410));
-  }
-  return r;
-}
-
 struct SteadyCoef {
   float scale;      // lr * 2^-(e - s)
   float pow2s_neg;  // -2^s
@@ -556,24 +289,6 @@ struct TileHot {       // the consumers' copy of the first 48 bytes of a TileDes
   unsigned char* comp;
   int tensor, n_bulk, count, flags;
 };
-
-// Three-input maximum / minimum (one instruction on sm_100a).  The .NaN form returns NaN as
-// soon as one input is NaN, which is how a NaN product reaches the range check below.
-__device__ __forceinline__ float max3_nan(float a, float b, float c) {
-  float d;
-  asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-  float d;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
-__device__ __forceinline__ float min3(float a, float b, float c) {
-  float d;
-  asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
 
 // The scans take two elements per instruction: the largest and smallest Pb give max|P|, and
 // |x|, |r0| go through three-input maxima.
@@ -874,32 +589,6 @@ __device__ __noinline__ void regrid_tile(const TileDesc* td, TileScan* slots, un
   if (wrote_stage) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// Next exponent from the max scan: the tight fit puts the largest mantissa in
-// (QMAX/2, QMAX].  With L = bit length of amax and QMAX = 2^(b-1)-1, the change is
-// L-(b-1), plus one more when amax still exceeds QMAX*2^change.
-__host__ __device__ __forceinline__ int bit_length(unsigned int x) {
-#ifdef __CUDA_ARCH__
-  return 32 - __clz(x);
-#else
-  int n = 0;
-  while (x) { ++n; x >>= 1; }
-  return n;
-#endif
-}
-
-__host__ __device__ __forceinline__ int next_exponent(unsigned int amax, int bits, int e_out, int amax_mode) {
-  if (!amax_mode || amax == 0u) return e_out;
-  const int L = bit_length(amax);
-  int change = L - (bits - 1);
-  if (change >= 1) {
-    const unsigned long long cap = (unsigned long long)((1 << (bits - 1)) - 1) << change;
-    if ((unsigned long long)amax > cap) ++change;
-  }
-  change = change < -kMaxDelta ? -kMaxDelta : (change > kMaxDelta ? kMaxDelta : change);
-  const int e = e_out + change;
-  return e < kExpMin ? kExpMin : (e > kExpMax ? kExpMax : e);
-}
-
 // Strict mode: the compensation's own next exponent.  The tight fit of its scan; an empty
 // scan (every increment rounded away, or none came) makes the grid 8 binades finer; the
 // result stays within [e_next - 36, e_next + 8] of theta's next exponent, which keeps every
@@ -911,51 +600,6 @@ __host__ __device__ __forceinline__ int next_exponent_acc(unsigned int amax, int
   if (amax_mode && amax == 0u) ec = ec_out - kMaxDelta;
   ec = ec < e_next - kStrictBelow ? e_next - kStrictBelow : (ec > e_next + kStrictAbove ? e_next + kStrictAbove : ec);
   return ec < kExpMin ? kExpMin : (ec > kExpMax ? kExpMax : ec);
-}
-
-struct __align__(128) BlockShared {
-  unsigned long long full[kSlots];     // producer -> consumers: the tile's bytes have landed
-  unsigned long long empty[kSlots];    // consumers -> producer: the tile's pages may be reused
-  TileDesc desc[kSlots];
-  TileScan scan[kSlots];
-  int slot_pages[kSlots];              // ring pages held by the tile in each slot
-  int abort_flag;   // set by the first thread whose bounded wait ran out
-  int never;        // stays 0: abort flag for waits that must not be cut short
-};
-
-constexpr size_t kSharedBytes = (size_t)kPages * kPageBytes + sizeof(BlockShared);
-
-// Producer side: scans of finished tiles are merged per tensor in registers and go to
-// global memory when the tensor changes (one set of atomics per block and tensor run).
-struct ScanAcc {
-  int tensor = -1;
-  unsigned int amax_t = 0, amax_c = 0, n_sat_t = 0, n_sat_c = 0, n_nonfinite = 0;
-};
-
-__device__ __forceinline__ void publish(const StepParams& p, ScanAcc& acc, TensorState* now) {
-  if (acc.tensor >= 0) {
-    const int t = acc.tensor, n = p.n_tensors;
-    if (acc.amax_t) atomicMax(&now[t].amax_t, acc.amax_t);
-    if (acc.amax_c) atomicMax(&now[t].amax_c, acc.amax_c);
-    if (acc.n_sat_t) atomicAdd(&p.ws.counters[t], (unsigned long long)acc.n_sat_t);
-    if (acc.n_sat_c) atomicAdd(&p.ws.counters[n + t], (unsigned long long)acc.n_sat_c);
-    if (acc.n_nonfinite) atomicAdd(&p.ws.counters[2 * n + t], (unsigned long long)acc.n_nonfinite);
-  }
-  acc = ScanAcc{};
-}
-
-__device__ __forceinline__ void take_back(const StepParams& p, ScanAcc& acc, TensorState* now,
-                                          TileScan* scan, int tensor) {
-  if (tensor != acc.tensor) {
-    publish(p, acc, now);
-    acc.tensor = tensor;
-  }
-  acc.amax_t = max(acc.amax_t, scan->amax_t);
-  acc.amax_c = max(acc.amax_c, scan->amax_c);
-  acc.n_sat_t += scan->n_sat_t;
-  acc.n_sat_c += scan->n_sat_c;
-  acc.n_nonfinite += scan->n_nonfinite;
-  scan->amax_t = scan->amax_c = scan->n_sat_t = scan->n_sat_c = scan->n_nonfinite = 0u;
 }
 
 // What the producer reads about a tile's tensor, fetched one tile ahead.
@@ -978,7 +622,7 @@ __device__ __forceinline__ void step_exponents(const StepParams& p, int t, int p
   const int4* rec = reinterpret_cast<const int4*>(&p.ws.state[(size_t)prev * p.ws.slab + t]);
   const int4 r0 = __ldcg(rec), r1 = __ldcg(rec + 1);
   m.e_in = r0.x;
-  m.e_out = r1.x ? r1.x - kOvrBias : next_exponent((unsigned)r0.z, m.ti.theta_bits, m.e_in, p.amax_mode);
+  m.e_out = r1.x ? r1.x - kOvrBias : next_exponent((unsigned)r0.z, m.ti.theta_bits, m.e_in, p.amax_mode);   // r0.z, r0.w: amax[0], amax[1]
   if (strict) {
     m.ec_in = r0.y;
     m.ec_out = r1.y ? r1.y - kOvrBias : next_exponent_acc((unsigned)r0.w, m.ti.comp_bits, m.ec_in, m.e_out, p.amax_mode);
@@ -1005,19 +649,18 @@ __device__ __forceinline__ void record_exponents(const StepParams& p, int t, int
 
 // ti: the tensor's table entry if the caller has it already (the table never changes).
 __device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const InlineArgs& a, int t, int ph, bool strict,
-                                                bool owner, const TensorInfo* ti = nullptr) {
+                                                const TensorInfo* ti) {
   TensorMeta m;
   m.ti = ti ? *ti : p.ws.info[t];
   m.grad = p.inline_args ? a.grads[t] : p.ws.grad_ptr[t];
   m.lr = p.inline_args ? a.lrs[t] : p.ws.lr[t];
   m.eg = 0;
   step_exponents(p, t, ph, strict, m);
-  if (owner) record_exponents(p, t, ph, strict, m);
   return m;
 }
 
 __device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const QGradArgs& a, int t, int ph, bool strict,
-                                                bool owner, const TensorInfo* ti = nullptr) {
+                                                const TensorInfo* ti) {
   TensorMeta m;
   m.ti = ti ? *ti : p.ws.info[t];
   m.grad = p.inline_args ? a.grads[t] : static_cast<const void*>(p.ws.grad_ptr[t]);
@@ -1025,272 +668,129 @@ __device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const QGrad
   if (p.exp_grad_dev) m.eg = max(kExpMin, min(kExpMax, __ldcg(p.exp_grad_dev + t)));
   else m.eg = p.inline_args ? (int)a.exp_grad[t] : p.ws.exp_grad[t];
   step_exponents(p, t, ph, strict, m);
-  if (owner) record_exponents(p, t, ph, strict, m);
   return m;
 }
 
-// The whole step.  GB = 32: binary32 gradients; 8 / 16: fixed-point gradients (one or two
-// bytes per parameter instead of four on the gradient stream).
-// STRICT: every statement of Algorithm 1 rounds into the stored format and the compensation
-// has its own exponent (comp_bits != 0 for every tensor).
-template <int GB, bool STRICT, typename Args>
-__device__ __forceinline__ void step_body(const StepParams& p, const Args& a) {
-  extern __shared__ __align__(128) unsigned char smem[];
-  BlockShared* sh = reinterpret_cast<BlockShared*>(smem + (size_t)kPages * kPageBytes);
-  grid_dependency_launch_dependents();   // the next step's blocks may take over SMs as ours exit
+// The plain optimizer as a policy of the ring (kahan_sgd_ring.cuh).  GB = 32: binary32
+// gradients; 8 / 16: fixed-point gradients (one or two bytes per parameter instead of four on
+// the gradient stream).  STRICT: every statement of Algorithm 1 rounds into the stored format
+// and the compensation has its own exponent (comp_bits != 0 for every tensor).
+template <int GB, bool STRICT>
+struct PlainPolicy {
+  static constexpr int kStreams = 3;          // gradient, theta, c
+  static constexpr int kConsumerWarps = ksgd::kConsumerWarps;
+  static constexpr int kAmax = 2, kCounts = 3;
+  using Params = StepParams;
+  using Info = TensorInfo;
+  using State = TensorState;
+  using TileDesc = ksgd::TileDesc;
+  using TileScan = ksgd::TileScan;
+  using Meta = TensorMeta;
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kSlots; ++s) {
-      mbar_init(&sh->full[s], 1u);
-      mbar_init(&sh->empty[s], (unsigned)kConsumerWarps);
-    }
-    sh->abort_flag = 0;
-    sh->never = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  template <typename Args>
+  static __device__ __forceinline__ Meta load_meta(const Params& p, const Args& a, int t, int ph, const Info* ti) {
+    return ksgd::load_meta(p, a, t, ph, STRICT, ti);
   }
-  if (threadIdx.x < kSlots * (int)(sizeof(TileScan) / 4))
-    reinterpret_cast<unsigned int*>(sh->scan)[threadIdx.x] = 0u;
-  __syncthreads();
-
-  if (warp == kConsumerWarps) {
-    // ------------------------------------------------------------------ producer
-    // Block b takes tiles b, b + gridDim.x, ...: neighbouring tiles run on neighbouring
-    // SMs at the same time, and the tiles of a tensor that needs the general path are
-    // spread evenly over all blocks.  Table entries are fetched two tiles ahead and the
-    // tensor's data one tile ahead, so none of these loads sits between a freed stage and
-    // the copy that refills it.
-    if (lane == 0) {
-      const int stride = (int)gridDim.x;
-      const int n_my = (p.tile_count - (int)blockIdx.x + stride - 1) / stride;
-      const int tile0 = p.tile_begin + (int)blockIdx.x;
-      const unsigned long long grad_policy = l2_policy_evict_first();
-      ScanAcc acc;
-      // the tile table is written once at init: read the first entries before waiting for
-      // the preceding kernel
-      ChunkRef cr = p.ws.chunks[tile0];
-      ChunkRef cr1{-1, -1};
-      if (n_my > 1) cr1 = p.ws.chunks[tile0 + stride];
-      const TensorInfo ti_first = p.ws.info[cr.tensor];       // the tensor table never changes either
-      // The step's phase.  The preceding step moves the word on as soon as all of its blocks
-      // have started, long before it ends, so the value read here, before the wait, is
-      // normally the right one already: the first record is fetched under it while the word
-      // is read again, and only fetched a second time if the two differ.  (The block's entry
-      // ticket, which tells the last block that all have read this word, is drawn by a
-      // consumer thread once the first tile has landed.)
-      int ph = (int)__ldcg(p.ws.phase);
-      grid_dependency_wait();
-      const int ph_now = (int)__ldcg(p.ws.phase);
-      TensorMeta meta = load_meta(p, a, cr.tensor, ph, STRICT, false, &ti_first);
-      if (ph_now != ph) {
-        ph = ph_now;
-        meta = load_meta(p, a, cr.tensor, ph, STRICT, false, &ti_first);
-      }
-      if (cr.index == 0) record_exponents(p, cr.tensor, ph, STRICT, meta);
-      TensorState* amax_now = p.ws.state + (size_t)ph * p.ws.slab;
-      int issued = 0;
-      // The ring: pages from `head` on are free, tiles are released in the order they were
-      // issued, `oldest` is the first tile whose pages have not been taken back yet.
-      int head = 0, free_pages = kPages, oldest = 0;
-      bool gave_up = false;
-      for (int i = 0; i < n_my; ++i) {
-        const int slot = i % kSlots;
-        ChunkRef cr2{-1, -1};
-        if (i + 2 < n_my) cr2 = p.ws.chunks[tile0 + (i + 2) * stride];
-        TensorMeta meta1 = meta;
-        if (i + 1 < n_my && cr1.tensor != cr.tensor) meta1 = load_meta(p, a, cr1.tensor, ph, STRICT, cr1.index == 0);
-
-        const TensorInfo& ti = meta.ti;
-        const int tbytes = ti.theta_bits >> 3, cbytes = ti.comp_bits >> 3;
-        // where the three arrays go (g, theta, c), and how many pages that takes including
-        // those skipped when a run does not fit before the end of the ring
-        constexpr int gbytes = GB / 8;
-        // kChunk == kPageBytes: an array of b-byte elements takes b pages (2b with the large tiles)
-        const int big = (ti.theta_bits == 8 && p.chunk8 != kChunk) ? 1 : 0;
-        const int chunk = kChunk << big;
-        const int run[3] = {gbytes << big, tbytes << big, cbytes << big};
-        int page[3] = {0, 0, 0}, h2 = head, need = 0;
-#pragma unroll
-        for (int r = 0; r < 3; ++r) {
-          if (run[r] == 0) continue;
-          if (h2 + run[r] > kPages) { need += kPages - h2; h2 = 0; }
-          page[r] = h2;
-          h2 += run[r];
-          need += run[r];
-        }
-        if (h2 == kPages) h2 = 0;
-        // take back pages, descriptor slots and scans from the oldest tiles until this one fits
-        while (free_pages < need || i - oldest >= kSlots) {
-          const int os = oldest % kSlots;
-          if (!mbar_wait(&sh->empty[os], (unsigned)(oldest / kSlots) & 1u, &sh->abort_flag)) {
-            gave_up = true;
-            break;
-          }
-          take_back(p, acc, amax_now, &sh->scan[os], sh->desc[os].tensor);
-          free_pages += sh->slot_pages[os];
-          ++oldest;
-        }
-        if (gave_up) {
-          sh->abort_flag = 1;
-          atomicCAS(p.ws.error, 0u, (unsigned)kErrEmptyWait);
-          break;
-        }
-        head = h2;
-        free_pages -= need;
-        sh->slot_pages[slot] = need;
-
-        const long long first = (long long)cr.index << (13 + big);
-        const long long left = ti.numel - first;
-        const int count = left < (long long)chunk ? (int)left : chunk;
-        const int n_bulk = count & ~15;
-        // The copies go out first and the descriptor is written while they are on their way:
-        // the tile's barrier completes only when the bytes have landed AND the producer has
-        // arrived, and it arrives after the descriptor is in place.
-        unsigned char* const theta_g = static_cast<unsigned char*>(ti.theta) + first * tbytes;
-        unsigned char* const comp_g = ti.comp ? static_cast<unsigned char*>(ti.comp) + first * cbytes : nullptr;
-        const unsigned char* const grad_g = static_cast<const unsigned char*>(meta.grad) + first * gbytes;
-        if (n_bulk > 0) {
-          mbar_expect_tx(&sh->full[slot], (unsigned)(n_bulk * (tbytes + cbytes + gbytes)));
-          bulk_load(smem + page[1] * kPageBytes, theta_g, (unsigned)(n_bulk * tbytes), &sh->full[slot]);
-          if (cbytes)
-            bulk_load(smem + page[2] * kPageBytes, comp_g, (unsigned)(n_bulk * cbytes), &sh->full[slot]);
-          // Gradients are read once.  When theta and c of the whole list fit in L2, letting
-          // the gradients leave it first keeps the state resident from step to step.
-          if (p.grad_evict_first)
-            bulk_load_hint(smem + page[0] * kPageBytes, grad_g, (unsigned)(n_bulk * gbytes), &sh->full[slot],
-                           grad_policy);
-          else
-            bulk_load(smem + page[0] * kPageBytes, grad_g, (unsigned)(n_bulk * gbytes), &sh->full[slot]);
-        }
-        const StepCoef coef = make_coef(ti, meta.e_in, meta.e_out, meta.ec_in, meta.ec_out, meta.lr, GB, meta.eg,
-                                        STRICT ? 1 : 0);
-        // fixed-point gradients: the exact-fp32 path multiplies the mantissa by scale * 2^eg,
-        // which must itself be exact (a normal number); otherwise the tile takes the general path
-        float scale_hot = coef.scale;
-        bool scale_ok = true;
-        if constexpr (GB != 32) {
-          const int ex = (int)((__float_as_uint(coef.scale) >> 23) & 0xffu);
-          scale_ok = ex != 0 && ex + meta.eg >= 1 && ex + meta.eg <= 254;
-          if (scale_ok) scale_hot = __int_as_float(__float_as_int(coef.scale) + (meta.eg << 23));
-        }
-        TileDesc& td = sh->desc[slot];
-        td.scale = scale_hot;
-        td.pow2s_neg = -pow2_float(coef.s);
-        td.inv2s = pow2_float(-coef.s);
-        td.pow2dc = pow2_float(-coef.delta_c);
-        td.theta = theta_g;
-        td.comp = comp_g;
-        td.tensor = cr.tensor;
-        td.n_bulk = n_bulk;
-        td.count = count;
-        td.flags = ((ti.theta_bits == 16 ? 3 : 0) + (ti.comp_bits >> 3)) |
-                   ((coef.delta == 0 && scale_ok && (!STRICT || coef.s >= 0)) ? kFlagSteady : 0) |
-                   // a coarser grid splits theta's mantissa at bit delta: that needs delta <= theta_bits - 1
-                   ((!STRICT && coef.delta != 0 && scale_ok && coef.delta <= ti.theta_bits - 1) ? kFlagRegrid : 0) |
-                   (page[1] << kFlagThetaPageShift) |
-                   (page[2] << kFlagCompPageShift) | (page[0] << kFlagGradPageShift);
-        td.coef = coef;
-        td.grad = grad_g;
-        mbar_arrive(&sh->full[slot]);
-        issued = i + 1;
-        cr = cr1;
-        cr1 = cr2;
-        meta = meta1;
-      }
-      // Collect the scans of the tiles still in the ring and publish.  The same waits make
-      // sure that every copy this block started has landed before the block exits.
-      for (int i = oldest; i < issued; ++i) {
-        const int os = i % kSlots;
-        if (mbar_wait(&sh->empty[os], (unsigned)(i / kSlots) & 1u, &sh->abort_flag))
-          take_back(p, acc, amax_now, &sh->scan[os], sh->desc[os].tensor);
-        else
-          mbar_wait(&sh->full[os], (unsigned)(i / kSlots) & 1u, &sh->never);
-      }
-      publish(p, acc, amax_now);
+  static __device__ __forceinline__ void record(const Params& p, int t, int ph, const Meta& m) {
+    record_exponents(p, t, ph, STRICT, m);
+  }
+  // Tensors with 8-bit theta take tiles of 2 * kChunk elements in lists long enough to keep
+  // every block busy with them (one vector per thread and tile leaves the per-tile work of a
+  // consumer -- wait, descriptor, scans, arrive -- a third of its instructions).
+  static __device__ __forceinline__ int tile_shift(const Params& p, const Meta& m) {
+    return (m.ti.theta_bits == 8 && p.chunk8 != kChunk) ? 1 : 0;
+  }
+  static __device__ __forceinline__ void streams(const Meta& m, const unsigned char* (&base)[kStreams],
+                                                 int (&bytes)[kStreams]) {
+    base[0] = static_cast<const unsigned char*>(m.grad);
+    bytes[0] = GB / 8;
+    base[1] = static_cast<const unsigned char*>(m.ti.theta);
+    bytes[1] = m.ti.theta_bits >> 3;
+    base[2] = static_cast<const unsigned char*>(m.ti.comp);
+    bytes[2] = m.ti.comp_bits >> 3;
+  }
+  static __device__ __forceinline__ void fill_desc(TileDesc& td, const Params& p, const Meta& meta, int tensor,
+                                                   int count, int n_bulk, const int (&page)[kStreams],
+                                                   const unsigned char* const (&gptr)[kStreams]) {
+    const TensorInfo& ti = meta.ti;
+    const StepCoef coef = make_coef(ti, meta.e_in, meta.e_out, meta.ec_in, meta.ec_out, meta.lr, GB, meta.eg,
+                    STRICT ? 1 : 0);
+    // fixed-point gradients: the exact-fp32 path multiplies the mantissa by scale * 2^eg,
+    // which must itself be exact (a normal number); otherwise the tile takes the general path
+    float scale_hot = coef.scale;
+    bool scale_ok = true;
+    if constexpr (GB != 32) {
+      const int ex = (int)((__float_as_uint(coef.scale) >> 23) & 0xffu);
+      scale_ok = ex != 0 && ex + meta.eg >= 1 && ex + meta.eg <= 254;
+      if (scale_ok) scale_hot = __int_as_float(__float_as_int(coef.scale) + (meta.eg << 23));
+    }
+    td.scale = scale_hot;
+    td.pow2s_neg = -pow2_float(coef.s);
+    td.inv2s = pow2_float(-coef.s);
+    td.pow2dc = pow2_float(-coef.delta_c);
+    td.theta = const_cast<unsigned char*>(gptr[1]);
+    td.comp = const_cast<unsigned char*>(gptr[2]);
+    td.tensor = tensor;
+    td.n_bulk = n_bulk;
+    td.count = count;
+    td.flags = ((ti.theta_bits == 16 ? 3 : 0) + (ti.comp_bits >> 3)) |
+           ((coef.delta == 0 && scale_ok && (!STRICT || coef.s >= 0)) ? kFlagSteady : 0) |
+           // a coarser grid splits theta's mantissa at bit delta: that needs delta <= theta_bits - 1
+           ((!STRICT && coef.delta != 0 && scale_ok && coef.delta <= ti.theta_bits - 1) ? kFlagRegrid : 0) |
+           (page[1] << kFlagThetaPageShift) |
+           (page[2] << kFlagCompPageShift) | (page[0] << kFlagGradPageShift);
+    td.coef = coef;
+    td.grad = gptr[0];
+  }
+  // One consumer thread's share of a tile: the exact-fp32 paths per format, the scans of its
+  // warp added to the tile's slot.
+  static __device__ __forceinline__ void consume(const TileDesc* td, TileScan* scan, unsigned char* smem, int ctid,
+                                                 int lane) {
+    unsigned char* st = smem;
+    if (!STRICT && (td->flags & kFlagRegrid)) {
+      regrid_tile<GB>(td, scan, st);
     } else {
-      grid_dependency_wait();
-    }
-  } else {
-    // ------------------------------------------------------------------ consumers
-    grid_dependency_wait();
-    const int ctid = threadIdx.x;
-    const int stride = (int)gridDim.x;
-    const int n_my = (p.tile_count - (int)blockIdx.x + stride - 1) / stride;
-    // Entry ticket (thread 0).  It is drawn after the block's first tile has landed, i.e. after
-    // the producer has read the phase word (it arrives on the tile's barrier later than that
-    // read returned, and the wait above has seen the arrival); the block that draws the last
-    // ticket therefore knows that every block of the step has read the word, and only then
-    // moves it on for the next step.  The answer is looked at when the block's tiles are done.
-    unsigned int ticket = 0u, ph0 = 0u;
-    for (int i = 0; i < n_my; ++i) {
-      const int stage = i % kSlots, use = i / kSlots;
-      if (!mbar_wait(&sh->full[stage], (unsigned)use & 1u, &sh->abort_flag)) {
-        if (lane == 0) {
-          sh->abort_flag = 1;
-          atomicCAS(p.ws.error, 0u, (unsigned)kErrFullWait);
-        }
-        break;
+      const TileHot h = load_tile_hot(td);
+      float amax_t = 0.0f, amax_c = 0.0f;
+      bool wrote_stage;
+      switch (h.flags & kFlagFormatMask) {
+        case 0: wrote_stage = consume_tile<8, 0, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 1: wrote_stage = consume_tile<8, 8, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 2: wrote_stage = consume_tile<8, 16, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 3: wrote_stage = consume_tile<16, 0, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        case 4: wrote_stage = consume_tile<16, 8, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
+        default: wrote_stage = consume_tile<16, 16, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
       }
-      if (i == 0 && threadIdx.x == 0 && p.advance) {
-        ph0 = __ldcg(p.ws.phase);
-        ticket = atomicAdd(p.ws.phase + 1 + (ph0 >> 8), 1u) + 1u;
-      }
-      const TileDesc* td = &sh->desc[stage];
-      TileScan* scan = &sh->scan[stage];
-      unsigned char* st = smem;
-      if (!STRICT && (td->flags & kFlagRegrid)) {
-        regrid_tile<GB>(td, scan, st);
-      } else {
-        const TileHot h = load_tile_hot(td);
-        float amax_t = 0.0f, amax_c = 0.0f;
-        bool wrote_stage;
-        switch (h.flags & kFlagFormatMask) {
-          case 0: wrote_stage = consume_tile<8, 0, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
-          case 1: wrote_stage = consume_tile<8, 8, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
-          case 2: wrote_stage = consume_tile<8, 16, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
-          case 3: wrote_stage = consume_tile<16, 0, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
-          case 4: wrote_stage = consume_tile<16, 8, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
-          default: wrote_stage = consume_tile<16, 16, GB, STRICT>(h, td, st, ctid, scan, amax_t, amax_c); break;
-        }
-        add_warp_scans(scan, lane, amax_t, amax_c);
-        // if the general path wrote into the stage, order those writes before the bulk copy
-        // that refills it
-        if (wrote_stage) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->empty[stage]);
-    }
-    if (threadIdx.x == 0 && ticket == gridDim.x) {
-      p.ws.phase[1] = 0u;
-      p.ws.phase[0] = ph0 == 2u ? 0u : ph0 + 1u;
+      add_warp_scans(scan, lane, amax_t, amax_c);
+      // if the general path wrote into the stage, order those writes before the bulk copy
+      // that refills it
+      if (wrote_stage) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
   }
+};
 
-  // Nothing follows: the step is complete when every block's producer has published its
-  // scans; the exponents they imply are worked out by the blocks of the next step.
-}
+constexpr size_t kSharedBytes = ring_shared_bytes<PlainPolicy<32, false>>();   // the same for every plain variant
 
 __global__ void __launch_bounds__(kBlockThreads, 1)
 ksgd_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ InlineArgs a) {
-  step_body<32, false>(p, a);
+  ring_step<PlainPolicy<32, false>>(p, a);
 }
 
 template <int GB>
 __global__ void __launch_bounds__(kBlockThreads, 1)
 ksgd_step_qgrad_kernel(const __grid_constant__ StepParams p, const __grid_constant__ QGradArgs a) {
-  step_body<GB, false>(p, a);
+  ring_step<PlainPolicy<GB, false>>(p, a);
 }
 
 __global__ void __launch_bounds__(kBlockThreads, 1)
 ksgd_strict_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ InlineArgs a) {
-  step_body<32, true>(p, a);
+  ring_step<PlainPolicy<32, true>>(p, a);
 }
 
 template <int GB>
 __global__ void __launch_bounds__(kBlockThreads, 1)
 ksgd_strict_step_qgrad_kernel(const __grid_constant__ StepParams p, const __grid_constant__ QGradArgs a) {
-  step_body<GB, true>(p, a);
+  ring_step<PlainPolicy<GB, true>>(p, a);
 }
 
 // Per-step arguments of long lists: written to the workspace from kernel parameters.

@@ -60,10 +60,52 @@ cudaError_t launch_step_kernel(void (*kernel)(KArgs...), unsigned grid, unsigned
 // kahan_sgd_amax fetches them with one copy.
 struct Layout {
   size_t phase, state, counters, error, stats_end;
-  size_t info, grad_ptr, lr, exp_grad, chunks, total;
+  size_t info, grad_ptr, lr, exp_grad /* the optimizers' extra per-tensor word: mu */, chunks, total;
   long long n_chunks;
   int slab;                // records per phase slab (a slab is a multiple of 128 bytes)
 };
+
+// The same layout for every optimizer: phase word, three slabs of per-step records (the
+// policy's State), counters, error word (all fetched by the read-out in one copy), then the
+// tensor table (the policy's Info), the per-step arguments of long lists, the tile table.
+Layout make_ring_layout(int32_t n, long long n_chunks, size_t state_bytes, size_t info_bytes, int n_counts) {
+  Layout L{};
+  L.n_chunks = n_chunks;
+  L.slab = (int)(align_up(state_bytes * (size_t)n, 128) / state_bytes);
+  size_t o = 0;
+  L.phase = o;     o += 128;
+  L.state = o;     o += state_bytes * 3 * L.slab;
+  L.counters = o;  o += sizeof(unsigned long long) * n_counts * n;
+  L.error = o;     o += 8;
+  L.stats_end = o;
+  o = align_up(o, 16);
+  L.info = o;      o += info_bytes * n;
+  o = align_up(o, 16);
+  L.grad_ptr = o;  o += sizeof(const float*) * n;
+  L.lr = o;        o += sizeof(float) * n;
+  L.exp_grad = o;  o += sizeof(int) * n;
+  o = align_up(o, 16);
+  L.chunks = o;    o += sizeof(ChunkRef) * (size_t)n_chunks;
+  L.total = align_up(o, 256);
+  return L;
+}
+
+// Tile table of a list cut into tiles of kChunk elements, into `chunks`; returns the count.
+long long plain_tile_count(const ksgd_tensor_desc* d, int32_t n) {
+  long long chunks = 0;
+  for (int32_t i = 0; i < n; ++i) chunks += (d[i].numel + kChunk - 1) / kChunk;
+  return chunks;
+}
+
+// What every init needs from the device, and the upload of the finished image.
+struct DeviceFacts { int sms = 0, l2_bytes = 0; };
+cudaError_t query_device(DeviceFacts& f) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&f.sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&f.l2_bytes, cudaDevAttrL2CacheSize, dev);
+  return e;
+}
 
 // Tile size of a tensor, given the list's tile size for 8-bit theta.
 inline long long tile_elems(const ksgd_tensor_desc& t, int chunk8) { return t.theta_bits == 8 ? chunk8 : kChunk; }
@@ -80,26 +122,9 @@ int pick_chunk8(const ksgd_tensor_desc* d, int32_t n) {
 }
 
 Layout make_layout(const ksgd_tensor_desc* d, int32_t n, int chunk8) {
-  Layout L{};
   long long chunks = 0;
   for (int32_t i = 0; i < n; ++i) chunks += (d[i].numel + tile_elems(d[i], chunk8) - 1) / tile_elems(d[i], chunk8);
-  L.n_chunks = chunks;
-  L.slab = (int)(align_up(sizeof(TensorState) * (size_t)n, 128) / sizeof(TensorState));
-  size_t o = 0;
-  L.phase = o;     o += 128;
-  L.state = o;     o += sizeof(TensorState) * 3 * L.slab;
-  L.counters = o;  o += sizeof(unsigned long long) * 3 * n;
-  L.error = o;     o += 8;
-  L.stats_end = o;
-  o = align_up(o, 16);
-  L.info = o;      o += sizeof(TensorInfo) * n;
-  L.grad_ptr = o;  o += sizeof(const float*) * n;
-  L.lr = o;        o += sizeof(float) * n;
-  L.exp_grad = o;  o += sizeof(int) * n;
-  o = align_up(o, 16);
-  L.chunks = o;    o += sizeof(ChunkRef) * (size_t)chunks;
-  L.total = align_up(o, 256);
-  return L;
+  return make_ring_layout(n, chunks, sizeof(TensorState), sizeof(TensorInfo), 3);
 }
 
 // Device-side view of a workspace at `b`.
@@ -829,39 +854,8 @@ int upload_long_list(cudaStream_t stream, int32_t n, const float* const* grads, 
   return KSGD_OK;
 }
 
-struct MomLayout {
-  size_t exp_cur, exp_next, expv_cur, expv_next, amax_last, counters, error, stats_end;
-  size_t amax_acc, info, chunks, ticket, grad_ptr, lr, mu, total;
-  long long n_chunks;
-};
-
-MomLayout make_mom_layout(const ksgd_tensor_desc* d, int32_t n) {
-  MomLayout L{};
-  long long chunks = 0;
-  for (int32_t i = 0; i < n; ++i) chunks += (d[i].numel + kChunk - 1) / kChunk;
-  L.n_chunks = chunks;
-  size_t o = 0;
-  L.exp_cur = o;   o += sizeof(int) * n;
-  L.exp_next = o;  o += sizeof(int) * n;
-  L.expv_cur = o;  o += sizeof(int) * n;
-  L.expv_next = o; o += sizeof(int) * n;
-  L.amax_last = o; o += sizeof(unsigned int) * 3 * n;
-  o = align_up(o, 8);
-  L.counters = o;  o += sizeof(unsigned long long) * 4 * n;
-  L.error = o;     o += 8;
-  L.stats_end = o;
-  L.amax_acc = o;  o += sizeof(unsigned int) * 3 * n;
-  o = align_up(o, 16);
-  L.info = o;      o += sizeof(mom::TensorInfo) * n;
-  o = align_up(o, 16);
-  L.chunks = o;    o += sizeof(ChunkRef) * (size_t)chunks;
-  o = align_up(o, 16);
-  L.ticket = o;    o += 16;
-  L.grad_ptr = o;  o += sizeof(float*) * n;
-  L.lr = o;        o += sizeof(float) * n;
-  L.mu = o;        o += sizeof(float) * n;
-  L.total = align_up(o, 256);
-  return L;
+Layout make_mom_layout(const ksgd_tensor_desc* d, int32_t n) {
+  return make_ring_layout(n, plain_tile_count(d, n), sizeof(mom::TensorState), sizeof(mom::TensorInfo), 4);
 }
 
 int validate_momentum(const ksgd_tensor_desc* d, const ksgd_momentum_desc* m, int32_t n) {
@@ -883,7 +877,8 @@ int validate_momentum(const ksgd_tensor_desc* d, const ksgd_momentum_desc* m, in
 }  // namespace
 
 struct ksgd_momentum_handle {
-  MomLayout layout;
+  Layout layout;
+  std::vector<int32_t> theta_bits, mom_bits;
   mom::StepParams params;
   char* ws_base;
   cudaStream_t stream;
@@ -908,7 +903,7 @@ int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* 
   if (mode != KSGD_EXP_FIXED && mode != KSGD_EXP_AMAX) return KSGD_ERR_MODE;
   if (!workspace) return KSGD_ERR_NULL;
   if (reinterpret_cast<uintptr_t>(workspace) % 256) return KSGD_ERR_ALIGN;
-  const MomLayout L = make_mom_layout(descs, n_tensors);
+  const Layout L = make_mom_layout(descs, n_tensors);
   if (workspace_bytes < L.total) return KSGD_ERR_WORKSPACE;
 
   ksgd_momentum_handle* h = new (std::nothrow) ksgd_momentum_handle();
@@ -919,21 +914,20 @@ int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* 
   h->stream = static_cast<cudaStream_t>(cuda_stream);
   h->stats_host.resize(L.stats_end);
 
+  // Host image: phase 0; in the records the first step reads (slab 2) the exponents of the
+  // stored mantissas and, as overrides, the exponents the first step must write.
   std::vector<unsigned char> img(L.total, 0);
-  int* e_cur = reinterpret_cast<int*>(img.data() + L.exp_cur);
-  int* e_next = reinterpret_cast<int*>(img.data() + L.exp_next);
-  int* ev_cur = reinterpret_cast<int*>(img.data() + L.expv_cur);
-  int* ev_next = reinterpret_cast<int*>(img.data() + L.expv_next);
+  mom::TensorState* last = reinterpret_cast<mom::TensorState*>(img.data() + L.state) + 2 * (size_t)L.slab;
   mom::TensorInfo* info = reinterpret_cast<mom::TensorInfo*>(img.data() + L.info);
   ChunkRef* chunks = reinterpret_cast<ChunkRef*>(img.data() + L.chunks);
   long long c = 0;
   double state_bytes = 0.0;
   for (int32_t i = 0; i < n_tensors; ++i) {
     const ksgd_tensor_desc& t = descs[i];
-    e_cur[i] = t.exp_theta;
-    e_next[i] = t.exp_theta_next;
-    ev_cur[i] = mdescs[i].exp_mom;
-    ev_next[i] = mdescs[i].exp_mom_next;
+    last[i].exp_theta = t.exp_theta;
+    last[i].ovr_theta = t.exp_theta_next + kOvrBias;
+    last[i].exp_mom = mdescs[i].exp_mom;
+    last[i].ovr_mom = mdescs[i].exp_mom_next + kOvrBias;
     info[i].theta = t.theta;
     info[i].comp = t.comp;
     info[i].mom = mdescs[i].mom;
@@ -942,6 +936,8 @@ int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* 
     info[i].comp_bits = t.comp_bits;
     info[i].mom_bits = mdescs[i].mom_bits;
     info[i].s = t.comp_bits - 1 - t.overlap_k;
+    h->theta_bits.push_back(t.theta_bits);
+    h->mom_bits.push_back(mdescs[i].mom_bits);
     const long long nc = (t.numel + kChunk - 1) / kChunk;
     for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
     state_bytes += (double)t.numel * ((t.theta_bits + t.comp_bits + mdescs[i].mom_bits) / 8);
@@ -949,29 +945,25 @@ int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* 
 
   mom::Workspace& w = h->params.ws;
   char* b = h->ws_base;
-  w.exp_cur = reinterpret_cast<int*>(b + L.exp_cur);
-  w.exp_next = reinterpret_cast<int*>(b + L.exp_next);
-  w.expv_cur = reinterpret_cast<int*>(b + L.expv_cur);
-  w.expv_next = reinterpret_cast<int*>(b + L.expv_next);
-  w.amax_last = reinterpret_cast<unsigned int*>(b + L.amax_last);
+  w.phase = reinterpret_cast<unsigned int*>(b + L.phase);
+  w.state = reinterpret_cast<mom::TensorState*>(b + L.state);
+  w.slab = L.slab;
   w.counters = reinterpret_cast<unsigned long long*>(b + L.counters);
   w.error = reinterpret_cast<unsigned int*>(b + L.error);
-  w.amax_acc = reinterpret_cast<unsigned int*>(b + L.amax_acc);
   w.info = reinterpret_cast<mom::TensorInfo*>(b + L.info);
   w.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
-  w.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
   w.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
   w.lr = reinterpret_cast<float*>(b + L.lr);
-  w.mu = reinterpret_cast<float*>(b + L.mu);
+  w.mu = reinterpret_cast<float*>(b + L.exp_grad);
   h->params.n_tensors = n_tensors;
-  h->params.n_chunks = (int)L.n_chunks;
+  h->params.tile_begin = 0;
+  h->params.tile_count = (int)L.n_chunks;
   h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
   h->params.inline_args = n_tensors <= kInlineArgs ? 1 : 0;
+  h->params.advance = 1;
 
-  int dev = 0, sms = 0, l2_bytes = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, dev);
+  DeviceFacts dev;
+  cudaError_t e = query_device(dev);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(mom::ksgd_momentum_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)mom::kSharedBytes);
@@ -979,8 +971,8 @@ int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* 
     delete h;
     return cuda_fail(e, "device query");
   }
-  h->grid = (int)(L.n_chunks < (long long)sms ? L.n_chunks : (long long)sms);
-  h->params.grad_evict_first = state_bytes <= 0.8 * (double)l2_bytes ? 1 : 0;
+  h->grid = (int)(L.n_chunks < (long long)dev.sms ? L.n_chunks : (long long)dev.sms);
+  h->params.grad_evict_first = state_bytes <= 0.8 * (double)dev.l2_bytes ? 1 : 0;
 
   e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
@@ -1021,19 +1013,32 @@ int kahan_sgd_momentum_amax(ksgd_momentum_handle* h, uint32_t* amax_theta, uint3
                             int32_t* exp_mom_cur, int32_t* exp_mom_next, uint64_t* n_sat_theta,
                             uint64_t* n_sat_comp, uint64_t* n_sat_mom, uint64_t* n_nonfinite) {
   if (!h) return KSGD_ERR_NULL;
-  const MomLayout& L = h->layout;
+  const Layout& L = h->layout;
   KSGD_CUDA(cudaMemcpyAsync(h->stats_host.data(), h->ws_base, L.stats_end, cudaMemcpyDeviceToHost,
                             h->stream));
   KSGD_CUDA(cudaStreamSynchronize(h->stream));
   const unsigned char* b = h->stats_host.data();
   const size_t n = (size_t)h->n;
-  if (exp_theta_cur) std::memcpy(exp_theta_cur, b + L.exp_cur, 4 * n);
-  if (exp_theta_next) std::memcpy(exp_theta_next, b + L.exp_next, 4 * n);
-  if (exp_mom_cur) std::memcpy(exp_mom_cur, b + L.expv_cur, 4 * n);
-  if (exp_mom_next) std::memcpy(exp_mom_next, b + L.expv_next, 4 * n);
-  if (amax_theta) std::memcpy(amax_theta, b + L.amax_last, 4 * n);
-  if (amax_comp) std::memcpy(amax_comp, b + L.amax_last + 4 * n, 4 * n);
-  if (amax_mom) std::memcpy(amax_mom, b + L.amax_last + 8 * n, 4 * n);
+  unsigned int ph = 0;
+  std::memcpy(&ph, b + L.phase, 4);
+  if (ph > 2) return KSGD_ERR_DEVICE;
+  // the records of the last finished step; the exponents the coming step will write are the
+  // overrides if set, else what the scans imply (the rule the kernel applies)
+  const mom::TensorState* last = reinterpret_cast<const mom::TensorState*>(b + L.state) + ((ph + 2) % 3) * (size_t)L.slab;
+  const int mode = h->params.amax_mode;
+  for (size_t i = 0; i < n; ++i) {
+    const mom::TensorState& r = last[i];
+    if (amax_theta) amax_theta[i] = r.amax[0];
+    if (amax_comp) amax_comp[i] = r.amax[1];
+    if (amax_mom) amax_mom[i] = r.amax[2];
+    if (exp_theta_cur) exp_theta_cur[i] = r.exp_theta;
+    if (exp_mom_cur) exp_mom_cur[i] = r.exp_mom;
+    if (exp_theta_next)
+      exp_theta_next[i] = r.ovr_theta ? r.ovr_theta - kOvrBias : next_exponent(r.amax[0], h->theta_bits[i], r.exp_theta, mode);
+    if (exp_mom_next)
+      exp_mom_next[i] = r.ovr_mom ? r.ovr_mom - kOvrBias
+                                  : mom::next_exponent_velocity(r.amax[2], h->mom_bits[i], r.exp_mom, mode);
+  }
   if (n_sat_theta) std::memcpy(n_sat_theta, b + L.counters, 8 * n);
   if (n_sat_comp) std::memcpy(n_sat_comp, b + L.counters + 8 * n, 8 * n);
   if (n_sat_mom) std::memcpy(n_sat_mom, b + L.counters + 16 * n, 8 * n);

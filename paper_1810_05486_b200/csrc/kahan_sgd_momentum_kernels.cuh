@@ -6,10 +6,10 @@
 // and three max scans per tensor (|P|, |Rq|, |V|) that steer the exponents of theta and of
 // the velocity independently.
 //
-// Same structure as ksgd_step_kernel (persistent blocks, one producer thread streaming
-// tiles into a paged shared-memory ring with bulk asynchronous copies, sixteen consumer
-// warps, producer-side publishing of the scans, exponent choice in the last block), with a
-// fourth array per tile.  HBM traffic: 2*m/8 + 2*n/8 + 2*b/8 + 4 bytes per parameter.
+// The persistent grid, the paged shared-memory ring, the scan publishing and the state that
+// steps hand to one another are those of kahan_sgd_ring.cuh; this file is the policy: four
+// arrays per tile (gradient, theta, c, v), the arithmetic of an element, three scans and two
+// exponents per tensor.  HBM traffic: 2*m/8 + 2*n/8 + 2*b/8 + 4 bytes per parameter.
 #pragma once
 
 #include "kahan_sgd_kernels.cuh"
@@ -28,18 +28,24 @@ struct TensorInfo {
   int s;       // grid distance: exp_comp = exp_theta - s
 };
 
+// What a step leaves behind for one tensor (see kahan_sgd_ring.cuh): one 32-byte record.
+struct __align__(32) TensorState {
+  int exp_theta;          // exponents as this step wrote them
+  int exp_mom;
+  unsigned int amax[3];   // this step's max scans: |P|, |Rq|, |V|
+  int ovr_theta;          // exponents the NEXT step must write instead of those the scans give
+  int ovr_mom;            //   (value + kOvrBias, 0 = none; set at init)
+  int pad;
+};
+
 struct Workspace {
-  int* exp_cur;                    // [n]  theta
-  int* exp_next;                   // [n]
-  int* expv_cur;                   // [n]  velocity
-  int* expv_next;                  // [n]
-  unsigned int* amax_last;         // [3n] theta | comp | mom, of the last finished step
+  unsigned int* phase;             // [0] phase of the coming step; [1] entry tickets of the running step
+  TensorState* state;              // [3][slab]
+  int slab;
   unsigned long long* counters;    // [4n] sat_theta | sat_comp | sat_mom | nonfinite
   unsigned int* error;             // [1]
-  unsigned int* amax_acc;          // [3n]
   TensorInfo* info;                // [n]
   ChunkRef* chunks;                // [n_chunks]
-  unsigned int* ticket;
   const float** grad_ptr;          // [n] per-step arguments for lists longer than kInlineArgs
   float* lr;                       // [n]
   float* mu;                       // [n]
@@ -48,10 +54,11 @@ struct Workspace {
 struct StepParams {
   Workspace ws;
   int n_tensors;
-  int n_chunks;
+  int tile_begin, tile_count;      // all tiles of the list
   int amax_mode;
   int grad_evict_first;
   int inline_args;                 // 1: grads/lrs/mus are in the StepArgs parameter
+  int advance;                     // 1 (every launch is a whole step)
 };
 
 struct StepArgs {                  // per-step arguments, passed as a kernel parameter
@@ -62,10 +69,7 @@ struct StepArgs {                  // per-step arguments, passed as a kernel par
 
 // Twelve consumer warps (three per scheduler, plus the producer's) leave 128 registers per
 // thread: a vector of eight elements with three mantissa arrays then stays in registers.
-#ifndef KSGD_MOM_WARPS
-#define KSGD_MOM_WARPS 12
-#endif
-constexpr int kWarps = KSGD_MOM_WARPS;         // consumer warps; one more warp produces
+constexpr int kWarps = 12;                     // consumer warps; one more warp produces
 constexpr int kThreads = 32 * kWarps;
 constexpr int kBlock = kThreads + 32;
 
@@ -100,6 +104,7 @@ constexpr int kFormatMask = 7;       // bit 0: theta 16, bit 1: comp 16, bit 2: 
 constexpr int kSteady = 8;
 constexpr int kThetaPageShift = 8, kCompPageShift = 13, kGradPageShift = 18, kMomPageShift = 23;
 
+// Three maxima, then four counts: the order the ring expects.
 struct TileScan {
   unsigned int amax_t, amax_c, amax_v, n_sat_t, n_sat_c, n_sat_v, n_nonfinite, pad;
 };
@@ -201,33 +206,26 @@ struct SteadyCoef {
 // theta', c' and v' are the low bits of Pm, r0 + M and Vm.  Returns false, nothing stored,
 // if a value could leave the exact range or a clamp is needed.
 template <int TB, int CB, int VB>
-__device__ __forceinline__ bool update_vector(Pack<TB> pt, Pack<CB> pc, Pack<VB> pv, const Pack<32>& pg,
-                                              const SteadyCoef& k, Pack<TB>& ot, Pack<CB>& oc, Pack<VB>& ov,
-                                              float& amax_t, float& amax_c, float& amax_v) {
+__device__ __forceinline__ bool update_vector(const Pack<TB>& pt, const Pack<CB>& pc, const Pack<VB>& pv,
+                                              const Pack<32>& pg, const SteadyCoef& k, Pack<TB>& ot, Pack<CB>& oc,
+                                              Pack<VB>& ov, float& amax_t, float& amax_c, float& amax_v) {
   constexpr int V = 8;
-  constexpr float bias_t = (float)(1 << (TB - 1)), bias_c = (float)(1 << (CB - 1)),
-                  bias_v = (float)(1 << (VB - 1));
-  constexpr float Mt = kMagic + bias_t;
-  flip_signs<TB>(pt);
-  flip_signs<CB>(pc);
-  flip_signs<VB>(pv);
-  // theta stays biased (qtB = M + 2^(TB-1) + Qt, the bias is even so ties fall as before; the
-  // packed result gets its sign bits flipped back); scans take two elements per instruction
+  // the scans take two elements per instruction
   float Pm[V], rm[V], Vm[V], va[2], ra[2];
-  float hiP = Mt, loP = Mt, aR = 0.0f, aV = 0.0f;
+  float hiP = kMagic, loP = kMagic, aR = 0.0f, aV = 0.0f;
 #pragma unroll
   for (int i = 0; i < V; ++i) {
-    const float qtB = magic_elem<TB>(pt, i);                                      // M + bias + Qt
-    const float qc = __fadd_rn(magic_elem<CB>(pc, i), -(kMagic + bias_c));        // Qc
-    const float qv = __fadd_rn(magic_elem<VB>(pv, i), -(kMagic + bias_v));        // Qv
+    const float qtM = magic_signed<TB>(pt, i);                                    // M + Qt
+    const float qc = __fadd_rn(magic_signed<CB>(pc, i), -kMagic);                 // Qc
+    const float qv = __fadd_rn(magic_signed<VB>(pv, i), -kMagic);                 // Qv
     const float g = __uint_as_float(pack_word(pg, i));
     const float y = __fmaf_rn(k.mu_s, qv, __fmul_rn(g, k.scale_v));
     const float vm = __fadd_rn(y, kMagic);              // M + rne(y)
     const float v = __fadd_rn(vm, -kMagic);             // Inf or NaN if y is
     const float d = __fadd_rn(__fmaf_rn(v, k.pow2k, kMagic), -kMagic);
     const float u = __fadd_rn(qc, -d);
-    const float P = __fmaf_rn(u, k.inv2s, qtB);
-    const float w = __fadd_rn(P, -qtB);
+    const float P = __fmaf_rn(u, k.inv2s, qtM);
+    const float w = __fadd_rn(P, -qtM);
     const float r0 = __fmaf_rn(w, k.pow2s_neg, u);
     Pm[i] = P;
     rm[i] = __fadd_rn(r0, kMagic);
@@ -241,7 +239,7 @@ __device__ __forceinline__ bool update_vector(Pack<TB> pt, Pack<CB> pc, Pack<VB>
       aR = max3(aR, ra[0], ra[1]);
     }
   }
-  const float aP = fmaxf(__fadd_rn(hiP, -Mt), __fadd_rn(Mt, -loP));
+  const float aP = fmaxf(__fadd_rn(hiP, -kMagic), __fadd_rn(kMagic, -loP));
   // |y| > 4e6 (where y + M stops being exact) shows as |V| far beyond QMAX_v, so the velocity
   // bound covers it; a NaN fails the same comparison
   if (!(aV <= k.qmax_v) | !(aV <= k.d_limit) | (aP > k.qmax_t)) return false;
@@ -249,7 +247,6 @@ __device__ __forceinline__ bool update_vector(Pack<TB> pt, Pack<CB> pc, Pack<VB>
   amax_c = fmaxf(amax_c, aR);
   amax_v = fmaxf(amax_v, aV);
   ot = pack_magic<TB, V>(Pm);
-  flip_signs<TB>(ot);
   oc = pack_magic<CB, V>(rm);
   ov = pack_magic<VB, V>(Vm);
   return true;
@@ -316,60 +313,13 @@ __device__ __forceinline__ bool consume_tile(const TileDesc* td, unsigned char* 
 // Exponent of the velocity for the next step.  The velocity's maximum moves with every
 // gradient, so it keeps its exponent while its largest mantissa stays in (QMAX/4, QMAX] and
 // otherwise takes the tight fit (coarser at once, finer only after a fourfold drop).
-__device__ __forceinline__ int next_exponent_velocity(unsigned int amax, int bits, int ev_out, int amax_mode) {
+__host__ __device__ __forceinline__ int next_exponent_velocity(unsigned int amax, int bits, int ev_out, int amax_mode) {
   const unsigned int q = (1u << (bits - 1)) - 1u;
   if (amax <= q && 4ull * amax > q) return ev_out;
   return next_exponent(amax, bits, ev_out, amax_mode);
 }
 
-struct __align__(128) BlockShared {
-  unsigned long long full[kSlots];
-  unsigned long long empty[kSlots];
-  TileDesc desc[kSlots];
-  TileScan scan[kSlots];
-  int slot_pages[kSlots];
-  int abort_flag;
-  int is_last;
-  int never;
-};
-
-constexpr size_t kSharedBytes = (size_t)kPages * kPageBytes + sizeof(BlockShared);
-
-struct ScanAcc {
-  int tensor = -1;
-  unsigned int amax_t = 0, amax_c = 0, amax_v = 0, n_sat_t = 0, n_sat_c = 0, n_sat_v = 0, n_nonfinite = 0;
-};
-
-__device__ __forceinline__ void publish(const StepParams& p, ScanAcc& acc) {
-  if (acc.tensor >= 0) {
-    const int t = acc.tensor, n = p.n_tensors;
-    if (acc.amax_t) atomicMax(&p.ws.amax_acc[t], acc.amax_t);
-    if (acc.amax_c) atomicMax(&p.ws.amax_acc[n + t], acc.amax_c);
-    if (acc.amax_v) atomicMax(&p.ws.amax_acc[2 * n + t], acc.amax_v);
-    if (acc.n_sat_t) atomicAdd(&p.ws.counters[t], (unsigned long long)acc.n_sat_t);
-    if (acc.n_sat_c) atomicAdd(&p.ws.counters[n + t], (unsigned long long)acc.n_sat_c);
-    if (acc.n_sat_v) atomicAdd(&p.ws.counters[2 * n + t], (unsigned long long)acc.n_sat_v);
-    if (acc.n_nonfinite) atomicAdd(&p.ws.counters[3 * n + t], (unsigned long long)acc.n_nonfinite);
-  }
-  acc = ScanAcc{};
-}
-
-__device__ __forceinline__ void take_back(const StepParams& p, ScanAcc& acc, TileScan* scan, int tensor) {
-  if (tensor != acc.tensor) {
-    publish(p, acc);
-    acc.tensor = tensor;
-  }
-  acc.amax_t = max(acc.amax_t, scan->amax_t);
-  acc.amax_c = max(acc.amax_c, scan->amax_c);
-  acc.amax_v = max(acc.amax_v, scan->amax_v);
-  acc.n_sat_t += scan->n_sat_t;
-  acc.n_sat_c += scan->n_sat_c;
-  acc.n_sat_v += scan->n_sat_v;
-  acc.n_nonfinite += scan->n_nonfinite;
-  scan->amax_t = scan->amax_c = scan->amax_v = 0u;
-  scan->n_sat_t = scan->n_sat_c = scan->n_sat_v = scan->n_nonfinite = 0u;
-}
-
+// What the producer knows about a tile's tensor.
 struct TensorMeta {
   TensorInfo ti;
   const float* grad;
@@ -377,224 +327,118 @@ struct TensorMeta {
   int e_in, e_out, ev_in, ev_out;
 };
 
-__device__ __forceinline__ TensorMeta load_meta(const StepParams& p, const StepArgs& a, int t) {
-  TensorMeta m;
-  m.ti = p.ws.info[t];
-  m.e_in = p.ws.exp_cur[t];
-  m.e_out = p.ws.exp_next[t];
-  m.ev_in = p.ws.expv_cur[t];
-  m.ev_out = p.ws.expv_next[t];
-  m.grad = p.inline_args ? a.grads[t] : p.ws.grad_ptr[t];
-  m.lr = p.inline_args ? a.lrs[t] : p.ws.lr[t];
-  m.mu = p.inline_args ? a.mus[t] : p.ws.mu[t];
-  return m;
-}
+struct Policy {
+  static constexpr int kStreams = 4;          // gradient, theta, c, v
+  static constexpr int kConsumerWarps = kWarps;
+  static constexpr int kAmax = 3, kCounts = 4;
+  using Params = StepParams;
+  using Info = TensorInfo;
+  using State = TensorState;
+  using TileDesc = mom::TileDesc;
+  using TileScan = mom::TileScan;
+  using Meta = TensorMeta;
+
+  // The exponents the tensor reads and writes in the step of phase ph, derived from the record
+  // the preceding step left (one 32-byte load), and the per-step arguments.
+  static __device__ __forceinline__ Meta load_meta(const Params& p, const StepArgs& a, int t, int ph, const Info* ti) {
+    Meta m;
+    m.ti = ti ? *ti : p.ws.info[t];
+    m.grad = p.inline_args ? a.grads[t] : p.ws.grad_ptr[t];
+    m.lr = p.inline_args ? a.lrs[t] : p.ws.lr[t];
+    m.mu = p.inline_args ? a.mus[t] : p.ws.mu[t];
+    const int prev = ph == 0 ? 2 : ph - 1;
+    const int4* rec = reinterpret_cast<const int4*>(&p.ws.state[(size_t)prev * p.ws.slab + t]);
+    const int4 r0 = __ldcg(rec), r1 = __ldcg(rec + 1);     // exp_theta exp_mom amax[0] amax[1] | amax[2] ovr_theta ovr_mom -
+    m.e_in = r0.x;
+    m.ev_in = r0.y;
+    m.e_out = r1.y ? r1.y - kOvrBias : next_exponent((unsigned)r0.z, m.ti.theta_bits, m.e_in, p.amax_mode);
+    m.ev_out = r1.z ? r1.z - kOvrBias : next_exponent_velocity((unsigned)r1.x, m.ti.mom_bits, m.ev_in, p.amax_mode);
+    return m;
+  }
+  static __device__ __forceinline__ void record(const Params& p, int t, int ph, const Meta& m) {
+    const int next = ph == 2 ? 0 : ph + 1;
+    TensorState* now = &p.ws.state[(size_t)ph * p.ws.slab + t];
+    now->exp_theta = m.e_out;
+    now->exp_mom = m.ev_out;
+    int4* nx = reinterpret_cast<int4*>(&p.ws.state[(size_t)next * p.ws.slab + t]);
+    nx[0] = make_int4(0, 0, 0, 0);
+    nx[1] = make_int4(0, 0, 0, 0);
+  }
+  static __device__ __forceinline__ int tile_shift(const Params&, const Meta&) { return 0; }
+  static __device__ __forceinline__ void streams(const Meta& m, const unsigned char* (&base)[kStreams],
+                                                 int (&bytes)[kStreams]) {
+    base[0] = reinterpret_cast<const unsigned char*>(m.grad);
+    bytes[0] = 4;
+    base[1] = static_cast<const unsigned char*>(m.ti.theta);
+    bytes[1] = m.ti.theta_bits >> 3;
+    base[2] = static_cast<const unsigned char*>(m.ti.comp);
+    bytes[2] = m.ti.comp_bits >> 3;
+    base[3] = static_cast<const unsigned char*>(m.ti.mom);
+    bytes[3] = m.ti.mom_bits >> 3;
+  }
+  static __device__ __forceinline__ void fill_desc(TileDesc& td, const Params&, const Meta& meta, int tensor, int count,
+                                                   int n_bulk, const int (&page)[kStreams],
+                                                   const unsigned char* const (&gptr)[kStreams]) {
+    const TensorInfo& ti = meta.ti;
+    const Coef coef = make_coef(ti, meta.e_in, meta.e_out, meta.ev_in, meta.ev_out, meta.lr, meta.mu);
+    // velocity LSB -> compensation LSBs as a float factor; beyond +-30 the steady path
+    // is never exact (k large) or the increment is always zero (k very negative)
+    const int kk = max(-40, min(30, coef.k));
+    td.scale_v = coef.scale_v;
+    td.mu_s = coef.mu_s;
+    td.pow2k = pow2_float(kk);
+    td.pow2s_neg = -pow2_float(coef.s);
+    td.inv2s = pow2_float(-coef.s);
+    td.qmax_t = (float)coef.qmax_t;
+    td.qmax_v = (float)coef.qmax_v;
+    td.d_limit = coef.k > 22 ? 0.5f : (coef.k > 0 ? 4000000.0f * pow2_float(-coef.k) : 4000000.0f);
+    td.theta = const_cast<unsigned char*>(gptr[1]);
+    td.comp = const_cast<unsigned char*>(gptr[2]);
+    td.mom = const_cast<unsigned char*>(gptr[3]);
+    td.n_bulk = n_bulk;
+    td.flags = ((ti.theta_bits == 16 ? 1 : 0) | (ti.comp_bits == 16 ? 2 : 0) | (ti.mom_bits == 16 ? 4 : 0)) |
+               (coef.delta == 0 ? kSteady : 0) | (page[1] << kThetaPageShift) |
+               (page[2] << kCompPageShift) | (page[0] << kGradPageShift) | (page[3] << kMomPageShift);
+    td.tensor = tensor;
+    td.count = count;
+    td.coef = coef;
+    td.grad = reinterpret_cast<const float*>(gptr[0]);
+  }
+  static __device__ __forceinline__ void consume(const TileDesc* td, TileScan* scan, unsigned char* smem, int ctid,
+                                                 int lane) {
+    float amax_t = 0.0f, amax_c = 0.0f, amax_v = 0.0f;
+    bool wrote_ring;
+    switch (td->flags & kFormatMask) {
+      case 0: wrote_ring = consume_tile<8, 8, 8>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+      case 1: wrote_ring = consume_tile<16, 8, 8>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+      case 2: wrote_ring = consume_tile<8, 16, 8>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+      case 3: wrote_ring = consume_tile<16, 16, 8>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+      case 4: wrote_ring = consume_tile<8, 8, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+      case 5: wrote_ring = consume_tile<16, 8, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+      case 6: wrote_ring = consume_tile<8, 16, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+      default: wrote_ring = consume_tile<16, 16, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
+    }
+    // the steady path's scans are exact integers below 2^23 held in floats
+    const unsigned int full = 0xffffffffu;
+    const unsigned int at = __reduce_max_sync(full, (unsigned int)amax_t);
+    const unsigned int ac = __reduce_max_sync(full, (unsigned int)amax_c);
+    const unsigned int av = __reduce_max_sync(full, (unsigned int)amax_v);
+    if (lane == 0) {
+      if (at) atomicMax(&scan->amax_t, at);
+      if (ac) atomicMax(&scan->amax_c, ac);
+      if (av) atomicMax(&scan->amax_v, av);
+    }
+    // if the general path wrote into the ring, order those writes before the bulk copy
+    // that refills the pages
+    if (wrote_ring) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+};
+
+constexpr size_t kSharedBytes = ring_shared_bytes<Policy>();
 
 __global__ void __launch_bounds__(kBlock, 1)
 ksgd_momentum_step_kernel(const __grid_constant__ StepParams p, const __grid_constant__ StepArgs a) {
-  extern __shared__ __align__(128) unsigned char smem[];
-  BlockShared* sh = reinterpret_cast<BlockShared*>(smem + (size_t)kPages * kPageBytes);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int stride = (int)gridDim.x;
-  const int n_my = ((int)p.n_chunks - (int)blockIdx.x + stride - 1) / stride;
-  grid_dependency_launch_dependents();
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kSlots; ++s) {
-      mbar_init(&sh->full[s], 1u);
-      mbar_init(&sh->empty[s], (unsigned)kWarps);
-    }
-    sh->abort_flag = 0;
-    sh->is_last = 0;
-    sh->never = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (threadIdx.x < kSlots * (int)(sizeof(TileScan) / 4))
-    reinterpret_cast<unsigned int*>(sh->scan)[threadIdx.x] = 0u;
-  __syncthreads();
-
-  if (warp == kWarps) {
-    // ------------------------------------------------------------------ producer
-    if (lane == 0) {
-      const unsigned long long grad_policy = l2_policy_evict_first();
-      ScanAcc acc;
-      ChunkRef cr = p.ws.chunks[blockIdx.x];
-      ChunkRef cr1{-1, -1};
-      if (n_my > 1) cr1 = p.ws.chunks[blockIdx.x + stride];
-      grid_dependency_wait();
-      TensorMeta meta = load_meta(p, a, cr.tensor);
-      int issued = 0, head = 0, free_pages = kPages, oldest = 0;
-      bool gave_up = false;
-      for (int i = 0; i < n_my; ++i) {
-        const int slot = i % kSlots;
-        ChunkRef cr2{-1, -1};
-        if (i + 2 < n_my) cr2 = p.ws.chunks[blockIdx.x + (i + 2) * stride];
-        TensorMeta meta1 = meta;
-        if (i + 1 < n_my && cr1.tensor != cr.tensor) meta1 = load_meta(p, a, cr1.tensor);
-
-        const TensorInfo& ti = meta.ti;
-        const int tbytes = ti.theta_bits >> 3, cbytes = ti.comp_bits >> 3, vbytes = ti.mom_bits >> 3;
-        const int run[4] = {kChunk * 4 / kPageBytes, kChunk * tbytes / kPageBytes,
-                            kChunk * cbytes / kPageBytes, kChunk * vbytes / kPageBytes};
-        int page[4] = {0, 0, 0, 0}, h2 = head, need = 0;
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          if (h2 + run[r] > kPages) { need += kPages - h2; h2 = 0; }
-          page[r] = h2;
-          h2 += run[r];
-          need += run[r];
-        }
-        if (h2 == kPages) h2 = 0;
-        while (free_pages < need || i - oldest >= kSlots) {
-          const int os = oldest % kSlots;
-          if (!mbar_wait(&sh->empty[os], (unsigned)(oldest / kSlots) & 1u, &sh->abort_flag)) {
-            gave_up = true;
-            break;
-          }
-          take_back(p, acc, &sh->scan[os], sh->desc[os].tensor);
-          free_pages += sh->slot_pages[os];
-          ++oldest;
-        }
-        if (gave_up) {
-          sh->abort_flag = 1;
-          atomicCAS(p.ws.error, 0u, (unsigned)kErrEmptyWait);
-          break;
-        }
-        head = h2;
-        free_pages -= need;
-        sh->slot_pages[slot] = need;
-
-        const Coef coef = make_coef(ti, meta.e_in, meta.e_out, meta.ev_in, meta.ev_out, meta.lr, meta.mu);
-        const long long first = (long long)cr.index * kChunk;
-        const long long left = ti.numel - first;
-        const int count = left < (long long)kChunk ? (int)left : kChunk;
-        const int n_bulk = count & ~15;
-        // velocity LSB -> compensation LSBs as a float factor; beyond +-30 the steady path
-        // is never exact (k large) or the increment is always zero (k very negative)
-        const int kk = max(-40, min(30, coef.k));
-        TileDesc& td = sh->desc[slot];
-        td.scale_v = coef.scale_v;
-        td.mu_s = coef.mu_s;
-        td.pow2k = pow2_float(kk);
-        td.pow2s_neg = -pow2_float(coef.s);
-        td.inv2s = pow2_float(-coef.s);
-        td.qmax_t = (float)coef.qmax_t;
-        td.qmax_v = (float)coef.qmax_v;
-        td.d_limit = coef.k > 22 ? 0.5f : (coef.k > 0 ? 4000000.0f * pow2_float(-coef.k) : 4000000.0f);
-        td.theta = static_cast<unsigned char*>(ti.theta) + first * tbytes;
-        td.comp = static_cast<unsigned char*>(ti.comp) + first * cbytes;
-        td.mom = static_cast<unsigned char*>(ti.mom) + first * vbytes;
-        td.n_bulk = n_bulk;
-        td.flags = ((ti.theta_bits == 16 ? 1 : 0) | (ti.comp_bits == 16 ? 2 : 0) | (ti.mom_bits == 16 ? 4 : 0)) |
-                   (coef.delta == 0 ? kSteady : 0) | (page[1] << kThetaPageShift) |
-                   (page[2] << kCompPageShift) | (page[0] << kGradPageShift) | (page[3] << kMomPageShift);
-        td.tensor = cr.tensor;
-        td.count = count;
-        td.coef = coef;
-        td.grad = meta.grad + first;
-        if (n_bulk > 0) {
-          mbar_arrive_expect_tx(&sh->full[slot], (unsigned)(n_bulk * (tbytes + cbytes + vbytes + 4)));
-          bulk_load(smem + page[1] * kPageBytes, td.theta, (unsigned)(n_bulk * tbytes), &sh->full[slot]);
-          bulk_load(smem + page[2] * kPageBytes, td.comp, (unsigned)(n_bulk * cbytes), &sh->full[slot]);
-          bulk_load(smem + page[3] * kPageBytes, td.mom, (unsigned)(n_bulk * vbytes), &sh->full[slot]);
-          if (p.grad_evict_first)
-            bulk_load_hint(smem + page[0] * kPageBytes, td.grad, (unsigned)(n_bulk * 4), &sh->full[slot],
-                           grad_policy);
-          else
-            bulk_load(smem + page[0] * kPageBytes, td.grad, (unsigned)(n_bulk * 4), &sh->full[slot]);
-        } else {
-          mbar_arrive(&sh->full[slot]);
-        }
-        issued = i + 1;
-        cr = cr1;
-        cr1 = cr2;
-        meta = meta1;
-      }
-      for (int i = oldest; i < issued; ++i) {
-        const int os = i % kSlots;
-        if (mbar_wait(&sh->empty[os], (unsigned)(i / kSlots) & 1u, &sh->abort_flag))
-          take_back(p, acc, &sh->scan[os], sh->desc[os].tensor);
-        else
-          mbar_wait(&sh->full[os], (unsigned)(i / kSlots) & 1u, &sh->never);
-      }
-      publish(p, acc);
-    } else {
-      grid_dependency_wait();
-    }
-  } else {
-    // ------------------------------------------------------------------ consumers
-    grid_dependency_wait();
-    const int ctid = threadIdx.x;
-    float amax_t = 0.0f, amax_c = 0.0f, amax_v = 0.0f;
-    for (int i = 0; i < n_my; ++i) {
-      const int slot = i % kSlots, use = i / kSlots;
-      if (!mbar_wait(&sh->full[slot], (unsigned)use & 1u, &sh->abort_flag)) {
-        if (lane == 0) {
-          sh->abort_flag = 1;
-          atomicCAS(p.ws.error, 0u, (unsigned)kErrFullWait);
-        }
-        break;
-      }
-      const TileDesc* td = &sh->desc[slot];
-      TileScan* scan = &sh->scan[slot];
-      bool wrote_ring;
-      switch (td->flags & kFormatMask) {
-        case 0: wrote_ring = consume_tile<8, 8, 8>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
-        case 1: wrote_ring = consume_tile<16, 8, 8>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
-        case 2: wrote_ring = consume_tile<8, 16, 8>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
-        case 3: wrote_ring = consume_tile<16, 16, 8>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
-        case 4: wrote_ring = consume_tile<8, 8, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
-        case 5: wrote_ring = consume_tile<16, 8, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
-        case 6: wrote_ring = consume_tile<8, 16, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
-        default: wrote_ring = consume_tile<16, 16, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
-      }
-      {
-        __syncwarp();
-        const unsigned int full = 0xffffffffu;
-        const unsigned int at = __reduce_max_sync(full, (unsigned int)amax_t);
-        const unsigned int ac = __reduce_max_sync(full, (unsigned int)amax_c);
-        const unsigned int av = __reduce_max_sync(full, (unsigned int)amax_v);
-        amax_t = amax_c = amax_v = 0.0f;
-        if (lane == 0) {
-          if (at) atomicMax(&scan->amax_t, at);
-          if (ac) atomicMax(&scan->amax_c, ac);
-          if (av) atomicMax(&scan->amax_v, av);
-        }
-      }
-      if (wrote_ring) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->empty[slot]);
-    }
-  }
-
-  // ---------------------------------------------------------------------- block done
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    const unsigned int done = atomicAdd(p.ws.ticket, 1u);
-    sh->is_last = (done == gridDim.x - 1u);
-  }
-  __syncthreads();
-  if (!sh->is_last) return;
-
-  // Last block: rotate and choose the exponents of theta and of the velocity.
-  __threadfence();
-  const int n = p.n_tensors;
-  for (int i = threadIdx.x; i < n; i += kBlock) {
-    const unsigned int at = __ldcg(&p.ws.amax_acc[i]);
-    const unsigned int ac = __ldcg(&p.ws.amax_acc[n + i]);
-    const unsigned int av = __ldcg(&p.ws.amax_acc[2 * n + i]);
-    const int eo = p.ws.exp_next[i], evo = p.ws.expv_next[i];
-    p.ws.exp_cur[i] = eo;
-    p.ws.exp_next[i] = next_exponent(at, p.ws.info[i].theta_bits, eo, p.amax_mode);
-    p.ws.expv_cur[i] = evo;
-    p.ws.expv_next[i] = next_exponent_velocity(av, p.ws.info[i].mom_bits, evo, p.amax_mode);
-    p.ws.amax_last[i] = at;
-    p.ws.amax_last[n + i] = ac;
-    p.ws.amax_last[2 * n + i] = av;
-    p.ws.amax_acc[i] = p.ws.amax_acc[n + i] = p.ws.amax_acc[2 * n + i] = 0u;
-  }
-  if (threadIdx.x == 0) *p.ws.ticket = 0u;
+  ring_step<Policy>(p, a);
 }
 
 }  // namespace mom

@@ -424,7 +424,6 @@ __device__ __forceinline__ void ring_step(const typename P::Params& p, const Arg
 
   extern __shared__ __align__(128) unsigned char smem[];
   Shared* sh = reinterpret_cast<Shared*>(smem + (size_t)kPages * kPageBytes);
-  grid_dependency_launch_dependents();   // the next step's blocks may take over SMs as ours exit
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -536,9 +535,6 @@ __device__ __forceinline__ void ring_step(const typename P::Params& p, const Arg
         const long long left = meta.ti.numel - first;
         const int count = left < (long long)chunk ? (int)left : chunk;
         const int n_bulk = count & ~15;
-        // The copies go out first and the descriptor is written while they are on their way:
-        // the tile's barrier completes only when the bytes have landed AND the producer has
-        // arrived, and it arrives after the descriptor is in place.
         const unsigned char* gptr[S];
         int row_bytes = 0;
 #pragma unroll
@@ -546,21 +542,36 @@ __device__ __forceinline__ void ring_step(const typename P::Params& p, const Arg
           gptr[r] = base[r] ? base[r] + first * bytes[r] : nullptr;
           row_bytes += bytes[r];
         }
-        if (n_bulk > 0) {
-          mbar_expect_tx(&sh->full[slot], (unsigned)(n_bulk * row_bytes));
+        auto issue_copies = [&]() {
+          if (n_bulk > 0) {
+            mbar_expect_tx(&sh->full[slot], (unsigned)(n_bulk * row_bytes));
 #pragma unroll
-          for (int r = 1; r < S; ++r)
-            if (bytes[r]) bulk_load(smem + page[r] * kPageBytes, gptr[r], (unsigned)(n_bulk * bytes[r]), &sh->full[slot]);
-          // Gradients are read once.  When the state of the whole list fits in L2, letting
-          // the gradients leave it first keeps the state resident from step to step.
-          if (p.grad_evict_first)
-            bulk_load_hint(smem + page[0] * kPageBytes, gptr[0], (unsigned)(n_bulk * bytes[0]), &sh->full[slot],
-                           grad_policy);
-          else
-            bulk_load(smem + page[0] * kPageBytes, gptr[0], (unsigned)(n_bulk * bytes[0]), &sh->full[slot]);
-        }
+            for (int r = 1; r < S; ++r)
+              if (bytes[r])
+                bulk_load(smem + page[r] * kPageBytes, gptr[r], (unsigned)(n_bulk * bytes[r]), &sh->full[slot]);
+            // Gradients are read once.  When the state of the whole list fits in L2, letting
+            // the gradients leave it first keeps the state resident from step to step.
+            if (p.grad_evict_first)
+              bulk_load_hint(smem + page[0] * kPageBytes, gptr[0], (unsigned)(n_bulk * bytes[0]), &sh->full[slot],
+                             grad_policy);
+            else
+              bulk_load(smem + page[0] * kPageBytes, gptr[0], (unsigned)(n_bulk * bytes[0]), &sh->full[slot]);
+          }
+        };
+        // The tile's barrier completes when its bytes have landed AND the producer has arrived,
+        // and it arrives after the descriptor is in place.  For the block's first tile the
+        // copies go out before the descriptor is built (the step's start-up latency); for
+        // the others after it, which measures better in long steps.
+        if (i == 0) issue_copies();
         P::fill_desc(sh->desc[slot], p, meta, cr.tensor, count, n_bulk, page, gptr);
+        if (i != 0) issue_copies();
         mbar_arrive(&sh->full[slot]);
+        // With its last tile on the way the block lets the next kernel of the stream go ahead:
+        // once every block has said so, blocks of that kernel take over SMs as ours exit, set
+        // up and wait (grid_dependency_wait) for this kernel to complete.  Said at the start
+        // instead, blocks of the next kernel sit on the early finishers' SMs for a large part
+        // of a long step, which measurably slows the blocks still at work.
+        if (i == n_my - 1) grid_dependency_launch_dependents();
         issued = i + 1;
         cr = cr1;
         cr1 = cr2;

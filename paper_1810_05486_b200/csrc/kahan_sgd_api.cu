@@ -1062,40 +1062,8 @@ int kahan_sgd_momentum_destroy(ksgd_momentum_handle* h) {
 
 namespace {
 
-struct AdamLayout {
-  size_t exp_cur, exp_next, expm_cur, expm_next, expv_cur, expv_next, amax_last, counters, error, stats_end;
-  size_t amax_acc, info, chunks, ticket, grad_ptr, lr, total;
-  long long n_chunks;
-};
-
-AdamLayout make_adam_layout(const ksgd_tensor_desc* d, int32_t n) {
-  AdamLayout L{};
-  long long chunks = 0;
-  for (int32_t i = 0; i < n; ++i) chunks += (d[i].numel + kChunk - 1) / kChunk;
-  L.n_chunks = chunks;
-  size_t o = 0;
-  L.exp_cur = o;   o += sizeof(int) * n;
-  L.exp_next = o;  o += sizeof(int) * n;
-  L.expm_cur = o;  o += sizeof(int) * n;
-  L.expm_next = o; o += sizeof(int) * n;
-  L.expv_cur = o;  o += sizeof(int) * n;
-  L.expv_next = o; o += sizeof(int) * n;
-  L.amax_last = o; o += sizeof(unsigned int) * 4 * n;
-  o = align_up(o, 8);
-  L.counters = o;  o += sizeof(unsigned long long) * 5 * n;
-  L.error = o;     o += 8;
-  L.stats_end = o;
-  L.amax_acc = o;  o += sizeof(unsigned int) * 4 * n;
-  o = align_up(o, 16);
-  L.info = o;      o += sizeof(adam::TensorInfo) * n;
-  o = align_up(o, 16);
-  L.chunks = o;    o += sizeof(ChunkRef) * (size_t)chunks;
-  o = align_up(o, 16);
-  L.ticket = o;    o += 16;
-  L.grad_ptr = o;  o += sizeof(float*) * n;
-  L.lr = o;        o += sizeof(float) * n;
-  L.total = align_up(o, 256);
-  return L;
+Layout make_adam_layout(const ksgd_tensor_desc* d, int32_t n) {
+  return make_ring_layout(n, plain_tile_count(d, n), sizeof(adam::TensorState), sizeof(adam::TensorInfo), 5);
 }
 
 bool exp_pair_ok(int32_t cur, int32_t next) {
@@ -1121,7 +1089,8 @@ int validate_adam(const ksgd_tensor_desc* d, const ksgd_adam_desc* a, int32_t n)
 }  // namespace
 
 struct ksgd_adam_handle {
-  AdamLayout layout;
+  Layout layout;
+  std::vector<int32_t> theta_bits;
   adam::StepParams params;
   char* ws_base;
   cudaStream_t stream;
@@ -1146,7 +1115,7 @@ int kahan_sgd_adam_init(ksgd_adam_handle** out, const ksgd_tensor_desc* descs, c
   if (mode != KSGD_EXP_FIXED && mode != KSGD_EXP_AMAX) return KSGD_ERR_MODE;
   if (!workspace) return KSGD_ERR_NULL;
   if (reinterpret_cast<uintptr_t>(workspace) % 256) return KSGD_ERR_ALIGN;
-  const AdamLayout L = make_adam_layout(descs, n_tensors);
+  const Layout L = make_adam_layout(descs, n_tensors);
   if (workspace_bytes < L.total) return KSGD_ERR_WORKSPACE;
 
   ksgd_adam_handle* h = new (std::nothrow) ksgd_adam_handle();
@@ -1157,20 +1126,22 @@ int kahan_sgd_adam_init(ksgd_adam_handle** out, const ksgd_tensor_desc* descs, c
   h->stream = static_cast<cudaStream_t>(cuda_stream);
   h->stats_host.resize(L.stats_end);
 
+  // Host image: phase 0; in the records the first step reads (slab 2) the exponents of the
+  // stored mantissas and, as overrides, the exponents the first step must write.
   std::vector<unsigned char> img(L.total, 0);
-  auto ints = [&](size_t off) { return reinterpret_cast<int*>(img.data() + off); };
+  adam::TensorState* last = reinterpret_cast<adam::TensorState*>(img.data() + L.state) + 2 * (size_t)L.slab;
   adam::TensorInfo* info = reinterpret_cast<adam::TensorInfo*>(img.data() + L.info);
   ChunkRef* chunks = reinterpret_cast<ChunkRef*>(img.data() + L.chunks);
   long long c = 0;
   double state_bytes = 0.0;
   for (int32_t i = 0; i < n_tensors; ++i) {
     const ksgd_tensor_desc& t = descs[i];
-    ints(L.exp_cur)[i] = t.exp_theta;
-    ints(L.exp_next)[i] = t.exp_theta_next;
-    ints(L.expm_cur)[i] = adescs[i].exp_m;
-    ints(L.expm_next)[i] = adescs[i].exp_m_next;
-    ints(L.expv_cur)[i] = adescs[i].exp_v;
-    ints(L.expv_next)[i] = adescs[i].exp_v_next;
+    last[i].exp_theta = t.exp_theta;
+    last[i].ovr_theta = t.exp_theta_next + kOvrBias;
+    last[i].exp_m = adescs[i].exp_m;
+    last[i].ovr_m = adescs[i].exp_m_next + kOvrBias;
+    last[i].exp_v = adescs[i].exp_v;
+    last[i].ovr_v = adescs[i].exp_v_next + kOvrBias;
     info[i].theta = t.theta;
     info[i].comp = t.comp;
     info[i].mom1 = adescs[i].mom1;
@@ -1180,6 +1151,7 @@ int kahan_sgd_adam_init(ksgd_adam_handle** out, const ksgd_tensor_desc* descs, c
     info[i].comp_bits = t.comp_bits;
     info[i].s = t.comp_bits - 1 - t.overlap_k;
     info[i].pad = 0;
+    h->theta_bits.push_back(t.theta_bits);
     const long long nc = (t.numel + kChunk - 1) / kChunk;
     for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
     state_bytes += (double)t.numel * ((t.theta_bits + t.comp_bits + 32) / 8);
@@ -1187,30 +1159,24 @@ int kahan_sgd_adam_init(ksgd_adam_handle** out, const ksgd_tensor_desc* descs, c
 
   adam::Workspace& w = h->params.ws;
   char* b = h->ws_base;
-  w.exp_cur = reinterpret_cast<int*>(b + L.exp_cur);
-  w.exp_next = reinterpret_cast<int*>(b + L.exp_next);
-  w.expm_cur = reinterpret_cast<int*>(b + L.expm_cur);
-  w.expm_next = reinterpret_cast<int*>(b + L.expm_next);
-  w.expv_cur = reinterpret_cast<int*>(b + L.expv_cur);
-  w.expv_next = reinterpret_cast<int*>(b + L.expv_next);
-  w.amax_last = reinterpret_cast<unsigned int*>(b + L.amax_last);
+  w.phase = reinterpret_cast<unsigned int*>(b + L.phase);
+  w.state = reinterpret_cast<adam::TensorState*>(b + L.state);
+  w.slab = L.slab;
   w.counters = reinterpret_cast<unsigned long long*>(b + L.counters);
   w.error = reinterpret_cast<unsigned int*>(b + L.error);
-  w.amax_acc = reinterpret_cast<unsigned int*>(b + L.amax_acc);
   w.info = reinterpret_cast<adam::TensorInfo*>(b + L.info);
   w.chunks = reinterpret_cast<ChunkRef*>(b + L.chunks);
-  w.ticket = reinterpret_cast<unsigned int*>(b + L.ticket);
   w.grad_ptr = reinterpret_cast<const float**>(b + L.grad_ptr);
   w.lr = reinterpret_cast<float*>(b + L.lr);
   h->params.n_tensors = n_tensors;
-  h->params.n_chunks = (int)L.n_chunks;
+  h->params.tile_begin = 0;
+  h->params.tile_count = (int)L.n_chunks;
   h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
   h->params.inline_args = n_tensors <= kInlineArgs ? 1 : 0;
+  h->params.advance = 1;
 
-  int dev = 0, sms = 0, l2_bytes = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, dev);
+  DeviceFacts dev;
+  cudaError_t e = query_device(dev);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(adam::ksgd_adam_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)adam::kSharedBytes);
@@ -1218,8 +1184,8 @@ int kahan_sgd_adam_init(ksgd_adam_handle** out, const ksgd_tensor_desc* descs, c
     delete h;
     return cuda_fail(e, "device query");
   }
-  h->grid = (int)(L.n_chunks < (long long)sms ? L.n_chunks : (long long)sms);
-  h->params.grad_evict_first = state_bytes <= 0.8 * (double)l2_bytes ? 1 : 0;
+  h->grid = (int)(L.n_chunks < (long long)dev.sms ? L.n_chunks : (long long)dev.sms);
+  h->params.grad_evict_first = state_bytes <= 0.8 * (double)dev.l2_bytes ? 1 : 0;
 
   e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
@@ -1261,23 +1227,37 @@ int kahan_sgd_adam_step(ksgd_adam_handle* h, const float* const* grads, const fl
 
 int kahan_sgd_adam_amax(ksgd_adam_handle* h, const ksgd_adam_stats* out) {
   if (!h || !out) return KSGD_ERR_NULL;
-  const AdamLayout& L = h->layout;
+  const Layout& L = h->layout;
   KSGD_CUDA(cudaMemcpyAsync(h->stats_host.data(), h->ws_base, L.stats_end, cudaMemcpyDeviceToHost,
                             h->stream));
   KSGD_CUDA(cudaStreamSynchronize(h->stream));
   const unsigned char* b = h->stats_host.data();
   const size_t n = (size_t)h->n;
+  unsigned int ph = 0;
+  std::memcpy(&ph, b + L.phase, 4);
+  if (ph > 2) return KSGD_ERR_DEVICE;
+  // the records of the last finished step; the exponents the coming step will write are the
+  // overrides if set, else what the scans imply (the rules the kernel applies)
+  const adam::TensorState* last = reinterpret_cast<const adam::TensorState*>(b + L.state) + ((ph + 2) % 3) * (size_t)L.slab;
+  const int mode = h->params.amax_mode;
+  for (size_t i = 0; i < n; ++i) {
+    const adam::TensorState& r = last[i];
+    if (out->amax_theta) out->amax_theta[i] = r.amax[0];
+    if (out->amax_comp) out->amax_comp[i] = r.amax[1];
+    if (out->amax_m) out->amax_m[i] = r.amax[2];
+    if (out->amax_v) out->amax_v[i] = r.amax[3];
+    if (out->exp_theta_cur) out->exp_theta_cur[i] = r.exp_theta;
+    if (out->exp_m_cur) out->exp_m_cur[i] = r.exp_m;
+    if (out->exp_v_cur) out->exp_v_cur[i] = r.exp_v;
+    if (out->exp_theta_next)
+      out->exp_theta_next[i] = r.ovr_theta ? r.ovr_theta - kOvrBias
+                                           : next_exponent(r.amax[0], h->theta_bits[i], r.exp_theta, mode);
+    if (out->exp_m_next)
+      out->exp_m_next[i] = r.ovr_m ? r.ovr_m - kOvrBias : adam::next_exponent_moment(r.amax[2], r.exp_m, mode);
+    if (out->exp_v_next)
+      out->exp_v_next[i] = r.ovr_v ? r.ovr_v - kOvrBias : adam::next_exponent_moment(r.amax[3], r.exp_v, mode);
+  }
   auto give = [&](void* dst, size_t off, size_t width) { if (dst) std::memcpy(dst, b + off, width * n); };
-  give(out->exp_theta_cur, L.exp_cur, 4);
-  give(out->exp_theta_next, L.exp_next, 4);
-  give(out->exp_m_cur, L.expm_cur, 4);
-  give(out->exp_m_next, L.expm_next, 4);
-  give(out->exp_v_cur, L.expv_cur, 4);
-  give(out->exp_v_next, L.expv_next, 4);
-  give(out->amax_theta, L.amax_last, 4);
-  give(out->amax_comp, L.amax_last + 4 * n, 4);
-  give(out->amax_m, L.amax_last + 8 * n, 4);
-  give(out->amax_v, L.amax_last + 12 * n, 4);
   give(out->n_sat_theta, L.counters, 8);
   give(out->n_sat_comp, L.counters + 8 * n, 8);
   give(out->n_sat_m, L.counters + 16 * n, 8);

@@ -355,7 +355,9 @@ __device__ __forceinline__ bool update_vector(const Pack<V * TB / 8>& pt, const 
 
 // The step in which theta's exponent changes by delta = e_out - e_in (ordinary mode: c's grid
 // moves with theta's), again on the FP32 pipe with every intermediate an exact integer below
-// 2^24.  k.pow2dc = 2^-delta.  d = rne(g*scale) is on the output compensation grid as always.
+// 2^24.  Statements 2-4 of Algorithm 1 for a vector whose increments d (on the output
+// compensation grid, as always) the caller has formed already; k.pow2dc = 2^-delta.  Shared
+// by the plain optimizer, the momentum optimizer and ADAM.
 //
 // Finer grid (delta < 0, a = -delta): the stored mantissas scale up exactly,
 //   base = M + qt*2^a (both even, so exact even beyond 2^24),  u = qc*2^a - d,
@@ -363,21 +365,29 @@ __device__ __forceinline__ bool update_vector(const Pack<V * TB / 8>& pt, const 
 // Coarser grid (delta > 0, a = delta, s' = s + a): theta's mantissa is split with two integer
 // operations per packed word, qt = A*2^a + B with 0 <= B < 2^a (on the sign-flipped lanes the
 // split is a logical shift and a mask), so that
-//   T = A*2^s' + v,  v = B*2^s + qc - d*2^a   (exact: |d|*2^a <= 4e6 is checked)
+//   T = A*2^s' + v,  v = B*2^s + qc - d*2^a   (exact when |d|*2^a <= 4e6)
 //   Pb = fma(v, 2^-s', M + A) = M + P,  w = Pb - (M + A),  R = fma(w, -2^s', v),
 //   Rm = fma(R, 2^-a, M) = M + Rq   (the second rounding of the coarser grid, ties on Rq's parity).
 // In both cases |Rq| <= 2^(s-1) whenever P needs no clamp, so c never clamps on this path.
-// Returns false (nothing stored: the vector goes to update_general) when some product is too
-// large, Inf or NaN, or some |P| exceeds QMAX.  A coarser change needs a <= TB - 1 (the
-// producer checks).
-template <int TB, int CB, int V, int GB>
-__device__ __forceinline__ bool update_vector_regrid(Pack<V * TB / 8> pt, Pack<(CB ? V * CB / 8 : 8)> pc,
-                                                     Pack<V * GB / 8> pg, const SteadyCoef& k,
-                                                     Pack<V * TB / 8>& ot, Pack<(CB ? V * CB / 8 : 8)>& oc,
-                                                     float& amax_t, float& amax_c) {
+// yM[i] = M + d_i.  The caller guarantees |d| <= regrid_d_limit(k) (and no NaN); the function
+// returns false (nothing stored: the vector goes to the general path) when some |P| exceeds
+// QMAX.  A coarser change needs a <= TB - 1 (the producer checks).
+struct RegridCoef {
+  float pow2dc;     // 2^-delta
+  float inv2s;      // 2^-s
+  float pow2s_neg;  // -2^s
+};
+
+__device__ __forceinline__ float regrid_d_limit(const RegridCoef& k) {
+  return k.pow2dc > 1.0f ? 4000000.0f : __fmul_rn(4000000.0f, k.pow2dc);   // coarser: |d| * 2^a stays exact
+}
+
+template <int TB, int CB, int V>
+__device__ __forceinline__ bool regrid_core(const Pack<V * TB / 8>& pt, const Pack<(CB ? V * CB / 8 : 8)>& pc,
+                                            const float (&yM)[V], const RegridCoef& k, Pack<V * TB / 8>& ot,
+                                            Pack<(CB ? V * CB / 8 : 8)>& oc, float& amax_t, float& amax_c) {
   constexpr bool HAS_COMP = CB != 0;
   constexpr int CBS = CB ? CB : 8;
-  constexpr int GBS = GB == 32 ? 8 : GB;
   constexpr float bias_t = (float)(1 << (TB - 1));
   const bool finer = k.pow2dc > 1.0f;
   // 2^a and 2^-a
@@ -402,22 +412,17 @@ __device__ __forceinline__ bool update_vector_regrid(Pack<V * TB / 8> pt, Pack<(
     pow2sp_neg = __fmul_rn(k.pow2s_neg, up);    // -2^s'
     biasA = __fmul_rn(bias_t, down);            // what the shifted lanes still carry of the sign flip
   }
-  float Pm[V], rm[V], xa[2], ra[2];
-  float aX = 0.0f, hiP = kMagic, loP = kMagic, aR = 0.0f;
+  float Pm[V], rm[V], ra[2];
+  float hiP = kMagic, loP = kMagic, aR = 0.0f;
 #pragma unroll
   for (int i = 0; i < V; ++i) {
-    float g;
-    if constexpr (GB == 32) g = __uint_as_float(pack_word(pg, i));
-    else g = __fadd_rn(magic_signed<GBS>(pg, i), -kMagic);
-    const float x = __fmul_rn(g, k.scale);              // the one binary32 multiply
-    const float y = __fadd_rn(x, kMagic);               // M + d
     float qc = 0.0f;
     if constexpr (HAS_COMP) qc = __fadd_rn(magic_signed<CBS>(pc, i), -kMagic);
     float P, r;
     if (finer) {
       const float qt = __fadd_rn(magic_signed<TB>(pt, i), -kMagic);
       const float base = __fmaf_rn(qt, up, kMagic);
-      const float u = __fmaf_rn(qc, up, __fadd_rn(kMagic, -y));
+      const float u = __fmaf_rn(qc, up, __fadd_rn(kMagic, -yM[i]));
       P = __fmaf_rn(u, inv2sp, base);
       const float w = __fadd_rn(P, -base);
       r = __fmaf_rn(w, pow2sp_neg, u);
@@ -425,7 +430,7 @@ __device__ __forceinline__ bool update_vector_regrid(Pack<V * TB / 8> pt, Pack<(
     } else {
       const float base = __fadd_rn(magic_elem<TB>(pA, i), -biasA);       // M + A
       const float B = __fadd_rn(magic_elem<TB>(pB, i), -kMagic);
-      const float d = __fadd_rn(y, -kMagic);
+      const float d = __fadd_rn(yM[i], -kMagic);
       const float v = __fmaf_rn(d, -up, __fmaf_rn(B, pow2s, qc));
       P = __fmaf_rn(v, inv2sp, base);
       const float w = __fadd_rn(P, -base);
@@ -434,10 +439,8 @@ __device__ __forceinline__ bool update_vector_regrid(Pack<V * TB / 8> pt, Pack<(
       r = __fadd_rn(rm[i], -kMagic);
     }
     Pm[i] = P;
-    xa[i & 1] = fabsf(x);
     ra[i & 1] = fabsf(r);
     if (i & 1) {
-      aX = max3_nan(aX, xa[0], xa[1]);                  // NaN if any product is
       hiP = max3(hiP, Pm[i - 1], P);
       loP = min3(loP, Pm[i - 1], P);
       if constexpr (HAS_COMP) aR = max3(aR, ra[0], ra[1]);
@@ -445,13 +448,36 @@ __device__ __forceinline__ bool update_vector_regrid(Pack<V * TB / 8> pt, Pack<(
   }
   const float aP = fmaxf(__fadd_rn(hiP, -kMagic), __fadd_rn(kMagic, -loP));
   constexpr float qmax_t = (float)((1 << (TB - 1)) - 1);
-  const float x_limit = finer ? 4000000.0f : __fmul_rn(4000000.0f, down);   // |d| * 2^a stays exact
-  if (!(aX <= x_limit) | (aP > qmax_t)) return false;   // also Inf and NaN products
+  if (aP > qmax_t) return false;
   amax_t = fmaxf(amax_t, aP);
   if constexpr (HAS_COMP) amax_c = fmaxf(amax_c, aR);
   ot = pack_magic<TB, V>(Pm);
   if constexpr (HAS_COMP) oc = pack_magic<CB, V>(rm);
   return true;
+}
+
+// The plain optimizer's increment for such a vector: d = rne(g * scale), as in update_vector.
+template <int TB, int CB, int V, int GB>
+__device__ __forceinline__ bool update_vector_regrid(const Pack<V * TB / 8>& pt, const Pack<(CB ? V * CB / 8 : 8)>& pc,
+                                                     const Pack<V * GB / 8>& pg, const SteadyCoef& k,
+                                                     Pack<V * TB / 8>& ot, Pack<(CB ? V * CB / 8 : 8)>& oc,
+                                                     float& amax_t, float& amax_c) {
+  constexpr int GBS = GB == 32 ? 8 : GB;
+  const RegridCoef rk{k.pow2dc, k.inv2s, k.pow2s_neg};
+  float yM[V], xa[2];
+  float aX = 0.0f;
+#pragma unroll
+  for (int i = 0; i < V; ++i) {
+    float g;
+    if constexpr (GB == 32) g = __uint_as_float(pack_word(pg, i));
+    else g = __fadd_rn(magic_signed<GBS>(pg, i), -kMagic);
+    const float x = __fmul_rn(g, k.scale);              // the one binary32 multiply
+    yM[i] = __fadd_rn(x, kMagic);                       // M + d
+    xa[i & 1] = fabsf(x);
+    if (i & 1) aX = max3_nan(aX, xa[0], xa[1]);         // NaN if any product is
+  }
+  if (!(aX <= regrid_d_limit(rk))) return false;        // also Inf and NaN products
+  return regrid_core<TB, CB, V>(pt, pc, yM, rk, ot, oc, amax_t, amax_c);
 }
 
 // All vectors of one tile that belong to this consumer thread (V consecutive elements,

@@ -102,6 +102,7 @@ struct __align__(16) TileDesc {
 };
 constexpr int kFormatMask = 7;       // bit 0: theta 16, bit 1: comp 16, bit 2: mom 16
 constexpr int kSteady = 8;
+constexpr int kRegrid = 16;      // theta's exponent changes: the exact-fp32 re-gridding path applies
 constexpr int kThetaPageShift = 8, kCompPageShift = 13, kGradPageShift = 18, kMomPageShift = 23;
 
 // Three maxima, then four counts: the order the ring expects.
@@ -310,6 +311,126 @@ __device__ __forceinline__ bool consume_tile(const TileDesc* td, unsigned char* 
   return wrote_ring;
 }
 
+// A vector of a tensor whose theta changes its exponent in this step: the velocity as in
+// update_vector, then statements 2-4 of Algorithm 1 through regrid_core (kahan_sgd_kernels.cuh).
+template <int TB, int CB, int VB>
+__device__ __forceinline__ bool update_vector_regrid(const Pack<TB>& pt, const Pack<CB>& pc, const Pack<VB>& pv,
+                                                     const Pack<32>& pg, const SteadyCoef& k, const RegridCoef& rk,
+                                                     Pack<TB>& ot, Pack<CB>& oc, Pack<VB>& ov, float& amax_t,
+                                                     float& amax_c, float& amax_v) {
+  constexpr int V = 8;
+  float yM[V], Vm[V], va[2], da[2];
+  float aV = 0.0f, aD = 0.0f;
+#pragma unroll
+  for (int i = 0; i < V; ++i) {
+    const float qv = __fadd_rn(magic_signed<VB>(pv, i), -kMagic);
+    const float g = __uint_as_float(pack_word(pg, i));
+    const float y = __fmaf_rn(k.mu_s, qv, __fmul_rn(g, k.scale_v));
+    const float vm = __fadd_rn(y, kMagic);
+    const float v = __fadd_rn(vm, -kMagic);
+    yM[i] = __fmaf_rn(v, k.pow2k, kMagic);              // M + d
+    Vm[i] = vm;
+    va[i & 1] = fabsf(v);
+    da[i & 1] = fabsf(__fadd_rn(yM[i], -kMagic));
+    if (i & 1) {
+      aV = max3_nan(aV, va[0], va[1]);
+      aD = max3(aD, da[0], da[1]);
+    }
+  }
+  if (!(aV <= k.qmax_v) | !(aV <= k.d_limit) | !(aD <= regrid_d_limit(rk))) return false;
+  float at = amax_t, ac = amax_c;
+  if (!regrid_core<TB, CB, V>(pt, pc, yM, rk, ot, oc, at, ac)) return false;
+  amax_t = at;
+  amax_c = ac;
+  amax_v = fmaxf(amax_v, aV);
+  ov = pack_magic<VB, V>(Vm);
+  return true;
+}
+
+template <int TB, int CB, int VB>
+__device__ __forceinline__ bool regrid_tile_format(const TileDesc* td, unsigned char* ring, int ctid, TileScan* scan,
+                                                   float& amax_t, float& amax_c, float& amax_v) {
+  constexpr int V = 8;
+  const uint4* q = reinterpret_cast<const uint4*>(td);
+  const uint4 q0 = q[0], q1 = q[1], q2 = q[2], q3 = q[3];
+  SteadyCoef k;
+  k.scale_v = __uint_as_float(q0.x);
+  k.mu_s = __uint_as_float(q0.y);
+  k.pow2k = __uint_as_float(q0.z);
+  k.pow2s_neg = __uint_as_float(q0.w);
+  k.inv2s = __uint_as_float(q1.x);
+  k.qmax_t = __uint_as_float(q1.y);
+  k.qmax_v = __uint_as_float(q1.z);
+  k.d_limit = __uint_as_float(q1.w);
+  const RegridCoef rk{pow2_float(-td->coef.delta), k.inv2s, k.pow2s_neg};
+  unsigned char* theta_g = reinterpret_cast<unsigned char*>(((unsigned long long)q2.y << 32) | q2.x);
+  unsigned char* comp_g = reinterpret_cast<unsigned char*>(((unsigned long long)q2.w << 32) | q2.z);
+  unsigned char* mom_g = reinterpret_cast<unsigned char*>(((unsigned long long)q3.y << 32) | q3.x);
+  const int n_bulk = (int)q3.z, flags = (int)q3.w;
+  unsigned char* theta_s = ring + ((flags >> kThetaPageShift) & 31) * kPageBytes;
+  unsigned char* comp_s = ring + ((flags >> kCompPageShift) & 31) * kPageBytes;
+  unsigned char* mom_s = ring + ((flags >> kMomPageShift) & 31) * kPageBytes;
+  const float* grad_s = reinterpret_cast<const float*>(ring + ((flags >> kGradPageShift) & 31) * kPageBytes);
+  bool wrote_ring = false;
+  const int n_vec = n_bulk / V;
+  for (int v = ctid; v < n_vec; v += kThreads) {
+    Pack<TB> ot;
+    Pack<CB> oc;
+    Pack<VB> ov;
+    const Pack<TB> pt = load_pack<TB>(theta_s + v * TB);
+    const Pack<CB> pc = load_pack<CB>(comp_s + v * CB);
+    const Pack<VB> pv = load_pack<VB>(mom_s + v * VB);
+    const Pack<32> pg = load_pack<32>(grad_s + v * V);
+    if (!update_vector_regrid<TB, CB, VB>(pt, pc, pv, pg, k, rk, ot, oc, ov, amax_t, amax_c, amax_v)) {
+      update_general(&td->coef, TB, CB, VB, theta_s, comp_s, mom_s, grad_s, v * V, V, scan);
+      ot = load_pack<TB>(theta_s + v * TB);
+      oc = load_pack<CB>(comp_s + v * CB);
+      ov = load_pack<VB>(mom_s + v * VB);
+      wrote_ring = true;
+    }
+    store_pack<TB>(theta_g + (size_t)v * TB, ot);
+    store_pack<CB>(comp_g + (size_t)v * CB, oc);
+    store_pack<VB>(mom_g + (size_t)v * VB, ov);
+  }
+  const int e = n_bulk + ctid;
+  if (e < td->count) update_general(&td->coef, TB, CB, VB, theta_g, comp_g, mom_g, td->grad, e, 1, scan);
+  return wrote_ring;
+}
+
+__device__ __forceinline__ void add_warp_scans(TileScan* scan, int lane, float amax_t, float amax_c, float amax_v) {
+  // the exact-fp32 paths' scans are exact integers below 2^23 held in floats
+  const unsigned int full = 0xffffffffu;
+  const unsigned int at = __reduce_max_sync(full, (unsigned int)amax_t);
+  const unsigned int ac = __reduce_max_sync(full, (unsigned int)amax_c);
+  const unsigned int av = __reduce_max_sync(full, (unsigned int)amax_v);
+  if (lane == 0) {
+    if (at) atomicMax(&scan->amax_t, at);
+    if (ac) atomicMax(&scan->amax_c, ac);
+    if (av) atomicMax(&scan->amax_v, av);
+  }
+}
+
+// A whole tile of a tensor whose theta changes its exponent, for one consumer thread.  Out of
+// line, called once per such tile with next to nothing live around the call, so that its
+// registers cost the tiles whose exponent does not change nothing.
+__device__ __noinline__ void regrid_tile(const TileDesc* td, TileScan* scan, unsigned char* ring) {
+  const int ctid = threadIdx.x;
+  float amax_t = 0.0f, amax_c = 0.0f, amax_v = 0.0f;
+  bool wrote_ring;
+  switch (td->flags & kFormatMask) {
+    case 0: wrote_ring = regrid_tile_format<8, 8, 8>(td, ring, ctid, scan, amax_t, amax_c, amax_v); break;
+    case 1: wrote_ring = regrid_tile_format<16, 8, 8>(td, ring, ctid, scan, amax_t, amax_c, amax_v); break;
+    case 2: wrote_ring = regrid_tile_format<8, 16, 8>(td, ring, ctid, scan, amax_t, amax_c, amax_v); break;
+    case 3: wrote_ring = regrid_tile_format<16, 16, 8>(td, ring, ctid, scan, amax_t, amax_c, amax_v); break;
+    case 4: wrote_ring = regrid_tile_format<8, 8, 16>(td, ring, ctid, scan, amax_t, amax_c, amax_v); break;
+    case 5: wrote_ring = regrid_tile_format<16, 8, 16>(td, ring, ctid, scan, amax_t, amax_c, amax_v); break;
+    case 6: wrote_ring = regrid_tile_format<8, 16, 16>(td, ring, ctid, scan, amax_t, amax_c, amax_v); break;
+    default: wrote_ring = regrid_tile_format<16, 16, 16>(td, ring, ctid, scan, amax_t, amax_c, amax_v); break;
+  }
+  add_warp_scans(scan, threadIdx.x & 31, amax_t, amax_c, amax_v);
+  if (wrote_ring) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
 // Exponent of the velocity for the next step.  The velocity's maximum moves with every
 // gradient, so it keeps its exponent while its largest mantissa stays in (QMAX/4, QMAX] and
 // otherwise takes the tight fit (coarser at once, finer only after a fourfold drop).
@@ -397,7 +518,9 @@ struct Policy {
     td.mom = const_cast<unsigned char*>(gptr[3]);
     td.n_bulk = n_bulk;
     td.flags = ((ti.theta_bits == 16 ? 1 : 0) | (ti.comp_bits == 16 ? 2 : 0) | (ti.mom_bits == 16 ? 4 : 0)) |
-               (coef.delta == 0 ? kSteady : 0) | (page[1] << kThetaPageShift) |
+               (coef.delta == 0 ? kSteady : 0) |
+               // a coarser grid splits theta's mantissa at bit delta: that needs delta <= theta_bits - 1
+               ((coef.delta != 0 && coef.delta <= ti.theta_bits - 1) ? kRegrid : 0) | (page[1] << kThetaPageShift) |
                (page[2] << kCompPageShift) | (page[0] << kGradPageShift) | (page[3] << kMomPageShift);
     td.tensor = tensor;
     td.count = count;
@@ -406,6 +529,10 @@ struct Policy {
   }
   static __device__ __forceinline__ void consume(const TileDesc* td, TileScan* scan, unsigned char* smem, int ctid,
                                                  int lane) {
+    if (td->flags & kRegrid) {
+      regrid_tile(td, scan, smem);
+      return;
+    }
     float amax_t = 0.0f, amax_c = 0.0f, amax_v = 0.0f;
     bool wrote_ring;
     switch (td->flags & kFormatMask) {
@@ -418,16 +545,7 @@ struct Policy {
       case 6: wrote_ring = consume_tile<8, 16, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
       default: wrote_ring = consume_tile<16, 16, 16>(td, smem, ctid, scan, amax_t, amax_c, amax_v); break;
     }
-    // the steady path's scans are exact integers below 2^23 held in floats
-    const unsigned int full = 0xffffffffu;
-    const unsigned int at = __reduce_max_sync(full, (unsigned int)amax_t);
-    const unsigned int ac = __reduce_max_sync(full, (unsigned int)amax_c);
-    const unsigned int av = __reduce_max_sync(full, (unsigned int)amax_v);
-    if (lane == 0) {
-      if (at) atomicMax(&scan->amax_t, at);
-      if (ac) atomicMax(&scan->amax_c, ac);
-      if (av) atomicMax(&scan->amax_v, av);
-    }
+    add_warp_scans(scan, lane, amax_t, amax_c, amax_v);
     // if the general path wrote into the ring, order those writes before the bulk copy
     // that refills the pages
     if (wrote_ring) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -134,6 +134,8 @@ def parse_args():
                     help="skip the per-size-bucket timing of c5_sweep")
     ap.add_argument("--no-extra-workloads", action="store_true",
                     help="skip the c3_resnet50 / c4_alexnet legs that the default run adds to its line")
+    ap.add_argument("--no-optimizers", action="store_true",
+                    help="skip the momentum / ADAM / int8-gradient legs that the default run adds to its line")
     ap.add_argument("--no-convert", action="store_true",
                     help="skip the fp32 <-> fixed-point conversion leg that the default run adds to its line")
     ap.add_argument("--sustained-s", type=float, default=0.35,
@@ -343,25 +345,44 @@ def convert_leg(torch, B, peak, numel=64 * 1024 * 1024, iters=10):
     return out
 
 
-def extra_workload(torch, B, W, name, args, peak, peak_src, barrier, gpu_index):
+OPTIMIZER_KERNELS = {"sgd": "ksgd_step_kernel", "sgd, int8 gradients": "ksgd_step_qgrad_kernel",
+                     "momentum 0.9, int16 velocity": "ksgd_momentum_step_kernel",
+                     "momentum 0.9, int8 velocity": "ksgd_momentum_step_kernel",
+                     "adam 0.9/0.999/1e-8, int16 moments": "ksgd_adam_step_kernel"}
+
+
+def extra_workload(torch, B, W, name, args, peak, peak_src, barrier, gpu_index, host=None, optimizer="sgd"):
     """One of the other workloads of at least 25 M parameters, timed like the headline: the
-    recipe's own number of steps (a fresh gradient set each), then the sustained leg."""
+    recipe's own number of steps (a fresh gradient set each), then the sustained leg.
+    optimizer: "sgd" (the path of the headline), or one of the optimizers and gradient formats
+    built around the same update (their extra arrays count as algorithmic bytes)."""
     from paper_1810_05486_b200.runner import DeviceRun, HostInputs
     wl = W.workload(name)
     n_sets = GRAD_SETS[name]
-    host = HostInputs(wl, args.seed, n_sets, pinned=False)
-    run = DeviceRun(host, B.KSGD_EXP_AMAX)
+    if host is None:
+        host = HostInputs(wl, args.seed, n_sets, pinned=False)
+    kw = {}
+    if optimizer.startswith("momentum"):
+        kw["mom_bits"] = 16 if "int16" in optimizer else 8
+    elif optimizer.startswith("adam"):
+        t0_ = wl.tensors[0]
+        kw["adam"] = dict(beta1=0.9, beta2=0.999, eps=1e-8,
+                          eta=1e-3 * 2.0 ** t0_.exp_theta * (2 ** (t0_.theta_bits - 1) - 1))
+    elif "int8 gradients" in optimizer:
+        kw["grad_bits"] = 8
+    run = DeviceRun(host, B.KSGD_EXP_AMAX, **kw)
     with torch.cuda.stream(run.stream):
         for i in range(args.warmup):
             run.step(i % n_sets)
         barrier()
         ms_total, quarters, launches, _ = timed_region(torch, B, run, n_sets, wl.steps, args.warmup, barrier)
         ms_step = ms_total / wl.steps
-        out = {"workload": name, "tensors": len(wl.tensors), "parameters": wl.numel,
+        out = {"workload": name, "optimizer": optimizer, "tensors": len(wl.tensors), "parameters": wl.numel,
                "bytes_per_step": run.bytes_per_step, "steps": wl.steps, "warmup": args.warmup,
                "ms_per_step": ms_step, "value": wl.numel / (ms_step * 1e-3), "unit": UNIT,
                "gpu_launches": launches, "l2": l2_note(wl, n_sets),
-               "roofline": roofline_of(wl, run.bytes_per_step, ms_step, peak, peak_src, "ksgd_step_kernel", True)}
+               "roofline": roofline_of(wl, run.bytes_per_step, ms_step, peak, peak_src,
+                                       OPTIMIZER_KERNELS[optimizer], optimizer == "sgd")}
         if args.sustained_s > 0:
             out["sustained"] = sustained_leg(torch, B, run, n_sets, ms_step, args.sustained_s,
                                              args.warmup + wl.steps, barrier, gpu_index, run.bytes_per_step, peak)
@@ -369,7 +390,7 @@ def extra_workload(torch, B, W, name, args, peak, peak_src, barrier, gpu_index):
     out["counters"] = {"n_sat_theta": int(sum(st["n_sat_theta"])), "n_sat_comp": int(sum(st["n_sat_comp"])),
                        "n_nonfinite": int(sum(st["n_nonfinite"]))}
     run.close()
-    del run, host
+    del run
     torch.cuda.empty_cache()
     return out
 
@@ -527,8 +548,18 @@ def run_ours(args, rank, world, local_rank):
         run.host = None
         del host        # page-locked host copies of the sweep (12 GB) go before the next workloads come
         torch.cuda.empty_cache()
-        line["workloads"] = [extra_workload(torch, B, W, name, args, peak, peak_src, barrier, local_rank)
-                             for name in ("c3_resnet50", "c4_alexnet")]
+        from paper_1810_05486_b200.runner import HostInputs
+        line["workloads"], line["optimizers"] = [], []
+        for name, others in (("c3_resnet50", ("adam 0.9/0.999/1e-8, int16 moments",)),
+                             ("c4_alexnet", ("momentum 0.9, int16 velocity", "sgd, int8 gradients"))):
+            h2 = HostInputs(W.workload(name), args.seed, GRAD_SETS[name], pinned=False)
+            line["workloads"].append(extra_workload(torch, B, W, name, args, peak, peak_src, barrier, local_rank, h2))
+            if not args.no_optimizers:
+                # the optimizers of Section 4 and the all-fixed-point gradient format, on the same inputs
+                for opt in others:
+                    line["optimizers"].append(extra_workload(torch, B, W, name, args, peak, peak_src, barrier,
+                                                             local_rank, h2, opt))
+            del h2
         if not args.no_convert:
             line["convert"] = convert_leg(torch, B, peak)
     print(json.dumps(line), flush=True)

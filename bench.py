@@ -42,19 +42,20 @@ GRAD_SETS = {"c5_sweep": 2, "c1_single": 100, "c2_resnet20": 200, "c3_resnet50":
 
 # DRAM traffic of ksgd_step_kernel from ncu captures (dram__bytes_read.sum +
 # dram__bytes_write.sum per launch, divided by the parameters of the captured launch; see
-# profiles/).  "cold": caches flushed before the launch (ncu's default), which is what a
-# list far larger than L2 sees at every step; c5_sweep was captured at 2e8 parameters and
-# its traffic is proportional to the parameter count, so a full launch is this figure times
-# its parameters.  "warm": the launch as it runs in the benchmark's loop, caches left as the
-# preceding steps left them (--cache-control none), which is what counts for a list whose
-# theta and c stay in L2 from step to step.  The record only counts while the kernel source
-# (kahan_sgd_kernels.cuh) still hashes to the value below.
+# profiles/).  "cold": caches flushed before the launch (ncu's default); c5_sweep was captured
+# at 2e8 parameters and its traffic is proportional to the parameter count, so a full launch
+# is this figure times its parameters.  "warm": the launch as it runs in the benchmark's loop,
+# caches left as the preceding steps left them (--cache-control none): the steady state,
+# which is what counts for a list whose theta and c partly stay in L2 from step to step (a
+# warm launch also writes back lines the preceding step left dirty, a cold one leaves some
+# of its own behind).  The record only counts while the kernel sources (kahan_sgd_ring.cuh,
+# kahan_sgd_kernels.cuh) still hash to the value below.
 TRAFFIC_RECORD = {
-    "sources_sha256": "2116fc351fe2f07e2b18bc9dcf183f78c3cd847a1bfd0bdc0e303bd140896441",
+    "sources_sha256": "389f2c4a0026120f2792de1392505d56ef66450fe2317b437ec2d8236459e00c",
     "dram_bytes_per_parameter": {
-        "c5_sweep": {"cold": 2355.328e6 / 2e8, "warm": None},
-        "c4_alexnet": {"cold": 469.794e6 / 61100840, "warm": None},
-        "c3_resnet50": {"cold": 200.325e6 / 25557032, "warm": None},
+        "c5_sweep": {"cold": 2357.049e6 / 2e8, "warm": None},
+        "c4_alexnet": {"cold": 470.839e6 / 61100840, "warm": 513.373e6 / 61100840},
+        "c3_resnet50": {"cold": 200.677e6 / 25557032, "warm": 218.487e6 / 25557032},
     },
 }
 
@@ -62,7 +63,7 @@ TRAFFIC_RECORD = {
 def kernel_sources_sha256():
     import hashlib
     h = hashlib.sha256()
-    for name in ("kahan_sgd_kernels.cuh",):
+    for name in ("kahan_sgd_ring.cuh", "kahan_sgd_kernels.cuh"):
         with open(os.path.join(ROOT, "paper_1810_05486_b200", "csrc", name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()
@@ -284,7 +285,7 @@ def roofline_of(wl, bytes_per_step, ms_step, peak, peak_src, kernel, plain):
          "traffic": None, "peak_source": peak_src, "frac_of_nominal_8000": achieved / 8000.0,
          "kernel": kernel, "launch_ms": ms_step, "l2_assisted": l2_resident_state(wl)}
     if plain:
-        kind = "warm" if r["l2_assisted"] else "cold"
+        kind = "warm" if TRAFFIC_RECORD["dram_bytes_per_parameter"].get(wl.name, {}).get("warm") else "cold"
         traffic = recorded_traffic(wl, kind)
         r["traffic"] = traffic
         r["traffic_capture"] = ("ncu --cache-control none (caches as the preceding steps left them)"

@@ -94,29 +94,30 @@ __global__ void __launch_bounds__(kThreads) absmax_fit_kernel(const float* __res
 // One element in binary32, every step exact except the two roundings of the definition:
 //   Q_theta = clamp(rne(x / 2^e)),  Q_c = clamp(rne((x - Q_theta*2^e) / 2^(e-s))).
 // x / 2^e is an exact scaling (a result below the normal range is far below half a unit and
-// rounds to 0 either way); the rounding is an addition of M = 1.5 * 2^23 after a clamp to
-// +-(QMAX + 1), which commutes with it; x/2^e - Q_theta is a difference of two floats that
-// either lie within a factor of two of each other or has a result of fewer bits than x/2^e,
-// so it is exact whenever the result can still matter (beyond 2^24 it only has to be large).
+// rounds to 0 either way).  Clamping to +-(QMAX + 1/4) first and rounding then gives the same
+// integer as rounding first and clamping to +-QMAX (everything from QMAX + 1/4 on rounds to
+// QMAX), and keeps the value where adding M = 1.5 * 2^23 rounds it to the nearest integer,
+// ties to even; the integer is then the low bits of M's bit pattern (no conversion
+// instruction).  x/2^e - Q_theta is a difference of two floats that either lie within a
+// factor of two of each other or has a result of fewer bits than x/2^e, so it is exact
+// whenever the result can still matter (beyond 2^24 it only has to be large).
 // NaN -> 0, +-Inf -> +-QMAX with nothing left for c.
 template <int TB, int CB>
 __device__ __forceinline__ void quantize_one(float x, float inv2e, float pow2s, int& qt, int& qc) {
   constexpr float kM = 12582912.0f;
-  constexpr float qmax_t = (float)((1 << (TB - 1)) - 1);
-  constexpr float qmax_c = (float)((1 << ((CB ? CB : 8) - 1)) - 1);
+  constexpr int kMBits = 0x4B400000;
+  constexpr float bound_t = (float)((1 << (TB - 1)) - 1) + 0.25f;
+  constexpr float bound_c = (float)((1 << ((CB ? CB : 8) - 1)) - 1) + 0.25f;
   const float xs = __fmul_rn(x, inv2e);
-  float t = fminf(fmaxf(xs, -(qmax_t + 1.0f)), qmax_t + 1.0f);      // NaN -> a finite bound, fixed below
-  t = __fadd_rn(__fadd_rn(t, kM), -kM);
-  t = fminf(fmaxf(t, -qmax_t), qmax_t);
+  const float tm = __fadd_rn(fminf(fmaxf(xs, -bound_t), bound_t), kM);   // NaN -> a finite bound, fixed below
   const bool nan = x != x, inf = fabsf(x) == __int_as_float(0x7f800000);
-  qt = nan ? 0 : (int)t;
+  qt = nan ? 0 : __float_as_int(tm) - kMBits;
   qc = 0;
   if constexpr (CB != 0) {
-    float r = __fmul_rn(__fadd_rn(xs, -t), pow2s);
-    r = fminf(fmaxf(r, -(qmax_c + 1.0f)), qmax_c + 1.0f);
-    r = __fadd_rn(__fadd_rn(r, kM), -kM);
-    r = fminf(fmaxf(r, -qmax_c), qmax_c);
-    qc = (nan || inf) ? 0 : (int)r;
+    const float t = __fadd_rn(tm, -kM);
+    const float r = __fmul_rn(__fadd_rn(xs, -t), pow2s);
+    const float rm = __fadd_rn(fminf(fmaxf(r, -bound_c), bound_c), kM);
+    qc = (nan || inf) ? 0 : __float_as_int(rm) - kMBits;
   }
 }
 
@@ -175,20 +176,23 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float* __restr
   }
 }
 
+// Four mantissas as floats: an integer dot product with a one-hot selector sign-extends a
+// mantissa and adds it to the bit pattern of M = 1.5 * 2^23 (for |q| < 2^22 integer addition
+// on the bits is addition of the values); subtracting M leaves q.  No conversion instruction.
 template <int BITS>
 __device__ __forceinline__ void load4(const void* base, long long i4, float (&q)[4]) {
+  constexpr float kM = 12582912.0f;
+  constexpr int kMBits = 0x4B400000;
   if constexpr (BITS == 8) {
-    const unsigned int w = reinterpret_cast<const unsigned int*>(base)[i4];
-    q[0] = (float)(signed char)(w & 0xff);
-    q[1] = (float)(signed char)((w >> 8) & 0xff);
-    q[2] = (float)(signed char)((w >> 16) & 0xff);
-    q[3] = (float)(signed char)(w >> 24);
+    const int w = (int)reinterpret_cast<const unsigned int*>(base)[i4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) q[j] = __fadd_rn(__int_as_float(__dp4a(w, 1 << (8 * j), kMBits)), -kM);
   } else {
     const uint2 w = reinterpret_cast<const uint2*>(base)[i4];
-    q[0] = (float)(short)(w.x & 0xffff);
-    q[1] = (float)(short)(w.x >> 16);
-    q[2] = (float)(short)(w.y & 0xffff);
-    q[3] = (float)(short)(w.y >> 16);
+    q[0] = __fadd_rn(__int_as_float(__dp2a_lo((int)w.x, 0x0001, kMBits)), -kM);
+    q[1] = __fadd_rn(__int_as_float(__dp2a_lo((int)w.x, 0x0100, kMBits)), -kM);
+    q[2] = __fadd_rn(__int_as_float(__dp2a_lo((int)w.y, 0x0001, kMBits)), -kM);
+    q[3] = __fadd_rn(__int_as_float(__dp2a_lo((int)w.y, 0x0100, kMBits)), -kM);
   }
 }
 

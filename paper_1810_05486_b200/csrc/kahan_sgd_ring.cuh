@@ -58,6 +58,8 @@ constexpr int kSlots = 6;              // tiles a block can have in its ring at 
 constexpr int kPageBytes = 8192;       // the ring is handed out in pages
 static_assert(kChunk == 8192 && kPageBytes == kChunk, "the producer's page arithmetic assumes 8192-element tiles and 8 KB pages");
 constexpr int kPages = 28;             // 224 KB of tile data per block
+constexpr int kLongStepTiles = 64;     // a block with at least this many tiles limits its tiles in flight
+constexpr int kTilesInFlight = 2;      // ... to this many
 constexpr int kInlineArgs = 256;     // lists up to this long pass grads/lrs as kernel parameters
 constexpr int kUploadBatch = 1024;   // tensors per launch of the argument-upload kernel
 constexpr int kDLimit = 1 << 30;     // clamp of the quantized increment, in compensation LSBs
@@ -480,8 +482,24 @@ __device__ __forceinline__ void ring_step(const typename P::Params& p, const Arg
       // issued, `oldest` is the first tile whose pages have not been taken back yet.
       int head = 0, free_pages = kPages, oldest = 0;
       bool gave_up = false;
+      // A long step is bound by DRAM, and DRAM serves it faster with fewer requests queued:
+      // there at most kTilesInFlight tiles are on their way at once (before issuing a tile the
+      // producer waits for the tile that many places back to have landed).  The pages still
+      // hold up to three and a half tiles, so landed tiles wait for the consumers as before.
+      // The wait stands before the tile's bookkeeping, not directly before its copies: the
+      // few hundred nanoseconds between are part of what the limit buys (measured both ways).
+      const bool long_step = n_my >= kLongStepTiles;
       for (int i = 0; i < n_my; ++i) {
         const int slot = i % kSlots;
+        if (long_step && i >= kTilesInFlight) {
+          const int w = i - kTilesInFlight;
+          if (!mbar_wait(&sh->full[w % kSlots], (unsigned)(w / kSlots) & 1u, &sh->abort_flag)) {
+            // this tile is never issued: its barrier stays open and the consumers leave on the flag
+            sh->abort_flag = 1;
+            atomicCAS(p.ws.error, 0u, (unsigned)kErrFullWait);
+            break;
+          }
+        }
         ChunkRef cr2{-1, -1};
         if (i + 2 < n_my) cr2 = p.ws.chunks[tile0 + (i + 2) * stride];
         Meta meta1 = meta;
@@ -566,13 +584,13 @@ __device__ __forceinline__ void ring_step(const typename P::Params& p, const Arg
         P::fill_desc(sh->desc[slot], p, meta, cr.tensor, count, n_bulk, page, gptr);
         if (i != 0) issue_copies();
         mbar_arrive(&sh->full[slot]);
+        issued = i + 1;
         // With its last tile on the way the block lets the next kernel of the stream go ahead:
         // once every block has said so, blocks of that kernel take over SMs as ours exit, set
         // up and wait (grid_dependency_wait) for this kernel to complete.  Said at the start
         // instead, blocks of the next kernel sit on the early finishers' SMs for a large part
         // of a long step, which measurably slows the blocks still at work.
         if (i == n_my - 1) grid_dependency_launch_dependents();
-        issued = i + 1;
         cr = cr1;
         cr1 = cr2;
         meta = meta1;

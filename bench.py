@@ -139,6 +139,8 @@ def parse_args():
                     help="skip the momentum / ADAM / int8-gradient legs that the default run adds to its line")
     ap.add_argument("--no-convert", action="store_true",
                     help="skip the fp32 <-> fixed-point conversion leg that the default run adds to its line")
+    ap.add_argument("--convert-only", action="store_true",
+                    help="time the fp32 <-> fixed-point conversion leg alone and print it as one JSON line")
     ap.add_argument("--sustained-s", type=float, default=0.35,
                     help="length of the sustained leg (the same steps repeated for about this long, with the "
                          "clocks sampled inside it); 0 skips it")
@@ -407,6 +409,14 @@ def run_ours(args, rank, world, local_rank):
     from paper_1810_05486_b200.runner import DeviceRun, HostInputs
 
     torch.cuda.set_device(local_rank)
+    if args.convert_only:
+        if rank == 0:
+            peak, peak_src = hbm_peak()
+            with torch.cuda.stream(torch.cuda.Stream()):
+                rows = convert_leg(torch, B, peak)
+            print(json.dumps({"convert": rows, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
+                              "gpu_launches": B.kahan_sgd_launch_count()}), flush=True)
+        return
     dist = None
     if world > 1:
         import torch.distributed as dist

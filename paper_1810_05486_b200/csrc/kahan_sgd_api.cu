@@ -363,7 +363,7 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   double state_bytes = 0.0;
   for (int32_t i = 0; i < n_tensors; ++i)
     state_bytes += (double)descs[i].numel * ((descs[i].theta_bits + descs[i].comp_bits) / 8);
-  h->params.grad_evict_first = state_bytes <= 0.8 * (double)l2_bytes ? 1 : 0;
+  h->params.state_in_l2 = state_bytes <= 0.8 * (double)l2_bytes ? 1 : 0;
   h->params.chunk8 = chunk8;
 
   e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
@@ -804,7 +804,7 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   params.tile_count = (int)L.n_chunks;
   params.tensor_begin = 0;
   params.tensor_count = n_tensors;
-  params.grad_evict_first = state_bytes <= 0.8 * (double)sd.l2_bytes ? 1 : 0;
+  params.state_in_l2 = state_bytes <= 0.8 * (double)sd.l2_bytes ? 1 : 0;
   params.chunk8 = kChunk;
   params.advance = 1;
   params.exp_grad_dev = nullptr;
@@ -972,7 +972,7 @@ int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* 
     return cuda_fail(e, "device query");
   }
   h->grid = (int)(L.n_chunks < (long long)dev.sms ? L.n_chunks : (long long)dev.sms);
-  h->params.grad_evict_first = state_bytes <= 0.8 * (double)dev.l2_bytes ? 1 : 0;
+  h->params.state_in_l2 = state_bytes <= 0.8 * (double)dev.l2_bytes ? 1 : 0;
 
   e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
@@ -1185,7 +1185,7 @@ int kahan_sgd_adam_init(ksgd_adam_handle** out, const ksgd_tensor_desc* descs, c
     return cuda_fail(e, "device query");
   }
   h->grid = (int)(L.n_chunks < (long long)dev.sms ? L.n_chunks : (long long)dev.sms);
-  h->params.grad_evict_first = state_bytes <= 0.8 * (double)dev.l2_bytes ? 1 : 0;
+  h->params.state_in_l2 = state_bytes <= 0.8 * (double)dev.l2_bytes ? 1 : 0;
 
   e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);

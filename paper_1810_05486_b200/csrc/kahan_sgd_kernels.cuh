@@ -68,7 +68,7 @@ struct StepParams {
   int n_chunks;
   int amax_mode;     // 1: exponents follow the max scan, 0: fixed
   int inline_args;   // 1: grads/lrs are in the InlineArgs parameter
-  int grad_evict_first;  // 1: gradient loads carry the L2 evict-first hint
+  int state_in_l2;       // 1: theta and c of the whole list fit in L2 and stay there from step to step
   const int* exp_grad_dev;   // fixed-point gradients: device array of their exponents (as a scan on the
                              // device left them), or nullptr: the exponents come with the per-step arguments
   int advance;           // 1: this launch ends a step (the phase word moves on); 0: more launches of the
@@ -143,6 +143,7 @@ struct __align__(16) TileDesc {
 constexpr int kFlagFormatMask = 7;   // 0..5 = (8,0) (8,8) (8,16) (16,0) (16,8) (16,16)
 constexpr int kFlagSteady = 8;       // no exponent change: the exact-fp32 path applies
 constexpr int kFlagRegrid = 16;      // theta's exponent changes: the exact-fp32 re-gridding path applies
+constexpr int kFlagStream = 32;      // the list does not stay in L2: results are stored with the streaming hint
 constexpr int kFlagThetaPageShift = 8;   // 5 bits each: first ring page of theta, c, g
 constexpr int kFlagCompPageShift = 13;
 constexpr int kFlagGradPageShift = 18;
@@ -491,6 +492,7 @@ __device__ __forceinline__ bool consume_tile(const TileHot& h, const TileDesc* t
   constexpr int CBYTES = HAS_COMP ? V * CB / 8 : 8;
   constexpr int GBYTES = V * GB / 8;
   const bool steady = (h.flags & kFlagSteady) != 0;
+  const bool stream = (h.flags & kFlagStream) != 0;
   unsigned char* theta_s = ring + ((h.flags >> kFlagThetaPageShift) & 31) * kPageBytes;
   unsigned char* comp_s = ring + ((h.flags >> kFlagCompPageShift) & 31) * kPageBytes;
   const unsigned char* grad_s = ring + ((h.flags >> kFlagGradPageShift) & 31) * kPageBytes;
@@ -514,8 +516,13 @@ __device__ __forceinline__ bool consume_tile(const TileHot& h, const TileDesc* t
       if constexpr (HAS_COMP) oc = load_pack<CBYTES>(comp_s + v * CBYTES);
       wrote_stage = true;
     }
-    store_pack<TBYTES>(h.theta + (size_t)v * TBYTES, ot);
-    if constexpr (HAS_COMP) store_pack<CBYTES>(h.comp + (size_t)v * CBYTES, oc);
+    if (stream) {
+      store_pack_streaming<TBYTES>(h.theta + (size_t)v * TBYTES, ot);
+      if constexpr (HAS_COMP) store_pack_streaming<CBYTES>(h.comp + (size_t)v * CBYTES, oc);
+    } else {
+      store_pack<TBYTES>(h.theta + (size_t)v * TBYTES, ot);
+      if constexpr (HAS_COMP) store_pack<CBYTES>(h.comp + (size_t)v * CBYTES, oc);
+    }
   }
   // ragged tail (fewer than 16 elements) that the bulk copies did not bring: in place in
   // global memory
@@ -706,6 +713,8 @@ struct PlainPolicy {
   static constexpr int kStreams = 3;          // gradient, theta, c
   static constexpr int kConsumerWarps = ksgd::kConsumerWarps;
   static constexpr int kAmax = 2, kCounts = 3;
+  static constexpr int kLongStepTiles = 16;   // tiles per block from which the ring limits its tiles in flight
+  static constexpr bool kGradEvictFirstBeyondL2 = true;
   using Params = StepParams;
   using Info = TensorInfo;
   using State = TensorState;
@@ -763,6 +772,7 @@ struct PlainPolicy {
            ((coef.delta == 0 && scale_ok && (!STRICT || coef.s >= 0)) ? kFlagSteady : 0) |
            // a coarser grid splits theta's mantissa at bit delta: that needs delta <= theta_bits - 1
            ((!STRICT && coef.delta != 0 && scale_ok && coef.delta <= ti.theta_bits - 1) ? kFlagRegrid : 0) |
+           (p.state_in_l2 ? 0 : kFlagStream) |
            (page[1] << kFlagThetaPageShift) |
            (page[2] << kFlagCompPageShift) | (page[0] << kFlagGradPageShift);
     td.coef = coef;

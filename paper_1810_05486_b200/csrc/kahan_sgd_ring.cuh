@@ -31,8 +31,10 @@
 //   kStreams            arrays per tile; stream 0 is the gradient (read once)
 //   kConsumerWarps      consumer warps per block (one more warp produces)
 //   kAmax, kCounts      max scans and counters per tensor
+//   kLongStepTiles      tiles per block from which a step beyond L2 limits its tiles in flight
+//   kGradEvictFirstBeyondL2   gradient loads carry the L2 evict-first hint also when the state does not fit in L2
 //   Params              kernel parameter with: ws.phase, ws.state, ws.slab, ws.counters, ws.error,
-//                       ws.info, ws.chunks; n_tensors, tile_begin, tile_count, advance, grad_evict_first
+//                       ws.info, ws.chunks; n_tensors, tile_begin, tile_count, advance, state_in_l2
 //   Info                the tensor table entry (with numel); State: the per-step record, whose
 //                       member amax[kAmax] the blocks add their scans to
 //   TileDesc, TileScan  what the producer tells the consumers about a tile; the tile's scan
@@ -58,8 +60,7 @@ constexpr int kSlots = 6;              // tiles a block can have in its ring at 
 constexpr int kPageBytes = 8192;       // the ring is handed out in pages
 static_assert(kChunk == 8192 && kPageBytes == kChunk, "the producer's page arithmetic assumes 8192-element tiles and 8 KB pages");
 constexpr int kPages = 28;             // 224 KB of tile data per block
-constexpr int kLongStepTiles = 64;     // a block with at least this many tiles limits its tiles in flight
-constexpr int kTilesInFlight = 2;      // ... to this many
+constexpr int kTilesInFlight = 2;      // tiles on their way at once in a step that streams from DRAM (ring_step)
 constexpr int kInlineArgs = 256;     // lists up to this long pass grads/lrs as kernel parameters
 constexpr int kUploadBatch = 1024;   // tensors per launch of the argument-upload kernel
 constexpr int kDLimit = 1 << 30;     // clamp of the quantized increment, in compensation LSBs
@@ -224,6 +225,20 @@ __device__ __forceinline__ void store_pack(void* p, const Pack<BYTES>& r) {
   } else {
 #pragma unroll
     for (int i = 0; i < BYTES / 16; ++i) reinterpret_cast<uint4*>(p)[i] = r.v[i];
+  }
+}
+
+// The same to global memory with the streaming (evict-first) hint: for results that will not
+// be read again before they have left L2 anyway, so that they leave it promptly and in order.
+template <int BYTES>
+__device__ __forceinline__ void store_pack_streaming(void* p, const Pack<BYTES>& r) {
+  if constexpr (BYTES == 8) {
+    __stcs(reinterpret_cast<uint2*>(p), r.v);
+  } else if constexpr (BYTES == 16) {
+    __stcs(reinterpret_cast<uint4*>(p), r.v);
+  } else {
+#pragma unroll
+    for (int i = 0; i < BYTES / 16; ++i) __stcs(reinterpret_cast<uint4*>(p) + i, r.v[i]);
   }
 }
 
@@ -482,13 +497,16 @@ __device__ __forceinline__ void ring_step(const typename P::Params& p, const Arg
       // issued, `oldest` is the first tile whose pages have not been taken back yet.
       int head = 0, free_pages = kPages, oldest = 0;
       bool gave_up = false;
-      // A long step is bound by DRAM, and DRAM serves it faster with fewer requests queued:
-      // there at most kTilesInFlight tiles are on their way at once (before issuing a tile the
-      // producer waits for the tile that many places back to have landed).  The pages still
+      // A step that streams everything from DRAM (state too large to stay in L2, at least
+      // P::kLongStepTiles tiles per block) is bound by DRAM, and DRAM serves it faster with
+      // fewer requests queued: there at most kTilesInFlight tiles are on their way at once
+      // (before issuing a tile the producer waits for the tile that many places back to have
+      // landed).  With the state resident in L2 the limit costs about 3 %, so it is left out;
+      // the tile count from which it pays is measured per optimizer.  The pages still
       // hold up to three and a half tiles, so landed tiles wait for the consumers as before.
       // The wait stands before the tile's bookkeeping, not directly before its copies: the
       // few hundred nanoseconds between are part of what the limit buys (measured both ways).
-      const bool long_step = n_my >= kLongStepTiles;
+      const bool long_step = n_my >= P::kLongStepTiles && !p.state_in_l2;
       for (int i = 0; i < n_my; ++i) {
         const int slot = i % kSlots;
         if (long_step && i >= kTilesInFlight) {
@@ -568,8 +586,11 @@ __device__ __forceinline__ void ring_step(const typename P::Params& p, const Arg
               if (bytes[r])
                 bulk_load(smem + page[r] * kPageBytes, gptr[r], (unsigned)(n_bulk * bytes[r]), &sh->full[slot]);
             // Gradients are read once.  When the state of the whole list fits in L2, letting
-            // the gradients leave it first keeps the state resident from step to step.
-            if (p.grad_evict_first)
+            // the gradients leave it first keeps the state resident from step to step.  When
+            // it does not, the hint makes their lines give way at once instead of ageing out:
+            // 1 to 3 % for the plain optimizer, a loss of 2 % with the three or four state
+            // arrays of the others (measured), hence the policy's say.
+            if (p.state_in_l2 || P::kGradEvictFirstBeyondL2)
               bulk_load_hint(smem + page[0] * kPageBytes, gptr[0], (unsigned)(n_bulk * bytes[0]), &sh->full[slot],
                              grad_policy);
             else

@@ -121,14 +121,16 @@ __device__ __forceinline__ void quantize_one(float x, float inv2e, float pow2s, 
   }
 }
 
+// (streaming stores: the mantissas are not read again soon, and must not push the source of an
+// import out of L2 before the quantization has read it)
 template <int BITS>
 __device__ __forceinline__ void store4(void* base, long long i4, const int (&q)[4]) {
   if constexpr (BITS == 8) {
-    reinterpret_cast<unsigned int*>(base)[i4] = (unsigned int)(q[0] & 0xff) | ((unsigned int)(q[1] & 0xff) << 8) |
-                                                ((unsigned int)(q[2] & 0xff) << 16) | ((unsigned int)q[3] << 24);
+    __stcs(reinterpret_cast<unsigned int*>(base) + i4, (unsigned int)(q[0] & 0xff) | ((unsigned int)(q[1] & 0xff) << 8) |
+                                                           ((unsigned int)(q[2] & 0xff) << 16) | ((unsigned int)q[3] << 24));
   } else {
-    reinterpret_cast<uint2*>(base)[i4] = make_uint2((unsigned int)(q[0] & 0xffff) | ((unsigned int)q[1] << 16),
-                                                    (unsigned int)(q[2] & 0xffff) | ((unsigned int)q[3] << 16));
+    __stcs(reinterpret_cast<uint2*>(base) + i4, make_uint2((unsigned int)(q[0] & 0xffff) | ((unsigned int)q[1] << 16),
+                                                           (unsigned int)(q[2] & 0xffff) | ((unsigned int)q[3] << 16)));
   }
 }
 

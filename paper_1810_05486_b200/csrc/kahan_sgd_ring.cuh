@@ -60,7 +60,8 @@ constexpr int kSlots = 6;              // tiles a block can have in its ring at 
 constexpr int kPageBytes = 8192;       // the ring is handed out in pages
 static_assert(kChunk == 8192 && kPageBytes == kChunk, "the producer's page arithmetic assumes 8192-element tiles and 8 KB pages");
 constexpr int kPages = 28;             // 224 KB of tile data per block
-constexpr int kTilesInFlight = 2;      // tiles on their way at once in a step that streams from DRAM (ring_step)
+constexpr int kTilesInFlight = 2;      // a step that streams from DRAM keeps this many tiles on their way, and more
+constexpr int kPagesInFlight = 18;     // only while they take no more than this many pages together (ring_step)
 constexpr int kInlineArgs = 256;     // lists up to this long pass grads/lrs as kernel parameters
 constexpr int kUploadBatch = 1024;   // tensors per launch of the argument-upload kernel
 constexpr int kDLimit = 1 << 30;     // clamp of the quantized increment, in compensation LSBs
@@ -499,19 +500,31 @@ __device__ __forceinline__ void ring_step(const typename P::Params& p, const Arg
       bool gave_up = false;
       // A step that streams everything from DRAM (state too large to stay in L2, at least
       // P::kLongStepTiles tiles per block) is bound by DRAM, and DRAM serves it faster with
-      // fewer requests queued: there at most kTilesInFlight tiles are on their way at once
-      // (before issuing a tile the producer waits for the tile that many places back to have
-      // landed).  With the state resident in L2 the limit costs about 3 %, so it is left out;
-      // the tile count from which it pays is measured per optimizer.  The pages still
-      // hold up to three and a half tiles, so landed tiles wait for the consumers as before.
-      // The wait stands before the tile's bookkeeping, not directly before its copies: the
-      // few hundred nanoseconds between are part of what the limit buys (measured both ways).
+      // fewer requests queued: there kTilesInFlight tiles are on their way at once, and more
+      // only while all of them together take at most kPagesInFlight pages (before issuing a
+      // tile the producer waits for the oldest tiles in flight to land until that holds).
+      // With the state resident in L2 the limit costs about 3 %, so it is left out; the tile
+      // count from which it pays is measured per optimizer.  The ring still holds up to three
+      // and a half tiles, so landed tiles wait for the consumers as before.  The wait stands
+      // before the tile's descriptor is built, not directly before its copies: the few
+      // hundred nanoseconds between are part of what the limit buys (measured both ways).
       const bool long_step = n_my >= P::kLongStepTiles && !p.state_in_l2;
+      int landed = 0, flight_pages = 0;   // first tile not known to have landed; pages of the tiles from there on
+      int last_need = 0;                  // pages of the tile issued last
       for (int i = 0; i < n_my; ++i) {
         const int slot = i % kSlots;
-        if (long_step && i >= kTilesInFlight) {
-          const int w = i - kTilesInFlight;
-          if (!mbar_wait(&sh->full[w % kSlots], (unsigned)(w / kSlots) & 1u, &sh->abort_flag)) {
+        if (long_step) {
+          // the limit on tiles in flight: wait for the oldest of them to land until this one
+          // fits (taken to need the pages its predecessor took: the wait comes first)
+          while (i - landed >= kTilesInFlight && flight_pages + last_need > kPagesInFlight) {
+            if (!mbar_wait(&sh->full[landed % kSlots], (unsigned)(landed / kSlots) & 1u, &sh->abort_flag)) {
+              gave_up = true;
+              break;
+            }
+            flight_pages -= sh->slot_pages[landed % kSlots];
+            ++landed;
+          }
+          if (gave_up) {
             // this tile is never issued: its barrier stays open and the consumers leave on the flag
             sh->abort_flag = 1;
             atomicCAS(p.ws.error, 0u, (unsigned)kErrFullWait);
@@ -561,6 +574,16 @@ __device__ __forceinline__ void ring_step(const typename P::Params& p, const Arg
           sh->abort_flag = 1;
           atomicCAS(p.ws.error, 0u, (unsigned)kErrEmptyWait);
           break;
+        }
+        if (long_step) {
+          // tiles taken back have landed: keep the count of those in flight in step (before
+          // the slot's page count is overwritten)
+          while (landed < oldest) {
+            flight_pages -= sh->slot_pages[landed % kSlots];
+            ++landed;
+          }
+          flight_pages += need;
+          last_need = need;
         }
         head = h2;
         free_pages -= need;

@@ -146,7 +146,8 @@ class DeviceRun:
                 self.dev_gq.append(q)
                 self.gq_ptr_sets.append((ctypes.c_void_p * self.n)(*[q.data_ptr() + o for o in self.q_offs]))
                 self.gq_exp_sets.append((ctypes.c_int32 * self.n)(*exps))
-            self.dev_g = self.dev_g[:1]            # the binary32 copies are no longer needed
+            self.dev_g = self.dev_g[:1]            # the binary32 copies are no longer needed ...
+            self.grad_ptr_sets = self.grad_ptr_sets[:1]   # ... and their addresses must not outlive them
             torch.cuda.empty_cache()
         self.lrs = (ctypes.c_float * self.n)(*([wl.lr] * self.n))
 

@@ -93,6 +93,31 @@ def test_int8_gradients_on_alexnet_shapes_quantized_by_the_import_kernel():
         run.close()
 
 
+def test_one_handle_alternating_int8_and_binary32_gradients_on_alexnet_shapes():
+    """Steps on 8-bit gradients use their own tile table (larger tiles for the 8-bit layers)
+    and leave their records where the next step, on binary32 gradients and the other table,
+    finds them: the two kinds of step alternate on one handle and every tensor is compared
+    after every step."""
+    from oracle import oracle_step
+    from paper_1810_05486_b200 import binding as B
+    wl, host, run, ost = _setup("c4_alexnet", grad_bits=8)
+    try:
+        for step in range(4):
+            if step % 2 == 0:
+                run.step(step)
+                exps = list(run.gq_exp_sets[step])
+                gq = [oracle_quantize(g, 8, 0, 0, e)[0] for g, e in zip(host.grads[step], exps)]
+                oracle_step_qgrad(ost, gq, exps, [wl.lr] * run.n)
+            else:
+                # the runner keeps only the first binary32 gradient set on the device in this mode
+                assert len(run.dev_g) == 1
+                B.kahan_sgd_step(run.handle, run.grad_ptr_sets[0], run.lrs)
+                oracle_step(ost, host.grads[0], [wl.lr] * run.n)
+            _check_common(run, ost, run.stats(), f"step {step}")
+    finally:
+        run.close()
+
+
 def test_strict_algorithm_1_on_resnet50_shapes():
     from paper_1810_05486_b200 import binding as B
     wl, host, run, ost = _setup("c3_resnet50", strict=True)

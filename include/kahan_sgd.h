@@ -135,8 +135,8 @@ int kahan_sgd_step(ksgd_handle* h, const float* const* grads, const float* lrs);
  * everything else as kahan_sgd_step.  Fixed-point gradients can be made from binary32
  * ones with kahan_sgd_import (comp_bits 0, KSGD_EXP_AUTO picks the exponent from the
  * maximum).  The gradient stream shrinks from 4 bytes per parameter to 1 or 2.  Steps on
- * 8-bit gradients of long lists walk a tile table of their own, with larger tiles for the
- * 8-bit tensors (it is part of the workspace that kahan_sgd_workspace_bytes sizes and
+ * 8-bit gradients of long lists walk a tile table of their own, with tiles twice as large
+ * (it is part of the workspace that kahan_sgd_workspace_bytes sizes and
  * kahan_sgd_init fills); which table a step uses changes no result, and steps of either kind
  * may follow one another on one handle.
  */
@@ -224,7 +224,8 @@ int kahan_sgd_set_exponents(ksgd_handle* h, const int32_t* exp_theta_next);
  * the one array and each call rewrites all of it, so two calls whose work overlaps on the
  * GPU (different streams, different threads) race: callers serialise them.  The list is
  * always cut into tiles of 8192 elements (the workspace path takes 16384-element tiles for
- * long lists of 8-bit tensors, 32768 in steps on 8-bit gradients), which changes no result.
+ * long lists of 8-bit tensors, and twice its usual sizes in steps on 8-bit gradients), which
+ * changes no result.
  */
 #define KSGD_STATIC_SCRATCH_BYTES (192 * 1024)
 #define KSGD_STATIC_MAX_TENSORS 256

@@ -127,30 +127,29 @@ long long tile_count(const ksgd_tensor_desc* d, int32_t n, int chunk8) {
   return chunks;
 }
 
-// Steps on 8-bit gradients move so few bytes per parameter (5 for an 8/8 tensor) that what a
-// consumer does per tile, not per element, is a fifth of its instructions with the tiles
-// above.  Lists long enough get a second tile table for those steps, with tiles of 4 * kChunk
-// elements for 8-bit theta (12 of the ring's 28 pages with an 8-bit c and an 8-bit gradient;
-// a 16-bit c would take 16, too many to keep two tiles in the ring, so such lists keep one
-// table).  Returns that tile size, or 0 for no second table.
-int pick_chunk8_qgrad(const ksgd_tensor_desc* d, int32_t n) {
+// Steps on 8-bit gradients move so few bytes per parameter (5 for an 8/8 tensor, 9 for 16/16)
+// that what a consumer does per tile, not per element, is a fifth or more of its instructions
+// with the tiles above.  Lists long enough get a second tile table for those steps, with
+// tiles twice as large as the largest of the first table: 4 * kChunk elements for 8-bit theta
+// (12 of the ring's 28 pages with an 8-bit c and an 8-bit gradient; 2 * kChunk with a 16-bit
+// c, which would take 16), 2 * kChunk for 16-bit theta (6 to 10 pages).  The kernel applies
+// the same rule (PlainPolicy::tile_shift).
+inline long long tile_elems_qgrad(const ksgd_tensor_desc& t) {
+  return t.theta_bits == 8 && t.comp_bits <= 8 ? 4 * kChunk : 2 * kChunk;
+}
+
+// Entries of that table, or 0 for none (short lists keep the small tiles of the first table,
+// with which every block has work).
+long long tile_count_qgrad(const ksgd_tensor_desc* d, int32_t n) {
   long long tiles = 0;
-  bool any8 = false;
-  for (int32_t i = 0; i < n; ++i) {
-    if (d[i].theta_bits == 8) {
-      if (d[i].comp_bits > 8) return 0;
-      any8 = true;
-    }
-    const long long c = tile_elems(d[i], 4 * kChunk);
-    tiles += (d[i].numel + c - 1) / c;
-  }
-  return any8 && tiles >= kBigTileMinTiles ? 4 * kChunk : 0;
+  for (int32_t i = 0; i < n; ++i) tiles += (d[i].numel + tile_elems_qgrad(d[i]) - 1) / tile_elems_qgrad(d[i]);
+  return tiles >= kBigTileMinTiles ? tiles : 0;
 }
 
 // The tile table is the layout's last region: the table for 8-bit gradients, if any, follows
 // the first one in it.
-Layout make_layout(const ksgd_tensor_desc* d, int32_t n, int chunk8, int chunk8_q) {
-  return make_ring_layout(n, tile_count(d, n, chunk8) + (chunk8_q ? tile_count(d, n, chunk8_q) : 0),
+Layout make_layout(const ksgd_tensor_desc* d, int32_t n, int chunk8, bool with_qgrad_table) {
+  return make_ring_layout(n, tile_count(d, n, chunk8) + (with_qgrad_table ? tile_count_qgrad(d, n) : 0),
                           sizeof(TensorState), sizeof(TensorInfo), 3);
 }
 
@@ -171,10 +170,11 @@ void bind_workspace(Workspace& w, char* b, const Layout& L) {
 // Host image of a fresh workspace (`img`: L.total zero bytes): phase 0; in the records the
 // first step reads (slab 2) the exponents of the stored mantissas and, as overrides, the
 // exponents the first step must write; zeroed scans and counters; tensor table; tile
-// table (and, for chunk8_qgrad != 0, the table for steps on 8-bit gradients behind it).
+// table (and, if asked for and the list is long enough for one, the table for steps on 8-bit
+// gradients behind it).
 // first_tile (optional) receives the first tile of every tensor, plus the total.
 void write_initial_image(unsigned char* img, const Layout& L, const ksgd_tensor_desc* descs, int32_t n,
-                         const int32_t* exp_comp, const int32_t* exp_comp_next, int chunk8, int chunk8_qgrad,
+                         const int32_t* exp_comp, const int32_t* exp_comp_next, int chunk8, bool with_qgrad_table,
                          std::vector<long long>* first_tile) {
   TensorState* last = reinterpret_cast<TensorState*>(img + L.state) + 2 * (size_t)L.slab;
   TensorInfo* info = reinterpret_cast<TensorInfo*>(img + L.info);
@@ -200,9 +200,9 @@ void write_initial_image(unsigned char* img, const Layout& L, const ksgd_tensor_
     for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
   }
   if (first_tile) first_tile->push_back(c);
-  if (chunk8_qgrad) {
+  if (with_qgrad_table && tile_count_qgrad(descs, n)) {
     for (int32_t i = 0; i < n; ++i) {
-      const long long nc = (descs[i].numel + tile_elems(descs[i], chunk8_qgrad) - 1) / tile_elems(descs[i], chunk8_qgrad);
+      const long long nc = (descs[i].numel + tile_elems_qgrad(descs[i]) - 1) / tile_elems_qgrad(descs[i]);
       for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
     }
   }
@@ -280,8 +280,8 @@ struct ksgd_handle {
   int sms;
   std::vector<unsigned char> stats_host;   // staging for kahan_sgd_amax
   std::vector<long long> first_tile;       // [n+1] first tile of every tensor
-  int chunk8_qgrad = 0;                    // tile size for 8-bit theta in steps on 8-bit gradients, 0: as in other steps
-  long long tiles_qgrad = 0;               // entries of the tile table for those steps (it follows the first one)
+  long long tiles_qgrad = 0;               // entries of the tile table for steps on 8-bit gradients (it follows
+                                           // the first one), 0: those steps use the first table too
   bool strict = false;                     // strict Algorithm 1: compensation with its own exponent
   // kahan_sgd_step_host: copy streams and events, created on first use
   cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
@@ -292,12 +292,12 @@ extern "C" {
 
 size_t kahan_sgd_workspace_bytes(const ksgd_tensor_desc* descs, int32_t n_tensors) {
   if (validate(descs, n_tensors) != KSGD_OK) return 0;
-  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), pick_chunk8_qgrad(descs, n_tensors)).total;
+  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), true).total;
 }
 
 size_t kahan_sgd_workspace_error_offset(const ksgd_tensor_desc* descs, int32_t n_tensors) {
   if (validate(descs, n_tensors) != KSGD_OK) return (size_t)-1;
-  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), pick_chunk8_qgrad(descs, n_tensors)).error;
+  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), true).error;
 }
 
 }  // extern "C"
@@ -336,8 +336,7 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   if (!workspace) return KSGD_ERR_NULL;
   if (reinterpret_cast<uintptr_t>(workspace) % 256) return KSGD_ERR_ALIGN;
   const int chunk8 = pick_chunk8(descs, n_tensors);
-  const int chunk8_q = pick_chunk8_qgrad(descs, n_tensors);
-  const Layout L = make_layout(descs, n_tensors, chunk8, chunk8_q);
+  const Layout L = make_layout(descs, n_tensors, chunk8, true);
   const long long tiles = tile_count(descs, n_tensors, chunk8);
   if (workspace_bytes < L.total) return KSGD_ERR_WORKSPACE;
 
@@ -352,10 +351,9 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   h->strict = strict;
 
   std::vector<unsigned char> img(L.total, 0);
-  write_initial_image(img.data(), L, descs, n_tensors, strict ? exp_comp : nullptr, exp_comp_next, chunk8, chunk8_q,
+  write_initial_image(img.data(), L, descs, n_tensors, strict ? exp_comp : nullptr, exp_comp_next, chunk8, true,
                       &h->first_tile);
-  h->chunk8_qgrad = chunk8_q;
-  h->tiles_qgrad = chunk8_q ? L.n_chunks - tiles : 0;
+  h->tiles_qgrad = tile_count_qgrad(descs, n_tensors);
   char* b = h->ws_base;
   bind_workspace(h->params.ws, b, L);
   h->params.n_tensors = n_tensors;
@@ -368,6 +366,7 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   h->params.tensor_count = n_tensors;
   h->params.advance = 1;
   h->params.exp_grad_dev = nullptr;
+  h->params.qgrad_tiles = 0;
 
   // Persistent grid: one block per SM (fewer if the list has fewer tiles).
   int dev = 0, sms = 0, l2_bytes = 0;
@@ -431,7 +430,7 @@ size_t kahan_sgd_strict_workspace_bytes(const ksgd_tensor_desc* descs, const int
                                         int32_t n_tensors) {
   if (validate(descs, n_tensors) != KSGD_OK) return 0;
   if (validate_strict(descs, exp_comp, nullptr, n_tensors) != KSGD_OK) return 0;
-  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), pick_chunk8_qgrad(descs, n_tensors)).total;
+  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), true).total;
 }
 
 int kahan_sgd_strict_init(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t* exp_comp,
@@ -566,10 +565,10 @@ static int step_qgrad_common(ksgd_handle* h, const void* const* grads, int32_t g
   StepParams p = h->params;
   p.exp_grad_dev = exp_grad_dev;
   unsigned grid = (unsigned)h->grid;
-  if (grad_bits == 8 && h->chunk8_qgrad) {      // the table of larger tiles, behind the first one
+  if (grad_bits == 8 && h->tiles_qgrad) {       // the table of larger tiles, behind the first one
     p.ws.chunks += p.n_chunks;
     p.n_chunks = p.tile_count = (int)h->tiles_qgrad;
-    p.chunk8 = h->chunk8_qgrad;
+    p.qgrad_tiles = 1;
     grid = (unsigned)(h->tiles_qgrad < (long long)h->sms ? h->tiles_qgrad : (long long)h->sms);
   }
   auto kernel = h->strict ? (grad_bits == 8 ? ksgd_strict_step_qgrad_kernel<8> : ksgd_strict_step_qgrad_kernel<16>)
@@ -800,7 +799,7 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   if (mode != KSGD_EXP_FIXED && mode != KSGD_EXP_AMAX) return KSGD_ERR_MODE;
   if (!grads || !lrs) return KSGD_ERR_NULL;
   if (n_tensors > KSGD_STATIC_MAX_TENSORS) return KSGD_ERR_WORKSPACE;
-  const Layout L = make_layout(descs, n_tensors, kChunk, 0);
+  const Layout L = make_layout(descs, n_tensors, kChunk, false);
   if (L.total > (size_t)KSGD_STATIC_SCRATCH_BYTES) return KSGD_ERR_WORKSPACE;
   for (int32_t i = 0; i < n_tensors; ++i) {
     if (!grads[i]) return KSGD_ERR_NULL;
@@ -833,7 +832,7 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   // Host image of the scratch, every byte of it: whatever the previous call left in the
   // array (scans, counters, phase and tickets) is overwritten.
   std::vector<unsigned char> img(L.total, 0);
-  write_initial_image(img.data(), L, descs, n_tensors, nullptr, nullptr, kChunk, 0, nullptr);
+  write_initial_image(img.data(), L, descs, n_tensors, nullptr, nullptr, kChunk, false, nullptr);
   double state_bytes = 0.0;
   for (int32_t i = 0; i < n_tensors; ++i)
     state_bytes += (double)descs[i].numel * ((descs[i].theta_bits + descs[i].comp_bits) / 8);
@@ -854,6 +853,7 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   params.chunk8 = kChunk;
   params.advance = 1;
   params.exp_grad_dev = nullptr;
+  params.qgrad_tiles = 0;
 
   InlineArgs inl;
   for (int32_t i = 0; i < n_tensors; ++i) { inl.grads[i] = grads[i]; inl.lrs[i] = lrs[i]; }

@@ -77,12 +77,14 @@ struct StepParams {
   // of tensors [tensor_begin, tensor_begin + tensor_count): the whole list for an ordinary
   // step, one group of tensors when the host-buffer entry point pipelines its copies.
   int tile_begin, tile_count, tensor_begin, tensor_count;
-  // Elements per tile of tensors with 8-bit theta in the tile table this launch uses:
-  // kChunk, or 2 * kChunk for lists long enough to keep every block busy with the larger
-  // tiles (one vector per thread and tile leaves the per-tile work of a consumer -- wait,
-  // descriptor, scans, arrive -- a third of its instructions), or 4 * kChunk in steps on
-  // 8-bit gradients of such lists.  Tensors with 16-bit theta always take kChunk.
+  // Elements per tile of tensors with 8-bit theta in the list's first tile table: kChunk, or
+  // 2 * kChunk for lists long enough to keep every block busy with the larger tiles (one
+  // vector per thread and tile leaves the per-tile work of a consumer -- wait, descriptor,
+  // scans, arrive -- a third of its instructions).  Tensors with 16-bit theta take kChunk.
   int chunk8;
+  // 1: this launch walks the table for steps on 8-bit gradients, whose tiles are twice as
+  // large again (4 * kChunk for 8-bit theta with an 8-bit or no c, 2 * kChunk otherwise)
+  int qgrad_tiles;
 };
 
 struct InlineArgs {
@@ -732,10 +734,12 @@ struct PlainPolicy {
   }
   // Tensors with 8-bit theta take tiles of 2 * kChunk elements in lists long enough to keep
   // every block busy with them (one vector per thread and tile leaves the per-tile work of a
-  // consumer -- wait, descriptor, scans, arrive -- a third of its instructions), and of
-  // 4 * kChunk in steps on 8-bit gradients (the host picks; p.chunk8 is the size).
+  // consumer -- wait, descriptor, scans, arrive -- a third of its instructions); the table
+  // for steps on 8-bit gradients has tiles twice as large again for every tensor (the same
+  // rule as the host's tile_elems_qgrad).
   static __device__ __forceinline__ int tile_shift(const Params& p, const Meta& m) {
-    return m.ti.theta_bits == 8 ? (p.chunk8 >> 14) : 0;   // 8192, 16384, 32768 -> 0, 1, 2
+    if (p.qgrad_tiles) return (m.ti.theta_bits == 8 && m.ti.comp_bits <= 8) ? 2 : 1;
+    return (m.ti.theta_bits == 8 && p.chunk8 != kChunk) ? 1 : 0;
   }
   static __device__ __forceinline__ void streams(const Meta& m, const unsigned char* (&base)[kStreams],
                                                  int (&bytes)[kStreams]) {

@@ -108,6 +108,8 @@ class LibraryRun:
             self.qgrad_arena = DeviceArena([s["numel"] * 2 for s in self.specs])
         for i, g in enumerate(grads_q):
             assert g.dtype == storage_dtype(bits) and g.size == self.specs[i]["numel"]
+            if g.nbytes < self.qgrad_arena.sizes[i]:      # narrower gradients than last time: the rest is guard again
+                self.qgrad_arena.view(i)[g.nbytes:] = CANARY
             self.qgrad_arena.sizes[i] = g.nbytes
             self.qgrad_arena.upload(i, g)
         self.B.kahan_sgd_step_qgrad(self.handle, [self.qgrad_arena.ptr(i) for i in range(self.n)], bits,

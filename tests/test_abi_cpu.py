@@ -94,17 +94,23 @@ def test_workspace_grows_with_the_chunk_table(B):
 
 
 def test_long_lists_of_8bit_theta_get_the_large_tiles(B):
-    """The tile table (8 bytes per tile) shows which tile size a list got: 8192 elements,
-    or 16384 for 8-bit theta once the list still has 1024 tiles with them; 16-bit theta
-    always keeps 8192."""
+    """The tile tables (8 bytes per tile) show which tile sizes a list got.  First table: 8192
+    elements, or 16384 for 8-bit theta once the list still has 1024 tiles with them; 16-bit
+    theta always keeps 8192.  A second table, for steps on 8-bit gradients, once the list has
+    1024 tiles of twice those sizes (32768 for 8-bit theta with an 8-bit c, 16384 otherwise)."""
     def table_bytes(numel, **kw):
         return (B.kahan_sgd_workspace_bytes(B.make_descs([good(numel=numel, **kw)])) -
                 B.kahan_sgd_workspace_bytes(B.make_descs([good(numel=1, **kw)])))
     short, long_ = 1023 * 16384, 1024 * 16384
-    assert abs(table_bytes(short) - 8 * (short // 8192)) <= 512          # small tiles
-    assert abs(table_bytes(long_) - 8 * 1024) <= 512                     # large tiles
+    assert abs(table_bytes(short) - 8 * (short // 8192)) <= 512          # small tiles, one table
+    assert abs(table_bytes(long_) - 8 * 1024) <= 512                     # large tiles, one table
+    longer = 1024 * 32768
+    assert abs(table_bytes(longer) - 8 * (2048 + 1024)) <= 512           # and 1024 tiles of 32768 in the second
     wide = dict(theta_bits=16, comp_bits=16)
-    assert abs(table_bytes(long_, **wide) - 8 * (long_ // 8192)) <= 512  # 16-bit theta: small tiles
+    assert abs(table_bytes(short, **wide) - 8 * (short // 8192)) <= 512  # 16-bit theta: small tiles, one table
+    assert abs(table_bytes(long_, **wide) - 8 * (long_ // 8192 + 1024)) <= 512   # second table: 1024 tiles of 16384
+    mixed = dict(theta_bits=8, comp_bits=16)                             # 8-bit theta with a 16-bit c: 16384 in both
+    assert abs(table_bytes(long_, **mixed) - 8 * (1024 + 1024)) <= 512
 
 
 def test_null_handles_and_strerror(B):

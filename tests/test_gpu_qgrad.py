@@ -115,3 +115,36 @@ def test_resnet20_shapes_with_gradients_quantized_by_the_import_rule():
         grads.append([oracle_quantize(g, 8, 0, 0, ei)[0] for g, ei in zip(gs, e)])
         exps.append(e)
     run_both(specs, thetas, comps, grads, exps, [wl.lr] * len(specs))
+
+
+def test_int8_gradients_on_a_list_long_enough_for_the_second_tile_table_every_format():
+    """Steps on 8-bit gradients of long lists walk their own tile table (32768 elements per
+    tile for 8-bit theta with an 8-bit or no c, 16384 for everything else).  Six tensors, one
+    per format, ragged sizes, 1300 such tiles in all; a step on 16-bit gradients and one on
+    8-bit gradients again, on the same handle, follow (the first table and back)."""
+    rng = np.random.default_rng(77)
+    sizes = {(8, 0): 250 * 32768 + 5, (8, 8): 250 * 32768 + 32767, (8, 16): 200 * 16384 + 16383,
+             (16, 0): 200 * 16384 + 1, (16, 8): 200 * 16384 + 8191, (16, 16): 200 * 16384 + 17}
+    specs, thetas, comps = [], [], []
+    for (tb, cb), n in sizes.items():
+        t, c = random_state(rng, n, tb, cb)
+        specs.append(dict(numel=n, theta_bits=tb, comp_bits=cb, exp_theta=-9 if tb == 8 else -15))
+        thetas.append(t); comps.append(c)
+
+    def grads(gb):
+        return [rng.integers(-2 ** (gb - 1), 2 ** (gb - 1), sp["numel"]).astype(storage_dtype(gb)) for sp in specs]
+
+    def exps(gb):
+        return [sp["exp_theta"] - (sp["comp_bits"] - 1 if sp["comp_bits"] else 0) - gb + 5 for sp in specs]
+    lrs = [0.1] * len(specs)
+    gpu = LibraryRun(specs, thetas, comps, EXP_AMAX)
+    ost = make_oracle_state(specs, thetas, comps, EXP_AMAX, oracle_max_threads())
+    try:
+        for step, gb in enumerate((8, 8, 16, 8)):
+            gq, eg = grads(gb), exps(gb)
+            gpu.step_qgrad(gq, eg, lrs)
+            oracle_step_qgrad(ost, gq, eg, lrs)
+            assert_same_state(gpu, ost, f"step {step} ({gb}-bit gradients)")
+        assert gpu.guards_intact()
+    finally:
+        gpu.close()

@@ -133,3 +133,26 @@ def test_strict_algorithm_1_on_resnet50_shapes():
         assert ec["exp_comp_next"] == [t.exp_comp_next for t in ost.tensors]
     finally:
         run.close()
+
+
+def test_strict_algorithm_1_on_int8_gradients_on_alexnet_shapes():
+    """Both of the paper's hardware-faithful modes together (INT8 gradients, the accumulator
+    rounded into n bits with its own exponent) at full size; these steps walk the tile table
+    of large tiles."""
+    from oracle import oracle_dequantize_gradient
+    from paper_1810_05486_b200 import binding as B
+    wl, host, run, ost = _setup("c4_alexnet", strict=True, grad_bits=8)
+    try:
+        for t in ost.tensors:
+            t.exp_comp = t.exp_comp_next = t.exp_theta - (t.comp_bits - 1 - t.overlap_k)
+        for step in range(4):
+            run.step(step)
+            exps = list(run.gq_exp_sets[step])
+            gq = [oracle_quantize(g, 8, 0, 0, e)[0] for g, e in zip(host.grads[step], exps)]
+            oracle_strict_step(ost, [oracle_dequantize_gradient(q, e) for q, e in zip(gq, exps)], [wl.lr] * run.n)
+        _check_common(run, ost, run.stats(), "strict, int8 gradients")
+        ec = B.kahan_sgd_strict_exponents(run.handle, run.n)
+        assert ec["exp_comp_cur"] == [t.exp_comp for t in ost.tensors]
+        assert ec["exp_comp_next"] == [t.exp_comp_next for t in ost.tensors]
+    finally:
+        run.close()

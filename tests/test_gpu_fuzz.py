@@ -1,0 +1,154 @@
+"""Randomised differential test of the CUDA library against the CPU oracle.
+
+Every case draws, from one seed, a ragged list of tensors (formats, overlaps, sizes around
+the tile borders, exponents), and then a sequence of steps in which the kind of gradient
+(binary32, INT8, INT16), its magnitude (from far below the compensation's unit to far above
+theta's range, so that exponents move both ways and both clamps fire), the learning rates
+and an occasional forced exponent all vary.  The whole state is compared bit for bit after
+every step (Algorithm 1 is defined per element, so every element is in scope)."""
+import numpy as np
+import pytest
+
+from harness import LibraryRun, assert_same_state, make_oracle_state, storage_dtype
+from oracle import (EXP_AMAX, EXP_FIXED, oracle_dequantize_gradient, oracle_max_threads, oracle_step,
+                    oracle_step_qgrad, oracle_strict_step)
+
+pytestmark = pytest.mark.gpu
+
+FORMATS = [(8, 0), (8, 8), (8, 16), (16, 0), (16, 8), (16, 16)]
+BORDER_SIZES = [1, 2, 15, 16, 17, 31, 33, 255, 4095, 4096, 8191, 8192, 8193, 16383, 16384, 16385, 24577,
+                32767, 32768, 32769, 65537]
+SPECIALS = np.array([np.inf, -np.inf, np.nan, 3.0e38, -3.0e38, 1.0e-45, -0.0], np.float32)
+
+
+def draw_size(rng):
+    kind = rng.integers(0, 3)
+    if kind == 0:
+        return int(BORDER_SIZES[rng.integers(0, len(BORDER_SIZES))])
+    if kind == 1:
+        return int(rng.integers(1, 3000))
+    return int(rng.integers(3000, 150000))
+
+
+def draw_list(rng, strict):
+    n_tensors = int(rng.integers(1, 14))
+    if rng.random() < 0.15:
+        n_tensors = int(rng.integers(257, 300))      # beyond the inline argument block
+    specs, thetas, comps = [], [], []
+    for _ in range(n_tensors):
+        tb, cb = FORMATS[rng.integers(0, len(FORMATS))]
+        if strict and cb == 0:
+            cb = 8 if rng.random() < 0.5 else 16
+        numel = draw_size(rng) if n_tensors < 100 else int(rng.integers(1, 2000))
+        k = int(rng.integers(0, cb)) if (cb and not strict and rng.random() < 0.3) else 0
+        e = int(rng.integers(-30, 10))
+        full = rng.random() < 0.3
+        lim_t = 2 ** (tb - 1) if full else 2 ** (tb - 2)
+        theta = rng.integers(-lim_t, lim_t, numel).astype(storage_dtype(tb))
+        comp = None
+        if cb:
+            lim_c = 2 ** (cb - 1) if full else 2 ** (cb - 2)
+            comp = rng.integers(-lim_c, lim_c, numel).astype(storage_dtype(cb))
+        spec = dict(numel=numel, theta_bits=tb, comp_bits=cb, overlap_k=k, exp_theta=e)
+        if strict:
+            # anywhere in the window the library accepts: 8 above to 36 below theta's exponent
+            spec["exp_comp"] = max(-64, e - int(rng.integers(-8, 37)))
+        specs.append(spec)
+        thetas.append(theta)
+        comps.append(comp)
+    return specs, thetas, comps
+
+
+def comp_unit_exponent(t, strict):
+    """Exponent of one compensation LSB of oracle tensor t as the coming step writes it."""
+    if strict:
+        return t.exp_comp_next
+    s = t.comp_bits - 1 - t.overlap_k if t.comp_bits else 0
+    return t.exp_theta_next - s
+
+
+def draw_float_grads(rng, ost, strict, lrs):
+    grads = []
+    for t, lr in zip(ost.tensors, lrs):
+        n = t.theta.size
+        # increments of 2^-6 compensation units up to a few units of theta (the exact
+        # steady path), in a third of the draws up to far beyond theta's range (clamps,
+        # coarser grids)
+        span = (t.comp_bits or 1) + 2
+        if rng.random() < 0.33:
+            span += t.theta_bits + 1
+        mag = 2.0 ** (comp_unit_exponent(t, strict) + float(rng.uniform(-6, span))) / lr
+        g = (rng.standard_normal(n) * mag).astype(np.float32)
+        if rng.random() < 0.25:
+            idx = rng.choice(n, min(n, 5), replace=False)
+            g[idx] = SPECIALS[rng.integers(0, len(SPECIALS), idx.size)]
+        if rng.random() < 0.1:
+            g[:] = 0.0
+        grads.append(g)
+    return grads
+
+
+def draw_fixed_grads(rng, ost, strict, lrs, gb):
+    grads, exps = [], []
+    for t, lr in zip(ost.tensors, lrs):
+        n = t.theta.size
+        g = rng.integers(-2 ** (gb - 1), 2 ** (gb - 1), n).astype(storage_dtype(gb))
+        if rng.random() < 0.3:                      # a grid fixed by one outlier, the rest small
+            g = (g // 2 ** (gb - 3)).astype(storage_dtype(gb))
+            g[rng.integers(0, n)] = 2 ** (gb - 1) - 1
+        # one gradient unit times lr worth 2^-5 .. 2^10 compensation units
+        eg = comp_unit_exponent(t, strict) + int(rng.integers(-5, 11)) - int(np.round(np.log2(lr)))
+        grads.append(g)
+        exps.append(int(np.clip(eg, -64, 64)))
+    return grads, exps
+
+
+def draw_lrs(rng, n):
+    if rng.random() < 0.5:
+        return [float(np.float32(2.0 ** rng.integers(-6, 3)))] * n
+    return [float(np.float32(rng.uniform(1e-3, 2.0))) for _ in range(n)]
+
+
+def run_case(seed, strict, steps):
+    rng = np.random.default_rng([seed, int(strict)])
+    specs, thetas, comps = draw_list(rng, strict)
+    mode = EXP_FIXED if rng.random() < 0.15 else EXP_AMAX
+    gpu = LibraryRun(specs, thetas, comps, mode, strict=strict)
+    ost = make_oracle_state(specs, thetas, comps, mode, oracle_max_threads())
+    n = len(specs)
+    kinds = []
+    try:
+        for step in range(steps):
+            lrs = draw_lrs(rng, n)
+            if not strict and rng.random() < 0.2:
+                want = [int(np.clip(t.exp_theta + rng.integers(-10, 11), -64, 64)) for t in ost.tensors]
+                gpu.set_exponents(want)
+                for t, e in zip(ost.tensors, want):       # the device limits the change to 8 binades
+                    t.exp_theta_next = max(t.exp_theta - 8, min(t.exp_theta + 8, e))
+            kind = (32, 32, 8, 16)[rng.integers(0, 4)]
+            kinds.append(kind)
+            if kind == 32:
+                grads = draw_float_grads(rng, ost, strict, lrs)
+                gpu.step(grads, lrs)
+                (oracle_strict_step if strict else oracle_step)(ost, [g.copy() for g in grads], lrs)
+            else:
+                gq, eg = draw_fixed_grads(rng, ost, strict, lrs, kind)
+                gpu.step_qgrad(gq, eg, lrs)
+                if strict:
+                    oracle_strict_step(ost, [oracle_dequantize_gradient(q, e) for q, e in zip(gq, eg)], lrs)
+                else:
+                    oracle_step_qgrad(ost, gq, eg, lrs)
+            assert_same_state(gpu, ost, f"seed {seed} strict {strict} step {step} kinds {kinds}")
+        assert gpu.guards_intact()
+    finally:
+        gpu.close()
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_random_lists_and_step_sequences_plain_handle(seed):
+    run_case(seed, strict=False, steps=7)
+
+
+@pytest.mark.parametrize("seed", range(30))
+def test_random_lists_and_step_sequences_strict_handle(seed):
+    run_case(seed, strict=True, steps=6)

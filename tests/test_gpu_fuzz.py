@@ -10,8 +10,8 @@ import numpy as np
 import pytest
 
 from harness import LibraryRun, assert_same_state, make_oracle_state, storage_dtype
-from oracle import (EXP_AMAX, EXP_FIXED, oracle_dequantize_gradient, oracle_max_threads, oracle_step,
-                    oracle_step_qgrad, oracle_strict_step)
+from oracle import (EXP_AMAX, EXP_FIXED, oracle_adam_step, oracle_dequantize_gradient, oracle_max_threads,
+                    oracle_momentum_step, oracle_step, oracle_step_qgrad, oracle_strict_step)
 
 pytestmark = pytest.mark.gpu
 
@@ -152,3 +152,113 @@ def test_random_lists_and_step_sequences_plain_handle(seed):
 @pytest.mark.parametrize("seed", range(30))
 def test_random_lists_and_step_sequences_strict_handle(seed):
     run_case(seed, strict=True, steps=6)
+
+
+# ------------------------------------------------------------------ momentum and ADAM
+
+def draw_optimizer_list(rng, with_velocity_bits):
+    """A short ragged list for the optimizers (comp_bits != 0), with exponents for the extra
+    state tensors placed around the size of the increments that will come."""
+    n_tensors = int(rng.integers(1, 9))
+    specs, thetas, comps = [], [], []
+    for _ in range(n_tensors):
+        tb = 8 if rng.random() < 0.5 else 16
+        cb = 8 if rng.random() < 0.5 else 16
+        numel = draw_size(rng)
+        k = int(rng.integers(0, cb)) if rng.random() < 0.25 else 0
+        e = int(rng.integers(-24, 4))
+        full = rng.random() < 0.25
+        lim_t = 2 ** (tb - 1) if full else 2 ** (tb - 2)
+        lim_c = 2 ** (cb - 1) if full else 2 ** (cb - 2)
+        spec = dict(numel=numel, theta_bits=tb, comp_bits=cb, overlap_k=k, exp_theta=e)
+        if with_velocity_bits:
+            spec["mom_bits"] = 8 if rng.random() < 0.5 else 16
+        specs.append(spec)
+        thetas.append(rng.integers(-lim_t, lim_t, numel).astype(storage_dtype(tb)))
+        comps.append(rng.integers(-lim_c, lim_c, numel).astype(storage_dtype(cb)))
+    return specs, thetas, comps
+
+
+def special_values(rng, g):
+    if rng.random() < 0.2:
+        idx = rng.choice(g.size, min(g.size, 5), replace=False)
+        g[idx] = SPECIALS[rng.integers(0, len(SPECIALS), idx.size)]
+    return g
+
+
+def run_momentum_case(seed, steps):
+    from test_gpu_momentum import MomentumRun, oracle_state
+    rng = np.random.default_rng([seed, 2])
+    specs, thetas, comps = draw_optimizer_list(rng, True)
+    moms = []
+    for s in specs:
+        vb = s["mom_bits"]
+        c_unit = s["exp_theta"] - (s["comp_bits"] - 1 - s["overlap_k"])
+        # the velocity's unit from 20 binades below the compensation's to 12 above
+        s["exp_mom"] = int(np.clip(c_unit + rng.integers(-20, 13), -64, 64))
+        lim = 2 ** (vb - 1) if rng.random() < 0.25 else 2 ** (vb - 3)
+        moms.append(rng.integers(-lim, lim, s["numel"]).astype(storage_dtype(vb)))
+    mode = EXP_FIXED if rng.random() < 0.15 else EXP_AMAX
+    gpu = MomentumRun(specs, thetas, comps, moms, mode)
+    ost = oracle_state(specs, thetas, comps, moms, mode)
+    try:
+        for step in range(steps):
+            lrs = draw_lrs(rng, len(specs))
+            mus = [float(np.float32(rng.choice([0.0, 0.5, 0.9, 0.99, 1.0])))] * len(specs)
+            grads = []
+            for t, lr in zip(ost.tensors, lrs):
+                # lr * g worth 2^-4 .. 2^(bits + 2) units of the velocity grid the step writes
+                mag = 2.0 ** (t.exp_mom_next + float(rng.uniform(-4, t.mom_bits + 2))) / lr
+                grads.append(special_values(rng, (rng.standard_normal(t.theta.size) * mag).astype(np.float32)))
+            gpu.step(grads, lrs, mus)
+            oracle_momentum_step(ost, [g.copy() for g in grads], lrs, mus)
+            gpu.check(ost, f"momentum seed {seed} step {step}")
+        assert gpu.guards_intact()
+    finally:
+        gpu.close()
+
+
+def run_adam_case(seed, steps):
+    from test_gpu_adam import AdamRun, oracle_state
+    rng = np.random.default_rng([seed, 3])
+    specs, thetas, comps = draw_optimizer_list(rng, False)
+    b1, b2, eps = [(0.9, 0.999, 1e-8), (0.5, 0.9, 1e-3), (0.9, 0.99, 0.0), (0.0, 0.999, 1e-6)][rng.integers(0, 4)]
+    m1s, m2s, sigmas = [], [], []
+    for s in specs:
+        sigma = 2.0 ** float(rng.uniform(-20, 4))
+        sigmas.append(sigma)
+        # grids that hold a first moment of about 4 sigma and a second of about 16 sigma^2,
+        # moved off by a few binades either way
+        s["exp_m"] = int(np.clip(np.ceil(np.log2(4 * sigma / 32767)) + rng.integers(-3, 4), -64, 64))
+        s["exp_v"] = int(np.clip(np.ceil(np.log2(16 * sigma ** 2 / 32767)) + rng.integers(-3, 4), -64, 64))
+        zero = rng.random() < 0.3
+        m1s.append(np.zeros(s["numel"], np.int16) if zero else rng.integers(-9000, 9000, s["numel"]).astype(np.int16))
+        m2s.append(np.zeros(s["numel"], np.int16) if zero else rng.integers(0, 9000, s["numel"]).astype(np.int16))
+    mode = EXP_FIXED if rng.random() < 0.15 else EXP_AMAX
+    gpu = AdamRun(specs, thetas, comps, m1s, m2s, mode)
+    ost = oracle_state(specs, thetas, comps, m1s, m2s, mode)
+    try:
+        for step in range(steps):
+            lrs = []
+            for t in ost.tensors:
+                # a unit step (m / sqrt(v) ~ 1) worth 2^-3 .. 2^(bits of c + 4) compensation units
+                c_unit = t.exp_theta_next - (t.comp_bits - 1 - t.overlap_k)
+                lrs.append(float(np.float32(2.0 ** (c_unit + float(rng.uniform(-3, t.comp_bits + 4))))))
+            grads = [special_values(rng, (rng.standard_normal(t.theta.size) * sg * 2.0 ** float(rng.uniform(-2, 2)))
+                                    .astype(np.float32)) for t, sg in zip(ost.tensors, sigmas)]
+            gpu.step(grads, lrs, b1, b2, eps)
+            oracle_adam_step(ost, [g.copy() for g in grads], lrs, b1, b2, eps)
+            gpu.check(ost, f"adam seed {seed} step {step}")
+        assert gpu.guards_intact()
+    finally:
+        gpu.close()
+
+
+@pytest.mark.parametrize("seed", range(30))
+def test_random_lists_and_gradients_momentum(seed):
+    run_momentum_case(seed, steps=6)
+
+
+@pytest.mark.parametrize("seed", range(30))
+def test_random_lists_and_gradients_adam(seed):
+    run_adam_case(seed, steps=6)

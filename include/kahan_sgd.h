@@ -257,7 +257,11 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
  * ignored; exponents outside [-64, 64] or outside the window above, or a first-step change
  * of c's exponent of more than 16 (the most the rule above ever asks for: 8 of its own fit
  * plus 8 of theta's move; the 64-bit sums of a step are only guaranteed up to there), give
- * KSGD_ERR_EXP_RANGE.
+ * KSGD_ERR_EXP_RANGE.  Both pairs are checked against their own window: (exp_theta,
+ * exp_comp) and (exp_theta_next, exp_comp_next); a state read from a running handle with
+ * kahan_sgd_amax and kahan_sgd_strict_exponents satisfies both, so it can be resumed.
+ * kahan_sgd_strict_workspace_bytes: the size for such a list, 0 if the list or a stored
+ * exponent pair is invalid (it does not see the first step's exponents and does not check them).
  * The handle then works with kahan_sgd_step, kahan_sgd_step_qgrad, kahan_sgd_amax and
  * kahan_sgd_destroy; kahan_sgd_step_host, kahan_sgd_set_exponents and
  * kahan_sgd_strict_exponents on the wrong kind of handle return KSGD_ERR_MODE.

@@ -306,14 +306,21 @@ namespace {
 
 bool strict_window_ok(int e, int ec) { return e - ec >= -kStrictAbove && e - ec <= kStrictBelow; }
 
-int validate_strict(const ksgd_tensor_desc* d, const int32_t* ec, const int32_t* ec_next, int32_t n) {
+// first_step: also check the exponents the first step writes (init).  The workspace size
+// does not depend on them, and c's stored exponent need not lie in the window of theta's
+// *next* exponent (a state taken from a running handle has it in the window of the stored
+// one only), so the size query checks the stored pair alone.
+int validate_strict(const ksgd_tensor_desc* d, const int32_t* ec, const int32_t* ec_next, int32_t n,
+                    bool first_step) {
   if (!ec) return KSGD_ERR_NULL;
   for (int32_t i = 0; i < n; ++i) {
     if (d[i].comp_bits == 0) return KSGD_ERR_BITS;          // the accumulator is the point of this mode
+    if (ec[i] < kExpMin || ec[i] > kExpMax) return KSGD_ERR_EXP_RANGE;
+    if (!strict_window_ok(d[i].exp_theta, ec[i])) return KSGD_ERR_EXP_RANGE;
+    if (!first_step) continue;
     const int32_t nx = ec_next ? ec_next[i] : ec[i];
-    if (ec[i] < kExpMin || ec[i] > kExpMax || nx < kExpMin || nx > kExpMax) return KSGD_ERR_EXP_RANGE;
-    if (!strict_window_ok(d[i].exp_theta, ec[i]) || !strict_window_ok(d[i].exp_theta_next, nx))
-      return KSGD_ERR_EXP_RANGE;
+    if (nx < kExpMin || nx > kExpMax) return KSGD_ERR_EXP_RANGE;
+    if (!strict_window_ok(d[i].exp_theta_next, nx)) return KSGD_ERR_EXP_RANGE;
     // the device never moves c's exponent by more than 2 * kMaxDelta in one step (its own
     // fit plus theta's move); a larger first-step change would shift past 64 bits
     if (std::abs(nx - ec[i]) > 2 * kMaxDelta) return KSGD_ERR_EXP_RANGE;
@@ -329,7 +336,7 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   const int v = validate(descs, n_tensors);
   if (v != KSGD_OK) return v;
   if (strict) {
-    const int vs = validate_strict(descs, exp_comp, exp_comp_next, n_tensors);
+    const int vs = validate_strict(descs, exp_comp, exp_comp_next, n_tensors, true);
     if (vs != KSGD_OK) return vs;
   }
   if (mode != KSGD_EXP_FIXED && mode != KSGD_EXP_AMAX) return KSGD_ERR_MODE;
@@ -429,7 +436,7 @@ int kahan_sgd_init(ksgd_handle** out, const ksgd_tensor_desc* descs, int32_t n_t
 size_t kahan_sgd_strict_workspace_bytes(const ksgd_tensor_desc* descs, const int32_t* exp_comp,
                                         int32_t n_tensors) {
   if (validate(descs, n_tensors) != KSGD_OK) return 0;
-  if (validate_strict(descs, exp_comp, nullptr, n_tensors) != KSGD_OK) return 0;
+  if (validate_strict(descs, exp_comp, nullptr, n_tensors, false) != KSGD_OK) return 0;
   return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), true).total;
 }
 

@@ -199,6 +199,14 @@ def test_strict_and_fixed_point_gradient_entry_points_reject_bad_arguments_witho
         with pytest.raises(B.KahanSgdError) as ei:
             B.kahan_sgd_strict_init(ds, ec, nxt, B.KSGD_EXP_AMAX, 0x100000, 1 << 20)
         assert ei.value.code == code
+    # A state taken from a running handle: c's stored exponent lies in the window of theta's
+    # stored exponent only (theta moves 8 up, c's next exponent with it).  The size query
+    # must accept it: the exponents of the first step are init's to check.
+    resumed = B.make_descs([good(exp_theta=0, exp_theta_next=8)])
+    assert B.kahan_sgd_strict_workspace_bytes(resumed, [-36]) > 0
+    with pytest.raises(B.KahanSgdError) as ei:       # ... and init refuses it without its next exponent
+        B.kahan_sgd_strict_init(resumed, [-36], None, B.KSGD_EXP_AMAX, 0x100000, 1 << 20)
+    assert ei.value.code == B.KSGD_ERR_EXP_RANGE
     assert B.lib.kahan_sgd_strict_init(None, descs, None, None, 1, 1, None, 0, None) == B.KSGD_ERR_NULL
     assert B.lib.kahan_sgd_strict_exponents(None, None, None) == B.KSGD_ERR_NULL
     assert B.lib.kahan_sgd_step_qgrad(None, None, 8, None, None) == B.KSGD_ERR_NULL

@@ -10,8 +10,9 @@ import numpy as np
 import pytest
 
 from harness import LibraryRun, assert_same_state, make_oracle_state, storage_dtype
-from oracle import (EXP_AMAX, EXP_FIXED, oracle_adam_step, oracle_dequantize_gradient, oracle_max_threads,
-                    oracle_momentum_step, oracle_step, oracle_step_qgrad, oracle_strict_step)
+from oracle import (EXP_AMAX, EXP_FIXED, oracle_adam_step, oracle_dequantize, oracle_dequantize_gradient,
+                    oracle_fit_exponent, oracle_max_threads, oracle_momentum_step, oracle_quantize, oracle_step,
+                    oracle_step_qgrad, oracle_strict_step)
 
 pytestmark = pytest.mark.gpu
 
@@ -125,6 +126,19 @@ def run_case(seed, strict, steps):
                 gpu.set_exponents(want)
                 for t, e in zip(ost.tensors, want):       # the device limits the change to 8 binades
                     t.exp_theta_next = max(t.exp_theta - 8, min(t.exp_theta + 8, e))
+            if step > 0 and rng.random() < 0.15:
+                # checkpoint and resume: a fresh handle (and a fresh oracle state) from the
+                # mantissas and exponents as they stand, the next exponents as first-step targets
+                kinds.append("resume")
+                gpu.close()
+                for sp, t in zip(specs, ost.tensors):
+                    sp["exp_theta"], sp["exp_theta_next"] = t.exp_theta, t.exp_theta_next
+                    if strict:
+                        sp["exp_comp"], sp["exp_comp_next"] = t.exp_comp, t.exp_comp_next
+                thetas = [t.theta.copy() for t in ost.tensors]
+                comps = [None if t.comp is None else t.comp.copy() for t in ost.tensors]
+                gpu = LibraryRun(specs, thetas, comps, mode, strict=strict)
+                ost = make_oracle_state(specs, thetas, comps, mode, oracle_max_threads())
             kind = (32, 32, 8, 16)[rng.integers(0, 4)]
             kinds.append(kind)
             if kind == 32:
@@ -262,3 +276,54 @@ def test_random_lists_and_gradients_momentum(seed):
 @pytest.mark.parametrize("seed", range(30))
 def test_random_lists_and_gradients_adam(seed):
     run_adam_case(seed, steps=6)
+
+
+# ------------------------------------------------------------------ fp32 <-> fixed point
+
+def run_convert_case(seed):
+    """Import and export of a random array at a random element offset (aligned and unaligned
+    paths), magnitudes over the whole exponent range, specials sprinkled in, against the oracle;
+    guard values before and after every output."""
+    import torch
+    from paper_1810_05486_b200 import binding as B
+    rng = np.random.default_rng([seed, 4])
+    st = torch.cuda.current_stream().cuda_stream
+    tb = 8 if rng.random() < 0.5 else 16
+    cb = int(rng.choice([0, 8, 16]))
+    k = int(rng.integers(0, cb)) if (cb and rng.random() < 0.3) else 0
+    n = draw_size(rng)
+    off = int(rng.choice([0, 0, 1, 2, 3, 4, 8]))
+    x = (rng.standard_t(3, n + off) * 2.0 ** float(rng.uniform(-70, 40))).astype(np.float32)
+    if rng.random() < 0.4:
+        idx = rng.choice(n + off, min(n + off, 6), replace=False)
+        x[idx] = SPECIALS[rng.integers(0, len(SPECIALS), idx.size)]
+    if rng.random() < 0.05:
+        x[:] = 0.0
+    src = np.ascontiguousarray(x[off:])
+    dx = torch.from_numpy(x).cuda()
+    tdt, cdt = (torch.int8 if tb == 8 else torch.int16), (torch.int8 if cb <= 8 else torch.int16)
+    th = torch.full((n + off + 32,), 0x5A, dtype=tdt, device="cuda")
+    c = torch.full((n + off + 32,), 0x5A, dtype=cdt, device="cuda")
+    scratch = torch.zeros(4, dtype=torch.int32, device="cuda")
+    e_req = B.KSGD_EXP_AUTO if rng.random() < 0.6 else int(rng.integers(-64, 65))
+    cptr = (c.data_ptr() + off * (max(cb, 8) // 8)) if cb else None
+    e = B.kahan_sgd_import(dx.data_ptr() + 4 * off, th.data_ptr() + off * (tb // 8), cptr, n, tb, cb, k, e_req,
+                           scratch.data_ptr(), st)
+    assert e == (oracle_fit_exponent(src, tb) if e_req == B.KSGD_EXP_AUTO else e_req), f"convert seed {seed}"
+    wt, wc = oracle_quantize(src, tb, cb, k, e)
+    assert np.array_equal(th[off:off + n].cpu().numpy(), wt), f"convert seed {seed}: theta"
+    assert bool((th[:off] == 0x5A).all()) and bool((th[off + n:] == 0x5A).all())
+    if cb:
+        assert np.array_equal(c[off:off + n].cpu().numpy(), wc), f"convert seed {seed}: comp"
+        assert bool((c[:off] == 0x5A).all()) and bool((c[off + n:] == 0x5A).all())
+    out = torch.full((n + off + 8,), 7.0, dtype=torch.float32, device="cuda")
+    B.kahan_sgd_export(th.data_ptr() + off * (tb // 8), cptr, out.data_ptr() + 4 * off, n, tb, cb, k, e, st)
+    want = oracle_dequantize(wt, wc, tb, cb, k, e)
+    assert np.array_equal(out[off:off + n].cpu().numpy().view(np.uint32), want.view(np.uint32)), \
+        f"convert seed {seed}: export"
+    assert bool((out[:off] == 7.0).all()) and bool((out[off + n:] == 7.0).all())
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_random_arrays_through_import_and_export(seed):
+    run_convert_case(seed)

@@ -139,9 +139,26 @@ def run_case(seed, strict, steps):
                 comps = [None if t.comp is None else t.comp.copy() for t in ost.tensors]
                 gpu = LibraryRun(specs, thetas, comps, mode, strict=strict)
                 ost = make_oracle_state(specs, thetas, comps, mode, oracle_max_threads())
-            kind = (32, 32, 8, 16)[rng.integers(0, 4)]
+            kind = (32, 32, 8, 16, "host")[rng.integers(0, 4 if strict else 5)]
             kinds.append(kind)
-            if kind == 32:
+            if kind == "host":
+                # the host-buffer entry point: state and gradients travel from host arrays (the
+                # oracle's copies, equal to the device's by the last comparison) and back
+                import torch
+                grads = draw_float_grads(rng, ost, strict, lrs)
+                th_h = [t.theta.copy() for t in ost.tensors]
+                c_h = [None if t.comp is None else t.comp.copy() for t in ost.tensors]
+                need = sum((sp["numel"] + 3) // 4 * 16 for sp in specs)
+                staging = torch.empty(need, dtype=torch.uint8, device="cuda")
+                gpu.B.kahan_sgd_step_host(gpu.handle, [t.ctypes.data for t in th_h],
+                                          [None if c is None else c.ctypes.data for c in c_h],
+                                          [g.ctypes.data for g in grads], lrs, staging.data_ptr(), need)
+                oracle_step(ost, [g.copy() for g in grads], lrs)
+                for i, t in enumerate(ost.tensors):
+                    assert np.array_equal(th_h[i], t.theta), f"seed {seed} step {step}: host theta of tensor {i}"
+                    assert t.comp is None or np.array_equal(c_h[i], t.comp), \
+                        f"seed {seed} step {step}: host comp of tensor {i}"
+            elif kind == 32:
                 grads = draw_float_grads(rng, ost, strict, lrs)
                 gpu.step(grads, lrs)
                 (oracle_strict_step if strict else oracle_step)(ost, [g.copy() for g in grads], lrs)
@@ -174,11 +191,13 @@ def draw_optimizer_list(rng, with_velocity_bits):
     """A short ragged list for the optimizers (comp_bits != 0), with exponents for the extra
     state tensors placed around the size of the increments that will come."""
     n_tensors = int(rng.integers(1, 9))
+    if rng.random() < 0.1:
+        n_tensors = int(rng.integers(257, 280))      # beyond the inline argument block
     specs, thetas, comps = [], [], []
     for _ in range(n_tensors):
         tb = 8 if rng.random() < 0.5 else 16
         cb = 8 if rng.random() < 0.5 else 16
-        numel = draw_size(rng)
+        numel = draw_size(rng) if n_tensors < 100 else int(rng.integers(1, 2000))
         k = int(rng.integers(0, cb)) if rng.random() < 0.25 else 0
         e = int(rng.integers(-24, 4))
         full = rng.random() < 0.25
@@ -217,6 +236,15 @@ def run_momentum_case(seed, steps):
     ost = oracle_state(specs, thetas, comps, moms, mode)
     try:
         for step in range(steps):
+            if step > 0 and rng.random() < 0.15:      # checkpoint and resume from the state as it stands
+                gpu.close()
+                for sp, t in zip(specs, ost.tensors):
+                    sp["exp_theta"], sp["exp_theta_next"] = t.exp_theta, t.exp_theta_next
+                    sp["exp_mom"], sp["exp_mom_next"] = t.exp_mom, t.exp_mom_next
+                thetas, comps = [t.theta.copy() for t in ost.tensors], [t.comp.copy() for t in ost.tensors]
+                moms = [t.mom.copy() for t in ost.tensors]
+                gpu = MomentumRun(specs, thetas, comps, moms, mode)
+                ost = oracle_state(specs, thetas, comps, moms, mode)
             lrs = draw_lrs(rng, len(specs))
             mus = [float(np.float32(rng.choice([0.0, 0.5, 0.9, 0.99, 1.0])))] * len(specs)
             grads = []
@@ -253,6 +281,16 @@ def run_adam_case(seed, steps):
     ost = oracle_state(specs, thetas, comps, m1s, m2s, mode)
     try:
         for step in range(steps):
+            if step > 0 and rng.random() < 0.15:      # checkpoint and resume from the state as it stands
+                gpu.close()
+                for sp, t in zip(specs, ost.tensors):
+                    sp["exp_theta"], sp["exp_theta_next"] = t.exp_theta, t.exp_theta_next
+                    sp["exp_m"], sp["exp_m_next"] = t.exp_mom, t.exp_mom_next
+                    sp["exp_v"], sp["exp_v_next"] = t.exp_mom2, t.exp_mom2_next
+                thetas, comps = [t.theta.copy() for t in ost.tensors], [t.comp.copy() for t in ost.tensors]
+                m1s, m2s = [t.mom.copy() for t in ost.tensors], [t.mom2.copy() for t in ost.tensors]
+                gpu = AdamRun(specs, thetas, comps, m1s, m2s, mode)
+                ost = oracle_state(specs, thetas, comps, m1s, m2s, mode)
             lrs = []
             for t in ost.tensors:
                 # a unit step (m / sqrt(v) ~ 1) worth 2^-3 .. 2^(bits of c + 4) compensation units

@@ -46,6 +46,17 @@
  * accumulation invariant and both directions of the velocity-to-compensation grid shift.
  * Accuracy tables of Section 4: parity unpinned
  * (datasets and trained weights are not available).
+ * Three rules of the optimizer variants are readings the paper neither states nor
+ * contradicts (Section 4 names momentum and ADAM and prints no arithmetic for them;
+ * Section 5 only cites max-scan schemes), and nothing outside this file fixes them, so
+ * for each of them parity is unpinned against the paper; their tests state the
+ * reading's own property:
+ *   - ksgd_oracle_next_exponent_velocity: the dead band (the velocity and the ADAM
+ *     moments keep their exponent while the largest mantissa lies in (QMAX/4, QMAX]);
+ *   - ksgd_oracle_adam_element: a stored second moment <= 0 enters the denominator
+ *     as one unit of its grid;
+ *   - ksgd_oracle_next_exponent_acc: an empty scan makes the strict accumulator's
+ *     grid 8 binades finer.
  *
  * Build: gcc -O2 -ffp-contract=off -fopenmp -shared -fPIC (see oracle/build.py).
  */

@@ -80,9 +80,10 @@ enum {
 
 /*
  * Bytes of device workspace kahan_sgd_init needs for this tensor list (per-tensor
- * exponents, max-scan scratch, counters, per-step arguments and the table that cuts
- * the ragged list into equal chunks).  Host-only computation.  Returns 0 if the list
- * is invalid (kahan_sgd_init reports why).
+ * exponents, max-scan scratch, counters, per-step arguments and the tables that cut
+ * the ragged list into tiles: about 8 bytes per 8192 elements, 170 bytes per tensor and
+ * 8 to 16 KB that do not depend on the list).  Host-only computation.  Returns 0 if the
+ * list is invalid (kahan_sgd_init reports why).  A tensor may have up to 2^40 elements.
  */
 size_t kahan_sgd_workspace_bytes(const ksgd_tensor_desc* descs, int32_t n_tensors);
 

@@ -90,13 +90,6 @@ Layout make_ring_layout(int32_t n, long long n_chunks, size_t state_bytes, size_
   return L;
 }
 
-// Tile table of a list cut into tiles of kChunk elements, into `chunks`; returns the count.
-long long plain_tile_count(const ksgd_tensor_desc* d, int32_t n) {
-  long long chunks = 0;
-  for (int32_t i = 0; i < n; ++i) chunks += (d[i].numel + kChunk - 1) / kChunk;
-  return chunks;
-}
-
 // What every init needs from the device, and the upload of the finished image.
 struct DeviceFacts { int sms = 0, l2_bytes = 0; };
 cudaError_t query_device(DeviceFacts& f) {
@@ -107,49 +100,102 @@ cudaError_t query_device(DeviceFacts& f) {
   return e;
 }
 
-// Tile size of a tensor, given the list's tile size for 8-bit theta.
-inline long long tile_elems(const ksgd_tensor_desc& t, int chunk8) { return t.theta_bits == 8 ? chunk8 : kChunk; }
+// ---- tile tables ----------------------------------------------------------------------
+// A list is cut into tiles of 2^lg elements of one tensor, lg by the tensor's format (the
+// rules below).  Block b of a step takes tiles b, b + blocks, ...: when the tile count is not a
+// multiple of the block count, the last round over the blocks has work for some of them only,
+// and the step ends with a tile's whole latency (load, compute, drain) during which the memory
+// system idles: on ResNet-50 shapes 19 of 148 blocks have a 22nd tile.  The builder therefore
+// cuts the tiles of that last round into 2^k equal pieces each, k the largest for which the
+// pieces still number at most one per block (and a piece has at least 512 elements), so
+// that the last round is short and spread over the blocks.  A list with fewer tiles than
+// blocks is one such round, which also puts more of the SMs to work on short lists.  The size
+// query does not know the device, so a table reserves room for kTailReserve more entries than
+// it has whole tiles.
+constexpr long long kTailReserve = 1024;   // more than any device has SMs; the pieces are capped to it anyway
 
-// Tile size for tensors with 8-bit theta: the large one if the list then still has
-// kBigTileMinTiles tiles (about seven per block), so that short lists keep every block busy.
-int pick_chunk8(const ksgd_tensor_desc* d, int32_t n) {
-  long long tiles = 0;
-  for (int32_t i = 0; i < n; ++i) {
-    const long long c = tile_elems(d[i], 2 * kChunk);
-    tiles += (d[i].numel + c - 1) / c;
-  }
-  return tiles >= kBigTileMinTiles ? 2 * kChunk : kChunk;
-}
-
-long long tile_count(const ksgd_tensor_desc* d, int32_t n, int chunk8) {
-  long long chunks = 0;
-  for (int32_t i = 0; i < n; ++i) chunks += (d[i].numel + tile_elems(d[i], chunk8) - 1) / tile_elems(d[i], chunk8);
-  return chunks;
-}
+inline int lg_plain(const ksgd_tensor_desc& t, int chunk8) { return t.theta_bits == 8 && chunk8 != kChunk ? 14 : 13; }
 
 // Steps on 8-bit gradients move so few bytes per parameter (5 for an 8/8 tensor, 9 for 16/16)
 // that what a consumer does per tile, not per element, is a fifth or more of its instructions
 // with the tiles above.  Lists long enough get a second tile table for those steps, with
 // tiles twice as large as the largest of the first table: 4 * kChunk elements for 8-bit theta
 // (12 of the ring's 28 pages with an 8-bit c and an 8-bit gradient; 2 * kChunk with a 16-bit
-// c, which would take 16), 2 * kChunk for 16-bit theta (6 to 10 pages).  The kernel applies
-// the same rule (PlainPolicy::tile_shift).
-inline long long tile_elems_qgrad(const ksgd_tensor_desc& t) {
-  return t.theta_bits == 8 && t.comp_bits <= 8 ? 4 * kChunk : 2 * kChunk;
+// c, which would take 16), 2 * kChunk for 16-bit theta (6 to 10 pages).
+inline int lg_qgrad(const ksgd_tensor_desc& t) { return t.theta_bits == 8 && t.comp_bits <= 8 ? 15 : 14; }
+
+template <class LgFn>
+long long whole_tiles(const ksgd_tensor_desc* d, int32_t n, LgFn lg_of) {
+  long long tiles = 0;
+  for (int32_t i = 0; i < n; ++i) tiles += (d[i].numel + (1LL << lg_of(d[i])) - 1) >> lg_of(d[i]);
+  return tiles;
 }
 
-// Entries of that table, or 0 for none (short lists keep the small tiles of the first table,
-// with which every block has work).
-long long tile_count_qgrad(const ksgd_tensor_desc* d, int32_t n) {
-  long long tiles = 0;
-  for (int32_t i = 0; i < n; ++i) tiles += (d[i].numel + tile_elems_qgrad(d[i]) - 1) / tile_elems_qgrad(d[i]);
+// Writes the table to `out` (nullptr: counts only) and returns the number of entries; sms > 0
+// cuts the last round into pieces as described above, sms == 0 leaves whole tiles.
+// first_tile (optional) receives the first entry of every tensor, plus the total.
+template <class LgFn>
+long long build_tile_table(const ksgd_tensor_desc* d, int32_t n, LgFn lg_of, int sms, ChunkRef* out,
+                           std::vector<long long>* first_tile) {
+  const long long tiles = whole_tiles(d, n, lg_of);
+  const long long r = sms > 0 ? tiles % sms : 0;
+  int k = 0;
+  if (r > 0) {
+    const long long room = (long long)sms < kTailReserve ? (long long)sms : kTailReserve;
+    while ((r << (k + 1)) <= room) ++k;
+  }
+  const long long cut_from = tiles - r;      // whole tiles from this one on are cut
+  long long c = 0, whole = 0;
+  if (first_tile) first_tile->clear();
+  for (int32_t i = 0; i < n; ++i) {
+    const int lg = lg_of(d[i]);
+    const long long nc = (d[i].numel + (1LL << lg) - 1) >> lg;
+    if (first_tile) first_tile->push_back(c);
+    for (long long j = 0; j < nc; ++j, ++whole) {
+      int kk = 0;
+      if (whole >= cut_from) {
+        kk = k < lg - kMinTileLog2 ? k : lg - kMinTileLog2;
+        while (kk > 0 && ((j + 1) << kk) > (1LL << kTileIndexBits)) --kk;    // the index field holds 27 bits
+      }
+      for (long long q = 0; q < (1LL << kk); ++q) {
+        const long long idx = (j << kk) + q;
+        if ((idx << (lg - kk)) >= d[i].numel) break;      // the tensor's short last tile: nothing left
+        if (out) out[c] = make_chunk_ref(i, idx, lg - kk);
+        ++c;
+      }
+    }
+  }
+  if (first_tile) first_tile->push_back(c);
+  return c;
+}
+
+// Tile size for tensors with 8-bit theta in the first table: the large one (2 * kChunk) if the
+// list then still has kBigTileMinTiles tiles (about seven per block), so that short lists
+// keep every block busy; with one 16-element vector per thread and tile, what a consumer does
+// per tile (wait, descriptor, scans, arrive) is a third of its instructions.
+int pick_chunk8(const ksgd_tensor_desc* d, int32_t n) {
+  const long long tiles = whole_tiles(d, n, [](const ksgd_tensor_desc& t) { return lg_plain(t, 2 * kChunk); });
+  return tiles >= kBigTileMinTiles ? 2 * kChunk : kChunk;
+}
+
+// Whole tiles of the table for steps on 8-bit gradients, or 0 for none (short lists keep the
+// smaller tiles of the first table, with which every block has work).
+long long whole_tiles_qgrad(const ksgd_tensor_desc* d, int32_t n) {
+  const long long tiles = whole_tiles(d, n, lg_qgrad);
   return tiles >= kBigTileMinTiles ? tiles : 0;
 }
 
-// The tile table is the layout's last region: the table for 8-bit gradients, if any, follows
-// the first one in it.
-Layout make_layout(const ksgd_tensor_desc* d, int32_t n, int chunk8, bool with_qgrad_table) {
-  return make_ring_layout(n, tile_count(d, n, chunk8) + (with_qgrad_table ? tile_count_qgrad(d, n) : 0),
+// Room for the two tables of the plain optimizer (the second follows the first at
+// qgrad_table_offset); reserve_tail: room for the pieces of the last round.
+long long plain_table_capacity(const ksgd_tensor_desc* d, int32_t n, int chunk8, bool reserve_tail) {
+  return whole_tiles(d, n, [chunk8](const ksgd_tensor_desc& t) { return lg_plain(t, chunk8); }) +
+         (reserve_tail ? kTailReserve : 0);
+}
+
+// The tile table is the layout's last region.
+Layout make_layout(const ksgd_tensor_desc* d, int32_t n, int chunk8, bool with_qgrad_table, bool reserve_tail) {
+  const long long q = with_qgrad_table ? whole_tiles_qgrad(d, n) : 0;
+  return make_ring_layout(n, plain_table_capacity(d, n, chunk8, reserve_tail) + (q ? q + kTailReserve : 0),
                           sizeof(TensorState), sizeof(TensorInfo), 3);
 }
 
@@ -171,15 +217,16 @@ void bind_workspace(Workspace& w, char* b, const Layout& L) {
 // first step reads (slab 2) the exponents of the stored mantissas and, as overrides, the
 // exponents the first step must write; zeroed scans and counters; tensor table; tile
 // table (and, if asked for and the list is long enough for one, the table for steps on 8-bit
-// gradients behind it).
+// gradients, at entry qgrad_offset of the table region).  sms: blocks of a step, for the
+// pieces of the tables' last round (0: whole tiles only).
 // first_tile (optional) receives the first tile of every tensor, plus the total.
-void write_initial_image(unsigned char* img, const Layout& L, const ksgd_tensor_desc* descs, int32_t n,
-                         const int32_t* exp_comp, const int32_t* exp_comp_next, int chunk8, bool with_qgrad_table,
-                         std::vector<long long>* first_tile) {
+struct TableCounts { long long plain = 0, qgrad = 0, qgrad_offset = 0; };
+TableCounts write_initial_image(unsigned char* img, const Layout& L, const ksgd_tensor_desc* descs, int32_t n,
+                                const int32_t* exp_comp, const int32_t* exp_comp_next, int chunk8,
+                                bool with_qgrad_table, int sms, std::vector<long long>* first_tile) {
   TensorState* last = reinterpret_cast<TensorState*>(img + L.state) + 2 * (size_t)L.slab;
   TensorInfo* info = reinterpret_cast<TensorInfo*>(img + L.info);
   ChunkRef* chunks = reinterpret_cast<ChunkRef*>(img + L.chunks);
-  long long c = 0;
   for (int32_t i = 0; i < n; ++i) {
     const ksgd_tensor_desc& t = descs[i];
     last[i].exp_theta = t.exp_theta;
@@ -195,17 +242,15 @@ void write_initial_image(unsigned char* img, const Layout& L, const ksgd_tensor_
     info[i].comp_bits = t.comp_bits;
     info[i].s = t.comp_bits ? t.comp_bits - 1 - t.overlap_k : 0;
     info[i].pad = 0;
-    const long long nc = (t.numel + tile_elems(t, chunk8) - 1) / tile_elems(t, chunk8);
-    if (first_tile) first_tile->push_back(c);
-    for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
   }
-  if (first_tile) first_tile->push_back(c);
-  if (with_qgrad_table && tile_count_qgrad(descs, n)) {
-    for (int32_t i = 0; i < n; ++i) {
-      const long long nc = (descs[i].numel + tile_elems_qgrad(descs[i]) - 1) / tile_elems_qgrad(descs[i]);
-      for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
-    }
+  TableCounts tc;
+  tc.plain = build_tile_table(descs, n, [chunk8](const ksgd_tensor_desc& t) { return lg_plain(t, chunk8); }, sms,
+                              chunks, first_tile);
+  if (with_qgrad_table && whole_tiles_qgrad(descs, n)) {
+    tc.qgrad_offset = plain_table_capacity(descs, n, chunk8, sms > 0);
+    tc.qgrad = build_tile_table(descs, n, lg_qgrad, sms, chunks + tc.qgrad_offset, nullptr);
   }
+  return tc;
 }
 
 // The caller's view of a copy of the stats region: scans and exponent of the last finished
@@ -261,8 +306,9 @@ int validate(const ksgd_tensor_desc* d, int32_t n) {
     if (std::abs(t.exp_theta_next - t.exp_theta) > kMaxDelta) return KSGD_ERR_EXP_RANGE;
     if (reinterpret_cast<uintptr_t>(t.theta) % 16 || reinterpret_cast<uintptr_t>(t.comp) % 16)
       return KSGD_ERR_ALIGN;
+    if (t.numel > (1LL << (kTileIndexBits + kChunkLog2))) return KSGD_ERR_NUMEL;   // the tile table's index field
     chunks += (t.numel + kChunk - 1) / kChunk;
-    if (chunks > 0x7fffffffLL) return KSGD_ERR_NUMEL;
+    if (chunks > 0x7fffffffLL - 2 * kTailReserve) return KSGD_ERR_NUMEL;
   }
   return KSGD_OK;
 }
@@ -280,8 +326,9 @@ struct ksgd_handle {
   int sms;
   std::vector<unsigned char> stats_host;   // staging for kahan_sgd_amax
   std::vector<long long> first_tile;       // [n+1] first tile of every tensor
-  long long tiles_qgrad = 0;               // entries of the tile table for steps on 8-bit gradients (it follows
-                                           // the first one), 0: those steps use the first table too
+  long long tiles_qgrad = 0;               // entries of the tile table for steps on 8-bit gradients, 0: those
+                                           // steps use the first table too
+  long long qgrad_offset = 0;              // where that table starts in the table region (in entries)
   bool strict = false;                     // strict Algorithm 1: compensation with its own exponent
   // kahan_sgd_step_host: copy streams and events, created on first use
   cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
@@ -292,12 +339,12 @@ extern "C" {
 
 size_t kahan_sgd_workspace_bytes(const ksgd_tensor_desc* descs, int32_t n_tensors) {
   if (validate(descs, n_tensors) != KSGD_OK) return 0;
-  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), true).total;
+  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), true, true).total;
 }
 
 size_t kahan_sgd_workspace_error_offset(const ksgd_tensor_desc* descs, int32_t n_tensors) {
   if (validate(descs, n_tensors) != KSGD_OK) return (size_t)-1;
-  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), true).error;
+  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), true, true).error;
 }
 
 }  // extern "C"
@@ -343,9 +390,13 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   if (!workspace) return KSGD_ERR_NULL;
   if (reinterpret_cast<uintptr_t>(workspace) % 256) return KSGD_ERR_ALIGN;
   const int chunk8 = pick_chunk8(descs, n_tensors);
-  const Layout L = make_layout(descs, n_tensors, chunk8, true);
-  const long long tiles = tile_count(descs, n_tensors, chunk8);
+  const Layout L = make_layout(descs, n_tensors, chunk8, true, true);
   if (workspace_bytes < L.total) return KSGD_ERR_WORKSPACE;
+  DeviceFacts dev_facts;      // the tile tables depend on the number of blocks a step has
+  {
+    const cudaError_t eq = query_device(dev_facts);
+    if (eq != cudaSuccess) return cuda_fail(eq, "device query");
+  }
 
   ksgd_handle* h = new (std::nothrow) ksgd_handle();
   if (!h) return KSGD_ERR_NULL;
@@ -358,9 +409,11 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   h->strict = strict;
 
   std::vector<unsigned char> img(L.total, 0);
-  write_initial_image(img.data(), L, descs, n_tensors, strict ? exp_comp : nullptr, exp_comp_next, chunk8, true,
-                      &h->first_tile);
-  h->tiles_qgrad = tile_count_qgrad(descs, n_tensors);
+  const TableCounts tc = write_initial_image(img.data(), L, descs, n_tensors, strict ? exp_comp : nullptr,
+                                             exp_comp_next, chunk8, true, dev_facts.sms, &h->first_tile);
+  const long long tiles = tc.plain;
+  h->tiles_qgrad = tc.qgrad;
+  h->qgrad_offset = tc.qgrad_offset;
   char* b = h->ws_base;
   bind_workspace(h->params.ws, b, L);
   h->params.n_tensors = n_tensors;
@@ -373,15 +426,10 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   h->params.tensor_count = n_tensors;
   h->params.advance = 1;
   h->params.exp_grad_dev = nullptr;
-  h->params.qgrad_tiles = 0;
 
   // Persistent grid: one block per SM (fewer if the list has fewer tiles).
-  int dev = 0, sms = 0, l2_bytes = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, dev);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(ksgd_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  const int sms = dev_facts.sms, l2_bytes = dev_facts.l2_bytes;
+  cudaError_t e = cudaFuncSetAttribute(ksgd_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)kSharedBytes);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(ksgd_step_qgrad_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -410,7 +458,6 @@ int init_common(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t*
   for (int32_t i = 0; i < n_tensors; ++i)
     state_bytes += (double)descs[i].numel * ((descs[i].theta_bits + descs[i].comp_bits) / 8);
   h->params.state_in_l2 = state_bytes <= 0.8 * (double)l2_bytes ? 1 : 0;
-  h->params.chunk8 = chunk8;
 
   e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
@@ -437,7 +484,7 @@ size_t kahan_sgd_strict_workspace_bytes(const ksgd_tensor_desc* descs, const int
                                         int32_t n_tensors) {
   if (validate(descs, n_tensors) != KSGD_OK) return 0;
   if (validate_strict(descs, exp_comp, nullptr, n_tensors, false) != KSGD_OK) return 0;
-  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), true).total;
+  return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), true, true).total;
 }
 
 int kahan_sgd_strict_init(ksgd_handle** out, const ksgd_tensor_desc* descs, const int32_t* exp_comp,
@@ -573,9 +620,8 @@ static int step_qgrad_common(ksgd_handle* h, const void* const* grads, int32_t g
   p.exp_grad_dev = exp_grad_dev;
   unsigned grid = (unsigned)h->grid;
   if (grad_bits == 8 && h->tiles_qgrad) {       // the table of larger tiles, behind the first one
-    p.ws.chunks += p.n_chunks;
+    p.ws.chunks += h->qgrad_offset;
     p.n_chunks = p.tile_count = (int)h->tiles_qgrad;
-    p.qgrad_tiles = 1;
     grid = (unsigned)(h->tiles_qgrad < (long long)h->sms ? h->tiles_qgrad : (long long)h->sms);
   }
   auto kernel = h->strict ? (grad_bits == 8 ? ksgd_strict_step_qgrad_kernel<8> : ksgd_strict_step_qgrad_kernel<16>)
@@ -806,7 +852,7 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   if (mode != KSGD_EXP_FIXED && mode != KSGD_EXP_AMAX) return KSGD_ERR_MODE;
   if (!grads || !lrs) return KSGD_ERR_NULL;
   if (n_tensors > KSGD_STATIC_MAX_TENSORS) return KSGD_ERR_WORKSPACE;
-  const Layout L = make_layout(descs, n_tensors, kChunk, false);
+  const Layout L = make_layout(descs, n_tensors, kChunk, false, false);
   if (L.total > (size_t)KSGD_STATIC_SCRATCH_BYTES) return KSGD_ERR_WORKSPACE;
   for (int32_t i = 0; i < n_tensors; ++i) {
     if (!grads[i]) return KSGD_ERR_NULL;
@@ -839,7 +885,7 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   // Host image of the scratch, every byte of it: whatever the previous call left in the
   // array (scans, counters, phase and tickets) is overwritten.
   std::vector<unsigned char> img(L.total, 0);
-  write_initial_image(img.data(), L, descs, n_tensors, nullptr, nullptr, kChunk, false, nullptr);
+  write_initial_image(img.data(), L, descs, n_tensors, nullptr, nullptr, kChunk, false, 0, nullptr);   // whole tiles of kChunk
   double state_bytes = 0.0;
   for (int32_t i = 0; i < n_tensors; ++i)
     state_bytes += (double)descs[i].numel * ((descs[i].theta_bits + descs[i].comp_bits) / 8);
@@ -857,10 +903,8 @@ int kahan_sgd_step_static(const ksgd_tensor_desc* descs, int32_t n_tensors, ksgd
   params.tensor_begin = 0;
   params.tensor_count = n_tensors;
   params.state_in_l2 = state_bytes <= 0.8 * (double)sd.l2_bytes ? 1 : 0;
-  params.chunk8 = kChunk;
   params.advance = 1;
   params.exp_grad_dev = nullptr;
-  params.qgrad_tiles = 0;
 
   InlineArgs inl;
   for (int32_t i = 0; i < n_tensors; ++i) { inl.grads[i] = grads[i]; inl.lrs[i] = lrs[i]; }
@@ -908,7 +952,8 @@ int upload_long_list(cudaStream_t stream, int32_t n, const float* const* grads, 
 }
 
 Layout make_mom_layout(const ksgd_tensor_desc* d, int32_t n) {
-  return make_ring_layout(n, plain_tile_count(d, n), sizeof(mom::TensorState), sizeof(mom::TensorInfo), 4);
+  return make_ring_layout(n, whole_tiles(d, n, [](const ksgd_tensor_desc&) { return kChunkLog2; }) + kTailReserve,
+                          sizeof(mom::TensorState), sizeof(mom::TensorInfo), 4);
 }
 
 int validate_momentum(const ksgd_tensor_desc* d, const ksgd_momentum_desc* m, int32_t n) {
@@ -959,6 +1004,11 @@ int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* 
   const Layout L = make_mom_layout(descs, n_tensors);
   if (workspace_bytes < L.total) return KSGD_ERR_WORKSPACE;
 
+  DeviceFacts dev;            // the tile table depends on the number of blocks a step has
+  {
+    const cudaError_t eq = query_device(dev);
+    if (eq != cudaSuccess) return cuda_fail(eq, "device query");
+  }
   ksgd_momentum_handle* h = new (std::nothrow) ksgd_momentum_handle();
   if (!h) return KSGD_ERR_NULL;
   h->layout = L;
@@ -973,7 +1023,6 @@ int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* 
   mom::TensorState* last = reinterpret_cast<mom::TensorState*>(img.data() + L.state) + 2 * (size_t)L.slab;
   mom::TensorInfo* info = reinterpret_cast<mom::TensorInfo*>(img.data() + L.info);
   ChunkRef* chunks = reinterpret_cast<ChunkRef*>(img.data() + L.chunks);
-  long long c = 0;
   double state_bytes = 0.0;
   for (int32_t i = 0; i < n_tensors; ++i) {
     const ksgd_tensor_desc& t = descs[i];
@@ -991,10 +1040,10 @@ int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* 
     info[i].s = t.comp_bits - 1 - t.overlap_k;
     h->theta_bits.push_back(t.theta_bits);
     h->mom_bits.push_back(mdescs[i].mom_bits);
-    const long long nc = (t.numel + kChunk - 1) / kChunk;
-    for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
     state_bytes += (double)t.numel * ((t.theta_bits + t.comp_bits + mdescs[i].mom_bits) / 8);
   }
+  const long long tiles = build_tile_table(descs, n_tensors, [](const ksgd_tensor_desc&) { return kChunkLog2; },
+                                           dev.sms, chunks, nullptr);
 
   mom::Workspace& w = h->params.ws;
   char* b = h->ws_base;
@@ -1010,21 +1059,18 @@ int kahan_sgd_momentum_init(ksgd_momentum_handle** out, const ksgd_tensor_desc* 
   w.mu = reinterpret_cast<float*>(b + L.exp_grad);
   h->params.n_tensors = n_tensors;
   h->params.tile_begin = 0;
-  h->params.tile_count = (int)L.n_chunks;
+  h->params.tile_count = (int)tiles;
   h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
   h->params.inline_args = n_tensors <= kInlineArgs ? 1 : 0;
   h->params.advance = 1;
 
-  DeviceFacts dev;
-  cudaError_t e = query_device(dev);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(mom::ksgd_momentum_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(mom::ksgd_momentum_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)mom::kSharedBytes);
   if (e != cudaSuccess) {
     delete h;
     return cuda_fail(e, "device query");
   }
-  h->grid = (int)(L.n_chunks < (long long)dev.sms ? L.n_chunks : (long long)dev.sms);
+  h->grid = (int)(tiles < (long long)dev.sms ? tiles : (long long)dev.sms);
   h->params.state_in_l2 = state_bytes <= 0.8 * (double)dev.l2_bytes ? 1 : 0;
 
   e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);
@@ -1116,7 +1162,8 @@ int kahan_sgd_momentum_destroy(ksgd_momentum_handle* h) {
 namespace {
 
 Layout make_adam_layout(const ksgd_tensor_desc* d, int32_t n) {
-  return make_ring_layout(n, plain_tile_count(d, n), sizeof(adam::TensorState), sizeof(adam::TensorInfo), 5);
+  return make_ring_layout(n, whole_tiles(d, n, [](const ksgd_tensor_desc&) { return kChunkLog2; }) + kTailReserve,
+                          sizeof(adam::TensorState), sizeof(adam::TensorInfo), 5);
 }
 
 bool exp_pair_ok(int32_t cur, int32_t next) {
@@ -1171,6 +1218,11 @@ int kahan_sgd_adam_init(ksgd_adam_handle** out, const ksgd_tensor_desc* descs, c
   const Layout L = make_adam_layout(descs, n_tensors);
   if (workspace_bytes < L.total) return KSGD_ERR_WORKSPACE;
 
+  DeviceFacts dev;            // the tile table depends on the number of blocks a step has
+  {
+    const cudaError_t eq = query_device(dev);
+    if (eq != cudaSuccess) return cuda_fail(eq, "device query");
+  }
   ksgd_adam_handle* h = new (std::nothrow) ksgd_adam_handle();
   if (!h) return KSGD_ERR_NULL;
   h->layout = L;
@@ -1185,7 +1237,6 @@ int kahan_sgd_adam_init(ksgd_adam_handle** out, const ksgd_tensor_desc* descs, c
   adam::TensorState* last = reinterpret_cast<adam::TensorState*>(img.data() + L.state) + 2 * (size_t)L.slab;
   adam::TensorInfo* info = reinterpret_cast<adam::TensorInfo*>(img.data() + L.info);
   ChunkRef* chunks = reinterpret_cast<ChunkRef*>(img.data() + L.chunks);
-  long long c = 0;
   double state_bytes = 0.0;
   for (int32_t i = 0; i < n_tensors; ++i) {
     const ksgd_tensor_desc& t = descs[i];
@@ -1205,10 +1256,10 @@ int kahan_sgd_adam_init(ksgd_adam_handle** out, const ksgd_tensor_desc* descs, c
     info[i].s = t.comp_bits - 1 - t.overlap_k;
     info[i].pad = 0;
     h->theta_bits.push_back(t.theta_bits);
-    const long long nc = (t.numel + kChunk - 1) / kChunk;
-    for (long long j = 0; j < nc; ++j) chunks[c++] = ChunkRef{i, (int)j};
     state_bytes += (double)t.numel * ((t.theta_bits + t.comp_bits + 32) / 8);
   }
+  const long long tiles = build_tile_table(descs, n_tensors, [](const ksgd_tensor_desc&) { return kChunkLog2; },
+                                           dev.sms, chunks, nullptr);
 
   adam::Workspace& w = h->params.ws;
   char* b = h->ws_base;
@@ -1223,21 +1274,18 @@ int kahan_sgd_adam_init(ksgd_adam_handle** out, const ksgd_tensor_desc* descs, c
   w.lr = reinterpret_cast<float*>(b + L.lr);
   h->params.n_tensors = n_tensors;
   h->params.tile_begin = 0;
-  h->params.tile_count = (int)L.n_chunks;
+  h->params.tile_count = (int)tiles;
   h->params.amax_mode = mode == KSGD_EXP_AMAX ? 1 : 0;
   h->params.inline_args = n_tensors <= kInlineArgs ? 1 : 0;
   h->params.advance = 1;
 
-  DeviceFacts dev;
-  cudaError_t e = query_device(dev);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(adam::ksgd_adam_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(adam::ksgd_adam_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)adam::kSharedBytes);
   if (e != cudaSuccess) {
     delete h;
     return cuda_fail(e, "device query");
   }
-  h->grid = (int)(L.n_chunks < (long long)dev.sms ? L.n_chunks : (long long)dev.sms);
+  h->grid = (int)(tiles < (long long)dev.sms ? tiles : (long long)dev.sms);
   h->params.state_in_l2 = state_bytes <= 0.8 * (double)dev.l2_bytes ? 1 : 0;
 
   e = cudaMemcpyAsync(b, img.data(), L.total, cudaMemcpyHostToDevice, h->stream);

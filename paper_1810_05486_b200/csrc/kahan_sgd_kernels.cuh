@@ -77,14 +77,6 @@ struct StepParams {
   // of tensors [tensor_begin, tensor_begin + tensor_count): the whole list for an ordinary
   // step, one group of tensors when the host-buffer entry point pipelines its copies.
   int tile_begin, tile_count, tensor_begin, tensor_count;
-  // Elements per tile of tensors with 8-bit theta in the list's first tile table: kChunk, or
-  // 2 * kChunk for lists long enough to keep every block busy with the larger tiles (one
-  // vector per thread and tile leaves the per-tile work of a consumer -- wait, descriptor,
-  // scans, arrive -- a third of its instructions).  Tensors with 16-bit theta take kChunk.
-  int chunk8;
-  // 1: this launch walks the table for steps on 8-bit gradients, whose tiles are twice as
-  // large again (4 * kChunk for 8-bit theta with an 8-bit or no c, 2 * kChunk otherwise)
-  int qgrad_tiles;
 };
 
 struct InlineArgs {
@@ -731,15 +723,6 @@ struct PlainPolicy {
   }
   static __device__ __forceinline__ void record(const Params& p, int t, int ph, const Meta& m) {
     record_exponents(p, t, ph, STRICT, m);
-  }
-  // Tensors with 8-bit theta take tiles of 2 * kChunk elements in lists long enough to keep
-  // every block busy with them (one vector per thread and tile leaves the per-tile work of a
-  // consumer -- wait, descriptor, scans, arrive -- a third of its instructions); the table
-  // for steps on 8-bit gradients has tiles twice as large again for every tensor (the same
-  // rule as the host's tile_elems_qgrad).
-  static __device__ __forceinline__ int tile_shift(const Params& p, const Meta& m) {
-    if (p.qgrad_tiles) return (m.ti.theta_bits == 8 && m.ti.comp_bits <= 8) ? 2 : 1;
-    return (m.ti.theta_bits == 8 && p.chunk8 != kChunk) ? 1 : 0;
   }
   static __device__ __forceinline__ void streams(const Meta& m, const unsigned char* (&base)[kStreams],
                                                  int (&bytes)[kStreams]) {

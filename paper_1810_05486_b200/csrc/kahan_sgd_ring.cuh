@@ -6,8 +6,9 @@
 // another.  What differs between the optimizers -- how many arrays a tile has, the arithmetic
 // of an element, how many scans steer how many exponents -- comes in as a policy class.
 //
-// Structure.  The tensor list is cut into tiles of kChunk elements (2 * kChunk where the policy
-// asks for it); block b takes tiles b, b + gridDim.x, ....  A tile's arrays go into a 224 KB
+// Structure.  The tensor list is cut into tiles of kChunk elements (a multiple where the host
+// chose larger ones, power-of-two pieces in the table's last round); block b takes tiles b,
+// b + gridDim.x, ....  A tile's arrays go into a 224 KB
 // ring handed out in 8 KB pages, so a tile takes only what its formats need and two to four
 // tiles are resident, independent of registers and occupancy.  The copies of a tile complete
 // an mbarrier; the consumers wait on it, compute, store their results straight to global
@@ -42,7 +43,6 @@
 //   Meta                what the producer knows about a tile's tensor (with .ti, the Info)
 //   load_meta(p, a, t, ph, ti)   read slab ph-1's record and the per-step arguments, derive exponents
 //   record(p, t, ph, m)          store the derived exponents into slab ph, clear the record in slab ph+1
-//   tile_shift(p, m)             0: tiles of kChunk elements, 1: of 2 * kChunk
 //   streams(m, base, bytes)      global base address and bytes per element of each array (0: absent)
 //   fill_desc(td, p, m, tensor, count, n_bulk, page, gptr)   gptr: the tile's first element in each array
 //   consume(td, scan, ring, ctid, lane)   one consumer thread's share of a tile, scans included
@@ -59,6 +59,7 @@ constexpr long long kBigTileMinTiles = 1024;   // a list gets the large 8-bit ti
 constexpr int kSlots = 6;              // tiles a block can have in its ring at once
 constexpr int kPageBytes = 8192;       // the ring is handed out in pages
 static_assert(kChunk == 8192 && kPageBytes == kChunk, "the producer's page arithmetic assumes 8192-element tiles and 8 KB pages");
+static_assert(kChunk == 1 << 13, "kChunkLog2");
 constexpr int kPages = 28;             // 224 KB of tile data per block
 constexpr int kTilesInFlight = 2;      // a step that streams from DRAM keeps this many tiles on their way, and more
 constexpr int kPagesInFlight = 18;     // only while they take no more than this many pages together (ring_step)
@@ -72,10 +73,26 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a barrier wait g
 enum DeviceError { kErrNone = 0, kErrFullWait = 1, kErrEmptyWait = 2 };
 
 
+// One entry of the tile table.  A tile is 2^lg consecutive elements of one tensor (only a
+// tensor's last tile is short), lg from kMinTileLog2 to 15, starting at element index << lg.
+// Most tiles of a list have the size its tensors' formats ask for (kChunk elements or a
+// multiple); the tiles of the table's last, incomplete round over the blocks are cut into
+// power-of-two pieces so that the round has about one piece per block (see the host's table
+// builder), which is why every entry carries its own size.
 struct ChunkRef {
-  int tensor;  // index into the tensor list
-  int index;   // tile number inside that tensor: elements [index*chunk, ...), chunk = the tensor's tile size
+  int tensor;          // index into the tensor list
+  unsigned int where;  // index (low kTileIndexBits bits) | lg << kTileIndexBits
 };
+constexpr int kTileIndexBits = 27;
+constexpr int kMinTileLog2 = 9;      // pieces of at least 512 elements (one 16-element vector per consumer thread)
+constexpr int kChunkLog2 = 13;
+__host__ __device__ __forceinline__ ChunkRef make_chunk_ref(int tensor, long long index, int lg) {
+  return ChunkRef{tensor, (unsigned int)index | ((unsigned int)lg << kTileIndexBits)};
+}
+__host__ __device__ __forceinline__ int chunk_log2(const ChunkRef& c) { return (int)(c.where >> kTileIndexBits); }
+__host__ __device__ __forceinline__ long long chunk_index(const ChunkRef& c) {
+  return (long long)(c.where & ((1u << kTileIndexBits) - 1u));
+}
 
 // Device-side view of the caller's workspace.
 // ----------------------------------------------------------------------------------------
@@ -474,7 +491,7 @@ __device__ __forceinline__ void ring_step(const typename P::Params& p, const Arg
       // the tile table and the tensor table are written once at init: read the first
       // entries before waiting for the preceding kernel
       ChunkRef cr = p.ws.chunks[tile0];
-      ChunkRef cr1{-1, -1};
+      ChunkRef cr1{-1, 0u};
       if (n_my > 1) cr1 = p.ws.chunks[tile0 + stride];
       const Info ti_first = p.ws.info[cr.tensor];
       // The step's phase.  The preceding step moves the word on as soon as all of its blocks
@@ -491,7 +508,7 @@ __device__ __forceinline__ void ring_step(const typename P::Params& p, const Arg
         ph = ph_now;
         meta = P::load_meta(p, a, cr.tensor, ph, &ti_first);
       }
-      if (cr.index == 0) P::record(p, cr.tensor, ph, meta);
+      if (chunk_index(cr) == 0) P::record(p, cr.tensor, ph, meta);
       State* now = p.ws.state + (size_t)ph * p.ws.slab;
       int issued = 0;
       // The ring: pages from `head` on are free, tiles are released in the order they were
@@ -531,19 +548,21 @@ __device__ __forceinline__ void ring_step(const typename P::Params& p, const Arg
             break;
           }
         }
-        ChunkRef cr2{-1, -1};
+        ChunkRef cr2{-1, 0u};
         if (i + 2 < n_my) cr2 = p.ws.chunks[tile0 + (i + 2) * stride];
         Meta meta1 = meta;
         if (i + 1 < n_my && cr1.tensor != cr.tensor) {
           meta1 = P::load_meta(p, a, cr1.tensor, ph, nullptr);
-          if (cr1.index == 0) P::record(p, cr1.tensor, ph, meta1);
+          if (chunk_index(cr1) == 0) P::record(p, cr1.tensor, ph, meta1);
         }
 
         // where the arrays go, and how many pages that takes including those skipped when
         // a run does not fit before the end of the ring (kChunk == kPageBytes: an array of
-        // b-byte elements takes b pages, 2b with the large tiles)
-        const int big = P::tile_shift(p, meta);
-        const int chunk = kChunk << big;
+        // b-byte elements takes b pages, 2b or 4b with the large tiles; the pieces of the
+        // table's last round are given the pages of a kChunk tile)
+        const int lg = chunk_log2(cr);
+        const int big = lg > kChunkLog2 ? lg - kChunkLog2 : 0;
+        const int chunk = 1 << lg;
         const unsigned char* base[S];
         int bytes[S];
         P::streams(meta, base, bytes);
@@ -590,7 +609,7 @@ __device__ __forceinline__ void ring_step(const typename P::Params& p, const Arg
         sh->slot_pages[slot] = need;
         sh->slot_tensor[slot] = cr.tensor;
 
-        const long long first = (long long)cr.index << (13 + big);
+        const long long first = chunk_index(cr) << lg;
         const long long left = meta.ti.numel - first;
         const int count = left < (long long)chunk ? (int)left : chunk;
         const int n_bulk = count & ~15;

@@ -54,6 +54,7 @@ def good(**over):
     (good(overlap_k=8), "KSGD_ERR_OVERLAP"),
     (good(overlap_k=-1), "KSGD_ERR_OVERLAP"),
     (good(numel=0), "KSGD_ERR_NUMEL"),
+    (good(numel=(1 << 40) + 1), "KSGD_ERR_NUMEL"),  # beyond the index field of a tile table entry
     (good(exp_theta=65), "KSGD_ERR_EXP_RANGE"),
     (good(exp_theta=-65), "KSGD_ERR_EXP_RANGE"),
     (good(exp_theta=0, exp_theta_next=9), "KSGD_ERR_EXP_RANGE"),
@@ -97,20 +98,26 @@ def test_long_lists_of_8bit_theta_get_the_large_tiles(B):
     """The tile tables (8 bytes per tile) show which tile sizes a list got.  First table: 8192
     elements, or 16384 for 8-bit theta once the list still has 1024 tiles with them; 16-bit
     theta always keeps 8192.  A second table, for steps on 8-bit gradients, once the list has
-    1024 tiles of twice those sizes (32768 for 8-bit theta with an 8-bit c, 16384 otherwise)."""
-    def table_bytes(numel, **kw):
+    1024 tiles of twice those sizes (32768 for 8-bit theta with an 8-bit c, 16384 otherwise).
+    Every table reserves 1024 entries more than it has whole tiles, for the pieces its last
+    round over the blocks is cut into (the size query does not know the device)."""
+    reserve = 8 * 1024
+
+    def table_bytes(numel, **kw):        # the first table's reserve cancels in the difference
         return (B.kahan_sgd_workspace_bytes(B.make_descs([good(numel=numel, **kw)])) -
                 B.kahan_sgd_workspace_bytes(B.make_descs([good(numel=1, **kw)])))
     short, long_ = 1023 * 16384, 1024 * 16384
     assert abs(table_bytes(short) - 8 * (short // 8192)) <= 512          # small tiles, one table
     assert abs(table_bytes(long_) - 8 * 1024) <= 512                     # large tiles, one table
     longer = 1024 * 32768
-    assert abs(table_bytes(longer) - 8 * (2048 + 1024)) <= 512           # and 1024 tiles of 32768 in the second
+    assert abs(table_bytes(longer) - 8 * (2048 + 1024) - reserve) <= 512   # and 1024 tiles of 32768 in the second
     wide = dict(theta_bits=16, comp_bits=16)
     assert abs(table_bytes(short, **wide) - 8 * (short // 8192)) <= 512  # 16-bit theta: small tiles, one table
-    assert abs(table_bytes(long_, **wide) - 8 * (long_ // 8192 + 1024)) <= 512   # second table: 1024 tiles of 16384
+    assert abs(table_bytes(long_, **wide) - 8 * (long_ // 8192 + 1024) - reserve) <= 512   # second table: 1024 tiles of 16384
     mixed = dict(theta_bits=8, comp_bits=16)                             # 8-bit theta with a 16-bit c: 16384 in both
-    assert abs(table_bytes(long_, **mixed) - 8 * (1024 + 1024)) <= 512
+    assert abs(table_bytes(long_, **mixed) - 8 * (1024 + 1024) - reserve) <= 512
+    # a one-element list: the table is the reserve and little else
+    assert B.kahan_sgd_workspace_bytes(B.make_descs([good(numel=1)])) < reserve + 4096
 
 
 def test_null_handles_and_strerror(B):

@@ -284,6 +284,28 @@ def test_long_lists_with_8bit_theta_take_the_large_tiles():
     run_both(specs, thetas, comps, grads, lrs, EXP_AMAX)
 
 
+@pytest.mark.parametrize("extra", [0, 1, 2, 19, 74, 75, 147])
+def test_last_round_of_the_tile_table_cut_into_pieces(extra):
+    """The tiles of a table's last, incomplete round over the blocks are cut into 2^k pieces
+    each (k the largest with at most one piece per block): one leftover tile becomes 16 pieces
+    of 512 elements, 19 become 133 of 1024, 75 and more stay whole, none is nothing to cut.
+    Two tensors, so that the round spans a tensor border, ragged ends, an exponent change."""
+    import torch
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    rng = np.random.default_rng(4000 + extra)
+    tiles = 2 * sms + extra
+    n0 = 8192 * (tiles - max(extra // 2, 1)) - 7          # ends inside a tile
+    n1 = 8192 * tiles - (n0 + 8191) // 8192 * 8192 - 3
+    specs, thetas, comps = [], [], []
+    for n in (n0, n1):
+        th, c = random_tensor(rng, n, 16, 8, full_range=False)
+        specs.append(dict(numel=n, theta_bits=16, comp_bits=8, overlap_k=0, exp_theta=-14))
+        thetas.append(th); comps.append(c)
+    grads = [[(rng.standard_normal(n) * 2.0 ** -19 * (1 + 40 * (k == 1))).astype(np.float32) for n in (n0, n1)]
+             for k in range(3)]
+    run_both(specs, thetas, comps, grads, [[1.0, 0.5]] * 3)
+
+
 def test_checkpoint_resume_is_bit_identical():
     """N steps in one go == N/2 steps, read the state back, re-init from it, N/2 more."""
     rng = np.random.default_rng(31)

@@ -70,7 +70,15 @@ def test_two_gloo_ranks_reproduce_the_single_process_result(tmp_path):
     import torch.multiprocessing as mp
     from oracle import EXP_AMAX, OracleState, OracleTensor, oracle_step
     world = 2
-    mp.spawn(_rank_main, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    # The port is free when it is drawn, not necessarily still when rank 0 binds it: a
+    # rendezvous that fails for that reason is tried once more on another port.
+    for attempt in range(2):
+        try:
+            mp.spawn(_rank_main, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+            break
+        except Exception:
+            if attempt == 1:
+                raise
 
     wl = W.scaled_sweep(600_000, 10)
     thetas, comps = W.initial_state(wl)

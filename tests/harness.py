@@ -101,8 +101,9 @@ class LibraryRun:
         self.B.kahan_sgd_step(self.handle, self.grad_ptrs, list(lrs))
 
     def step_qgrad(self, grads_q: Sequence[np.ndarray], exp_grads: Sequence[int],
-                   lrs: Sequence[float]) -> None:
-        """Fixed-point gradients (all int8 or all int16), in a guarded arena of their own."""
+                   lrs: Sequence[float], exponents_on_device: bool = False) -> None:
+        """Fixed-point gradients (all int8 or all int16), in a guarded arena of their own;
+        their exponents from the host, or from a device array the step reads when it runs."""
         bits = 8 * grads_q[0].dtype.itemsize
         if getattr(self, "qgrad_arena", None) is None:
             self.qgrad_arena = DeviceArena([s["numel"] * 2 for s in self.specs])
@@ -112,8 +113,13 @@ class LibraryRun:
                 self.qgrad_arena.view(i)[g.nbytes:] = CANARY
             self.qgrad_arena.sizes[i] = g.nbytes
             self.qgrad_arena.upload(i, g)
-        self.B.kahan_sgd_step_qgrad(self.handle, [self.qgrad_arena.ptr(i) for i in range(self.n)], bits,
-                                    [int(e) for e in exp_grads], list(lrs))
+        ptrs = [self.qgrad_arena.ptr(i) for i in range(self.n)]
+        if exponents_on_device:
+            self.exp_grad_dev = self.torch.tensor([int(e) for e in exp_grads], dtype=self.torch.int32, device="cuda")
+            self.torch.cuda.current_stream().synchronize()      # the upload is torch's; the step may run on another stream
+            self.B.kahan_sgd_step_qgrad_dev(self.handle, ptrs, bits, self.exp_grad_dev.data_ptr(), list(lrs))
+        else:
+            self.B.kahan_sgd_step_qgrad(self.handle, ptrs, bits, [int(e) for e in exp_grads], list(lrs))
 
     def set_exponents(self, exps: Sequence[int]) -> None:
         self.B.kahan_sgd_set_exponents(self.handle, list(exps))

@@ -164,7 +164,7 @@ def run_case(seed, strict, steps):
                 (oracle_strict_step if strict else oracle_step)(ost, [g.copy() for g in grads], lrs)
             else:
                 gq, eg = draw_fixed_grads(rng, ost, strict, lrs, kind)
-                gpu.step_qgrad(gq, eg, lrs)
+                gpu.step_qgrad(gq, eg, lrs, exponents_on_device=bool(rng.random() < 0.4))
                 if strict:
                     oracle_strict_step(ost, [oracle_dequantize_gradient(q, e) for q, e in zip(gq, eg)], lrs)
                 else:

@@ -98,6 +98,20 @@ size_t kahan_sgd_workspace_bytes(const ksgd_tensor_desc* descs, int32_t n_tensor
 size_t kahan_sgd_workspace_error_offset(const ksgd_tensor_desc* descs, int32_t n_tensors);
 
 /*
+ * The tile table kahan_sgd_init would build for this list on a device with `sms`
+ * multiprocessors (0: whole tiles only), for diagnostics and tests: how a step cuts the ragged
+ * list into the pieces its blocks take in turn (block b takes entries b, b + sms, ...).
+ * which: 0 = the table of ordinary steps, 1 = the table of steps on 8-bit gradients (0
+ * entries for lists too short to have one).  out: host array of 3 * capacity values, or NULL
+ * to count only; entry i is out[3i] = tensor, out[3i+1] = first element, out[3i+2] = number
+ * of elements.  Returns the number of entries of the table (which may exceed capacity; only
+ * capacity entries are written), or a negative error code for an invalid list or argument.
+ * Host-only computation.  (No counterpart in the paper: the partition is this library's.)
+ */
+int64_t kahan_sgd_tile_table(const ksgd_tensor_desc* descs, int32_t n_tensors, int32_t sms, int32_t which,
+                             int64_t* out, int64_t capacity);
+
+/*
  * Validate the list, lay out the workspace and copy the chunk table and initial
  * exponents to it.  descs: host array of n_tensors entries, copied.  workspace: device,
  * caller-owned, at least kahan_sgd_workspace_bytes, 256-byte aligned; it must stay

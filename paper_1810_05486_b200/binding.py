@@ -28,7 +28,7 @@ KSGD_ERR_MODE = -10
 KSGD_ERR_DEVICE = -11
 
 EXPORTS = (
-    "kahan_sgd_workspace_bytes", "kahan_sgd_workspace_error_offset", "kahan_sgd_init", "kahan_sgd_step", "kahan_sgd_step_qgrad",
+    "kahan_sgd_workspace_bytes", "kahan_sgd_workspace_error_offset", "kahan_sgd_tile_table", "kahan_sgd_init", "kahan_sgd_step", "kahan_sgd_step_qgrad",
     "kahan_sgd_step_qgrad_dev", "kahan_sgd_import_dev",
     "kahan_sgd_step_host", "kahan_sgd_strict_workspace_bytes", "kahan_sgd_strict_init",
     "kahan_sgd_strict_exponents",
@@ -85,6 +85,9 @@ def _load() -> ctypes.CDLL:
     lib.kahan_sgd_workspace_bytes.argtypes = [P(ksgd_tensor_desc), ctypes.c_int32]
     lib.kahan_sgd_workspace_error_offset.restype = ctypes.c_size_t
     lib.kahan_sgd_workspace_error_offset.argtypes = [P(ksgd_tensor_desc), ctypes.c_int32]
+    lib.kahan_sgd_tile_table.restype = ctypes.c_int64
+    lib.kahan_sgd_tile_table.argtypes = [P(ksgd_tensor_desc), ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                         P(ctypes.c_int64), ctypes.c_int64]
     lib.kahan_sgd_init.restype = ctypes.c_int
     lib.kahan_sgd_init.argtypes = [P(ctypes.c_void_p), P(ksgd_tensor_desc), ctypes.c_int32,
                                    ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
@@ -204,6 +207,17 @@ def kahan_sgd_workspace_error_offset(descs) -> int:
     if off == ctypes.c_size_t(-1).value:
         raise KahanSgdError(KSGD_ERR_NUMEL, "invalid tensor list")
     return off
+
+
+def kahan_sgd_tile_table(descs, sms: int, which: int = 0):
+    """The tile table of this list on a device with `sms` multiprocessors, as a list of
+    (tensor, first element, number of elements); which = 1: the table of steps on 8-bit gradients."""
+    n = int(lib.kahan_sgd_tile_table(descs, len(descs), sms, which, None, 0))
+    if n < 0:
+        _check(n)
+    out = (ctypes.c_int64 * (3 * max(n, 1)))()
+    _check(min(0, int(lib.kahan_sgd_tile_table(descs, len(descs), sms, which, out, n))))
+    return [(int(out[3 * i]), int(out[3 * i + 1]), int(out[3 * i + 2])) for i in range(n)]
 
 
 def kahan_sgd_init(descs, mode: int, workspace: int, workspace_bytes: int, stream: int = 0):

@@ -347,6 +347,31 @@ size_t kahan_sgd_workspace_error_offset(const ksgd_tensor_desc* descs, int32_t n
   return make_layout(descs, n_tensors, pick_chunk8(descs, n_tensors), true, true).error;
 }
 
+int64_t kahan_sgd_tile_table(const ksgd_tensor_desc* descs, int32_t n_tensors, int32_t sms, int32_t which,
+                             int64_t* out, int64_t capacity) {
+  const int v = validate(descs, n_tensors);
+  if (v != KSGD_OK) return v;
+  if (sms < 0 || (which != 0 && which != 1) || capacity < 0) return KSGD_ERR_MODE;
+  const int chunk8 = pick_chunk8(descs, n_tensors);
+  if (which == 1 && whole_tiles_qgrad(descs, n_tensors) == 0) return 0;
+  auto lg_first = [chunk8](const ksgd_tensor_desc& t) { return lg_plain(t, chunk8); };
+  const long long count = which == 0 ? build_tile_table(descs, n_tensors, lg_first, sms, nullptr, nullptr)
+                                     : build_tile_table(descs, n_tensors, lg_qgrad, sms, nullptr, nullptr);
+  if (!out) return count;
+  std::vector<ChunkRef> table((size_t)count);
+  if (which == 0) build_tile_table(descs, n_tensors, lg_first, sms, table.data(), nullptr);
+  else build_tile_table(descs, n_tensors, lg_qgrad, sms, table.data(), nullptr);
+  for (long long i = 0; i < count && i < capacity; ++i) {
+    const ChunkRef& c = table[(size_t)i];
+    const long long first = chunk_index(c) << chunk_log2(c);
+    const long long left = descs[c.tensor].numel - first;
+    out[3 * i] = c.tensor;
+    out[3 * i + 1] = first;
+    out[3 * i + 2] = left < (1LL << chunk_log2(c)) ? left : (1LL << chunk_log2(c));
+  }
+  return count;
+}
+
 }  // extern "C"
 
 namespace {
